@@ -1,0 +1,246 @@
+"""ctypes front end of the CPU oracle (``rtma_oracle.cpp``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg, never by the product package.  Argument
+marshalling only; all arithmetic lives in the C++ file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rtma_oracle.cpp")
+_LIB = os.path.join(_HERE, "librtma_oracle.so")
+_lib = None
+
+c_i32p = ctypes.POINTER(ctypes.c_int32)
+c_i64p = ctypes.POINTER(ctypes.c_int64)
+c_f32p = ctypes.POINTER(ctypes.c_float)
+c_f64p = ctypes.POINTER(ctypes.c_double)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ -O2 (single-threaded, no CUDA)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.run(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-o", tmp, _SRC], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.orc_splitmix64.restype = ctypes.c_uint64
+        _lib.orc_splitmix64.argtypes = [ctypes.c_uint64]
+        _lib.orc_induced_csr.restype = ctypes.c_int64
+        _lib.orc_param_count.restype = ctypes.c_int64
+        _lib.orc_forward_backward_f32.restype = ctypes.c_double
+        _lib.orc_forward_backward_f64.restype = ctypes.c_double
+    return _lib
+
+
+def _p(a, ty):
+    return None if a is None else a.ctypes.data_as(ty)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def splitmix64(x: int) -> int:
+    return int(lib().orc_splitmix64(ctypes.c_uint64(x & (2**64 - 1))))
+
+
+def assign(n: int, group_id, seed: int, M: int) -> np.ndarray:
+    part_id = np.empty(n, dtype=np.int32)
+    g = None if group_id is None else _i32(group_id)
+    lib().orc_assign(ctypes.c_int64(n), _p(g, c_i32p), ctypes.c_uint64(seed), ctypes.c_int32(M),
+                     _p(part_id, c_i32p))
+    return part_id
+
+
+def relabel(part_id: np.ndarray, M: int):
+    n = part_id.size
+    part_id = _i32(part_id)
+    part_offsets = np.empty(M + 1, dtype=np.int64)
+    perm = np.empty(n, dtype=np.int32)
+    local_id = np.empty(n, dtype=np.int32)
+    lib().orc_relabel(ctypes.c_int64(n), ctypes.c_int32(M), _p(part_id, c_i32p),
+                      _p(part_offsets, c_i64p), _p(perm, c_i32p), _p(local_id, c_i32p))
+    return part_offsets, perm, local_id
+
+
+def partition(n: int, group_id, seed: int, M: int):
+    part_id = assign(n, group_id, seed, M)
+    part_offsets, perm, local_id = relabel(part_id, M)
+    return part_id, part_offsets, perm, local_id
+
+
+def induced_csr(rowptr, col, M, part_id, part_offsets, perm, local_id):
+    """Returns (rowptr_out[n+M], col_out[E_kept], edge_offsets[M+1], kept, cut)."""
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    n = rowptr.size - 1
+    rowptr_out = np.empty(n + M, dtype=np.int64)
+    edge_offsets = np.empty(M + 1, dtype=np.int64)
+    kept_cut = np.empty(2, dtype=np.int64)
+    args = [ctypes.c_int64(n), _p(rowptr, c_i64p), _p(col, c_i32p), ctypes.c_int32(M),
+            _p(_i32(part_id), c_i32p), _p(_i64(part_offsets), c_i64p), _p(_i32(perm), c_i32p),
+            _p(_i32(local_id), c_i32p), _p(rowptr_out, c_i64p)]
+    tail = [_p(edge_offsets, c_i64p), _p(kept_cut, c_i64p)]
+    kept = lib().orc_induced_csr(*args, None, *tail)
+    col_out = np.empty(kept, dtype=np.int32)
+    lib().orc_induced_csr(*args, _p(col_out, c_i32p), *tail)
+    return rowptr_out, col_out, edge_offsets, int(kept_cut[0]), int(kept_cut[1])
+
+
+def gather_rows(src: np.ndarray, perm: np.ndarray) -> np.ndarray:
+    src = np.ascontiguousarray(src)
+    perm = _i32(perm)
+    dst = np.empty((perm.size,) + src.shape[1:], dtype=src.dtype)
+    row_bytes = src.dtype.itemsize * int(np.prod(src.shape[1:], dtype=np.int64))
+    lib().orc_gather_rows(ctypes.c_int64(perm.size), ctypes.c_int64(row_bytes),
+                          src.ctypes.data_as(ctypes.c_void_p), _p(perm, c_i32p),
+                          dst.ctypes.data_as(ctypes.c_void_p))
+    return dst
+
+
+def param_count(dims) -> int:
+    d = _i32(dims)
+    return int(lib().orc_param_count(ctypes.c_int32(len(dims) - 1), _p(d, c_i32p)))
+
+
+def _fp(dtype):
+    if np.dtype(dtype) == np.float32:
+        return "f32", c_f32p, np.float32
+    return "f64", c_f64p, np.float64
+
+
+def spmm_mean(rowptr, col, H: np.ndarray) -> np.ndarray:
+    tag, ptr, dt = _fp(H.dtype)
+    H = np.ascontiguousarray(H, dtype=dt)
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    n = rowptr.size - 1
+    d = H.shape[1]
+    N = np.empty((n, d), dtype=dt)
+    getattr(lib(), f"orc_spmm_mean_{tag}")(ctypes.c_int64(n), _p(rowptr, c_i64p), _p(col, c_i32p),
+                                          ctypes.c_int64(d), _p(H, ptr), _p(N, ptr))
+    return N
+
+
+def acts_layout(dims, n: int):
+    """[(name, offset, rows, width)] of the activation record of one part."""
+    out, off = [], 0
+    for l in range(len(dims) - 1):
+        out.append((f"N{l}", off, n, dims[l]))
+        off += n * dims[l]
+        out.append((f"H{l + 1}", off, n, dims[l + 1]))
+        off += n * dims[l + 1]
+    return out, off
+
+
+def forward_backward(dims, rowptr, col, X, y, params, want_grads=True, want_acts=False):
+    """Returns (loss, grads or None, {name: array} or None) for one part."""
+    tag, ptr, dt = _fp(params.dtype)
+    X = np.ascontiguousarray(X, dtype=dt)
+    params = np.ascontiguousarray(params, dtype=dt)
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    y = _i32(y)
+    n = rowptr.size - 1
+    d = _i32(dims)
+    grads = np.empty(params.size, dtype=dt) if want_grads else None
+    acts = None
+    layout = None
+    if want_acts:
+        layout, total = acts_layout(dims, n)
+        acts = np.empty(total, dtype=dt)
+    loss = getattr(lib(), f"orc_forward_backward_{tag}")(
+        ctypes.c_int32(len(dims) - 1), _p(d, c_i32p), ctypes.c_int64(n), _p(rowptr, c_i64p),
+        _p(col, c_i32p), _p(X, ptr), _p(y, c_i32p), _p(params, ptr), _p(grads, ptr), _p(acts, ptr))
+    named = None
+    if want_acts:
+        named = {nm: acts[o:o + r * w].reshape(r, w) for nm, o, r, w in layout}
+    return float(loss), grads, named
+
+
+def local_steps(dims, lr, rowptr, col, X, y, params, K):
+    """K plain-SGD steps on one part.  Returns (new params, loss[K])."""
+    tag, ptr, dt = _fp(params.dtype)
+    X = np.ascontiguousarray(X, dtype=dt)
+    params = np.array(params, dtype=dt, copy=True)
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    y = _i32(y)
+    d = _i32(dims)
+    loss = np.empty(K, dtype=np.float64)
+    getattr(lib(), f"orc_local_steps_{tag}")(
+        ctypes.c_int32(len(dims) - 1), _p(d, c_i32p), ctypes.c_double(lr),
+        ctypes.c_int64(rowptr.size - 1), _p(rowptr, c_i64p), _p(col, c_i32p), _p(X, ptr),
+        _p(y, c_i32p), _p(params, ptr), ctypes.c_int32(K), _p(loss, c_f64p))
+    return params, loss
+
+
+def average(params: np.ndarray):
+    """params [M, P] -> (averaged copies [M, P], global [P])."""
+    tag, ptr, dt = _fp(params.dtype)
+    out = np.array(params, dtype=dt, copy=True, order="C")
+    M, P = out.shape
+    glob = np.empty(P, dtype=dt)
+    getattr(lib(), f"orc_average_{tag}")(_p(out, ptr), ctypes.c_int64(P), ctypes.c_int32(M), _p(glob, ptr))
+    return out, glob
+
+
+def sigmoid_l2_grad(rowptr, col, X, y, w):
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    n, d = X.shape
+    g = np.empty((n, d), dtype=np.float64)
+    lib().orc_sigmoid_l2_grad(ctypes.c_int64(n), _p(rowptr, c_i64p), _p(col, c_i32p), ctypes.c_int64(d),
+                              _p(X, c_f64p), _p(y, c_f64p), _p(w, c_f64p), _p(g, c_f64p))
+    return g
+
+
+def part_graph(rowptr_out, col_out, part_offsets, edge_offsets, p: int):
+    """Slice part p's CSR out of the packed induced-CSR arrays."""
+    lo = int(part_offsets[p]) + p
+    n_p = int(part_offsets[p + 1] - part_offsets[p])
+    rp = rowptr_out[lo:lo + n_p + 1]
+    cp = col_out[int(edge_offsets[p]):int(edge_offsets[p + 1])]
+    return rp, cp
+
+
+def run_method(rowptr, col, X, y, dims, M, K, R, lr, seed, params0, group_id=None, dtype=np.float64):
+    """The whole path on the CPU: partition, induced CSR, R rounds of K local
+    steps on each of the M parts followed by averaging.  Returns a dict."""
+    n = len(rowptr) - 1
+    part_id, part_offsets, perm, local_id = partition(n, group_id, seed, M)
+    rowptr_out, col_out, edge_offsets, kept, cut = induced_csr(
+        rowptr, col, M, part_id, part_offsets, perm, local_id)
+    Xp = gather_rows(X, perm)
+    yp = gather_rows(y, perm)
+    params = np.tile(np.asarray(params0, dtype=dtype), (M, 1))
+    losses = np.zeros((R, M, K))
+    for r in range(R):
+        for p in range(M):
+            rp, cp = part_graph(rowptr_out, col_out, part_offsets, edge_offsets, p)
+            lo, hi = int(part_offsets[p]), int(part_offsets[p + 1])
+            params[p], losses[r, p] = local_steps(dims, lr, rp, cp, Xp[lo:hi], yp[lo:hi], params[p], K)
+        params, _ = average(params)
+    return dict(part_id=part_id, part_offsets=part_offsets, perm=perm, local_id=local_id,
+                rowptr_out=rowptr_out, col_out=col_out, edge_offsets=edge_offsets,
+                kept=kept, cut=cut, Xp=Xp, yp=yp, params=params, losses=losses)

@@ -1,0 +1,355 @@
+// CPU oracle for the RandomTMA / SuperTMA data-parallel path.
+//
+// TEST INFRASTRUCTURE ONLY.  Plain, single-threaded, slow and meant to be
+// checked against the paper by eye.  It shares no code with the CUDA library
+// and must never be called from the product path; only the tests, the smoke
+// check and the benchmark's CPU-baseline leg use it.
+//
+// What each function follows:
+//   orc_splitmix64        one step of the SplitMix64 generator (Steele, Lea,
+//                         Flood 2014): the counter-based source of the paper's
+//                         "randomly and independently assigned" (Sec. 3.2.2).
+//   orc_assign            RandomTMA (node level) and SuperTMA (super-node
+//                         level) assignment, Sec. 3.2.2.
+//   orc_relabel           alpha^{-1}(i) as ordered lists (Preliminaries).
+//   orc_induced_csr       the node-induced subgraph G^(i) (Preliminaries).
+//   orc_spmm_mean         row-normalised aggregation, A-bar X of Theorem 2 /
+//                         Eq. (proof-2-pred): (1/d_v) sum over the effective
+//                         (local) neighbourhood.
+//   orc_forward_backward  GraphSAGE-mean layers, softmax cross-entropy, chain
+//                         rule (the structure of Eq. (proof-2-grad)).
+//   orc_local_steps       Algorithm 2's loop body with a plain SGD optimizer.
+//   orc_average           Algorithm 1's aggregation phi = plain average, then
+//                         Algorithm 2's overwrite of every local copy.
+//   orc_sigmoid_l2_grad   the 1-layer sigmoid / L2 model of Theorem 2, used
+//                         only to pin the aggregation against Eq.
+//                         (proof-2-exp-grad-central).
+//
+// Floating point: storage type T (float or double), every sum accumulated in
+// double and rounded to T once per output element.
+// Parity pins: every function above has at least one pin in tests/ that does
+// not come from this file (printed values, closed forms, brute force,
+// finite differences).  Convergence / accuracy against the paper's tables:
+// parity unpinned (different task, datasets not available).
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+namespace {
+
+inline uint64_t splitmix64_step(uint64_t x) {
+    uint64_t z = x + 0x9E3779B97F4A7C15ULL;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+struct LayerView {
+    int64_t d_in, d_out;
+    int64_t w_self, w_neigh, bias;  // offsets into the flat parameter vector
+};
+
+std::vector<LayerView> layer_views(int32_t L, const int32_t* dims) {
+    std::vector<LayerView> v(L);
+    int64_t off = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        v[l].d_in = dims[l];
+        v[l].d_out = dims[l + 1];
+        v[l].w_self = off;
+        off += v[l].d_in * v[l].d_out;
+        v[l].w_neigh = off;
+        off += v[l].d_in * v[l].d_out;
+        v[l].bias = off;
+        off += v[l].d_out;
+    }
+    return v;
+}
+
+int64_t total_params(int32_t L, const int32_t* dims) {
+    int64_t p = 0;
+    for (int32_t l = 0; l < L; ++l) p += 2LL * dims[l] * dims[l + 1] + dims[l + 1];
+    return p;
+}
+
+// N[v] = (1/deg(v)) * sum_{u in row v} H[u];  deg(v) == 0 -> zero row.
+template <class T>
+void spmm_mean(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, const T* H, T* N) {
+    std::vector<double> acc(d);
+    for (int64_t v = 0; v < n; ++v) {
+        for (int64_t j = 0; j < d; ++j) acc[j] = 0.0;
+        const int64_t deg = rowptr[v + 1] - rowptr[v];
+        for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+            const T* h = H + (int64_t)col[e] * d;
+            for (int64_t j = 0; j < d; ++j) acc[j] += (double)h[j];
+        }
+        for (int64_t j = 0; j < d; ++j) N[v * d + j] = deg > 0 ? (T)(acc[j] / (double)deg) : (T)0;
+    }
+}
+
+// One forward + backward pass over one part.  Returns the loss.
+// acts (optional): for l = 0..L-1: N^l [n x d_l] then H^{l+1} [n x d_{l+1}]
+// (post-ReLU for hidden layers, the logits for the last layer).
+template <class T>
+double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
+                        const int32_t* col, const T* X, const int32_t* y, const T* params,
+                        T* grads, T* acts) {
+    const std::vector<LayerView> lv = layer_views(L, dims);
+    const int64_t P = total_params(L, dims);
+    if (grads) for (int64_t i = 0; i < P; ++i) grads[i] = (T)0;
+    if (n == 0) return 0.0;
+
+    std::vector<std::vector<T>> H(L + 1), N(L), Z(L);
+    H[0].assign(X, X + n * lv[0].d_in);
+    for (int32_t l = 0; l < L; ++l) {
+        const int64_t di = lv[l].d_in, dn = lv[l].d_out;
+        N[l].resize(n * di);
+        spmm_mean<T>(n, rowptr, col, di, H[l].data(), N[l].data());
+        Z[l].resize(n * dn);
+        H[l + 1].resize(n * dn);
+        const T* Ws = params + lv[l].w_self;
+        const T* Wn = params + lv[l].w_neigh;
+        const T* b = params + lv[l].bias;
+        std::vector<double> acc(dn);
+        for (int64_t v = 0; v < n; ++v) {
+            for (int64_t j = 0; j < dn; ++j) acc[j] = (double)b[j];
+            for (int64_t k = 0; k < di; ++k) {
+                const double hs = (double)H[l][v * di + k];
+                const double hn = (double)N[l][v * di + k];
+                const T* ws = Ws + k * dn;
+                const T* wn = Wn + k * dn;
+                for (int64_t j = 0; j < dn; ++j) acc[j] += hs * (double)ws[j] + hn * (double)wn[j];
+            }
+            for (int64_t j = 0; j < dn; ++j) {
+                const T z = (T)acc[j];
+                Z[l][v * dn + j] = z;
+                H[l + 1][v * dn + j] = (l < L - 1) ? (z > (T)0 ? z : (T)0) : z;
+            }
+        }
+    }
+    if (acts) {
+        T* a = acts;
+        for (int32_t l = 0; l < L; ++l) {
+            std::memcpy(a, N[l].data(), sizeof(T) * N[l].size());
+            a += N[l].size();
+            std::memcpy(a, H[l + 1].data(), sizeof(T) * H[l + 1].size());
+            a += H[l + 1].size();
+        }
+    }
+
+    // Softmax cross-entropy, mean over the part's nodes.
+    const int64_t C = lv[L - 1].d_out;
+    std::vector<T> dZ(n * C);
+    double loss = 0.0;
+    for (int64_t v = 0; v < n; ++v) {
+        const T* z = &Z[L - 1][v * C];
+        double zmax = (double)z[0];
+        for (int64_t c = 1; c < C; ++c) zmax = std::fmax(zmax, (double)z[c]);
+        double s = 0.0;
+        for (int64_t c = 0; c < C; ++c) s += std::exp((double)z[c] - zmax);
+        const double lse = zmax + std::log(s);
+        loss += lse - (double)z[y[v]];
+        for (int64_t c = 0; c < C; ++c) {
+            const double p = std::exp((double)z[c] - lse);
+            dZ[v * C + c] = (T)((p - (c == y[v] ? 1.0 : 0.0)) / (double)n);
+        }
+    }
+    loss /= (double)n;
+    if (!grads) return loss;
+
+    // Backward.
+    for (int32_t l = L - 1; l >= 0; --l) {
+        const int64_t di = lv[l].d_in, dn = lv[l].d_out;
+        const T* Ws = params + lv[l].w_self;
+        const T* Wn = params + lv[l].w_neigh;
+        {   // dWs = H^T dZ, dWn = N^T dZ, db = column sums of dZ
+            std::vector<double> gs(di * dn, 0.0), gn(di * dn, 0.0), gb(dn, 0.0);
+            for (int64_t v = 0; v < n; ++v) {
+                const T* dz = &dZ[v * dn];
+                for (int64_t j = 0; j < dn; ++j) gb[j] += (double)dz[j];
+                for (int64_t k = 0; k < di; ++k) {
+                    const double hs = (double)H[l][v * di + k];
+                    const double hn = (double)N[l][v * di + k];
+                    double* rs = &gs[k * dn];
+                    double* rn = &gn[k * dn];
+                    for (int64_t j = 0; j < dn; ++j) {
+                        rs[j] += hs * (double)dz[j];
+                        rn[j] += hn * (double)dz[j];
+                    }
+                }
+            }
+            for (int64_t i = 0; i < di * dn; ++i) grads[lv[l].w_self + i] = (T)gs[i];
+            for (int64_t i = 0; i < di * dn; ++i) grads[lv[l].w_neigh + i] = (T)gn[i];
+            for (int64_t j = 0; j < dn; ++j) grads[lv[l].bias + j] = (T)gb[j];
+        }
+        if (l == 0) break;
+        // dH = dZ Ws^T + A-bar^T (dZ Wn^T);  dZ_prev = dH where Z_prev > 0
+        std::vector<double> dH(n * di, 0.0);
+        std::vector<double> dN(di);
+        for (int64_t v = 0; v < n; ++v) {
+            const T* dz = &dZ[v * dn];
+            for (int64_t k = 0; k < di; ++k) {
+                double s = 0.0, t = 0.0;
+                for (int64_t j = 0; j < dn; ++j) {
+                    s += (double)dz[j] * (double)Ws[k * dn + j];
+                    t += (double)dz[j] * (double)Wn[k * dn + j];
+                }
+                dH[v * di + k] += s;
+                dN[k] = (double)(T)t;
+            }
+            const int64_t deg = rowptr[v + 1] - rowptr[v];
+            for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+                double* dst = &dH[(int64_t)col[e] * di];
+                for (int64_t k = 0; k < di; ++k) dst[k] += dN[k] / (double)deg;
+            }
+        }
+        std::vector<T> dZprev(n * di);
+        for (int64_t i = 0; i < n * di; ++i)
+            dZprev[i] = Z[l - 1][i] > (T)0 ? (T)dH[i] : (T)0;
+        dZ.swap(dZprev);
+    }
+    return loss;
+}
+
+template <class T>
+void local_steps(int32_t L, const int32_t* dims, double lr, int64_t n, const int64_t* rowptr,
+                 const int32_t* col, const T* X, const int32_t* y, T* params, int32_t K,
+                 double* loss_out) {
+    const int64_t P = total_params(L, dims);
+    std::vector<T> g(P);
+    for (int32_t k = 0; k < K; ++k) {
+        const double loss = forward_backward<T>(L, dims, n, rowptr, col, X, y, params, g.data(), nullptr);
+        if (loss_out) loss_out[k] = loss;
+        for (int64_t i = 0; i < P; ++i) params[i] = (T)((double)params[i] - lr * (double)g[i]);
+    }
+}
+
+template <class T>
+void average(T* params, int64_t P, int32_t M, T* global_out) {
+    for (int64_t j = 0; j < P; ++j) {
+        double s = 0.0;
+        for (int32_t i = 0; i < M; ++i) s += (double)params[(int64_t)i * P + j];
+        const T mean = (T)(s / (double)M);
+        for (int32_t i = 0; i < M; ++i) params[(int64_t)i * P + j] = mean;
+        if (global_out) global_out[j] = mean;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+uint64_t orc_splitmix64(uint64_t x) { return splitmix64_step(x); }
+
+// part_id[v] = h(seed xor g(v)) mod M, g(v) = v or the node's super-node id.
+void orc_assign(int64_t n, const int32_t* group_id, uint64_t seed, int32_t M, int32_t* part_id) {
+    for (int64_t v = 0; v < n; ++v) {
+        const uint64_t g = group_id ? (uint64_t)(int64_t)group_id[v] : (uint64_t)v;
+        part_id[v] = (int32_t)(splitmix64_step(seed ^ g) % (uint64_t)M);
+    }
+}
+
+// Sizes, exclusive scan, and the ordered lists alpha^{-1}(i): within a part
+// nodes keep ascending global id.
+void orc_relabel(int64_t n, int32_t M, const int32_t* part_id, int64_t* part_offsets,
+                 int32_t* perm, int32_t* local_id) {
+    std::vector<int64_t> size(M, 0), cursor(M, 0);
+    for (int64_t v = 0; v < n; ++v) size[part_id[v]]++;
+    part_offsets[0] = 0;
+    for (int32_t p = 0; p < M; ++p) part_offsets[p + 1] = part_offsets[p] + size[p];
+    for (int64_t v = 0; v < n; ++v) {
+        const int32_t p = part_id[v];
+        local_id[v] = (int32_t)cursor[p];
+        perm[part_offsets[p] + cursor[p]] = (int32_t)v;
+        cursor[p]++;
+    }
+}
+
+// E^(i) = {(u,v) in E : u, v in alpha^{-1}(i)}, as one CSR per part over local
+// ids.  rowptr_out has n+M entries: part p's n_p+1 zero-based offsets start at
+// part_offsets[p]+p.  col_out (may be null to count only) holds part p's
+// entries from edge_offsets[p].  Returns the number of kept entries.
+int64_t orc_induced_csr(int64_t n, const int64_t* rowptr, const int32_t* col, int32_t M,
+                        const int32_t* part_id, const int64_t* part_offsets, const int32_t* perm,
+                        const int32_t* local_id, int64_t* rowptr_out, int32_t* col_out,
+                        int64_t* edge_offsets, int64_t* kept_cut) {
+    int64_t kept = 0;
+    for (int32_t p = 0; p < M; ++p) {
+        edge_offsets[p] = kept;
+        const int64_t n_p = part_offsets[p + 1] - part_offsets[p];
+        int64_t* rp = rowptr_out + part_offsets[p] + p;
+        rp[0] = 0;
+        for (int64_t i = 0; i < n_p; ++i) {
+            const int64_t u = perm[part_offsets[p] + i];
+            for (int64_t e = rowptr[u]; e < rowptr[u + 1]; ++e) {
+                const int32_t v = col[e];
+                if (part_id[v] == p) {
+                    if (col_out) col_out[kept] = local_id[v];
+                    kept++;
+                }
+            }
+            rp[i + 1] = kept - edge_offsets[p];
+        }
+    }
+    edge_offsets[M] = kept;
+    kept_cut[0] = kept;
+    kept_cut[1] = rowptr[n] - kept;
+    return kept;
+}
+
+void orc_gather_rows(int64_t n, int64_t row_bytes, const void* src, const int32_t* perm, void* dst) {
+    for (int64_t i = 0; i < n; ++i)
+        std::memcpy((char*)dst + i * row_bytes, (const char*)src + (int64_t)perm[i] * row_bytes, row_bytes);
+}
+
+int64_t orc_param_count(int32_t L, const int32_t* dims) { return total_params(L, dims); }
+
+void orc_spmm_mean_f32(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, const float* H, float* N) {
+    spmm_mean<float>(n, rowptr, col, d, H, N);
+}
+void orc_spmm_mean_f64(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, const double* H, double* N) {
+    spmm_mean<double>(n, rowptr, col, d, H, N);
+}
+
+double orc_forward_backward_f32(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
+                                const int32_t* col, const float* X, const int32_t* y,
+                                const float* params, float* grads, float* acts) {
+    return forward_backward<float>(L, dims, n, rowptr, col, X, y, params, grads, acts);
+}
+double orc_forward_backward_f64(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
+                                const int32_t* col, const double* X, const int32_t* y,
+                                const double* params, double* grads, double* acts) {
+    return forward_backward<double>(L, dims, n, rowptr, col, X, y, params, grads, acts);
+}
+
+void orc_local_steps_f32(int32_t L, const int32_t* dims, double lr, int64_t n, const int64_t* rowptr,
+                         const int32_t* col, const float* X, const int32_t* y, float* params,
+                         int32_t K, double* loss_out) {
+    local_steps<float>(L, dims, lr, n, rowptr, col, X, y, params, K, loss_out);
+}
+void orc_local_steps_f64(int32_t L, const int32_t* dims, double lr, int64_t n, const int64_t* rowptr,
+                         const int32_t* col, const double* X, const int32_t* y, double* params,
+                         int32_t K, double* loss_out) {
+    local_steps<double>(L, dims, lr, n, rowptr, col, X, y, params, K, loss_out);
+}
+
+void orc_average_f32(float* params, int64_t P, int32_t M, float* global_out) { average<float>(params, P, M, global_out); }
+void orc_average_f64(double* params, int64_t P, int32_t M, double* global_out) { average<double>(params, P, M, global_out); }
+
+// Theorem 2's model: z_v = sigmoid((A-bar X w)_v), L = 1/2 (y_v - z_v)^2 per
+// node.  Writes the per-node gradient dL/dw [n x d] (Eq. (proof-2-grad)).
+void orc_sigmoid_l2_grad(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d,
+                         const double* X, const double* y, const double* w, double* grad_per_node) {
+    std::vector<double> N(n * d);
+    spmm_mean<double>(n, rowptr, col, d, X, N.data());
+    for (int64_t v = 0; v < n; ++v) {
+        double g = 0.0;
+        for (int64_t j = 0; j < d; ++j) g += N[v * d + j] * w[j];
+        const double z = 1.0 / (1.0 + std::exp(-g));
+        const double f = (z - y[v]) * z * (1.0 - z);
+        for (int64_t j = 0; j < d; ++j) grad_per_node[v * d + j] = f * N[v * d + j];
+    }
+}
+
+}  // extern "C"

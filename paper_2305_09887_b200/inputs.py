@@ -1,0 +1,285 @@
+"""Seeded synthetic inputs: graphs, features, labels and initial weights.
+
+Everything here is input plumbing.  It holds none of the method's arithmetic
+(no partition hash, no aggregation, no training maths): randomness comes from
+numpy's ``default_rng(seed)``, and the arrays produced are handed unchanged to
+whichever implementation consumes them.  The shapes stand in for the paper's
+workloads (Table 1: social / citation / e-commerce graphs with power-law
+degrees, 100-768 wide features), which are not redistributed with this code.
+
+Graph convention: CSR over directed entries, both directions of every
+undirected edge stored, no self loops, no duplicates, columns sorted.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import numpy as np
+
+
+@dataclasses.dataclass
+class Graph:
+    n: int
+    rowptr: np.ndarray  # int32 or int64, [n+1]
+    col: np.ndarray     # int32, [E]
+    group_id: np.ndarray | None = None  # int32 [n], super-node id per node
+
+    @property
+    def num_entries(self) -> int:
+        return int(self.rowptr[-1])
+
+
+@dataclasses.dataclass
+class Workload:
+    name: str
+    graph: Graph
+    X: np.ndarray        # float32 [n, F]
+    y: np.ndarray        # int32 [n]
+    dims: tuple          # (F, hidden..., C)
+    M: int
+    K: int               # local steps per round
+    R: int               # aggregation rounds
+    lr: float
+    partition_seed: int
+    params0: np.ndarray  # float32 [P], identical start for every trainer
+    use_groups: bool = False
+    gemm_dtype: int = 0  # 0: fp32-accurate GEMMs, 1: bf16 inputs / fp32 accumulate
+
+
+def _csr_from_pairs(n: int, u: np.ndarray, v: np.ndarray, wide_rowptr: bool) -> Graph:
+    """Symmetrise, drop loops and duplicates, sort, and build CSR."""
+    keep = u != v
+    u = u[keep].astype(np.int64)
+    v = v[keep].astype(np.int64)
+    key = np.concatenate([u * n + v, v * n + u])
+    del u, v
+    key = np.unique(key)  # sorted by (row, col), duplicates removed
+    rows = key // n
+    col = (key - rows * n).astype(np.int32)
+    del key
+    counts = np.bincount(rows, minlength=n)
+    del rows
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(counts, out=rowptr[1:])
+    if not wide_rowptr:
+        assert rowptr[-1] < 2**31
+        rowptr = rowptr.astype(np.int32)
+    return Graph(n=n, rowptr=rowptr, col=col)
+
+
+def uniform_graph(n: int, m_undirected: int, seed: int, wide_rowptr: bool = False) -> Graph:
+    """G(n, m): m distinct undirected pairs chosen uniformly, no loops."""
+    rng = np.random.default_rng(seed)
+    have = np.empty(0, dtype=np.int64)
+    while have.size < m_undirected:
+        need = m_undirected - have.size
+        a = rng.integers(0, n, size=need + need // 8 + 16, dtype=np.int64)
+        b = rng.integers(0, n, size=a.size, dtype=np.int64)
+        ok = a != b
+        lo = np.minimum(a[ok], b[ok])
+        hi = np.maximum(a[ok], b[ok])
+        have = np.unique(np.concatenate([have, lo * n + hi]))
+    if have.size > m_undirected:
+        have = rng.permutation(have)[:m_undirected]
+    return _csr_from_pairs(n, have // n, have % n, wide_rowptr)
+
+
+def _power_law_cdf(n: int, gamma: float, target_entries: float) -> np.ndarray:
+    """CDF of endpoint weights w_i ~ (i+i0)^(-1/(gamma-1)); i0 caps the largest
+    expected degree at sqrt(target_entries)."""
+    expo = -1.0 / (gamma - 1.0)
+    idx = np.arange(n, dtype=np.float64)
+    cap = math.sqrt(target_entries)
+
+    def top_degree(i0: float) -> float:
+        w = (idx + i0) ** expo
+        return target_entries * w[0] / w.sum()
+
+    lo, hi = 1e-3, float(n)
+    if top_degree(lo) <= cap:
+        i0 = lo
+    else:
+        for _ in range(60):
+            mid = math.sqrt(lo * hi)
+            if top_degree(mid) > cap:
+                lo = mid
+            else:
+                hi = mid
+        i0 = hi
+    w = (idx + i0) ** expo
+    cdf = np.cumsum(w)
+    cdf /= cdf[-1]
+    return cdf
+
+
+def chung_lu_graph(n: int, avg_degree: float, gamma: float, seed: int,
+                   wide_rowptr: bool = False) -> Graph:
+    """Chung-Lu power-law graph by endpoint sampling, node ids shuffled so that
+    hubs are spread over the id range."""
+    rng = np.random.default_rng(seed)
+    target = float(n) * avg_degree
+    cdf = _power_law_cdf(n, gamma, target)
+    m = int(target // 2)
+    shuffle = rng.permutation(n).astype(np.int64)
+    u = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
+    v = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
+    return _csr_from_pairs(n, u, v, wide_rowptr)
+
+
+def planted_community_graph(n_clusters: int, cluster_size: int, intra_degree: float,
+                            inter_degree: float, gamma: float, seed: int,
+                            wide_rowptr: bool = False) -> Graph:
+    """Clusters of equal size with Bernoulli edges inside each cluster and a
+    power-law Chung-Lu overlay between clusters.  ``group_id`` holds each
+    node's cluster; clusters are scattered over the node-id range."""
+    rng = np.random.default_rng(seed)
+    n = n_clusters * cluster_size
+    node_of_slot = rng.permutation(n).astype(np.int64)  # slot = cluster*size + k
+    group_id = np.empty(n, dtype=np.int32)
+    group_id[node_of_slot] = (np.arange(n) // cluster_size).astype(np.int32)
+
+    iu, iv = np.triu_indices(cluster_size, k=1)
+    pairs_per = iu.size
+    p = intra_degree / (cluster_size - 1)
+    us, vs = [], []
+    chunk = max(1, (1 << 24) // pairs_per)
+    for c0 in range(0, n_clusters, chunk):
+        c1 = min(n_clusters, c0 + chunk)
+        hit = np.flatnonzero(rng.random((c1 - c0) * pairs_per) < p)
+        c = hit // pairs_per + c0
+        k = hit % pairs_per
+        us.append(node_of_slot[c * cluster_size + iu[k]])
+        vs.append(node_of_slot[c * cluster_size + iv[k]])
+
+    target = float(n) * inter_degree
+    if target > 0:
+        cdf = _power_law_cdf(n, gamma, target)
+        m = int(target // 2)
+        shuffle = rng.permutation(n).astype(np.int64)
+        a = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
+        b = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
+        differ = group_id[a] != group_id[b]
+        us.append(a[differ])
+        vs.append(b[differ])
+    g = _csr_from_pairs(n, np.concatenate(us), np.concatenate(vs), wide_rowptr)
+    g.group_id = group_id
+    return g
+
+
+def two_class_block_graph(n: int, avg_degree: float, h: float, seed: int):
+    """Two equal classes; an edge joins same-class nodes with probability
+    proportional to h and different-class nodes proportional to 1-h (the
+    compatibility-matrix model of Lemma 1).  Returns (graph, labels)."""
+    rng = np.random.default_rng(seed)
+    y = (rng.permutation(n) % 2).astype(np.int32)
+    m = int(n * avg_degree / 2)
+    u = rng.integers(0, n, size=m, dtype=np.int64)
+    same = rng.random(m) < h
+    members = [np.flatnonzero(y == 0), np.flatnonzero(y == 1)]
+    v = np.empty(m, dtype=np.int64)
+    for cls in (0, 1):
+        for want_same in (False, True):
+            sel = (y[u] == cls) & (same == want_same)
+            pool = members[cls if want_same else 1 - cls]
+            v[sel] = pool[rng.integers(0, pool.size, size=int(sel.sum()))]
+    return _csr_from_pairs(n, u, v, False), y
+
+
+def normal_features(n: int, F: int, seed: int, y: np.ndarray | None = None,
+                    n_classes: int = 0, shift: float = 0.0) -> np.ndarray:
+    """N(0,1) features; with ``shift`` a class-dependent mean shift*mu_y, mu_c ~ N(0,I)."""
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((n, F), dtype=np.float32)
+    if shift != 0.0 and y is not None:
+        mu = rng.standard_normal((n_classes, F), dtype=np.float32)
+        X += np.float32(shift) * mu[y]
+    return X
+
+
+def uniform_labels(n: int, n_classes: int, seed: int) -> np.ndarray:
+    return np.random.default_rng(seed).integers(0, n_classes, size=n, dtype=np.int32)
+
+
+def rare_positive_labels(n: int, positive_rate: float, seed: int) -> np.ndarray:
+    return (np.random.default_rng(seed).random(n) < positive_rate).astype(np.int32)
+
+
+def param_count(dims) -> int:
+    return sum(2 * dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
+
+
+def xavier_params(dims, seed: int) -> np.ndarray:
+    """Flat parameter vector, layer-major: W_self[d_in][d_out], W_neigh[d_in][d_out],
+    b[d_out].  Weights U(-a, a) with a = sqrt(6/(d_in+d_out)); biases zero."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for l in range(len(dims) - 1):
+        d_in, d_out = dims[l], dims[l + 1]
+        a = math.sqrt(6.0 / (d_in + d_out))
+        out.append(rng.uniform(-a, a, size=2 * d_in * d_out).astype(np.float32))
+        out.append(np.zeros(d_out, dtype=np.float32))
+    return np.concatenate(out)
+
+
+SEED_GRAPH, SEED_FEAT, SEED_LABEL, SEED_WEIGHT, SEED_PART = (
+    0x5EED0001, 0x5EED0002, 0x5EED0003, 0x5EED0004, 0x5EED0005)
+
+
+def tiny() -> Workload:
+    """2,000 nodes, 10,000 undirected edges, 64-d features, 8 classes, M=4."""
+    g = uniform_graph(2000, 10000, SEED_GRAPH)
+    y = uniform_labels(g.n, 8, SEED_LABEL)
+    X = normal_features(g.n, 64, SEED_FEAT)
+    dims = (64, 64, 8)
+    return Workload("tiny", g, X, y, dims, M=4, K=5, R=1, lr=0.01,
+                    partition_seed=SEED_PART, params0=xavier_params(dims, SEED_WEIGHT))
+
+
+def medium(scale: float = 1.0) -> Workload:
+    """Chung-Lu, 200k nodes, exponent 2.1, average degree 25, 128-d class-shifted
+    features, 47 classes, M=8, three layers of width 256, 20 steps x 5 rounds."""
+    n = int(200_000 * scale)
+    g = chung_lu_graph(n, 25.0, 2.1, SEED_GRAPH + 1)
+    y = uniform_labels(n, 47, SEED_LABEL + 1)
+    X = normal_features(n, 128, SEED_FEAT + 1, y, 47, 0.5)
+    dims = (128, 256, 256, 47)
+    return Workload("medium" if scale == 1.0 else f"medium_x{scale:g}", g, X, y, dims,
+                    M=8, K=20, R=5, lr=0.01, partition_seed=SEED_PART + 1,
+                    params0=xavier_params(dims, SEED_WEIGHT + 1))
+
+
+def supertma(scale: float = 1.0, width: int | None = None, M: int = 16,
+             use_groups: bool = True, gemm_dtype: int = 0) -> Workload:
+    """Planted communities: 20,000 super-nodes of 100 nodes, intra degree 20,
+    inter-cluster power-law degree 10, labels constant per cluster, 100-d
+    features, 47 classes, three layers of width 256, 10 steps x 3 rounds.
+    ``width`` = 512 gives the trainer-count / width sweep shape."""
+    n_clusters = max(2, int(20_000 * scale))
+    g = planted_community_graph(n_clusters, 100, 20.0, 10.0, 2.1, SEED_GRAPH + 2)
+    cluster_label = uniform_labels(n_clusters, 47, SEED_LABEL + 2)
+    y = cluster_label[g.group_id].astype(np.int32)
+    F = 100 if width is None else width
+    hid = 256 if width is None else width
+    X = normal_features(g.n, F, SEED_FEAT + 2, y, 47, 0.5)
+    dims = (F, hid, hid, 47)
+    K, R = (10, 3) if width is None else (5, 1)
+    name = "supertma" if width is None else f"sweep_w{width}_M{M}_{'super' if use_groups else 'node'}"
+    if scale != 1.0:
+        name += f"_x{scale:g}"
+    return Workload(name, g, X, y, dims, M=M, K=K, R=R, lr=0.01,
+                    partition_seed=SEED_PART + 2, params0=xavier_params(dims, SEED_WEIGHT + 2),
+                    use_groups=use_groups, gemm_dtype=gemm_dtype)
+
+
+def large(scale: float = 1.0) -> Workload:
+    """Chung-Lu, 25M nodes, exponent 2.0, ~1.3B directed entries (int64 row
+    offsets), 128-d features, 2 classes with 1% positives, M=32, two layers."""
+    n = int(25_000_000 * scale)
+    g = chung_lu_graph(n, 52.0, 2.0, SEED_GRAPH + 3, wide_rowptr=True)
+    y = rare_positive_labels(n, 0.01, SEED_LABEL + 3)
+    X = normal_features(n, 128, SEED_FEAT + 3)
+    dims = (128, 256, 2)
+    return Workload("large" if scale == 1.0 else f"large_x{scale:g}", g, X, y, dims,
+                    M=32, K=5, R=1, lr=0.01, partition_seed=SEED_PART + 3,
+                    params0=xavier_params(dims, SEED_WEIGHT + 3))
