@@ -1,0 +1,175 @@
+/*
+ * rtma.h -- C ABI of the RandomTMA / SuperTMA data-parallel hot path on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * "TMA" is the paper's Time-based Model Aggregation (Sec. 3.1), not the GPU's
+ * tensor-memory unit.  The calls follow the paper's problem statement (Sec. 3,
+ * requirements R1 and R2): a partition function alpha that maps nodes to the M
+ * trainers, the node-induced subgraph of every part, independent local training
+ * on each part (Algorithm 2), and the aggregation of the trainers' parameters
+ * (Algorithm 1).
+ *
+ * Conventions
+ *  - Every function returns an int32_t status: RTMA_OK (0) or a negative
+ *    RTMA_ERR_* code.  Nothing throws or aborts across this boundary;
+ *    rtma_last_error(ctx) gives the text of the last failure on that context.
+ *  - Unless a parameter says "host", every array pointer is a DEVICE pointer to
+ *    memory that the caller allocated and owns (for instance the data pointer
+ *    of a torch tensor).  The library never frees it and keeps no reference to
+ *    it after the call returns.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Calls only enqueue work on it and return without synchronising,
+ *    except where stated.  Outputs are valid once the stream has drained.
+ *  - The context owns one scratch arena on its device; it grows (cudaMalloc +
+ *    cudaFree, which synchronise the device) only when a call needs more than
+ *    any call before it.  Every call on a context uses that scratch, so calls on
+ *    one context must be ordered: the same stream, or the earlier call's stream
+ *    drained first (rtma_local_steps orders its own streams).  A context must not
+ *    be used from two host threads at the same time.
+ *  - Node ids and column indices are int32; row offsets are int32 or int64 on
+ *    input and int64 on output.  At most RTMA_MAX_PARTS trainers.
+ */
+#ifndef RTMA_H_
+#define RTMA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RTMA_MAX_PARTS 64
+#define RTMA_MAX_LAYERS 8
+
+enum {
+    RTMA_OK = 0,
+    RTMA_ERR_INVALID_ARG = -1, /* null pointer, negative size, M out of range ...        */
+    RTMA_ERR_UNSUPPORTED = -2, /* a shape or mode this build does not implement           */
+    RTMA_ERR_WORKSPACE = -3,   /* the scratch arena cannot be made large enough           */
+    RTMA_ERR_OVERFLOW = -4,    /* a count does not fit the index type of its output       */
+    RTMA_ERR_CUDA = -5,        /* a CUDA runtime call failed; text in rtma_last_error     */
+    RTMA_ERR_TIMEOUT = -6      /* a bounded device-side wait ran out (kernel gave up)     */
+};
+
+typedef struct rtma_ctx rtma_ctx;
+
+/* Creates a context on CUDA device `device` and reserves `workspace_bytes` of scratch
+ * (0 = reserve lazily).  Synchronous.  *out is NULL on failure.                          */
+int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_bytes);
+/* Synchronises the device, frees the scratch arena and the context.                      */
+int32_t rtma_destroy(rtma_ctx* ctx);
+/* Text of the last error on this context ("" if none).  Owned by the context.            */
+const char* rtma_last_error(const rtma_ctx* ctx);
+/* Bytes of scratch currently held by the context.                                        */
+size_t rtma_workspace_bytes(const rtma_ctx* ctx);
+
+/* ---- R1: partition function (Sec. 3.2.2, RandomTMA and SuperTMA) -----------------------
+ * part_id[v] = h(seed XOR g(v)) mod M, where h is one step of the SplitMix64 generator and
+ * g(v) = v when group_id is NULL (RandomTMA: every node assigned independently) or
+ * g(v) = group_id[v] (SuperTMA: every super-node / mini-cluster assigned as a whole; ids
+ * need not be dense).  Also produces the ordered member lists alpha^{-1}(i) of the
+ * Preliminaries: part_offsets[M+1] (exclusive scan of part sizes), perm[n] (global ids
+ * sorted by (part, id)), local_id[n] (rank of v inside its part).
+ * 1 <= M <= RTMA_MAX_PARTS, 0 <= n < 2^31.  All four outputs are always written.          */
+int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group_id, uint64_t seed,
+                       int32_t M, int32_t* part_id, int64_t* part_offsets, int32_t* perm,
+                       int32_t* local_id, void* stream);
+
+/* ---- node-induced subgraphs G^(i) (Preliminaries) --------------------------------------
+ * Keeps CSR entry (u,v) iff part_id[u] == part_id[v] and emits, for every part, a CSR over
+ * local ids with rows in local order and the input's column order preserved.
+ *   rowptr       [n+1], int64 if rowptr_is_64 else int32;  col [rowptr[n]] int32.
+ *   rowptr_out   [n+M] int64: part p's n_p+1 zero-based offsets start at part_offsets[p]+p.
+ *   edge_offsets [M+1] int64: part p's entries are col_out[edge_offsets[p] .. edge_offsets[p+1]).
+ *   kept_cut     [2]   int64: entries kept, entries dropped (kept + cut = rowptr[n]).
+ * Two phases.  col_out == NULL: COUNT -- writes rowptr_out, edge_offsets and kept_cut; read
+ * edge_offsets[M] back (after draining the stream) to size col_out.  col_out != NULL: FILL --
+ * reads rowptr_out and edge_offsets as the count phase left them and writes col_out only.
+ * part_id / part_offsets / perm / local_id are rtma_partition's outputs.                  */
+int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_64, const void* rowptr,
+                               const int32_t* col, int32_t M, const int32_t* part_id,
+                               const int64_t* part_offsets, const int32_t* perm,
+                               const int32_t* local_id, int64_t* rowptr_out, int32_t* col_out,
+                               int64_t* edge_offsets, int64_t* kept_cut, void* stream);
+
+/* dst[i] = src[perm[i]] for rows of row_bytes bytes: brings features and labels into
+ * partition order ("load G_train^(i)", Algorithm 2).  src and dst must not overlap.       */
+int32_t rtma_gather_rows(rtma_ctx* ctx, int64_t n, int64_t row_bytes, const void* src,
+                         const int32_t* perm, void* dst, void* stream);
+
+/* ---- local training (Algorithm 2, the loop body with a plain SGD optimizer) ------------
+ * Model: L GraphSAGE-mean layers, Z^l = H^l Ws^l + (Abar H^l) Wn^l + b^l, ReLU between
+ * layers, softmax cross-entropy averaged over the part's nodes.  Abar is the part's
+ * row-normalised adjacency (Theorem 2): the mean over LOCAL neighbours, zero for a node
+ * without any.  dims[0] = feature width, dims[L] = number of classes.
+ * Parameters of one trainer: flat float vector of rtma_param_count() entries, layer after
+ * layer: Ws[d_l][d_{l+1}], Wn[d_l][d_{l+1}], b[d_{l+1}], all row-major.                    */
+typedef struct {
+    int32_t L;
+    int32_t dims[RTMA_MAX_LAYERS + 1];
+    int32_t gemm_dtype; /* 0: fp32-accurate products; 1: bf16 operands, fp32 accumulate   */
+    float lr;
+} rtma_model_desc;
+
+int64_t rtma_param_count(const rtma_model_desc* model);
+
+/* Optional record of one step's intermediates, for verification.  Any pointer may be NULL.
+ * acts: for part 0..M-1 in turn, for l = 0..L-1: Abar H^l [n_p x d_l] then H^{l+1}
+ * [n_p x d_{l+1}] (post-ReLU; the logits for l = L-1), densely packed.  grads: [M][P], the
+ * gradient that step applied.  step: which local step (0-based) to record.                */
+typedef struct {
+    float* acts;
+    float* grads;
+    int32_t step;
+} rtma_taps;
+
+/* Runs K local SGD steps on each of the M parts: W_i <- W_i - lr * grad L_i(W_i).
+ *   part_offsets_host, edge_offsets_host  HOST arrays [M+1] (copies of the device outputs).
+ *   rowptr_out, col_out                   as produced by rtma_build_induced_csr.  The
+ *                                         subgraphs must be symmetric (undirected graph,
+ *                                         both directions stored), as the paper's "simple
+ *                                         graph" is; symmetric != 1 is RTMA_ERR_UNSUPPORTED.
+ *   Xp [n][dims[0]] float, yp [n] int32   features / labels in partition order.
+ *   params [M][P]                         in/out, one replica per trainer.
+ *   loss_out [M][K] float or NULL         loss of every step of every trainer.
+ *   streams  HOST array of M cudaStream_t: trainer i runs on streams[i].  Trainers that
+ *            share a stream are batched into common launches; distinct streams run
+ *            concurrently.  The call returns once everything is enqueued.
+ * Scratch is taken from the context (grows if needed).                                    */
+int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* model, int32_t M,
+                         const int64_t* part_offsets_host, const int64_t* edge_offsets_host,
+                         const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                         const float* Xp, const int32_t* yp, float* params, int32_t K,
+                         float* loss_out, const rtma_taps* taps, void* const* streams);
+
+/* ---- R2: aggregation (Algorithm 1, phi = plain average; Algorithm 2, overwrite) ---------
+ * Wbar[j] = (1/M) sum_i params[i][j]; every replica is overwritten with Wbar; global_out
+ * [P] (or NULL) also receives it.  M = 1 leaves the parameters unchanged.                 */
+int32_t rtma_aggregate(rtma_ctx* ctx, float* params, int64_t P, int32_t M, float* global_out,
+                       void* stream);
+
+/* The last local step fused with the aggregation: Wbar = (1/M) sum_i (params[i] - lr *
+ * grads[i]), written to every replica (and global_out).  grads [M][P].                    */
+int32_t rtma_sgd_aggregate(rtma_ctx* ctx, float* params, const float* grads, float lr, int64_t P,
+                           int32_t M, float* global_out, void* stream);
+
+/* ---- the whole path on HOST buffers (Sec. 3: partition, Algorithm 2, Algorithm 1) --------
+ * Every pointer here is a HOST pointer (pageable or pinned).  Copies the graph (CSR as for
+ * rtma_build_induced_csr), group_id_h (NULL = RandomTMA), features X_h [n][dims[0]], labels
+ * y_h [n] and the common initial parameters params0_h [P] to the device, runs rtma_partition,
+ * rtma_build_induced_csr, rtma_gather_rows, then R rounds of (rtma_local_steps with K steps on
+ * every part, rtma_aggregate), and copies back params_out_h [P] (the averaged parameters),
+ * loss_out_h [R][M][K] (or NULL) and kept_cut_h [2] (or NULL).  The graph must be undirected
+ * with both directions stored.  Allocates and frees its device buffers with cudaMalloc /
+ * cudaFree and SYNCHRONISES the stream before returning.                                   */
+int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_64, const void* rowptr_h,
+                        const int32_t* col_h, const int32_t* group_id_h, const float* X_h,
+                        const int32_t* y_h, const rtma_model_desc* model, int32_t M, uint64_t seed,
+                        int32_t K, int32_t R, const float* params0_h, float* params_out_h,
+                        float* loss_out_h, int64_t* kept_cut_h, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RTMA_H_ */

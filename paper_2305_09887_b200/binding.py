@@ -1,0 +1,263 @@
+"""Thin ctypes binding over the CUDA C-ABI library (``librtma.so``, see ``include/rtma.h``).
+
+Argument marshalling only: tensors are allocated with torch (device memory and streams are
+all torch is used for) and handed to the library as raw pointers; every step of the path
+runs in the library's kernels.  There is no CPU fallback: if the library is missing or no
+CUDA device is present the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librtma.so")
+MAX_PARTS = 64
+MAX_LAYERS = 8
+
+EXPORTS = (
+    "rtma_create", "rtma_destroy", "rtma_last_error", "rtma_workspace_bytes", "rtma_partition",
+    "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
+    "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host",
+)
+
+_lib = None
+
+
+class RtmaError(RuntimeError):
+    pass
+
+
+class ModelDesc(ctypes.Structure):
+    _fields_ = [("L", ctypes.c_int32), ("dims", ctypes.c_int32 * (MAX_LAYERS + 1)),
+                ("gemm_dtype", ctypes.c_int32), ("lr", ctypes.c_float)]
+
+
+class Taps(ctypes.Structure):
+    _fields_ = [("acts", ctypes.c_void_p), ("grads", ctypes.c_void_p), ("step", ctypes.c_int32)]
+
+
+def load_library():
+    """Loads the shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RtmaError(f"{LIB_PATH} not found: build it with `python -m paper_2305_09887_b200.build` "
+                            "(there is no CPU fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        lib.rtma_last_error.restype = ctypes.c_char_p
+        lib.rtma_last_error.argtypes = [ctypes.c_void_p]
+        lib.rtma_workspace_bytes.restype = ctypes.c_size_t
+        lib.rtma_workspace_bytes.argtypes = [ctypes.c_void_p]
+        lib.rtma_param_count.restype = ctypes.c_int64
+        _lib = lib
+    return _lib
+
+
+def model_desc(dims, lr: float = 0.01, gemm_dtype: int = 0) -> ModelDesc:
+    L = len(dims) - 1
+    if not 1 <= L <= MAX_LAYERS:
+        raise ValueError(f"number of layers {L} outside [1, {MAX_LAYERS}]")
+    md = ModelDesc()
+    md.L = L
+    for i, d in enumerate(dims):
+        md.dims[i] = int(d)
+    md.gemm_dtype = int(gemm_dtype)
+    md.lr = float(lr)
+    return md
+
+
+def param_count(dims) -> int:
+    return int(load_library().rtma_param_count(ctypes.byref(model_desc(dims))))
+
+
+def _ptr(t):
+    if t is None:
+        return ctypes.c_void_p(0)
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        return int(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)
+
+
+def _need(t, dtype, name, device=None):
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if device is not None and t.device != device:
+        raise ValueError(f"{name} must live on {device}, got {t.device}")
+    return t
+
+
+class Context:
+    """One library context on one CUDA device.  Calls are enqueued on the given (or the
+    current torch) stream and share the context's scratch, so keep them stream-ordered."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        if not torch.cuda.is_available():
+            raise RtmaError("no CUDA device: this library has no CPU path")
+        self._lib = load_library()
+        self.device = torch.device("cuda", device)
+        torch.cuda.init()
+        with torch.cuda.device(self.device):
+            torch.zeros(1, device=self.device)  # make sure the primary context exists
+        h = ctypes.c_void_p()
+        st = self._lib.rtma_create(ctypes.byref(h), ctypes.c_int32(device), ctypes.c_size_t(workspace_bytes))
+        if st != 0:
+            raise RtmaError(f"rtma_create failed with status {st}")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.rtma_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st, what):
+        if st != 0:
+            raise RtmaError(f"{what} failed ({st}): {self._lib.rtma_last_error(self._h).decode()}")
+
+    @property
+    def workspace_bytes(self) -> int:
+        return int(self._lib.rtma_workspace_bytes(self._h))
+
+    # ---- R1 -------------------------------------------------------------------------
+    def partition(self, n: int, group_id, seed: int, M: int, stream=None):
+        """Returns (part_id[n] i32, part_offsets[M+1] i64, perm[n] i32, local_id[n] i32)."""
+        dev = self.device
+        if group_id is not None:
+            _need(group_id, torch.int32, "group_id", dev)
+        part_id = torch.empty(n, dtype=torch.int32, device=dev)
+        part_offsets = torch.empty(M + 1, dtype=torch.int64, device=dev)
+        perm = torch.empty(n, dtype=torch.int32, device=dev)
+        local_id = torch.empty(n, dtype=torch.int32, device=dev)
+        st = self._lib.rtma_partition(self._h, ctypes.c_int64(n), _ptr(group_id), ctypes.c_uint64(seed),
+                                      ctypes.c_int32(M), _ptr(part_id), _ptr(part_offsets), _ptr(perm),
+                                      _ptr(local_id), ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_partition")
+        return part_id, part_offsets, perm, local_id
+
+    def build_induced_csr(self, rowptr, col, M: int, part_id, part_offsets, perm, local_id, stream=None):
+        """Count, size, fill.  Returns (rowptr_out[n+M] i64, col_out[E_kept] i32,
+        edge_offsets[M+1] i64 (device), kept_cut[2] i64 (device), edge_offsets_host list)."""
+        dev = self.device
+        n = rowptr.numel() - 1
+        is64 = 1 if rowptr.dtype == torch.int64 else 0
+        if rowptr.dtype not in (torch.int32, torch.int64):
+            raise TypeError("rowptr must be int32 or int64")
+        _need(col, torch.int32, "col", dev)
+        rowptr_out = torch.empty(n + M, dtype=torch.int64, device=dev)
+        edge_offsets = torch.empty(M + 1, dtype=torch.int64, device=dev)
+        kept_cut = torch.empty(2, dtype=torch.int64, device=dev)
+        s = ctypes.c_void_p(_stream_handle(stream))
+
+        def call(col_out):
+            st = self._lib.rtma_build_induced_csr(
+                self._h, ctypes.c_int64(n), ctypes.c_int32(is64), _ptr(rowptr), _ptr(col), ctypes.c_int32(M),
+                _ptr(part_id), _ptr(part_offsets), _ptr(perm), _ptr(local_id), _ptr(rowptr_out), _ptr(col_out),
+                _ptr(edge_offsets), _ptr(kept_cut), s)
+            self._check(st, "rtma_build_induced_csr")
+
+        call(None)
+        edge_host = edge_offsets.cpu().tolist()  # drains the stream: the size must come back
+        col_out = torch.empty(max(edge_host[-1], 1), dtype=torch.int32, device=dev)[:edge_host[-1]]
+        if edge_host[-1] > 0:
+            call(col_out)
+        return rowptr_out, col_out, edge_offsets, kept_cut, edge_host
+
+    def gather_rows(self, src, perm, stream=None):
+        n = perm.numel()
+        dst = torch.empty((n,) + tuple(src.shape[1:]), dtype=src.dtype, device=self.device)
+        row_bytes = src.element_size() * int(src[0].numel()) if src.shape[0] > 0 else src.element_size()
+        st = self._lib.rtma_gather_rows(self._h, ctypes.c_int64(n), ctypes.c_int64(row_bytes), _ptr(src),
+                                        _ptr(perm), _ptr(dst), ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_gather_rows")
+        return dst
+
+    # ---- Algorithm 2 ----------------------------------------------------------------
+    def local_steps(self, dims, lr, M, part_offsets_host, edge_offsets_host, rowptr_out, col_out, Xp, yp,
+                    params, K, loss_out=None, streams=None, gemm_dtype=0, taps=None, symmetric=True):
+        """K SGD steps on each of the M parts, in place on params [M, P].
+        streams: None (all trainers on the current stream), or a list of M torch streams.
+        taps: None or (acts tensor or None, grads tensor or None, step)."""
+        dev = self.device
+        md = model_desc(dims, lr, gemm_dtype)
+        _need(params, torch.float32, "params", dev)
+        _need(Xp, torch.float32, "Xp", dev)
+        _need(yp, torch.int32, "yp", dev)
+        _need(rowptr_out, torch.int64, "rowptr_out", dev)
+        _need(col_out, torch.int32, "col_out", dev)
+        if loss_out is not None:
+            _need(loss_out, torch.float32, "loss_out", dev)
+        po = (ctypes.c_int64 * (M + 1))(*[int(v) for v in part_offsets_host])
+        eo = (ctypes.c_int64 * (M + 1))(*[int(v) for v in edge_offsets_host])
+        if streams is None:
+            handles = [_stream_handle(None)] * M
+        else:
+            handles = [_stream_handle(s) for s in streams]
+        sarr = (ctypes.c_void_p * M)(*handles)
+        tap_struct = None
+        if taps is not None:
+            acts, grads, step = taps
+            tap_struct = Taps(_ptr(acts), _ptr(grads), int(step))
+        st = self._lib.rtma_local_steps(
+            self._h, ctypes.byref(md), ctypes.c_int32(M), po, eo, _ptr(rowptr_out), _ptr(col_out),
+            ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), _ptr(yp), _ptr(params), ctypes.c_int32(K),
+            _ptr(loss_out), ctypes.byref(tap_struct) if tap_struct is not None else None, sarr)
+        self._check(st, "rtma_local_steps")
+
+    # ---- R2 -------------------------------------------------------------------------
+    def aggregate(self, params, global_out=None, stream=None):
+        M, P = params.shape
+        _need(params, torch.float32, "params", self.device)
+        st = self._lib.rtma_aggregate(self._h, _ptr(params), ctypes.c_int64(P), ctypes.c_int32(M),
+                                      _ptr(global_out), ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_aggregate")
+
+    def sgd_aggregate(self, params, grads, lr, global_out=None, stream=None):
+        M, P = params.shape
+        st = self._lib.rtma_sgd_aggregate(self._h, _ptr(params), _ptr(grads), ctypes.c_float(lr),
+                                          ctypes.c_int64(P), ctypes.c_int32(M), _ptr(global_out),
+                                          ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_sgd_aggregate")
+
+    # ---- whole path from host buffers -----------------------------------------------
+    def train_host(self, rowptr, col, X, y, dims, M, K, R, lr, seed, params0, group_id=None, gemm_dtype=0):
+        """The whole path on HOST (numpy) buffers: copies the inputs to the device, runs
+        partition, induced CSR, row gather, R rounds of (K local steps + aggregation), and
+        copies the result back.  Returns (params[P] f32, losses[R, M, K] f32, kept, cut)."""
+        import numpy as np
+        rowptr = np.ascontiguousarray(rowptr)
+        is64 = 1 if rowptr.dtype == np.int64 else 0
+        if rowptr.dtype not in (np.int32, np.int64):
+            raise TypeError("rowptr must be int32 or int64")
+        col = np.ascontiguousarray(col, dtype=np.int32)
+        X = np.ascontiguousarray(X, dtype=np.float32)
+        y = np.ascontiguousarray(y, dtype=np.int32)
+        params0 = np.ascontiguousarray(params0, dtype=np.float32)
+        gid = None if group_id is None else np.ascontiguousarray(group_id, dtype=np.int32)
+        n = rowptr.size - 1
+        md = model_desc(dims, lr, gemm_dtype)
+        out = np.empty(params0.size, dtype=np.float32)
+        losses = np.empty((R, M, K), dtype=np.float32)
+        kept_cut = np.empty(2, dtype=np.int64)
+        vp = lambda a: ctypes.c_void_p(0) if a is None else ctypes.c_void_p(a.ctypes.data)
+        st = self._lib.rtma_train_host(
+            self._h, ctypes.c_int64(n), ctypes.c_int32(is64), vp(rowptr), vp(col), vp(gid), vp(X), vp(y),
+            ctypes.byref(md), ctypes.c_int32(M), ctypes.c_uint64(seed), ctypes.c_int32(K), ctypes.c_int32(R),
+            vp(params0), vp(out), vp(losses), vp(kept_cut), ctypes.c_void_p(_stream_handle(None)))
+        self._check(st, "rtma_train_host")
+        return out, losses, int(kept_cut[0]), int(kept_cut[1])

@@ -1,0 +1,71 @@
+// Shared host-side plumbing of the library: context, error reporting, scratch arena.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+
+#include "rtma.h"
+
+struct rtma_ctx {
+    int device = 0;
+    char* arena = nullptr;        // device scratch
+    size_t arena_bytes = 0;
+    void* pinned = nullptr;       // small pinned staging block for descriptors
+    size_t pinned_bytes = 0;
+    char error[512] = {0};
+};
+
+inline int32_t rtma_fail(rtma_ctx* ctx, int32_t code, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->error, sizeof(ctx->error), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+#define RTMA_CUDA(ctx, expr)                                                              \
+    do {                                                                                  \
+        cudaError_t e__ = (expr);                                                         \
+        if (e__ != cudaSuccess)                                                           \
+            return rtma_fail((ctx), RTMA_ERR_CUDA, "%s failed: %s (%s:%d)", #expr,        \
+                             cudaGetErrorString(e__), __FILE__, __LINE__);                \
+    } while (0)
+
+#define RTMA_LAUNCH_CHECK(ctx) RTMA_CUDA(ctx, cudaGetLastError())
+
+#define RTMA_TRY(expr)                      \
+    do {                                    \
+        int32_t s__ = (expr);               \
+        if (s__ != RTMA_OK) return s__;     \
+    } while (0)
+
+// Makes the arena at least `bytes` large.  Growing synchronises the device.
+int32_t rtma_reserve(rtma_ctx* ctx, size_t bytes);
+
+// Bump allocator over the arena (256-byte granules).
+struct ArenaCursor {
+    char* base;
+    size_t used = 0;
+    explicit ArenaCursor(char* b) : base(b) {}
+    template <class T>
+    T* take(size_t count) {
+        T* p = reinterpret_cast<T*>(base + used);
+        used += (count * sizeof(T) + 255) / 256 * 256;
+        return p;
+    }
+    static size_t granule(size_t bytes) { return (bytes + 255) / 256 * 256; }
+};
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---- generic device-wide exclusive scan (three passes, no inter-block waits) ----
+// out[i] = sum_{k<i} in[k] for i = 0..n (n+1 outputs).  scratch: scan_scratch_elems(n) int64.
+size_t scan_scratch_elems(int64_t n);
+int32_t exclusive_scan_i32_to_i64(rtma_ctx* ctx, const int32_t* in, int64_t n, int64_t* out,
+                                  int64_t* scratch, cudaStream_t stream);

@@ -1,0 +1,166 @@
+// Context life cycle, scratch arena, and the device-wide exclusive scan shared by the
+// partition and induced-subgraph stages.
+#include "common.cuh"
+
+extern "C" int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_bytes) {
+    if (!out) return RTMA_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return RTMA_ERR_CUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return RTMA_ERR_CUDA;
+    rtma_ctx* ctx = new rtma_ctx();
+    ctx->device = device;
+    ctx->pinned_bytes = 1 << 16;
+    if (cudaMallocHost(&ctx->pinned, ctx->pinned_bytes) != cudaSuccess) {
+        delete ctx;
+        return RTMA_ERR_CUDA;
+    }
+    if (workspace_bytes) {
+        int32_t s = rtma_reserve(ctx, workspace_bytes);
+        if (s != RTMA_OK) {
+            cudaFreeHost(ctx->pinned);
+            delete ctx;
+            return s;
+        }
+    }
+    *out = ctx;
+    return RTMA_OK;
+}
+
+extern "C" int32_t rtma_destroy(rtma_ctx* ctx) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->arena) cudaFree(ctx->arena);
+    if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    delete ctx;
+    return RTMA_OK;
+}
+
+extern "C" const char* rtma_last_error(const rtma_ctx* ctx) { return ctx ? ctx->error : "null context"; }
+
+extern "C" size_t rtma_workspace_bytes(const rtma_ctx* ctx) { return ctx ? ctx->arena_bytes : 0; }
+
+int32_t rtma_reserve(rtma_ctx* ctx, size_t bytes) {
+    if (bytes <= ctx->arena_bytes) return RTMA_OK;
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_CUDA(ctx, cudaDeviceSynchronize());
+    if (ctx->arena) {
+        RTMA_CUDA(ctx, cudaFree(ctx->arena));
+        ctx->arena = nullptr;
+        ctx->arena_bytes = 0;
+    }
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return rtma_fail(ctx, RTMA_ERR_WORKSPACE, "cannot reserve %zu bytes of scratch: %s", bytes,
+                         cudaGetErrorString(e));
+    }
+    ctx->arena = static_cast<char*>(p);
+    ctx->arena_bytes = bytes;
+    return RTMA_OK;
+}
+
+// ------------------------------------------------------------------------------------
+// Exclusive scan: reduce per block, scan the block sums in one block, re-scan per block.
+// ------------------------------------------------------------------------------------
+namespace {
+
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = 8;
+constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
+
+// Exclusive prefix of `v` over the block; *total gets the block sum.  All threads call.
+__device__ __forceinline__ int64_t block_exclusive_scan(int64_t v, int64_t* total) {
+    __shared__ int64_t warp_sums[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int64_t incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int64_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();  // protects warp_sums against a previous call
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    const int nwarps = (blockDim.x + 31) >> 5;
+    if (warp == 0) {
+        int64_t w = lane < nwarps ? warp_sums[lane] : 0;
+        int64_t wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int64_t t = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        warp_sums[lane] = wi - w;  // exclusive prefix of the warp sums
+        if (lane == 31) *total = wi;
+    }
+    __syncthreads();
+    return warp_sums[warp] + incl - v;
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS) scan_reduce_kernel(const int32_t* __restrict__ in, int64_t n,
+                                                                    int64_t* __restrict__ block_sums) {
+    __shared__ int64_t total;
+    const int64_t base = (int64_t)blockIdx.x * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
+    int64_t s = 0;
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
+        const int64_t i = base + k;
+        if (i < n) s += in[i];
+    }
+    block_exclusive_scan(s, &total);
+    if (threadIdx.x == 0) block_sums[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(1024) scan_spine_kernel(int64_t* __restrict__ block_sums, int64_t nb) {
+    __shared__ int64_t total;
+    int64_t carry = 0;
+    for (int64_t start = 0; start < nb; start += blockDim.x) {
+        const int64_t i = start + threadIdx.x;
+        const int64_t v = i < nb ? block_sums[i] : 0;
+        const int64_t ex = block_exclusive_scan(v, &total);
+        if (i < nb) block_sums[i] = carry + ex;
+        carry += total;
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(const int32_t* __restrict__ in, int64_t n,
+                                                                   const int64_t* __restrict__ block_sums,
+                                                                   int64_t* __restrict__ out) {
+    __shared__ int64_t total;
+    const int64_t base = (int64_t)blockIdx.x * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
+    int32_t v[SCAN_ITEMS];
+    int64_t s = 0;
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
+        const int64_t i = base + k;
+        v[k] = i < n ? in[i] : 0;
+        s += v[k];
+    }
+    int64_t run = block_exclusive_scan(s, &total) + block_sums[blockIdx.x];
+#pragma unroll
+    for (int k = 0; k < SCAN_ITEMS; ++k) {
+        const int64_t i = base + k;
+        if (i <= n) out[i] = run;
+        run += v[k];
+    }
+}
+
+}  // namespace
+
+size_t scan_scratch_elems(int64_t n) { return (size_t)ceil_div(n + 1, SCAN_TILE) + 1; }
+
+int32_t exclusive_scan_i32_to_i64(rtma_ctx* ctx, const int32_t* in, int64_t n, int64_t* out,
+                                  int64_t* scratch, cudaStream_t stream) {
+    const int64_t nb = ceil_div(n + 1, SCAN_TILE);
+    scan_reduce_kernel<<<(unsigned)nb, SCAN_THREADS, 0, stream>>>(in, n, scratch);
+    RTMA_LAUNCH_CHECK(ctx);
+    scan_spine_kernel<<<1, 1024, 0, stream>>>(scratch, nb);
+    RTMA_LAUNCH_CHECK(ctx);
+    scan_apply_kernel<<<(unsigned)nb, SCAN_THREADS, 0, stream>>>(in, n, scratch, out);
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}

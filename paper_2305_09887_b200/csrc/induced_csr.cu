@@ -1,0 +1,204 @@
+// Node-induced subgraph of every part (Preliminaries: E^(i) = {(u,v) in E : u,v in
+// alpha^{-1}(i)}), emitted as one CSR per part over local ids, plus the row gather that
+// brings features and labels into partition order.
+//
+// COUNT: one warp per output row (rows taken in partition order, so part p's rows are
+// contiguous) counts the entries whose endpoint lies in the same part; an exclusive scan of
+// the counts gives every row's slot in col_out, from which the per-part zero-based offsets
+// and edge_offsets follow.  FILL: the same walk, with a warp ballot turning the keep
+// predicate into compact, order-preserving output positions.
+#include "common.cuh"
+
+namespace {
+
+constexpr int CSR_THREADS = 256;
+constexpr int CSR_WARPS = CSR_THREADS / 32;
+
+__device__ __forceinline__ int find_part(const int64_t* __restrict__ offs, int M, int64_t row) {
+    int lo = 0, hi = M;  // largest p with offs[p] <= row and offs[p+1] > row
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (offs[mid] <= row) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <class RowT>
+__global__ void __launch_bounds__(CSR_THREADS)
+induced_count_kernel(int64_t n, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
+                     const int32_t* __restrict__ part_id, const int32_t* __restrict__ perm,
+                     int32_t* __restrict__ counts) {
+    const int lane = threadIdx.x & 31;
+    const int64_t j = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
+    if (j >= n) return;
+    const int32_t u = perm[j];
+    const int32_t p = part_id[u];
+    const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
+    int kept = 0;
+    for (int64_t e = begin + lane; e < end; e += 32) kept += (part_id[col[e]] == p);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
+    if (lane == 0) counts[j] = kept;
+}
+
+// slots[j] = global slot of row j's first kept entry (exclusive scan of counts), j = 0..n.
+template <class RowT>
+__global__ void __launch_bounds__(CSR_THREADS)
+induced_offsets_kernel(int64_t n, int M, const int64_t* __restrict__ part_offsets,
+                       const int64_t* __restrict__ slots, const RowT* __restrict__ rowptr,
+                       int64_t* __restrict__ rowptr_out, int64_t* __restrict__ edge_offsets,
+                       int64_t* __restrict__ kept_cut) {
+    __shared__ int64_t offs[RTMA_MAX_PARTS + 1];
+    for (int b = threadIdx.x; b <= M; b += CSR_THREADS) offs[b] = part_offsets[b];
+    __syncthreads();
+    // index space: i in [0, n+M): part p owns i in [offs[p]+p, offs[p+1]+p+1)
+    const int64_t i = (int64_t)blockIdx.x * CSR_THREADS + threadIdx.x;
+    if (i < n + M) {
+        int lo = 0, hi = M;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (offs[mid] + mid <= i) lo = mid; else hi = mid;
+        }
+        const int p = lo;
+        const int64_t row = i - p;  // partition-order row index, may equal offs[p+1]
+        rowptr_out[i] = slots[row] - slots[offs[p]];
+    }
+    if (blockIdx.x == 0) {
+        for (int b = threadIdx.x; b <= M; b += CSR_THREADS) edge_offsets[b] = slots[offs[b]];
+        if (threadIdx.x == 0) {
+            kept_cut[0] = slots[n];
+            kept_cut[1] = (int64_t)rowptr[n] - slots[n];
+        }
+    }
+}
+
+template <class RowT>
+__global__ void __launch_bounds__(CSR_THREADS)
+induced_fill_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
+                    const int32_t* __restrict__ part_id, const int64_t* __restrict__ part_offsets,
+                    const int32_t* __restrict__ perm, const int32_t* __restrict__ local_id,
+                    const int64_t* __restrict__ rowptr_out, const int64_t* __restrict__ edge_offsets,
+                    int32_t* __restrict__ col_out) {
+    __shared__ int64_t offs[RTMA_MAX_PARTS + 1];
+    for (int b = threadIdx.x; b <= M; b += CSR_THREADS) offs[b] = part_offsets[b];
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t j = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
+    if (j >= n) return;
+    const int p = find_part(offs, M, j);
+    const int32_t u = perm[j];
+    const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
+    int64_t out = edge_offsets[p] + rowptr_out[j + p];
+    const unsigned below = (1u << lane) - 1u;
+    for (int64_t e0 = begin; e0 < end; e0 += 32) {
+        const int64_t e = e0 + lane;
+        int32_t v = 0;
+        bool keep = false;
+        if (e < end) {
+            v = col[e];
+            keep = part_id[v] == p;
+        }
+        const unsigned votes = __ballot_sync(0xffffffffu, keep);
+        if (keep) col_out[out + __popc(votes & below)] = local_id[v];
+        out += __popc(votes);
+    }
+}
+
+template <int VEC_BYTES>
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(int64_t n, int64_t row_bytes, const char* __restrict__ src, const int32_t* __restrict__ perm,
+                   char* __restrict__ dst) {
+    const int lane = threadIdx.x & 31;
+    const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (i >= n) return;
+    const char* s = src + (int64_t)perm[i] * row_bytes;
+    char* d = dst + i * row_bytes;
+    if (VEC_BYTES == 16) {
+        for (int64_t o = lane * 16; o < row_bytes; o += 32 * 16)
+            *reinterpret_cast<int4*>(d + o) = __ldg(reinterpret_cast<const int4*>(s + o));
+    } else if (VEC_BYTES == 4) {
+        for (int64_t o = lane * 4; o < row_bytes; o += 32 * 4)
+            *reinterpret_cast<int32_t*>(d + o) = __ldg(reinterpret_cast<const int32_t*>(s + o));
+    } else {
+        for (int64_t o = lane; o < row_bytes; o += 32) d[o] = s[o];
+    }
+}
+
+}  // namespace
+
+extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_64, const void* rowptr,
+                                          const int32_t* col, int32_t M, const int32_t* part_id,
+                                          const int64_t* part_offsets, const int32_t* perm, const int32_t* local_id,
+                                          int64_t* rowptr_out, int32_t* col_out, int64_t* edge_offsets,
+                                          int64_t* kept_cut, void* stream_) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
+    if (n < 0 || n >= (int64_t(1) << 31)) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "n=%lld outside [0,2^31)", (long long)n);
+    if (!rowptr || !part_offsets || !rowptr_out || !edge_offsets || !kept_cut || (n > 0 && (!part_id || !perm || !local_id)))
+        return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_build_induced_csr: null pointer");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    const unsigned row_blocks = (unsigned)ceil_div(n, CSR_WARPS);
+
+    if (col_out) {  // FILL
+        if (n == 0) return RTMA_OK;
+        if (rowptr_is_64)
+            induced_fill_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+                n, M, static_cast<const int64_t*>(rowptr), col, part_id, part_offsets, perm, local_id, rowptr_out,
+                edge_offsets, col_out);
+        else
+            induced_fill_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+                n, M, static_cast<const int32_t*>(rowptr), col, part_id, part_offsets, perm, local_id, rowptr_out,
+                edge_offsets, col_out);
+        RTMA_LAUNCH_CHECK(ctx);
+        return RTMA_OK;
+    }
+
+    // COUNT
+    const size_t need = ArenaCursor::granule(sizeof(int32_t) * (n + 1)) + ArenaCursor::granule(sizeof(int64_t) * (n + 2)) +
+                        ArenaCursor::granule(sizeof(int64_t) * scan_scratch_elems(n));
+    RTMA_TRY(rtma_reserve(ctx, need));
+    ArenaCursor cur(ctx->arena);
+    int32_t* counts = cur.take<int32_t>(n + 1);
+    int64_t* slots = cur.take<int64_t>(n + 2);
+    int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(n));
+    if (n > 0) {
+        if (rowptr_is_64)
+            induced_count_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+                n, static_cast<const int64_t*>(rowptr), col, part_id, perm, counts);
+        else
+            induced_count_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+                n, static_cast<const int32_t*>(rowptr), col, part_id, perm, counts);
+        RTMA_LAUNCH_CHECK(ctx);
+    }
+    RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, n, slots, scratch, stream));
+    const unsigned off_blocks = (unsigned)ceil_div(n + M, CSR_THREADS);
+    if (rowptr_is_64)
+        induced_offsets_kernel<int64_t><<<off_blocks, CSR_THREADS, 0, stream>>>(
+            n, M, part_offsets, slots, static_cast<const int64_t*>(rowptr), rowptr_out, edge_offsets, kept_cut);
+    else
+        induced_offsets_kernel<int32_t><<<off_blocks, CSR_THREADS, 0, stream>>>(
+            n, M, part_offsets, slots, static_cast<const int32_t*>(rowptr), rowptr_out, edge_offsets, kept_cut);
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}
+
+extern "C" int32_t rtma_gather_rows(rtma_ctx* ctx, int64_t n, int64_t row_bytes, const void* src,
+                                    const int32_t* perm, void* dst, void* stream_) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    if (n < 0 || row_bytes <= 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_gather_rows: bad size");
+    if (n == 0) return RTMA_OK;
+    if (!src || !perm || !dst) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_gather_rows: null pointer");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    const unsigned blocks = (unsigned)ceil_div(n, 8);
+    const uintptr_t align = reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst) | (uintptr_t)row_bytes;
+    if (align % 16 == 0)
+        gather_rows_kernel<16><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst));
+    else if (align % 4 == 0)
+        gather_rows_kernel<4><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst));
+    else
+        gather_rows_kernel<1><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst));
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}

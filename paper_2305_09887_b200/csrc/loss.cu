@@ -1,0 +1,88 @@
+// Softmax cross-entropy over a part's logits, averaged over the part's nodes, and its
+// gradient (softmax - onehot) / n_p written over the logits.
+//
+// One warp per row; three sweeps over the row (max, sum of exponentials, gradient), which
+// stay in L1 for the class counts used here.  Loss sums are reduced in a fixed order
+// (warp -> block -> part), so results do not change from run to run.
+#include "train.cuh"
+
+namespace {
+
+constexpr int LOSS_THREADS = 256;
+constexpr int LOSS_TILE_ROWS = 64;
+
+__global__ void __launch_bounds__(LOSS_THREADS)
+softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
+                    float* __restrict__ tile_loss) {
+    __shared__ float warp_loss[LOSS_THREADS / 32];
+    int k, r0;
+    if (!locate_tile(g, LOSS_TILE_ROWS, blockIdx.x, &k, &r0)) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_p = g.rows[k];
+    const float inv_n = 1.0f / (float)n_p;
+    float loss = 0.f;
+    for (int q = 0; q < LOSS_TILE_ROWS / (LOSS_THREADS / 32); ++q) {
+        const int i = r0 + warp * (LOSS_TILE_ROWS / (LOSS_THREADS / 32)) + q;
+        if (i >= n_p) break;
+        float* z = logits.ptr + (g.row_ws[k] + i) * logits.ld;
+        const int label = yp[g.row_abs[k] + i];
+        float zmax = -INFINITY;
+        for (int c = lane; c < C; c += 32) zmax = fmaxf(zmax, z[c]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+        float sum = 0.f;
+        for (int c = lane; c < C; c += 32) sum += expf(z[c] - zmax);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float lse = zmax + logf(sum);
+        if (lane == 0) loss += lse - z[label];
+        __syncwarp();
+        for (int c = lane; c < C; c += 32) {
+            const float p = expf(z[c] - lse);
+            z[c] = (p - (c == label ? 1.f : 0.f)) * inv_n;
+        }
+    }
+    if (lane == 0) warp_loss[warp] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int w = 0; w < LOSS_THREADS / 32; ++w) s += warp_loss[w];
+        tile_loss[blockIdx.x] = s;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+loss_finalize_kernel(const __grid_constant__ GroupDesc g, const float* __restrict__ tile_loss,
+                     float* __restrict__ loss_out, const int64_t loss_stride, const int64_t loss_col) {
+    __shared__ float red[256];
+    const int k = blockIdx.x;
+    int64_t first = 0;
+    for (int q = 0; q < k; ++q) first += (g.rows[q] + LOSS_TILE_ROWS - 1) / LOSS_TILE_ROWS;
+    const int64_t count = (g.rows[k] + LOSS_TILE_ROWS - 1) / LOSS_TILE_ROWS;
+    float s = 0.f;
+    for (int64_t t = threadIdx.x; t < count; t += 256) s += tile_loss[first + t];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0)
+        loss_out[(int64_t)g.part[k] * loss_stride + loss_col] = g.rows[k] > 0 ? red[0] / (float)g.rows[k] : 0.f;
+}
+
+}  // namespace
+
+int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp, float* tile_loss,
+                            float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s) {
+    const int64_t tiles = group_tiles(g, LOSS_TILE_ROWS);
+    if (tiles > 0) {
+        softmax_xent_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, tile_loss);
+        RTMA_LAUNCH_CHECK(ctx);
+    }
+    if (loss_out && g.num > 0) {
+        loss_finalize_kernel<<<g.num, 256, 0, s>>>(g, tile_loss, loss_out, loss_stride, loss_col);
+        RTMA_LAUNCH_CHECK(ctx);
+    }
+    return RTMA_OK;
+}

@@ -1,0 +1,121 @@
+// Randomized assignment of nodes (RandomTMA) or super-nodes (SuperTMA) to M trainers
+// (Sec. 3.2.2) and the ordered member lists alpha^{-1}(i) (Preliminaries).
+//
+// Three launches, no atomics on global memory and no inter-block waits, so the result is
+// the unique stable order (ascending node id inside every part):
+//   1. every warp hashes a chunk of 1024 consecutive nodes and counts them per part;
+//   2. an exclusive scan over the counts, laid out part-major, gives for every
+//      (part, chunk) the first output slot of that chunk's members;
+//   3. every warp hashes its chunk again and ranks its nodes inside the warp with
+//      match.any, 32 nodes per round, which keeps id order.
+#include "common.cuh"
+
+namespace {
+
+constexpr int PART_THREADS = 256;
+constexpr int PART_WARPS = PART_THREADS / 32;
+constexpr int PART_ROUNDS = 32;
+constexpr int PART_CHUNK = 32 * PART_ROUNDS;
+
+// One step of the SplitMix64 generator (Steele, Lea, Flood 2014): add the golden-ratio
+// increment, then the 64-bit finaliser.
+__device__ __forceinline__ uint64_t splitmix64_step(uint64_t x) {
+    uint64_t z = x + 0x9E3779B97F4A7C15ULL;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+__device__ __forceinline__ int part_of(int64_t v, const int32_t* __restrict__ group_id, uint64_t seed, int M) {
+    const uint64_t g = group_id ? (uint64_t)(int64_t)group_id[v] : (uint64_t)v;
+    return (int)(splitmix64_step(seed ^ g) % (uint64_t)M);
+}
+
+__global__ void __launch_bounds__(PART_THREADS)
+part_count_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t seed, int M, int64_t num_chunks,
+                  int32_t* __restrict__ counts) {
+    __shared__ int32_t hist[PART_WARPS][RTMA_MAX_PARTS + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t chunk = (int64_t)blockIdx.x * PART_WARPS + warp;
+    for (int b = lane; b <= RTMA_MAX_PARTS; b += 32) hist[warp][b] = 0;
+    __syncwarp();
+    if (chunk >= num_chunks) return;
+    for (int r = 0; r < PART_ROUNDS; ++r) {
+        const int64_t v = chunk * PART_CHUNK + r * 32 + lane;
+        const int pid = v < n ? part_of(v, group_id, seed, M) : M;
+        const unsigned peers = __match_any_sync(0xffffffffu, pid);
+        if (lane == __ffs(peers) - 1) hist[warp][pid] += __popc(peers);
+        __syncwarp();
+    }
+    for (int b = lane; b < M; b += 32) counts[(int64_t)b * num_chunks + chunk] = hist[warp][b];
+}
+
+__global__ void __launch_bounds__(PART_THREADS)
+part_scatter_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t seed, int M, int64_t num_chunks,
+                    const int64_t* __restrict__ scanned, int32_t* __restrict__ part_id,
+                    int64_t* __restrict__ part_offsets, int32_t* __restrict__ perm,
+                    int32_t* __restrict__ local_id) {
+    __shared__ int32_t cursor[PART_WARPS][RTMA_MAX_PARTS + 1];
+    __shared__ int32_t first_slot[RTMA_MAX_PARTS + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t chunk = (int64_t)blockIdx.x * PART_WARPS + warp;
+    for (int b = threadIdx.x; b < M; b += PART_THREADS) first_slot[b] = (int32_t)scanned[(int64_t)b * num_chunks];
+    if (blockIdx.x == 0)
+        for (int b = threadIdx.x; b <= M; b += PART_THREADS)
+            part_offsets[b] = b < M ? scanned[(int64_t)b * num_chunks] : n;
+    if (chunk < num_chunks)
+        for (int b = lane; b < M; b += 32) cursor[warp][b] = (int32_t)scanned[(int64_t)b * num_chunks + chunk];
+    __syncthreads();
+    if (chunk >= num_chunks) return;
+    const unsigned below = (1u << lane) - 1u;
+    for (int r = 0; r < PART_ROUNDS; ++r) {
+        const int64_t v = chunk * PART_CHUNK + r * 32 + lane;
+        const bool live = v < n;
+        const int pid = live ? part_of(v, group_id, seed, M) : M;
+        const unsigned peers = __match_any_sync(0xffffffffu, pid);
+        const int slot = live ? cursor[warp][pid] + __popc(peers & below) : 0;
+        __syncwarp();
+        if (live && lane == __ffs(peers) - 1) cursor[warp][pid] += __popc(peers);
+        __syncwarp();
+        if (live) {
+            part_id[v] = pid;
+            local_id[v] = slot - first_slot[pid];
+            perm[slot] = (int32_t)v;
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group_id, uint64_t seed, int32_t M,
+                                  int32_t* part_id, int64_t* part_offsets, int32_t* perm, int32_t* local_id,
+                                  void* stream_) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
+    if (n < 0 || n >= (int64_t(1) << 31)) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "n=%lld outside [0,2^31)", (long long)n);
+    if (!part_offsets || (n > 0 && (!part_id || !perm || !local_id)))
+        return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_partition: null output pointer");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    if (n == 0) {
+        RTMA_CUDA(ctx, cudaMemsetAsync(part_offsets, 0, sizeof(int64_t) * (M + 1), stream));
+        return RTMA_OK;
+    }
+    const int64_t num_chunks = ceil_div(n, PART_CHUNK);
+    const int64_t cells = num_chunks * M;
+    const size_t need = ArenaCursor::granule(sizeof(int32_t) * cells) + ArenaCursor::granule(sizeof(int64_t) * (cells + 1)) +
+                        ArenaCursor::granule(sizeof(int64_t) * scan_scratch_elems(cells));
+    RTMA_TRY(rtma_reserve(ctx, need));
+    ArenaCursor cur(ctx->arena);
+    int32_t* counts = cur.take<int32_t>(cells);
+    int64_t* scanned = cur.take<int64_t>(cells + 1);
+    int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(cells));
+    const unsigned blocks = (unsigned)ceil_div(num_chunks, PART_WARPS);
+    part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts);
+    RTMA_LAUNCH_CHECK(ctx);
+    RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, cells, scanned, scratch, stream));
+    part_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, scanned, part_id,
+                                                             part_offsets, perm, local_id);
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}

@@ -1,0 +1,95 @@
+// Declarations shared by the local-training kernels (Algorithm 2's loop body) and the
+// host code that sequences them.
+#pragma once
+
+#include "common.cuh"
+
+// A group = the trainers that share one stream and one scratch region.  Its kernels cover
+// all of the group's parts in one launch; a tile never straddles two parts because every
+// part multiplies by its own parameter replica.
+struct GroupDesc {
+    int32_t num;                        // parts in the group
+    int32_t part[RTMA_MAX_PARTS];       // trainer index i of each part
+    int32_t rows[RTMA_MAX_PARTS];       // n_p
+    int64_t row_abs[RTMA_MAX_PARTS];    // first row in partition order (Xp, yp; rowptr_out at row_abs + part)
+    int64_t row_ws[RTMA_MAX_PARTS];     // first row inside the group's scratch matrices
+    int64_t edge_abs[RTMA_MAX_PARTS];   // first entry of the part in col_out
+};
+
+// Tiles of `tile_rows` rows, numbered part after part.
+inline int64_t group_tiles(const GroupDesc& g, int tile_rows) {
+    int64_t t = 0;
+    for (int k = 0; k < g.num; ++k) t += ceil_div(g.rows[k], tile_rows);
+    return t;
+}
+
+#ifdef __CUDACC__
+// Maps a tile number to (slot k in the group, first row of the tile inside the part).
+__device__ __forceinline__ bool locate_tile(const GroupDesc& g, int tile_rows, int64_t tile, int* k_out, int* row_out) {
+    for (int k = 0; k < g.num; ++k) {
+        const int64_t t = (g.rows[k] + tile_rows - 1) / tile_rows;
+        if (tile < t) {
+            *k_out = k;
+            *row_out = (int)tile * tile_rows;
+            return true;
+        }
+        tile -= t;
+    }
+    return false;
+}
+#endif
+
+// A matrix of activations: rows addressed either by absolute partition-order row (the
+// caller's Xp) or by the group's scratch row.
+struct Mat {
+    float* ptr;
+    int64_t ld;       // floats between rows
+    int32_t absolute; // 1: row index = row_abs[k] + i, 0: row_ws[k] + i
+};
+
+inline size_t padded_ld(int64_t d) { return (size_t)((d + 3) / 4 * 4); }
+
+// ---- spmm.cu --------------------------------------------------------------------------
+// inv_deg[row_ws + i] = 1 / local degree (0 for an isolated node).
+int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s);
+// out[r] = inv_deg[r] * sum_{u in N(r)} src[u]                      (forward, mean)
+int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                         const float* inv_deg, Mat src, Mat out, int d, cudaStream_t s);
+// out[r] = (self[r] + sum_{u in N(r)} src[u]) where gate[r] > 0 else 0   (backward through the
+// symmetric aggregation and the ReLU; out may alias gate)
+int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                             Mat src, Mat self, Mat gate, Mat out, int d, cudaStream_t s);
+
+// ---- gemm_simt.cu ---------------------------------------------------------------------
+struct LayerShape {
+    int32_t d_in, d_out;
+    int64_t param_offset;  // of Ws inside one replica; Ws, Wn, b are contiguous: a (2 d_in + 1) x d_out matrix
+    int64_t P;             // parameters per replica
+};
+// out = act([H | N | 1] * [Ws; Wn; b])
+int32_t launch_layer_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const float* params, Mat H, Mat N,
+                             Mat out, bool relu, cudaStream_t s);
+// ST[:, 0:d_in] = dZ Ws^T ;  ST[:, d_in:2 d_in] = inv_deg * (dZ Wn^T)
+int32_t launch_layer_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const float* params, Mat dZ,
+                           const float* inv_deg, Mat ST, cudaStream_t s);
+// partial[slot][(2 d_in + 1) x d_out] = [H | N | 1]^T dZ over one chunk of rows; chunks of part k
+// occupy slots split_begin[k] .. split_begin[k+1].
+struct SplitPlan {
+    int32_t split_begin[RTMA_MAX_PARTS + 1];
+    int32_t rows_per_split[RTMA_MAX_PARTS];
+};
+int32_t launch_layer_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, Mat H, Mat N, Mat dZ,
+                           float* partial, cudaStream_t s);
+
+// ---- loss.cu --------------------------------------------------------------------------
+// Softmax cross-entropy over logits (in place: logits become dL/dlogits), mean over the part.
+// loss_out[part * loss_stride + loss_col] receives the part's loss when loss_out != NULL.
+int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp,
+                            float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s);
+
+// ---- optim.cu -------------------------------------------------------------------------
+// grad = sum of the part's partial slots; params -= lr * grad; optionally records grad.
+int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, const float* partial,
+                          float lr, float* params, float* grads_record, cudaStream_t s);
+int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float* dst, int64_t ld_dst, int64_t rows,
+                         int width, cudaStream_t s);

@@ -1,0 +1,98 @@
+"""GPU parity, integer half: partition ids, relabels and induced CSR arrays must be
+bit-identical to the oracle's on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2305_09887_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def util():
+    import gpu_util
+    return gpu_util
+
+
+@pytest.mark.parametrize("n,M", [(1, 1), (7, 3), (1000, 64), (1024, 5), (1025, 5), (8192, 32), (8193, 23),
+                                 (100_003, 4), (1_000_000, 32)])
+def test_partition_matches_oracle(util, n, M):
+    seed = 0x5EED0005 + n
+    got = util.ctx().partition(n, None, seed, M)
+    want = oracle.partition(n, None, seed, M)
+    for a, b in zip(got, want):
+        assert np.array_equal(a.cpu().numpy(), b)
+
+
+def test_partition_empty_and_supernodes(util):
+    part_id, part_offsets, perm, local_id = util.ctx().partition(0, None, 1, 4)
+    assert part_offsets.cpu().tolist() == [0] * 5 and part_id.numel() == 0
+    n, M, seed = 250_000, 16, 99
+    group = (np.random.default_rng(0).integers(0, 2500, size=n) * 11 - 7).astype(np.int32)  # sparse, some negative
+    got = util.ctx().partition(n, util.dev(group), seed, M)
+    want = oracle.partition(n, group, seed, M)
+    for a, b in zip(got, want):
+        assert np.array_equal(a.cpu().numpy(), b)
+
+
+def test_partition_is_deterministic(util):
+    a = util.ctx().partition(300_000, None, 5, 8)
+    b = util.ctx().partition(300_000, None, 5, 8)
+    assert all(torch.equal(x, y) for x, y in zip(a, b))
+
+
+@pytest.mark.parametrize("M", [1, 4, 23])
+def test_induced_csr_tiny(util, tiny_workload, M):
+    util.assert_preprocess_equal(util.gpu_preprocess(tiny_workload, M=M), util.oracle_preprocess(tiny_workload, M=M))
+
+
+def test_induced_csr_power_law_int64_rowptr(util):
+    w = inputs.medium(0.25)
+    w.graph.rowptr = w.graph.rowptr.astype(np.int64)
+    got = util.gpu_preprocess(w, M=8)
+    want = util.oracle_preprocess(w, M=8)
+    util.assert_preprocess_equal(got, want)
+    assert abs(want["kept"] / w.graph.num_entries - 1 / 8) < 0.01     # Sec. 3.2.2: kept fraction 1/M
+
+
+def test_induced_csr_supernodes(util):
+    w = inputs.supertma(0.02)
+    got = util.gpu_preprocess(w)
+    want = util.oracle_preprocess(w)
+    util.assert_preprocess_equal(got, want)
+    assert want["kept"] / w.graph.num_entries > 0.6                   # most edges live inside super-nodes
+
+
+def test_induced_csr_degenerate_graphs(util):
+    c = util.ctx()
+    # no edges at all
+    n, M = 100, 4
+    rowptr = np.zeros(n + 1, dtype=np.int32)
+    col = np.zeros(0, dtype=np.int32)
+    p = c.partition(n, None, 3, M)
+    rowptr_out, col_out, edge_offsets, kept_cut, edge_host = c.build_induced_csr(
+        util.dev(rowptr), torch.empty(0, dtype=torch.int32, device="cuda"), M, *p)
+    assert edge_host == [0] * (M + 1) and kept_cut.cpu().tolist() == [0, 0]
+    assert rowptr_out.cpu().abs().sum().item() == 0
+    # one hub row much longer than a warp, directed entries, self loop, duplicates
+    rowptr = np.array([0, 1000, 1001, 1001, 1003], dtype=np.int64)
+    col = np.concatenate([np.arange(1000) % 4, [1], [3, 3]]).astype(np.int32)
+    part_id = oracle.assign(4, None, 11, 2)
+    po, perm, lid = oracle.relabel(part_id, 2)
+    want = oracle.induced_csr(rowptr, col, 2, part_id, po, perm, lid)
+    gp = c.partition(4, None, 11, 2)
+    got = c.build_induced_csr(util.dev(rowptr), util.dev(col), 2, *gp)
+    assert np.array_equal(got[0].cpu().numpy(), want[0]) and np.array_equal(got[1].cpu().numpy(), want[1])
+    assert got[3].cpu().tolist() == [want[3], want[4]]
+
+
+@pytest.mark.parametrize("shape,dtype", [((1000, 100), np.float32), ((1000,), np.int32), ((333, 3), np.uint8),
+                                         ((257, 129), np.float32)])
+def test_gather_rows(util, shape, dtype):
+    rng = np.random.default_rng(0)
+    src = (rng.standard_normal(shape) * 100).astype(dtype)
+    perm = rng.permutation(shape[0]).astype(np.int32)
+    got = util.ctx().gather_rows(util.dev(src), util.dev(perm)).cpu().numpy()
+    assert np.array_equal(got, src[perm])

@@ -1,0 +1,213 @@
+"""GPU parity, floating-point half: activations, gradients, losses and parameters after
+K local steps and after averaging, against the fp64 oracle on the same seeded inputs.
+
+Tolerances (relative = max|a-b| / max|b| per tensor): 1e-4 on forward activations, 1e-3 on
+gradients and on parameters after K steps / after averaging (fp32-accurate GEMM path);
+5e-3 when GEMM operands are bf16.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2305_09887_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_ACT, TOL_GRAD, TOL_PARAM = 1e-4, 1e-3, 1e-3
+
+
+@pytest.fixture(scope="module")
+def util():
+    import gpu_util
+    return gpu_util
+
+
+def _oracle_parts(w, pre):
+    """Per-part (rowptr, col, X, y) from the oracle's preprocessing."""
+    out = []
+    for p in range(pre["M"]):
+        rp, cp = oracle.part_graph(pre["rowptr_out"], pre["col_out"], pre["part_offsets"], pre["edge_offsets"], p)
+        lo, hi = int(pre["part_offsets"][p]), int(pre["part_offsets"][p + 1])
+        out.append((rp, cp, pre["Xp"][lo:hi].astype(np.float64), pre["yp"][lo:hi]))
+    return out
+
+
+def _check_one_step(util, w, M=None, gemm_dtype=0, tol_scale=1.0, streams=None):
+    """Step 0 intermediates and gradients, then K steps and the average."""
+    c = util.ctx()
+    got = util.gpu_preprocess(w, M=M)
+    want = util.oracle_preprocess(w, M=M)
+    util.assert_preprocess_equal(got, want)
+    M = got["M"]
+    dims, n = w.dims, w.graph.n
+    P = inputs.param_count(dims)
+    rec = sum(dims[l] + dims[l + 1] for l in range(len(dims) - 1))
+    params = util.dev(np.tile(w.params0, (M, 1)))
+    acts = torch.zeros(n * rec, dtype=torch.float32, device="cuda")
+    grads = torch.zeros(M, P, dtype=torch.float32, device="cuda")
+    loss = torch.zeros(M, 1, dtype=torch.float32, device="cuda")
+    c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
+                  got["Xp"], got["yp"], params, 1, loss_out=loss, taps=(acts, grads, 0), gemm_dtype=gemm_dtype,
+                  streams=streams)
+    torch.cuda.synchronize()
+    acts, grads, loss, params1 = acts.cpu().numpy(), grads.cpu().numpy(), loss.cpu().numpy(), params.cpu().numpy()
+    p0 = w.params0.astype(np.float64)
+    for p, (rp, cp, X, y) in enumerate(_oracle_parts(w, want)):
+        n_p = rp.size - 1
+        o_loss, o_grads, o_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True)
+        layout, total = oracle.acts_layout(dims, n_p)
+        base = int(want["part_offsets"][p]) * rec
+        for name, off, r, wd in layout:
+            a = acts[base + off: base + off + r * wd].reshape(r, wd)
+            assert util.rel_err(a, o_acts[name]) <= TOL_ACT * tol_scale, (p, name)
+        if n_p:
+            assert abs(loss[p, 0] - o_loss) <= 1e-5 * tol_scale * max(1.0, abs(o_loss)), p
+        # gradients: per parameter tensor
+        off = 0
+        for l in range(len(dims) - 1):
+            for nm, size in (("Ws", dims[l] * dims[l + 1]), ("Wn", dims[l] * dims[l + 1]), ("b", dims[l + 1])):
+                gg, og = grads[p, off:off + size], o_grads[off:off + size]
+                if np.abs(og).max() > 0:
+                    assert util.rel_err(gg, og) <= TOL_GRAD * tol_scale, (p, l, nm)
+                else:
+                    assert np.abs(gg).max() == 0
+                off += size
+        assert util.rel_err(params1[p], p0 - w.lr * o_grads) <= TOL_PARAM * tol_scale
+    return got, want
+
+
+def _check_k_steps_and_average(util, w, got, want, K, gemm_dtype=0, tol_scale=1.0, streams=None):
+    c = util.ctx()
+    M, dims = got["M"], w.dims
+    params = util.dev(np.tile(w.params0, (M, 1)))
+    loss = torch.zeros(M, K, dtype=torch.float32, device="cuda")
+    c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
+                  got["Xp"], got["yp"], params, K, loss_out=loss, gemm_dtype=gemm_dtype, streams=streams)
+    torch.cuda.synchronize()
+    after = params.cpu().numpy().copy()
+    glob = torch.empty(params.shape[1], dtype=torch.float32, device="cuda")
+    c.aggregate(params, glob)
+    torch.cuda.synchronize()
+    o_params = np.empty((M, params.shape[1]))
+    for p, (rp, cp, X, y) in enumerate(_oracle_parts(w, want)):
+        o_params[p], o_loss = oracle.local_steps(dims, w.lr, rp, cp, X, y, w.params0.astype(np.float64), K)
+        assert util.rel_err(after[p], o_params[p]) <= TOL_PARAM * tol_scale, p
+        if rp.size > 1:
+            assert np.abs(loss[p].cpu().numpy() - o_loss).max() <= 1e-4 * tol_scale * max(1.0, np.abs(o_loss).max())
+    o_avg, o_glob = oracle.average(o_params)
+    assert util.rel_err(glob.cpu().numpy(), o_glob) <= TOL_PARAM * tol_scale
+    pa = params.cpu().numpy()
+    for p in range(M):
+        assert np.array_equal(pa[p], glob.cpu().numpy())     # every local copy overwritten
+    return after
+
+
+def test_tiny_config_end_to_end(util, tiny_workload):
+    w = tiny_workload
+    got, want = _check_one_step(util, w)
+    _check_k_steps_and_average(util, w, got, want, w.K)
+
+
+def test_medium_shape_scaled(util):
+    # the Medium model (128-256-256-47, M=8) on a 12k-node power-law graph: several row tiles
+    # per part plus a ragged tail, hubs, isolated local nodes
+    w = inputs.medium(0.06)
+    got, want = _check_one_step(util, w)
+    _check_k_steps_and_average(util, w, got, want, 2)
+
+
+def test_supertma_shape_scaled_feature_width_100(util):
+    w = inputs.supertma(0.02, M=4)   # 40k nodes, F=100 (rows of 400 bytes), super-node assignment
+    w.dims = (100, 64, 47)
+    w.params0 = inputs.xavier_params(w.dims, 5)
+    got, want = _check_one_step(util, w)
+    _check_k_steps_and_average(util, w, got, want, 2)
+
+
+@pytest.mark.parametrize("dims", [(6, 5, 3), (33, 2), (17, 130, 7, 2)])
+def test_odd_widths_and_binary_head(util, tiny_workload, dims):
+    w = inputs.tiny()
+    w.dims = dims
+    w.X = inputs.normal_features(w.graph.n, dims[0], 3)
+    w.y = inputs.rare_positive_labels(w.graph.n, 0.1, 4) if dims[-1] == 2 else inputs.uniform_labels(w.graph.n, dims[-1], 4)
+    w.params0 = inputs.xavier_params(dims, 6)
+    got, want = _check_one_step(util, w, M=3)
+    _check_k_steps_and_average(util, w, got, want, 3)
+
+
+def test_more_trainers_than_busy_parts(util):
+    # 40 nodes over 64 trainers: many empty parts, most nodes isolated
+    w = inputs.tiny()
+    g = inputs.uniform_graph(40, 100, 3)
+    w.graph, w.X, w.y = g, w.X[:40].copy(), w.y[:40].copy()
+    got, want = _check_one_step(util, w, M=64)
+    assert min(np.diff(want["part_offsets"])) == 0
+    _check_k_steps_and_average(util, w, got, want, 2)
+
+
+def test_streams_do_not_change_the_result(util, tiny_workload):
+    w = tiny_workload
+    got = util.gpu_preprocess(w)
+    want = util.oracle_preprocess(w)
+    one = _check_k_steps_and_average(util, w, got, want, 3)
+    streams = [torch.cuda.Stream() for _ in range(w.M)]
+    torch.cuda.synchronize()
+    many = _check_k_steps_and_average(util, w, got, want, 3, streams=streams)
+    pairs = [streams[0], streams[1], streams[0], streams[1]]
+    two = _check_k_steps_and_average(util, w, got, want, 3, streams=pairs)
+    assert np.array_equal(one, many) and np.array_equal(one, two)
+
+
+def test_zero_steps_and_zero_learning_rate(util, tiny_workload):
+    w = tiny_workload
+    c = util.ctx()
+    got = util.gpu_preprocess(w)
+    params = util.dev(np.tile(w.params0, (w.M, 1)))
+    args = (w.M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"], got["Xp"], got["yp"], params)
+    c.local_steps(w.dims, w.lr, *args, 0)
+    c.aggregate(params)
+    torch.cuda.synchronize()
+    assert np.array_equal(params.cpu().numpy(), np.tile(w.params0, (w.M, 1)))   # K = 0: initial weights
+    c.local_steps(w.dims, 0.0, *args, 2)
+    torch.cuda.synchronize()
+    assert np.array_equal(params.cpu().numpy(), np.tile(w.params0, (w.M, 1)))   # lr = 0: unchanged
+
+
+@pytest.mark.parametrize("M,P", [(1, 1000), (4, 9288), (7, 1001), (32, 66818), (64, 4096)])
+def test_aggregate_matches_oracle(util, M, P):
+    rng = np.random.default_rng(M * 1000 + P)
+    W = rng.standard_normal((M, P)).astype(np.float32)
+    params = util.dev(W)
+    glob = torch.empty(P, dtype=torch.float32, device="cuda")
+    util.ctx().aggregate(params, glob)
+    torch.cuda.synchronize()
+    o_avg, o_glob = oracle.average(W.astype(np.float64))
+    assert util.rel_err(glob.cpu().numpy(), o_glob) <= 1e-6
+    assert np.array_equal(params.cpu().numpy(), np.tile(glob.cpu().numpy(), (M, 1)))
+    if M == 1:
+        assert np.array_equal(params.cpu().numpy(), W)
+
+
+def test_sgd_aggregate_is_step_then_average(util):
+    rng = np.random.default_rng(0)
+    M, P, lr = 8, 20000, 0.05
+    W = rng.standard_normal((M, P)).astype(np.float32)
+    G = rng.standard_normal((M, P)).astype(np.float32)
+    params = util.dev(W)
+    util.ctx().sgd_aggregate(params, util.dev(G), lr)
+    torch.cuda.synchronize()
+    _, o_glob = oracle.average(W.astype(np.float64) - lr * G.astype(np.float64))
+    assert util.rel_err(params.cpu().numpy()[3], o_glob) <= 1e-6
+
+
+def test_whole_path_from_host_buffers(util, tiny_workload):
+    w = tiny_workload
+    g = w.graph
+    R = 2
+    params, losses, kept, cut = util.ctx().train_host(g.rowptr, g.col, w.X, w.y, w.dims, w.M, w.K, R, w.lr,
+                                                      w.partition_seed, w.params0)
+    res = oracle.run_method(g.rowptr, g.col, w.X, w.y, w.dims, w.M, w.K, R, w.lr, w.partition_seed, w.params0)
+    assert (kept, cut) == (res["kept"], res["cut"])
+    assert util.rel_err(params, res["params"][0]) <= TOL_PARAM
+    assert np.abs(losses - res["losses"]).max() <= 1e-4
