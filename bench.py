@@ -1,0 +1,392 @@
+#!/usr/bin/env python
+"""Benchmark of the whole RandomTMA hot path on one B200 (or N independent replicas).
+
+One step = one pass of the whole path over the Medium workload (Chung-Lu power-law graph,
+200k nodes, ~5M directed entries, 128-d features, 47 classes, M=8 trainers, 128-256-256-47
+GraphSAGE-mean, 20 local steps per round, 5 aggregation rounds): broadcast of the initial
+weights, partition, induced CSR (count + fill), row gather, then 5 x (20 local steps on all
+8 parts + aggregation).
+
+Metric: aggregated edges/s = (sum over parts of kept entries) x (SpMM passes per local step:
+L forward + L-1 backward) x (local steps) / time.  Local trainer-steps/s is reported beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints one JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "aggregated_edges_per_s"
+UNIT = "edges/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+SM_COUNT, FP32_LANES_PER_SM = 148, 128
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS, bf16_tflops_sustained=1400.0,
+                sm_max_mhz=1965.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------------------
+# workload arithmetic (algorithmic work per kernel class for one bench step)
+# ---------------------------------------------------------------------------------------
+def algorithmic_work(dims, n_parts, e_parts, K, R):
+    """Per kernel class: (bound, algorithmic bytes, algorithmic flops) summed over one bench
+    step.  Bytes are compulsory traffic (every operand read once, every result written once)."""
+    L = len(dims) - 1
+    n, e = float(sum(n_parts)), float(sum(e_parts))
+    steps = K * R
+    work = {}
+    spmm_f = sum(n * 8 * dims[l] + 4 * e + 8 * n for l in range(L))
+    spmm_b = sum(n * (4 * dims[l] * 2 + 4 * dims[l] * 2) + 4 * e + 8 * n for l in range(1, L))
+    work["spmm_forward"] = ("hbm", steps * spmm_f, steps * sum(e * dims[l] for l in range(L)))
+    work["spmm_backward"] = ("hbm", steps * spmm_b, steps * sum(e * dims[l] for l in range(1, L)))
+    Mtr = len(n_parts)
+    gf_b = sum(4 * n * (2 * dims[l] + dims[l + 1]) + 4 * Mtr * (2 * dims[l] + 1) * dims[l + 1] for l in range(L))
+    gf_f = sum(2 * n * (2 * dims[l] + 1) * dims[l + 1] for l in range(L))
+    work["gemm_forward"] = ("flops", steps * gf_b, steps * gf_f)
+    work["gemm_wgrad"] = ("flops", steps * gf_b, steps * gf_f)
+    gd_b = sum(4 * n * (2 * dims[l] + dims[l + 1]) + 4 * Mtr * 2 * dims[l] * dims[l + 1] for l in range(1, L))
+    gd_f = sum(2 * n * 2 * dims[l] * dims[l + 1] for l in range(1, L))
+    work["gemm_dgrad"] = ("flops", steps * gd_b, steps * gd_f)
+    P = sum((2 * dims[l] + 1) * dims[l + 1] for l in range(L))
+    work["softmax_xent"] = ("hbm", steps * (8 * n * dims[L] + 4 * n), 0.0)
+    work["reduce_sgd"] = ("hbm", steps * 12.0 * Mtr * P, 0.0)
+    work["aggregate"] = ("hbm", R * 8.0 * Mtr * P, 0.0)
+    return work
+
+
+# ---------------------------------------------------------------------------------------
+# clock sampling during the timed region
+# ---------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------
+# CPU baseline: the checker program as it stands, on a bounded sample
+# ---------------------------------------------------------------------------------------
+def cpu_sample(w, local_steps=1):
+    """Times the CPU checker on a bounded sample of the workload: partition + induced CSR + row
+    gather of the whole graph, then `local_steps` local steps of trainer 0 only.  Returns the
+    whole-workload figure extrapolated from it (every other trainer-step costed like trainer 0's)."""
+    import oracle
+    g = w.graph
+    L = len(w.dims) - 1
+    t0 = time.perf_counter()
+    part_id, part_offsets, perm, local_id = oracle.partition(g.n, None, w.partition_seed, w.M)
+    rowptr_out, col_out, edge_offsets, kept, cut = oracle.induced_csr(
+        g.rowptr, g.col, w.M, part_id, part_offsets, perm, local_id)
+    Xp = oracle.gather_rows(w.X, perm)
+    yp = oracle.gather_rows(w.y, perm)
+    t_pre = time.perf_counter() - t0
+    rp, cp = oracle.part_graph(rowptr_out, col_out, part_offsets, edge_offsets, 0)
+    hi = int(part_offsets[1])
+    t1 = time.perf_counter()
+    oracle.local_steps(w.dims, w.lr, rp, cp, Xp[:hi], yp[:hi], w.params0, local_steps)
+    t_step = (time.perf_counter() - t1) / local_steps
+    passes = 2 * L - 1
+    units_full = float(kept) * passes * w.K * w.R
+    est_full_s = t_pre + w.K * w.R * w.M * t_step
+    return dict(value=units_full / est_full_s, t_pre_s=t_pre, t_step_s=t_step, sample_s=t_pre + t_step * local_steps,
+                trainer_steps_per_s=1.0 / t_step,
+                sample=(f"partition+induced CSR+row gather of all {g.n} nodes ({t_pre:.2f} s), then {local_steps} "
+                        f"local step(s) of trainer 0 ({hi} nodes, {cp.size} entries; {t_step:.2f} s/step); "
+                        f"whole workload extrapolated as t_pre + K*R*M*t_step"))
+
+
+def run_reference(args, w):
+    """`--impl reference`: the CPU checker, single-threaded, timed on the host cores."""
+    steps, warmup = args.steps, args.warmup
+    for _ in range(warmup):
+        cpu_sample(w)
+    t0 = time.perf_counter()
+    samples = [cpu_sample(w) for _ in range(steps)]
+    wall = time.perf_counter() - t0
+    value = statistics.mean(s["value"] for s in samples)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": 1e3 * wall / max(steps, 1), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "nodes": w.graph.n, "entries": w.graph.num_entries, "M": w.M,
+                   "dims": list(w.dims), "K": w.K, "R": w.R, "timing": "host wall clock, bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": samples[-1]["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "trainer_steps_per_s": statistics.mean(s["trainer_steps_per_s"] for s in samples),
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------
+def max_over_ranks(seconds: float, dist_mod=None, device=None) -> float:
+    """Largest value over all ranks (the slowest rank sets the job's time)."""
+    if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
+        return seconds
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist_mod.all_reduce(t, op=dist_mod.ReduceOp.MAX)
+    return float(t.item())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_2305_09887_b200 import inputs
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, inputs.medium())
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2305_09887_b200 import binding
+
+    if args.warmup < 3:
+        args.warmup = 3
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    w = inputs.medium()
+    g = w.graph
+    L = len(w.dims) - 1
+    ctx = binding.Context(local_rank)
+    d_rowptr = torch.from_numpy(g.rowptr).to(device)
+    d_col = torch.from_numpy(g.col).to(device)
+    d_X = torch.from_numpy(w.X).to(device)
+    d_y = torch.from_numpy(w.y).to(device)
+    d_params0 = torch.from_numpy(w.params0).to(device)
+    P = w.params0.size
+    params = torch.empty(w.M, P, dtype=torch.float32, device=device)
+    loss = torch.zeros(w.R, w.M, w.K, dtype=torch.float32, device=device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)  # > 126 MB of L2
+    state = {}
+
+    def step():
+        params.copy_(d_params0.expand(w.M, P))                      # W_global[0] broadcast to the trainers
+        part_id, part_offsets, perm, local_id = ctx.partition(g.n, None, w.partition_seed, w.M)
+        rowptr_out, col_out, edge_offsets, kept_cut, edge_host = ctx.build_induced_csr(
+            d_rowptr, d_col, w.M, part_id, part_offsets, perm, local_id)
+        Xp = ctx.gather_rows(d_X, perm)
+        yp = ctx.gather_rows(d_y, perm)
+        part_host = part_offsets.cpu().tolist()
+        for r in range(w.R):
+            ctx.local_steps(w.dims, w.lr, w.M, part_host, edge_host, rowptr_out, col_out, Xp, yp, params, w.K,
+                            loss_out=loss[r])
+            ctx.aggregate(params)
+        state.update(part_host=part_host, edge_host=edge_host)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    ctx.profile_read()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ctx.profile(True)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)                                       # evict L2 between timed steps
+        starts[i].record()
+        step()
+        stops[i].record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    ctx.profile(False)
+    prof = ctx.profile_read()
+    clocks = sampler.stop()
+    elapsed_s = sum(a.elapsed_time(b) for a, b in zip(starts, stops)) / 1e3
+    elapsed_s = max_over_ranks(elapsed_s, dist if world > 1 else None, device)
+
+    n_parts = np.diff(state["part_host"]).tolist()
+    e_parts = np.diff(state["edge_host"]).tolist()
+    kept = float(sum(e_parts))
+    passes = 2 * L - 1
+    units_per_step = kept * passes * w.K * w.R
+    trainer_steps = w.M * w.K * w.R
+    value = world * args.steps * units_per_step / elapsed_s
+    final_loss = loss[-1, :, -1].mean().item()
+    first_loss = loss[0, :, 0].mean().item()
+
+    # ---- roofline of the dominant kernel class --------------------------------------
+    peaks = load_peaks()
+    work = algorithmic_work(w.dims, n_parts, e_parts, w.K, w.R)
+    total_kernel_ms = sum(ms for ms, _ in prof.values())
+    shares = {k: ms / total_kernel_ms for k, (ms, _) in prof.items() if ms > 0}
+    top = max(shares, key=shares.get)
+    top_ms, top_launches = prof[top]
+    gemm_dtype_note = "fp32 FMA on CUDA cores"
+    if top in work:
+        bound, abytes, aflops = work[top]
+        if bound == "hbm":
+            achieved = abytes * args.steps / (top_ms / 1e3) / 1e9
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        else:
+            achieved = aflops * args.steps / (top_ms / 1e3) / 1e12
+            alu_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+            roof = {"bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s", "note": gemm_dtype_note}
+    else:
+        roof = {"bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof.update({"frac": (roof["achieved"] / roof["peak"]) if roof["achieved"] else None, "traffic": None,
+                 "kernel": top, "launches_per_step": top_launches / args.steps,
+                 "avg_launch_us": 1e3 * top_ms / max(top_launches, 1), "share_of_kernel_time": shares[top],
+                 "peak_source": peaks["source"]})
+    per_class = {}
+    for k, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        entry = {"ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps,
+                 "share": ms / total_kernel_ms if total_kernel_ms else None}
+        if k in work and ms > 0:
+            bound, abytes, aflops = work[k]
+            entry["GBps"] = abytes * args.steps / (ms / 1e3) / 1e9
+            if aflops:
+                entry["TFLOPps"] = aflops * args.steps / (ms / 1e3) / 1e12
+        per_class[k] = entry
+    gpu_launches = int(sum(cnt for _, cnt in prof.values()))
+
+    # ---- end to end through the host-buffer entry point ------------------------------
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
+    h_rowptr, h_col, h_X, h_y, h_p0 = pin(g.rowptr), pin(g.col), pin(w.X), pin(w.y), pin(w.params0)
+    e2e_steps = max(1, min(args.steps, 3))
+    ctx.train_host(h_rowptr, h_col, h_X, h_y, w.dims, w.M, w.K, w.R, w.lr, w.partition_seed, h_p0)  # warm-up
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        out_params, out_losses, _, _ = ctx.train_host(h_rowptr, h_col, h_X, h_y, w.dims, w.M, w.K, w.R, w.lr,
+                                                      w.partition_seed, h_p0)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_s = max_over_ranks(e0.elapsed_time(e1) / 1e3, dist if world > 1 else None, device)
+    h2d = h_rowptr.nbytes + h_col.nbytes + h_X.nbytes + h_y.nbytes + w.M * h_p0.nbytes
+    d2h = out_params.nbytes + out_losses.nbytes + 16 + 2 * 8 * (w.M + 1)
+    e2e_value = world * e2e_steps * units_per_step / e2e_s
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * elapsed_s / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "nodes": g.n, "entries": g.num_entries, "kept_entries": int(kept), "M": w.M,
+                   "dims": list(w.dims), "K": w.K, "R": w.R, "spmm_passes_per_local_step": passes,
+                   "parallelism": "replicas only" if world > 1 else "single GPU, 8 trainers batched on one stream",
+                   "l2": "256 MB written between timed steps; per-step working set 1.5 GB > L2"},
+        "trainer_steps_per_s": world * args.steps * trainer_steps / elapsed_s,
+        "loss_first_last": [first_loss, final_loss],
+        "roofline": roof,
+        "kernels": per_class,
+        "gpu_launches": gpu_launches,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": 1e3 * e2e_s / e2e_steps, "steps": e2e_steps},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        cb = cpu_sample(w, local_steps=2)
+        line["cpu_baseline"] = {"value": cb["value"], "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": cb["sample"], "sample_seconds": cb["sample_s"],
+                                "trainer_steps_per_s": cb["trainer_steps_per_s"]}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

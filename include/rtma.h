@@ -154,6 +154,18 @@ int32_t rtma_aggregate(rtma_ctx* ctx, float* params, int64_t P, int32_t M, float
 int32_t rtma_sgd_aggregate(rtma_ctx* ctx, float* params, const float* grads, float lr, int64_t P,
                            int32_t M, float* global_out, void* stream);
 
+/* ---- instrumentation --------------------------------------------------------------------
+ * The library counts its kernel launches per class (RTMA_KERNEL_CLASSES classes, named by
+ * rtma_kernel_class_name).  rtma_profile(ctx, 1) additionally brackets every launch with CUDA
+ * events on the launching stream; rtma_profile_read synchronises the device, writes the time
+ * summed per class (ms [RTMA_KERNEL_CLASSES], milliseconds; zeros if profiling was off) and the
+ * launch counts (launches [RTMA_KERNEL_CLASSES]) since the previous read, and resets both.
+ * Either output may be NULL.  The paper has no counterpart; these feed the roofline report.  */
+#define RTMA_KERNEL_CLASSES 17
+int32_t rtma_profile(rtma_ctx* ctx, int32_t enable);
+int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launches);
+const char* rtma_kernel_class_name(int32_t cls);
+
 /* ---- the whole path on HOST buffers (Sec. 3: partition, Algorithm 2, Algorithm 1) --------
  * Every pointer here is a HOST pointer (pageable or pinned).  Copies the graph (CSR as for
  * rtma_build_induced_csr), group_id_h (NULL = RandomTMA), features X_h [n][dims[0]], labels

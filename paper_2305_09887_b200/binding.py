@@ -20,8 +20,10 @@ MAX_LAYERS = 8
 EXPORTS = (
     "rtma_create", "rtma_destroy", "rtma_last_error", "rtma_workspace_bytes", "rtma_partition",
     "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
-    "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host",
+    "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
+    "rtma_kernel_class_name",
 )
+KERNEL_CLASSES = 17
 
 _lib = None
 
@@ -52,6 +54,7 @@ def load_library():
         lib.rtma_workspace_bytes.restype = ctypes.c_size_t
         lib.rtma_workspace_bytes.argtypes = [ctypes.c_void_p]
         lib.rtma_param_count.restype = ctypes.c_int64
+        lib.rtma_kernel_class_name.restype = ctypes.c_char_p
         _lib = lib
     return _lib
 
@@ -133,6 +136,18 @@ class Context:
     @property
     def workspace_bytes(self) -> int:
         return int(self._lib.rtma_workspace_bytes(self._h))
+
+    # ---- instrumentation ------------------------------------------------------------
+    def profile(self, enable: bool):
+        self._check(self._lib.rtma_profile(self._h, ctypes.c_int32(1 if enable else 0)), "rtma_profile")
+
+    def profile_read(self):
+        """{class name: (milliseconds, launches)} since the previous read; synchronises."""
+        ms = (ctypes.c_double * KERNEL_CLASSES)()
+        cnt = (ctypes.c_int64 * KERNEL_CLASSES)()
+        self._check(self._lib.rtma_profile_read(self._h, ms, cnt), "rtma_profile_read")
+        return {self._lib.rtma_kernel_class_name(ctypes.c_int32(i)).decode(): (float(ms[i]), int(cnt[i]))
+                for i in range(KERNEL_CLASSES)}
 
     # ---- R1 -------------------------------------------------------------------------
     def partition(self, n: int, group_id, seed: int, M: int, stream=None):

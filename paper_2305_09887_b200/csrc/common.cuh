@@ -7,11 +7,29 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 #include "rtma.h"
 
+// Kernel classes, for launch counting and optional per-class timing.
+enum KernelClass {
+    KC_PART_COUNT = 0, KC_SCAN, KC_PART_SCATTER, KC_CSR_COUNT, KC_CSR_OFFSETS, KC_CSR_FILL, KC_GATHER_ROWS,
+    KC_INV_DEGREE, KC_SPMM_FWD, KC_SPMM_BWD, KC_GEMM_FWD, KC_GEMM_DGRAD, KC_GEMM_WGRAD, KC_LOSS, KC_REDUCE_SGD,
+    KC_AGGREGATE, KC_COPY, KC_COUNT
+};
+static_assert(KC_COUNT == RTMA_KERNEL_CLASSES, "kernel class table out of step with rtma.h");
+
+struct ProfSpan {
+    int cls;
+    cudaEvent_t start, stop;
+};
+
 struct rtma_ctx {
     int device = 0;
+    bool profiling = false;
+    int64_t launches[KC_COUNT] = {0};
+    std::vector<ProfSpan> spans;        // recorded since the last read
+    std::vector<cudaEvent_t> event_pool;  // spare events
     char* arena = nullptr;        // device scratch
     size_t arena_bytes = 0;
     void* pinned = nullptr;       // small pinned staging block for descriptors
@@ -44,6 +62,40 @@ inline int32_t rtma_fail(rtma_ctx* ctx, int32_t code, const char* fmt, ...) {
         int32_t s__ = (expr);               \
         if (s__ != RTMA_OK) return s__;     \
     } while (0)
+
+// Counts one kernel launch of class `cls`; with profiling on, brackets it with CUDA events on
+// the launching stream.  Use as:  { KernelScope ks(ctx, KC_X, stream); kernel<<<...>>>(...); }
+struct KernelScope {
+    rtma_ctx* ctx;
+    cudaStream_t stream;
+    cudaEvent_t stop = nullptr;
+    static cudaEvent_t event(rtma_ctx* c) {
+        cudaEvent_t e = nullptr;
+        if (!c->event_pool.empty()) {
+            e = c->event_pool.back();
+            c->event_pool.pop_back();
+        } else if (cudaEventCreate(&e) != cudaSuccess) {
+            e = nullptr;
+        }
+        return e;
+    }
+    KernelScope(rtma_ctx* c, int cls, cudaStream_t s) : ctx(c), stream(s) {
+        c->launches[cls]++;
+        if (c->profiling) {
+            cudaEvent_t start = event(c);
+            stop = event(c);
+            if (start && stop) {
+                cudaEventRecord(start, s);
+                c->spans.push_back(ProfSpan{cls, start, stop});
+            } else {
+                stop = nullptr;
+            }
+        }
+    }
+    ~KernelScope() {
+        if (stop) cudaEventRecord(stop, stream);
+    }
+};
 
 // Makes the arena at least `bytes` large.  Growing synchronises the device.
 int32_t rtma_reserve(rtma_ctx* ctx, size_t bytes);

@@ -33,6 +33,11 @@ extern "C" int32_t rtma_destroy(rtma_ctx* ctx) {
     cudaDeviceSynchronize();
     if (ctx->arena) cudaFree(ctx->arena);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    for (const ProfSpan& sp : ctx->spans) {
+        cudaEventDestroy(sp.start);
+        cudaEventDestroy(sp.stop);
+    }
+    for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
     delete ctx;
     return RTMA_OK;
 }
@@ -40,6 +45,41 @@ extern "C" int32_t rtma_destroy(rtma_ctx* ctx) {
 extern "C" const char* rtma_last_error(const rtma_ctx* ctx) { return ctx ? ctx->error : "null context"; }
 
 extern "C" size_t rtma_workspace_bytes(const rtma_ctx* ctx) { return ctx ? ctx->arena_bytes : 0; }
+
+static const char* const kKernelClassNames[KC_COUNT] = {
+    "partition_count", "scan", "partition_scatter", "induced_count", "induced_offsets", "induced_fill", "gather_rows",
+    "inv_degree", "spmm_forward", "spmm_backward", "gemm_forward", "gemm_dgrad", "gemm_wgrad", "softmax_xent",
+    "reduce_sgd", "aggregate", "copy_rows"};
+
+extern "C" const char* rtma_kernel_class_name(int32_t cls) {
+    return cls >= 0 && cls < KC_COUNT ? kKernelClassNames[cls] : "";
+}
+
+extern "C" int32_t rtma_profile(rtma_ctx* ctx, int32_t enable) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    ctx->profiling = enable != 0;
+    return RTMA_OK;
+}
+
+extern "C" int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launches) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_CUDA(ctx, cudaDeviceSynchronize());
+    for (int c = 0; c < KC_COUNT; ++c) {
+        if (ms) ms[c] = 0.0;
+        if (launches) launches[c] = ctx->launches[c];
+        ctx->launches[c] = 0;
+    }
+    for (const ProfSpan& sp : ctx->spans) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, sp.start, sp.stop) == cudaSuccess && ms) ms[sp.cls] += (double)t;
+        ctx->event_pool.push_back(sp.start);
+        ctx->event_pool.push_back(sp.stop);
+    }
+    cudaGetLastError();
+    ctx->spans.clear();
+    return RTMA_OK;
+}
 
 int32_t rtma_reserve(rtma_ctx* ctx, size_t bytes) {
     if (bytes <= ctx->arena_bytes) return RTMA_OK;
@@ -156,11 +196,11 @@ size_t scan_scratch_elems(int64_t n) { return (size_t)ceil_div(n + 1, SCAN_TILE)
 int32_t exclusive_scan_i32_to_i64(rtma_ctx* ctx, const int32_t* in, int64_t n, int64_t* out,
                                   int64_t* scratch, cudaStream_t stream) {
     const int64_t nb = ceil_div(n + 1, SCAN_TILE);
-    scan_reduce_kernel<<<(unsigned)nb, SCAN_THREADS, 0, stream>>>(in, n, scratch);
+    { KernelScope ks(ctx, KC_SCAN, stream); scan_reduce_kernel<<<(unsigned)nb, SCAN_THREADS, 0, stream>>>(in, n, scratch); }
     RTMA_LAUNCH_CHECK(ctx);
-    scan_spine_kernel<<<1, 1024, 0, stream>>>(scratch, nb);
+    { KernelScope ks(ctx, KC_SCAN, stream); scan_spine_kernel<<<1, 1024, 0, stream>>>(scratch, nb); }
     RTMA_LAUNCH_CHECK(ctx);
-    scan_apply_kernel<<<(unsigned)nb, SCAN_THREADS, 0, stream>>>(in, n, scratch, out);
+    { KernelScope ks(ctx, KC_SCAN, stream); scan_apply_kernel<<<(unsigned)nb, SCAN_THREADS, 0, stream>>>(in, n, scratch, out); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

@@ -164,7 +164,7 @@ int32_t launch_layer_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, c
     const int64_t tiles = group_tiles(g, BM);
     if (tiles == 0) return RTMA_OK;
     dim3 grid((unsigned)tiles, (unsigned)ceil_div(ls.d_out, BN));
-    layer_forward_kernel<<<grid, GEMM_THREADS, 0, s>>>(g, ls, params, H, N, out, relu ? 1 : 0);
+    { KernelScope ks(ctx, KC_GEMM_FWD, s); layer_forward_kernel<<<grid, GEMM_THREADS, 0, s>>>(g, ls, params, H, N, out, relu ? 1 : 0); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
@@ -174,7 +174,7 @@ int32_t launch_layer_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, con
     const int64_t tiles = group_tiles(g, BM);
     if (tiles == 0) return RTMA_OK;
     dim3 grid((unsigned)tiles, (unsigned)ceil_div(2 * ls.d_in, BN));
-    layer_dgrad_kernel<<<grid, GEMM_THREADS, 0, s>>>(g, ls, params, dZ, inv_deg, ST);
+    { KernelScope ks(ctx, KC_GEMM_DGRAD, s); layer_dgrad_kernel<<<grid, GEMM_THREADS, 0, s>>>(g, ls, params, dZ, inv_deg, ST); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
@@ -185,7 +185,7 @@ int32_t launch_layer_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& s
     if (slots == 0) return RTMA_OK;
     if (slots > 65535) return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "too many weight-gradient chunks (%d)", slots);
     dim3 grid((unsigned)ceil_div(2 * ls.d_in + 1, BM), (unsigned)ceil_div(ls.d_out, BN), (unsigned)slots);
-    layer_wgrad_kernel<<<grid, GEMM_THREADS, 0, s>>>(g, sp, ls, H, N, dZ, partial);
+    { KernelScope ks(ctx, KC_GEMM_WGRAD, s); layer_wgrad_kernel<<<grid, GEMM_THREADS, 0, s>>>(g, sp, ls, H, N, dZ, partial); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

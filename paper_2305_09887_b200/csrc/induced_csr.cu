@@ -143,13 +143,13 @@ extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowp
     if (col_out) {  // FILL
         if (n == 0) return RTMA_OK;
         if (rowptr_is_64)
-            induced_fill_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+            { KernelScope ks(ctx, KC_CSR_FILL, stream); induced_fill_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
                 n, M, static_cast<const int64_t*>(rowptr), col, part_id, part_offsets, perm, local_id, rowptr_out,
-                edge_offsets, col_out);
+                edge_offsets, col_out); }
         else
-            induced_fill_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+            { KernelScope ks(ctx, KC_CSR_FILL, stream); induced_fill_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
                 n, M, static_cast<const int32_t*>(rowptr), col, part_id, part_offsets, perm, local_id, rowptr_out,
-                edge_offsets, col_out);
+                edge_offsets, col_out); }
         RTMA_LAUNCH_CHECK(ctx);
         return RTMA_OK;
     }
@@ -164,21 +164,21 @@ extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowp
     int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(n));
     if (n > 0) {
         if (rowptr_is_64)
-            induced_count_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, static_cast<const int64_t*>(rowptr), col, part_id, perm, counts);
+            { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+                n, static_cast<const int64_t*>(rowptr), col, part_id, perm, counts); }
         else
-            induced_count_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, static_cast<const int32_t*>(rowptr), col, part_id, perm, counts);
+            { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+                n, static_cast<const int32_t*>(rowptr), col, part_id, perm, counts); }
         RTMA_LAUNCH_CHECK(ctx);
     }
     RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, n, slots, scratch, stream));
     const unsigned off_blocks = (unsigned)ceil_div(n + M, CSR_THREADS);
     if (rowptr_is_64)
-        induced_offsets_kernel<int64_t><<<off_blocks, CSR_THREADS, 0, stream>>>(
-            n, M, part_offsets, slots, static_cast<const int64_t*>(rowptr), rowptr_out, edge_offsets, kept_cut);
+        { KernelScope ks(ctx, KC_CSR_OFFSETS, stream); induced_offsets_kernel<int64_t><<<off_blocks, CSR_THREADS, 0, stream>>>(
+            n, M, part_offsets, slots, static_cast<const int64_t*>(rowptr), rowptr_out, edge_offsets, kept_cut); }
     else
-        induced_offsets_kernel<int32_t><<<off_blocks, CSR_THREADS, 0, stream>>>(
-            n, M, part_offsets, slots, static_cast<const int32_t*>(rowptr), rowptr_out, edge_offsets, kept_cut);
+        { KernelScope ks(ctx, KC_CSR_OFFSETS, stream); induced_offsets_kernel<int32_t><<<off_blocks, CSR_THREADS, 0, stream>>>(
+            n, M, part_offsets, slots, static_cast<const int32_t*>(rowptr), rowptr_out, edge_offsets, kept_cut); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
@@ -194,11 +194,11 @@ extern "C" int32_t rtma_gather_rows(rtma_ctx* ctx, int64_t n, int64_t row_bytes,
     const unsigned blocks = (unsigned)ceil_div(n, 8);
     const uintptr_t align = reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst) | (uintptr_t)row_bytes;
     if (align % 16 == 0)
-        gather_rows_kernel<16><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst));
+        { KernelScope ks(ctx, KC_GATHER_ROWS, stream); gather_rows_kernel<16><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst)); }
     else if (align % 4 == 0)
-        gather_rows_kernel<4><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst));
+        { KernelScope ks(ctx, KC_GATHER_ROWS, stream); gather_rows_kernel<4><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst)); }
     else
-        gather_rows_kernel<1><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst));
+        { KernelScope ks(ctx, KC_GATHER_ROWS, stream); gather_rows_kernel<1><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst)); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

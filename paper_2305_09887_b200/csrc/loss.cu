@@ -77,11 +77,11 @@ int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C
                             float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s) {
     const int64_t tiles = group_tiles(g, LOSS_TILE_ROWS);
     if (tiles > 0) {
-        softmax_xent_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, tile_loss);
+        { KernelScope ks(ctx, KC_LOSS, s); softmax_xent_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, tile_loss); }
         RTMA_LAUNCH_CHECK(ctx);
     }
     if (loss_out && g.num > 0) {
-        loss_finalize_kernel<<<g.num, 256, 0, s>>>(g, tile_loss, loss_out, loss_stride, loss_col);
+        { KernelScope ks(ctx, KC_LOSS, s); loss_finalize_kernel<<<g.num, 256, 0, s>>>(g, tile_loss, loss_out, loss_stride, loss_col); }
         RTMA_LAUNCH_CHECK(ctx);
     }
     return RTMA_OK;

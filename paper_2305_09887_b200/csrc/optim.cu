@@ -95,11 +95,11 @@ int32_t aggregate_impl(rtma_ctx* ctx, float* params, const float* grads, float l
     const int64_t packs = vec ? P / 4 : P;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(packs, 256), (int64_t)sm_count(ctx->device) * 8);
     if (vec) {
-        if (grads) aggregate_kernel<4, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, global_out);
-        else aggregate_kernel<4, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, global_out);
+        if (grads) { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<4, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, global_out); }
+        else { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<4, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, global_out); }
     } else {
-        if (grads) aggregate_kernel<1, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, global_out);
-        else aggregate_kernel<1, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, global_out);
+        if (grads) { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<1, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, global_out); }
+        else { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<1, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, global_out); }
     }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
@@ -112,7 +112,7 @@ int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp
     if (g.num == 0) return RTMA_OK;
     const int64_t count = (int64_t)(2 * ls.d_in + 1) * ls.d_out;
     dim3 grid((unsigned)ceil_div(count, 256), (unsigned)g.num);
-    reduce_sgd_kernel<<<grid, 256, 0, s>>>(g, sp, ls, partial, lr, params, grads_record);
+    { KernelScope ks(ctx, KC_REDUCE_SGD, s); reduce_sgd_kernel<<<grid, 256, 0, s>>>(g, sp, ls, partial, lr, params, grads_record); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
@@ -121,7 +121,7 @@ int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float*
                          int width, cudaStream_t s) {
     if (rows <= 0 || width <= 0) return RTMA_OK;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(rows * width, 256), 148 * 16);
-    copy_rows_kernel<<<grid, 256, 0, s>>>(src, ld_src, dst, ld_dst, rows, width);
+    { KernelScope ks(ctx, KC_COPY, s); copy_rows_kernel<<<grid, 256, 0, s>>>(src, ld_src, dst, ld_dst, rows, width); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

@@ -111,11 +111,11 @@ extern "C" int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group
     int64_t* scanned = cur.take<int64_t>(cells + 1);
     int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(cells));
     const unsigned blocks = (unsigned)ceil_div(num_chunks, PART_WARPS);
-    part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts);
+    { KernelScope ks(ctx, KC_PART_COUNT, stream); part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts); }
     RTMA_LAUNCH_CHECK(ctx);
     RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, cells, scanned, scratch, stream));
-    part_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, scanned, part_id,
-                                                             part_offsets, perm, local_id);
+    { KernelScope ks(ctx, KC_PART_SCATTER, stream); part_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, scanned, part_id,
+                                                             part_offsets, perm, local_id); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

@@ -123,7 +123,7 @@ int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_o
     if (tiles == 0) return RTMA_OK;
     const unsigned grid = (unsigned)tiles;
     const bool vec = d % 4 == 0 && aligned16(src) && aligned16(self) && aligned16(gate) && aligned16(out);
-#define RTMA_SPMM(V, N) spmm_kernel<V, N, BACKWARD><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, self, gate, out, d)
+#define RTMA_SPMM(V, N) do { KernelScope ks(ctx, BACKWARD ? KC_SPMM_BWD : KC_SPMM_FWD, s); spmm_kernel<V, N, BACKWARD><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, self, gate, out, d); } while (0)
     if (vec) {
         if (d <= 128) RTMA_SPMM(4, 1);
         else if (d <= 256) RTMA_SPMM(4, 2);
@@ -145,7 +145,7 @@ int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_o
 int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s) {
     const int64_t tiles = group_tiles(g, 256);
     if (tiles == 0) return RTMA_OK;
-    inv_degree_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, rowptr_out, inv_deg);
+    { KernelScope ks(ctx, KC_INV_DEGREE, s); inv_degree_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, rowptr_out, inv_deg); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
