@@ -150,8 +150,12 @@ def acts_layout(dims, n: int):
     return out, off
 
 
-def forward_backward(dims, rowptr, col, X, y, params, want_grads=True, want_acts=False):
-    """Returns (loss, grads or None, {name: array} or None) for one part."""
+def forward_backward(dims, rowptr, col, X, y, params, want_grads=True, want_acts=False, want_preact=False,
+                     gates=None):
+    """Returns (loss, grads or None, {name: array} or None) for one part.
+    want_preact adds the hidden pre-activations as "Z1".."Z{L-1}" to the dict.
+    gates: None, or a list of int8 arrays [n, d_{l+1}] for l = 0..L-2 (-1 natural, 0 closed,
+    1 open) overriding the ReLU branch of individual units."""
     tag, ptr, dt = _fp(params.dtype)
     X = np.ascontiguousarray(X, dtype=dt)
     params = np.ascontiguousarray(params, dtype=dt)
@@ -166,12 +170,27 @@ def forward_backward(dims, rowptr, col, X, y, params, want_grads=True, want_acts
     if want_acts:
         layout, total = acts_layout(dims, n)
         acts = np.empty(total, dtype=dt)
+    hidden = [n * dims[l + 1] for l in range(len(dims) - 2)]
+    preact = np.empty(sum(hidden), dtype=dt) if want_preact else None
+    gate_buf = None
+    if gates is not None:
+        gate_buf = np.concatenate([np.ascontiguousarray(g, dtype=np.int8).ravel() for g in gates]) if gates else \
+            np.empty(0, dtype=np.int8)
+        assert gate_buf.size == sum(hidden)
     loss = getattr(lib(), f"orc_forward_backward_{tag}")(
         ctypes.c_int32(len(dims) - 1), _p(d, c_i32p), ctypes.c_int64(n), _p(rowptr, c_i64p),
-        _p(col, c_i32p), _p(X, ptr), _p(y, c_i32p), _p(params, ptr), _p(grads, ptr), _p(acts, ptr))
+        _p(col, c_i32p), _p(X, ptr), _p(y, c_i32p), _p(params, ptr), _p(grads, ptr), _p(acts, ptr),
+        _p(preact, ptr), _p(gate_buf, ctypes.POINTER(ctypes.c_int8)))
     named = None
-    if want_acts:
-        named = {nm: acts[o:o + r * w].reshape(r, w) for nm, o, r, w in layout}
+    if want_acts or want_preact:
+        named = {}
+        if want_acts:
+            named.update({nm: acts[o:o + r * w].reshape(r, w) for nm, o, r, w in layout})
+        if want_preact:
+            off = 0
+            for l, size in enumerate(hidden):
+                named[f"Z{l + 1}"] = preact[off:off + size].reshape(n, dims[l + 1])
+                off += size
     return float(loss), grads, named
 
 

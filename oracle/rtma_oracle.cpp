@@ -91,16 +91,24 @@ void spmm_mean(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, 
 // One forward + backward pass over one part.  Returns the loss.
 // acts (optional): for l = 0..L-1: N^l [n x d_l] then H^{l+1} [n x d_{l+1}]
 // (post-ReLU for hidden layers, the logits for the last layer).
+// preact (optional): the hidden pre-activations Z^l, l = 0..L-2, [n x d_{l+1}] each.
+// gates (optional): same shape as preact; -1 = the unit's ReLU is open iff Z > 0 (the rule),
+// 0 / 1 = closed / open regardless.  ReLU is not differentiable at 0 and a pre-activation
+// within rounding error of 0 has no determined branch; the override lets a test evaluate
+// either branch for such a unit.
 template <class T>
 double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
                         const int32_t* col, const T* X, const int32_t* y, const T* params,
-                        T* grads, T* acts) {
+                        T* grads, T* acts, T* preact = nullptr, const int8_t* gates = nullptr) {
     const std::vector<LayerView> lv = layer_views(L, dims);
     const int64_t P = total_params(L, dims);
     if (grads) for (int64_t i = 0; i < P; ++i) grads[i] = (T)0;
     if (n == 0) return 0.0;
 
     std::vector<std::vector<T>> H(L + 1), N(L), Z(L);
+    std::vector<std::vector<char>> open(L);  // ReLU branch taken by every hidden unit
+    std::vector<int64_t> gate_off(L, 0);
+    for (int32_t l = 1; l < L; ++l) gate_off[l] = gate_off[l - 1] + n * lv[l - 1].d_out;
     H[0].assign(X, X + n * lv[0].d_in);
     for (int32_t l = 0; l < L; ++l) {
         const int64_t di = lv[l].d_in, dn = lv[l].d_out;
@@ -108,6 +116,7 @@ double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t
         spmm_mean<T>(n, rowptr, col, di, H[l].data(), N[l].data());
         Z[l].resize(n * dn);
         H[l + 1].resize(n * dn);
+        open[l].assign(n * dn, 1);
         const T* Ws = params + lv[l].w_self;
         const T* Wn = params + lv[l].w_neigh;
         const T* b = params + lv[l].bias;
@@ -124,10 +133,19 @@ double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t
             for (int64_t j = 0; j < dn; ++j) {
                 const T z = (T)acc[j];
                 Z[l][v * dn + j] = z;
-                H[l + 1][v * dn + j] = (l < L - 1) ? (z > (T)0 ? z : (T)0) : z;
+                if (l < L - 1) {
+                    const int8_t forced = gates ? gates[gate_off[l] + v * dn + j] : (int8_t)-1;
+                    const bool is_open = forced < 0 ? (z > (T)0) : (forced != 0);
+                    open[l][v * dn + j] = is_open ? 1 : 0;
+                    H[l + 1][v * dn + j] = is_open ? z : (T)0;
+                } else {
+                    H[l + 1][v * dn + j] = z;
+                }
             }
         }
     }
+    if (preact)
+        for (int32_t l = 0; l + 1 < L; ++l) std::memcpy(preact + gate_off[l], Z[l].data(), sizeof(T) * Z[l].size());
     if (acts) {
         T* a = acts;
         for (int32_t l = 0; l < L; ++l) {
@@ -206,7 +224,7 @@ double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t
         }
         std::vector<T> dZprev(n * di);
         for (int64_t i = 0; i < n * di; ++i)
-            dZprev[i] = Z[l - 1][i] > (T)0 ? (T)dH[i] : (T)0;
+            dZprev[i] = open[l - 1][i] ? (T)dH[i] : (T)0;
         dZ.swap(dZprev);
     }
     return loss;
@@ -314,13 +332,15 @@ void orc_spmm_mean_f64(int64_t n, const int64_t* rowptr, const int32_t* col, int
 
 double orc_forward_backward_f32(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
                                 const int32_t* col, const float* X, const int32_t* y,
-                                const float* params, float* grads, float* acts) {
-    return forward_backward<float>(L, dims, n, rowptr, col, X, y, params, grads, acts);
+                                const float* params, float* grads, float* acts, float* preact,
+                                const int8_t* gates) {
+    return forward_backward<float>(L, dims, n, rowptr, col, X, y, params, grads, acts, preact, gates);
 }
 double orc_forward_backward_f64(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
                                 const int32_t* col, const double* X, const int32_t* y,
-                                const double* params, double* grads, double* acts) {
-    return forward_backward<double>(L, dims, n, rowptr, col, X, y, params, grads, acts);
+                                const double* params, double* grads, double* acts, double* preact,
+                                const int8_t* gates) {
+    return forward_backward<double>(L, dims, n, rowptr, col, X, y, params, grads, acts, preact, gates);
 }
 
 void orc_local_steps_f32(int32_t L, const int32_t* dims, double lr, int64_t n, const int64_t* rowptr,

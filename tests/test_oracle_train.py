@@ -250,3 +250,42 @@ def test_whole_method_on_tiny(tiny_workload):
     assert res["kept"] + res["cut"] == w.graph.num_entries
     for i in range(1, w.M):
         assert np.array_equal(res["params"][i], res["params"][0])
+
+
+def test_relu_branch_override_only_moves_the_chosen_units(tiny_workload):
+    # The override exists for units whose pre-activation is within rounding error of 0, where
+    # the ReLU branch is not determined.  Natural gates (-1 everywhere) must reproduce the plain
+    # result; forcing one unit's branch must agree with finite differences of the loss in which
+    # that unit is replaced by the identity (open) or by zero (closed) -- checked here through
+    # the bias gradient of that unit, which is the sum over rows of dL/dZ.
+    rp, cp, X, y = _part(tiny_workload, 1)
+    dims = tiny_workload.dims
+    params = tiny_workload.params0.astype(np.float64)
+    loss, g, named = oracle.forward_backward(dims, rp, cp, X, y, params, want_preact=True)
+    Z1 = named["Z1"]
+    natural = [np.full(Z1.shape, -1, dtype=np.int8)]
+    loss_n, g_n, _ = oracle.forward_backward(dims, rp, cp, X, y, params, gates=natural)
+    assert loss_n == loss and np.array_equal(g_n, g)
+    same = [(Z1 > 0).astype(np.int8)]
+    loss_s, g_s, _ = oracle.forward_backward(dims, rp, cp, X, y, params, gates=same)
+    assert loss_s == loss and np.array_equal(g_s, g)
+    # close the open unit closest to the kink (its value is ~1e-5, so the forward pass barely
+    # moves): node v stops contributing to column j of the first layer's gradients, by exactly
+    # x_v (and the mean of its neighbours) times dL/dz, and nothing else moves beyond O(z).
+    pos = np.where(Z1 > 0, Z1, np.inf)
+    v, j = np.unravel_index(np.argmin(pos), pos.shape)
+    z = Z1[v, j]
+    assert 0 < z < 1e-3
+    forced = [np.full(Z1.shape, -1, dtype=np.int8)]
+    forced[0][v, j] = 0
+    _, g_f, _ = oracle.forward_backward(dims, rp, cp, X, y, params, gates=forced)
+    d0, d1 = dims[0], dims[1]
+    delta_b = (g - g_f)[2 * d0 * d1: 2 * d0 * d1 + d1]
+    dldz = delta_b[j]
+    assert abs(dldz) > 1e-7
+    assert np.abs(np.delete(delta_b, j)).max() < 50 * z * abs(dldz) + 1e-12
+    dWs = (g - g_f)[:d0 * d1].reshape(d0, d1)
+    assert np.allclose(dWs[:, j], X[v] * dldz, rtol=0, atol=50 * z * abs(dldz) * np.abs(X[v]).max() + 1e-12)
+    dWn = (g - g_f)[d0 * d1:2 * d0 * d1].reshape(d0, d1)
+    Nv = (_dense_mean_adjacency(rp, cp) @ X)[v]
+    assert np.allclose(dWn[:, j], Nv * dldz, rtol=0, atol=50 * z * abs(dldz) * max(np.abs(Nv).max(), 1e-3) + 1e-12)
