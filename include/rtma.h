@@ -61,6 +61,11 @@ int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_bytes);
 int32_t rtma_destroy(rtma_ctx* ctx);
 /* Text of the last error on this context ("" if none).  Owned by the context.            */
 const char* rtma_last_error(const rtma_ctx* ctx);
+/* Synchronises the device and reports RTMA_ERR_TIMEOUT if any kernel launched through this
+ * context since the last check gave up on one of its bounded device-side waits (the
+ * tensor-core kernels wait on mbarriers with an iteration limit instead of spinning for
+ * ever); RTMA_OK otherwise.  rtma_train_host calls it before returning.                    */
+int32_t rtma_check(rtma_ctx* ctx);
 /* Bytes of scratch currently held by the context.                                        */
 size_t rtma_workspace_bytes(const rtma_ctx* ctx);
 
@@ -161,7 +166,7 @@ int32_t rtma_sgd_aggregate(rtma_ctx* ctx, float* params, const float* grads, flo
  * summed per class (ms [RTMA_KERNEL_CLASSES], milliseconds; zeros if profiling was off) and the
  * launch counts (launches [RTMA_KERNEL_CLASSES]) since the previous read, and resets both.
  * Either output may be NULL.  The paper has no counterpart; these feed the roofline report.  */
-#define RTMA_KERNEL_CLASSES 17
+#define RTMA_KERNEL_CLASSES 18
 int32_t rtma_profile(rtma_ctx* ctx, int32_t enable);
 int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launches);
 const char* rtma_kernel_class_name(int32_t cls);

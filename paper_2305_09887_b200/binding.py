@@ -21,9 +21,9 @@ EXPORTS = (
     "rtma_create", "rtma_destroy", "rtma_last_error", "rtma_workspace_bytes", "rtma_partition",
     "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
-    "rtma_kernel_class_name",
+    "rtma_kernel_class_name", "rtma_check",
 )
-KERNEL_CLASSES = 17
+KERNEL_CLASSES = 18
 
 _lib = None
 
@@ -136,6 +136,10 @@ class Context:
     @property
     def workspace_bytes(self) -> int:
         return int(self._lib.rtma_workspace_bytes(self._h))
+
+    def check(self):
+        """Synchronises and raises if a kernel gave up on a bounded device-side wait."""
+        self._check(self._lib.rtma_check(self._h), "rtma_check")
 
     # ---- instrumentation ------------------------------------------------------------
     def profile(self, enable: bool):

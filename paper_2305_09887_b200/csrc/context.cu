@@ -1,5 +1,7 @@
 // Context life cycle, scratch arena, and the device-wide exclusive scan shared by the
 // partition and induced-subgraph stages.
+#include <cstdlib>
+
 #include "common.cuh"
 
 extern "C" int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_bytes) {
@@ -15,6 +17,13 @@ extern "C" int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_
         delete ctx;
         return RTMA_ERR_CUDA;
     }
+    if (cudaMalloc(&ctx->error_word, 256) != cudaSuccess || cudaMemset(ctx->error_word, 0, 256) != cudaSuccess) {
+        cudaFreeHost(ctx->pinned);
+        delete ctx;
+        return RTMA_ERR_CUDA;
+    }
+    const char* mode = getenv("RTMA_GEMM");
+    if (mode && strcmp(mode, "simt") == 0) ctx->use_tensor_cores = false;
     if (workspace_bytes) {
         int32_t s = rtma_reserve(ctx, workspace_bytes);
         if (s != RTMA_OK) {
@@ -32,6 +41,7 @@ extern "C" int32_t rtma_destroy(rtma_ctx* ctx) {
     cudaSetDevice(ctx->device);
     cudaDeviceSynchronize();
     if (ctx->arena) cudaFree(ctx->arena);
+    if (ctx->error_word) cudaFree(ctx->error_word);
     if (ctx->pinned) cudaFreeHost(ctx->pinned);
     for (const ProfSpan& sp : ctx->spans) {
         cudaEventDestroy(sp.start);
@@ -49,10 +59,23 @@ extern "C" size_t rtma_workspace_bytes(const rtma_ctx* ctx) { return ctx ? ctx->
 static const char* const kKernelClassNames[KC_COUNT] = {
     "partition_count", "scan", "partition_scatter", "induced_count", "induced_offsets", "induced_fill", "gather_rows",
     "inv_degree", "spmm_forward", "spmm_backward", "gemm_forward", "gemm_dgrad", "gemm_wgrad", "softmax_xent",
-    "reduce_sgd", "aggregate", "copy_rows"};
+    "reduce_sgd", "aggregate", "copy_rows", "weight_prep"};
 
 extern "C" const char* rtma_kernel_class_name(int32_t cls) {
     return cls >= 0 && cls < KC_COUNT ? kKernelClassNames[cls] : "";
+}
+
+extern "C" int32_t rtma_check(rtma_ctx* ctx) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_CUDA(ctx, cudaDeviceSynchronize());
+    int word = 0;
+    RTMA_CUDA(ctx, cudaMemcpy(&word, ctx->error_word, sizeof(int), cudaMemcpyDeviceToHost));
+    if (word != 0) {
+        cudaMemset(ctx->error_word, 0, sizeof(int));
+        return rtma_fail(ctx, RTMA_ERR_TIMEOUT, "a kernel gave up on a bounded wait (device error word %d)", word);
+    }
+    return RTMA_OK;
 }
 
 extern "C" int32_t rtma_profile(rtma_ctx* ctx, int32_t enable) {

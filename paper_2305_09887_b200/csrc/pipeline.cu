@@ -91,5 +91,5 @@ extern "C" int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_6
         RTMA_CUDA(ctx, cudaMemcpyAsync(loss_out_h, loss, 4 * (size_t)R * M * K, cudaMemcpyDeviceToHost, stream));
     if (kept_cut_h) RTMA_CUDA(ctx, cudaMemcpyAsync(kept_cut_h, kept_cut, 16, cudaMemcpyDeviceToHost, stream));
     RTMA_CUDA(ctx, cudaStreamSynchronize(stream));
-    return RTMA_OK;
+    return rtma_check(ctx);
 }

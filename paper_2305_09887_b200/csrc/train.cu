@@ -41,6 +41,7 @@ int32_t parse_model(rtma_ctx* ctx, const rtma_model_desc* md, Model* m) {
 struct ScratchPlan {
     size_t per_row_floats;   // activations, gradients, 1/deg
     size_t max_layer_params; // largest (2 d_in + 1) d_out
+    size_t prep_floats;      // repacked weights for the tensor-core path, per part
 };
 
 ScratchPlan plan_scratch(const Model& m) {
@@ -55,6 +56,7 @@ ScratchPlan plan_scratch(const Model& m) {
     }
     per_row += 2 * widest_hidden;  // [S | T]
     sp.per_row_floats = per_row;
+    for (int l = 0; l < m.L; ++l) sp.prep_floats += tc_prep_floats(tc_plan_layer(m.layer[l]), l >= 1) + 256;
     return sp;
 }
 
@@ -62,9 +64,9 @@ int splits_for(int64_t n_p) { return (int)std::min<int64_t>(64, std::max<int64_t
 
 size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
     // every matrix start is rounded up to 256 bytes; allow for that once per matrix
-    const size_t matrices = 2 * m.L + 4;
+    const size_t matrices = 6 * m.L + 4;
     return sizeof(float) * (sp.per_row_floats * (size_t)n_p + (size_t)splits_for(n_p) * sp.max_layer_params +
-                            (size_t)ceil_div(n_p, 64) + 256) + 256 * matrices;
+                            (size_t)ceil_div(n_p, 64) + 256 + sp.prep_floats) + 256 * matrices;
 }
 
 }  // namespace
@@ -191,6 +193,20 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
             Mat ST{cur.take<float>((size_t)rows * 2 * widest_hidden + 4), (int64_t)(2 * widest_hidden), 0};
             float* partial = cur.take<float>((size_t)slots * plan.max_layer_params + 4);
             float* tile_loss = cur.take<float>((size_t)group_tiles(g, 64) + 4);
+            // tensor-core path: per layer, repacked weights (forward and dgrad operands, hi and lo)
+            TcLayerPlan tcp[RTMA_MAX_LAYERS];
+            bool tc_on[RTMA_MAX_LAYERS];
+            float *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
+            for (int l = 0; l < m.L; ++l) {
+                tcp[l] = tc_plan_layer(m.layer[l]);
+                tc_on[l] = ctx->use_tensor_cores && rows > 0 && tc_layer_supported(m.layer[l], Hl[l], Nl[l], Hl[l + 1]);
+                const size_t nf = (size_t)g.num * tcp[l].Npad_f * tcp[l].Kf;
+                const size_t nd = l >= 1 ? (size_t)g.num * tcp[l].Npad_d * tcp[l].Kd : 0;
+                Bf_hi[l] = cur.take<float>(nf);
+                Bf_lo[l] = cur.take<float>(nf);
+                Bd_hi[l] = nd ? cur.take<float>(nd) : nullptr;
+                Bd_lo[l] = nd ? cur.take<float>(nd) : nullptr;
+            }
             if (cur.used > share)
                 return rtma_fail(ctx, RTMA_ERR_WORKSPACE, "internal: wave needs %zu bytes, share is %zu", cur.used, share);
 
@@ -198,9 +214,16 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
             for (int step = 0; step < K; ++step) {
                 const bool tap = taps && taps->step == step;
                 // ---- forward ----
+                for (int l = 0; l < m.L; ++l)
+                    if (tc_on[l])
+                        RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
                 for (int l = 0; l < m.L; ++l) {
                     RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], s));
-                    RTMA_TRY(launch_layer_forward(ctx, g, m.layer[l], params, Hl[l], Nl[l], Hl[l + 1], l < m.L - 1, s));
+                    if (tc_on[l])
+                        RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, n, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
+                                                   Hl[l + 1], l < m.L - 1, s));
+                    else
+                        RTMA_TRY(launch_layer_forward(ctx, g, m.layer[l], params, Hl[l], Nl[l], Hl[l + 1], l < m.L - 1, s));
                 }
                 if (tap && taps->acts) {
                     size_t rec = 0;  // floats per row in the record
@@ -221,9 +244,15 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                 // ---- backward + SGD ----
                 for (int l = m.L - 1; l >= 0; --l) {
                     const Mat dZ = Hl[l + 1];
-                    RTMA_TRY(launch_layer_wgrad(ctx, g, sp, m.layer[l], Hl[l], Nl[l], dZ, partial, s));
+                    if (tc_on[l])
+                        RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, n, Hl[l], Nl[l], dZ, partial, s));
+                    else
+                        RTMA_TRY(launch_layer_wgrad(ctx, g, sp, m.layer[l], Hl[l], Nl[l], dZ, partial, s));
                     if (l > 0) {
-                        RTMA_TRY(launch_layer_dgrad(ctx, g, m.layer[l], params, dZ, inv_deg, ST, s));
+                        if (tc_on[l])
+                            RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, s));
+                        else
+                            RTMA_TRY(launch_layer_dgrad(ctx, g, m.layer[l], params, dZ, inv_deg, ST, s));
                         const Mat S{ST.ptr, ST.ld, 0};
                         const Mat T{ST.ptr + m.dims[l], ST.ld, 0};
                         // dZ^{l-1} overwrites H^l, whose sign is the ReLU gate

@@ -93,3 +93,22 @@ int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp
                           float lr, float* params, float* grads_record, cudaStream_t s);
 int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float* dst, int64_t ld_dst, int64_t rows,
                          int width, cudaStream_t s);
+
+// ---- gemm_tc.cu (tensor-core path) ------------------------------------------------------
+struct TcLayerPlan {
+    int Kf, BN_f, Npad_f;  // forward: padded K (2 x 32-blocks over d_in), column tile, padded N
+    int Kd, BN_d, Npad_d;  // dgrad: padded K over d_out, column tile, padded N over 2 d_in
+};
+bool tc_available();
+TcLayerPlan tc_plan_layer(LayerShape ls);
+size_t tc_prep_floats(const TcLayerPlan& p, bool with_dgrad);  // per part, hi and lo together
+bool tc_layer_supported(LayerShape ls, Mat H, Mat N, Mat Hout);
+int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, const float* params,
+                              float* Bf_hi, float* Bf_lo, float* Bd_hi, float* Bd_lo, cudaStream_t s);
+int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
+                          int64_t abs_rows, const float* params, Mat H, Mat N, const float* Bf_hi, const float* Bf_lo,
+                          Mat out, bool relu, cudaStream_t s);
+int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
+                        Mat dZ, const float* Bd_hi, const float* Bd_lo, const float* inv_deg, Mat ST, cudaStream_t s);
+int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
+                        int64_t abs_rows, Mat H, Mat N, Mat dZ, float* partial, cudaStream_t s);

@@ -55,12 +55,31 @@ def _check_one_step(util, w, M=None, gemm_dtype=0, tol_scale=1.0, streams=None):
     p0 = w.params0.astype(np.float64)
     for p, (rp, cp, X, y) in enumerate(_oracle_parts(w, want)):
         n_p = rp.size - 1
-        o_loss, o_grads, o_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True)
+        o_loss, o_grads, o_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True, want_preact=True)
         layout, total = oracle.acts_layout(dims, n_p)
         base = int(want["part_offsets"][p]) * rec
+        gpu_acts = {}
         for name, off, r, wd in layout:
             a = acts[base + off: base + off + r * wd].reshape(r, wd)
+            gpu_acts[name] = a
             assert util.rel_err(a, o_acts[name]) <= TOL_ACT * tol_scale, (p, name)
+        # ReLU has no derivative at 0: a hidden unit whose pre-activation is within the rounding
+        # error of an fp32 forward pass of 0 may legitimately take either branch, and the branch
+        # decides a finite part of the gradient.  For such units only (judged on the oracle's own
+        # pre-activations) the oracle is re-evaluated on the branch the kernel took; any other
+        # unit on the wrong branch fails the activation check above.
+        gates, flipped = [], 0
+        for l in range(len(dims) - 2):
+            Z = o_acts[f"Z{l + 1}"]
+            ambiguous = np.abs(Z) < 2e-5 * tol_scale * max(1.0, np.abs(Z).max(initial=0.0))
+            differ = ambiguous & ((gpu_acts[f"H{l + 1}"] > 0) != (Z > 0))
+            flipped += int(differ.sum())
+            g8 = np.full(Z.shape, -1, dtype=np.int8)
+            g8[differ] = (gpu_acts[f"H{l + 1}"] > 0)[differ]
+            gates.append(g8)
+        assert flipped <= 8
+        if flipped:
+            o_loss, o_grads, _ = oracle.forward_backward(dims, rp, cp, X, y, p0, gates=gates)
         if n_p:
             assert abs(loss[p, 0] - o_loss) <= 1e-5 * tol_scale * max(1.0, abs(o_loss)), p
         # gradients: per parameter tensor
