@@ -18,6 +18,7 @@
 // (each warp reads its quarter of the 128 TMEM lanes).  Every mbarrier wait is bounded; a
 // wait that runs out raises the context's device error word and the block winds down.
 #include <algorithm>
+#include <cstdlib>
 
 #include "tc_common.cuh"
 #include "train.cuh"
@@ -27,7 +28,6 @@ namespace {
 constexpr int TC_THREADS = 192;
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 32;                 // floats per 128-byte swizzle row
-constexpr int A_TILE_BYTES = TC_BM * 128;  // 16 KB
 constexpr int MAX_STAGES = 4;
 constexpr int SMEM_BUDGET = 200 * 1024;
 
@@ -107,6 +107,7 @@ struct RowsArgs {
     int kb0, kb1;          // 32-wide k blocks taken from source 0 / source 1
     int a0_absolute;       // source 0 addressed by absolute (partition-order) rows
     int BN, Npad, N;       // column tile, B rows per part, valid output columns
+    int bk;                // floats per k block: 32 (128-byte swizzle rows) or 16 (64-byte rows)
     int tmem_cols, stages;
     float* out;
     int64_t ld_out;
@@ -125,14 +126,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
     if (!locate_tile(a.g, TC_BM, blockIdx.x, &k, &r0)) return;
     uint8_t* smem = align_1024(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int BN = a.BN, stages = a.stages, KB = a.kb0 + a.kb1;
+    const int BN = a.BN, stages = a.stages, KB = a.kb0 + a.kb1, bk = a.bk;
     const int n0 = blockIdx.y * BN;
-    const uint32_t b_tile_bytes = (uint32_t)BN * 128u;
-    const uint32_t stage_bytes = 2u * A_TILE_BYTES + 2u * b_tile_bytes;
+    const uint32_t row_bytes = (uint32_t)bk * 4u;
+    const uint32_t a_tile_bytes = TC_BM * row_bytes;
+    const uint32_t b_tile_bytes = (uint32_t)BN * row_bytes;
+    const uint32_t stage_bytes = 2u * a_tile_bytes + 2u * b_tile_bytes;
     auto a_hi = [&](int s) { return smem + (size_t)s * stage_bytes; };
-    auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + A_TILE_BYTES; };
-    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * A_TILE_BYTES; };
-    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * A_TILE_BYTES + b_tile_bytes; };
+    auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + a_tile_bytes; };
+    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * a_tile_bytes; };
+    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * a_tile_bytes + b_tile_bytes; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -165,27 +168,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % stages;
                 if (!wait_or_abort(&pb.empty[s], ((kb / stages) & 1) ^ 1, &pb, a.error_word)) break;
-                tc::mbar_arrive_expect_tx(&pb.full[s], A_TILE_BYTES + 2u * b_tile_bytes);
-                if (kb < a.kb0) tc::tma_load_2d(a_hi(s), &a.mapA0, &pb.full[s], kb * TC_BK, row0);
-                else tc::tma_load_2d(a_hi(s), &a.mapA1, &pb.full[s], (kb - a.kb0) * TC_BK, row1);
-                tc::tma_load_2d(b_hi(s), &a.mapBhi, &pb.full[s], kb * TC_BK, brow);
-                tc::tma_load_2d(b_lo(s), &a.mapBlo, &pb.full[s], kb * TC_BK, brow);
+                tc::mbar_arrive_expect_tx(&pb.full[s], a_tile_bytes + 2u * b_tile_bytes);
+                if (kb < a.kb0) tc::tma_load_2d(a_hi(s), &a.mapA0, &pb.full[s], kb * bk, row0);
+                else tc::tma_load_2d(a_hi(s), &a.mapA1, &pb.full[s], (kb - a.kb0) * bk, row1);
+                tc::tma_load_2d(b_hi(s), &a.mapBhi, &pb.full[s], kb * bk, brow);
+                tc::tma_load_2d(b_lo(s), &a.mapBlo, &pb.full[s], kb * bk, brow);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = tc::idesc_tf32(TC_BM, BN, false, false);
+            const uint32_t layout = bk == 32 ? tc::LAYOUT_SW128 : tc::LAYOUT_SW64;
+            const uint32_t sbo = 8u * row_bytes;  // eight rows of the swizzle pattern
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % stages;
                 if (!wait_or_abort(&pb.split[s], (kb / stages) & 1, &pb, a.error_word)) break;
                 tc::tc_fence_after_sync();
                 const uint32_t ah = tc::smem_u32(a_hi(s)), al = tc::smem_u32(a_lo(s));
                 const uint32_t bh = tc::smem_u32(b_hi(s)), bl = tc::smem_u32(b_lo(s));
-#pragma unroll
-                for (int ks = 0; ks < TC_BK / 8; ++ks) {
+                for (int ks = 0; ks < bk / 8; ++ks) {
                     const uint32_t off = ks * 32;  // 8 tf32 = 32 bytes along K inside the swizzle row
-                    const uint64_t dah = tc::smem_desc_sw128(ah + off, 16, 1024), dal = tc::smem_desc_sw128(al + off, 16, 1024);
-                    const uint64_t dbh = tc::smem_desc_sw128(bh + off, 16, 1024), dbl = tc::smem_desc_sw128(bl + off, 16, 1024);
+                    const uint64_t dah = tc::smem_desc(ah + off, 16, sbo, layout), dal = tc::smem_desc(al + off, 16, sbo, layout);
+                    const uint64_t dbh = tc::smem_desc(bh + off, 16, sbo, layout), dbl = tc::smem_desc(bl + off, 16, sbo, layout);
                     tc::mma_tf32(tmem_base, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
                     tc::mma_tf32(tmem_base, dah, dbl, idesc, 1u);
                     tc::mma_tf32(tmem_base, dah, dbh, idesc, 1u);
@@ -203,8 +207,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
             if (!ok) break;
             float4* hi = reinterpret_cast<float4*>(a_hi(s));
             float4* lo = reinterpret_cast<float4*>(a_lo(s));
-#pragma unroll
-            for (int i = 0; i < A_TILE_BYTES / 16 / 128; ++i) {
+#pragma unroll 4
+            for (int i = 0; i < (int)(a_tile_bytes / 16 / 128); ++i) {
                 const int idx = tw + 128 * i;
                 float4 h, l;
                 tc::split4(hi[idx], h, l);
@@ -272,6 +276,7 @@ struct WgradArgs {
     int jt_per_src;   // 128-wide tiles over d_in, per source
     int h_absolute;
     int n_atoms;      // 32-wide atoms over d_out (all column tiles together); a tile takes up to 8
+    int bk;           // rows (k) per pipeline stage: 16 or 32
     int tmem_cols, stages;
     float* partial;   // [slot][(2 d_in + 1) x d_out]
     int* error_word;
@@ -287,7 +292,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     const int n_p = a.g.rows[k];
     const int v0 = min(n_p, chunk * a.sp.rows_per_split[k]);
     const int v1 = min(n_p, v0 + a.sp.rows_per_split[k]);
-    const int KB = (v1 - v0 + TC_BK - 1) / TC_BK;
+    const int bk = a.bk;
+    const int KB = (v1 - v0 + bk - 1) / bk;
     const int src = blockIdx.x / a.jt_per_src;
     const int j0 = (blockIdx.x % a.jt_per_src) * TC_BM;
     const int d_in = a.d_in, d_out = a.d_out;
@@ -309,12 +315,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 
     uint8_t* smem = align_1024(smem_raw);
     const int stages = a.stages, NA = min(8, a.n_atoms - 8 * (int)blockIdx.z);
-    const uint32_t b_tile_bytes = (uint32_t)NA * 4096u;
-    const uint32_t stage_bytes = 2u * A_TILE_BYTES + 2u * b_tile_bytes;
+    const uint32_t atom_bytes = (uint32_t)bk * 128u;  // one 32-wide column of bk k-rows
+    const uint32_t a_tile_bytes = 4u * atom_bytes;
+    const uint32_t b_tile_bytes = (uint32_t)NA * atom_bytes;
+    const uint32_t stage_bytes = 2u * a_tile_bytes + 2u * b_tile_bytes;
     auto a_hi = [&](int s) { return smem + (size_t)s * stage_bytes; };
-    auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + A_TILE_BYTES; };
-    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * A_TILE_BYTES; };
-    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * A_TILE_BYTES + b_tile_bytes; };
+    auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + a_tile_bytes; };
+    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * a_tile_bytes; };
+    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * a_tile_bytes + b_tile_bytes; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -346,11 +354,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % stages;
                 if (!wait_or_abort(&pb.empty[s], ((kb / stages) & 1) ^ 1, &pb, a.error_word)) break;
-                tc::mbar_arrive_expect_tx(&pb.full[s], A_TILE_BYTES + b_tile_bytes);
+                tc::mbar_arrive_expect_tx(&pb.full[s], a_tile_bytes + b_tile_bytes);
                 for (int t = 0; t < 4; ++t)
-                    tc::tma_load_2d(a_hi(s) + t * 4096, mapA, &pb.full[s], j0 + 32 * t, arow + kb * TC_BK);
+                    tc::tma_load_2d(a_hi(s) + t * atom_bytes, mapA, &pb.full[s], j0 + 32 * t, arow + kb * bk);
                 for (int t = 0; t < NA; ++t)
-                    tc::tma_load_2d(b_hi(s) + t * 4096, &a.mapZ, &pb.full[s], cbase + 32 * t, zrow + kb * TC_BK);
+                    tc::tma_load_2d(b_hi(s) + t * atom_bytes, &a.mapZ, &pb.full[s], cbase + 32 * t, zrow + kb * bk);
             }
         }
     } else if (warp == 1) {
@@ -362,13 +370,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                 tc::tc_fence_after_sync();
                 const uint32_t ah = tc::smem_u32(a_hi(s)), al = tc::smem_u32(a_lo(s));
                 const uint32_t bh = tc::smem_u32(b_hi(s)), bl = tc::smem_u32(b_lo(s));
-#pragma unroll
-                for (int ks = 0; ks < TC_BK / 8; ++ks) {
+                for (int ks = 0; ks < bk / 8; ++ks) {
                     const uint32_t off = ks * 1024;  // 8 k-rows of 128 bytes
-                    const uint64_t dah = tc::smem_desc(ah + off, 4096, 512, tc::LAYOUT_SW128_BASE32);
-                    const uint64_t dal = tc::smem_desc(al + off, 4096, 512, tc::LAYOUT_SW128_BASE32);
-                    const uint64_t dbh = tc::smem_desc(bh + off, 4096, 512, tc::LAYOUT_SW128_BASE32);
-                    const uint64_t dbl = tc::smem_desc(bl + off, 4096, 512, tc::LAYOUT_SW128_BASE32);
+                    const uint64_t dah = tc::smem_desc(ah + off, atom_bytes, 512, tc::LAYOUT_SW128_BASE32);
+                    const uint64_t dal = tc::smem_desc(al + off, atom_bytes, 512, tc::LAYOUT_SW128_BASE32);
+                    const uint64_t dbh = tc::smem_desc(bh + off, atom_bytes, 512, tc::LAYOUT_SW128_BASE32);
+                    const uint64_t dbl = tc::smem_desc(bl + off, atom_bytes, 512, tc::LAYOUT_SW128_BASE32);
                     tc::mma_tf32(tmem_base, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
                     tc::mma_tf32(tmem_base, dah, dbl, idesc, 1u);
                     tc::mma_tf32(tmem_base, dah, dbh, idesc, 1u);
@@ -392,13 +399,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
             const int s = kb % stages;
             ok = wait_or_abort(&pb.full[s], (kb / stages) & 1, &pb, a.error_word);
             if (!ok) break;
-            const int valid = min(TC_BK, (v1 - v0) - kb * TC_BK);  // k-rows of this block inside the chunk
+            const int valid = min(bk, (v1 - v0) - kb * bk);  // k-rows of this block inside the chunk
+            const int halves = bk >> 4;                       // 16 k-rows = 128 chunks per pass over an atom
             float4* ahi = reinterpret_cast<float4*>(a_hi(s));
             float4* alo = reinterpret_cast<float4*>(a_lo(s));
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int idx = tw + 128 * i;
-                const int r = (idx >> 3) & 31;
+            for (int i = 0; i < 4 * halves; ++i) {
+                const int idx = tw + 128 * i;                 // atoms are contiguous: chunk id over the whole tile
+                const int r = (idx >> 3) % bk;
                 float4 h = make_float4(0.f, 0.f, 0.f, 0.f), l = h;
                 if (r < valid) tc::split4(ahi[idx], h, l);
                 ahi[idx] = h;
@@ -409,9 +416,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
                 if (t < NA) {
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const int idx = t * 256 + half * 128 + tw;
+                    for (int half = 0; half < halves; ++half) {
+                        const int idx = t * (bk * 8) + half * 128 + tw;
                         const int r = half * 16 + r_lo;
                         float4 x = make_float4(0.f, 0.f, 0.f, 0.f), h = x, l = x;
                         if (r < valid) {
@@ -512,6 +518,16 @@ int stages_for(size_t stage_bytes, int kblocks) {
     return s;
 }
 
+// k-block depth: 16 gives twice as many, half as large pipeline stages as 32.
+int tuned_bk() {
+    static int bk = 0;
+    if (!bk) {
+        const char* e = getenv("RTMA_TC_BK");
+        bk = (e && atoi(e) == 32) ? 32 : 16;
+    }
+    return bk;
+}
+
 bool tma_ok(const Mat& m) { return m.ptr && reinterpret_cast<uintptr_t>(m.ptr) % 16 == 0 && m.ld % 4 == 0; }
 
 int32_t set_smem_limit(rtma_ctx* ctx, const void* kernel) {
@@ -522,7 +538,7 @@ int32_t set_smem_limit(rtma_ctx* ctx, const void* kernel) {
 }  // namespace
 
 bool make_tensor_map_2d(CUtensorMap* out, const float* base, uint64_t rows, uint64_t cols, uint64_t ld,
-                        uint32_t box_cols, uint32_t box_rows, bool chunk32) {
+                        uint32_t box_cols, uint32_t box_rows, TmaSwizzle swizzle) {
     EncodeTiledFn fn = encode_tiled();
     if (!fn || rows == 0 || cols == 0) return false;
     const cuuint64_t gdim[2] = {cols, rows};
@@ -530,7 +546,9 @@ bool make_tensor_map_2d(CUtensorMap* out, const float* base, uint64_t rows, uint
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estride[2] = {1, 1};
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), gdim, gstride, box, estride,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, chunk32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle == TmaSwizzle::B128 ? CU_TENSOR_MAP_SWIZZLE_128B
+              : swizzle == TmaSwizzle::B64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -572,7 +590,7 @@ static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t 
         RTMA_TRY(set_smem_limit(ctx, reinterpret_cast<const void*>(tc_rows_kernel)));
         configured = true;
     }
-    const size_t stage_bytes = 2 * (size_t)A_TILE_BYTES + 2 * (size_t)a.BN * 128;
+    const size_t stage_bytes = 2 * (size_t)TC_BM * a.bk * 4 + 2 * (size_t)a.BN * a.bk * 4;
     a.stages = stages_for(stage_bytes, a.kb0 + a.kb1);
     a.tmem_cols = (int)tmem_columns_for(a.BN);
     a.error_word = ctx->error_word;
@@ -590,12 +608,14 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
     RowsArgs a{};
     a.g = g;
     const uint64_t hrows = H.absolute ? (uint64_t)abs_rows : (uint64_t)rows_total;
-    if (!make_tensor_map_2d(&a.mapA0, H.ptr, hrows, ls.d_in, H.ld, TC_BK, TC_BM) ||
-        !make_tensor_map_2d(&a.mapA1, N.ptr, rows_total, ls.d_in, N.ld, TC_BK, TC_BM) ||
-        !make_tensor_map_2d(&a.mapBhi, Bf_hi, (uint64_t)g.num * p.Npad_f, p.Kf, p.Kf, TC_BK, p.BN_f) ||
-        !make_tensor_map_2d(&a.mapBlo, Bf_lo, (uint64_t)g.num * p.Npad_f, p.Kf, p.Kf, TC_BK, p.BN_f))
+    a.bk = tuned_bk();
+    const TmaSwizzle sw = a.bk == 32 ? TmaSwizzle::B128 : TmaSwizzle::B64;
+    if (!make_tensor_map_2d(&a.mapA0, H.ptr, hrows, ls.d_in, H.ld, a.bk, TC_BM, sw) ||
+        !make_tensor_map_2d(&a.mapA1, N.ptr, rows_total, ls.d_in, N.ld, a.bk, TC_BM, sw) ||
+        !make_tensor_map_2d(&a.mapBhi, Bf_hi, (uint64_t)g.num * p.Npad_f, p.Kf, p.Kf, a.bk, p.BN_f, sw) ||
+        !make_tensor_map_2d(&a.mapBlo, Bf_lo, (uint64_t)g.num * p.Npad_f, p.Kf, p.Kf, a.bk, p.BN_f, sw))
         return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the forward operands");
-    a.kb0 = a.kb1 = p.Kf / (2 * TC_BK);
+    a.kb0 = a.kb1 = p.Kf / (2 * a.bk);
     a.a0_absolute = H.absolute;
     a.BN = p.BN_f;
     a.Npad = p.Npad_f;
@@ -615,12 +635,14 @@ int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const 
                         Mat dZ, const float* Bd_hi, const float* Bd_lo, const float* inv_deg, Mat ST, cudaStream_t s) {
     RowsArgs a{};
     a.g = g;
-    if (!make_tensor_map_2d(&a.mapA0, dZ.ptr, rows_total, ls.d_out, dZ.ld, TC_BK, TC_BM) ||
-        !make_tensor_map_2d(&a.mapBhi, Bd_hi, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d) ||
-        !make_tensor_map_2d(&a.mapBlo, Bd_lo, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d))
+    a.bk = tuned_bk();
+    const TmaSwizzle sw = a.bk == 32 ? TmaSwizzle::B128 : TmaSwizzle::B64;
+    if (!make_tensor_map_2d(&a.mapA0, dZ.ptr, rows_total, ls.d_out, dZ.ld, a.bk, TC_BM, sw) ||
+        !make_tensor_map_2d(&a.mapBhi, Bd_hi, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, a.bk, p.BN_d, sw) ||
+        !make_tensor_map_2d(&a.mapBlo, Bd_lo, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, a.bk, p.BN_d, sw))
         return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the dgrad operands");
     a.mapA1 = a.mapA0;
-    a.kb0 = p.Kd / TC_BK;
+    a.kb0 = (int)ceil_div(ls.d_out, a.bk);
     a.kb1 = 0;
     a.a0_absolute = 0;
     a.BN = p.BN_d;
@@ -651,9 +673,10 @@ int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, 
     a.g = g;
     a.sp = sp;
     const uint64_t hrows = H.absolute ? (uint64_t)abs_rows : (uint64_t)rows_total;
-    if (!make_tensor_map_2d(&a.mapH, H.ptr, hrows, ls.d_in, H.ld, 32, TC_BK, true) ||
-        !make_tensor_map_2d(&a.mapN, N.ptr, rows_total, ls.d_in, N.ld, 32, TC_BK, true) ||
-        !make_tensor_map_2d(&a.mapZ, dZ.ptr, rows_total, ls.d_out, dZ.ld, 32, TC_BK, true))
+    a.bk = tuned_bk();
+    if (!make_tensor_map_2d(&a.mapH, H.ptr, hrows, ls.d_in, H.ld, 32, a.bk, TmaSwizzle::B128_CHUNK32) ||
+        !make_tensor_map_2d(&a.mapN, N.ptr, rows_total, ls.d_in, N.ld, 32, a.bk, TmaSwizzle::B128_CHUNK32) ||
+        !make_tensor_map_2d(&a.mapZ, dZ.ptr, rows_total, ls.d_out, dZ.ld, 32, a.bk, TmaSwizzle::B128_CHUNK32))
         return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the wgrad operands");
     a.d_in = ls.d_in;
     a.d_out = ls.d_out;
@@ -662,7 +685,7 @@ int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, 
     a.n_atoms = (int)ceil_div(ls.d_out, 32);
     const int tile_atoms = a.n_atoms < 8 ? a.n_atoms : 8;
     a.tmem_cols = (int)tmem_columns_for(32 * tile_atoms);
-    const size_t stage_bytes = 2 * (size_t)A_TILE_BYTES + 2 * (size_t)tile_atoms * 4096;
+    const size_t stage_bytes = (2 * (size_t)4 + 2 * (size_t)tile_atoms) * a.bk * 128;
     a.stages = stages_for(stage_bytes, MAX_STAGES);
     a.partial = partial;
     a.error_word = ctx->error_word;

@@ -104,8 +104,9 @@ __device__ __forceinline__ void tmem_load_32x32(uint32_t taddr, float (&v)[32]) 
 //   MN-major tf32 operand: the only layout the tensor core accepts is the 128-byte swizzle of
 //     32-byte chunks (rows of 128 B = 32 tf32 along M/N, one row per k, chunk index xor
 //     (row mod 4)): lbo = bytes between 32-wide M/N atoms, sbo = bytes between 4-row k groups.
-constexpr uint32_t LAYOUT_SW128 = 2;         // 16-byte chunks
-constexpr uint32_t LAYOUT_SW128_BASE32 = 1;  // 32-byte chunks
+constexpr uint32_t LAYOUT_SW128 = 2;         // 128-byte rows, 16-byte chunks
+constexpr uint32_t LAYOUT_SW64 = 4;          // 64-byte rows, 16-byte chunks
+constexpr uint32_t LAYOUT_SW128_BASE32 = 1;  // 128-byte rows, 32-byte chunks
 __device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
@@ -156,7 +157,8 @@ __device__ __forceinline__ void split4(const float4 x, float4& hi, float4& lo) {
 
 // ---- host side: tensor-map encoding through the driver entry point ------------------------
 // 2-D row-major float matrix [rows x cols], `ld` floats between rows, box = box_cols x box_rows,
-// 128-byte swizzle of 16-byte chunks (or of 32-byte chunks when chunk32), out-of-range elements
-// read as zero.  Returns false if the driver refuses.
+// swizzled in shared memory as asked, out-of-range elements read as zero.  Returns false if
+// the driver refuses.
+enum class TmaSwizzle { B128, B64, B128_CHUNK32 };
 bool make_tensor_map_2d(CUtensorMap* out, const float* base, uint64_t rows, uint64_t cols, uint64_t ld,
-                        uint32_t box_cols, uint32_t box_rows, bool chunk32 = false);
+                        uint32_t box_cols, uint32_t box_rows, TmaSwizzle swizzle);
