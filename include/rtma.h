@@ -166,7 +166,7 @@ int32_t rtma_sgd_aggregate(rtma_ctx* ctx, float* params, const float* grads, flo
  * summed per class (ms [RTMA_KERNEL_CLASSES], milliseconds; zeros if profiling was off) and the
  * launch counts (launches [RTMA_KERNEL_CLASSES]) since the previous read, and resets both.
  * Either output may be NULL.  The paper has no counterpart; these feed the roofline report.  */
-#define RTMA_KERNEL_CLASSES 18
+#define RTMA_KERNEL_CLASSES 19
 int32_t rtma_profile(rtma_ctx* ctx, int32_t enable);
 int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launches);
 const char* rtma_kernel_class_name(int32_t cls);

@@ -23,7 +23,7 @@ EXPORTS = (
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check",
 )
-KERNEL_CLASSES = 18
+KERNEL_CLASSES = 19
 
 _lib = None
 

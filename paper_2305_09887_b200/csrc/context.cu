@@ -22,8 +22,6 @@ extern "C" int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_
         delete ctx;
         return RTMA_ERR_CUDA;
     }
-    const char* mode = getenv("RTMA_GEMM");
-    if (mode && strcmp(mode, "simt") == 0) ctx->use_tensor_cores = false;
     if (workspace_bytes) {
         int32_t s = rtma_reserve(ctx, workspace_bytes);
         if (s != RTMA_OK) {
@@ -59,7 +57,7 @@ extern "C" size_t rtma_workspace_bytes(const rtma_ctx* ctx) { return ctx ? ctx->
 static const char* const kKernelClassNames[KC_COUNT] = {
     "partition_count", "scan", "partition_scatter", "induced_count", "induced_offsets", "induced_fill", "gather_rows",
     "inv_degree", "spmm_forward", "spmm_backward", "gemm_forward", "gemm_dgrad", "gemm_wgrad", "softmax_xent",
-    "reduce_sgd", "aggregate", "copy_rows", "weight_prep"};
+    "reduce_sgd", "aggregate", "copy_rows", "weight_prep", "to_planes"};
 
 extern "C" const char* rtma_kernel_class_name(int32_t cls) {
     return cls >= 0 && cls < KC_COUNT ? kKernelClassNames[cls] : "";

@@ -1,16 +1,22 @@
 // Mean aggregation over the local neighbourhood (the row-normalised adjacency Abar of
-// Theorem 2 / Eq. (proof-2-pred)) and its transpose for the backward pass.
+// Theorem 2 / Eq. (proof-2-pred)) and its transpose for the backward pass, on activations
+// stored as split bf16 planes; plus the conversions between fp32 rows and planes.
 //
-// Gather-bound: one warp per row, the row's column indices are read coalesced (32 at a time)
-// and broadcast with shuffles, each neighbour's feature row is fetched with 128-bit loads.
-// Local degrees are tiny after random partitioning (about deg/M), so a block covers 32 rows
-// and each warp walks 4 of them.
+// Gather-bound and, at the tiny local degrees random partitioning leaves (about deg/M),
+// latency-bound: a warp owns 8 consecutive rows, reads their offsets with one load and their
+// column indices with one coalesced load per 32 entries (consecutive rows are consecutive
+// in the CSR), and walks the entries with four neighbours' rows in flight per lane.  Lanes
+// split the feature width in pieces of 8 values (16 bytes per plane).
+#include <algorithm>
+
 #include "train.cuh"
 
 namespace {
 
 constexpr int SPMM_THREADS = 256;
-constexpr int SPMM_TILE_ROWS = 32;
+constexpr int SPMM_ROWS_PER_WARP = 8;
+constexpr int SPMM_TILE_ROWS = SPMM_ROWS_PER_WARP * (SPMM_THREADS / 32);  // 64 = two bias tiles
+static_assert(SPMM_TILE_ROWS == 2 * BIAS_TILE_ROWS && BIAS_TILE_ROWS % SPMM_ROWS_PER_WARP == 0, "bias tiles");
 
 __global__ void __launch_bounds__(256)
 inv_degree_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, float* __restrict__ inv_deg) {
@@ -23,124 +29,241 @@ inv_degree_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict
     inv_deg[g.row_ws[k] + i] = deg > 0 ? 1.0f / (float)deg : 0.0f;
 }
 
-template <int VEC>
-struct Pack;
-template <>
-struct Pack<4> {
-    float4 v;
-    __device__ __forceinline__ void zero() { v = make_float4(0.f, 0.f, 0.f, 0.f); }
-    __device__ __forceinline__ void load(const float* p) { v = __ldg(reinterpret_cast<const float4*>(p)); }
-    __device__ __forceinline__ void load_plain(const float* p) { v = *reinterpret_cast<const float4*>(p); }
-    __device__ __forceinline__ void add(const Pack& o) { v.x += o.v.x; v.y += o.v.y; v.z += o.v.z; v.w += o.v.w; }
-    __device__ __forceinline__ void scale(float s) { v.x *= s; v.y *= s; v.z *= s; v.w *= s; }
-    __device__ __forceinline__ void gate(const Pack& m) {
-        v.x = m.v.x > 0.f ? v.x : 0.f; v.y = m.v.y > 0.f ? v.y : 0.f;
-        v.z = m.v.z > 0.f ? v.z : 0.f; v.w = m.v.w > 0.f ? v.w : 0.f;
+__global__ void __launch_bounds__(256)
+to_planes_kernel(const __grid_constant__ GroupDesc g, const float* __restrict__ X, const int d, const Planes out) {
+    int k, r0;
+    if (!locate_tile(g, 32, blockIdx.x, &k, &r0)) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int q = 0; q < 4; ++q) {
+        const int i = r0 + warp * 4 + q;
+        if (i >= g.rows[k]) return;
+        const float* x = X + (g.row_abs[k] + i) * (int64_t)d;
+        const int64_t o = (g.row_ws[k] + i) * out.ld;
+        for (int c0 = lane * 8; c0 < out.ld; c0 += 256) {
+            Pack8 p;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) p.v[e] = c0 + e < d ? __ldg(x + c0 + e) : 0.f;
+            uint4 h, l;
+            p.to_planes(h, l);
+            *reinterpret_cast<uint4*>(out.hi + o + c0) = h;
+            *reinterpret_cast<uint4*>(out.lo + o + c0) = l;
+        }
     }
-    __device__ __forceinline__ void store(float* p) const { *reinterpret_cast<float4*>(p) = v; }
-};
-template <>
-struct Pack<1> {
-    float v;
-    __device__ __forceinline__ void zero() { v = 0.f; }
-    __device__ __forceinline__ void load(const float* p) { v = __ldg(p); }
-    __device__ __forceinline__ void load_plain(const float* p) { v = *p; }
-    __device__ __forceinline__ void add(const Pack& o) { v += o.v; }
-    __device__ __forceinline__ void scale(float s) { v *= s; }
-    __device__ __forceinline__ void gate(const Pack& m) { v = m.v > 0.f ? v : 0.f; }
-    __device__ __forceinline__ void store(float* p) const { *p = v; }
-};
+}
 
-// BACKWARD == false: out = inv_deg * sum src[nbr].  BACKWARD == true: out = gate(self + sum src[nbr]).
-template <int VEC, int NCH, bool BACKWARD>
+__global__ void __launch_bounds__(256)
+from_planes_kernel(const Planes src, const int64_t first_row, const int64_t rows, const int d, float* __restrict__ dst) {
+    const int64_t total = rows * d;
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (int64_t)gridDim.x * 256) {
+        const int64_t r = i / d;
+        const int c = (int)(i - r * d);
+        const int64_t at = (first_row + r) * src.ld + c;
+        dst[i] = join_bf16(src.hi[at], src.lo[at]);
+    }
+}
+
+// BACKWARD == false: out = inv_deg * sum src[nbr]                              (src, out: planes)
+// BACKWARD == true : out <- gate_out(S + sum T[nbr]); S, T = the two halves of ST (fp32), out
+//                    holds H on entry (the ReLU gate) and dZ on exit.
+template <int NCH, bool BACKWARD>
 __global__ void __launch_bounds__(SPMM_THREADS)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
-            const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Mat src, const Mat self,
-            const Mat gate, const Mat out, const int d) {
+            const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
+            const Mat ST, const int d, float* __restrict__ bias_partial, const int64_t ld_bias) {
+    __shared__ float bias_red[BACKWARD ? SPMM_THREADS / 32 : 1][BACKWARD ? NCH * 256 : 1];
     int k, r0;
     if (!locate_tile(g, SPMM_TILE_ROWS, blockIdx.x, &k, &r0)) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n_p = g.rows[k];
     const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
     const int32_t* cols = col_out + g.edge_abs[k];
-    const int64_t src_base = src.absolute ? g.row_abs[k] : g.row_ws[k];
     const int64_t ws = g.row_ws[k];
-    constexpr int ROWS_PER_WARP = SPMM_TILE_ROWS / (SPMM_THREADS / 32);
+    const int i0 = r0 + warp * SPMM_ROWS_PER_WARP;
+    const int nrows = max(0, min(SPMM_ROWS_PER_WARP, n_p - i0));
 
-    for (int q = 0; q < ROWS_PER_WARP; ++q) {
-        const int i = r0 + warp * ROWS_PER_WARP + q;
-        if (i >= n_p) return;
-        const int64_t begin = rp[i], end = rp[i + 1];
-        Pack<VEC> acc[NCH];
+    // offsets of the warp's rows: lane j holds rp[i0 + j], j = 0..nrows
+    const int64_t my_off = (nrows > 0 && lane <= nrows) ? rp[i0 + lane] : 0;
+    const int64_t e_begin = __shfl_sync(0xffffffffu, my_off, 0);
+    const int64_t e_end = __shfl_sync(0xffffffffu, my_off, nrows);
+
+    Pack8 acc[NCH], colsum[NCH];
 #pragma unroll
-        for (int c = 0; c < NCH; ++c) acc[c].zero();
-        for (int64_t e0 = begin; e0 < end; e0 += 32) {
-            const int cnt = (int)min((int64_t)32, end - e0);
-            const int32_t mine = lane < cnt ? __ldg(cols + e0 + lane) : 0;
-#pragma unroll 4
-            for (int t = 0; t < cnt; ++t) {
-                const int32_t nb = __shfl_sync(0xffffffffu, mine, t);
-                const float* row = src.ptr + (src_base + nb) * src.ld;
+    for (int c = 0; c < NCH; ++c) {
+        acc[c].zero();
+        colsum[c].zero();
+    }
+    int cur = 0;  // row (relative to i0) the accumulators belong to
+
+    // finishes row `row`: scale or gate, store, clear
+    auto flush = [&](int row) {
+        const int64_t r = ws + i0 + row;
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int colx = (c * 32 + lane) * VEC;
-                    if (colx < d) {
-                        Pack<VEC> x;
-                        x.load(row + colx);
-                        acc[c].add(x);
+        for (int c = 0; c < NCH; ++c) {
+            const int colx = (c * 32 + lane) * 8;
+            if (colx < d) {
+                if (BACKWARD) {
+                    const float* s = ST.ptr + r * ST.ld + colx;
+                    const float4 s0 = *reinterpret_cast<const float4*>(s), s1 = *reinterpret_cast<const float4*>(s + 4);
+                    const uint4 gh = *reinterpret_cast<const uint4*>(out.hi + r * out.ld + colx);
+                    const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gh);
+                    const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float gate = (e & 1) ? __high2float(gp[e >> 1]) : __low2float(gp[e >> 1]);
+                        const float v = gate > 0.f ? acc[c].v[e] + sv[e] : 0.f;
+                        acc[c].v[e] = v;
+                        colsum[c].v[e] += v;
                     }
+                } else {
+                    const float w = inv_deg[r];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[c].v[e] *= w;
+                }
+                uint4 h, l;
+                acc[c].to_planes(h, l);
+                *reinterpret_cast<uint4*>(out.hi + r * out.ld + colx) = h;
+                *reinterpret_cast<uint4*>(out.lo + r * out.ld + colx) = l;
+            }
+            acc[c].zero();
+        }
+    };
+
+    const __nv_bfloat16* sh = BACKWARD ? nullptr : src.hi + ws * src.ld;
+    const __nv_bfloat16* sl = BACKWARD ? nullptr : src.lo + ws * src.ld;
+    const float* tsrc = BACKWARD ? ST.ptr + ws * ST.ld + (ST.ld >> 1) : nullptr;  // the T half
+
+    for (int64_t e0 = e_begin; e0 < e_end; e0 += 32) {
+        const int cnt = (int)min((int64_t)32, e_end - e0);
+        const int64_t e = e0 + lane;
+        // row of entry e = how many of the offsets rp[i0 + 1 ..] are <= e
+        int my_row = 0;
+#pragma unroll
+        for (int j = 1; j < SPMM_ROWS_PER_WARP; ++j) {
+            const int64_t oj = __shfl_sync(0xffffffffu, my_off, j);
+            my_row += (j < nrows && oj <= e) ? 1 : 0;
+        }
+        const int32_t mine = lane < cnt ? __ldg(cols + e) : 0;
+        for (int t = 0; t < cnt; t += 4) {
+            int32_t nb[4];
+            int row[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int tj = min(t + j, cnt - 1);
+                nb[j] = __shfl_sync(0xffffffffu, mine, tj);
+                row[j] = __shfl_sync(0xffffffffu, my_row, tj);
+                if (t + j >= cnt) nb[j] = -1;
+            }
+            if (BACKWARD) {
+                float4 x[4][NCH][2];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        const int colx = (c * 32 + lane) * 8;
+                        x[j][c][0] = x[j][c][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (nb[j] >= 0 && colx < d) {
+                            const float* p = tsrc + (int64_t)nb[j] * ST.ld + colx;
+                            x[j][c][0] = __ldg(reinterpret_cast<const float4*>(p));
+                            x[j][c][1] = __ldg(reinterpret_cast<const float4*>(p + 4));
+                        }
+                    }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (nb[j] < 0) continue;
+                    while (cur < row[j]) flush(cur++);
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        acc[c].v[0] += x[j][c][0].x; acc[c].v[1] += x[j][c][0].y;
+                        acc[c].v[2] += x[j][c][0].z; acc[c].v[3] += x[j][c][0].w;
+                        acc[c].v[4] += x[j][c][1].x; acc[c].v[5] += x[j][c][1].y;
+                        acc[c].v[6] += x[j][c][1].z; acc[c].v[7] += x[j][c][1].w;
+                    }
+                }
+            } else {
+                uint4 xh[4][NCH], xl[4][NCH];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        const int colx = (c * 32 + lane) * 8;
+                        xh[j][c] = xl[j][c] = make_uint4(0u, 0u, 0u, 0u);
+                        if (nb[j] >= 0 && colx < d) {
+                            xh[j][c] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)nb[j] * src.ld + colx));
+                            xl[j][c] = __ldg(reinterpret_cast<const uint4*>(sl + (int64_t)nb[j] * src.ld + colx));
+                        }
+                    }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (nb[j] < 0) continue;
+                    while (cur < row[j]) flush(cur++);
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) acc[c].add_planes(xh[j][c], xl[j][c]);
                 }
             }
         }
-        const int64_t self_row = BACKWARD ? ((self.absolute ? g.row_abs[k] : ws) + i) : 0;
-        const int64_t gate_row = BACKWARD ? ((gate.absolute ? g.row_abs[k] : ws) + i) : 0;
-        const float scale = BACKWARD ? 1.0f : inv_deg[ws + i];
+    }
+    while (cur < nrows) flush(cur++);
+
+    if (BACKWARD) {
+        // column sums of the block's two bias tiles (warps 0-3 and 4-7), added in warp order
 #pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-            const int colx = (c * 32 + lane) * VEC;
-            if (colx < d) {
-                if (BACKWARD) {
-                    Pack<VEC> s, m;
-                    s.load_plain(self.ptr + self_row * self.ld + colx);
-                    m.load_plain(gate.ptr + gate_row * gate.ld + colx);  // may alias out: ordinary load
-                    acc[c].add(s);
-                    acc[c].gate(m);
-                } else {
-                    acc[c].scale(scale);
-                }
-                acc[c].store(out.ptr + (ws + i) * out.ld + colx);
-            }
+        for (int c = 0; c < NCH; ++c)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) bias_red[warp][c * 256 + lane * 8 + e] = colsum[c].v[e];
+        __syncthreads();
+        int64_t tile0 = 0;  // bias tile number of the block's first tile
+        for (int q = 0; q < k; ++q) tile0 += (g.rows[q] + BIAS_TILE_ROWS - 1) / BIAS_TILE_ROWS;
+        tile0 += r0 / BIAS_TILE_ROWS;
+        constexpr int WARPS_PER_TILE = BIAS_TILE_ROWS / SPMM_ROWS_PER_WARP;
+        for (int idx = threadIdx.x; idx < 2 * d; idx += SPMM_THREADS) {
+            const int half = idx / d, c = idx - half * d;
+            if (r0 + half * BIAS_TILE_ROWS >= n_p) continue;
+            float s = 0.f;
+            for (int w = 0; w < WARPS_PER_TILE; ++w) s += bias_red[half * WARPS_PER_TILE + w][c];
+            bias_partial[(tile0 + half) * ld_bias + c] = s;
         }
     }
 }
 
-bool aligned16(const Mat& m) { return m.ptr == nullptr || (reinterpret_cast<uintptr_t>(m.ptr) % 16 == 0 && m.ld % 4 == 0); }
-
 template <bool BACKWARD>
 int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                      const float* inv_deg, Mat src, Mat self, Mat gate, Mat out, int d, cudaStream_t s) {
+                      const float* inv_deg, Planes src, Planes out, Mat ST, int d, float* bias_partial, int64_t ld_bias,
+                      cudaStream_t s) {
     const int64_t tiles = group_tiles(g, SPMM_TILE_ROWS);
     if (tiles == 0) return RTMA_OK;
     const unsigned grid = (unsigned)tiles;
-    const bool vec = d % 4 == 0 && aligned16(src) && aligned16(self) && aligned16(gate) && aligned16(out);
-#define RTMA_SPMM(V, N) do { KernelScope ks(ctx, BACKWARD ? KC_SPMM_BWD : KC_SPMM_FWD, s); spmm_kernel<V, N, BACKWARD><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, self, gate, out, d); } while (0)
-    if (vec) {
-        if (d <= 128) RTMA_SPMM(4, 1);
-        else if (d <= 256) RTMA_SPMM(4, 2);
-        else if (d <= 512) RTMA_SPMM(4, 4);
-        else return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "aggregation width %d > 512", d);
-    } else {
-        if (d <= 64) RTMA_SPMM(1, 2);
-        else if (d <= 128) RTMA_SPMM(1, 4);
-        else if (d <= 512) RTMA_SPMM(1, 16);
-        else return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "aggregation width %d > 512", d);
-    }
+#define RTMA_SPMM(N)                                                                                      \
+    do {                                                                                                  \
+        KernelScope ks(ctx, BACKWARD ? KC_SPMM_BWD : KC_SPMM_FWD, s);                                     \
+        spmm_kernel<N, BACKWARD><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, \
+                                                               ST, d, bias_partial, ld_bias);             \
+    } while (0)
+    if (d <= 256) RTMA_SPMM(1);
+    else if (d <= 512) RTMA_SPMM(2);
+    else if (d <= 1024) RTMA_SPMM(4);
+    else return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "aggregation width %d > 1024", d);
 #undef RTMA_SPMM
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
 
 }  // namespace
+
+int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, int d, Planes out, cudaStream_t s) {
+    const int64_t tiles = group_tiles(g, 32);
+    if (tiles == 0) return RTMA_OK;
+    { KernelScope ks(ctx, KC_TO_PLANES, s); to_planes_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, X, d, out); }
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}
+
+int32_t launch_from_planes(rtma_ctx* ctx, Planes src, int64_t first_row, int64_t rows, int d, float* dst, cudaStream_t s) {
+    if (rows <= 0 || d <= 0) return RTMA_OK;
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(rows * d, 256), 148 * 16);
+    { KernelScope ks(ctx, KC_COPY, s); from_planes_kernel<<<grid, 256, 0, s>>>(src, first_row, rows, d, dst); }
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}
 
 int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s) {
     const int64_t tiles = group_tiles(g, 256);
@@ -151,12 +274,12 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 }
 
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                         const float* inv_deg, Mat src, Mat out, int d, cudaStream_t s) {
-    const Mat none{nullptr, 0, 0};
-    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, none, none, out, d, s);
+                         const float* inv_deg, Planes src, Planes out, int d, cudaStream_t s) {
+    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, Mat{nullptr, 0}, d, nullptr, 0, s);
 }
 
 int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat src, Mat self, Mat gate, Mat out, int d, cudaStream_t s) {
-    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, nullptr, src, self, gate, out, d, s);
+                             Mat ST, Planes h, int d, float* bias_partial, int64_t ld_bias, cudaStream_t s) {
+    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, nullptr, Planes{nullptr, nullptr, 0}, h, ST, d, bias_partial,
+                               ld_bias, s);
 }

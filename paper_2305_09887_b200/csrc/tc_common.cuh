@@ -1,7 +1,6 @@
 // Blackwell (sm_100a) building blocks for the tensor-core layer products: mbarriers with
 // bounded waits, bulk-tensor (cp.async.bulk.tensor) loads, tcgen05 MMA / commit / TMEM
-// access, shared-memory matrix descriptors, and the hi/lo split that gives fp32-accurate
-// products out of TF32 MMAs.
+// access and shared-memory matrix descriptors.
 #pragma once
 
 #include <cuda.h>
@@ -98,39 +97,32 @@ __device__ __forceinline__ void tmem_load_32x32(uint32_t taddr, float (&v)[32]) 
 }
 
 // ---- MMA --------------------------------------------------------------------------------
-// Shared-memory matrix descriptor.  Addresses and offsets are stored in 16-byte units.
-//   K-major operand, 128-byte swizzle of 16-byte chunks (rows of 128 B = 32 tf32 along K):
-//     sbo = bytes between 8-row groups.
-//   MN-major tf32 operand: the only layout the tensor core accepts is the 128-byte swizzle of
-//     32-byte chunks (rows of 128 B = 32 tf32 along M/N, one row per k, chunk index xor
-//     (row mod 4)): lbo = bytes between 32-wide M/N atoms, sbo = bytes between 4-row k groups.
-constexpr uint32_t LAYOUT_SW128 = 2;         // 128-byte rows, 16-byte chunks
-constexpr uint32_t LAYOUT_SW64 = 4;          // 64-byte rows, 16-byte chunks
-constexpr uint32_t LAYOUT_SW128_BASE32 = 1;  // 128-byte rows, 32-byte chunks
-__device__ __forceinline__ uint64_t smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+// Shared-memory matrix descriptor for bf16 operands in the 128-byte swizzle of 16-byte chunks
+// (the layout a bulk-tensor load with 128-byte swizzle produces).  Fields are stored in
+// 16-byte units.
+//   K-major operand  (rows of 128 B = 64 bf16 along K): sbo = bytes between 8-row groups.
+//   MN-major operand (rows of 128 B = 64 bf16 along M/N, one row per k): lbo = bytes between
+//     64-wide M/N atoms, sbo = bytes between 8-row k groups.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
     d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
     d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
     d |= (uint64_t)1 << 46;  // descriptor version of this architecture
-    d |= (uint64_t)layout << 61;
+    d |= (uint64_t)2 << 61;  // 128-byte swizzle, 16-byte chunks
     return d;
 }
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return smem_desc(smem_addr, lbo_bytes, sbo_bytes, LAYOUT_SW128);
-}
-// Instruction descriptor: TF32 x TF32 -> FP32, dense.
-__device__ __host__ constexpr uint32_t idesc_tf32(int M, int N, bool a_mn_major, bool b_mn_major) {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+// Instruction descriptor: BF16 x BF16 -> FP32, dense.
+__device__ __host__ constexpr uint32_t idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-// D[tmem] (+)= A[smem] * B[smem]; issued by one thread.
-__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t"
         ".reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
         "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -139,26 +131,11 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// ---- fp32 = tf32 hi + tf32 lo -----------------------------------------------------------
-// hi is x rounded to TF32 (so the tensor core reads it exactly), lo = x - hi is exact in
-// fp32 and has at most 13 significant bits.  A*B ~= Ah*Bh + Al*Bh + Ah*Bl with a relative
-// error of about 2^-21 per product.
-__device__ __forceinline__ float tf32_hi(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
-}
-__device__ __forceinline__ void split4(const float4 x, float4& hi, float4& lo) {
-    hi.x = tf32_hi(x.x); hi.y = tf32_hi(x.y); hi.z = tf32_hi(x.z); hi.w = tf32_hi(x.w);
-    lo.x = x.x - hi.x; lo.y = x.y - hi.y; lo.z = x.z - hi.z; lo.w = x.w - hi.w;
-}
-
 }  // namespace tc
 
 // ---- host side: tensor-map encoding through the driver entry point ------------------------
-// 2-D row-major float matrix [rows x cols], `ld` floats between rows, box = box_cols x box_rows,
-// swizzled in shared memory as asked, out-of-range elements read as zero.  Returns false if
-// the driver refuses.
-enum class TmaSwizzle { B128, B64, B128_CHUNK32 };
-bool make_tensor_map_2d(CUtensorMap* out, const float* base, uint64_t rows, uint64_t cols, uint64_t ld,
-                        uint32_t box_cols, uint32_t box_rows, TmaSwizzle swizzle);
+// 2-D row-major bf16 matrix [rows x cols], `ld` elements between rows, box = box_cols x box_rows
+// (box_cols <= 64), 128-byte swizzle of 16-byte chunks in shared memory, out-of-range elements
+// read as zero.  Returns false if the driver refuses.
+bool make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                          uint32_t box_cols, uint32_t box_rows);

@@ -37,36 +37,51 @@ int32_t parse_model(rtma_ctx* ctx, const rtma_model_desc* md, Model* m) {
     return RTMA_OK;
 }
 
-// Scratch floats one part of n_p rows needs.
+// Scratch one part of n_p rows needs.
 struct ScratchPlan {
-    size_t per_row_floats;   // activations, gradients, 1/deg
-    size_t max_layer_params; // largest (2 d_in + 1) d_out
-    size_t prep_floats;      // repacked weights for the tensor-core path, per part
+    size_t per_row_bytes;     // planes, logits, [S|T], 1/deg
+    size_t max_layer_params;  // largest (2 d_in + 1) d_out
+    size_t max_bias_ld;       // widest d_out, padded
+    size_t prep_bytes;        // repacked weights, per part
+    size_t st_half;           // floats in one half of [S | T]
 };
+
+int64_t aligned_rows(int64_t n_p) { return ceil_div(n_p, GROUP_ROW_ALIGN) * GROUP_ROW_ALIGN; }
 
 ScratchPlan plan_scratch(const Model& m) {
     ScratchPlan sp{};
-    size_t per_row = 1;  // inv_deg
+    size_t per_row = sizeof(float);              // inv_deg
+    per_row += 4 * planes_ld(m.dims[0]);         // X as planes
     size_t widest_hidden = 0;
     for (int l = 0; l < m.L; ++l) {
-        per_row += padded_ld(m.dims[l]);      // Abar H^l
-        per_row += padded_ld(m.dims[l + 1]);  // H^{l+1} (later overwritten by dZ^l)
-        if (l >= 1) widest_hidden = std::max(widest_hidden, padded_ld(m.dims[l]));
+        per_row += 4 * planes_ld(m.dims[l]);     // Abar H^l
+        if (l < m.L - 1) per_row += 4 * planes_ld(m.dims[l + 1]);  // H^{l+1}, later overwritten by dZ^l
+        if (l >= 1) widest_hidden = std::max(widest_hidden, planes_ld(m.dims[l]));
         sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(2 * m.dims[l] + 1) * m.dims[l + 1]);
+        sp.max_bias_ld = std::max(sp.max_bias_ld, planes_ld(m.dims[l + 1]));
+        sp.prep_bytes += sizeof(__nv_bfloat16) * tc_prep_elems(tc_plan_layer(m.layer[l]), l >= 1) + 4 * 256;
     }
-    per_row += 2 * widest_hidden;  // [S | T]
-    sp.per_row_floats = per_row;
-    for (int l = 0; l < m.L; ++l) sp.prep_floats += tc_prep_floats(tc_plan_layer(m.layer[l]), l >= 1) + 256;
+    per_row += sizeof(float) * planes_ld(m.dims[m.L]);  // logits
+    per_row += 4 * planes_ld(m.dims[m.L]);              // dZ of the last layer
+    sp.st_half = widest_hidden;
+    per_row += sizeof(float) * 2 * widest_hidden;       // [S | T]
+    sp.per_row_bytes = per_row;
     return sp;
 }
 
-int splits_for(int64_t n_p) { return (int)std::min<int64_t>(64, std::max<int64_t>(1, ceil_div(n_p, 4096))); }
+// Row chunks of the weight gradient: enough of them to give the GPU a few blocks per SM,
+// each a multiple of the row alignment.
+int splits_for(int64_t n_p, int parts_in_flight) {
+    const int64_t want = std::max<int64_t>(1, 296 / std::max(1, 4 * parts_in_flight));
+    const int64_t by_rows = std::max<int64_t>(1, ceil_div(n_p, 1024));
+    return (int)std::min<int64_t>(64, std::min(want, by_rows));
+}
 
 size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
-    // every matrix start is rounded up to 256 bytes; allow for that once per matrix
-    const size_t matrices = 6 * m.L + 4;
-    return sizeof(float) * (sp.per_row_floats * (size_t)n_p + (size_t)splits_for(n_p) * sp.max_layer_params +
-                            (size_t)ceil_div(n_p, 64) + 256 + sp.prep_floats) + 256 * matrices;
+    const size_t rows = (size_t)aligned_rows(n_p);
+    const size_t matrices = 8 * m.L + 12;  // every matrix start is rounded up to 256 bytes
+    return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, BIAS_TILE_ROWS) * (1 + sp.max_bias_ld) + 256) +
+           sp.prep_bytes + 256 * matrices;
 }
 
 }  // namespace
@@ -90,6 +105,8 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
     if (K < 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "K=%d negative", K);
     if (!part_offsets || !edge_offsets || !rowptr_out || !params || !streams)
         return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_local_steps: null pointer");
+    if (!tc_available())
+        return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "the driver does not provide cuTensorMapEncodeTiled");
     if (symmetric != 1)
         return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "directed subgraphs are not implemented: pass an undirected graph with both directions stored and symmetric=1");
     const int64_t n = part_offsets[M];
@@ -157,7 +174,6 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
             SplitPlan sp{};
             size_t bytes = 0;
             int64_t rows = 0;
-            int slots = 0;
             while (at < parts.size()) {
                 const int p = parts[at];
                 const int64_t n_p = part_offsets[p + 1] - part_offsets[p];
@@ -169,61 +185,75 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                 g.row_abs[k] = part_offsets[p];
                 g.row_ws[k] = rows;
                 g.edge_abs[k] = edge_offsets[p];
-                sp.split_begin[k] = slots;
-                const int nsplit = splits_for(n_p);
-                sp.rows_per_split[k] = (int32_t)std::max<int64_t>(1, ceil_div(n_p, nsplit));
-                slots += nsplit;
-                rows += n_p;
+                rows += aligned_rows(n_p);
                 bytes += b;
                 ++at;
+            }
+            int slots = 0;
+            for (int k = 0; k < g.num; ++k) {
+                sp.split_begin[k] = slots;
+                const int nsplit = splits_for(g.rows[k], g.num);
+                sp.rows_per_split[k] = (int32_t)std::max<int64_t>(GROUP_ROW_ALIGN, aligned_rows(ceil_div(g.rows[k], nsplit)));
+                slots += (int)std::max<int64_t>(1, ceil_div(g.rows[k], sp.rows_per_split[k]));
             }
             sp.split_begin[g.num] = slots;
 
             // ---- carve the share ----
             ArenaCursor cur(ctx->arena + gi * share);
+            auto take_planes = [&](int d) {
+                Planes pl;
+                pl.ld = (int64_t)planes_ld(d);
+                pl.hi = cur.take<__nv_bfloat16>((size_t)rows * pl.ld + 8);
+                pl.lo = cur.take<__nv_bfloat16>((size_t)rows * pl.ld + 8);
+                return pl;
+            };
             float* inv_deg = cur.take<float>((size_t)rows + 1);
-            Mat Nl[RTMA_MAX_LAYERS], Hl[RTMA_MAX_LAYERS + 1];
-            Hl[0] = Mat{const_cast<float*>(Xp), (int64_t)m.dims[0], 1};
-            size_t widest_hidden = 0;
+            Planes Nl[RTMA_MAX_LAYERS], Hl[RTMA_MAX_LAYERS];
+            Hl[0] = take_planes(m.dims[0]);
             for (int l = 0; l < m.L; ++l) {
-                Nl[l] = Mat{cur.take<float>((size_t)rows * padded_ld(m.dims[l]) + 4), (int64_t)padded_ld(m.dims[l]), 0};
-                Hl[l + 1] = Mat{cur.take<float>((size_t)rows * padded_ld(m.dims[l + 1]) + 4), (int64_t)padded_ld(m.dims[l + 1]), 0};
-                if (l >= 1) widest_hidden = std::max(widest_hidden, padded_ld(m.dims[l]));
+                Nl[l] = take_planes(m.dims[l]);
+                if (l < m.L - 1) Hl[l + 1] = take_planes(m.dims[l + 1]);
             }
-            Mat ST{cur.take<float>((size_t)rows * 2 * widest_hidden + 4), (int64_t)(2 * widest_hidden), 0};
+            const int C = m.dims[m.L];
+            Mat logits{cur.take<float>((size_t)rows * planes_ld(C) + 8), (int64_t)planes_ld(C)};
+            Planes dZlast = take_planes(C);
+            Mat ST{cur.take<float>((size_t)rows * 2 * plan.st_half + 8), (int64_t)(2 * plan.st_half)};
             float* partial = cur.take<float>((size_t)slots * plan.max_layer_params + 4);
-            float* tile_loss = cur.take<float>((size_t)group_tiles(g, 64) + 4);
-            // tensor-core path: per layer, repacked weights (forward and dgrad operands, hi and lo)
+            const int64_t bias_tiles = group_tiles(g, BIAS_TILE_ROWS);
+            float* tile_loss = cur.take<float>((size_t)bias_tiles + 4);
+            float* bias_partial = cur.take<float>((size_t)bias_tiles * plan.max_bias_ld + 4);
+            const int64_t ld_bias = (int64_t)plan.max_bias_ld;
+            const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
-            bool tc_on[RTMA_MAX_LAYERS];
-            float *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
+            __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
             for (int l = 0; l < m.L; ++l) {
                 tcp[l] = tc_plan_layer(m.layer[l]);
-                tc_on[l] = ctx->use_tensor_cores && rows > 0 && tc_layer_supported(m.layer[l], Hl[l], Nl[l], Hl[l + 1]);
                 const size_t nf = (size_t)g.num * tcp[l].Npad_f * tcp[l].Kf;
                 const size_t nd = l >= 1 ? (size_t)g.num * tcp[l].Npad_d * tcp[l].Kd : 0;
-                Bf_hi[l] = cur.take<float>(nf);
-                Bf_lo[l] = cur.take<float>(nf);
-                Bd_hi[l] = nd ? cur.take<float>(nd) : nullptr;
-                Bd_lo[l] = nd ? cur.take<float>(nd) : nullptr;
+                Bf_hi[l] = cur.take<__nv_bfloat16>(nf);
+                Bf_lo[l] = cur.take<__nv_bfloat16>(nf);
+                Bd_hi[l] = nd ? cur.take<__nv_bfloat16>(nd) : nullptr;
+                Bd_lo[l] = nd ? cur.take<__nv_bfloat16>(nd) : nullptr;
             }
             if (cur.used > share)
                 return rtma_fail(ctx, RTMA_ERR_WORKSPACE, "internal: wave needs %zu bytes, share is %zu", cur.used, share);
+            if (rows == 0) continue;
 
+            RTMA_CUDA(ctx, cudaMemsetAsync(ctx->arena + gi * share, 0, zero_bytes, s));
             RTMA_TRY(launch_inv_degree(ctx, g, rowptr_out, inv_deg, s));
+            RTMA_TRY(launch_to_planes(ctx, g, Xp, m.dims[0], Hl[0], s));
+            const Planes no_planes{nullptr, nullptr, 0};
+            const Mat no_mat{nullptr, 0};
             for (int step = 0; step < K; ++step) {
                 const bool tap = taps && taps->step == step;
                 // ---- forward ----
                 for (int l = 0; l < m.L; ++l)
-                    if (tc_on[l])
-                        RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
+                    RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
                 for (int l = 0; l < m.L; ++l) {
                     RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], s));
-                    if (tc_on[l])
-                        RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, n, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
-                                                   Hl[l + 1], l < m.L - 1, s));
-                    else
-                        RTMA_TRY(launch_layer_forward(ctx, g, m.layer[l], params, Hl[l], Nl[l], Hl[l + 1], l < m.L - 1, s));
+                    const bool last = l == m.L - 1;
+                    RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
+                                               last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, s));
                 }
                 if (tap && taps->acts) {
                     size_t rec = 0;  // floats per row in the record
@@ -232,34 +262,29 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                         float* dst = taps->acts + (size_t)g.row_abs[k] * rec;
                         const int64_t n_p = g.rows[k];
                         for (int l = 0; l < m.L; ++l) {
-                            RTMA_TRY(launch_copy_rows(ctx, Nl[l].ptr + g.row_ws[k] * Nl[l].ld, Nl[l].ld, dst, m.dims[l], n_p, m.dims[l], s));
+                            RTMA_TRY(launch_from_planes(ctx, Nl[l], g.row_ws[k], n_p, m.dims[l], dst, s));
                             dst += (size_t)n_p * m.dims[l];
-                            RTMA_TRY(launch_copy_rows(ctx, Hl[l + 1].ptr + g.row_ws[k] * Hl[l + 1].ld, Hl[l + 1].ld, dst, m.dims[l + 1], n_p, m.dims[l + 1], s));
+                            if (l < m.L - 1)
+                                RTMA_TRY(launch_from_planes(ctx, Hl[l + 1], g.row_ws[k], n_p, m.dims[l + 1], dst, s));
+                            else
+                                RTMA_TRY(launch_copy_rows(ctx, logits.ptr + g.row_ws[k] * logits.ld, logits.ld, dst, C, n_p, C, s));
                             dst += (size_t)n_p * m.dims[l + 1];
                         }
                     }
                 }
-                // ---- loss; logits become dZ^{L-1} ----
-                RTMA_TRY(launch_softmax_xent(ctx, g, Hl[m.L], m.dims[m.L], yp, tile_loss, loss_out, K, step, s));
+                // ---- loss; dZ of the last layer and its tile column sums ----
+                RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, K, step, bias_partial, ld_bias, s));
                 // ---- backward + SGD ----
                 for (int l = m.L - 1; l >= 0; --l) {
-                    const Mat dZ = Hl[l + 1];
-                    if (tc_on[l])
-                        RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, n, Hl[l], Nl[l], dZ, partial, s));
-                    else
-                        RTMA_TRY(launch_layer_wgrad(ctx, g, sp, m.layer[l], Hl[l], Nl[l], dZ, partial, s));
-                    if (l > 0) {
-                        if (tc_on[l])
-                            RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, s));
-                        else
-                            RTMA_TRY(launch_layer_dgrad(ctx, g, m.layer[l], params, dZ, inv_deg, ST, s));
-                        const Mat S{ST.ptr, ST.ld, 0};
-                        const Mat T{ST.ptr + m.dims[l], ST.ld, 0};
-                        // dZ^{l-1} overwrites H^l, whose sign is the ReLU gate
-                        RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, T, S, Hl[l], Hl[l], m.dims[l], s));
-                    }
-                    RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params,
+                    const Planes dZ = l == m.L - 1 ? dZlast : Hl[l + 1];
+                    RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, s));
+                    if (l > 0) RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, s));
+                    // the bias gradient of layer l comes from the tile sums written with dZ^l; reduce
+                    // them before the next aggregation overwrites the tile sums with those of dZ^{l-1}
+                    RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, bias_partial, ld_bias, m.lr, params,
                                                tap ? taps->grads : nullptr, s));
+                    if (l > 0)  // dZ^{l-1} overwrites H^l, whose sign is the ReLU gate
+                        RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, ST, Hl[l], m.dims[l], bias_partial, ld_bias, s));
                 }
             }
         }

@@ -3,10 +3,14 @@
 #pragma once
 
 #include "common.cuh"
+#include "planes.cuh"
 
 // A group = the trainers that share one stream and one scratch region.  Its kernels cover
 // all of the group's parts in one launch; a tile never straddles two parts because every
-// part multiplies by its own parameter replica.
+// part multiplies by its own parameter replica.  Inside the scratch matrices every part
+// starts at a multiple of GROUP_ROW_ALIGN rows and the rows between parts stay zero, so a
+// tile that runs past the end of a part reads zeros.
+constexpr int GROUP_ROW_ALIGN = 64;
 struct GroupDesc {
     int32_t num;                        // parts in the group
     int32_t part[RTMA_MAX_PARTS];       // trainer index i of each part
@@ -39,76 +43,85 @@ __device__ __forceinline__ bool locate_tile(const GroupDesc& g, int tile_rows, i
 }
 #endif
 
-// A matrix of activations: rows addressed either by absolute partition-order row (the
-// caller's Xp) or by the group's scratch row.
+// An fp32 scratch matrix addressed by the group's scratch rows.
 struct Mat {
     float* ptr;
-    int64_t ld;       // floats between rows
-    int32_t absolute; // 1: row index = row_abs[k] + i, 0: row_ws[k] + i
+    int64_t ld;  // floats between rows, a multiple of 4
 };
 
 inline size_t padded_ld(int64_t d) { return (size_t)((d + 3) / 4 * 4); }
 
-// ---- spmm.cu --------------------------------------------------------------------------
-// inv_deg[row_ws + i] = 1 / local degree (0 for an isolated node).
-int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s);
-// out[r] = inv_deg[r] * sum_{u in N(r)} src[u]                      (forward, mean)
-int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                         const float* inv_deg, Mat src, Mat out, int d, cudaStream_t s);
-// out[r] = (self[r] + sum_{u in N(r)} src[u]) where gate[r] > 0 else 0   (backward through the
-// symmetric aggregation and the ReLU; out may alias gate)
-int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat src, Mat self, Mat gate, Mat out, int d, cudaStream_t s);
-
-// ---- gemm_simt.cu ---------------------------------------------------------------------
 struct LayerShape {
     int32_t d_in, d_out;
     int64_t param_offset;  // of Ws inside one replica; Ws, Wn, b are contiguous: a (2 d_in + 1) x d_out matrix
     int64_t P;             // parameters per replica
 };
-// out = act([H | N | 1] * [Ws; Wn; b])
-int32_t launch_layer_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const float* params, Mat H, Mat N,
-                             Mat out, bool relu, cudaStream_t s);
-// ST[:, 0:d_in] = dZ Ws^T ;  ST[:, d_in:2 d_in] = inv_deg * (dZ Wn^T)
-int32_t launch_layer_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const float* params, Mat dZ,
-                           const float* inv_deg, Mat ST, cudaStream_t s);
-// partial[slot][(2 d_in + 1) x d_out] = [H | N | 1]^T dZ over one chunk of rows; chunks of part k
-// occupy slots split_begin[k] .. split_begin[k+1].
+
+// Chunks of rows over which the weight gradient is accumulated before the reduction: chunks of
+// part k occupy slots split_begin[k] .. split_begin[k+1], rows_per_split[k] rows each
+// (a multiple of GROUP_ROW_ALIGN).
 struct SplitPlan {
     int32_t split_begin[RTMA_MAX_PARTS + 1];
     int32_t rows_per_split[RTMA_MAX_PARTS];
 };
-int32_t launch_layer_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, Mat H, Mat N, Mat dZ,
-                           float* partial, cudaStream_t s);
+
+// Column sums of dZ are produced by the kernels that write dZ, one row of sums per tile of
+// BIAS_TILE_ROWS rows (tiles numbered part after part), and reduced with the bias update.
+constexpr int BIAS_TILE_ROWS = 32;
+
+// ---- spmm.cu --------------------------------------------------------------------------
+// fp32 rows in partition order -> split planes in scratch rows.
+int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, int d, Planes out, cudaStream_t s);
+// Split planes -> dense fp32 [rows x d] (verification taps).
+int32_t launch_from_planes(rtma_ctx* ctx, Planes src, int64_t first_row, int64_t rows, int d, float* dst, cudaStream_t s);
+// inv_deg[row_ws + i] = 1 / local degree (0 for an isolated node).
+int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s);
+// out[r] = inv_deg[r] * sum_{u in N(r)} src[u]                      (forward, mean)
+int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                         const float* inv_deg, Planes src, Planes out, int d, cudaStream_t s);
+// h[r] <- (S[r] + sum_{u in N(r)} T[u]) where h[r] > 0 else 0, S = ST[:, 0:d], T = ST[:, d:2d]
+// (backward through the symmetric aggregation and the ReLU; h holds H on entry, dZ on exit).
+// Also writes the column sums of every BIAS_TILE_ROWS-row tile of the result to bias_partial.
+int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                             Mat ST, Planes h, int d, float* bias_partial, int64_t ld_bias, cudaStream_t s);
 
 // ---- loss.cu --------------------------------------------------------------------------
-// Softmax cross-entropy over logits (in place: logits become dL/dlogits), mean over the part.
-// loss_out[part * loss_stride + loss_col] receives the part's loss when loss_out != NULL.
-int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp,
-                            float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s);
+// Softmax cross-entropy over fp32 logits, mean over the part; dZ = (softmax - onehot) / n_p is
+// written as split planes, its tile column sums to bias_partial, and the part's loss to
+// loss_out[part * loss_stride + loss_col] when loss_out != NULL.
+int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp, Planes dZ,
+                            float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col,
+                            float* bias_partial, int64_t ld_bias, cudaStream_t s);
 
 // ---- optim.cu -------------------------------------------------------------------------
-// grad = sum of the part's partial slots; params -= lr * grad; optionally records grad.
+// Weight rows: grad = sum of the part's chunk slots; bias row: grad = sum of the part's tile
+// column sums; params -= lr * grad; optionally records grad.
 int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, const float* partial,
-                          float lr, float* params, float* grads_record, cudaStream_t s);
+                          const float* bias_partial, int64_t ld_bias, float lr, float* params, float* grads_record,
+                          cudaStream_t s);
 int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float* dst, int64_t ld_dst, int64_t rows,
                          int width, cudaStream_t s);
 
-// ---- gemm_tc.cu (tensor-core path) ------------------------------------------------------
+// ---- gemm_tc.cu (layer products on the tensor cores) --------------------------------------
 struct TcLayerPlan {
-    int Kf, BN_f, Npad_f;  // forward: padded K (2 x 32-blocks over d_in), column tile, padded N
+    int Kf, BN_f, Npad_f;  // forward: padded K (2 x 64-blocks over d_in), column tile, padded N
     int Kd, BN_d, Npad_d;  // dgrad: padded K over d_out, column tile, padded N over 2 d_in
 };
 bool tc_available();
 TcLayerPlan tc_plan_layer(LayerShape ls);
-size_t tc_prep_floats(const TcLayerPlan& p, bool with_dgrad);  // per part, hi and lo together
-bool tc_layer_supported(LayerShape ls, Mat H, Mat N, Mat Hout);
+size_t tc_prep_elems(const TcLayerPlan& p, bool with_dgrad);  // bf16 elements per part, hi and lo together
+// Repack one layer's weights of every part: transposed, zero padded, split into hi / lo.
 int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, const float* params,
-                              float* Bf_hi, float* Bf_lo, float* Bd_hi, float* Bd_lo, cudaStream_t s);
+                              __nv_bfloat16* Bf_hi, __nv_bfloat16* Bf_lo, __nv_bfloat16* Bd_hi, __nv_bfloat16* Bd_lo,
+                              cudaStream_t s);
+// out = act([H | N] [Ws; Wn] + b): split planes when out_planes.hi != NULL, else fp32 out_f32.
 int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
-                          int64_t abs_rows, const float* params, Mat H, Mat N, const float* Bf_hi, const float* Bf_lo,
-                          Mat out, bool relu, cudaStream_t s);
+                          const float* params, Planes H, Planes N, const __nv_bfloat16* Bf_hi,
+                          const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, cudaStream_t s);
+// ST[:, 0:d_in] = dZ Ws^T ;  ST[:, d_in:2 d_in] = inv_deg * (dZ Wn^T)
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
-                        Mat dZ, const float* Bd_hi, const float* Bd_lo, const float* inv_deg, Mat ST, cudaStream_t s);
+                        Planes dZ, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, const float* inv_deg, Mat ST,
+                        cudaStream_t s);
+// partial[slot][0 : 2 d_in][d_out] = [H | N]^T dZ over one chunk of rows (the bias row is not touched).
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
-                        int64_t abs_rows, Mat H, Mat N, Mat dZ, float* partial, cudaStream_t s);
+                        Planes H, Planes N, Planes dZ, float* partial, cudaStream_t s);
