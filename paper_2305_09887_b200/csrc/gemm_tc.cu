@@ -14,10 +14,10 @@
 //                 operands are MN-major straight from the planes.  Rows between parts are
 //                 zero in every plane, so chunks need no masking.
 //
-// Warp roles in a 192-thread block: warp 0 = loader (one lane), warp 1 = TMEM owner and MMA
-// issuer (one lane), warps 2-5 = epilogue (each warp reads its quarter of the 128 TMEM lanes).
-// Every mbarrier wait is bounded; a wait that runs out raises the context's device error word
-// and the block winds down.
+// Warp roles: warp 0 = loader (one lane), warp 1 = TMEM owner and MMA issuer (one lane), the
+// remaining warps = epilogue (each warp reads its quarter of the 128 TMEM lanes).  Every
+// mbarrier wait is bounded; a wait that runs out raises the context's device error word and
+// the block winds down.
 #include <algorithm>
 #include <cstdlib>
 
@@ -105,7 +105,8 @@ struct RowsArgs {
     CUtensorMap mapA0h, mapA0l, mapA1h, mapA1l, mapBh, mapBl;
     int kb0, kb1;          // 64-wide k blocks taken from source 0 / source 1
     int BN, Npad, N;       // column tile, B rows per part, valid output columns
-    int tmem_cols, stages;
+    int tmem_cols, stages; // columns of one accumulator buffer (two are allocated); pipeline depth
+    int64_t row_tiles;     // 128-row tiles over all parts
     Planes out_planes;     // hi != NULL: write split planes
     float* out;            // else: fp32
     int64_t ld_out;
@@ -118,15 +119,41 @@ struct RowsArgs {
     int* error_word;
 };
 
-__global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_constant__ RowsArgs a) {
+// Persistent: a block walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... (tile = row tile x
+// column tile, column tiles of one row tile adjacent).  Two accumulator buffers in tensor
+// memory let the epilogue of one tile overlap the main loop of the next; the shared-memory
+// ring keeps running across tiles.  Warps: 0 = loader, 1 = MMA issuer / TMEM owner,
+// 2..9 = epilogue (two warps per TMEM lane quarter, alternating 32-column chunks).
+constexpr int ROWS_THREADS = 320;
+constexpr int ROWS_EPI_THREADS = 256;
+
+struct RowsBarriers {
+    uint64_t full[MAX_STAGES];
+    uint64_t empty[MAX_STAGES];
+    uint64_t acc_full[2];   // all MMAs of the tile in this buffer finished
+    uint64_t acc_empty[2];  // the epilogue has drained this buffer
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ bool rows_wait(uint64_t* bar, uint32_t parity, RowsBarriers* pb, int* error_word) {
+    for (uint32_t i = 0; i < tc::WAIT_POLLS; ++i) {
+        if (tc::mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int*>(&pb->abort)) break;
+    }
+    *reinterpret_cast<volatile int*>(&pb->abort) = 1;
+    atomicExch(error_word, 1);
+    return false;
+}
+
+__global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_constant__ RowsArgs a) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ PipeBarriers pb;
-    int k, r0;
-    if (!locate_tile(a.g, TC_BM, blockIdx.x, &k, &r0)) return;
+    __shared__ RowsBarriers pb;
     uint8_t* smem = align_1024(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = a.BN, stages = a.stages, KB = a.kb0 + a.kb1;
-    const int n0 = blockIdx.y * BN;
+    const int n_tiles = a.Npad / BN;
+    const int64_t total_tiles = a.row_tiles * n_tiles;
     const uint32_t b_tile_bytes = (uint32_t)BN * 128u;
     const uint32_t stage_bytes = 2u * PLANE_TILE_BYTES + 2u * b_tile_bytes;
     auto a_hi = [&](int s) { return smem + (size_t)s * stage_bytes; };
@@ -139,7 +166,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
             tc::mbar_init(&pb.full[s], 1);
             tc::mbar_init(&pb.empty[s], 1);
         }
-        tc::mbar_init(&pb.accum, 1);
+        for (int b = 0; b < 2; ++b) {
+            tc::mbar_init(&pb.acc_full[b], 1);
+            tc::mbar_init(&pb.acc_empty[b], ROWS_EPI_THREADS);
+        }
         pb.abort = 0;
         tc::fence_barrier_init();
         tc::prefetch_tensormap(&a.mapA0h);
@@ -150,7 +180,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
         tc::prefetch_tensormap(&a.mapBl);
     }
     if (warp == 1) {
-        tc::tmem_alloc(&pb.tmem_base, (uint32_t)a.tmem_cols);
+        tc::tmem_alloc(&pb.tmem_base, 2u * (uint32_t)a.tmem_cols);
         tc::tmem_relinquish();
     }
     tc::tc_fence_before_sync();
@@ -160,60 +190,86 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
 
     if (warp == 0) {
         if (lane == 0) {
-            const int arow = (int)(a.g.row_ws[k] + r0);
-            const int brow = k * a.Npad + n0;
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % stages;
-                if (!wait_or_abort(&pb.empty[s], ((kb / stages) & 1) ^ 1, &pb, a.error_word)) break;
-                tc::mbar_arrive_expect_tx(&pb.full[s], 2u * PLANE_TILE_BYTES + 2u * b_tile_bytes);
-                if (kb < a.kb0) {
-                    tc::tma_load_2d(a_hi(s), &a.mapA0h, &pb.full[s], kb * TC_BK, arow);
-                    tc::tma_load_2d(a_lo(s), &a.mapA0l, &pb.full[s], kb * TC_BK, arow);
-                } else {
-                    tc::tma_load_2d(a_hi(s), &a.mapA1h, &pb.full[s], (kb - a.kb0) * TC_BK, arow);
-                    tc::tma_load_2d(a_lo(s), &a.mapA1l, &pb.full[s], (kb - a.kb0) * TC_BK, arow);
+            int64_t it = 0;  // k blocks issued so far by this block
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                int k, r0;
+                if (!locate_tile(a.g, TC_BM, tile / n_tiles, &k, &r0)) break;
+                const int n0 = (int)(tile % n_tiles) * BN;
+                const int arow = (int)(a.g.row_ws[k] + r0);
+                const int brow = k * a.Npad + n0;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = (int)(it % stages);
+                    ok = rows_wait(&pb.empty[s], (uint32_t)((it / stages) & 1) ^ 1u, &pb, a.error_word);
+                    if (!ok) break;
+                    tc::mbar_arrive_expect_tx(&pb.full[s], 2u * PLANE_TILE_BYTES + 2u * b_tile_bytes);
+                    if (kb < a.kb0) {
+                        tc::tma_load_2d(a_hi(s), &a.mapA0h, &pb.full[s], kb * TC_BK, arow);
+                        tc::tma_load_2d(a_lo(s), &a.mapA0l, &pb.full[s], kb * TC_BK, arow);
+                    } else {
+                        tc::tma_load_2d(a_hi(s), &a.mapA1h, &pb.full[s], (kb - a.kb0) * TC_BK, arow);
+                        tc::tma_load_2d(a_lo(s), &a.mapA1l, &pb.full[s], (kb - a.kb0) * TC_BK, arow);
+                    }
+                    tc::tma_load_2d(b_hi(s), &a.mapBh, &pb.full[s], kb * TC_BK, brow);
+                    tc::tma_load_2d(b_lo(s), &a.mapBl, &pb.full[s], kb * TC_BK, brow);
                 }
-                tc::tma_load_2d(b_hi(s), &a.mapBh, &pb.full[s], kb * TC_BK, brow);
-                tc::tma_load_2d(b_lo(s), &a.mapBl, &pb.full[s], kb * TC_BK, brow);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = tc::idesc_bf16(TC_BM, BN, false, false);
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % stages;
-                if (!wait_or_abort(&pb.full[s], (kb / stages) & 1, &pb, a.error_word)) break;
+            int64_t it = 0, t = 0;  // k blocks consumed, tiles started
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+                const int buf = (int)(t & 1);
+                ok = rows_wait(&pb.acc_empty[buf], (uint32_t)((t >> 1) & 1) ^ 1u, &pb, a.error_word);
+                if (!ok) break;
                 tc::tc_fence_after_sync();
-                const uint32_t ah = tc::smem_u32(a_hi(s)), al = tc::smem_u32(a_lo(s));
-                const uint32_t bh = tc::smem_u32(b_hi(s)), bl = tc::smem_u32(b_lo(s));
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.tmem_cols);
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = (int)(it % stages);
+                    ok = rows_wait(&pb.full[s], (uint32_t)((it / stages) & 1), &pb, a.error_word);
+                    if (!ok) break;
+                    tc::tc_fence_after_sync();
+                    const uint32_t ah = tc::smem_u32(a_hi(s)), al = tc::smem_u32(a_lo(s));
+                    const uint32_t bh = tc::smem_u32(b_hi(s)), bl = tc::smem_u32(b_lo(s));
 #pragma unroll
-                for (int ks = 0; ks < TC_BK / 16; ++ks) {
-                    const uint32_t off = ks * 32;  // 16 bf16 = 32 bytes along K inside the swizzle row
-                    const uint64_t dah = tc::smem_desc_sw128(ah + off, 16, 1024), dal = tc::smem_desc_sw128(al + off, 16, 1024);
-                    const uint64_t dbh = tc::smem_desc_sw128(bh + off, 16, 1024), dbl = tc::smem_desc_sw128(bl + off, 16, 1024);
-                    tc::mma_bf16(tmem_base, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
-                    tc::mma_bf16(tmem_base, dah, dbl, idesc, 1u);
-                    tc::mma_bf16(tmem_base, dah, dbh, idesc, 1u);
+                    for (int ks = 0; ks < TC_BK / 16; ++ks) {
+                        const uint32_t off = ks * 32;  // 16 bf16 = 32 bytes along K inside the swizzle row
+                        const uint64_t dah = tc::smem_desc_sw128(ah + off, 16, 1024), dal = tc::smem_desc_sw128(al + off, 16, 1024);
+                        const uint64_t dbh = tc::smem_desc_sw128(bh + off, 16, 1024), dbl = tc::smem_desc_sw128(bl + off, 16, 1024);
+                        tc::mma_bf16(d_tmem, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
+                        tc::mma_bf16(d_tmem, dah, dbl, idesc, 1u);
+                        tc::mma_bf16(d_tmem, dah, dbh, idesc, 1u);
+                    }
+                    tc::mma_commit(&pb.empty[s]);
                 }
-                tc::mma_commit(&pb.empty[s]);
+                if (ok) tc::mma_commit(&pb.acc_full[buf]);
             }
-            tc::mma_commit(&pb.accum);
         }
     } else {
-        bool ok = wait_or_abort(&pb.accum, 0, &pb, a.error_word);
-        asm volatile("bar.sync 1, 128;" ::: "memory");  // the four epilogue warps agree on the outcome
-        ok = *reinterpret_cast<volatile int*>(&pb.abort) == 0;
-        tc::tc_fence_after_sync();
-        if (ok) {
-            const int q = warp & 3;  // the TMEM lane quarter this warp may read
+        const int ew = warp - 2;          // 0..7
+        const int q = warp & 3;           // the TMEM lane quarter this warp may read
+        const int col_phase = ew >> 2;    // which of the two warps of the quarter: even or odd chunks
+        int64_t t = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
+            int k, r0;
+            if (!locate_tile(a.g, TC_BM, tile / n_tiles, &k, &r0)) break;
+            const int n0 = (int)(tile % n_tiles) * BN;
+            const int buf = (int)(t & 1);
+            ok = rows_wait(&pb.acc_full[buf], (uint32_t)((t >> 1) & 1), &pb, a.error_word);
+            if (!ok) break;
+            tc::tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.tmem_cols);
             const int i = r0 + q * 32 + lane;
             const bool live = i < a.g.rows[k];
             const int64_t orow = a.g.row_ws[k] + i;
             const float* bias = a.bias_offset >= 0 ? a.params + (int64_t)a.g.part[k] * a.P + a.bias_offset : nullptr;
             const float w = (a.scale_from >= 0 && live) ? a.inv_deg[orow] : 1.f;
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = col_phase * 32; c0 < BN; c0 += 64) {
                 float v[32];
-                tc::tmem_load_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+                tc::tmem_load_32x32(d_tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
                 if (!live) continue;
 #pragma unroll
                 for (int j = 0; j < 32; j += 8) {
@@ -222,15 +278,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
                     Pack8 x;
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        float t = v[j + e];
+                        float tv = v[j + e];
                         if (n + e < a.N) {
-                            if (bias) t += __ldg(bias + n + e);
-                            if (a.scale_from >= 0 && n + e >= a.scale_from) t *= w;
-                            if (a.relu) t = fmaxf(t, 0.f);
+                            if (bias) tv += __ldg(bias + n + e);
+                            if (a.scale_from >= 0 && n + e >= a.scale_from) tv *= w;
+                            if (a.relu) tv = fmaxf(tv, 0.f);
                         } else {
-                            t = 0.f;
+                            tv = 0.f;
                         }
-                        x.v[e] = t;
+                        x.v[e] = tv;
                     }
                     if (a.out_planes.hi) {
                         uint4 h, l;  // the padded row length is a multiple of 8: whole packs fit
@@ -251,11 +307,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_rows_kernel(const __grid_con
                     }
                 }
             }
+            tc::tc_fence_before_sync();
+            tc::mbar_arrive(&pb.acc_empty[buf]);  // all 256 epilogue threads arrive: the buffer may be overwritten
         }
     }
     tc::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) tc::tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+    if (warp == 1) tc::tmem_dealloc(tmem_base, 2u * (uint32_t)a.tmem_cols);
 }
 
 // ------------------------------------------------------------------------------------
@@ -447,6 +505,16 @@ int32_t set_smem_limit(rtma_ctx* ctx, const void* kernel) {
     return RTMA_OK;
 }
 
+int sm_count_of(int device) {
+    static int cached = 0;
+    if (!cached) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || v <= 0) v = 148;
+        cached = v;
+    }
+    return cached;
+}
+
 bool plane_maps(CUtensorMap* hi, CUtensorMap* lo, Planes p, uint64_t rows, uint64_t cols, uint32_t box_cols,
                 uint32_t box_rows) {
     return make_tensor_map_bf16(hi, p.hi, rows, cols, p.ld, box_cols, box_rows) &&
@@ -509,10 +577,11 @@ static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t 
     a.stages = stages_for(stage_bytes, a.kb0 + a.kb1);
     a.tmem_cols = (int)tmem_columns_for(a.BN);
     a.error_word = ctx->error_word;
-    const int64_t tiles = group_tiles(a.g, TC_BM);
-    if (tiles == 0) return RTMA_OK;
-    dim3 grid((unsigned)tiles, (unsigned)(a.Npad / a.BN));
-    { KernelScope ks(ctx, kclass, s); tc_rows_kernel<<<grid, TC_THREADS, a.stages * stage_bytes + 1024, s>>>(a); }
+    a.row_tiles = group_tiles(a.g, TC_BM);
+    if (a.row_tiles == 0) return RTMA_OK;
+    const int64_t total_tiles = a.row_tiles * (a.Npad / a.BN);
+    const unsigned grid = (unsigned)std::min<int64_t>(total_tiles, sm_count_of(ctx->device));
+    { KernelScope ks(ctx, kclass, s); tc_rows_kernel<<<grid, ROWS_THREADS, a.stages * stage_bytes + 1024, s>>>(a); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
