@@ -66,7 +66,7 @@ from_planes_kernel(const Planes src, const int64_t first_row, const int64_t rows
 // BACKWARD == true : out <- gate_out(S + sum T[nbr]); S, T = the two halves of ST (fp32), out
 //                    holds H on entry (the ReLU gate) and dZ on exit.
 template <int NCH, bool BACKWARD>
-__global__ void __launch_bounds__(SPMM_THREADS)
+__global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 3 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
             const Mat ST, const int d, float* __restrict__ bias_partial, const int64_t ld_bias) {
