@@ -81,6 +81,32 @@ int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group_id, uint64
                        int32_t M, int32_t* part_id, int64_t* part_offsets, int32_t* perm,
                        int32_t* local_id, void* stream);
 
+/* The same partition for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of rtma_partition.)  Some hosts of this library
+ * cannot call cudaMalloc at the point where they partition: code running while a CUDA graph is
+ * being captured or inside a memory pool whose size is fixed in advance, services that pin their
+ * whole device budget at start-up, and callers holding locks under which an allocation (which may
+ * synchronise the device) is forbidden.  rtma_partition takes its scratch from the context's
+ * arena, which it may have to grow; this entry point needs no context and takes its scratch from
+ * a fixed array compiled into the library (about 3 MB, held on every GPU that loads the library
+ * until the process exits).  It calls no cudaMalloc / cudaFree and no allocating routine.
+ *   Limit: ceil(n / 1024) * M <= RTMA_PARTITION_STATIC_MAX_CELLS (e.g. 4,194,304 nodes at M = 64,
+ *   33,554,432 nodes at M = 8); beyond it the call returns RTMA_ERR_WORKSPACE and does nothing.
+ *   Arguments and results are exactly those of rtma_partition (device pointers, same outputs bit
+ *   for bit); `device` is the CUDA device the pointers live on and is made current.
+ *   The first call on a device looks up the scratch array's device address (cudaGetSymbolAddress);
+ *   make that first call before any stream capture begins.
+ *   All calls share the one array, which keeps the previous call's contents (nothing in it needs
+ *   clearing: every cell is rewritten before it is read).  Two calls whose kernels overlap on the
+ *   GPU -- different streams without ordering, or different host threads -- race on it: order them.
+ *   Errors: RTMA_ERR_* as elsewhere; rtma_partition_static_error() returns the text of the last
+ *   failure of this entry point (one buffer for the process, not thread safe).               */
+#define RTMA_PARTITION_STATIC_MAX_CELLS 262144
+int32_t rtma_partition_static(int32_t device, int64_t n, const int32_t* group_id, uint64_t seed,
+                              int32_t M, int32_t* part_id, int64_t* part_offsets, int32_t* perm,
+                              int32_t* local_id, void* stream);
+const char* rtma_partition_static_error(void);
+
 /* ---- node-induced subgraphs G^(i) (Preliminaries) --------------------------------------
  * Keeps CSR entry (u,v) iff part_id[u] == part_id[v] and emits, for every part, a CSR over
  * local ids with rows in local order and the input's column order preserved.

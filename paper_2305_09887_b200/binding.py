@@ -21,7 +21,7 @@ EXPORTS = (
     "rtma_create", "rtma_destroy", "rtma_last_error", "rtma_workspace_bytes", "rtma_partition",
     "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
-    "rtma_kernel_class_name", "rtma_check",
+    "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
 )
 KERNEL_CLASSES = 19
 
@@ -55,6 +55,7 @@ def load_library():
         lib.rtma_workspace_bytes.argtypes = [ctypes.c_void_p]
         lib.rtma_param_count.restype = ctypes.c_int64
         lib.rtma_kernel_class_name.restype = ctypes.c_char_p
+        lib.rtma_partition_static_error.restype = ctypes.c_char_p
         _lib = lib
     return _lib
 
@@ -98,6 +99,31 @@ def _need(t, dtype, name, device=None):
     if device is not None and t.device != device:
         raise ValueError(f"{name} must live on {device}, got {t.device}")
     return t
+
+
+PARTITION_STATIC_MAX_CELLS = 262144
+
+
+def partition_static(n: int, group_id, seed: int, M: int, device: int = 0, stream=None):
+    """rtma_partition for callers that must not allocate while partitioning: no context, scratch
+    in a fixed array inside the library, limited to ceil(n/1024)*M <= PARTITION_STATIC_MAX_CELLS.
+    The four output tensors are still the caller's (allocated here with torch for convenience;
+    a caller that cannot allocate passes its own buffers through the C ABI).  Same results as
+    Context.partition, bit for bit.  Calls share the fixed scratch: keep them stream-ordered."""
+    lib = load_library()
+    dev = torch.device("cuda", device)
+    if group_id is not None:
+        _need(group_id, torch.int32, "group_id", dev)
+    part_id = torch.empty(n, dtype=torch.int32, device=dev)
+    part_offsets = torch.empty(M + 1, dtype=torch.int64, device=dev)
+    perm = torch.empty(n, dtype=torch.int32, device=dev)
+    local_id = torch.empty(n, dtype=torch.int32, device=dev)
+    st = lib.rtma_partition_static(ctypes.c_int32(device), ctypes.c_int64(n), _ptr(group_id), ctypes.c_uint64(seed),
+                                   ctypes.c_int32(M), _ptr(part_id), _ptr(part_offsets), _ptr(perm), _ptr(local_id),
+                                   ctypes.c_void_p(_stream_handle(stream)))
+    if st != 0:
+        raise RtmaError(f"rtma_partition_static failed ({st}): {lib.rtma_partition_static_error().decode()}")
+    return part_id, part_offsets, perm, local_id
 
 
 class Context:

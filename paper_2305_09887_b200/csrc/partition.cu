@@ -119,3 +119,111 @@ extern "C" int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
+
+// ------------------------------------------------------------------------------------
+// The same partition without any allocation: scratch lives in a fixed device array.
+// ------------------------------------------------------------------------------------
+namespace {
+
+// counts [cells] int32 followed by scanned [cells + 1] int64, cells = ceil(n / 1024) * M
+constexpr int64_t STATIC_MAX_CELLS = RTMA_PARTITION_STATIC_MAX_CELLS;
+constexpr size_t STATIC_COUNTS_BYTES = (sizeof(int32_t) * STATIC_MAX_CELLS + 255) / 256 * 256;
+constexpr size_t STATIC_SCRATCH_BYTES = STATIC_COUNTS_BYTES + sizeof(int64_t) * (STATIC_MAX_CELLS + 1);
+static __device__ __align__(256) unsigned char g_partition_scratch[STATIC_SCRATCH_BYTES];
+
+// In host code the array's name is only a handle for the runtime, not a device address: the
+// address is looked up once per device (with that device current) and kept here.
+constexpr int STATIC_MAX_DEVICES = 64;
+unsigned char* g_partition_scratch_ptr[STATIC_MAX_DEVICES] = {nullptr};
+char g_static_error[256] = {0};
+
+int32_t static_fail(int32_t code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_static_error, sizeof(g_static_error), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+// Exclusive scan of `cells` counts (cells + 1 outputs) by one block of 1024 threads.
+__global__ void __launch_bounds__(1024)
+part_scan_one_block_kernel(const int32_t* __restrict__ counts, int64_t cells, int64_t* __restrict__ scanned) {
+    __shared__ int64_t warp_sums[32];
+    __shared__ int64_t carry;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int64_t start = 0; start <= cells; start += 1024) {
+        const int64_t i = start + threadIdx.x;
+        const int64_t v = i < cells ? counts[i] : 0;
+        int64_t incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int64_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            const int64_t w = warp_sums[lane];
+            int64_t wi = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int64_t t = __shfl_up_sync(0xffffffffu, wi, o);
+                if (lane >= o) wi += t;
+            }
+            warp_sums[lane] = wi - w;
+        }
+        __syncthreads();
+        const int64_t base = carry;
+        if (i <= cells) scanned[i] = base + warp_sums[warp] + incl - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = base + warp_sums[31] + incl;
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+extern "C" const char* rtma_partition_static_error(void) { return g_static_error; }
+
+extern "C" int32_t rtma_partition_static(int32_t device, int64_t n, const int32_t* group_id, uint64_t seed, int32_t M,
+                                         int32_t* part_id, int64_t* part_offsets, int32_t* perm, int32_t* local_id,
+                                         void* stream_) {
+    if (device < 0 || device >= STATIC_MAX_DEVICES) return static_fail(RTMA_ERR_INVALID_ARG, "device %d outside [0,%d)", device, STATIC_MAX_DEVICES);
+    if (M < 1 || M > RTMA_MAX_PARTS) return static_fail(RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
+    if (n < 0 || n >= (int64_t(1) << 31)) return static_fail(RTMA_ERR_INVALID_ARG, "n=%lld outside [0,2^31)", (long long)n);
+    if (!part_offsets || (n > 0 && (!part_id || !perm || !local_id)))
+        return static_fail(RTMA_ERR_INVALID_ARG, "rtma_partition_static: null output pointer");
+    const int64_t num_chunks = ceil_div(n, PART_CHUNK);
+    const int64_t cells = num_chunks * M;
+    if (cells > STATIC_MAX_CELLS)
+        return static_fail(RTMA_ERR_WORKSPACE,
+                           "rtma_partition_static: ceil(n/1024)*M = %lld exceeds the fixed scratch of %lld cells (n=%lld, M=%d); "
+                           "use rtma_partition",
+                           (long long)cells, (long long)STATIC_MAX_CELLS, (long long)n, M);
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) return static_fail(RTMA_ERR_CUDA, "cudaSetDevice(%d): %s", device, cudaGetErrorString(e));
+    if (!g_partition_scratch_ptr[device]) {  // first call on this device: resolve the array's device address
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_partition_scratch);
+        if (e != cudaSuccess || !p) return static_fail(RTMA_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        g_partition_scratch_ptr[device] = static_cast<unsigned char*>(p);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (n == 0) {
+        e = cudaMemsetAsync(part_offsets, 0, sizeof(int64_t) * (M + 1), stream);
+        return e == cudaSuccess ? RTMA_OK : static_fail(RTMA_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    }
+    // Nothing in the scratch has to start from zero: the count pass writes every cell it owns
+    // and the scan writes every prefix before the scatter pass reads them.
+    int32_t* counts = reinterpret_cast<int32_t*>(g_partition_scratch_ptr[device]);
+    int64_t* scanned = reinterpret_cast<int64_t*>(g_partition_scratch_ptr[device] + STATIC_COUNTS_BYTES);
+    const unsigned blocks = (unsigned)ceil_div(num_chunks, PART_WARPS);
+    part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts);
+    part_scan_one_block_kernel<<<1, 1024, 0, stream>>>(counts, cells, scanned);
+    part_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, scanned, part_id,
+                                                             part_offsets, perm, local_id);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? RTMA_OK : static_fail(RTMA_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+}
