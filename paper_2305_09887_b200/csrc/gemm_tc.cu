@@ -12,7 +12,9 @@
 //                 are K-major straight from the planes, B from the repacked weights.
 //   wgrad kernel  D[128 x d_out] = A^T * dZ over a chunk of rows, A = H or Abar H.  Both
 //                 operands are MN-major straight from the planes.  Rows between parts are
-//                 zero in every plane, so chunks need no masking.
+//                 zero in every plane, so chunks need no masking.  The bias gradient (column
+//                 sums of dZ) is added up from the staged dZ tiles by the otherwise idle
+//                 epilogue warps.
 //
 // Warp roles: warp 0 = loader (one lane), warp 1 = TMEM owner and MMA issuer (one lane), the
 // remaining warps = epilogue (each warp reads its quarter of the 128 TMEM lanes).  Every
@@ -350,11 +352,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     const int ccount = min(256, d_out - cbase);               // valid columns in it
     float* P = a.partial + (int64_t)slot * (2 * d_in + 1) * d_out;
 
+    const bool bias_tile = blockIdx.x == 0;  // these blocks also produce the bias gradient of their columns
+
     if (KB == 0) {  // empty chunk: the gradient contribution is zero
         for (int idx = threadIdx.x; idx < TC_BM * ccount; idx += TC_THREADS) {
             const int j = j0 + idx / ccount;
             if (j < d_in) P[(int64_t)(src * d_in + j) * d_out + cbase + idx % ccount] = 0.f;
         }
+        if (bias_tile)
+            for (int c = threadIdx.x; c < ccount; c += TC_THREADS) P[(int64_t)2 * d_in * d_out + cbase + c] = 0.f;
         return;
     }
 
@@ -372,7 +378,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             tc::mbar_init(&pb.full[s], 1);
-            tc::mbar_init(&pb.empty[s], 1);
+            tc::mbar_init(&pb.empty[s], bias_tile ? 1 + 128 : 1);  // MMA commit (+ the column-sum readers)
         }
         tc::mbar_init(&pb.accum, 1);
         pb.abort = 0;
@@ -433,10 +439,60 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
             tc::mma_commit(&pb.accum);
         }
     } else {
-        bool ok = wait_or_abort(&pb.accum, 0, &pb, a.error_word);
+        const int tw = threadIdx.x - 64;  // 0..127
+        // Bias gradient = column sums of dZ.  While the MMAs run, the epilogue warps of the bias
+        // blocks add up the dZ tiles sitting in shared memory.  In an 8 KB atom a 16-byte chunk id
+        // is (k-row r = id / 8, stored chunk s = id % 8) and holds logical chunk s ^ (r % 8).
+        // Thread tw takes ids tw, tw + 128, tw + 256, tw + 384: rows tw / 8 + 16 i, which agree
+        // mod 8, so it always sums the same 8 columns of every atom.
+        float colsum[4][8];
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) colsum[t][e] = 0.f;
+        bool ok = true;
+        if (bias_tile) {
+            for (int kb = 0; kb < KB && ok; ++kb) {
+                const int s = kb % stages;
+                ok = wait_or_abort(&pb.full[s], (kb / stages) & 1, &pb, a.error_word);
+                if (!ok) break;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    if (t < NA) {
+                        const uint4* bh = reinterpret_cast<const uint4*>(b_hi(s) + t * ATOM_BYTES);
+                        const uint4* bl = reinterpret_cast<const uint4*>(b_lo(s) + t * ATOM_BYTES);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            Pack8 p;
+                            p.zero();
+                            p.add_planes(bh[tw + 128 * i], bl[tw + 128 * i]);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) colsum[t][e] += p.v[e];
+                        }
+                    }
+                }
+                tc::mbar_arrive(&pb.empty[s]);
+            }
+        }
+        if (ok) ok = wait_or_abort(&pb.accum, 0, &pb, a.error_word);
         asm volatile("bar.sync 1, 128;" ::: "memory");  // the four epilogue warps agree on the outcome
         ok = *reinterpret_cast<volatile int*>(&pb.abort) == 0;
         tc::tc_fence_after_sync();
+        if (ok && bias_tile) {
+            // every load has landed and every MMA has finished: stage 0 is free to hold the sums
+            float* red = reinterpret_cast<float*>(a_hi(0));  // [128 threads][32]
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) red[tw * 32 + t * 8 + e] = colsum[t][e];
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int c = tw; c < ccount; c += 128) {
+                const int t = c >> 6, lc = (c & 63) >> 3, e = c & 7;
+                float sum = 0.f;
+                for (int h = 0; h < 16; ++h) sum += red[(h * 8 + (lc ^ (h & 7))) * 32 + t * 8 + e];  // fixed order
+                P[(int64_t)2 * d_in * d_out + cbase + c] = sum;
+            }
+        }
         if (ok) {
             const int q = warp & 3;
             const int j = j0 + q * 32 + lane;

@@ -1,22 +1,23 @@
 // Softmax cross-entropy over a part's fp32 logits, averaged over the part's nodes; its
 // gradient (softmax - onehot) / n_p is written as split bf16 planes (it feeds the tensor-core
-// products of the backward pass), together with its per-tile column sums (the bias gradient).
+// products of the backward pass).
 //
-// One warp per row, three sweeps over the row (max, sum of exponentials, gradient), which
-// stay in L1 for the class counts used here.  Every reduction runs in a fixed order
-// (warp -> block -> part), so results do not change from run to run.
+// One warp per row.  With up to 128 classes a lane keeps its (at most four) logits in registers,
+// so the row is read once; wider rows are swept three times (max, sum of exponentials, gradient).
+// Loss sums are reduced in a fixed order (warp -> block -> part): results do not change from
+// run to run.
 #include "train.cuh"
 
 namespace {
 
 constexpr int LOSS_THREADS = 256;
-constexpr int LOSS_TILE_ROWS = BIAS_TILE_ROWS;
+constexpr int LOSS_TILE_ROWS = 64;
 constexpr int LOSS_ROWS_PER_WARP = LOSS_TILE_ROWS / (LOSS_THREADS / 32);
+constexpr int LOSS_REG_CLASSES = 128;
 
 __global__ void __launch_bounds__(LOSS_THREADS)
 softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
-                    const Planes dZ, float* __restrict__ tile_loss, float* __restrict__ bias_partial,
-                    const int64_t ld_bias) {
+                    const Planes dZ, float* __restrict__ tile_loss) {
     __shared__ float warp_loss[LOSS_THREADS / 32];
     int k, r0;
     if (!locate_tile(g, LOSS_TILE_ROWS, blockIdx.x, &k, &r0)) return;
@@ -30,22 +31,52 @@ softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const
         const int64_t r = g.row_ws[k] + i;
         const float* z = logits.ptr + r * logits.ld;
         const int label = yp[g.row_abs[k] + i];
-        float zmax = -INFINITY;
-        for (int c = lane; c < C; c += 32) zmax = fmaxf(zmax, z[c]);
+        if (C <= LOSS_REG_CLASSES) {
+            float v[4];
+            float zmax = -INFINITY;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
-        float sum = 0.f;
-        for (int c = lane; c < C; c += 32) sum += expf(z[c] - zmax);
+            for (int j = 0; j < 4; ++j) {
+                const int c = lane + 32 * j;
+                v[j] = c < C ? z[c] : -INFINITY;
+                zmax = fmaxf(zmax, v[j]);
+            }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        const float lse = zmax + logf(sum);
-        if (lane == 0) loss += lse - z[label];
-        for (int c = lane; c < C; c += 32) {
-            const float p = expf(z[c] - lse);
-            __nv_bfloat16 h, l;
-            split_bf16((p - (c == label ? 1.f : 0.f)) * inv_n, h, l);
-            dZ.hi[r * dZ.ld + c] = h;
-            dZ.lo[r * dZ.ld + c] = l;
+            for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+            float sum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) sum += lane + 32 * j < C ? expf(v[j] - zmax) : 0.f;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            const float lse = zmax + logf(sum);
+            const float zl = __shfl_sync(0xffffffffu, v[label >> 5], label & 31);
+            if (lane == 0) loss += lse - zl;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int c = lane + 32 * j;
+                if (c < C) {
+                    __nv_bfloat16 h, l;
+                    split_bf16((expf(v[j] - lse) - (c == label ? 1.f : 0.f)) * inv_n, h, l);
+                    dZ.hi[r * dZ.ld + c] = h;
+                    dZ.lo[r * dZ.ld + c] = l;
+                }
+            }
+        } else {
+            float zmax = -INFINITY;
+            for (int c = lane; c < C; c += 32) zmax = fmaxf(zmax, z[c]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+            float sum = 0.f;
+            for (int c = lane; c < C; c += 32) sum += expf(z[c] - zmax);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            const float lse = zmax + logf(sum);
+            if (lane == 0) loss += lse - z[label];
+            for (int c = lane; c < C; c += 32) {
+                __nv_bfloat16 h, l;
+                split_bf16((expf(z[c] - lse) - (c == label ? 1.f : 0.f)) * inv_n, h, l);
+                dZ.hi[r * dZ.ld + c] = h;
+                dZ.lo[r * dZ.ld + c] = l;
+            }
         }
     }
     if (lane == 0) warp_loss[warp] = loss;
@@ -54,16 +85,6 @@ softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const
         float s = 0.f;
         for (int w = 0; w < LOSS_THREADS / 32; ++w) s += warp_loss[w];
         tile_loss[blockIdx.x] = s;
-    }
-    // bias gradient of this tile: column sums of the rows just written, in row order
-    const int rows_here = min(LOSS_TILE_ROWS, n_p - r0);
-    for (int c = threadIdx.x; c < C; c += LOSS_THREADS) {
-        float s = 0.f;
-        for (int q = 0; q < rows_here; ++q) {
-            const int64_t at = (g.row_ws[k] + r0 + q) * dZ.ld + c;
-            s += join_bf16(dZ.hi[at], dZ.lo[at]);
-        }
-        bias_partial[(int64_t)blockIdx.x * ld_bias + c] = s;
     }
 }
 
@@ -89,12 +110,13 @@ loss_finalize_kernel(const __grid_constant__ GroupDesc g, const float* __restric
 
 }  // namespace
 
+int64_t loss_tiles(const GroupDesc& g) { return group_tiles(g, LOSS_TILE_ROWS); }
+
 int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp, Planes dZ,
-                            float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col,
-                            float* bias_partial, int64_t ld_bias, cudaStream_t s) {
+                            float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s) {
     const int64_t tiles = group_tiles(g, LOSS_TILE_ROWS);
     if (tiles > 0) {
-        { KernelScope ks(ctx, KC_LOSS, s); softmax_xent_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss, bias_partial, ld_bias); }
+        { KernelScope ks(ctx, KC_LOSS, s); softmax_xent_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss); }
         RTMA_LAUNCH_CHECK(ctx);
     }
     if (loss_out && g.num > 0) {

@@ -13,40 +13,14 @@ reduce_sgd_kernel(const __grid_constant__ GroupDesc g, const __grid_constant__ S
                   const float* __restrict__ partial, const float lr, float* __restrict__ params,
                   float* __restrict__ grads_record) {
     const int k = blockIdx.y;
-    const int64_t count = (int64_t)2 * ls.d_in * ls.d_out;          // the weight rows
-    const int64_t slot_stride = count + ls.d_out;                   // a slot also holds an (unused) bias row
+    const int64_t count = (int64_t)(2 * ls.d_in + 1) * ls.d_out;  // Ws, Wn and the bias row
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (i >= count) return;
     float gsum = 0.f;
-    for (int s = sp.split_begin[k]; s < sp.split_begin[k + 1]; ++s) gsum += partial[(int64_t)s * slot_stride + i];
+    for (int s = sp.split_begin[k]; s < sp.split_begin[k + 1]; ++s) gsum += partial[(int64_t)s * count + i];
     const int64_t at = (int64_t)g.part[k] * ls.P + ls.param_offset + i;
     if (grads_record) grads_record[at] = gsum;
     params[at] -= lr * gsum;
-}
-
-// Bias row: sum of the part's per-tile column sums.  A block takes 32 columns; its 8 row
-// groups each add every 8th tile, then the groups are added in order.
-__global__ void __launch_bounds__(256)
-bias_sgd_kernel(const __grid_constant__ GroupDesc g, const LayerShape ls, const float* __restrict__ bias_partial,
-                const int64_t ld_bias, const float lr, float* __restrict__ params, float* __restrict__ grads_record) {
-    __shared__ float red[8][32];
-    const int k = blockIdx.y;
-    const int c = blockIdx.x * 32 + (threadIdx.x & 31), rg = threadIdx.x >> 5;
-    int64_t first = 0;
-    for (int q = 0; q < k; ++q) first += (g.rows[q] + BIAS_TILE_ROWS - 1) / BIAS_TILE_ROWS;
-    const int64_t count = (g.rows[k] + BIAS_TILE_ROWS - 1) / BIAS_TILE_ROWS;
-    float s = 0.f;
-    if (c < ls.d_out)
-        for (int64_t t = rg; t < count; t += 8) s += bias_partial[(first + t) * ld_bias + c];
-    red[rg][threadIdx.x & 31] = s;
-    __syncthreads();
-    if (rg == 0 && c < ls.d_out) {
-        float gsum = 0.f;
-        for (int q = 0; q < 8; ++q) gsum += red[q][threadIdx.x];
-        const int64_t at = (int64_t)g.part[k] * ls.P + ls.param_offset + (int64_t)2 * ls.d_in * ls.d_out + c;
-        if (grads_record) grads_record[at] = gsum;
-        params[at] -= lr * gsum;
-    }
 }
 
 __global__ void __launch_bounds__(256)
@@ -134,15 +108,11 @@ int32_t aggregate_impl(rtma_ctx* ctx, float* params, const float* grads, float l
 }  // namespace
 
 int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, const float* partial,
-                          const float* bias_partial, int64_t ld_bias, float lr, float* params, float* grads_record,
-                          cudaStream_t s) {
+                          float lr, float* params, float* grads_record, cudaStream_t s) {
     if (g.num == 0) return RTMA_OK;
-    const int64_t count = (int64_t)2 * ls.d_in * ls.d_out;
+    const int64_t count = (int64_t)(2 * ls.d_in + 1) * ls.d_out;
     dim3 grid((unsigned)ceil_div(count, 256), (unsigned)g.num);
     { KernelScope ks(ctx, KC_REDUCE_SGD, s); reduce_sgd_kernel<<<grid, 256, 0, s>>>(g, sp, ls, partial, lr, params, grads_record); }
-    RTMA_LAUNCH_CHECK(ctx);
-    dim3 bgrid((unsigned)ceil_div(ls.d_out, 32), (unsigned)g.num);
-    { KernelScope ks(ctx, KC_REDUCE_SGD, s); bias_sgd_kernel<<<bgrid, 256, 0, s>>>(g, ls, bias_partial, ld_bias, lr, params, grads_record); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

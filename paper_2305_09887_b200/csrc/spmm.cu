@@ -15,8 +15,7 @@ namespace {
 
 constexpr int SPMM_THREADS = 256;
 constexpr int SPMM_ROWS_PER_WARP = 8;
-constexpr int SPMM_TILE_ROWS = SPMM_ROWS_PER_WARP * (SPMM_THREADS / 32);  // 64 = two bias tiles
-static_assert(SPMM_TILE_ROWS == 2 * BIAS_TILE_ROWS && BIAS_TILE_ROWS % SPMM_ROWS_PER_WARP == 0, "bias tiles");
+constexpr int SPMM_TILE_ROWS = SPMM_ROWS_PER_WARP * (SPMM_THREADS / 32);
 
 __global__ void __launch_bounds__(256)
 inv_degree_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, float* __restrict__ inv_deg) {
@@ -69,8 +68,7 @@ template <int NCH, bool BACKWARD>
 __global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 3 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
-            const Mat ST, const int d, float* __restrict__ bias_partial, const int64_t ld_bias) {
-    __shared__ float bias_red[BACKWARD ? SPMM_THREADS / 32 : 1][BACKWARD ? NCH * 256 : 1];
+            const Mat ST, const int d) {
     int k, r0;
     if (!locate_tile(g, SPMM_TILE_ROWS, blockIdx.x, &k, &r0)) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -86,12 +84,9 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     const int64_t e_begin = __shfl_sync(0xffffffffu, my_off, 0);
     const int64_t e_end = __shfl_sync(0xffffffffu, my_off, nrows);
 
-    Pack8 acc[NCH], colsum[NCH];
+    Pack8 acc[NCH];
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-        acc[c].zero();
-        colsum[c].zero();
-    }
+    for (int c = 0; c < NCH; ++c) acc[c].zero();
     int cur = 0;  // row (relative to i0) the accumulators belong to
 
     // finishes row `row`: scale or gate, store, clear
@@ -110,9 +105,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const float gate = (e & 1) ? __high2float(gp[e >> 1]) : __low2float(gp[e >> 1]);
-                        const float v = gate > 0.f ? acc[c].v[e] + sv[e] : 0.f;
-                        acc[c].v[e] = v;
-                        colsum[c].v[e] += v;
+                        acc[c].v[e] = gate > 0.f ? acc[c].v[e] + sv[e] : 0.f;
                     }
                 } else {
                     const float w = inv_deg[r];
@@ -204,31 +197,11 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     }
     while (cur < nrows) flush(cur++);
 
-    if (BACKWARD) {
-        // column sums of the block's two bias tiles (warps 0-3 and 4-7), added in warp order
-#pragma unroll
-        for (int c = 0; c < NCH; ++c)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) bias_red[warp][c * 256 + lane * 8 + e] = colsum[c].v[e];
-        __syncthreads();
-        int64_t tile0 = 0;  // bias tile number of the block's first tile
-        for (int q = 0; q < k; ++q) tile0 += (g.rows[q] + BIAS_TILE_ROWS - 1) / BIAS_TILE_ROWS;
-        tile0 += r0 / BIAS_TILE_ROWS;
-        constexpr int WARPS_PER_TILE = BIAS_TILE_ROWS / SPMM_ROWS_PER_WARP;
-        for (int idx = threadIdx.x; idx < 2 * d; idx += SPMM_THREADS) {
-            const int half = idx / d, c = idx - half * d;
-            if (r0 + half * BIAS_TILE_ROWS >= n_p) continue;
-            float s = 0.f;
-            for (int w = 0; w < WARPS_PER_TILE; ++w) s += bias_red[half * WARPS_PER_TILE + w][c];
-            bias_partial[(tile0 + half) * ld_bias + c] = s;
-        }
-    }
 }
 
 template <bool BACKWARD>
 int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                      const float* inv_deg, Planes src, Planes out, Mat ST, int d, float* bias_partial, int64_t ld_bias,
-                      cudaStream_t s) {
+                      const float* inv_deg, Planes src, Planes out, Mat ST, int d, cudaStream_t s) {
     const int64_t tiles = group_tiles(g, SPMM_TILE_ROWS);
     if (tiles == 0) return RTMA_OK;
     const unsigned grid = (unsigned)tiles;
@@ -236,7 +209,7 @@ int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_o
     do {                                                                                                  \
         KernelScope ks(ctx, BACKWARD ? KC_SPMM_BWD : KC_SPMM_FWD, s);                                     \
         spmm_kernel<N, BACKWARD><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, \
-                                                               ST, d, bias_partial, ld_bias);             \
+                                                               ST, d);                                    \
     } while (0)
     if (d <= 256) RTMA_SPMM(1);
     else if (d <= 512) RTMA_SPMM(2);
@@ -275,11 +248,10 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                          const float* inv_deg, Planes src, Planes out, int d, cudaStream_t s) {
-    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, Mat{nullptr, 0}, d, nullptr, 0, s);
+    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, Mat{nullptr, 0}, d, s);
 }
 
 int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat ST, Planes h, int d, float* bias_partial, int64_t ld_bias, cudaStream_t s) {
-    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, nullptr, Planes{nullptr, nullptr, 0}, h, ST, d, bias_partial,
-                               ld_bias, s);
+                             Mat ST, Planes h, int d, cudaStream_t s) {
+    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, nullptr, Planes{nullptr, nullptr, 0}, h, ST, d, s);
 }

@@ -41,7 +41,6 @@ int32_t parse_model(rtma_ctx* ctx, const rtma_model_desc* md, Model* m) {
 struct ScratchPlan {
     size_t per_row_bytes;     // planes, logits, [S|T], 1/deg
     size_t max_layer_params;  // largest (2 d_in + 1) d_out
-    size_t max_bias_ld;       // widest d_out, padded
     size_t prep_bytes;        // repacked weights, per part
     size_t st_half;           // floats in one half of [S | T]
 };
@@ -58,7 +57,6 @@ ScratchPlan plan_scratch(const Model& m) {
         if (l < m.L - 1) per_row += 4 * planes_ld(m.dims[l + 1]);  // H^{l+1}, later overwritten by dZ^l
         if (l >= 1) widest_hidden = std::max(widest_hidden, planes_ld(m.dims[l]));
         sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(2 * m.dims[l] + 1) * m.dims[l + 1]);
-        sp.max_bias_ld = std::max(sp.max_bias_ld, planes_ld(m.dims[l + 1]));
         sp.prep_bytes += sizeof(__nv_bfloat16) * tc_prep_elems(tc_plan_layer(m.layer[l]), l >= 1) + 4 * 256;
     }
     per_row += sizeof(float) * planes_ld(m.dims[m.L]);  // logits
@@ -80,7 +78,7 @@ int splits_for(int64_t n_p, int parts_in_flight) {
 size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
     const size_t rows = (size_t)aligned_rows(n_p);
     const size_t matrices = 8 * m.L + 12;  // every matrix start is rounded up to 256 bytes
-    return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, BIAS_TILE_ROWS) * (1 + sp.max_bias_ld) + 256) +
+    return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, 32) + 256) +
            sp.prep_bytes + 256 * matrices;
 }
 
@@ -219,10 +217,7 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
             Planes dZlast = take_planes(C);
             Mat ST{cur.take<float>((size_t)rows * 2 * plan.st_half + 8), (int64_t)(2 * plan.st_half)};
             float* partial = cur.take<float>((size_t)slots * plan.max_layer_params + 4);
-            const int64_t bias_tiles = group_tiles(g, BIAS_TILE_ROWS);
-            float* tile_loss = cur.take<float>((size_t)bias_tiles + 4);
-            float* bias_partial = cur.take<float>((size_t)bias_tiles * plan.max_bias_ld + 4);
-            const int64_t ld_bias = (int64_t)plan.max_bias_ld;
+            float* tile_loss = cur.take<float>((size_t)loss_tiles(g) + 4);
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
             __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
@@ -273,18 +268,15 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                     }
                 }
                 // ---- loss; dZ of the last layer and its tile column sums ----
-                RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, K, step, bias_partial, ld_bias, s));
+                RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, K, step, s));
                 // ---- backward + SGD ----
                 for (int l = m.L - 1; l >= 0; --l) {
                     const Planes dZ = l == m.L - 1 ? dZlast : Hl[l + 1];
                     RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, s));
                     if (l > 0) RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, s));
-                    // the bias gradient of layer l comes from the tile sums written with dZ^l; reduce
-                    // them before the next aggregation overwrites the tile sums with those of dZ^{l-1}
-                    RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, bias_partial, ld_bias, m.lr, params,
-                                               tap ? taps->grads : nullptr, s));
+                    RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
                     if (l > 0)  // dZ^{l-1} overwrites H^l, whose sign is the ReLU gate
-                        RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, ST, Hl[l], m.dims[l], bias_partial, ld_bias, s));
+                        RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, ST, Hl[l], m.dims[l], s));
                 }
             }
         }

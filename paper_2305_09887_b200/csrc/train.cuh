@@ -65,10 +65,6 @@ struct SplitPlan {
     int32_t rows_per_split[RTMA_MAX_PARTS];
 };
 
-// Column sums of dZ are produced by the kernels that write dZ, one row of sums per tile of
-// BIAS_TILE_ROWS rows (tiles numbered part after part), and reduced with the bias update.
-constexpr int BIAS_TILE_ROWS = 32;
-
 // ---- spmm.cu --------------------------------------------------------------------------
 // fp32 rows in partition order -> split planes in scratch rows.
 int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, int d, Planes out, cudaStream_t s);
@@ -81,24 +77,21 @@ int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowpt
                          const float* inv_deg, Planes src, Planes out, int d, cudaStream_t s);
 // h[r] <- (S[r] + sum_{u in N(r)} T[u]) where h[r] > 0 else 0, S = ST[:, 0:d], T = ST[:, d:2d]
 // (backward through the symmetric aggregation and the ReLU; h holds H on entry, dZ on exit).
-// Also writes the column sums of every BIAS_TILE_ROWS-row tile of the result to bias_partial.
 int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat ST, Planes h, int d, float* bias_partial, int64_t ld_bias, cudaStream_t s);
+                             Mat ST, Planes h, int d, cudaStream_t s);
 
 // ---- loss.cu --------------------------------------------------------------------------
 // Softmax cross-entropy over fp32 logits, mean over the part; dZ = (softmax - onehot) / n_p is
-// written as split planes, its tile column sums to bias_partial, and the part's loss to
-// loss_out[part * loss_stride + loss_col] when loss_out != NULL.
+// written as split planes and the part's loss to loss_out[part * loss_stride + loss_col] when
+// loss_out != NULL.  tile_loss: loss_tiles(g) floats of scratch.
+int64_t loss_tiles(const GroupDesc& g);
 int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp, Planes dZ,
-                            float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col,
-                            float* bias_partial, int64_t ld_bias, cudaStream_t s);
+                            float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s);
 
 // ---- optim.cu -------------------------------------------------------------------------
-// Weight rows: grad = sum of the part's chunk slots; bias row: grad = sum of the part's tile
-// column sums; params -= lr * grad; optionally records grad.
+// grad = sum of the part's chunk slots; params -= lr * grad; optionally records grad.
 int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, const float* partial,
-                          const float* bias_partial, int64_t ld_bias, float lr, float* params, float* grads_record,
-                          cudaStream_t s);
+                          float lr, float* params, float* grads_record, cudaStream_t s);
 int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float* dst, int64_t ld_dst, int64_t rows,
                          int width, cudaStream_t s);
 
@@ -122,6 +115,6 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                         Planes dZ, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, const float* inv_deg, Mat ST,
                         cudaStream_t s);
-// partial[slot][0 : 2 d_in][d_out] = [H | N]^T dZ over one chunk of rows (the bias row is not touched).
+// partial[slot][(2 d_in + 1) x d_out] = [H | N | 1]^T dZ over one chunk of rows.
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
                         Planes H, Planes N, Planes dZ, float* partial, cudaStream_t s);
