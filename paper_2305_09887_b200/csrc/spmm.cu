@@ -3,7 +3,7 @@
 // stored as split bf16 planes; plus the conversions between fp32 rows and planes.
 //
 // Gather-bound and, at the tiny local degrees random partitioning leaves (about deg/M),
-// latency-bound: a warp owns 8 consecutive rows, reads their offsets with one load and their
+// latency-bound: a warp takes 8 consecutive rows at a time, reads their offsets with one load and their
 // column indices with one coalesced load per 32 entries (consecutive rows are consecutive
 // in the CSR), and walks the entries with four neighbours' rows in flight per lane.  Lanes
 // split the feature width in pieces of 8 values (16 bytes per plane).
@@ -15,7 +15,6 @@ namespace {
 
 constexpr int SPMM_THREADS = 256;
 constexpr int SPMM_ROWS_PER_WARP = 8;
-constexpr int SPMM_TILE_ROWS = SPMM_ROWS_PER_WARP * (SPMM_THREADS / 32);
 
 __global__ void __launch_bounds__(256)
 inv_degree_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, float* __restrict__ inv_deg) {
@@ -68,15 +67,22 @@ template <int NCH, bool BACKWARD>
 __global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 3 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
-            const Mat ST, const int d) {
-    int k, r0;
-    if (!locate_tile(g, SPMM_TILE_ROWS, blockIdx.x, &k, &r0)) return;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            const Mat ST, const int d, const int64_t total_groups, int* __restrict__ ticket) {
+    const int lane = threadIdx.x & 31;
+  // Warps draw groups of 8 consecutive rows from a shared ticket counter until none are left:
+  // degrees are power-law distributed, and a fixed assignment would leave most warps idle while
+  // a few finish their hub rows.
+  for (;;) {
+    int64_t grp = 0;
+    if (lane == 0) grp = atomicAdd(ticket, 1);
+    grp = __shfl_sync(0xffffffffu, grp, 0);
+    if (grp >= total_groups) break;
+    int k, i0;
+    if (!locate_tile(g, SPMM_ROWS_PER_WARP, grp, &k, &i0)) break;
     const int n_p = g.rows[k];
     const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
     const int32_t* cols = col_out + g.edge_abs[k];
     const int64_t ws = g.row_ws[k];
-    const int i0 = r0 + warp * SPMM_ROWS_PER_WARP;
     const int nrows = max(0, min(SPMM_ROWS_PER_WARP, n_p - i0));
 
     // offsets of the warp's rows: lane j holds rp[i0 + j], j = 0..nrows
@@ -196,20 +202,32 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
         }
     }
     while (cur < nrows) flush(cur++);
-
+  }
+    // the last warp to run dry re-arms the ticket for the next launch
+    if (lane == 0) {
+        const int total_warps = gridDim.x * (SPMM_THREADS / 32);
+        if (atomicAdd(ticket + 1, 1) == total_warps - 1) {
+            ticket[0] = 0;
+            ticket[1] = 0;
+        }
+    }
 }
 
 template <bool BACKWARD>
 int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                      const float* inv_deg, Planes src, Planes out, Mat ST, int d, cudaStream_t s) {
-    const int64_t tiles = group_tiles(g, SPMM_TILE_ROWS);
-    if (tiles == 0) return RTMA_OK;
-    const unsigned grid = (unsigned)tiles;
+                      const float* inv_deg, Planes src, Planes out, Mat ST, int d, int* ticket, cudaStream_t s) {
+    const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
+    if (groups == 0) return RTMA_OK;
+    if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
+    static int sms = 0;
+    if (!sms && (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess || sms <= 0)) sms = 148;
+    const int blocks_per_sm = d <= 256 ? 3 : 1;
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, SPMM_THREADS / 32), (int64_t)sms * blocks_per_sm);
 #define RTMA_SPMM(N)                                                                                      \
     do {                                                                                                  \
         KernelScope ks(ctx, BACKWARD ? KC_SPMM_BWD : KC_SPMM_FWD, s);                                     \
         spmm_kernel<N, BACKWARD><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, \
-                                                               ST, d);                                    \
+                                                               ST, d, groups, ticket);                    \
     } while (0)
     if (d <= 256) RTMA_SPMM(1);
     else if (d <= 512) RTMA_SPMM(2);
@@ -247,11 +265,11 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 }
 
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                         const float* inv_deg, Planes src, Planes out, int d, cudaStream_t s) {
-    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, Mat{nullptr, 0}, d, s);
+                         const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s) {
+    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, Mat{nullptr, 0}, d, ticket, s);
 }
 
 int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat ST, Planes h, int d, cudaStream_t s) {
-    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, nullptr, Planes{nullptr, nullptr, 0}, h, ST, d, s);
+                             Mat ST, Planes h, int d, int* ticket, cudaStream_t s) {
+    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, nullptr, Planes{nullptr, nullptr, 0}, h, ST, d, ticket, s);
 }

@@ -218,6 +218,7 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
             Mat ST{cur.take<float>((size_t)rows * 2 * plan.st_half + 8), (int64_t)(2 * plan.st_half)};
             float* partial = cur.take<float>((size_t)slots * plan.max_layer_params + 4);
             float* tile_loss = cur.take<float>((size_t)loss_tiles(g) + 4);
+            int* ticket = cur.take<int>(64);  // work counter of the aggregation kernels (zero between launches)
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
             __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
@@ -245,7 +246,7 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                 for (int l = 0; l < m.L; ++l)
                     RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
                 for (int l = 0; l < m.L; ++l) {
-                    RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], s));
+                    RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], ticket, s));
                     const bool last = l == m.L - 1;
                     RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
                                                last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, s));
@@ -276,7 +277,7 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                     if (l > 0) RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, s));
                     RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
                     if (l > 0)  // dZ^{l-1} overwrites H^l, whose sign is the ReLU gate
-                        RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, ST, Hl[l], m.dims[l], s));
+                        RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, ST, Hl[l], m.dims[l], ticket, s));
                 }
             }
         }

@@ -73,12 +73,13 @@ int32_t launch_from_planes(rtma_ctx* ctx, Planes src, int64_t first_row, int64_t
 // inv_deg[row_ws + i] = 1 / local degree (0 for an isolated node).
 int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s);
 // out[r] = inv_deg[r] * sum_{u in N(r)} src[u]                      (forward, mean)
+// ticket: two ints of scratch, zero on entry and zero again when the kernel has finished.
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                         const float* inv_deg, Planes src, Planes out, int d, cudaStream_t s);
+                         const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s);
 // h[r] <- (S[r] + sum_{u in N(r)} T[u]) where h[r] > 0 else 0, S = ST[:, 0:d], T = ST[:, d:2d]
 // (backward through the symmetric aggregation and the ReLU; h holds H on entry, dZ on exit).
 int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat ST, Planes h, int d, cudaStream_t s);
+                             Mat ST, Planes h, int d, int* ticket, cudaStream_t s);
 
 // ---- loss.cu --------------------------------------------------------------------------
 // Softmax cross-entropy over fp32 logits, mean over the part; dZ = (softmax - onehot) / n_p is
