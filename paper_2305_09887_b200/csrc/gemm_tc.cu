@@ -128,6 +128,9 @@ struct RowsArgs {
 // 2..9 = epilogue (two warps per TMEM lane quarter, alternating 32-column chunks).
 constexpr int ROWS_THREADS = 320;
 constexpr int ROWS_EPI_THREADS = 256;
+constexpr int ROWS_STAGING_BYTES = 4096;          // per epilogue warp: a 32 x 32 fp32 block (or two 32 x 32 bf16)
+constexpr int ROWS_RING_BUDGET = 192 * 1024;      // shared memory for the operand ring
+constexpr int ROWS_SMEM_MAX = ROWS_RING_BUDGET + 1024 + 8 * ROWS_STAGING_BYTES;
 
 struct RowsBarriers {
     uint64_t full[MAX_STAGES];
@@ -148,6 +151,7 @@ __device__ __forceinline__ bool rows_wait(uint64_t* bar, uint32_t parity, RowsBa
     return false;
 }
 
+template <bool PLANES_OUT>
 __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_constant__ RowsArgs a) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ RowsBarriers pb;
@@ -253,6 +257,7 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
         const int ew = warp - 2;          // 0..7
         const int q = warp & 3;           // the TMEM lane quarter this warp may read
         const int col_phase = ew >> 2;    // which of the two warps of the quarter: even or odd chunks
+        uint8_t* stg = smem + (size_t)stages * stage_bytes + (size_t)ew * ROWS_STAGING_BYTES;  // 4 KB per warp
         int64_t t = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++t) {
@@ -266,47 +271,88 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.tmem_cols);
             const int i = r0 + q * 32 + lane;
             const bool live = i < a.g.rows[k];
-            const int64_t orow = a.g.row_ws[k] + i;
             const float* bias = a.bias_offset >= 0 ? a.params + (int64_t)a.g.part[k] * a.P + a.bias_offset : nullptr;
-            const float w = (a.scale_from >= 0 && live) ? a.inv_deg[orow] : 1.f;
+            const float w = (a.scale_from >= 0 && live) ? a.inv_deg[a.g.row_ws[k] + i] : 1.f;
+            const int rows_here = min(32, a.g.rows[k] - (r0 + q * 32));  // live rows of this warp's quarter
+            const int64_t orow0 = a.g.row_ws[k] + r0 + q * 32;
             for (int c0 = col_phase * 32; c0 < BN; c0 += 64) {
                 float v[32];
                 tc::tmem_load_32x32(d_tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-                if (!live) continue;
+                if (rows_here <= 0) continue;
+                const int nbase = n0 + c0;
+                if constexpr (!PLANES_OUT) {
+                    // fp32 output (logits, [S | T]): each thread stores its own row, pack by pack
+                    if (!live) continue;
+                    float* o = a.out + (orow0 + lane) * a.ld_out;
 #pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    const int n = n0 + c0 + j;
-                    if (n >= a.N || c0 + j >= BN) break;  // BN is a multiple of 16, not always of 32
-                    Pack8 x;
+                    for (int j = 0; j < 32; j += 8) {
+                        const int n = nbase + j;
+                        if (n >= a.N || c0 + j >= BN) break;  // BN is a multiple of 16, not always of 32
+                        float x[8];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        float tv = v[j + e];
-                        if (n + e < a.N) {
-                            if (bias) tv += __ldg(bias + n + e);
-                            if (a.scale_from >= 0 && n + e >= a.scale_from) tv *= w;
-                            if (a.relu) tv = fmaxf(tv, 0.f);
-                        } else {
-                            tv = 0.f;
+                        for (int e = 0; e < 8; ++e) {
+                            float tv = v[j + e];
+                            if (n + e < a.N) {
+                                if (bias) tv += __ldg(bias + n + e);
+                                if (a.scale_from >= 0 && n + e >= a.scale_from) tv *= w;
+                                if (a.relu) tv = fmaxf(tv, 0.f);
+                            }
+                            x[e] = tv;
                         }
-                        x.v[e] = tv;
-                    }
-                    if (a.out_planes.hi) {
-                        uint4 h, l;  // the padded row length is a multiple of 8: whole packs fit
-                        x.to_planes(h, l);
-                        *reinterpret_cast<uint4*>(a.out_planes.hi + orow * a.out_planes.ld + n) = h;
-                        *reinterpret_cast<uint4*>(a.out_planes.lo + orow * a.out_planes.ld + n) = l;
-                    } else {
-                        float* o = a.out + orow * a.ld_out;
                         const bool straddles = a.scale_from >= 0 && n < a.scale_from && n + 7 >= a.scale_from;
                         const int dst0 = (a.scale_from >= 0 && n >= a.scale_from) ? n + a.scale_shift : n;
                         if (!straddles && n + 7 < a.N && (dst0 & 3) == 0) {
-                            *reinterpret_cast<float4*>(o + dst0) = make_float4(x.v[0], x.v[1], x.v[2], x.v[3]);
-                            *reinterpret_cast<float4*>(o + dst0 + 4) = make_float4(x.v[4], x.v[5], x.v[6], x.v[7]);
+                            *reinterpret_cast<float4*>(o + dst0) = make_float4(x[0], x[1], x[2], x[3]);
+                            *reinterpret_cast<float4*>(o + dst0 + 4) = make_float4(x[4], x[5], x[6], x[7]);
                         } else {
                             for (int e = 0; e < 8 && n + e < a.N; ++e)
-                                o[(a.scale_from >= 0 && n + e >= a.scale_from) ? n + e + a.scale_shift : n + e] = x.v[e];
+                                o[(a.scale_from >= 0 && n + e >= a.scale_from) ? n + e + a.scale_shift : n + e] = x[e];
                         }
                     }
+                } else {
+                // plane output: bias, ReLU on the thread's own row; columns past N (or past the tile) become 0
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int n = nbase + e;
+                    float tv = v[e];
+                    if (n < a.N && c0 + e < BN) {
+                        if (bias) tv += __ldg(bias + n);
+                        if (a.relu) tv = fmaxf(tv, 0.f);
+                    } else {
+                        tv = 0.f;
+                    }
+                    v[e] = tv;
+                }
+                // Transpose through the warp's staging slab so that every store instruction writes
+                // whole 128-byte (fp32) or 64-byte (plane) row segments instead of 32 scattered pieces.
+                __syncwarp();
+                {
+                    uint4* sh = reinterpret_cast<uint4*>(stg);        // [32 rows][4 pieces of 8 bf16], hi
+                    uint4* sl = sh + 128;                             // lo
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        Pack8 x;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) x.v[e] = v[8 * p + e];
+                        uint4 h, l;
+                        x.to_planes(h, l);
+                        const int slot = lane * 4 + (p ^ ((lane >> 1) & 3));
+                        sh[slot] = h;
+                        sl[slot] = l;
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const int row = it * 8 + (lane >> 2), p = lane & 3;
+                        const int n = nbase + 8 * p;
+                        if (row < rows_here && n < a.out_planes.ld && c0 + 8 * p < BN) {
+                            const int slot = row * 4 + (p ^ ((row >> 1) & 3));
+                            const int64_t at = (orow0 + row) * a.out_planes.ld + n;
+                            *reinterpret_cast<uint4*>(a.out_planes.hi + at) = sh[slot];
+                            *reinterpret_cast<uint4*>(a.out_planes.lo + at) = sl[slot];
+                        }
+                    }
+                }
                 }
             }
             tc::tc_fence_before_sync();
@@ -626,18 +672,27 @@ int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, 
 static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
-        RTMA_TRY(set_smem_limit(ctx, reinterpret_cast<const void*>(tc_rows_kernel)));
+        RTMA_CUDA(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(tc_rows_kernel<true>),
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, ROWS_SMEM_MAX));
+        RTMA_CUDA(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(tc_rows_kernel<false>),
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, ROWS_SMEM_MAX));
         configured = true;
     }
     const size_t stage_bytes = 2 * (size_t)PLANE_TILE_BYTES + 2 * (size_t)a.BN * 128;
-    a.stages = stages_for(stage_bytes, a.kb0 + a.kb1);
+    a.stages = std::max(1, std::min<int>(MAX_STAGES, (int)(ROWS_RING_BUDGET / stage_bytes)));
     a.tmem_cols = (int)tmem_columns_for(a.BN);
     a.error_word = ctx->error_word;
     a.row_tiles = group_tiles(a.g, TC_BM);
     if (a.row_tiles == 0) return RTMA_OK;
     const int64_t total_tiles = a.row_tiles * (a.Npad / a.BN);
     const unsigned grid = (unsigned)std::min<int64_t>(total_tiles, sm_count_of(ctx->device));
-    { KernelScope ks(ctx, kclass, s); tc_rows_kernel<<<grid, ROWS_THREADS, a.stages * stage_bytes + 1024, s>>>(a); }
+    // the epilogue staging slabs are only allocated for plane output: shared memory comes out of L1
+    {
+        KernelScope ks(ctx, kclass, s);
+        const size_t ring = a.stages * stage_bytes + 1024;
+        if (a.out_planes.hi) tc_rows_kernel<true><<<grid, ROWS_THREADS, ring + 8 * ROWS_STAGING_BYTES, s>>>(a);
+        else tc_rows_kernel<false><<<grid, ROWS_THREADS, ring, s>>>(a);
+    }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
