@@ -20,14 +20,29 @@ struct Planes {
 inline size_t planes_ld(int64_t d) { return (size_t)((d + 7) / 8 * 8); }
 
 #ifdef __CUDACC__
+// Conversions are written with integer arithmetic on purpose: the dedicated conversion
+// instructions issue on the narrow special-function pipe, which became the limit of the
+// aggregation kernels.  Round-to-nearest-even; inputs are assumed finite.
+__device__ __forceinline__ uint32_t bf16_bits_rn(float x) {
+    const uint32_t u = __float_as_uint(x);
+    return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+// x -> (hi bits, lo bits): hi = bf16(x), lo = bf16(x - hi)
+__device__ __forceinline__ void split_bits(float x, uint32_t& hi, uint32_t& lo) {
+    hi = bf16_bits_rn(x);
+    lo = bf16_bits_rn(x - bf16_bits_to_float(hi));
+}
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
-    hi = __float2bfloat16_rn(x);
-    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+    uint32_t h, l;
+    split_bits(x, h, l);
+    hi = __ushort_as_bfloat16((unsigned short)h);
+    lo = __ushort_as_bfloat16((unsigned short)l);
 }
 __device__ __forceinline__ float join_bf16(__nv_bfloat16 hi, __nv_bfloat16 lo) {
-    return __bfloat162float(hi) + __bfloat162float(lo);
+    return bf16_bits_to_float(__bfloat16_as_ushort(hi)) + bf16_bits_to_float(__bfloat16_as_ushort(lo));
 }
-// Eight consecutive elements (16 bytes per plane).
+// Eight consecutive elements (16 bytes per plane); a 32-bit word holds elements 2i (low half) and 2i+1.
 struct Pack8 {
     float v[8];
     __device__ __forceinline__ void zero() {
@@ -35,27 +50,25 @@ struct Pack8 {
         for (int i = 0; i < 8; ++i) v[i] = 0.f;
     }
     __device__ __forceinline__ void add_planes(const uint4 h, const uint4 l) {
-        const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&h);
-        const __nv_bfloat162* lp = reinterpret_cast<const __nv_bfloat162*>(&l);
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w}, lw[4] = {l.x, l.y, l.z, l.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float2 a = __bfloat1622float2(hp[i]);
-            const float2 b = __bfloat1622float2(lp[i]);
-            v[2 * i] += a.x + b.x;
-            v[2 * i + 1] += a.y + b.y;
+            v[2 * i] += __uint_as_float(hw[i] << 16) + __uint_as_float(lw[i] << 16);
+            v[2 * i + 1] += __uint_as_float(hw[i] & 0xFFFF0000u) + __uint_as_float(lw[i] & 0xFFFF0000u);
         }
     }
     __device__ __forceinline__ void to_planes(uint4& h, uint4& l) const {
-        __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&h);
-        __nv_bfloat162* lp = reinterpret_cast<__nv_bfloat162*>(&l);
+        uint32_t hw[4], lw[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            __nv_bfloat16 h0, l0, h1, l1;
-            split_bf16(v[2 * i], h0, l0);
-            split_bf16(v[2 * i + 1], h1, l1);
-            hp[i] = __halves2bfloat162(h0, h1);
-            lp[i] = __halves2bfloat162(l0, l1);
+            uint32_t h0, l0, h1, l1;
+            split_bits(v[2 * i], h0, l0);
+            split_bits(v[2 * i + 1], h1, l1);
+            hw[i] = h0 | (h1 << 16);
+            lw[i] = l0 | (l1 << 16);
         }
+        h = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        l = make_uint4(lw[0], lw[1], lw[2], lw[3]);
     }
 };
 #endif

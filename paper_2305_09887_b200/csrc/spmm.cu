@@ -106,11 +106,11 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                     const float* s = ST.ptr + r * ST.ld + colx;
                     const float4 s0 = *reinterpret_cast<const float4*>(s), s1 = *reinterpret_cast<const float4*>(s + 4);
                     const uint4 gh = *reinterpret_cast<const uint4*>(out.hi + r * out.ld + colx);
-                    const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gh);
+                    const uint32_t gw[4] = {gh.x, gh.y, gh.z, gh.w};
                     const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const float gate = (e & 1) ? __high2float(gp[e >> 1]) : __low2float(gp[e >> 1]);
+                        const float gate = __uint_as_float((e & 1) ? (gw[e >> 1] & 0xFFFF0000u) : (gw[e >> 1] << 16));
                         acc[c].v[e] = gate > 0.f ? acc[c].v[e] + sv[e] : 0.f;
                     }
                 } else {
