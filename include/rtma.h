@@ -174,11 +174,37 @@ int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* model, int32_t M,
                          const float* Xp, const int32_t* yp, float* params, int32_t K,
                          float* loss_out, const rtma_taps* taps, void* const* streams);
 
+/* Local training with a step count of its own for every trainer.  Aggregation is triggered by
+ * wall time, not by a step count (Sec. 3.1), so trainers arrive at an aggregation with
+ * different numbers of finished steps (Table 4 reports up to 28.8% fewer on the slowest one):
+ * trainer i runs steps_host[i] steps.  steps_host[i] = 0 is a trainer that did not run at all,
+ * e.g. one that failed to start (Sec. 4.5): its replica is left untouched and it takes neither
+ * scratch nor launches.
+ *   steps_host  HOST array [M], every entry >= 0.
+ *   loss_out    [M][loss_stride] float or NULL, loss_stride >= max_i steps_host[i]; entries
+ *               [i][s] with s >= steps_host[i] are not written.
+ * Everything else as for rtma_local_steps, which is this call with every entry equal to K and
+ * loss_stride = K.  Trainers that have finished drop out of the later launches.              */
+int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* model, int32_t M,
+                             const int64_t* part_offsets_host, const int64_t* edge_offsets_host,
+                             const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                             const float* Xp, const int32_t* yp, float* params,
+                             const int32_t* steps_host, int32_t loss_stride, float* loss_out,
+                             const rtma_taps* taps, void* const* streams);
+
 /* ---- R2: aggregation (Algorithm 1, phi = plain average; Algorithm 2, overwrite) ---------
  * Wbar[j] = (1/M) sum_i params[i][j]; every replica is overwritten with Wbar; global_out
  * [P] (or NULL) also receives it.  M = 1 leaves the parameters unchanged.                 */
 int32_t rtma_aggregate(rtma_ctx* ctx, float* params, int64_t P, int32_t M, float* global_out,
                        void* stream);
+
+/* Aggregation when some trainers are offline (Sec. 4.5: training continues with the remaining
+ * trainers): Wbar[j] = (1/|A|) sum_{i in A} params[i][j], A = { i : active_host[i] != 0 }.
+ * Every replica, the inactive ones included, is overwritten with Wbar, as a trainer that
+ * comes back would receive it.  active_host: HOST array [M] of bytes; an empty A is
+ * RTMA_ERR_INVALID_ARG.  With every byte set this is rtma_aggregate, bit for bit.            */
+int32_t rtma_aggregate_masked(rtma_ctx* ctx, float* params, int64_t P, int32_t M,
+                              const uint8_t* active_host, float* global_out, void* stream);
 
 /* The last local step fused with the aggregation: Wbar = (1/M) sum_i (params[i] - lr *
  * grads[i]), written to every replica (and global_out).  grads [M][P].                    */

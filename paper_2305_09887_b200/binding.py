@@ -22,6 +22,7 @@ EXPORTS = (
     "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
+    "rtma_local_steps_var", "rtma_aggregate_masked",
 )
 KERNEL_CLASSES = 19
 
@@ -235,7 +236,8 @@ class Context:
     # ---- Algorithm 2 ----------------------------------------------------------------
     def local_steps(self, dims, lr, M, part_offsets_host, edge_offsets_host, rowptr_out, col_out, Xp, yp,
                     params, K, loss_out=None, streams=None, gemm_dtype=0, taps=None, symmetric=True):
-        """K SGD steps on each of the M parts, in place on params [M, P].
+        """K SGD steps on each of the M parts, in place on params [M, P].  K: an int, or a sequence
+        of M per-trainer step counts (0 = the trainer does not run; rtma_local_steps_var).
         streams: None (all trainers on the current stream), or a list of M torch streams.
         taps: None or (acts tensor or None, grads tensor or None, step)."""
         dev = self.device
@@ -258,11 +260,23 @@ class Context:
         if taps is not None:
             acts, grads, step = taps
             tap_struct = Taps(_ptr(acts), _ptr(grads), int(step))
-        st = self._lib.rtma_local_steps(
-            self._h, ctypes.byref(md), ctypes.c_int32(M), po, eo, _ptr(rowptr_out), _ptr(col_out),
-            ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), _ptr(yp), _ptr(params), ctypes.c_int32(K),
-            _ptr(loss_out), ctypes.byref(tap_struct) if tap_struct is not None else None, sarr)
-        self._check(st, "rtma_local_steps")
+        tap_ref = ctypes.byref(tap_struct) if tap_struct is not None else None
+        if isinstance(K, int):
+            st = self._lib.rtma_local_steps(
+                self._h, ctypes.byref(md), ctypes.c_int32(M), po, eo, _ptr(rowptr_out), _ptr(col_out),
+                ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), _ptr(yp), _ptr(params), ctypes.c_int32(K),
+                _ptr(loss_out), tap_ref, sarr)
+            self._check(st, "rtma_local_steps")
+        else:
+            if len(K) != M:
+                raise ValueError("one step count per trainer")
+            steps = (ctypes.c_int32 * M)(*[int(v) for v in K])
+            stride = int(loss_out.shape[1]) if loss_out is not None else max([int(v) for v in K] + [0])
+            st = self._lib.rtma_local_steps_var(
+                self._h, ctypes.byref(md), ctypes.c_int32(M), po, eo, _ptr(rowptr_out), _ptr(col_out),
+                ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), _ptr(yp), _ptr(params), steps,
+                ctypes.c_int32(stride), _ptr(loss_out), tap_ref, sarr)
+            self._check(st, "rtma_local_steps_var")
 
     # ---- R2 -------------------------------------------------------------------------
     def aggregate(self, params, global_out=None, stream=None):
@@ -271,6 +285,17 @@ class Context:
         st = self._lib.rtma_aggregate(self._h, _ptr(params), ctypes.c_int64(P), ctypes.c_int32(M),
                                       _ptr(global_out), ctypes.c_void_p(_stream_handle(stream)))
         self._check(st, "rtma_aggregate")
+
+    def aggregate_masked(self, params, active, global_out=None, stream=None):
+        """Average over the replicas whose entry of `active` (M truthy / falsy values) is set."""
+        M, P = params.shape
+        _need(params, torch.float32, "params", self.device)
+        if len(active) != M:
+            raise ValueError("one flag per trainer")
+        mask = (ctypes.c_uint8 * M)(*[1 if a else 0 for a in active])
+        st = self._lib.rtma_aggregate_masked(self._h, _ptr(params), ctypes.c_int64(P), ctypes.c_int32(M), mask,
+                                             _ptr(global_out), ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_aggregate_masked")
 
     def sgd_aggregate(self, params, grads, lr, global_out=None, stream=None):
         M, P = params.shape

@@ -115,6 +115,7 @@ struct RowsArgs {
     const float* params;   // bias = params + part * P + bias_offset (bias_offset < 0: none)
     int64_t P, bias_offset;
     int relu;
+    int single;            // 1: operands rounded to bf16 (hi planes only, one MMA per product)
     const float* inv_deg;  // fp32 output only: columns >= scale_from are multiplied by inv_deg[row]
     int scale_from;        // and stored scale_shift columns further right; scale_from < 0: none
     int scale_shift;
@@ -161,11 +162,13 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
     const int n_tiles = a.Npad / BN;
     const int64_t total_tiles = a.row_tiles * n_tiles;
     const uint32_t b_tile_bytes = (uint32_t)BN * 128u;
-    const uint32_t stage_bytes = 2u * PLANE_TILE_BYTES + 2u * b_tile_bytes;
+    const bool single = a.single != 0;
+    const uint32_t np = single ? 1u : 2u;  // planes staged per operand
+    const uint32_t stage_bytes = np * (PLANE_TILE_BYTES + b_tile_bytes);
     auto a_hi = [&](int s) { return smem + (size_t)s * stage_bytes; };
     auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + PLANE_TILE_BYTES; };
-    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * PLANE_TILE_BYTES; };
-    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * PLANE_TILE_BYTES + b_tile_bytes; };
+    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + np * PLANE_TILE_BYTES; };
+    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + np * PLANE_TILE_BYTES + b_tile_bytes; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -208,16 +211,16 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                     const int s = (int)(it % stages);
                     ok = rows_wait(&pb.empty[s], (uint32_t)((it / stages) & 1) ^ 1u, &pb, a.error_word);
                     if (!ok) break;
-                    tc::mbar_arrive_expect_tx(&pb.full[s], 2u * PLANE_TILE_BYTES + 2u * b_tile_bytes);
+                    tc::mbar_arrive_expect_tx(&pb.full[s], stage_bytes);
                     if (kb < a.kb0) {
                         tc::tma_load_2d(a_hi(s), &a.mapA0h, &pb.full[s], kb * TC_BK, arow);
-                        tc::tma_load_2d(a_lo(s), &a.mapA0l, &pb.full[s], kb * TC_BK, arow);
+                        if (!single) tc::tma_load_2d(a_lo(s), &a.mapA0l, &pb.full[s], kb * TC_BK, arow);
                     } else {
                         tc::tma_load_2d(a_hi(s), &a.mapA1h, &pb.full[s], (kb - a.kb0) * TC_BK, arow);
-                        tc::tma_load_2d(a_lo(s), &a.mapA1l, &pb.full[s], (kb - a.kb0) * TC_BK, arow);
+                        if (!single) tc::tma_load_2d(a_lo(s), &a.mapA1l, &pb.full[s], (kb - a.kb0) * TC_BK, arow);
                     }
                     tc::tma_load_2d(b_hi(s), &a.mapBh, &pb.full[s], kb * TC_BK, brow);
-                    tc::tma_load_2d(b_lo(s), &a.mapBl, &pb.full[s], kb * TC_BK, brow);
+                    if (!single) tc::tma_load_2d(b_lo(s), &a.mapBl, &pb.full[s], kb * TC_BK, brow);
                 }
             }
         }
@@ -242,11 +245,15 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
 #pragma unroll
                     for (int ks = 0; ks < TC_BK / 16; ++ks) {
                         const uint32_t off = ks * 32;  // 16 bf16 = 32 bytes along K inside the swizzle row
-                        const uint64_t dah = tc::smem_desc_sw128(ah + off, 16, 1024), dal = tc::smem_desc_sw128(al + off, 16, 1024);
-                        const uint64_t dbh = tc::smem_desc_sw128(bh + off, 16, 1024), dbl = tc::smem_desc_sw128(bl + off, 16, 1024);
-                        tc::mma_bf16(d_tmem, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
-                        tc::mma_bf16(d_tmem, dah, dbl, idesc, 1u);
-                        tc::mma_bf16(d_tmem, dah, dbh, idesc, 1u);
+                        const uint64_t dah = tc::smem_desc_sw128(ah + off, 16, 1024), dbh = tc::smem_desc_sw128(bh + off, 16, 1024);
+                        if (single) {
+                            tc::mma_bf16(d_tmem, dah, dbh, idesc, (kb | ks) ? 1u : 0u);
+                        } else {
+                            const uint64_t dal = tc::smem_desc_sw128(al + off, 16, 1024), dbl = tc::smem_desc_sw128(bl + off, 16, 1024);
+                            tc::mma_bf16(d_tmem, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
+                            tc::mma_bf16(d_tmem, dah, dbl, idesc, 1u);
+                            tc::mma_bf16(d_tmem, dah, dbh, idesc, 1u);
+                        }
                     }
                     tc::mma_commit(&pb.empty[s]);
                 }
@@ -375,6 +382,7 @@ struct WgradArgs {
     int jt_per_src;   // 128-wide tiles over d_in, per source
     int n_atoms;      // 64-wide atoms over d_out (all column tiles together); a tile takes up to 4
     int tmem_cols, stages;
+    int single;       // 1: operands rounded to bf16 (hi planes only)
     float* partial;   // [slot][(2 d_in + 1) x d_out]
     int* error_word;
 };
@@ -415,11 +423,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     constexpr uint32_t ATOM_BYTES = TC_BK * 128u;  // one 64-wide column of 64 k-rows: 8 KB
     const uint32_t a_plane_bytes = 2u * ATOM_BYTES;
     const uint32_t b_plane_bytes = (uint32_t)NA * ATOM_BYTES;
-    const uint32_t stage_bytes = 2u * a_plane_bytes + 2u * b_plane_bytes;
+    const bool single = a.single != 0;
+    const uint32_t np = single ? 1u : 2u;  // planes staged per operand
+    const uint32_t stage_bytes = np * (a_plane_bytes + b_plane_bytes);
     auto a_hi = [&](int s) { return smem + (size_t)s * stage_bytes; };
     auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + a_plane_bytes; };
-    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * a_plane_bytes; };
-    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + 2 * a_plane_bytes + b_plane_bytes; };
+    auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + np * a_plane_bytes; };
+    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + np * a_plane_bytes + b_plane_bytes; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -451,14 +461,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % stages;
                 if (!wait_or_abort(&pb.empty[s], ((kb / stages) & 1) ^ 1, &pb, a.error_word)) break;
-                tc::mbar_arrive_expect_tx(&pb.full[s], 2u * a_plane_bytes + 2u * b_plane_bytes);
+                tc::mbar_arrive_expect_tx(&pb.full[s], stage_bytes);
                 for (int t = 0; t < 2; ++t) {
                     tc::tma_load_2d(a_hi(s) + t * ATOM_BYTES, mapAh, &pb.full[s], j0 + 64 * t, row + kb * TC_BK);
-                    tc::tma_load_2d(a_lo(s) + t * ATOM_BYTES, mapAl, &pb.full[s], j0 + 64 * t, row + kb * TC_BK);
+                    if (!single) tc::tma_load_2d(a_lo(s) + t * ATOM_BYTES, mapAl, &pb.full[s], j0 + 64 * t, row + kb * TC_BK);
                 }
                 for (int t = 0; t < NA; ++t) {
                     tc::tma_load_2d(b_hi(s) + t * ATOM_BYTES, &a.mapZh, &pb.full[s], cbase + 64 * t, row + kb * TC_BK);
-                    tc::tma_load_2d(b_lo(s) + t * ATOM_BYTES, &a.mapZl, &pb.full[s], cbase + 64 * t, row + kb * TC_BK);
+                    if (!single) tc::tma_load_2d(b_lo(s) + t * ATOM_BYTES, &a.mapZl, &pb.full[s], cbase + 64 * t, row + kb * TC_BK);
                 }
             }
         }
@@ -474,11 +484,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 #pragma unroll
                 for (int ks = 0; ks < TC_BK / 16; ++ks) {
                     const uint32_t off = ks * 2048;  // 16 k-rows of 128 bytes
-                    const uint64_t dah = tc::smem_desc_sw128(ah + off, ATOM_BYTES, 1024), dal = tc::smem_desc_sw128(al + off, ATOM_BYTES, 1024);
-                    const uint64_t dbh = tc::smem_desc_sw128(bh + off, ATOM_BYTES, 1024), dbl = tc::smem_desc_sw128(bl + off, ATOM_BYTES, 1024);
-                    tc::mma_bf16(tmem_base, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
-                    tc::mma_bf16(tmem_base, dah, dbl, idesc, 1u);
-                    tc::mma_bf16(tmem_base, dah, dbh, idesc, 1u);
+                    const uint64_t dah = tc::smem_desc_sw128(ah + off, ATOM_BYTES, 1024), dbh = tc::smem_desc_sw128(bh + off, ATOM_BYTES, 1024);
+                    if (single) {
+                        tc::mma_bf16(tmem_base, dah, dbh, idesc, (kb | ks) ? 1u : 0u);
+                    } else {
+                        const uint64_t dal = tc::smem_desc_sw128(al + off, ATOM_BYTES, 1024), dbl = tc::smem_desc_sw128(bl + off, ATOM_BYTES, 1024);
+                        tc::mma_bf16(tmem_base, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
+                        tc::mma_bf16(tmem_base, dah, dbl, idesc, 1u);
+                        tc::mma_bf16(tmem_base, dah, dbh, idesc, 1u);
+                    }
                 }
                 tc::mma_commit(&pb.empty[s]);
             }
@@ -511,7 +525,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                         for (int i = 0; i < 4; ++i) {
                             Pack8 p;
                             p.zero();
-                            p.add_planes(bh[tw + 128 * i], bl[tw + 128 * i]);
+                            p.add_planes(bh[tw + 128 * i], single ? make_uint4(0u, 0u, 0u, 0u) : bl[tw + 128 * i]);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) colsum[t][e] += p.v[e];
                         }
@@ -678,7 +692,7 @@ static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t 
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, ROWS_SMEM_MAX));
         configured = true;
     }
-    const size_t stage_bytes = 2 * (size_t)PLANE_TILE_BYTES + 2 * (size_t)a.BN * 128;
+    const size_t stage_bytes = (a.single ? 1 : 2) * ((size_t)PLANE_TILE_BYTES + (size_t)a.BN * 128);
     a.stages = std::max(1, std::min<int>(MAX_STAGES, (int)(ROWS_RING_BUDGET / stage_bytes)));
     a.tmem_cols = (int)tmem_columns_for(a.BN);
     a.error_word = ctx->error_word;
@@ -699,9 +713,11 @@ static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t 
 
 int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                           const float* params, Planes H, Planes N, const __nv_bfloat16* Bf_hi,
-                          const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, cudaStream_t s) {
+                          const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, bool single,
+                          cudaStream_t s) {
     RowsArgs a{};
     a.g = g;
+    a.single = single ? 1 : 0;
     if (!plane_maps(&a.mapA0h, &a.mapA0l, H, rows_total, ls.d_in, TC_BK, TC_BM) ||
         !plane_maps(&a.mapA1h, &a.mapA1l, N, rows_total, ls.d_in, TC_BK, TC_BM) ||
         !make_tensor_map_bf16(&a.mapBh, Bf_hi, (uint64_t)g.num * p.Npad_f, p.Kf, p.Kf, TC_BK, p.BN_f) ||
@@ -726,9 +742,10 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
 
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                         Planes dZ, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, const float* inv_deg, Mat ST,
-                        cudaStream_t s) {
+                        bool single, cudaStream_t s) {
     RowsArgs a{};
     a.g = g;
+    a.single = single ? 1 : 0;
     if (!plane_maps(&a.mapA0h, &a.mapA0l, dZ, rows_total, ls.d_out, TC_BK, TC_BM) ||
         !make_tensor_map_bf16(&a.mapBh, Bd_hi, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d) ||
         !make_tensor_map_bf16(&a.mapBl, Bd_lo, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d))
@@ -754,7 +771,7 @@ int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const 
 }
 
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
-                        Planes H, Planes N, Planes dZ, float* partial, cudaStream_t s) {
+                        Planes H, Planes N, Planes dZ, float* partial, bool single, cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
         RTMA_TRY(set_smem_limit(ctx, reinterpret_cast<const void*>(tc_wgrad_kernel)));
@@ -776,7 +793,8 @@ int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, 
     a.n_atoms = (int)ceil_div(ls.d_out, 64);
     const int tile_atoms = a.n_atoms < 4 ? a.n_atoms : 4;
     a.tmem_cols = (int)tmem_columns_for(64 * tile_atoms);
-    const size_t stage_bytes = (2 * (size_t)2 + 2 * (size_t)tile_atoms) * TC_BK * 128;
+    a.single = single ? 1 : 0;
+    const size_t stage_bytes = (single ? 1 : 2) * ((size_t)2 + (size_t)tile_atoms) * TC_BK * 128;
     a.stages = stages_for(stage_bytes, MAX_STAGES);
     a.partial = partial;
     a.error_word = ctx->error_word;

@@ -34,17 +34,19 @@ copy_rows_kernel(const float* __restrict__ src, const int64_t ld_src, float* __r
     }
 }
 
-// out_j = (1/M) sum_i (params[i][j] - lr * grads[i][j]); written to every replica.
+// out_j = (1/|A|) sum_{i in A} (params[i][j] - lr * grads[i][j]), A = the replicas whose bit is
+// set in `active`; written to every replica, the inactive ones included.
 template <int VEC, bool WITH_GRADS>
 __global__ void __launch_bounds__(256)
 aggregate_kernel(float* __restrict__ params, const float* __restrict__ grads, const float lr, const int64_t P,
-                 const int M, float* __restrict__ global_out) {
-    const float inv_m = 1.0f / (float)M;
+                 const int M, const uint64_t active, float* __restrict__ global_out) {
+    const float inv_m = 1.0f / (float)__popcll(active);
     const int64_t packs = P / VEC;
     for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < packs; j += (int64_t)gridDim.x * 256) {
         if (VEC == 4) {
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int i = 0; i < M; ++i) {
+                if (!((active >> i) & 1)) continue;
                 float4 w = *reinterpret_cast<const float4*>(params + (int64_t)i * P + j * 4);
                 if (WITH_GRADS) {
                     const float4 gr = __ldg(reinterpret_cast<const float4*>(grads + (int64_t)i * P + j * 4));
@@ -58,6 +60,7 @@ aggregate_kernel(float* __restrict__ params, const float* __restrict__ grads, co
         } else {
             float acc = 0.f;
             for (int i = 0; i < M; ++i) {
+                if (!((active >> i) & 1)) continue;
                 float w = params[(int64_t)i * P + j];
                 if (WITH_GRADS) w -= lr * __ldg(grads + (int64_t)i * P + j);
                 acc += w;
@@ -81,10 +84,14 @@ int sm_count(int device) {
 }
 
 int32_t aggregate_impl(rtma_ctx* ctx, float* params, const float* grads, float lr, int64_t P, int32_t M,
-                       float* global_out, void* stream_) {
+                       const uint8_t* active_host, float* global_out, void* stream_) {
     if (!ctx) return RTMA_ERR_INVALID_ARG;
     if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
     if (P < 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "P=%lld negative", (long long)P);
+    uint64_t active = 0;
+    for (int i = 0; i < M; ++i)
+        if (!active_host || active_host[i]) active |= uint64_t(1) << i;
+    if (active == 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "aggregate: no active trainer among %d", M);
     if (P == 0) return RTMA_OK;
     if (!params) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "aggregate: null params");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -95,11 +102,11 @@ int32_t aggregate_impl(rtma_ctx* ctx, float* params, const float* grads, float l
     const int64_t packs = vec ? P / 4 : P;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(packs, 256), (int64_t)sm_count(ctx->device) * 8);
     if (vec) {
-        if (grads) { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<4, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, global_out); }
-        else { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<4, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, global_out); }
+        if (grads) { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<4, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, active, global_out); }
+        else { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<4, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, active, global_out); }
     } else {
-        if (grads) { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<1, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, global_out); }
-        else { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<1, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, global_out); }
+        if (grads) { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<1, true><<<grid, 256, 0, stream>>>(params, grads, lr, P, M, active, global_out); }
+        else { KernelScope ks(ctx, KC_AGGREGATE, stream); aggregate_kernel<1, false><<<grid, 256, 0, stream>>>(params, nullptr, 0.f, P, M, active, global_out); }
     }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
@@ -127,11 +134,17 @@ int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float*
 }
 
 extern "C" int32_t rtma_aggregate(rtma_ctx* ctx, float* params, int64_t P, int32_t M, float* global_out, void* stream) {
-    return aggregate_impl(ctx, params, nullptr, 0.f, P, M, global_out, stream);
+    return aggregate_impl(ctx, params, nullptr, 0.f, P, M, nullptr, global_out, stream);
+}
+
+extern "C" int32_t rtma_aggregate_masked(rtma_ctx* ctx, float* params, int64_t P, int32_t M, const uint8_t* active,
+                                         float* global_out, void* stream) {
+    if (ctx && !active) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_aggregate_masked: null mask");
+    return aggregate_impl(ctx, params, nullptr, 0.f, P, M, active, global_out, stream);
 }
 
 extern "C" int32_t rtma_sgd_aggregate(rtma_ctx* ctx, float* params, const float* grads, float lr, int64_t P, int32_t M,
                                       float* global_out, void* stream) {
     if (!grads) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_sgd_aggregate: null grads");
-    return aggregate_impl(ctx, params, grads, lr, P, M, global_out, stream);
+    return aggregate_impl(ctx, params, grads, lr, P, M, nullptr, global_out, stream);
 }

@@ -75,6 +75,18 @@ int splits_for(int64_t n_p, int parts_in_flight) {
     return (int)std::min<int64_t>(64, std::min(want, by_rows));
 }
 
+int plan_splits(const GroupDesc& g, SplitPlan* sp) {
+    int slots = 0;
+    for (int k = 0; k < g.num; ++k) {
+        sp->split_begin[k] = slots;
+        const int nsplit = splits_for(g.rows[k], g.num);
+        sp->rows_per_split[k] = (int32_t)std::max<int64_t>(GROUP_ROW_ALIGN, aligned_rows(ceil_div(g.rows[k], nsplit)));
+        slots += (int)std::max<int64_t>(1, ceil_div(g.rows[k], sp->rows_per_split[k]));
+    }
+    sp->split_begin[g.num] = slots;
+    return slots;
+}
+
 size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
     const size_t rows = (size_t)aligned_rows(n_p);
     const size_t matrices = 8 * m.L + 12;  // every matrix start is rounded up to 256 bytes
@@ -91,18 +103,24 @@ extern "C" int64_t rtma_param_count(const rtma_model_desc* md) {
     return p;
 }
 
-extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,
-                                    const int64_t* part_offsets, const int64_t* edge_offsets,
-                                    const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
-                                    const float* Xp, const int32_t* yp, float* params, int32_t K, float* loss_out,
-                                    const rtma_taps* taps, void* const* streams) {
+extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,
+                                        const int64_t* part_offsets, const int64_t* edge_offsets,
+                                        const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                                        const float* Xp, const int32_t* yp, float* params, const int32_t* steps,
+                                        int32_t loss_stride, float* loss_out, const rtma_taps* taps,
+                                        void* const* streams) {
     if (!ctx) return RTMA_ERR_INVALID_ARG;
     Model m;
     RTMA_TRY(parse_model(ctx, md, &m));
     if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
-    if (K < 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "K=%d negative", K);
-    if (!part_offsets || !edge_offsets || !rowptr_out || !params || !streams)
+    if (!part_offsets || !edge_offsets || !rowptr_out || !params || !streams || !steps)
         return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_local_steps: null pointer");
+    int32_t K = 0;
+    for (int p = 0; p < M; ++p) {
+        if (steps[p] < 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "steps[%d]=%d negative", p, steps[p]);
+        K = std::max(K, steps[p]);
+    }
+    if (loss_out && loss_stride < K) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "loss_stride=%d < largest step count %d", loss_stride, K);
     if (!tc_available())
         return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "the driver does not provide cuTensorMapEncodeTiled");
     if (symmetric != 1)
@@ -116,11 +134,13 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
             return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "part %d has inconsistent offsets", p);
     if (K == 0) return RTMA_OK;
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    const bool single_pass = md->gemm_dtype == 1;
 
     // Trainers grouped by stream, in order of first appearance.
     std::vector<cudaStream_t> group_stream;
     std::vector<std::vector<int>> group_parts;
     for (int p = 0; p < M; ++p) {
+        if (steps[p] == 0) continue;  // a trainer that does not run takes no scratch and no launches
         cudaStream_t s = static_cast<cudaStream_t>(streams[p]);
         size_t gi = 0;
         while (gi < group_stream.size() && group_stream[gi] != s) ++gi;
@@ -187,14 +207,9 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                 bytes += b;
                 ++at;
             }
-            int slots = 0;
-            for (int k = 0; k < g.num; ++k) {
-                sp.split_begin[k] = slots;
-                const int nsplit = splits_for(g.rows[k], g.num);
-                sp.rows_per_split[k] = (int32_t)std::max<int64_t>(GROUP_ROW_ALIGN, aligned_rows(ceil_div(g.rows[k], nsplit)));
-                slots += (int)std::max<int64_t>(1, ceil_div(g.rows[k], sp.rows_per_split[k]));
-            }
-            sp.split_begin[g.num] = slots;
+            const int slots = plan_splits(g, &sp);
+            int wave_steps = 0;
+            for (int k = 0; k < g.num; ++k) wave_steps = std::max(wave_steps, steps[g.part[k]]);
 
             // ---- carve the share ----
             ArenaCursor cur(ctx->arena + gi * share);
@@ -240,8 +255,36 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
             RTMA_TRY(launch_to_planes(ctx, g, Xp, m.dims[0], Hl[0], s));
             const Planes no_planes{nullptr, nullptr, 0};
             const Mat no_mat{nullptr, 0};
-            for (int step = 0; step < K; ++step) {
+            const GroupDesc wave = g;   // all parts of the wave, with their scratch rows
+            const SplitPlan wave_sp = sp;
+            for (int step = 0; step < wave_steps; ++step) {
                 const bool tap = taps && taps->step == step;
+                // trainers that have finished their steps drop out (time-based aggregation lets
+                // trainers reach the aggregation point with different step counts)
+                bool all_run = true;
+                for (int k = 0; k < wave.num; ++k) all_run = all_run && steps[wave.part[k]] > step;
+                if (all_run) {
+                    g = wave;
+                    sp = wave_sp;
+                } else {
+                    g.num = 0;
+                    int slot = 0;
+                    for (int k = 0; k < wave.num; ++k) {
+                        if (steps[wave.part[k]] <= step) continue;
+                        const int j = g.num++;
+                        // same chunking as in the whole wave: the slots still fit `partial`, and a
+                        // trainer's gradient sums do not depend on who else is still running
+                        sp.split_begin[j] = slot;
+                        sp.rows_per_split[j] = wave_sp.rows_per_split[k];
+                        slot += wave_sp.split_begin[k + 1] - wave_sp.split_begin[k];
+                        sp.split_begin[j + 1] = slot;
+                        g.part[j] = wave.part[k];
+                        g.rows[j] = wave.rows[k];
+                        g.row_abs[j] = wave.row_abs[k];
+                        g.row_ws[j] = wave.row_ws[k];
+                        g.edge_abs[j] = wave.edge_abs[k];
+                    }
+                }
                 // ---- forward ----
                 for (int l = 0; l < m.L; ++l)
                     RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
@@ -249,7 +292,7 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                     RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], ticket, s));
                     const bool last = l == m.L - 1;
                     RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
-                                               last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, s));
+                                               last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, single_pass, s));
                 }
                 if (tap && taps->acts) {
                     size_t rec = 0;  // floats per row in the record
@@ -269,12 +312,12 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
                     }
                 }
                 // ---- loss; dZ of the last layer and its tile column sums ----
-                RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, K, step, s));
+                RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, loss_stride, step, s));
                 // ---- backward + SGD ----
                 for (int l = m.L - 1; l >= 0; --l) {
                     const Planes dZ = l == m.L - 1 ? dZlast : Hl[l + 1];
-                    RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, s));
-                    if (l > 0) RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, s));
+                    RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, single_pass, s));
+                    if (l > 0) RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, single_pass, s));
                     RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
                     if (l > 0)  // dZ^{l-1} overwrites H^l, whose sign is the ReLU gate
                         RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, ST, Hl[l], m.dims[l], ticket, s));
@@ -283,4 +326,18 @@ extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, in
         }
     }
     return RTMA_OK;
+}
+
+extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,
+                                    const int64_t* part_offsets, const int64_t* edge_offsets,
+                                    const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                                    const float* Xp, const int32_t* yp, float* params, int32_t K, float* loss_out,
+                                    const rtma_taps* taps, void* const* streams) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    if (K < 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "K=%d negative", K);
+    if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
+    int32_t steps[RTMA_MAX_PARTS];
+    for (int p = 0; p < M; ++p) steps[p] = K;
+    return rtma_local_steps_var(ctx, md, M, part_offsets, edge_offsets, rowptr_out, col_out, symmetric, Xp, yp, params,
+                                steps, K, loss_out, taps, streams);
 }

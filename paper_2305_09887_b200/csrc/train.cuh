@@ -97,6 +97,8 @@ int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float*
                          int width, cudaStream_t s);
 
 // ---- gemm_tc.cu (layer products on the tensor cores) --------------------------------------
+// `single` = operands rounded to bf16: only the hi planes are loaded and each product is one MMA
+// instead of three.
 struct TcLayerPlan {
     int Kf, BN_f, Npad_f;  // forward: padded K (2 x 64-blocks over d_in), column tile, padded N
     int Kd, BN_d, Npad_d;  // dgrad: padded K over d_out, column tile, padded N over 2 d_in
@@ -111,11 +113,12 @@ int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, 
 // out = act([H | N] [Ws; Wn] + b): split planes when out_planes.hi != NULL, else fp32 out_f32.
 int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                           const float* params, Planes H, Planes N, const __nv_bfloat16* Bf_hi,
-                          const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, cudaStream_t s);
+                          const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, bool single,
+                          cudaStream_t s);
 // ST[:, 0:d_in] = dZ Ws^T ;  ST[:, d_in:2 d_in] = inv_deg * (dZ Wn^T)
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                         Planes dZ, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, const float* inv_deg, Mat ST,
-                        cudaStream_t s);
+                        bool single, cudaStream_t s);
 // partial[slot][(2 d_in + 1) x d_out] = [H | N | 1]^T dZ over one chunk of rows.
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
-                        Planes H, Planes N, Planes dZ, float* partial, cudaStream_t s);
+                        Planes H, Planes N, Planes dZ, float* partial, bool single, cudaStream_t s);
