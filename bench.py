@@ -1,16 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the whole RandomTMA hot path on one B200 (or N independent replicas).
 
-One step = one pass of the whole path over the Medium workload (Chung-Lu power-law graph,
-200k nodes, ~5M directed entries, 128-d features, 47 classes, M=8 trainers, 128-256-256-47
-GraphSAGE-mean, 20 local steps per round, 5 aggregation rounds): broadcast of the initial
-weights, partition, induced CSR (count + fill), row gather, then 5 x (20 local steps on all
-8 parts + aggregation).
+One step = one pass of the whole path over the workload: broadcast of the initial weights,
+partition, induced CSR (count + fill), row gather, then R x (K local steps on all M parts +
+aggregation).  The default workload is Medium (Chung-Lu power-law graph, 200k nodes, ~5M
+directed entries, 128-d features, 47 classes, M=8 trainers, 128-256-256-47 GraphSAGE-mean,
+20 local steps per round, 5 aggregation rounds).  --workload selects the other shapes:
+supertma (planted communities, super-node assignment, M=16), sweep (the same graph at width
+512 with bf16 GEMM operands; --M and --assign pick the point of the sweep) and large
+(--scale shrinks it; the full size needs ~60 GB of host memory to generate).
 
 Metric: aggregated edges/s = (sum over parts of kept entries) x (SpMM passes per local step:
 L forward + L-1 backward) x (local steps) / time.  Local trainer-steps/s is reported beside it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                    [--workload medium|supertma|sweep|large] [--scale S] [--M M] [--assign node|super]
 
 Prints one JSON line (rank 0).
 """
@@ -148,7 +152,8 @@ def cpu_sample(w, local_steps=1):
     g = w.graph
     L = len(w.dims) - 1
     t0 = time.perf_counter()
-    part_id, part_offsets, perm, local_id = oracle.partition(g.n, None, w.partition_seed, w.M)
+    part_id, part_offsets, perm, local_id = oracle.partition(g.n, g.group_id if w.use_groups else None,
+                                                             w.partition_seed, w.M)
     rowptr_out, col_out, edge_offsets, kept, cut = oracle.induced_csr(
         g.rowptr, g.col, w.M, part_id, part_offsets, perm, local_id)
     Xp = oracle.gather_rows(w.X, perm)
@@ -193,6 +198,19 @@ def run_reference(args, w):
 
 
 # ---------------------------------------------------------------------------------------
+def make_workload(args):
+    from paper_2305_09887_b200 import inputs
+    s = args.scale
+    if args.workload == "medium":
+        return inputs.medium(1.0 if s is None else s)
+    if args.workload == "supertma":
+        return inputs.supertma(1.0 if s is None else s, M=args.M or 16)
+    if args.workload == "sweep":
+        return inputs.supertma(1.0 if s is None else s, width=512, M=args.M or 16,
+                               use_groups=args.assign == "super", gemm_dtype=1)
+    return inputs.large(1.0 if s is None else s)
+
+
 def max_over_ranks(seconds: float, dist_mod=None, device=None) -> float:
     """Largest value over all ranks (the slowest rank sets the job's time)."""
     if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
@@ -210,15 +228,18 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="medium", choices=["medium", "supertma", "sweep", "large"])
+    ap.add_argument("--scale", type=float, default=None, help="shrink (or grow) the workload's graph")
+    ap.add_argument("--M", type=int, default=None, help="trainers (supertma / sweep)")
+    ap.add_argument("--assign", default="super", choices=["node", "super"], help="sweep: assignment scheme")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
-    from paper_2305_09887_b200 import inputs
     if args.impl == "reference":
         if rank == 0:
-            run_reference(args, inputs.medium())
+            run_reference(args, make_workload(args))
         return
 
     import torch
@@ -232,7 +253,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
-    w = inputs.medium()
+    w = make_workload(args)
     g = w.graph
     L = len(w.dims) - 1
     ctx = binding.Context(local_rank)
@@ -241,6 +262,7 @@ def main():
     d_X = torch.from_numpy(w.X).to(device)
     d_y = torch.from_numpy(w.y).to(device)
     d_params0 = torch.from_numpy(w.params0).to(device)
+    d_gid = torch.from_numpy(g.group_id).to(device) if w.use_groups else None
     P = w.params0.size
     params = torch.empty(w.M, P, dtype=torch.float32, device=device)
     loss = torch.zeros(w.R, w.M, w.K, dtype=torch.float32, device=device)
@@ -249,7 +271,7 @@ def main():
 
     def step():
         params.copy_(d_params0.expand(w.M, P))                      # W_global[0] broadcast to the trainers
-        part_id, part_offsets, perm, local_id = ctx.partition(g.n, None, w.partition_seed, w.M)
+        part_id, part_offsets, perm, local_id = ctx.partition(g.n, d_gid, w.partition_seed, w.M)
         rowptr_out, col_out, edge_offsets, kept_cut, edge_host = ctx.build_induced_csr(
             d_rowptr, d_col, w.M, part_id, part_offsets, perm, local_id)
         Xp = ctx.gather_rows(d_X, perm)
@@ -257,7 +279,7 @@ def main():
         part_host = part_offsets.cpu().tolist()
         for r in range(w.R):
             ctx.local_steps(w.dims, w.lr, w.M, part_host, edge_host, rowptr_out, col_out, Xp, yp, params, w.K,
-                            loss_out=loss[r])
+                            loss_out=loss[r], gemm_dtype=w.gemm_dtype)
             ctx.aggregate(params)
         state.update(part_host=part_host, edge_host=edge_host)
 
@@ -308,7 +330,7 @@ def main():
     # A layer product is three bf16 MMAs (hi*hi + lo*hi + hi*lo): the tensor pipe executes 3x the
     # algorithmic flops.  Its roofline is whichever is slower for the algorithmic work: the operand
     # bytes at the HBM peak or 3x the flops at the bf16 peak (sustained figure: timed inside a long step).
-    MMAS_PER_PRODUCT = 3
+    MMAS_PER_PRODUCT = 1 if w.gemm_dtype == 1 else 3
     if top in work:
         bound, abytes, aflops = work[top]
         seconds = top_ms / 1e3
@@ -322,7 +344,7 @@ def main():
         else:
             roof = {"bound": "tensor", "achieved": aflops * args.steps / seconds / 1e12,
                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "note": "algorithmic flops; the tensor pipe executes 3 bf16 MMAs per product"}
+                    "note": f"algorithmic flops; the tensor pipe executes {MMAS_PER_PRODUCT} bf16 MMA(s) per product"}
     else:
         roof = {"bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof.update({"frac": (roof["achieved"] / roof["peak"]) if roof["achieved"] else None, "traffic": None,
@@ -347,7 +369,9 @@ def main():
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
     h_rowptr, h_col, h_X, h_y, h_p0 = pin(g.rowptr), pin(g.col), pin(w.X), pin(w.y), pin(w.params0)
     e2e_steps = max(1, min(args.steps, 3))
-    ctx.train_host(h_rowptr, h_col, h_X, h_y, w.dims, w.M, w.K, w.R, w.lr, w.partition_seed, h_p0)  # warm-up
+    h_gid = pin(g.group_id) if w.use_groups else None
+    host_kw = dict(group_id=h_gid, gemm_dtype=w.gemm_dtype)
+    ctx.train_host(h_rowptr, h_col, h_X, h_y, w.dims, w.M, w.K, w.R, w.lr, w.partition_seed, h_p0, **host_kw)  # warm-up
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if world > 1:
@@ -355,11 +379,11 @@ def main():
     e0.record()
     for _ in range(e2e_steps):
         out_params, out_losses, _, _ = ctx.train_host(h_rowptr, h_col, h_X, h_y, w.dims, w.M, w.K, w.R, w.lr,
-                                                      w.partition_seed, h_p0)
+                                                      w.partition_seed, h_p0, **host_kw)
     e1.record()
     torch.cuda.synchronize()
     e2e_s = max_over_ranks(e0.elapsed_time(e1) / 1e3, dist if world > 1 else None, device)
-    h2d = h_rowptr.nbytes + h_col.nbytes + h_X.nbytes + h_y.nbytes + w.M * h_p0.nbytes
+    h2d = h_rowptr.nbytes + h_col.nbytes + h_X.nbytes + h_y.nbytes + w.M * h_p0.nbytes + (h_gid.nbytes if w.use_groups else 0)
     d2h = out_params.nbytes + out_losses.nbytes + 16 + 2 * 8 * (w.M + 1)
     e2e_value = world * e2e_steps * units_per_step / e2e_s
 
@@ -371,11 +395,14 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * elapsed_s / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16x3-split products, f32 accumulate and elementwise", "data": "synthetic",
+        "dtype": ("bf16 products, f32 accumulate and elementwise" if w.gemm_dtype == 1 else
+                  "bf16x3-split products, f32 accumulate and elementwise"), "data": "synthetic",
         "config": {"workload": w.name, "nodes": g.n, "entries": g.num_entries, "kept_entries": int(kept), "M": w.M,
                    "dims": list(w.dims), "K": w.K, "R": w.R, "spmm_passes_per_local_step": passes,
-                   "parallelism": "replicas only" if world > 1 else "single GPU, 8 trainers batched on one stream",
-                   "l2": "256 MB written between timed steps; per-step working set 1.5 GB > L2"},
+                   "assignment": "super-node" if w.use_groups else "node",
+                   "kept_fraction": kept / g.num_entries,
+                   "parallelism": "replicas only" if world > 1 else f"single GPU, {w.M} trainers batched on one stream",
+                   "l2": "256 MB written between timed steps"},
         "trainer_steps_per_s": world * args.steps * trainer_steps / elapsed_s,
         "loss_first_last": [first_loss, final_loss],
         "roofline": roof,

@@ -47,6 +47,17 @@ class Workload:
     gemm_dtype: int = 0  # 0: fp32-accurate GEMMs, 1: bf16 inputs / fp32 accumulate
 
 
+def _sorted_unique(key: np.ndarray) -> np.ndarray:
+    """np.unique by an in-place sort (several times faster on tens of millions of keys)."""
+    key.sort()
+    if key.size == 0:
+        return key
+    keep = np.empty(key.size, dtype=bool)
+    keep[0] = True
+    np.not_equal(key[1:], key[:-1], out=keep[1:])
+    return key[keep]
+
+
 def _csr_from_pairs(n: int, u: np.ndarray, v: np.ndarray, wide_rowptr: bool) -> Graph:
     """Symmetrise, drop loops and duplicates, sort, and build CSR."""
     keep = u != v
@@ -54,7 +65,7 @@ def _csr_from_pairs(n: int, u: np.ndarray, v: np.ndarray, wide_rowptr: bool) -> 
     v = v[keep].astype(np.int64)
     key = np.concatenate([u * n + v, v * n + u])
     del u, v
-    key = np.unique(key)  # sorted by (row, col), duplicates removed
+    key = _sorted_unique(key)  # sorted by (row, col), duplicates removed
     rows = key // n
     col = (key - rows * n).astype(np.int32)
     del key

@@ -3,7 +3,11 @@ import numpy as np
 import torch
 
 import oracle
-from paper_2305_09887_b200 import binding
+from paper_2305_09887_b200 import binding, inputs
+
+# relative = max|a-b| / max|b| per tensor
+TOL_ACT, TOL_GRAD, TOL_PARAM = 1e-4, 1e-3, 1e-3
+TOL_BF16 = 5e-3
 
 _ctx = None
 
@@ -68,3 +72,124 @@ def assert_preprocess_equal(got, want):
     assert kc == [want["kept"], want["cut"]]
     assert np.array_equal(got["Xp"].cpu().numpy(), want["Xp"])
     assert np.array_equal(got["yp"].cpu().numpy(), want["yp"])
+
+
+def oracle_part(w, pre, p):
+    """(rowptr, col, X, y) of part p from the oracle's preprocessing."""
+    rp, cp = oracle.part_graph(pre["rowptr_out"], pre["col_out"], pre["part_offsets"], pre["edge_offsets"], p)
+    lo, hi = int(pre["part_offsets"][p]), int(pre["part_offsets"][p + 1])
+    return rp, cp, pre["Xp"][lo:hi].astype(np.float64), pre["yp"][lo:hi]
+
+
+def oracle_parts(w, pre):
+    return [oracle_part(w, pre, p) for p in range(pre["M"])]
+
+
+def tols(gemm_dtype):
+    """(activations, gradients, parameters, loss, |z| below which a ReLU branch is ambiguous as a
+    fraction of max|z|, flips allowed per part as a fraction of the hidden units)."""
+    if gemm_dtype == 1:   # operands rounded to bf16 (2^-9 each), fp32 accumulation
+        return TOL_BF16, TOL_BF16, TOL_BF16, TOL_BF16, 4e-3, 0.01
+    # fp32-accurate products: the kernel's pre-activations carry about 1e-6 of relative error, so
+    # of the order of 1e-6 of all units straddle the kink differently from the fp64 oracle
+    return TOL_ACT, TOL_GRAD, TOL_PARAM, 1e-5, 2e-5, 1e-5
+
+
+def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None):
+    """Partition + induced CSR against the oracle (bit-exact), then step 0 of all M trainers
+    batched as one call: every recorded intermediate, the loss, the gradient and the updated
+    parameters of every part (or of the parts in only_parts) against the oracle."""
+    tol_act, tol_grad, tol_param, tol_loss, amb, flip_frac = tols(gemm_dtype)
+    c = ctx()
+    got = gpu_preprocess(w, M=M)
+    want = oracle_preprocess(w, M=M)
+    assert_preprocess_equal(got, want)
+    M = got["M"]
+    dims, n = w.dims, w.graph.n
+    P = inputs.param_count(dims)
+    rec = sum(dims[l] + dims[l + 1] for l in range(len(dims) - 1))
+    params = dev(np.tile(w.params0, (M, 1)))
+    acts = torch.zeros(n * rec, dtype=torch.float32, device="cuda")
+    grads = torch.zeros(M, P, dtype=torch.float32, device="cuda")
+    loss = torch.zeros(M, 1, dtype=torch.float32, device="cuda")
+    c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
+                  got["Xp"], got["yp"], params, 1, loss_out=loss, taps=(acts, grads, 0), gemm_dtype=gemm_dtype,
+                  streams=streams)
+    torch.cuda.synchronize()
+    grads, loss, params1 = grads.cpu().numpy(), loss.cpu().numpy(), params.cpu().numpy()
+    p0 = w.params0.astype(np.float64)
+    for p in range(M) if only_parts is None else only_parts:
+        rp, cp, X, y = oracle_part(w, want, p)
+        n_p = rp.size - 1
+        o_loss, o_grads, o_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True, want_preact=True)
+        layout, total = oracle.acts_layout(dims, n_p)
+        base = int(want["part_offsets"][p]) * rec
+        gpu_acts = {}
+        for name, off, r, wd in layout:
+            a = acts[base + off: base + off + r * wd].cpu().numpy().reshape(r, wd)
+            gpu_acts[name] = a
+            assert rel_err(a, o_acts[name]) <= tol_act, (p, name)
+        # ReLU has no derivative at 0: a hidden unit whose pre-activation is within the rounding
+        # error of an fp32 forward pass of 0 may legitimately take either branch, and the branch
+        # decides a finite part of the gradient.  For such units only (judged on the oracle's own
+        # pre-activations) the oracle is re-evaluated on the branch the kernel took; any other
+        # unit on the wrong branch fails the activation check above.
+        gates, flipped, units = [], 0, 0
+        for l in range(len(dims) - 2):
+            Z = o_acts[f"Z{l + 1}"]
+            ambiguous = np.abs(Z) < amb * max(1.0, np.abs(Z).max(initial=0.0))
+            units += Z.size
+            differ = ambiguous & ((gpu_acts[f"H{l + 1}"] > 0) != (Z > 0))
+            flipped += int(differ.sum())
+            g8 = np.full(Z.shape, -1, dtype=np.int8)
+            g8[differ] = (gpu_acts[f"H{l + 1}"] > 0)[differ]
+            gates.append(g8)
+        assert flipped <= 8 + flip_frac * units
+        if flipped:
+            o_loss, o_grads, _ = oracle.forward_backward(dims, rp, cp, X, y, p0, gates=gates)
+        if n_p:
+            assert abs(loss[p, 0] - o_loss) <= tol_loss * max(1.0, abs(o_loss)), p
+        # gradients: per parameter tensor
+        off = 0
+        for l in range(len(dims) - 1):
+            for nm, size in (("Ws", dims[l] * dims[l + 1]), ("Wn", dims[l] * dims[l + 1]), ("b", dims[l + 1])):
+                gg, og = grads[p, off:off + size], o_grads[off:off + size]
+                if np.abs(og).max() > 0:
+                    assert rel_err(gg, og) <= tol_grad, (p, l, nm)
+                else:
+                    assert np.abs(gg).max() == 0
+                off += size
+        assert rel_err(params1[p], p0 - w.lr * o_grads) <= tol_param
+    return got, want
+
+
+def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_parts=None):
+    """K local steps of all M trainers and the aggregation.  Parameters and losses of every part
+    (or of the parts in only_parts) against the oracle; the average against the oracle's, or,
+    when only some parts were recomputed, against the fp64 mean of the kernel's own replicas."""
+    tol_param = tols(gemm_dtype)[2]
+    tol_loss = 10 * tols(gemm_dtype)[3]
+    c = ctx()
+    M, dims = got["M"], w.dims
+    params = dev(np.tile(w.params0, (M, 1)))
+    loss = torch.zeros(M, K, dtype=torch.float32, device="cuda")
+    c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
+                  got["Xp"], got["yp"], params, K, loss_out=loss, gemm_dtype=gemm_dtype, streams=streams)
+    torch.cuda.synchronize()
+    after = params.cpu().numpy().copy()
+    glob = torch.empty(params.shape[1], dtype=torch.float32, device="cuda")
+    c.aggregate(params, glob)
+    torch.cuda.synchronize()
+    o_params = after.astype(np.float64)
+    for p in range(M) if only_parts is None else only_parts:
+        rp, cp, X, y = oracle_part(w, want, p)
+        o_params[p], o_loss = oracle.local_steps(dims, w.lr, rp, cp, X, y, w.params0.astype(np.float64), K)
+        assert rel_err(after[p], o_params[p]) <= tol_param, p
+        if rp.size > 1:
+            assert np.abs(loss[p].cpu().numpy() - o_loss).max() <= tol_loss * max(1.0, np.abs(o_loss).max())
+    o_avg, o_glob = oracle.average(o_params)
+    assert rel_err(glob.cpu().numpy(), o_glob) <= tol_param
+    pa = params.cpu().numpy()
+    for p in range(M):
+        assert np.array_equal(pa[p], glob.cpu().numpy())     # every local copy overwritten
+    return after

@@ -14,8 +14,7 @@ from paper_2305_09887_b200 import inputs
 
 pytestmark = pytest.mark.gpu
 
-TOL_ACT, TOL_GRAD, TOL_PARAM = 1e-4, 1e-3, 1e-3
-TOL_BF16 = 5e-3
+TOL_PARAM = 1e-3
 
 
 @pytest.fixture(scope="module")
@@ -24,150 +23,39 @@ def util():
     return gpu_util
 
 
-def _oracle_parts(w, pre):
-    """Per-part (rowptr, col, X, y) from the oracle's preprocessing."""
-    out = []
-    for p in range(pre["M"]):
-        rp, cp = oracle.part_graph(pre["rowptr_out"], pre["col_out"], pre["part_offsets"], pre["edge_offsets"], p)
-        lo, hi = int(pre["part_offsets"][p]), int(pre["part_offsets"][p + 1])
-        out.append((rp, cp, pre["Xp"][lo:hi].astype(np.float64), pre["yp"][lo:hi]))
-    return out
-
-
-def _tols(gemm_dtype):
-    """(activations, gradients, parameters, loss, |z| below which a ReLU branch is ambiguous as a
-    fraction of max|z|, flips allowed per part as a fraction of the hidden units)."""
-    if gemm_dtype == 1:   # operands rounded to bf16 (2^-9 each), fp32 accumulation
-        return TOL_BF16, TOL_BF16, TOL_BF16, TOL_BF16, 4e-3, 0.01
-    return TOL_ACT, TOL_GRAD, TOL_PARAM, 1e-5, 2e-5, 0.0
-
-
-def _check_one_step(util, w, M=None, gemm_dtype=0, streams=None):
-    """Step 0 intermediates and gradients, then K steps and the average."""
-    tol_act, tol_grad, tol_param, tol_loss, amb, flip_frac = _tols(gemm_dtype)
-    c = util.ctx()
-    got = util.gpu_preprocess(w, M=M)
-    want = util.oracle_preprocess(w, M=M)
-    util.assert_preprocess_equal(got, want)
-    M = got["M"]
-    dims, n = w.dims, w.graph.n
-    P = inputs.param_count(dims)
-    rec = sum(dims[l] + dims[l + 1] for l in range(len(dims) - 1))
-    params = util.dev(np.tile(w.params0, (M, 1)))
-    acts = torch.zeros(n * rec, dtype=torch.float32, device="cuda")
-    grads = torch.zeros(M, P, dtype=torch.float32, device="cuda")
-    loss = torch.zeros(M, 1, dtype=torch.float32, device="cuda")
-    c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
-                  got["Xp"], got["yp"], params, 1, loss_out=loss, taps=(acts, grads, 0), gemm_dtype=gemm_dtype,
-                  streams=streams)
-    torch.cuda.synchronize()
-    acts, grads, loss, params1 = acts.cpu().numpy(), grads.cpu().numpy(), loss.cpu().numpy(), params.cpu().numpy()
-    p0 = w.params0.astype(np.float64)
-    for p, (rp, cp, X, y) in enumerate(_oracle_parts(w, want)):
-        n_p = rp.size - 1
-        o_loss, o_grads, o_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True, want_preact=True)
-        layout, total = oracle.acts_layout(dims, n_p)
-        base = int(want["part_offsets"][p]) * rec
-        gpu_acts = {}
-        for name, off, r, wd in layout:
-            a = acts[base + off: base + off + r * wd].reshape(r, wd)
-            gpu_acts[name] = a
-            assert util.rel_err(a, o_acts[name]) <= tol_act, (p, name)
-        # ReLU has no derivative at 0: a hidden unit whose pre-activation is within the rounding
-        # error of an fp32 forward pass of 0 may legitimately take either branch, and the branch
-        # decides a finite part of the gradient.  For such units only (judged on the oracle's own
-        # pre-activations) the oracle is re-evaluated on the branch the kernel took; any other
-        # unit on the wrong branch fails the activation check above.
-        gates, flipped, units = [], 0, 0
-        for l in range(len(dims) - 2):
-            Z = o_acts[f"Z{l + 1}"]
-            ambiguous = np.abs(Z) < amb * max(1.0, np.abs(Z).max(initial=0.0))
-            units += Z.size
-            differ = ambiguous & ((gpu_acts[f"H{l + 1}"] > 0) != (Z > 0))
-            flipped += int(differ.sum())
-            g8 = np.full(Z.shape, -1, dtype=np.int8)
-            g8[differ] = (gpu_acts[f"H{l + 1}"] > 0)[differ]
-            gates.append(g8)
-        assert flipped <= 8 + flip_frac * units
-        if flipped:
-            o_loss, o_grads, _ = oracle.forward_backward(dims, rp, cp, X, y, p0, gates=gates)
-        if n_p:
-            assert abs(loss[p, 0] - o_loss) <= tol_loss * max(1.0, abs(o_loss)), p
-        # gradients: per parameter tensor
-        off = 0
-        for l in range(len(dims) - 1):
-            for nm, size in (("Ws", dims[l] * dims[l + 1]), ("Wn", dims[l] * dims[l + 1]), ("b", dims[l + 1])):
-                gg, og = grads[p, off:off + size], o_grads[off:off + size]
-                if np.abs(og).max() > 0:
-                    assert util.rel_err(gg, og) <= tol_grad, (p, l, nm)
-                else:
-                    assert np.abs(gg).max() == 0
-                off += size
-        assert util.rel_err(params1[p], p0 - w.lr * o_grads) <= tol_param
-    return got, want
-
-
-def _check_k_steps_and_average(util, w, got, want, K, gemm_dtype=0, streams=None):
-    tol_param = _tols(gemm_dtype)[2]
-    tol_loss = 10 * _tols(gemm_dtype)[3]
-    c = util.ctx()
-    M, dims = got["M"], w.dims
-    params = util.dev(np.tile(w.params0, (M, 1)))
-    loss = torch.zeros(M, K, dtype=torch.float32, device="cuda")
-    c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
-                  got["Xp"], got["yp"], params, K, loss_out=loss, gemm_dtype=gemm_dtype, streams=streams)
-    torch.cuda.synchronize()
-    after = params.cpu().numpy().copy()
-    glob = torch.empty(params.shape[1], dtype=torch.float32, device="cuda")
-    c.aggregate(params, glob)
-    torch.cuda.synchronize()
-    o_params = np.empty((M, params.shape[1]))
-    for p, (rp, cp, X, y) in enumerate(_oracle_parts(w, want)):
-        o_params[p], o_loss = oracle.local_steps(dims, w.lr, rp, cp, X, y, w.params0.astype(np.float64), K)
-        assert util.rel_err(after[p], o_params[p]) <= tol_param, p
-        if rp.size > 1:
-            assert np.abs(loss[p].cpu().numpy() - o_loss).max() <= tol_loss * max(1.0, np.abs(o_loss).max())
-    o_avg, o_glob = oracle.average(o_params)
-    assert util.rel_err(glob.cpu().numpy(), o_glob) <= tol_param
-    pa = params.cpu().numpy()
-    for p in range(M):
-        assert np.array_equal(pa[p], glob.cpu().numpy())     # every local copy overwritten
-    return after
-
-
 def test_tiny_config_end_to_end(util, tiny_workload):
     w = tiny_workload
-    got, want = _check_one_step(util, w)
-    _check_k_steps_and_average(util, w, got, want, w.K)
+    got, want = util.check_one_step(w)
+    util.check_k_steps_and_average(w, got, want, w.K)
 
 
 def test_medium_shape_scaled(util):
     # the Medium model (128-256-256-47, M=8) on a 12k-node power-law graph: several row tiles
     # per part plus a ragged tail, hubs, isolated local nodes
     w = inputs.medium(0.06)
-    got, want = _check_one_step(util, w)
-    _check_k_steps_and_average(util, w, got, want, 2)
+    got, want = util.check_one_step(w)
+    util.check_k_steps_and_average(w, got, want, 2)
 
 
 def test_supertma_shape_scaled_feature_width_100(util):
     w = inputs.supertma(0.02, M=4)   # 40k nodes, F=100 (rows of 400 bytes), super-node assignment
     w.dims = (100, 64, 47)
     w.params0 = inputs.xavier_params(w.dims, 5)
-    got, want = _check_one_step(util, w)
-    _check_k_steps_and_average(util, w, got, want, 2)
+    got, want = util.check_one_step(w)
+    util.check_k_steps_and_average(w, got, want, 2)
 
 
 def test_bf16_operand_mode(util, tiny_workload):
     # gemm_dtype = 1: every product takes its operands rounded to bf16 and accumulates in fp32
     w = tiny_workload
-    got, want = _check_one_step(util, w, gemm_dtype=1)
-    _check_k_steps_and_average(util, w, got, want, w.K, gemm_dtype=1)
+    got, want = util.check_one_step(w, gemm_dtype=1)
+    util.check_k_steps_and_average(w, got, want, w.K, gemm_dtype=1)
     # the width-512 sweep shape (512-512-512-47) on a scaled planted-community graph, node and
     # super-node assignment
     for use_groups in (True, False):
         w = inputs.supertma(0.004, width=512, M=2, use_groups=use_groups, gemm_dtype=1)
-        got, want = _check_one_step(util, w, gemm_dtype=1)
-    _check_k_steps_and_average(util, w, got, want, 2, gemm_dtype=1)
+        got, want = util.check_one_step(w, gemm_dtype=1)
+    util.check_k_steps_and_average(w, got, want, 2, gemm_dtype=1)
 
 
 def test_bf16_operand_mode_is_not_the_accurate_mode(util, tiny_workload):
@@ -204,7 +92,7 @@ def test_heterogeneous_step_counts(util, tiny_workload):
         c.local_steps(*args, params, steps, loss_out=loss, streams=streams)
         torch.cuda.synchronize()
         after, loss_h = params.cpu().numpy(), loss.cpu().numpy()
-        for p, (rp, cp, X, y) in enumerate(_oracle_parts(w, want)):
+        for p, (rp, cp, X, y) in enumerate(util.oracle_parts(w, want)):
             if steps[p] == 0:
                 assert np.array_equal(after[p], w.params0)
             else:
@@ -231,7 +119,7 @@ def test_failed_trainer_is_left_out_of_the_average(util, tiny_workload):
     got = util.gpu_preprocess(w)
     want = util.oracle_preprocess(w)
     M, dims = got["M"], w.dims
-    parts = _oracle_parts(w, want)
+    parts = util.oracle_parts(w, want)
     for failed in range(M):
         steps = [0 if p == failed else w.K for p in range(M)]
         alive = [p != failed for p in range(M)]
@@ -278,8 +166,8 @@ def test_odd_widths_and_binary_head(util, tiny_workload, dims):
     w.X = inputs.normal_features(w.graph.n, dims[0], 3)
     w.y = inputs.rare_positive_labels(w.graph.n, 0.1, 4) if dims[-1] == 2 else inputs.uniform_labels(w.graph.n, dims[-1], 4)
     w.params0 = inputs.xavier_params(dims, 6)
-    got, want = _check_one_step(util, w, M=3)
-    _check_k_steps_and_average(util, w, got, want, 3)
+    got, want = util.check_one_step(w, M=3)
+    util.check_k_steps_and_average(w, got, want, 3)
 
 
 def test_more_trainers_than_busy_parts(util):
@@ -287,21 +175,21 @@ def test_more_trainers_than_busy_parts(util):
     w = inputs.tiny()
     g = inputs.uniform_graph(40, 100, 3)
     w.graph, w.X, w.y = g, w.X[:40].copy(), w.y[:40].copy()
-    got, want = _check_one_step(util, w, M=64)
+    got, want = util.check_one_step(w, M=64)
     assert min(np.diff(want["part_offsets"])) == 0
-    _check_k_steps_and_average(util, w, got, want, 2)
+    util.check_k_steps_and_average(w, got, want, 2)
 
 
 def test_streams_do_not_change_the_result(util, tiny_workload):
     w = tiny_workload
     got = util.gpu_preprocess(w)
     want = util.oracle_preprocess(w)
-    one = _check_k_steps_and_average(util, w, got, want, 3)
+    one = util.check_k_steps_and_average(w, got, want, 3)
     streams = [torch.cuda.Stream() for _ in range(w.M)]
     torch.cuda.synchronize()
-    many = _check_k_steps_and_average(util, w, got, want, 3, streams=streams)
+    many = util.check_k_steps_and_average(w, got, want, 3, streams=streams)
     pairs = [streams[0], streams[1], streams[0], streams[1]]
-    two = _check_k_steps_and_average(util, w, got, want, 3, streams=pairs)
+    two = util.check_k_steps_and_average(w, got, want, 3, streams=pairs)
     assert np.array_equal(one, many) and np.array_equal(one, two)
 
 
