@@ -317,49 +317,45 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                         }
                     }
                 } else {
-                // plane output: bias, ReLU on the thread's own row; columns past N (or past the tile) become 0
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const int n = nbase + e;
-                    float tv = v[e];
-                    if (n < a.N && c0 + e < BN) {
-                        if (bias) tv += __ldg(bias + n);
-                        if (a.relu) tv = fmaxf(tv, 0.f);
-                    } else {
-                        tv = 0.f;
-                    }
-                    v[e] = tv;
-                }
-                // Transpose through the warp's staging slab so that every store instruction writes
-                // whole 128-byte (fp32) or 64-byte (plane) row segments instead of 32 scattered pieces.
-                __syncwarp();
-                {
-                    uint4* sh = reinterpret_cast<uint4*>(stg);        // [32 rows][4 pieces of 8 bf16], hi
-                    uint4* sl = sh + 128;                             // lo
-#pragma unroll
-                    for (int p = 0; p < 4; ++p) {
-                        Pack8 x;
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) x.v[e] = v[8 * p + e];
-                        uint4 h, l;
-                        x.to_planes(h, l);
-                        const int slot = lane * 4 + (p ^ ((lane >> 1) & 3));
-                        sh[slot] = h;
-                        sl[slot] = l;
-                    }
+                    // Plane output.  The warp's 32 x 32 block goes through its staging slab as fp32
+                    // (16-byte chunk j of row r stored at chunk j ^ (r & 7): conflict free both ways),
+                    // so that afterwards a thread owns 8 consecutive columns of a row: bias is two
+                    // vector loads per chunk, and every store instruction writes whole 64-byte row
+                    // segments of a plane.
+                    float4* st = reinterpret_cast<float4*>(stg);  // [32 rows][8 chunks of 4 floats]
                     __syncwarp();
 #pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        st[lane * 8 + (j ^ (lane & 7))] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    __syncwarp();
+                    const int p = lane & 3;
+                    const int n = nbase + 8 * p;
+                    const bool col_ok = n < a.out_planes.ld && c0 + 8 * p < BN;
+                    float bv[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) bv[e] = (bias && col_ok && n + e < a.N) ? __ldg(bias + n + e) : 0.f;
+#pragma unroll
                     for (int it = 0; it < 4; ++it) {
-                        const int row = it * 8 + (lane >> 2), p = lane & 3;
-                        const int n = nbase + 8 * p;
-                        if (row < rows_here && n < a.out_planes.ld && c0 + 8 * p < BN) {
-                            const int slot = row * 4 + (p ^ ((row >> 1) & 3));
+                        const int row = it * 8 + (lane >> 2);
+                        const float4 x0 = st[row * 8 + ((2 * p) ^ (row & 7))];
+                        const float4 x1 = st[row * 8 + ((2 * p + 1) ^ (row & 7))];
+                        if (row < rows_here && col_ok) {
+                            Pack8 x;
+                            x.v[0] = x0.x; x.v[1] = x0.y; x.v[2] = x0.z; x.v[3] = x0.w;
+                            x.v[4] = x1.x; x.v[5] = x1.y; x.v[6] = x1.z; x.v[7] = x1.w;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                float tv = x.v[e] + bv[e];
+                                if (a.relu) tv = fmaxf(tv, 0.f);
+                                x.v[e] = (n + e < a.N) ? tv : 0.f;  // padding columns of the planes stay zero
+                            }
+                            uint4 h, l;
+                            x.to_planes_cvt(h, l);
                             const int64_t at = (orow0 + row) * a.out_planes.ld + n;
-                            *reinterpret_cast<uint4*>(a.out_planes.hi + at) = sh[slot];
-                            *reinterpret_cast<uint4*>(a.out_planes.lo + at) = sl[slot];
+                            *reinterpret_cast<uint4*>(a.out_planes.hi + at) = h;
+                            *reinterpret_cast<uint4*>(a.out_planes.lo + at) = l;
                         }
                     }
-                }
                 }
             }
             tc::tc_fence_before_sync();
