@@ -64,15 +64,16 @@ def algorithmic_work(dims, n_parts, e_parts, K, R):
     steps = K * R
     work = {}
     spmm_f = sum(n * 8 * dims[l] + 4 * e + 8 * n for l in range(L))
-    spmm_b = sum(n * (4 * dims[l] * 2 + 4 * dims[l] * 2) + 4 * e + 8 * n for l in range(1, L))
+    spmm_b = sum(n * 8 * dims[l + 1] + 4 * e + 12 * n for l in range(1, L))
     work["spmm_forward"] = ("hbm", steps * spmm_f, steps * sum(e * dims[l] for l in range(L)))
-    work["spmm_backward"] = ("hbm", steps * spmm_b, steps * sum(e * dims[l] for l in range(1, L)))
+    work["spmm_backward"] = ("hbm", steps * spmm_b, steps * sum(2 * e * dims[l + 1] for l in range(1, L)))
     Mtr = len(n_parts)
     gf_b = sum(4 * n * (2 * dims[l] + dims[l + 1]) + 4 * Mtr * (2 * dims[l] + 1) * dims[l + 1] for l in range(L))
     gf_f = sum(2 * n * (2 * dims[l] + 1) * dims[l + 1] for l in range(L))
     work["gemm_forward"] = ("gemm", steps * gf_b, steps * gf_f)
     work["gemm_wgrad"] = ("gemm", steps * gf_b, steps * gf_f)
-    gd_b = sum(4 * n * (2 * dims[l] + dims[l + 1]) + 4 * Mtr * 2 * dims[l] * dims[l + 1] for l in range(1, L))
+    # dgrad reads dZ and Abar^T dZ (planes), the gate (hi plane of H) and writes dZ of the layer below
+    gd_b = sum(n * (8 * dims[l + 1] + 2 * dims[l] + 4 * dims[l]) + 4 * Mtr * 2 * dims[l] * dims[l + 1] for l in range(1, L))
     gd_f = sum(2 * n * 2 * dims[l] * dims[l + 1] for l in range(1, L))
     work["gemm_dgrad"] = ("gemm", steps * gd_b, steps * gd_f)
     P = sum((2 * dims[l] + 1) * dims[l + 1] for l in range(L))

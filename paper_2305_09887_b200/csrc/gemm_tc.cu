@@ -8,8 +8,9 @@
 //
 //   rows kernel   D[128 rows x BN] = [A0 | A1] * B^T   -- forward ([H | Abar H] times [Ws; Wn],
 //                 bias + ReLU epilogue, written back as planes, or as fp32 logits for the last
-//                 layer) and dgrad (dZ times [Ws; Wn]^T, 1/deg on the T half, fp32).  A tiles
-//                 are K-major straight from the planes, B from the repacked weights.
+//                 layer) and dgrad ([dZ | Abar^T dZ] times [Ws^T; Wn^T], gated by the sign of H
+//                 and written as planes over H).  A tiles are K-major straight from the planes,
+//                 B from the repacked weights.
 //   wgrad kernel  D[128 x d_out] = A^T * dZ over a chunk of rows, A = H or Abar H.  Both
 //                 operands are MN-major straight from the planes.  Rows between parts are
 //                 zero in every plane, so chunks need no masking.  The bias gradient (column
@@ -62,7 +63,9 @@ __device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
 //   forward  Bf[n][kk], n < Npad_f, kk < Kf = 2 * 64 * ceil(d_in / 64):
 //            kk <  Kf/2 : Ws[kk][n]          (zero beyond d_in / d_out)
 //            kk >= Kf/2 : Wn[kk - Kf/2][n]
-//   dgrad    Bd[j][c],  j < Npad_d (2 d_in valid), c < Kd = 64 * ceil(d_out / 64): Wcat[j][c]
+//   dgrad    Bd[j][kk], j < Npad_d (d_in valid), kk < Kd = 2 * 64 * ceil(d_out / 64):
+//            kk <  Kd/2 : Ws[j][kk]          (zero beyond d_in / d_out)
+//            kk >= Kd/2 : Wn[j][kk - Kd/2]
 // each written as a hi and a lo bf16 matrix.
 // ------------------------------------------------------------------------------------
 struct PrepArgs {
@@ -90,8 +93,10 @@ tc_weight_prep_kernel(const __grid_constant__ GroupDesc g, const PrepArgs a, con
             lo = a.Bf_lo + (int64_t)k * nf + i;
         } else {
             const int64_t ii = i - nf;
-            const int j = (int)(ii / a.Kd), c = (int)(ii % a.Kd);
-            if (j < 2 * d_in && c < d_out) x = W[(int64_t)j * d_out + c];
+            const int j = (int)(ii / a.Kd), kk = (int)(ii % a.Kd);
+            const int half = a.Kd / 2;
+            const int c = kk < half ? kk : kk - half;
+            if (j < d_in && c < d_out) x = W[(int64_t)(kk < half ? j : d_in + j) * d_out + c];
             hi = a.Bd_hi + (int64_t)k * nd + ii;
             lo = a.Bd_lo + (int64_t)k * nd + ii;
         }
@@ -116,9 +121,8 @@ struct RowsArgs {
     int64_t P, bias_offset;
     int relu;
     int single;            // 1: operands rounded to bf16 (hi planes only, one MMA per product)
-    const float* inv_deg;  // fp32 output only: columns >= scale_from are multiplied by inv_deg[row]
-    int scale_from;        // and stored scale_shift columns further right; scale_from < 0: none
-    int scale_shift;
+    const __nv_bfloat16* gate_hi;  // plane output only: entries whose gate value (same row and column,
+                                   // leading dimension of out_planes) is <= 0 become 0; NULL: none
     int* error_word;
 };
 
@@ -279,7 +283,6 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
             const int i = r0 + q * 32 + lane;
             const bool live = i < a.g.rows[k];
             const float* bias = a.bias_offset >= 0 ? a.params + (int64_t)a.g.part[k] * a.P + a.bias_offset : nullptr;
-            const float w = (a.scale_from >= 0 && live) ? a.inv_deg[a.g.row_ws[k] + i] : 1.f;
             const int rows_here = min(32, a.g.rows[k] - (r0 + q * 32));  // live rows of this warp's quarter
             const int64_t orow0 = a.g.row_ws[k] + r0 + q * 32;
             for (int c0 = col_phase * 32; c0 < BN; c0 += 64) {
@@ -288,7 +291,7 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                 if (rows_here <= 0) continue;
                 const int nbase = n0 + c0;
                 if constexpr (!PLANES_OUT) {
-                    // fp32 output (logits, [S | T]): each thread stores its own row, pack by pack
+                    // fp32 output (logits): each thread stores its own row, pack by pack
                     if (!live) continue;
                     float* o = a.out + (orow0 + lane) * a.ld_out;
 #pragma unroll
@@ -301,19 +304,15 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                             float tv = v[j + e];
                             if (n + e < a.N) {
                                 if (bias) tv += __ldg(bias + n + e);
-                                if (a.scale_from >= 0 && n + e >= a.scale_from) tv *= w;
                                 if (a.relu) tv = fmaxf(tv, 0.f);
                             }
                             x[e] = tv;
                         }
-                        const bool straddles = a.scale_from >= 0 && n < a.scale_from && n + 7 >= a.scale_from;
-                        const int dst0 = (a.scale_from >= 0 && n >= a.scale_from) ? n + a.scale_shift : n;
-                        if (!straddles && n + 7 < a.N && (dst0 & 3) == 0) {
-                            *reinterpret_cast<float4*>(o + dst0) = make_float4(x[0], x[1], x[2], x[3]);
-                            *reinterpret_cast<float4*>(o + dst0 + 4) = make_float4(x[4], x[5], x[6], x[7]);
+                        if (n + 7 < a.N) {
+                            *reinterpret_cast<float4*>(o + n) = make_float4(x[0], x[1], x[2], x[3]);
+                            *reinterpret_cast<float4*>(o + n + 4) = make_float4(x[4], x[5], x[6], x[7]);
                         } else {
-                            for (int e = 0; e < 8 && n + e < a.N; ++e)
-                                o[(a.scale_from >= 0 && n + e >= a.scale_from) ? n + e + a.scale_shift : n + e] = x[e];
+                            for (int e = 0; e < 8 && n + e < a.N; ++e) o[n + e] = x[e];
                         }
                     }
                 } else {
@@ -349,9 +348,18 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                                 if (a.relu) tv = fmaxf(tv, 0.f);
                                 x.v[e] = (n + e < a.N) ? tv : 0.f;  // padding columns of the planes stay zero
                             }
+                            const int64_t at = (orow0 + row) * a.out_planes.ld + n;
+                            if (a.gate_hi) {
+                                const uint4 gq = *reinterpret_cast<const uint4*>(a.gate_hi + at);
+                                const uint32_t gw[4] = {gq.x, gq.y, gq.z, gq.w};
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const float gate = __uint_as_float((e & 1) ? (gw[e >> 1] & 0xFFFF0000u) : (gw[e >> 1] << 16));
+                                    if (!(gate > 0.f)) x.v[e] = 0.f;
+                                }
+                            }
                             uint4 h, l;
                             x.to_planes_cvt(h, l);
-                            const int64_t at = (orow0 + row) * a.out_planes.ld + n;
                             *reinterpret_cast<uint4*>(a.out_planes.hi + at) = h;
                             *reinterpret_cast<uint4*>(a.out_planes.lo + at) = l;
                         }
@@ -654,9 +662,9 @@ TcLayerPlan tc_plan_layer(LayerShape ls) {
     int tiles = (int)ceil_div(ls.d_out, 256);
     p.BN_f = (int)ceil_div(ceil_div(ls.d_out, tiles), 16) * 16;
     p.Npad_f = p.BN_f * tiles;
-    p.Kd = TC_BK * (int)ceil_div(ls.d_out, TC_BK);
-    tiles = (int)ceil_div(2 * ls.d_in, 256);
-    p.BN_d = (int)ceil_div(ceil_div(2 * ls.d_in, tiles), 16) * 16;
+    p.Kd = 2 * TC_BK * (int)ceil_div(ls.d_out, TC_BK);
+    tiles = (int)ceil_div(ls.d_in, 256);
+    p.BN_d = (int)ceil_div(ceil_div(ls.d_in, tiles), 16) * 16;
     p.Npad_d = p.BN_d * tiles;
     return p;
 }
@@ -730,39 +738,33 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
     a.P = ls.P;
     a.bias_offset = ls.param_offset + (int64_t)2 * ls.d_in * ls.d_out;
     a.relu = relu ? 1 : 0;
-    a.inv_deg = nullptr;
-    a.scale_from = -1;
-    a.scale_shift = 0;
+    a.gate_hi = nullptr;
     return launch_rows(ctx, a, KC_GEMM_FWD, s);
 }
 
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
-                        Planes dZ, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, const float* inv_deg, Mat ST,
-                        bool single, cudaStream_t s) {
+                        Planes dZ, Planes Q, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, Planes H, bool single,
+                        cudaStream_t s) {
     RowsArgs a{};
     a.g = g;
     a.single = single ? 1 : 0;
     if (!plane_maps(&a.mapA0h, &a.mapA0l, dZ, rows_total, ls.d_out, TC_BK, TC_BM) ||
+        !plane_maps(&a.mapA1h, &a.mapA1l, Q, rows_total, ls.d_out, TC_BK, TC_BM) ||
         !make_tensor_map_bf16(&a.mapBh, Bd_hi, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d) ||
         !make_tensor_map_bf16(&a.mapBl, Bd_lo, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d))
         return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the dgrad operands");
-    a.mapA1h = a.mapA0h;
-    a.mapA1l = a.mapA0l;
-    a.kb0 = p.Kd / TC_BK;
-    a.kb1 = 0;
+    a.kb0 = a.kb1 = p.Kd / (2 * TC_BK);
     a.BN = p.BN_d;
     a.Npad = p.Npad_d;
-    a.N = 2 * ls.d_in;
-    a.out_planes = Planes{nullptr, nullptr, 0};
-    a.out = ST.ptr;
-    a.ld_out = ST.ld;
+    a.N = ls.d_in;
+    a.out_planes = H;  // every tile reads the gate of exactly the block it then overwrites
+    a.out = nullptr;
+    a.ld_out = 0;
     a.params = nullptr;
     a.P = 0;
     a.bias_offset = -1;
     a.relu = 0;
-    a.inv_deg = inv_deg;
-    a.scale_from = ls.d_in;  // S = columns [0, d_in); T = the second half of ST, scaled by 1/deg
-    a.scale_shift = (int)(ST.ld / 2) - ls.d_in;
+    a.gate_hi = H.hi;
     return launch_rows(ctx, a, KC_GEMM_DGRAD, s);
 }
 

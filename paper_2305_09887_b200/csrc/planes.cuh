@@ -57,6 +57,15 @@ struct Pack8 {
             v[2 * i + 1] += __uint_as_float(hw[i] & 0xFFFF0000u) + __uint_as_float(lw[i] & 0xFFFF0000u);
         }
     }
+    // v += w * (hi + lo); hi + lo is exact in fp32
+    __device__ __forceinline__ void fma_planes(const float w, const uint4 h, const uint4 l) {
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w}, lw[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = fmaf(w, __uint_as_float(hw[i] << 16) + __uint_as_float(lw[i] << 16), v[2 * i]);
+            v[2 * i + 1] = fmaf(w, __uint_as_float(hw[i] & 0xFFFF0000u) + __uint_as_float(lw[i] & 0xFFFF0000u), v[2 * i + 1]);
+        }
+    }
     __device__ __forceinline__ void to_planes(uint4& h, uint4& l) const {
         uint32_t hw[4], lw[4];
 #pragma unroll

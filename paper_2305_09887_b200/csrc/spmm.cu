@@ -1,6 +1,10 @@
 // Mean aggregation over the local neighbourhood (the row-normalised adjacency Abar of
-// Theorem 2 / Eq. (proof-2-pred)) and its transpose for the backward pass, on activations
-// stored as split bf16 planes; plus the conversions between fp32 rows and planes.
+// Theorem 2) and its transpose for the backward pass, on activations stored as split bf16
+// planes; plus the conversions between fp32 rows and planes.
+//
+// Forward:  N[v] = (1/deg v) sum_{u in N(v)} H[u]           (Abar H: weight on the destination)
+// Backward: Q[v] = sum_{u in N(v)} (1/deg u) dZ[u]          (Abar^T dZ on a symmetric graph: weight
+//           on the source), so that dH = [dZ | Q] [Ws^T ; Wn^T] is one product.
 //
 // Gather-bound and, at the tiny local degrees random partitioning leaves (about deg/M),
 // latency-bound: a warp takes 8 consecutive rows at a time, reads their offsets with one load and their
@@ -60,14 +64,13 @@ from_planes_kernel(const Planes src, const int64_t first_row, const int64_t rows
     }
 }
 
-// BACKWARD == false: out = inv_deg * sum src[nbr]                              (src, out: planes)
-// BACKWARD == true : out <- gate_out(S + sum T[nbr]); S, T = the two halves of ST (fp32), out
-//                    holds H on entry (the ReLU gate) and dZ on exit.
-template <int NCH, bool BACKWARD>
+// SRC_WEIGHTED == false: out[v] = inv_deg[v] * sum_u src[u]
+// SRC_WEIGHTED == true : out[v] = sum_u inv_deg[u] * src[u]
+template <int NCH, bool SRC_WEIGHTED>
 __global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 3 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
-            const Mat ST, const int d, const int64_t total_groups, int* __restrict__ ticket) {
+            const int d, const int64_t total_groups, int* __restrict__ ticket) {
     const int lane = threadIdx.x & 31;
   // Warps draw groups of 8 consecutive rows from a shared ticket counter until none are left:
   // degrees are power-law distributed, and a fixed assignment would leave most warps idle while
@@ -95,26 +98,15 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     for (int c = 0; c < NCH; ++c) acc[c].zero();
     int cur = 0;  // row (relative to i0) the accumulators belong to
 
-    // finishes row `row`: scale or gate, store, clear
+    // finishes row `row`: scale, store, clear
     auto flush = [&](int row) {
         const int64_t r = ws + i0 + row;
+        const float w = SRC_WEIGHTED ? 1.f : inv_deg[r];
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
             const int colx = (c * 32 + lane) * 8;
             if (colx < d) {
-                if (BACKWARD) {
-                    const float* s = ST.ptr + r * ST.ld + colx;
-                    const float4 s0 = *reinterpret_cast<const float4*>(s), s1 = *reinterpret_cast<const float4*>(s + 4);
-                    const uint4 gh = *reinterpret_cast<const uint4*>(out.hi + r * out.ld + colx);
-                    const uint32_t gw[4] = {gh.x, gh.y, gh.z, gh.w};
-                    const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float gate = __uint_as_float((e & 1) ? (gw[e >> 1] & 0xFFFF0000u) : (gw[e >> 1] << 16));
-                        acc[c].v[e] = gate > 0.f ? acc[c].v[e] + sv[e] : 0.f;
-                    }
-                } else {
-                    const float w = inv_deg[r];
+                if (!SRC_WEIGHTED) {
 #pragma unroll
                     for (int e = 0; e < 8; ++e) acc[c].v[e] *= w;
                 }
@@ -127,9 +119,8 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
         }
     };
 
-    const __nv_bfloat16* sh = BACKWARD ? nullptr : src.hi + ws * src.ld;
-    const __nv_bfloat16* sl = BACKWARD ? nullptr : src.lo + ws * src.ld;
-    const float* tsrc = BACKWARD ? ST.ptr + ws * ST.ld + (ST.ld >> 1) : nullptr;  // the T half
+    const __nv_bfloat16* sh = src.hi + ws * src.ld;
+    const __nv_bfloat16* sl = src.lo + ws * src.ld;
 
     for (int64_t e0 = e_begin; e0 < e_end; e0 += 32) {
         const int cnt = (int)min((int64_t)32, e_end - e0);
@@ -142,43 +133,20 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
             my_row += (j < nrows && oj <= e) ? 1 : 0;
         }
         const int32_t mine = lane < cnt ? __ldg(cols + e) : 0;
+        const float mine_w = (SRC_WEIGHTED && lane < cnt) ? __ldg(inv_deg + ws + mine) : 0.f;
         for (int t = 0; t < cnt; t += 4) {
             int32_t nb[4];
             int row[4];
+            float wt[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int tj = min(t + j, cnt - 1);
                 nb[j] = __shfl_sync(0xffffffffu, mine, tj);
                 row[j] = __shfl_sync(0xffffffffu, my_row, tj);
+                wt[j] = SRC_WEIGHTED ? __shfl_sync(0xffffffffu, mine_w, tj) : 1.f;
                 if (t + j >= cnt) nb[j] = -1;
             }
-            if (BACKWARD) {
-                float4 x[4][NCH][2];
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        const int colx = (c * 32 + lane) * 8;
-                        x[j][c][0] = x[j][c][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (nb[j] >= 0 && colx < d) {
-                            const float* p = tsrc + (int64_t)nb[j] * ST.ld + colx;
-                            x[j][c][0] = __ldg(reinterpret_cast<const float4*>(p));
-                            x[j][c][1] = __ldg(reinterpret_cast<const float4*>(p + 4));
-                        }
-                    }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (nb[j] < 0) continue;
-                    while (cur < row[j]) flush(cur++);
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        acc[c].v[0] += x[j][c][0].x; acc[c].v[1] += x[j][c][0].y;
-                        acc[c].v[2] += x[j][c][0].z; acc[c].v[3] += x[j][c][0].w;
-                        acc[c].v[4] += x[j][c][1].x; acc[c].v[5] += x[j][c][1].y;
-                        acc[c].v[6] += x[j][c][1].z; acc[c].v[7] += x[j][c][1].w;
-                    }
-                }
-            } else {
+            {
                 uint4 xh[4][NCH], xl[4][NCH];
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
@@ -196,7 +164,10 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                     if (nb[j] < 0) continue;
                     while (cur < row[j]) flush(cur++);
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c) acc[c].add_planes(xh[j][c], xl[j][c]);
+                    for (int c = 0; c < NCH; ++c) {
+                        if (SRC_WEIGHTED) acc[c].fma_planes(wt[j], xh[j][c], xl[j][c]);
+                        else acc[c].add_planes(xh[j][c], xl[j][c]);
+                    }
                 }
             }
         }
@@ -213,9 +184,9 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     }
 }
 
-template <bool BACKWARD>
+template <bool SRC_WEIGHTED>
 int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                      const float* inv_deg, Planes src, Planes out, Mat ST, int d, int* ticket, cudaStream_t s) {
+                      const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s) {
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
     if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
@@ -225,9 +196,9 @@ int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_o
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, SPMM_THREADS / 32), (int64_t)sms * blocks_per_sm);
 #define RTMA_SPMM(N)                                                                                      \
     do {                                                                                                  \
-        KernelScope ks(ctx, BACKWARD ? KC_SPMM_BWD : KC_SPMM_FWD, s);                                     \
-        spmm_kernel<N, BACKWARD><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, \
-                                                               ST, d, groups, ticket);                    \
+        KernelScope ks(ctx, SRC_WEIGHTED ? KC_SPMM_BWD : KC_SPMM_FWD, s);                                 \
+        spmm_kernel<N, SRC_WEIGHTED><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src,  \
+                                                                   out, d, groups, ticket);               \
     } while (0)
     if (d <= 256) RTMA_SPMM(1);
     else if (d <= 512) RTMA_SPMM(2);
@@ -266,10 +237,10 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                          const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s) {
-    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, Mat{nullptr, 0}, d, ticket, s);
+    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, ticket, s);
 }
 
-int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat ST, Planes h, int d, int* ticket, cudaStream_t s) {
-    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, nullptr, Planes{nullptr, nullptr, 0}, h, ST, d, ticket, s);
+int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                               const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s) {
+    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, ticket, s);
 }

@@ -39,10 +39,10 @@ int32_t parse_model(rtma_ctx* ctx, const rtma_model_desc* md, Model* m) {
 
 // Scratch one part of n_p rows needs.
 struct ScratchPlan {
-    size_t per_row_bytes;     // planes, logits, [S|T], 1/deg
+    size_t per_row_bytes;     // planes, logits, 1/deg
     size_t max_layer_params;  // largest (2 d_in + 1) d_out
     size_t prep_bytes;        // repacked weights, per part
-    size_t st_half;           // floats in one half of [S | T]
+    int q_width;              // widest Abar^T dZ (widths of the layers above the first)
 };
 
 int64_t aligned_rows(int64_t n_p) { return ceil_div(n_p, GROUP_ROW_ALIGN) * GROUP_ROW_ALIGN; }
@@ -51,18 +51,18 @@ ScratchPlan plan_scratch(const Model& m) {
     ScratchPlan sp{};
     size_t per_row = sizeof(float);              // inv_deg
     per_row += 4 * planes_ld(m.dims[0]);         // X as planes
-    size_t widest_hidden = 0;
+    int q_width = 0;
     for (int l = 0; l < m.L; ++l) {
         per_row += 4 * planes_ld(m.dims[l]);     // Abar H^l
         if (l < m.L - 1) per_row += 4 * planes_ld(m.dims[l + 1]);  // H^{l+1}, later overwritten by dZ^l
-        if (l >= 1) widest_hidden = std::max(widest_hidden, planes_ld(m.dims[l]));
+        if (l >= 1) q_width = std::max(q_width, m.dims[l + 1]);
         sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(2 * m.dims[l] + 1) * m.dims[l + 1]);
         sp.prep_bytes += sizeof(__nv_bfloat16) * tc_prep_elems(tc_plan_layer(m.layer[l]), l >= 1) + 4 * 256;
     }
     per_row += sizeof(float) * planes_ld(m.dims[m.L]);  // logits
     per_row += 4 * planes_ld(m.dims[m.L]);              // dZ of the last layer
-    sp.st_half = widest_hidden;
-    per_row += sizeof(float) * 2 * widest_hidden;       // [S | T]
+    sp.q_width = q_width;
+    if (q_width) per_row += 4 * planes_ld(q_width);     // Abar^T dZ
     sp.per_row_bytes = per_row;
     return sp;
 }
@@ -230,7 +230,9 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             const int C = m.dims[m.L];
             Mat logits{cur.take<float>((size_t)rows * planes_ld(C) + 8), (int64_t)planes_ld(C)};
             Planes dZlast = take_planes(C);
-            Mat ST{cur.take<float>((size_t)rows * 2 * plan.st_half + 8), (int64_t)(2 * plan.st_half)};
+            // Abar^T dZ of the layer in hand; carved at the widest layer, addressed at each layer's own width
+            __nv_bfloat16* q_hi = plan.q_width ? cur.take<__nv_bfloat16>((size_t)rows * planes_ld(plan.q_width) + 8) : nullptr;
+            __nv_bfloat16* q_lo = plan.q_width ? cur.take<__nv_bfloat16>((size_t)rows * planes_ld(plan.q_width) + 8) : nullptr;
             float* partial = cur.take<float>((size_t)slots * plan.max_layer_params + 4);
             float* tile_loss = cur.take<float>((size_t)loss_tiles(g) + 4);
             int* ticket = cur.take<int>(64);  // work counter of the aggregation kernels (zero between launches)
@@ -317,10 +319,15 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 for (int l = m.L - 1; l >= 0; --l) {
                     const Planes dZ = l == m.L - 1 ? dZlast : Hl[l + 1];
                     RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, single_pass, s));
-                    if (l > 0) RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Bd_hi[l], Bd_lo[l], inv_deg, ST, single_pass, s));
+                    if (l > 0) {
+                        // dH^l = dZ Ws^T + Abar^T (dZ Wn^T) = [dZ | Abar^T dZ] [Ws^T ; Wn^T]: aggregate first,
+                        // at the layer's output width, then one product whose epilogue applies the ReLU
+                        // gate and writes dZ^{l-1} over H^l
+                        const Planes Q{q_hi, q_lo, (int64_t)planes_ld(m.dims[l + 1])};
+                        RTMA_TRY(launch_spmm_transposed(ctx, g, rowptr_out, col_out, inv_deg, dZ, Q, m.dims[l + 1], ticket, s));
+                        RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Q, Bd_hi[l], Bd_lo[l], Hl[l], single_pass, s));
+                    }
                     RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
-                    if (l > 0)  // dZ^{l-1} overwrites H^l, whose sign is the ReLU gate
-                        RTMA_TRY(launch_spmm_backward(ctx, g, rowptr_out, col_out, ST, Hl[l], m.dims[l], ticket, s));
                 }
             }
         }

@@ -76,10 +76,9 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 // ticket: two ints of scratch, zero on entry and zero again when the kernel has finished.
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                          const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s);
-// h[r] <- (S[r] + sum_{u in N(r)} T[u]) where h[r] > 0 else 0, S = ST[:, 0:d], T = ST[:, d:2d]
-// (backward through the symmetric aggregation and the ReLU; h holds H on entry, dZ on exit).
-int32_t launch_spmm_backward(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                             Mat ST, Planes h, int d, int* ticket, cudaStream_t s);
+// out[r] = sum_{u in N(r)} inv_deg[u] * src[u]                     (backward: Abar^T on a symmetric graph)
+int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                               const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s);
 
 // ---- loss.cu --------------------------------------------------------------------------
 // Softmax cross-entropy over fp32 logits, mean over the part; dZ = (softmax - onehot) / n_p is
@@ -101,7 +100,7 @@ int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float*
 // instead of three.
 struct TcLayerPlan {
     int Kf, BN_f, Npad_f;  // forward: padded K (2 x 64-blocks over d_in), column tile, padded N
-    int Kd, BN_d, Npad_d;  // dgrad: padded K over d_out, column tile, padded N over 2 d_in
+    int Kd, BN_d, Npad_d;  // dgrad: padded K (2 x 64-blocks over d_out), column tile, padded N over d_in
 };
 bool tc_available();
 TcLayerPlan tc_plan_layer(LayerShape ls);
@@ -115,10 +114,12 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
                           const float* params, Planes H, Planes N, const __nv_bfloat16* Bf_hi,
                           const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, bool single,
                           cudaStream_t s);
-// ST[:, 0:d_in] = dZ Ws^T ;  ST[:, d_in:2 d_in] = inv_deg * (dZ Wn^T)
+// H <- ([dZ | Q] [Ws^T ; Wn^T]) where H > 0 else 0: on entry H holds the layer's input activations
+// (their sign is the ReLU gate), on exit the gradient with respect to the previous layer's
+// pre-activations.  Q = Abar^T dZ.
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
-                        Planes dZ, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, const float* inv_deg, Mat ST,
-                        bool single, cudaStream_t s);
+                        Planes dZ, Planes Q, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, Planes H, bool single,
+                        cudaStream_t s);
 // partial[slot][(2 d_in + 1) x d_out] = [H | N | 1]^T dZ over one chunk of rows.
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
                         Planes H, Planes N, Planes dZ, float* partial, bool single, cudaStream_t s);
