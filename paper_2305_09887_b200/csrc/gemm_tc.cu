@@ -286,6 +286,22 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
             const int rows_here = min(32, a.g.rows[k] - (r0 + q * 32));  // live rows of this warp's quarter
             const int64_t orow0 = a.g.row_ws[k] + r0 + q * 32;
             for (int c0 = col_phase * 32; c0 < BN; c0 += 64) {
+                // the gate words this thread will need after the transpose, requested before the
+                // accumulator is read so that their latency hides behind it
+                uint4 gq[4];
+                if constexpr (PLANES_OUT) {
+                    if (a.gate_hi) {
+                        const int gn = n0 + c0 + 8 * (lane & 3);
+                        const bool g_ok = gn < a.out_planes.ld && c0 + 8 * (lane & 3) < BN;
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) {
+                            const int row = it * 8 + (lane >> 2);
+                            gq[it] = (g_ok && row < rows_here)
+                                         ? *reinterpret_cast<const uint4*>(a.gate_hi + (orow0 + row) * a.out_planes.ld + gn)
+                                         : make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+                }
                 float v[32];
                 tc::tmem_load_32x32(d_tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
                 if (rows_here <= 0) continue;
@@ -350,8 +366,7 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                             }
                             const int64_t at = (orow0 + row) * a.out_planes.ld + n;
                             if (a.gate_hi) {
-                                const uint4 gq = *reinterpret_cast<const uint4*>(a.gate_hi + at);
-                                const uint32_t gw[4] = {gq.x, gq.y, gq.z, gq.w};
+                                const uint32_t gw[4] = {gq[it].x, gq[it].y, gq[it].z, gq[it].w};
 #pragma unroll
                                 for (int e = 0; e < 8; ++e) {
                                     const float gate = __uint_as_float((e & 1) ? (gw[e >> 1] & 0xFFFF0000u) : (gw[e >> 1] << 16));
