@@ -42,6 +42,12 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 __device__ __forceinline__ float join_bf16(__nv_bfloat16 hi, __nv_bfloat16 lo) {
     return bf16_bits_to_float(__bfloat16_as_ushort(hi)) + bf16_bits_to_float(__bfloat16_as_ushort(lo));
 }
+// acc + x with x a bf16 number (bits in a 16-bit register): exact conversion, one fp32 rounding
+__device__ __forceinline__ float add_f32_bf16(float acc, unsigned short x_bits) {
+    float d;
+    asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(x_bits), "f"(acc));
+    return d;
+}
 // Eight consecutive elements (16 bytes per plane); a 32-bit word holds elements 2i (low half) and 2i+1.
 struct Pack8 {
     float v[8];
@@ -55,6 +61,27 @@ struct Pack8 {
         for (int i = 0; i < 4; ++i) {
             v[2 * i] += __uint_as_float(hw[i] << 16) + __uint_as_float(lw[i] << 16);
             v[2 * i + 1] += __uint_as_float(hw[i] & 0xFFFF0000u) + __uint_as_float(lw[i] & 0xFFFF0000u);
+        }
+    }
+    // v += hi, v += lo with the mixed-precision add (fp32 accumulator, bf16 addend): no unpacking
+    // arithmetic on the integer pipe
+    __device__ __forceinline__ void add_planes_mixed(const uint4 h, const uint4 l) {
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w}, lw[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = add_f32_bf16(add_f32_bf16(v[2 * i], (unsigned short)(hw[i] & 0xFFFFu)), (unsigned short)(lw[i] & 0xFFFFu));
+            v[2 * i + 1] = add_f32_bf16(add_f32_bf16(v[2 * i + 1], (unsigned short)(hw[i] >> 16)), (unsigned short)(lw[i] >> 16));
+        }
+    }
+    // v += w * (hi + lo), hi + lo formed exactly by two mixed-precision adds
+    __device__ __forceinline__ void fma_planes_mixed(const float w, const uint4 h, const uint4 l) {
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w}, lw[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float t0 = add_f32_bf16(add_f32_bf16(0.f, (unsigned short)(lw[i] & 0xFFFFu)), (unsigned short)(hw[i] & 0xFFFFu));
+            const float t1 = add_f32_bf16(add_f32_bf16(0.f, (unsigned short)(lw[i] >> 16)), (unsigned short)(hw[i] >> 16));
+            v[2 * i] = fmaf(w, t0, v[2 * i]);
+            v[2 * i + 1] = fmaf(w, t1, v[2 * i + 1]);
         }
     }
     // v += w * (hi + lo); hi + lo is exact in fp32

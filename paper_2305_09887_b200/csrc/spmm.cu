@@ -9,7 +9,7 @@
 // Gather-bound and, at the tiny local degrees random partitioning leaves (about deg/M),
 // latency-bound: a warp takes 8 consecutive rows at a time, reads their offsets with one load and their
 // column indices with one coalesced load per 32 entries (consecutive rows are consecutive
-// in the CSR), and walks the entries with four neighbours' rows in flight per lane.  Lanes
+// in the CSR), and walks the entries with eight (four for rows wider than 256) neighbours' rows in flight per lane.  Lanes
 // split the feature width in pieces of 8 values (16 bytes per plane).
 #include <algorithm>
 
@@ -64,13 +64,63 @@ from_planes_kernel(const Planes src, const int64_t first_row, const int64_t rows
     }
 }
 
+// Heavy row groups first.  Local degrees are power-law distributed: a group that holds a hub takes
+// tens of times longer than the average one, and if a warp draws it late the whole launch waits
+// for it.  Groups are therefore bucketed once per call by the logarithm of their entry count and
+// the aggregation kernels walk the buckets from the heaviest down (longest job first).  The order
+// inside a bucket is arbitrary and does not influence any result.
+constexpr int ORDER_BUCKETS = 16;
+__device__ __forceinline__ int order_bucket(int64_t entries) {
+    const int lg = entries <= 0 ? 0 : min(ORDER_BUCKETS - 1, 64 - __clzll(entries));  // 1 | 2-3 | 4-7 | ...
+    return ORDER_BUCKETS - 1 - lg;
+}
+__device__ __forceinline__ int64_t group_entries(const GroupDesc& g, const int64_t* rowptr_out, int64_t grp) {
+    int k, i0;
+    if (!locate_tile(g, SPMM_ROWS_PER_WARP, grp, &k, &i0)) return 0;
+    const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
+    return rp[min(i0 + SPMM_ROWS_PER_WARP, g.rows[k])] - rp[i0];
+}
+
+__global__ void __launch_bounds__(256)
+order_count_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, const int64_t total_groups,
+                   int* __restrict__ hist) {
+    __shared__ int h[ORDER_BUCKETS];
+    if (threadIdx.x < ORDER_BUCKETS) h[threadIdx.x] = 0;
+    __syncthreads();
+    for (int64_t grp = (int64_t)blockIdx.x * 256 + threadIdx.x; grp < total_groups; grp += (int64_t)gridDim.x * 256)
+        atomicAdd(&h[order_bucket(group_entries(g, rowptr_out, grp))], 1);
+    __syncthreads();
+    if (threadIdx.x < ORDER_BUCKETS && h[threadIdx.x]) atomicAdd(hist + threadIdx.x, h[threadIdx.x]);
+}
+
+__global__ void __launch_bounds__(256)
+order_scatter_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, const int64_t total_groups,
+                     const int* __restrict__ hist, int* __restrict__ cursor, int* __restrict__ order) {
+    __shared__ int base[ORDER_BUCKETS];
+    if (threadIdx.x == 0) {
+        int at = 0;
+        for (int b = 0; b < ORDER_BUCKETS; ++b) {
+            base[b] = at;
+            at += hist[b];
+        }
+    }
+    __syncthreads();
+    for (int64_t grp = (int64_t)blockIdx.x * 256 + threadIdx.x; grp < total_groups; grp += (int64_t)gridDim.x * 256) {
+        const int b = order_bucket(group_entries(g, rowptr_out, grp));
+        order[base[b] + atomicAdd(cursor + b, 1)] = (int)grp;
+    }
+}
+
 // SRC_WEIGHTED == false: out[v] = inv_deg[v] * sum_u src[u]
 // SRC_WEIGHTED == true : out[v] = sum_u inv_deg[u] * src[u]
 template <int NCH, bool SRC_WEIGHTED>
-__global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 3 : 1)
+__global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 2 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
-            const int d, const int64_t total_groups, int* __restrict__ ticket) {
+            const int d, const int64_t total_groups, const int* __restrict__ order, int* __restrict__ ticket) {
+    // neighbours' rows a lane has in flight: a hub row is a chain of entries / SPMM_INFLIGHT memory
+    // round trips, and that chain sets the length of the whole launch
+    constexpr int SPMM_INFLIGHT = NCH == 1 ? 8 : 4;
     const int lane = threadIdx.x & 31;
   // Warps draw groups of 8 consecutive rows from a shared ticket counter until none are left:
   // degrees are power-law distributed, and a fixed assignment would leave most warps idle while
@@ -80,6 +130,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     if (lane == 0) grp = atomicAdd(ticket, 1);
     grp = __shfl_sync(0xffffffffu, grp, 0);
     if (grp >= total_groups) break;
+    if (order) grp = order[grp];
     int k, i0;
     if (!locate_tile(g, SPMM_ROWS_PER_WARP, grp, &k, &i0)) break;
     const int n_p = g.rows[k];
@@ -134,12 +185,12 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
         }
         const int32_t mine = lane < cnt ? __ldg(cols + e) : 0;
         const float mine_w = (SRC_WEIGHTED && lane < cnt) ? __ldg(inv_deg + ws + mine) : 0.f;
-        for (int t = 0; t < cnt; t += 4) {
-            int32_t nb[4];
-            int row[4];
-            float wt[4];
+        for (int t = 0; t < cnt; t += SPMM_INFLIGHT) {
+            int32_t nb[SPMM_INFLIGHT];
+            int row[SPMM_INFLIGHT];
+            float wt[SPMM_INFLIGHT];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < SPMM_INFLIGHT; ++j) {
                 const int tj = min(t + j, cnt - 1);
                 nb[j] = __shfl_sync(0xffffffffu, mine, tj);
                 row[j] = __shfl_sync(0xffffffffu, my_row, tj);
@@ -147,9 +198,9 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                 if (t + j >= cnt) nb[j] = -1;
             }
             {
-                uint4 xh[4][NCH], xl[4][NCH];
+                uint4 xh[SPMM_INFLIGHT][NCH], xl[SPMM_INFLIGHT][NCH];
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
+                for (int j = 0; j < SPMM_INFLIGHT; ++j)
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
                         const int colx = (c * 32 + lane) * 8;
@@ -160,13 +211,13 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                         }
                     }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < SPMM_INFLIGHT; ++j) {
                     if (nb[j] < 0) continue;
                     while (cur < row[j]) flush(cur++);
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
-                        if (SRC_WEIGHTED) acc[c].fma_planes(wt[j], xh[j][c], xl[j][c]);
-                        else acc[c].add_planes(xh[j][c], xl[j][c]);
+                        if (SRC_WEIGHTED) acc[c].fma_planes_mixed(wt[j], xh[j][c], xl[j][c]);
+                        else acc[c].add_planes_mixed(xh[j][c], xl[j][c]);
                     }
                 }
             }
@@ -186,19 +237,19 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
 
 template <bool SRC_WEIGHTED>
 int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                      const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s) {
+                      const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket, cudaStream_t s) {
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
     if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
     static int sms = 0;
     if (!sms && (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess || sms <= 0)) sms = 148;
-    const int blocks_per_sm = d <= 256 ? 3 : 1;
+    const int blocks_per_sm = d <= 256 ? 2 : 1;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, SPMM_THREADS / 32), (int64_t)sms * blocks_per_sm);
 #define RTMA_SPMM(N)                                                                                      \
     do {                                                                                                  \
         KernelScope ks(ctx, SRC_WEIGHTED ? KC_SPMM_BWD : KC_SPMM_FWD, s);                                 \
         spmm_kernel<N, SRC_WEIGHTED><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src,  \
-                                                                   out, d, groups, ticket);               \
+                                                                   out, d, groups, order, ticket);        \
     } while (0)
     if (d <= 256) RTMA_SPMM(1);
     else if (d <= 512) RTMA_SPMM(2);
@@ -236,11 +287,28 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 }
 
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                         const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s) {
-    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, ticket, s);
+                         const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket,
+                         cudaStream_t s) {
+    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
 }
 
 int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                               const float* inv_deg, Planes src, Planes out, int d, int* ticket, cudaStream_t s) {
-    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, ticket, s);
+                               const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket,
+                               cudaStream_t s) {
+    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
+}
+
+int64_t spmm_order_entries(const GroupDesc& g) { return group_tiles(g, SPMM_ROWS_PER_WARP); }
+
+int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, int* counters, int* order,
+                          cudaStream_t s) {
+    const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
+    if (groups == 0) return RTMA_OK;
+    if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, 256), 148 * 4);
+    { KernelScope ks(ctx, KC_INV_DEGREE, s); order_count_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, groups, counters); }
+    RTMA_LAUNCH_CHECK(ctx);
+    { KernelScope ks(ctx, KC_INV_DEGREE, s); order_scatter_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, groups, counters, counters + ORDER_BUCKETS, order); }
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
 }

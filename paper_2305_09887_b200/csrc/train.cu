@@ -91,6 +91,7 @@ size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
     const size_t rows = (size_t)aligned_rows(n_p);
     const size_t matrices = 8 * m.L + 12;  // every matrix start is rounded up to 256 bytes
     return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, 32) + 256) +
+           sizeof(int) * ((size_t)ceil_div(n_p, 8) + 64) +  // processing order of the aggregation kernels
            sp.prep_bytes + 256 * matrices;
 }
 
@@ -237,6 +238,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             float* tile_loss = cur.take<float>((size_t)loss_tiles(g) + 4);
             int* ticket = cur.take<int>(64);  // work counter of the aggregation kernels (zero between launches)
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
+            int* spmm_order = cur.take<int>((size_t)spmm_order_entries(g) + 4);
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
             __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
             for (int l = 0; l < m.L; ++l) {
@@ -254,6 +256,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
 
             RTMA_CUDA(ctx, cudaMemsetAsync(ctx->arena + gi * share, 0, zero_bytes, s));
             RTMA_TRY(launch_inv_degree(ctx, g, rowptr_out, inv_deg, s));
+            RTMA_TRY(launch_spmm_order(ctx, g, rowptr_out, ticket + 16, spmm_order, s));
             RTMA_TRY(launch_to_planes(ctx, g, Xp, m.dims[0], Hl[0], s));
             const Planes no_planes{nullptr, nullptr, 0};
             const Mat no_mat{nullptr, 0};
@@ -265,6 +268,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 // trainers reach the aggregation point with different step counts)
                 bool all_run = true;
                 for (int k = 0; k < wave.num; ++k) all_run = all_run && steps[wave.part[k]] > step;
+                const int* order = all_run ? spmm_order : nullptr;  // the order was built for the whole wave
                 if (all_run) {
                     g = wave;
                     sp = wave_sp;
@@ -291,7 +295,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 for (int l = 0; l < m.L; ++l)
                     RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
                 for (int l = 0; l < m.L; ++l) {
-                    RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], ticket, s));
+                    RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], order, ticket, s));
                     const bool last = l == m.L - 1;
                     RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
                                                last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, single_pass, s));
@@ -324,7 +328,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                         // at the layer's output width, then one product whose epilogue applies the ReLU
                         // gate and writes dZ^{l-1} over H^l
                         const Planes Q{q_hi, q_lo, (int64_t)planes_ld(m.dims[l + 1])};
-                        RTMA_TRY(launch_spmm_transposed(ctx, g, rowptr_out, col_out, inv_deg, dZ, Q, m.dims[l + 1], ticket, s));
+                        RTMA_TRY(launch_spmm_transposed(ctx, g, rowptr_out, col_out, inv_deg, dZ, Q, m.dims[l + 1], order, ticket, s));
                         RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Q, Bd_hi[l], Bd_lo[l], Hl[l], single_pass, s));
                     }
                     RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
