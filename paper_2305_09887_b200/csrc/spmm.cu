@@ -66,14 +66,9 @@ from_planes_kernel(const Planes src, const int64_t first_row, const int64_t rows
 
 // Heavy row groups first.  Local degrees are power-law distributed: a group that holds a hub takes
 // tens of times longer than the average one, and if a warp draws it late the whole launch waits
-// for it.  Groups are therefore bucketed once per call by the logarithm of their entry count and
-// the aggregation kernels walk the buckets from the heaviest down (longest job first).  The order
-// inside a bucket is arbitrary and does not influence any result.
-constexpr int ORDER_BUCKETS = 16;
-__device__ __forceinline__ int order_bucket(int64_t entries) {
-    const int lg = entries <= 0 ? 0 : min(ORDER_BUCKETS - 1, 64 - __clzll(entries));  // 1 | 2-3 | 4-7 | ...
-    return ORDER_BUCKETS - 1 - lg;
-}
+// for it.  Once per call the groups with at least `heavy` entries are listed; the aggregation
+// kernels hand those out first (longest jobs first) and then walk all groups in row order,
+// part after part (which keeps one part's source rows in L2), skipping the listed ones.
 __device__ __forceinline__ int64_t group_entries(const GroupDesc& g, const int64_t* rowptr_out, int64_t grp) {
     int k, i0;
     if (!locate_tile(g, SPMM_ROWS_PER_WARP, grp, &k, &i0)) return 0;
@@ -82,33 +77,10 @@ __device__ __forceinline__ int64_t group_entries(const GroupDesc& g, const int64
 }
 
 __global__ void __launch_bounds__(256)
-order_count_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, const int64_t total_groups,
-                   int* __restrict__ hist) {
-    __shared__ int h[ORDER_BUCKETS];
-    if (threadIdx.x < ORDER_BUCKETS) h[threadIdx.x] = 0;
-    __syncthreads();
+heavy_list_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, const int64_t total_groups,
+                  const int64_t heavy, int* __restrict__ count, int* __restrict__ list) {
     for (int64_t grp = (int64_t)blockIdx.x * 256 + threadIdx.x; grp < total_groups; grp += (int64_t)gridDim.x * 256)
-        atomicAdd(&h[order_bucket(group_entries(g, rowptr_out, grp))], 1);
-    __syncthreads();
-    if (threadIdx.x < ORDER_BUCKETS && h[threadIdx.x]) atomicAdd(hist + threadIdx.x, h[threadIdx.x]);
-}
-
-__global__ void __launch_bounds__(256)
-order_scatter_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, const int64_t total_groups,
-                     const int* __restrict__ hist, int* __restrict__ cursor, int* __restrict__ order) {
-    __shared__ int base[ORDER_BUCKETS];
-    if (threadIdx.x == 0) {
-        int at = 0;
-        for (int b = 0; b < ORDER_BUCKETS; ++b) {
-            base[b] = at;
-            at += hist[b];
-        }
-    }
-    __syncthreads();
-    for (int64_t grp = (int64_t)blockIdx.x * 256 + threadIdx.x; grp < total_groups; grp += (int64_t)gridDim.x * 256) {
-        const int b = order_bucket(group_entries(g, rowptr_out, grp));
-        order[base[b] + atomicAdd(cursor + b, 1)] = (int)grp;
-    }
+        if (group_entries(g, rowptr_out, grp) >= heavy) list[atomicAdd(count, 1)] = (int)grp;
 }
 
 // SRC_WEIGHTED == false: out[v] = inv_deg[v] * sum_u src[u]
@@ -117,7 +89,7 @@ template <int NCH, bool SRC_WEIGHTED>
 __global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 2 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
-            const int d, const int64_t total_groups, const int* __restrict__ order, int* __restrict__ ticket) {
+            const int d, const int64_t total_groups, const SpmmOrder order, int* __restrict__ ticket) {
     // neighbours' rows a lane has in flight: a hub row is a chain of entries / SPMM_INFLIGHT memory
     // round trips, and that chain sets the length of the whole launch
     constexpr int SPMM_INFLIGHT = NCH == 1 ? 8 : 4;
@@ -129,8 +101,11 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     int64_t grp = 0;
     if (lane == 0) grp = atomicAdd(ticket, 1);
     grp = __shfl_sync(0xffffffffu, grp, 0);
-    if (grp >= total_groups) break;
-    if (order) grp = order[grp];
+    // tickets 0 .. n_heavy-1 are the listed heavy groups, the rest all groups in row order
+    const int64_t n_heavy = order.heavy_count ? *order.heavy_count : 0;
+    if (grp >= n_heavy + total_groups) break;
+    const bool listed = grp < n_heavy;
+    grp = listed ? order.heavy_list[grp] : grp - n_heavy;
     int k, i0;
     if (!locate_tile(g, SPMM_ROWS_PER_WARP, grp, &k, &i0)) break;
     const int n_p = g.rows[k];
@@ -143,6 +118,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     const int64_t my_off = (nrows > 0 && lane <= nrows) ? rp[i0 + lane] : 0;
     const int64_t e_begin = __shfl_sync(0xffffffffu, my_off, 0);
     const int64_t e_end = __shfl_sync(0xffffffffu, my_off, nrows);
+    if (!listed && order.heavy_count && e_end - e_begin >= order.heavy) continue;  // done as a listed group
 
     Pack8 acc[NCH];
 #pragma unroll
@@ -237,7 +213,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
 
 template <bool SRC_WEIGHTED>
 int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                      const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket, cudaStream_t s) {
+                      const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket, cudaStream_t s) {
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
     if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
@@ -287,28 +263,30 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 }
 
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                         const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket,
+                         const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                          cudaStream_t s) {
     return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
 }
 
 int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                               const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket,
+                               const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                                cudaStream_t s) {
     return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
 }
 
 int64_t spmm_order_entries(const GroupDesc& g) { return group_tiles(g, SPMM_ROWS_PER_WARP); }
 
-int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, int* counters, int* order,
-                          cudaStream_t s) {
+int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, int64_t entries, int* count,
+                          int* list, SpmmOrder* order, cudaStream_t s) {
+    *order = SpmmOrder{nullptr, nullptr, 0};
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
-    if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
+    if (groups >= (int64_t(1) << 30)) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
+    // heavy = several times the average group, and enough entries to be worth the detour
+    const int64_t heavy = std::max<int64_t>(128, 4 * ceil_div(entries, groups));
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, 256), 148 * 4);
-    { KernelScope ks(ctx, KC_INV_DEGREE, s); order_count_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, groups, counters); }
+    { KernelScope ks(ctx, KC_INV_DEGREE, s); heavy_list_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, groups, heavy, count, list); }
     RTMA_LAUNCH_CHECK(ctx);
-    { KernelScope ks(ctx, KC_INV_DEGREE, s); order_scatter_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, groups, counters, counters + ORDER_BUCKETS, order); }
-    RTMA_LAUNCH_CHECK(ctx);
+    *order = SpmmOrder{count, list, heavy};
     return RTMA_OK;
 }

@@ -238,7 +238,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             float* tile_loss = cur.take<float>((size_t)loss_tiles(g) + 4);
             int* ticket = cur.take<int>(64);  // work counter of the aggregation kernels (zero between launches)
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
-            int* spmm_order = cur.take<int>((size_t)spmm_order_entries(g) + 4);
+            int* heavy_list = cur.take<int>((size_t)spmm_order_entries(g) + 4);
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
             __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
             for (int l = 0; l < m.L; ++l) {
@@ -256,7 +256,10 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
 
             RTMA_CUDA(ctx, cudaMemsetAsync(ctx->arena + gi * share, 0, zero_bytes, s));
             RTMA_TRY(launch_inv_degree(ctx, g, rowptr_out, inv_deg, s));
-            RTMA_TRY(launch_spmm_order(ctx, g, rowptr_out, ticket + 16, spmm_order, s));
+            int64_t wave_entries = 0;
+            for (int k = 0; k < g.num; ++k) wave_entries += edge_offsets[g.part[k] + 1] - edge_offsets[g.part[k]];
+            SpmmOrder wave_order;
+            RTMA_TRY(launch_spmm_order(ctx, g, rowptr_out, wave_entries, ticket + 16, heavy_list, &wave_order, s));
             RTMA_TRY(launch_to_planes(ctx, g, Xp, m.dims[0], Hl[0], s));
             const Planes no_planes{nullptr, nullptr, 0};
             const Mat no_mat{nullptr, 0};
@@ -268,7 +271,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 // trainers reach the aggregation point with different step counts)
                 bool all_run = true;
                 for (int k = 0; k < wave.num; ++k) all_run = all_run && steps[wave.part[k]] > step;
-                const int* order = all_run ? spmm_order : nullptr;  // the order was built for the whole wave
+                const SpmmOrder order = all_run ? wave_order : SpmmOrder{nullptr, nullptr, 0};  // built for the whole wave
                 if (all_run) {
                     g = wave;
                     sp = wave_sp;

@@ -72,20 +72,26 @@ int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, int 
 int32_t launch_from_planes(rtma_ctx* ctx, Planes src, int64_t first_row, int64_t rows, int d, float* dst, cudaStream_t s);
 // inv_deg[row_ws + i] = 1 / local degree (0 for an isolated node).
 int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s);
-// Processing order of the aggregation kernels' row groups for group g, heaviest first:
-// order[spmm_order_entries(g)]; counters: 32 ints of scratch, zero on entry.
+// Processing order of the aggregation kernels' row groups (8 consecutive rows): the groups with at
+// least `heavy` entries, listed once per call, go first.  A zeroed SpmmOrder means plain row order.
+struct SpmmOrder {
+    const int* heavy_count;  // device: number of listed groups
+    const int* heavy_list;   // device: their indices
+    int64_t heavy;           // entries from which a group is listed
+};
+// list: spmm_order_entries(g) ints; count: one int, zero on entry; entries: kept entries of g's parts.
 int64_t spmm_order_entries(const GroupDesc& g);
-int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, int* counters, int* order,
-                          cudaStream_t s);
+int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, int64_t entries, int* count,
+                          int* list, SpmmOrder* order, cudaStream_t s);
 // out[r] = inv_deg[r] * sum_{u in N(r)} src[u]                      (forward, mean)
 // ticket: two ints of scratch, zero on entry and zero again when the kernel has finished.
-// order: from launch_spmm_order for this very g, or NULL (row order).
+// order: from launch_spmm_order for this very g, or zeroed.
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                         const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket,
+                         const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                          cudaStream_t s);
 // out[r] = sum_{u in N(r)} inv_deg[u] * src[u]                     (backward: Abar^T on a symmetric graph)
 int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
-                               const float* inv_deg, Planes src, Planes out, int d, const int* order, int* ticket,
+                               const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                                cudaStream_t s);
 
 // ---- loss.cu --------------------------------------------------------------------------
