@@ -233,6 +233,8 @@ def main():
     ap.add_argument("--scale", type=float, default=None, help="shrink (or grow) the workload's graph")
     ap.add_argument("--M", type=int, default=None, help="trainers (supertma / sweep)")
     ap.add_argument("--assign", default="super", choices=["node", "super"], help="sweep: assignment scheme")
+    ap.add_argument("--streams", type=int, default=1,
+                    help="CUDA streams the trainers are spread over (trainers sharing a stream are batched)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -268,6 +270,9 @@ def main():
     params = torch.empty(w.M, P, dtype=torch.float32, device=device)
     loss = torch.zeros(w.R, w.M, w.K, dtype=torch.float32, device=device)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)  # > 126 MB of L2
+    n_streams = max(1, min(args.streams, w.M))
+    pool = [torch.cuda.Stream(device=device) for _ in range(n_streams)] if n_streams > 1 else None
+    trainer_streams = [pool[i * n_streams // w.M] for i in range(w.M)] if pool else None
     state = {}
 
     def step():
@@ -279,8 +284,14 @@ def main():
         yp = ctx.gather_rows(d_y, perm)
         part_host = part_offsets.cpu().tolist()
         for r in range(w.R):
+            if pool:  # the trainers' streams start after the preprocessing / the previous aggregation
+                for st in pool:
+                    st.wait_stream(torch.cuda.current_stream())
             ctx.local_steps(w.dims, w.lr, w.M, part_host, edge_host, rowptr_out, col_out, Xp, yp, params, w.K,
-                            loss_out=loss[r], gemm_dtype=w.gemm_dtype)
+                            loss_out=loss[r], gemm_dtype=w.gemm_dtype, streams=trainer_streams)
+            if pool:
+                for st in pool:
+                    torch.cuda.current_stream().wait_stream(st)
             ctx.aggregate(params)
         state.update(part_host=part_host, edge_host=edge_host)
 
@@ -402,7 +413,8 @@ def main():
                    "dims": list(w.dims), "K": w.K, "R": w.R, "spmm_passes_per_local_step": passes,
                    "assignment": "super-node" if w.use_groups else "node",
                    "kept_fraction": kept / g.num_entries,
-                   "parallelism": "replicas only" if world > 1 else f"single GPU, {w.M} trainers batched on one stream",
+                   "parallelism": ("replicas only" if world > 1 else
+                                   f"single GPU, {w.M} trainers batched on {n_streams} stream(s)"),
                    "l2": "256 MB written between timed steps"},
         "trainer_steps_per_s": world * args.steps * trainer_steps / elapsed_s,
         "loss_first_last": [first_loss, final_loss],

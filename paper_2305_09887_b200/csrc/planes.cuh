@@ -20,9 +20,9 @@ struct Planes {
 inline size_t planes_ld(int64_t d) { return (size_t)((d + 7) / 8 * 8); }
 
 #ifdef __CUDACC__
-// Conversions are written with integer arithmetic on purpose: the dedicated conversion
-// instructions issue on the narrow special-function pipe, which became the limit of the
-// aggregation kernels.  Round-to-nearest-even; inputs are assumed finite.
+// fp32 -> bf16 bits in integer arithmetic (round-to-nearest-even; inputs are assumed finite), for
+// code whose conversion pipe is busy; Pack8::to_planes_cvt is the same split through the paired
+// conversion instruction.
 __device__ __forceinline__ uint32_t bf16_bits_rn(float x) {
     const uint32_t u = __float_as_uint(x);
     return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;

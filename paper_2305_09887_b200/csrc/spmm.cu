@@ -138,7 +138,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                     for (int e = 0; e < 8; ++e) acc[c].v[e] *= w;
                 }
                 uint4 h, l;
-                acc[c].to_planes(h, l);
+                acc[c].to_planes_cvt(h, l);
                 *reinterpret_cast<uint4*>(out.hi + r * out.ld + colx) = h;
                 *reinterpret_cast<uint4*>(out.lo + r * out.ld + colx) = l;
             }
