@@ -211,6 +211,119 @@ def local_steps(dims, lr, rowptr, col, X, y, params, K):
     return params, loss
 
 
+# ---- model variants: (encoder, act, norm); encoder 0 = GraphSAGE-mean, 1 = GCN; act 0 = ReLU,
+# 1 = PReLU; norm 0 = none, 1 = Layer Normalization before the activation -------------------
+SAGE_RELU = (0, 0, 0)
+
+
+def _variant(v):
+    return _i32(list(v))
+
+
+def variant_param_count(variant, dims) -> int:
+    d = _i32(dims)
+    f = lib().orc_variant_param_count
+    f.restype = ctypes.c_int64
+    return int(f(_p(_variant(variant), c_i32p), ctypes.c_int32(len(dims) - 1), _p(d, c_i32p)))
+
+
+def variant_layout(variant, dims):
+    """Per layer a dict of offsets into the flat parameter vector: w0, w1, bias, gamma, beta,
+    slope (-1 = absent).  GraphSAGE: w0 = Ws, w1 = Wn; GCN: w0 = W."""
+    L = len(dims) - 1
+    off = np.empty(6 * L, dtype=np.int64)
+    lib().orc_variant_layout(_p(_variant(variant), c_i32p), ctypes.c_int32(L), _p(_i32(dims), c_i32p), _p(off, c_i64p))
+    names = ("w0", "w1", "bias", "gamma", "beta", "slope")
+    return [dict(zip(names, (int(x) for x in off[6 * l:6 * l + 6]))) for l in range(L)]
+
+
+def variant_init_params(variant, dims, seed) -> np.ndarray:
+    """Xavier-uniform weights, zero biases, gamma = 1, beta = 0, PReLU slope = 0.25 (fp64)."""
+    rng = np.random.default_rng(seed)
+    P = variant_param_count(variant, dims)
+    p = np.zeros(P, dtype=np.float64)
+    for l, lay in enumerate(variant_layout(variant, dims)):
+        d_in, d_out = dims[l], dims[l + 1]
+        a = np.sqrt(6.0 / (d_in + d_out))
+        for key in ("w0", "w1"):
+            if lay[key] >= 0:
+                p[lay[key]:lay[key] + d_in * d_out] = rng.uniform(-a, a, size=d_in * d_out)
+        if lay["gamma"] >= 0:
+            p[lay["gamma"]:lay["gamma"] + d_out] = 1.0
+        if lay["slope"] >= 0:
+            p[lay["slope"]] = 0.25
+    return p
+
+
+def spmm_gcn(rowptr, col, H: np.ndarray) -> np.ndarray:
+    H = np.ascontiguousarray(H, dtype=np.float64)
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    n, d = rowptr.size - 1, H.shape[1]
+    N = np.empty((n, d), dtype=np.float64)
+    lib().orc_spmm_gcn_f64(ctypes.c_int64(n), _p(rowptr, c_i64p), _p(col, c_i32p), ctypes.c_int64(d),
+                           _p(H, c_f64p), _p(N, c_f64p))
+    return N
+
+
+def forward_backward_variant(variant, dims, rowptr, col, X, y, params, want_grads=True, want_acts=False,
+                             want_preact=False, gates=None):
+    """forward_backward for a model variant (fp64).  want_preact adds the activations' inputs
+    (after the normalisation, if any) of the hidden layers as "Z1".."Z{L-1}"."""
+    dt, ptr = np.float64, c_f64p
+    X = np.ascontiguousarray(X, dtype=dt)
+    params = np.ascontiguousarray(params, dtype=dt)
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    y = _i32(y)
+    n = rowptr.size - 1
+    d = _i32(dims)
+    assert params.size == variant_param_count(variant, dims)
+    grads = np.empty(params.size, dtype=dt) if want_grads else None
+    acts, layout = None, None
+    if want_acts:
+        layout, total = acts_layout(dims, n)
+        acts = np.empty(total, dtype=dt)
+    hidden = [n * dims[l + 1] for l in range(len(dims) - 2)]
+    preact = np.empty(sum(hidden), dtype=dt) if want_preact else None
+    gate_buf = None
+    if gates is not None:
+        gate_buf = np.concatenate([np.ascontiguousarray(g, dtype=np.int8).ravel() for g in gates]) if gates else \
+            np.empty(0, dtype=np.int8)
+        assert gate_buf.size == sum(hidden)
+    f = lib().orc_forward_backward_variant_f64
+    f.restype = ctypes.c_double
+    loss = f(_p(_variant(variant), c_i32p), ctypes.c_int32(len(dims) - 1), _p(d, c_i32p), ctypes.c_int64(n),
+             _p(rowptr, c_i64p), _p(col, c_i32p), _p(X, ptr), _p(y, c_i32p), _p(params, ptr), _p(grads, ptr),
+             _p(acts, ptr), _p(preact, ptr), _p(gate_buf, ctypes.POINTER(ctypes.c_int8)))
+    named = None
+    if want_acts or want_preact:
+        named = {}
+        if want_acts:
+            named.update({nm: acts[o:o + r * w].reshape(r, w) for nm, o, r, w in layout})
+        if want_preact:
+            off = 0
+            for l, size in enumerate(hidden):
+                named[f"Z{l + 1}"] = preact[off:off + size].reshape(n, dims[l + 1])
+                off += size
+    return float(loss), grads, named
+
+
+def local_steps_variant(variant, dims, lr, rowptr, col, X, y, params, K):
+    """K plain-SGD steps on one part for a model variant.  Returns (new params, loss[K])."""
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    params = np.array(params, dtype=np.float64, copy=True)
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    y = _i32(y)
+    loss = np.empty(K, dtype=np.float64)
+    lib().orc_local_steps_variant_f64(
+        _p(_variant(variant), c_i32p), ctypes.c_int32(len(dims) - 1), _p(_i32(dims), c_i32p), ctypes.c_double(lr),
+        ctypes.c_int64(rowptr.size - 1), _p(rowptr, c_i64p), _p(col, c_i32p), _p(X, c_f64p), _p(y, c_i32p),
+        _p(params, c_f64p), ctypes.c_int32(K), _p(loss, c_f64p))
+    return params, loss
+
+
 def average(params: np.ndarray):
     """params [M, P] -> (averaged copies [M, P], global [P])."""
     tag, ptr, dt = _fp(params.dtype)

@@ -21,6 +21,9 @@
 //   orc_local_steps       Algorithm 2's loop body with a plain SGD optimizer.
 //   orc_average           Algorithm 1's aggregation phi = plain average, then
 //                         Algorithm 2's overwrite of every local copy.
+//   orc_*_variant         the encoders the paper's experiments use (Sec. 4.1): GCN
+//                         (Kipf & Welling) or GraphSAGE-mean layers, PReLU, Layer
+//                         Normalization before the activation.
 //   orc_sigmoid_l2_grad   the 1-layer sigmoid / L2 model of Theorem 2, used
 //                         only to pin the aggregation against Eq.
 //                         (proof-2-exp-grad-central).
@@ -243,6 +246,318 @@ void local_steps(int32_t L, const int32_t* dims, double lr, int64_t n, const int
     }
 }
 
+// ---- model variants (Sec. 4.1 "GNN Encoders"): GCN or GraphSAGE-mean layers, ReLU or PReLU,
+// optional Layer Normalization before the activation ---------------------------------------
+//   GraphSAGE-mean  Z = H Ws + (A-bar H) Wn + b                       params: Ws, Wn, b
+//   GCN             Z = (A-hat H) W + b,  A-hat = D~^-1/2 (A + I) D~^-1/2, D~ = local degree + 1
+//                   (Kipf & Welling's renormalised adjacency)         params: W, b
+//   hidden layers   U = gamma * (Z - mean) / sqrt(var + eps) + beta over the row's features
+//                   (Ba et al.; biased variance, eps = 1e-5)          params: gamma, beta
+//                   H = U if U > 0 else a * U (PReLU, one learnable slope per layer; He et al.)
+//                                                                     params: a
+// The last layer has neither normalisation nor activation.  Parameter order inside a layer:
+// weights, b, [gamma, beta], [a].
+struct Variant {
+    int32_t encoder;  // 0 GraphSAGE-mean, 1 GCN
+    int32_t act;      // 0 ReLU, 1 PReLU
+    int32_t norm;     // 0 none, 1 Layer Normalization before the activation
+};
+constexpr double LN_EPS = 1e-5;
+
+struct VLayer {
+    int64_t d_in, d_out;
+    int64_t w0, w1, bias, gamma, beta, slope;  // offsets; -1 = absent
+};
+
+std::vector<VLayer> variant_layers(const Variant& m, int32_t L, const int32_t* dims, int64_t* total) {
+    std::vector<VLayer> v(L);
+    int64_t off = 0;
+    for (int32_t l = 0; l < L; ++l) {
+        VLayer& x = v[l];
+        x.d_in = dims[l];
+        x.d_out = dims[l + 1];
+        x.w0 = off;
+        off += x.d_in * x.d_out;
+        x.w1 = -1;
+        if (m.encoder == 0) {
+            x.w1 = off;
+            off += x.d_in * x.d_out;
+        }
+        x.bias = off;
+        off += x.d_out;
+        x.gamma = x.beta = x.slope = -1;
+        if (l < L - 1 && m.norm == 1) {
+            x.gamma = off;
+            off += x.d_out;
+            x.beta = off;
+            off += x.d_out;
+        }
+        if (l < L - 1 && m.act == 1) {
+            x.slope = off;
+            off += 1;
+        }
+    }
+    *total = off;
+    return v;
+}
+
+// N = A-hat H:  N[v] = s_v * (s_v H[v] + sum_{u in row v} s_u H[u]),  s_v = (deg(v) + 1)^-1/2
+template <class T>
+void spmm_gcn(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, const T* H, T* N) {
+    std::vector<double> acc(d);
+    for (int64_t v = 0; v < n; ++v) {
+        const double sv = 1.0 / std::sqrt((double)(rowptr[v + 1] - rowptr[v] + 1));
+        for (int64_t j = 0; j < d; ++j) acc[j] = sv * (double)H[v * d + j];
+        for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+            const int64_t u = col[e];
+            const double su = 1.0 / std::sqrt((double)(rowptr[u + 1] - rowptr[u] + 1));
+            for (int64_t j = 0; j < d; ++j) acc[j] += su * (double)H[u * d + j];
+        }
+        for (int64_t j = 0; j < d; ++j) N[v * d + j] = (T)(sv * acc[j]);
+    }
+}
+
+// Same outputs and conventions as forward_backward; preact holds U (the activation's input) of
+// the hidden layers; gates override the branch U > 0 of single units (see forward_backward).
+template <class T>
+double forward_backward_variant(const Variant& m, int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
+                                const int32_t* col, const T* X, const int32_t* y, const T* params, T* grads,
+                                T* acts, T* preact, const int8_t* gates) {
+    int64_t P = 0;
+    const std::vector<VLayer> lv = variant_layers(m, L, dims, &P);
+    if (grads) for (int64_t i = 0; i < P; ++i) grads[i] = (T)0;
+    if (n == 0) return 0.0;
+
+    std::vector<std::vector<T>> H(L + 1), N(L), Z(L), U(L), XH(L);   // XH = normalised Z
+    std::vector<std::vector<double>> rstd(L);
+    std::vector<std::vector<char>> open(L);
+    std::vector<int64_t> gate_off(L, 0);
+    for (int32_t l = 1; l < L; ++l) gate_off[l] = gate_off[l - 1] + n * lv[l - 1].d_out;
+    H[0].assign(X, X + n * lv[0].d_in);
+    for (int32_t l = 0; l < L; ++l) {
+        const int64_t di = lv[l].d_in, dn = lv[l].d_out;
+        const bool hidden = l < L - 1;
+        N[l].resize(n * di);
+        if (m.encoder == 0) spmm_mean<T>(n, rowptr, col, di, H[l].data(), N[l].data());
+        else spmm_gcn<T>(n, rowptr, col, di, H[l].data(), N[l].data());
+        Z[l].resize(n * dn);
+        U[l].resize(n * dn);
+        H[l + 1].resize(n * dn);
+        open[l].assign(n * dn, 1);
+        if (hidden && m.norm == 1) {
+            XH[l].resize(n * dn);
+            rstd[l].resize(n);
+        }
+        const T* W0 = params + lv[l].w0;
+        const T* W1 = lv[l].w1 >= 0 ? params + lv[l].w1 : nullptr;
+        const T* b = params + lv[l].bias;
+        const double slope = !hidden ? 1.0 : (m.act == 1 ? (double)params[lv[l].slope] : 0.0);
+        std::vector<double> acc(dn);
+        for (int64_t v = 0; v < n; ++v) {
+            for (int64_t j = 0; j < dn; ++j) acc[j] = (double)b[j];
+            for (int64_t k = 0; k < di; ++k) {
+                // GraphSAGE: self term on W0, neighbour term on W1; GCN: the aggregate on W0
+                const double a0 = m.encoder == 0 ? (double)H[l][v * di + k] : (double)N[l][v * di + k];
+                const double a1 = m.encoder == 0 ? (double)N[l][v * di + k] : 0.0;
+                const T* w0 = W0 + k * dn;
+                for (int64_t j = 0; j < dn; ++j) acc[j] += a0 * (double)w0[j];
+                if (W1) {
+                    const T* w1 = W1 + k * dn;
+                    for (int64_t j = 0; j < dn; ++j) acc[j] += a1 * (double)w1[j];
+                }
+            }
+            for (int64_t j = 0; j < dn; ++j) Z[l][v * dn + j] = (T)acc[j];
+            if (!hidden) {
+                for (int64_t j = 0; j < dn; ++j) U[l][v * dn + j] = H[l + 1][v * dn + j] = Z[l][v * dn + j];
+                continue;
+            }
+            if (m.norm == 1) {
+                double mean = 0.0, var = 0.0;
+                for (int64_t j = 0; j < dn; ++j) mean += (double)Z[l][v * dn + j];
+                mean /= (double)dn;
+                for (int64_t j = 0; j < dn; ++j) {
+                    const double c = (double)Z[l][v * dn + j] - mean;
+                    var += c * c;
+                }
+                var /= (double)dn;
+                const double rs = 1.0 / std::sqrt(var + LN_EPS);
+                rstd[l][v] = rs;
+                const T* gamma = params + lv[l].gamma;
+                const T* beta = params + lv[l].beta;
+                for (int64_t j = 0; j < dn; ++j) {
+                    const double xh = ((double)Z[l][v * dn + j] - mean) * rs;
+                    XH[l][v * dn + j] = (T)xh;
+                    U[l][v * dn + j] = (T)((double)gamma[j] * xh + (double)beta[j]);
+                }
+            } else {
+                for (int64_t j = 0; j < dn; ++j) U[l][v * dn + j] = Z[l][v * dn + j];
+            }
+            for (int64_t j = 0; j < dn; ++j) {
+                const T u = U[l][v * dn + j];
+                const int8_t forced = gates ? gates[gate_off[l] + v * dn + j] : (int8_t)-1;
+                const bool is_open = forced < 0 ? (u > (T)0) : (forced != 0);
+                open[l][v * dn + j] = is_open ? 1 : 0;
+                H[l + 1][v * dn + j] = is_open ? u : (T)(slope * (double)u);
+            }
+        }
+    }
+    if (preact)
+        for (int32_t l = 0; l + 1 < L; ++l) std::memcpy(preact + gate_off[l], U[l].data(), sizeof(T) * U[l].size());
+    if (acts) {
+        T* a = acts;
+        for (int32_t l = 0; l < L; ++l) {
+            std::memcpy(a, N[l].data(), sizeof(T) * N[l].size());
+            a += N[l].size();
+            std::memcpy(a, H[l + 1].data(), sizeof(T) * H[l + 1].size());
+            a += H[l + 1].size();
+        }
+    }
+
+    // Softmax cross-entropy, mean over the part's nodes.
+    const int64_t C = lv[L - 1].d_out;
+    std::vector<T> dZ(n * C);
+    double loss = 0.0;
+    for (int64_t v = 0; v < n; ++v) {
+        const T* z = &Z[L - 1][v * C];
+        double zmax = (double)z[0];
+        for (int64_t c = 1; c < C; ++c) zmax = std::fmax(zmax, (double)z[c]);
+        double s = 0.0;
+        for (int64_t c = 0; c < C; ++c) s += std::exp((double)z[c] - zmax);
+        const double lse = zmax + std::log(s);
+        loss += lse - (double)z[y[v]];
+        for (int64_t c = 0; c < C; ++c) {
+            const double p = std::exp((double)z[c] - lse);
+            dZ[v * C + c] = (T)((p - (c == y[v] ? 1.0 : 0.0)) / (double)n);
+        }
+    }
+    loss /= (double)n;
+    if (!grads) return loss;
+
+    for (int32_t l = L - 1; l >= 0; --l) {
+        const int64_t di = lv[l].d_in, dn = lv[l].d_out;
+        const T* W0 = params + lv[l].w0;
+        const T* W1 = lv[l].w1 >= 0 ? params + lv[l].w1 : nullptr;
+        {   // weight gradients: (input of each weight matrix)^T dZ; db = column sums of dZ
+            std::vector<double> g0(di * dn, 0.0), g1(W1 ? di * dn : 0, 0.0), gb(dn, 0.0);
+            for (int64_t v = 0; v < n; ++v) {
+                const T* dz = &dZ[v * dn];
+                for (int64_t j = 0; j < dn; ++j) gb[j] += (double)dz[j];
+                for (int64_t k = 0; k < di; ++k) {
+                    const double a0 = m.encoder == 0 ? (double)H[l][v * di + k] : (double)N[l][v * di + k];
+                    double* r0 = &g0[k * dn];
+                    for (int64_t j = 0; j < dn; ++j) r0[j] += a0 * (double)dz[j];
+                    if (W1) {
+                        const double a1 = (double)N[l][v * di + k];
+                        double* r1 = &g1[k * dn];
+                        for (int64_t j = 0; j < dn; ++j) r1[j] += a1 * (double)dz[j];
+                    }
+                }
+            }
+            for (int64_t i = 0; i < di * dn; ++i) grads[lv[l].w0 + i] = (T)g0[i];
+            if (W1) for (int64_t i = 0; i < di * dn; ++i) grads[lv[l].w1 + i] = (T)g1[i];
+            for (int64_t j = 0; j < dn; ++j) grads[lv[l].bias + j] = (T)gb[j];
+        }
+        if (l == 0) break;
+        // gradient with respect to this layer's input H^l
+        std::vector<double> dH(n * di, 0.0);
+        std::vector<double> dN(di);
+        for (int64_t v = 0; v < n; ++v) {
+            const T* dz = &dZ[v * dn];
+            for (int64_t k = 0; k < di; ++k) {
+                double s = 0.0, t = 0.0;
+                for (int64_t j = 0; j < dn; ++j) {
+                    s += (double)dz[j] * (double)W0[k * dn + j];
+                    if (W1) t += (double)dz[j] * (double)W1[k * dn + j];
+                }
+                if (m.encoder == 0) {
+                    dH[v * di + k] += s;          // self term
+                    dN[k] = (double)(T)t;         // gradient of the aggregate
+                } else {
+                    dN[k] = (double)(T)s;
+                }
+            }
+            if (m.encoder == 0) {
+                const int64_t deg = rowptr[v + 1] - rowptr[v];
+                for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+                    double* dst = &dH[(int64_t)col[e] * di];
+                    for (int64_t k = 0; k < di; ++k) dst[k] += dN[k] / (double)deg;
+                }
+            } else {
+                // transpose of spmm_gcn, entry by entry
+                const double sv = 1.0 / std::sqrt((double)(rowptr[v + 1] - rowptr[v] + 1));
+                for (int64_t k = 0; k < di; ++k) dH[v * di + k] += sv * sv * dN[k];
+                for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+                    const int64_t u = col[e];
+                    const double su = 1.0 / std::sqrt((double)(rowptr[u + 1] - rowptr[u] + 1));
+                    double* dst = &dH[u * di];
+                    for (int64_t k = 0; k < di; ++k) dst[k] += sv * su * dN[k];
+                }
+            }
+        }
+        // back through the activation and the normalisation of layer l-1 (whose output is H^l)
+        const int32_t q = l - 1;
+        const double slope = m.act == 1 ? (double)params[lv[q].slope] : 0.0;
+        std::vector<T> dZprev(n * di);
+        std::vector<double> g_gamma(m.norm == 1 ? di : 0, 0.0), g_beta(m.norm == 1 ? di : 0, 0.0);
+        double g_slope = 0.0;
+        std::vector<double> dU(di);
+        for (int64_t v = 0; v < n; ++v) {
+            for (int64_t k = 0; k < di; ++k) {
+                const int64_t i = v * di + k;
+                const double g = (double)(T)dH[i];
+                if (open[q][i]) {
+                    dU[k] = g;
+                } else {
+                    dU[k] = slope * g;
+                    g_slope += g * (double)U[q][i];
+                }
+            }
+            if (m.norm == 1) {
+                const T* gamma = params + lv[q].gamma;
+                double m1 = 0.0, m2 = 0.0;
+                for (int64_t k = 0; k < di; ++k) {
+                    const double xh = (double)XH[q][v * di + k];
+                    g_gamma[k] += dU[k] * xh;
+                    g_beta[k] += dU[k];
+                    const double dx = dU[k] * (double)gamma[k];
+                    m1 += dx;
+                    m2 += dx * xh;
+                }
+                m1 /= (double)di;
+                m2 /= (double)di;
+                for (int64_t k = 0; k < di; ++k) {
+                    const double xh = (double)XH[q][v * di + k];
+                    const double dx = dU[k] * (double)gamma[k];
+                    dZprev[v * di + k] = (T)(rstd[q][v] * (dx - m1 - xh * m2));
+                }
+            } else {
+                for (int64_t k = 0; k < di; ++k) dZprev[v * di + k] = (T)dU[k];
+            }
+        }
+        if (m.norm == 1) {
+            for (int64_t k = 0; k < di; ++k) grads[lv[q].gamma + k] = (T)g_gamma[k];
+            for (int64_t k = 0; k < di; ++k) grads[lv[q].beta + k] = (T)g_beta[k];
+        }
+        if (m.act == 1) grads[lv[q].slope] = (T)g_slope;
+        dZ.swap(dZprev);
+    }
+    return loss;
+}
+
+template <class T>
+void local_steps_variant(const Variant& m, int32_t L, const int32_t* dims, double lr, int64_t n, const int64_t* rowptr,
+                         const int32_t* col, const T* X, const int32_t* y, T* params, int32_t K, double* loss_out) {
+    int64_t P = 0;
+    variant_layers(m, L, dims, &P);
+    std::vector<T> g(P);
+    for (int32_t k = 0; k < K; ++k) {
+        const double loss = forward_backward_variant<T>(m, L, dims, n, rowptr, col, X, y, params, g.data(), nullptr,
+                                                        nullptr, nullptr);
+        if (loss_out) loss_out[k] = loss;
+        for (int64_t i = 0; i < P; ++i) params[i] = (T)((double)params[i] - lr * (double)g[i]);
+    }
+}
+
 template <class T>
 void average(T* params, int64_t P, int32_t M, T* global_out) {
     for (int64_t j = 0; j < P; ++j) {
@@ -356,6 +671,38 @@ void orc_local_steps_f64(int32_t L, const int32_t* dims, double lr, int64_t n, c
 
 void orc_average_f32(float* params, int64_t P, int32_t M, float* global_out) { average<float>(params, P, M, global_out); }
 void orc_average_f64(double* params, int64_t P, int32_t M, double* global_out) { average<double>(params, P, M, global_out); }
+
+// ---- model variants: variant = {encoder, act, norm} ------------------------------------------
+int64_t orc_variant_param_count(const int32_t* variant, int32_t L, const int32_t* dims) {
+    int64_t P = 0;
+    variant_layers(Variant{variant[0], variant[1], variant[2]}, L, dims, &P);
+    return P;
+}
+// offsets[l * 6 + {0..5}] = w0, w1, bias, gamma, beta, slope of layer l (-1 = absent)
+void orc_variant_layout(const int32_t* variant, int32_t L, const int32_t* dims, int64_t* offsets) {
+    int64_t P = 0;
+    const std::vector<VLayer> lv = variant_layers(Variant{variant[0], variant[1], variant[2]}, L, dims, &P);
+    for (int32_t l = 0; l < L; ++l) {
+        const int64_t o[6] = {lv[l].w0, lv[l].w1, lv[l].bias, lv[l].gamma, lv[l].beta, lv[l].slope};
+        for (int i = 0; i < 6; ++i) offsets[l * 6 + i] = o[i];
+    }
+}
+void orc_spmm_gcn_f64(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, const double* H, double* N) {
+    spmm_gcn<double>(n, rowptr, col, d, H, N);
+}
+double orc_forward_backward_variant_f64(const int32_t* variant, int32_t L, const int32_t* dims, int64_t n,
+                                        const int64_t* rowptr, const int32_t* col, const double* X, const int32_t* y,
+                                        const double* params, double* grads, double* acts, double* preact,
+                                        const int8_t* gates) {
+    return forward_backward_variant<double>(Variant{variant[0], variant[1], variant[2]}, L, dims, n, rowptr, col, X, y,
+                                            params, grads, acts, preact, gates);
+}
+void orc_local_steps_variant_f64(const int32_t* variant, int32_t L, const int32_t* dims, double lr, int64_t n,
+                                 const int64_t* rowptr, const int32_t* col, const double* X, const int32_t* y,
+                                 double* params, int32_t K, double* loss_out) {
+    local_steps_variant<double>(Variant{variant[0], variant[1], variant[2]}, L, dims, lr, n, rowptr, col, X, y, params, K,
+                                loss_out);
+}
 
 // Theorem 2's model: z_v = sigmoid((A-bar X w)_v), L = 1/2 (y_v - z_v)^2 per
 // node.  Writes the per-node gradient dL/dw [n x d] (Eq. (proof-2-grad)).
