@@ -135,12 +135,26 @@ int32_t rtma_gather_rows(rtma_ctx* ctx, int64_t n, int64_t row_bytes, const void
  * row-normalised adjacency (Theorem 2): the mean over LOCAL neighbours, zero for a node
  * without any.  dims[0] = feature width, dims[L] = number of classes.
  * Parameters of one trainer: flat float vector of rtma_param_count() entries, layer after
- * layer: Ws[d_l][d_{l+1}], Wn[d_l][d_{l+1}], b[d_{l+1}], all row-major.                    */
+ * layer: Ws[d_l][d_{l+1}], Wn[d_l][d_{l+1}], b[d_{l+1}], all row-major.
+ *
+ * Variants (Sec. 4.1 "GNN Encoders": GCN or GraphSAGE encoders, PReLU, Layer Normalization
+ * before the activation), all zero = the model above:
+ *   encoder = 1  GCN layers, Z^l = (Ahat H^l) W^l + b^l with Ahat = D~^-1/2 (A + I) D~^-1/2,
+ *                D~ = local degree + 1 (Kipf & Welling's renormalised adjacency); one weight
+ *                matrix W[d_l][d_{l+1}] per layer instead of Ws, Wn.
+ *   norm = 1     hidden layers: U = gamma * (Z - mean) / sqrt(var + 1e-5) + beta over the row's
+ *                features (biased variance), parameters gamma[d_{l+1}], beta[d_{l+1}].
+ *   act = 1      hidden layers: H = U if U > 0 else a * U, one learnable slope a per layer.
+ * The last layer has neither.  Parameter order inside a layer: weight matrices, b, then
+ * (hidden layers only) gamma, beta if norm = 1, then a if act = 1.                          */
 typedef struct {
     int32_t L;
     int32_t dims[RTMA_MAX_LAYERS + 1];
     int32_t gemm_dtype; /* 0: fp32-accurate products; 1: bf16 operands, fp32 accumulate   */
     float lr;
+    int32_t encoder;    /* 0: GraphSAGE-mean; 1: GCN                                        */
+    int32_t act;        /* 0: ReLU; 1: PReLU                                                */
+    int32_t norm;       /* 0: none; 1: Layer Normalization before the activation            */
 } rtma_model_desc;
 
 int64_t rtma_param_count(const rtma_model_desc* model);
@@ -218,7 +232,7 @@ int32_t rtma_sgd_aggregate(rtma_ctx* ctx, float* params, const float* grads, flo
  * summed per class (ms [RTMA_KERNEL_CLASSES], milliseconds; zeros if profiling was off) and the
  * launch counts (launches [RTMA_KERNEL_CLASSES]) since the previous read, and resets both.
  * Either output may be NULL.  The paper has no counterpart; these feed the roofline report.  */
-#define RTMA_KERNEL_CLASSES 19
+#define RTMA_KERNEL_CLASSES 20
 int32_t rtma_profile(rtma_ctx* ctx, int32_t enable);
 int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launches);
 const char* rtma_kernel_class_name(int32_t cls);

@@ -24,7 +24,7 @@ EXPORTS = (
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
     "rtma_local_steps_var", "rtma_aggregate_masked",
 )
-KERNEL_CLASSES = 19
+KERNEL_CLASSES = 20
 
 _lib = None
 
@@ -35,7 +35,8 @@ class RtmaError(RuntimeError):
 
 class ModelDesc(ctypes.Structure):
     _fields_ = [("L", ctypes.c_int32), ("dims", ctypes.c_int32 * (MAX_LAYERS + 1)),
-                ("gemm_dtype", ctypes.c_int32), ("lr", ctypes.c_float)]
+                ("gemm_dtype", ctypes.c_int32), ("lr", ctypes.c_float), ("encoder", ctypes.c_int32),
+                ("act", ctypes.c_int32), ("norm", ctypes.c_int32)]
 
 
 class Taps(ctypes.Structure):
@@ -61,7 +62,7 @@ def load_library():
     return _lib
 
 
-def model_desc(dims, lr: float = 0.01, gemm_dtype: int = 0) -> ModelDesc:
+def model_desc(dims, lr: float = 0.01, gemm_dtype: int = 0, variant=(0, 0, 0)) -> ModelDesc:
     L = len(dims) - 1
     if not 1 <= L <= MAX_LAYERS:
         raise ValueError(f"number of layers {L} outside [1, {MAX_LAYERS}]")
@@ -71,11 +72,12 @@ def model_desc(dims, lr: float = 0.01, gemm_dtype: int = 0) -> ModelDesc:
         md.dims[i] = int(d)
     md.gemm_dtype = int(gemm_dtype)
     md.lr = float(lr)
+    md.encoder, md.act, md.norm = (int(v) for v in variant)
     return md
 
 
-def param_count(dims) -> int:
-    return int(load_library().rtma_param_count(ctypes.byref(model_desc(dims))))
+def param_count(dims, variant=(0, 0, 0)) -> int:
+    return int(load_library().rtma_param_count(ctypes.byref(model_desc(dims, variant=variant))))
 
 
 def _ptr(t):
@@ -235,13 +237,15 @@ class Context:
 
     # ---- Algorithm 2 ----------------------------------------------------------------
     def local_steps(self, dims, lr, M, part_offsets_host, edge_offsets_host, rowptr_out, col_out, Xp, yp,
-                    params, K, loss_out=None, streams=None, gemm_dtype=0, taps=None, symmetric=True):
+                    params, K, loss_out=None, streams=None, gemm_dtype=0, taps=None, symmetric=True,
+                    variant=(0, 0, 0)):
         """K SGD steps on each of the M parts, in place on params [M, P].  K: an int, or a sequence
         of M per-trainer step counts (0 = the trainer does not run; rtma_local_steps_var).
         streams: None (all trainers on the current stream), or a list of M torch streams.
-        taps: None or (acts tensor or None, grads tensor or None, step)."""
+        taps: None or (acts tensor or None, grads tensor or None, step).
+        variant: (encoder, act, norm) of rtma_model_desc."""
         dev = self.device
-        md = model_desc(dims, lr, gemm_dtype)
+        md = model_desc(dims, lr, gemm_dtype, variant)
         _need(params, torch.float32, "params", dev)
         _need(Xp, torch.float32, "Xp", dev)
         _need(yp, torch.int32, "yp", dev)

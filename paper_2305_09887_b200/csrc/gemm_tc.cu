@@ -86,7 +86,7 @@ tc_weight_prep_kernel(const __grid_constant__ GroupDesc g, const PrepArgs a, con
         __nv_bfloat16 *hi, *lo;
         if (i < nf) {
             const int n = (int)(i / a.Kf), kk = (int)(i % a.Kf);
-            const int half = a.Kf / 2;
+            const int half = a.Kf / a.ls.nsrc;  // one block of K per weight matrix
             const int src = kk < half ? kk : kk - half;
             if (n < d_out && src < d_in) x = W[(int64_t)(kk < half ? src : d_in + src) * d_out + n];
             hi = a.Bf_hi + (int64_t)k * nf + i;
@@ -94,7 +94,7 @@ tc_weight_prep_kernel(const __grid_constant__ GroupDesc g, const PrepArgs a, con
         } else {
             const int64_t ii = i - nf;
             const int j = (int)(ii / a.Kd), kk = (int)(ii % a.Kd);
-            const int half = a.Kd / 2;
+            const int half = a.Kd / a.ls.nsrc;
             const int c = kk < half ? kk : kk - half;
             if (j < d_in && c < d_out) x = W[(int64_t)(kk < half ? j : d_in + j) * d_out + c];
             hi = a.Bd_hi + (int64_t)k * nd + ii;
@@ -397,7 +397,7 @@ struct WgradArgs {
     GroupDesc g;
     SplitPlan sp;
     CUtensorMap mapHh, mapHl, mapNh, mapNl, mapZh, mapZl;
-    int d_in, d_out;
+    int d_in, d_out, nsrc;
     int jt_per_src;   // 128-wide tiles over d_in, per source
     int n_atoms;      // 64-wide atoms over d_out (all column tiles together); a tile takes up to 4
     int tmem_cols, stages;
@@ -423,7 +423,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cbase = blockIdx.z * 256;                       // first output column of this tile
     const int ccount = min(256, d_out - cbase);               // valid columns in it
-    float* P = a.partial + (int64_t)slot * (2 * d_in + 1) * d_out;
+    float* P = a.partial + (int64_t)slot * (a.nsrc * d_in + 1) * d_out;
 
     const bool bias_tile = blockIdx.x == 0;  // these blocks also produce the bias gradient of their columns
 
@@ -433,7 +433,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
             if (j < d_in) P[(int64_t)(src * d_in + j) * d_out + cbase + idx % ccount] = 0.f;
         }
         if (bias_tile)
-            for (int c = threadIdx.x; c < ccount; c += TC_THREADS) P[(int64_t)2 * d_in * d_out + cbase + c] = 0.f;
+            for (int c = threadIdx.x; c < ccount; c += TC_THREADS) P[(int64_t)a.nsrc * d_in * d_out + cbase + c] = 0.f;
         return;
     }
 
@@ -569,7 +569,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                 const int t = c >> 6, lc = (c & 63) >> 3, e = c & 7;
                 float sum = 0.f;
                 for (int h = 0; h < 16; ++h) sum += red[(h * 8 + (lc ^ (h & 7))) * 32 + t * 8 + e];  // fixed order
-                P[(int64_t)2 * d_in * d_out + cbase + c] = sum;
+                P[(int64_t)a.nsrc * d_in * d_out + cbase + c] = sum;
             }
         }
         if (ok) {
@@ -673,11 +673,11 @@ bool make_tensor_map_bf16(CUtensorMap* out, const void* base, uint64_t rows, uin
 
 TcLayerPlan tc_plan_layer(LayerShape ls) {
     TcLayerPlan p{};
-    p.Kf = 2 * TC_BK * (int)ceil_div(ls.d_in, TC_BK);
+    p.Kf = ls.nsrc * TC_BK * (int)ceil_div(ls.d_in, TC_BK);
     int tiles = (int)ceil_div(ls.d_out, 256);
     p.BN_f = (int)ceil_div(ceil_div(ls.d_out, tiles), 16) * 16;
     p.Npad_f = p.BN_f * tiles;
-    p.Kd = 2 * TC_BK * (int)ceil_div(ls.d_out, TC_BK);
+    p.Kd = ls.nsrc * TC_BK * (int)ceil_div(ls.d_out, TC_BK);
     tiles = (int)ceil_div(ls.d_in, 256);
     p.BN_d = (int)ceil_div(ceil_div(ls.d_in, tiles), 16) * 16;
     p.Npad_d = p.BN_d * tiles;
@@ -742,7 +742,14 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
         !make_tensor_map_bf16(&a.mapBh, Bf_hi, (uint64_t)g.num * p.Npad_f, p.Kf, p.Kf, TC_BK, p.BN_f) ||
         !make_tensor_map_bf16(&a.mapBl, Bf_lo, (uint64_t)g.num * p.Npad_f, p.Kf, p.Kf, TC_BK, p.BN_f))
         return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the forward operands");
-    a.kb0 = a.kb1 = p.Kf / (2 * TC_BK);
+    if (ls.nsrc == 2) {
+        a.kb0 = a.kb1 = p.Kf / (2 * TC_BK);
+    } else {  // one weight matrix: the aggregate is the only operand
+        a.mapA0h = a.mapA1h;
+        a.mapA0l = a.mapA1l;
+        a.kb0 = p.Kf / TC_BK;
+        a.kb1 = 0;
+    }
     a.BN = p.BN_f;
     a.Npad = p.Npad_f;
     a.N = ls.d_out;
@@ -751,15 +758,15 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
     a.ld_out = out_f32.ld;
     a.params = params;
     a.P = ls.P;
-    a.bias_offset = ls.param_offset + (int64_t)2 * ls.d_in * ls.d_out;
+    a.bias_offset = ls.param_offset + (int64_t)ls.nsrc * ls.d_in * ls.d_out;
     a.relu = relu ? 1 : 0;
     a.gate_hi = nullptr;
     return launch_rows(ctx, a, KC_GEMM_FWD, s);
 }
 
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
-                        Planes dZ, Planes Q, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, Planes H, bool single,
-                        cudaStream_t s) {
+                        Planes dZ, Planes Q, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, Planes H, bool gate,
+                        bool single, cudaStream_t s) {
     RowsArgs a{};
     a.g = g;
     a.single = single ? 1 : 0;
@@ -768,7 +775,14 @@ int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const 
         !make_tensor_map_bf16(&a.mapBh, Bd_hi, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d) ||
         !make_tensor_map_bf16(&a.mapBl, Bd_lo, (uint64_t)g.num * p.Npad_d, p.Kd, p.Kd, TC_BK, p.BN_d))
         return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the dgrad operands");
-    a.kb0 = a.kb1 = p.Kd / (2 * TC_BK);
+    if (ls.nsrc == 2) {
+        a.kb0 = a.kb1 = p.Kd / (2 * TC_BK);
+    } else {
+        a.mapA0h = a.mapA1h;
+        a.mapA0l = a.mapA1l;
+        a.kb0 = p.Kd / TC_BK;
+        a.kb1 = 0;
+    }
     a.BN = p.BN_d;
     a.Npad = p.Npad_d;
     a.N = ls.d_in;
@@ -779,7 +793,7 @@ int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const 
     a.P = 0;
     a.bias_offset = -1;
     a.relu = 0;
-    a.gate_hi = H.hi;
+    a.gate_hi = gate ? H.hi : nullptr;
     return launch_rows(ctx, a, KC_GEMM_DGRAD, s);
 }
 
@@ -802,6 +816,11 @@ int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, 
         return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the wgrad operands");
     a.d_in = ls.d_in;
     a.d_out = ls.d_out;
+    a.nsrc = ls.nsrc;
+    if (ls.nsrc == 1) {  // the aggregate is the only source
+        a.mapHh = a.mapNh;
+        a.mapHl = a.mapNl;
+    }
     a.jt_per_src = (int)ceil_div(ls.d_in, TC_BM);
     a.n_atoms = (int)ceil_div(ls.d_out, 64);
     const int tile_atoms = a.n_atoms < 4 ? a.n_atoms : 4;
@@ -811,7 +830,7 @@ int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, 
     a.stages = stages_for(stage_bytes, MAX_STAGES);
     a.partial = partial;
     a.error_word = ctx->error_word;
-    dim3 grid((unsigned)(2 * a.jt_per_src), (unsigned)slots, (unsigned)ceil_div(a.n_atoms, 4));
+    dim3 grid((unsigned)(ls.nsrc * a.jt_per_src), (unsigned)slots, (unsigned)ceil_div(a.n_atoms, 4));
     { KernelScope ks(ctx, KC_GEMM_WGRAD, s); tc_wgrad_kernel<<<grid, TC_THREADS, a.stages * stage_bytes + 1024, s>>>(a); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;

@@ -13,7 +13,7 @@ reduce_sgd_kernel(const __grid_constant__ GroupDesc g, const __grid_constant__ S
                   const float* __restrict__ partial, const float lr, float* __restrict__ params,
                   float* __restrict__ grads_record) {
     const int k = blockIdx.y;
-    const int64_t count = (int64_t)(2 * ls.d_in + 1) * ls.d_out;  // Ws, Wn and the bias row
+    const int64_t count = (int64_t)(ls.nsrc * ls.d_in + 1) * ls.d_out;  // the weight matrices and the bias row
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (i >= count) return;
     float gsum = 0.f;
@@ -117,7 +117,7 @@ int32_t aggregate_impl(rtma_ctx* ctx, float* params, const float* grads, float l
 int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, const float* partial,
                           float lr, float* params, float* grads_record, cudaStream_t s) {
     if (g.num == 0) return RTMA_OK;
-    const int64_t count = (int64_t)(2 * ls.d_in + 1) * ls.d_out;
+    const int64_t count = (int64_t)(ls.nsrc * ls.d_in + 1) * ls.d_out;
     dim3 grid((unsigned)ceil_div(count, 256), (unsigned)g.num);
     { KernelScope ks(ctx, KC_REDUCE_SGD, s); reduce_sgd_kernel<<<grid, 256, 0, s>>>(g, sp, ls, partial, lr, params, grads_record); }
     RTMA_LAUNCH_CHECK(ctx);

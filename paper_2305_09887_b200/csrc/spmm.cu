@@ -5,6 +5,9 @@
 // Forward:  N[v] = (1/deg v) sum_{u in N(v)} H[u]           (Abar H: weight on the destination)
 // Backward: Q[v] = sum_{u in N(v)} (1/deg u) dZ[u]          (Abar^T dZ on a symmetric graph: weight
 //           on the source), so that dH = [dZ | Q] [Ws^T ; Wn^T] is one product.
+// GCN:      N[v] = s_v (s_v H[v] + sum_{u in N(v)} s_u H[u]), s = (deg + 1)^-1/2: the renormalised
+//           adjacency D~^-1/2 (A + I) D~^-1/2 of Kipf & Welling, symmetric, so the same kernel
+//           serves the backward pass.
 //
 // Gather-bound and, at the tiny local degrees random partitioning leaves (about deg/M),
 // latency-bound: a warp takes 8 consecutive rows at a time, reads their offsets with one load and their
@@ -29,6 +32,17 @@ inv_degree_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict
     const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
     const int64_t deg = rp[i + 1] - rp[i];
     inv_deg[g.row_ws[k] + i] = deg > 0 ? 1.0f / (float)deg : 0.0f;
+}
+
+// s[v] = (deg(v) + 1)^-1/2
+__global__ void __launch_bounds__(256)
+gcn_scale_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out, float* __restrict__ scale) {
+    int k, r0;
+    if (!locate_tile(g, 256, blockIdx.x, &k, &r0)) return;
+    const int i = r0 + threadIdx.x;
+    if (i >= g.rows[k]) return;
+    const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
+    scale[g.row_ws[k] + i] = rsqrtf((float)(rp[i + 1] - rp[i] + 1));
 }
 
 __global__ void __launch_bounds__(256)
@@ -83,9 +97,10 @@ heavy_list_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict
         if (group_entries(g, rowptr_out, grp) >= heavy) list[atomicAdd(count, 1)] = (int)grp;
 }
 
-// SRC_WEIGHTED == false: out[v] = inv_deg[v] * sum_u src[u]
-// SRC_WEIGHTED == true : out[v] = sum_u inv_deg[u] * src[u]
-template <int NCH, bool SRC_WEIGHTED>
+// MODE 0: out[v] = w[v] * sum_u src[u]                      (w = 1 / deg)
+// MODE 1: out[v] = sum_u w[u] * src[u]                      (w = 1 / deg)
+// MODE 2: out[v] = w[v] * (w[v] * src[v] + sum_u w[u] * src[u])   (w = (deg + 1)^-1/2)
+template <int NCH, int MODE>
 __global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 2 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
@@ -128,12 +143,15 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     // finishes row `row`: scale, store, clear
     auto flush = [&](int row) {
         const int64_t r = ws + i0 + row;
-        const float w = SRC_WEIGHTED ? 1.f : inv_deg[r];
+        const float w = MODE == 1 ? 1.f : inv_deg[r];
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
             const int colx = (c * 32 + lane) * 8;
             if (colx < d) {
-                if (!SRC_WEIGHTED) {
+                if (MODE == 2)  // the self loop
+                    acc[c].fma_planes_mixed(w, *reinterpret_cast<const uint4*>(src.hi + r * src.ld + colx),
+                                            *reinterpret_cast<const uint4*>(src.lo + r * src.ld + colx));
+                if (MODE != 1) {
 #pragma unroll
                     for (int e = 0; e < 8; ++e) acc[c].v[e] *= w;
                 }
@@ -160,7 +178,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
             my_row += (j < nrows && oj <= e) ? 1 : 0;
         }
         const int32_t mine = lane < cnt ? __ldg(cols + e) : 0;
-        const float mine_w = (SRC_WEIGHTED && lane < cnt) ? __ldg(inv_deg + ws + mine) : 0.f;
+        const float mine_w = (MODE != 0 && lane < cnt) ? __ldg(inv_deg + ws + mine) : 0.f;
         for (int t = 0; t < cnt; t += SPMM_INFLIGHT) {
             int32_t nb[SPMM_INFLIGHT];
             int row[SPMM_INFLIGHT];
@@ -170,7 +188,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                 const int tj = min(t + j, cnt - 1);
                 nb[j] = __shfl_sync(0xffffffffu, mine, tj);
                 row[j] = __shfl_sync(0xffffffffu, my_row, tj);
-                wt[j] = SRC_WEIGHTED ? __shfl_sync(0xffffffffu, mine_w, tj) : 1.f;
+                wt[j] = MODE != 0 ? __shfl_sync(0xffffffffu, mine_w, tj) : 1.f;
                 if (t + j >= cnt) nb[j] = -1;
             }
             {
@@ -192,7 +210,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                     while (cur < row[j]) flush(cur++);
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
-                        if (SRC_WEIGHTED) acc[c].fma_planes_mixed(wt[j], xh[j][c], xl[j][c]);
+                        if (MODE != 0) acc[c].fma_planes_mixed(wt[j], xh[j][c], xl[j][c]);
                         else acc[c].add_planes_mixed(xh[j][c], xl[j][c]);
                     }
                 }
@@ -211,8 +229,8 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     }
 }
 
-template <bool SRC_WEIGHTED>
-int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+template <int MODE>
+int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                       const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket, cudaStream_t s) {
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
@@ -223,9 +241,9 @@ int32_t dispatch_spmm(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_o
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, SPMM_THREADS / 32), (int64_t)sms * blocks_per_sm);
 #define RTMA_SPMM(N)                                                                                      \
     do {                                                                                                  \
-        KernelScope ks(ctx, SRC_WEIGHTED ? KC_SPMM_BWD : KC_SPMM_FWD, s);                                 \
-        spmm_kernel<N, SRC_WEIGHTED><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src,  \
-                                                                   out, d, groups, order, ticket);        \
+        KernelScope ks(ctx, kclass, s);                                                                   \
+        spmm_kernel<N, MODE><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, d,  \
+                                                           groups, order, ticket);                        \
     } while (0)
     if (d <= 256) RTMA_SPMM(1);
     else if (d <= 512) RTMA_SPMM(2);
@@ -265,13 +283,28 @@ int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
 int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                          const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                          cudaStream_t s) {
-    return dispatch_spmm<false>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
+    return dispatch_spmm<0>(ctx, KC_SPMM_FWD, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
 }
 
 int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                                const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                                cudaStream_t s) {
-    return dispatch_spmm<true>(ctx, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
+    return dispatch_spmm<1>(ctx, KC_SPMM_BWD, g, rowptr_out, col_out, inv_deg, src, out, d, order, ticket, s);
+}
+
+int32_t launch_spmm_gcn(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                        const float* scale, Planes src, Planes out, int d, bool backward, SpmmOrder order, int* ticket,
+                        cudaStream_t s) {
+    return dispatch_spmm<2>(ctx, backward ? KC_SPMM_BWD : KC_SPMM_FWD, g, rowptr_out, col_out, scale, src, out, d, order,
+                            ticket, s);
+}
+
+int32_t launch_gcn_scale(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* scale, cudaStream_t s) {
+    const int64_t tiles = group_tiles(g, 256);
+    if (tiles == 0) return RTMA_OK;
+    { KernelScope ks(ctx, KC_INV_DEGREE, s); gcn_scale_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, rowptr_out, scale); }
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
 }
 
 int64_t spmm_order_entries(const GroupDesc& g) { return group_tiles(g, SPMM_ROWS_PER_WARP); }

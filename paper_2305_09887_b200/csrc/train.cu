@@ -1,5 +1,5 @@
 // Host-side sequencing of Algorithm 2's loop body for M trainers on one GPU: K plain-SGD
-// steps of a GraphSAGE-mean network on every part, trainers grouped by stream.
+// steps of a GraphSAGE-mean (or GCN) network on every part, trainers grouped by stream.
 #include <algorithm>
 #include <vector>
 
@@ -13,27 +13,51 @@ struct Model {
     LayerShape layer[RTMA_MAX_LAYERS];
     int64_t P;
     float lr;
+    bool gcn;   // GCN layers (one weight matrix, renormalised adjacency) instead of GraphSAGE-mean
+    bool post;  // hidden layers normalise and / or use PReLU: the activation is a pass of its own
 };
+
+// The parameter layout of one replica (also rtma_param_count).
+int64_t layout_model(const rtma_model_desc* md, LayerShape* layer) {
+    const int nsrc = md->encoder == 1 ? 1 : 2;
+    int64_t off = 0;
+    for (int l = 0; l < md->L; ++l) {
+        LayerShape ls{};
+        ls.d_in = md->dims[l];
+        ls.d_out = md->dims[l + 1];
+        ls.nsrc = nsrc;
+        ls.param_offset = off;
+        off += (int64_t)(nsrc * md->dims[l] + 1) * md->dims[l + 1];
+        ls.gamma_offset = ls.beta_offset = ls.slope_offset = -1;
+        if (l < md->L - 1 && md->norm == 1) {
+            ls.gamma_offset = off;
+            off += ls.d_out;
+            ls.beta_offset = off;
+            off += ls.d_out;
+        }
+        if (l < md->L - 1 && md->act == 1) ls.slope_offset = off++;
+        if (layer) layer[l] = ls;
+    }
+    if (layer)
+        for (int l = 0; l < md->L; ++l) layer[l].P = off;
+    return off;
+}
 
 int32_t parse_model(rtma_ctx* ctx, const rtma_model_desc* md, Model* m) {
     if (!md) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "null model description");
     if (md->L < 1 || md->L > RTMA_MAX_LAYERS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "L=%d outside [1,%d]", md->L, RTMA_MAX_LAYERS);
     if (md->gemm_dtype != 0 && md->gemm_dtype != 1) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "gemm_dtype=%d", md->gemm_dtype);
+    if ((md->encoder | 1) != 1 || (md->act | 1) != 1 || (md->norm | 1) != 1)
+        return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "encoder=%d act=%d norm=%d: each must be 0 or 1", md->encoder, md->act, md->norm);
     m->L = md->L;
     m->lr = md->lr;
-    int64_t off = 0;
     for (int l = 0; l <= md->L; ++l) {
         if (md->dims[l] < 1) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "dims[%d]=%d", l, md->dims[l]);
         m->dims[l] = md->dims[l];
     }
-    for (int l = 0; l < md->L; ++l) {
-        m->layer[l].d_in = md->dims[l];
-        m->layer[l].d_out = md->dims[l + 1];
-        m->layer[l].param_offset = off;
-        off += (int64_t)(2 * md->dims[l] + 1) * md->dims[l + 1];
-    }
-    m->P = off;
-    for (int l = 0; l < md->L; ++l) m->layer[l].P = off;
+    m->P = layout_model(md, m->layer);
+    m->gcn = md->encoder == 1;
+    m->post = md->L > 1 && (md->act == 1 || md->norm == 1);
     return RTMA_OK;
 }
 
@@ -43,6 +67,7 @@ struct ScratchPlan {
     size_t max_layer_params;  // largest (2 d_in + 1) d_out
     size_t prep_bytes;        // repacked weights, per part
     int q_width;              // widest Abar^T dZ (widths of the layers above the first)
+    size_t post_width;        // widest normalised / PReLU layer output (0: none)
 };
 
 int64_t aligned_rows(int64_t n_p) { return ceil_div(n_p, GROUP_ROW_ALIGN) * GROUP_ROW_ALIGN; }
@@ -55,8 +80,10 @@ ScratchPlan plan_scratch(const Model& m) {
     for (int l = 0; l < m.L; ++l) {
         per_row += 4 * planes_ld(m.dims[l]);     // Abar H^l
         if (l < m.L - 1) per_row += 4 * planes_ld(m.dims[l + 1]);  // H^{l+1}, later overwritten by dZ^l
+        if (l < m.L - 1 && m.post) per_row += 4 * planes_ld(m.dims[l + 1]) + sizeof(float2);  // Z^{l}, (mean, 1/std)
         if (l >= 1) q_width = std::max(q_width, m.dims[l + 1]);
-        sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(2 * m.dims[l] + 1) * m.dims[l + 1]);
+        sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(m.layer[l].nsrc * m.dims[l] + 1) * m.dims[l + 1]);
+        if (l < m.L - 1 && m.post) sp.post_width = std::max(sp.post_width, (size_t)m.dims[l + 1]);
         sp.prep_bytes += sizeof(__nv_bfloat16) * tc_prep_elems(tc_plan_layer(m.layer[l]), l >= 1) + 4 * 256;
     }
     per_row += sizeof(float) * planes_ld(m.dims[m.L]);  // logits
@@ -92,6 +119,7 @@ size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
     const size_t matrices = 8 * m.L + 12;  // every matrix start is rounded up to 256 bytes
     return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, 32) + 256) +
            sizeof(int) * ((size_t)ceil_div(n_p, 8) + 64) +  // processing order of the aggregation kernels
+           sizeof(float) * ((size_t)ceil_div(n_p, 64) + 1) * (2 * sp.post_width + 1) +  // per-tile sums of d gamma, d beta, d a
            sp.prep_bytes + 256 * matrices;
 }
 
@@ -99,9 +127,7 @@ size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
 
 extern "C" int64_t rtma_param_count(const rtma_model_desc* md) {
     if (!md || md->L < 1 || md->L > RTMA_MAX_LAYERS) return -1;
-    int64_t p = 0;
-    for (int l = 0; l < md->L; ++l) p += (int64_t)(2 * md->dims[l] + 1) * md->dims[l + 1];
-    return p;
+    return layout_model(md, nullptr);
 }
 
 extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,
@@ -223,10 +249,16 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             };
             float* inv_deg = cur.take<float>((size_t)rows + 1);
             Planes Nl[RTMA_MAX_LAYERS], Hl[RTMA_MAX_LAYERS];
+            Planes Zl[RTMA_MAX_LAYERS];       // pre-activations of the hidden layers (only with a separate activation pass)
+            float2* stats[RTMA_MAX_LAYERS];   // their (mean, 1/std)
             Hl[0] = take_planes(m.dims[0]);
             for (int l = 0; l < m.L; ++l) {
                 Nl[l] = take_planes(m.dims[l]);
                 if (l < m.L - 1) Hl[l + 1] = take_planes(m.dims[l + 1]);
+                if (l < m.L - 1 && m.post) {
+                    Zl[l] = take_planes(m.dims[l + 1]);
+                    stats[l] = cur.take<float2>((size_t)rows + 1);
+                }
             }
             const int C = m.dims[m.L];
             Mat logits{cur.take<float>((size_t)rows * planes_ld(C) + 8), (int64_t)planes_ld(C)};
@@ -239,6 +271,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             int* ticket = cur.take<int>(64);  // work counter of the aggregation kernels (zero between launches)
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
             int* heavy_list = cur.take<int>((size_t)spmm_order_entries(g) + 4);
+            float* post_partial = m.post ? cur.take<float>((size_t)post_tiles(g) * (2 * plan.post_width + 1) + 4) : nullptr;
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
             __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
             for (int l = 0; l < m.L; ++l) {
@@ -255,7 +288,8 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             if (rows == 0) continue;
 
             RTMA_CUDA(ctx, cudaMemsetAsync(ctx->arena + gi * share, 0, zero_bytes, s));
-            RTMA_TRY(launch_inv_degree(ctx, g, rowptr_out, inv_deg, s));
+            if (m.gcn) RTMA_TRY(launch_gcn_scale(ctx, g, rowptr_out, inv_deg, s));  // (deg + 1)^-1/2 in the same array
+            else RTMA_TRY(launch_inv_degree(ctx, g, rowptr_out, inv_deg, s));
             int64_t wave_entries = 0;
             for (int k = 0; k < g.num; ++k) wave_entries += edge_offsets[g.part[k] + 1] - edge_offsets[g.part[k]];
             SpmmOrder wave_order;
@@ -298,10 +332,17 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 for (int l = 0; l < m.L; ++l)
                     RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
                 for (int l = 0; l < m.L; ++l) {
-                    RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], order, ticket, s));
+                    if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], false, order, ticket, s));
+                    else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], order, ticket, s));
                     const bool last = l == m.L - 1;
-                    RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
-                                               last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, single_pass, s));
+                    if (last || !m.post) {
+                        RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
+                                                   last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, single_pass, s));
+                    } else {  // pre-activations kept; normalisation and PReLU in a pass of their own
+                        RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
+                                                   Zl[l], no_mat, false, single_pass, s));
+                        RTMA_TRY(launch_post_forward(ctx, g, m.layer[l], params, Zl[l], Hl[l + 1], stats[l], s));
+                    }
                 }
                 if (tap && taps->acts) {
                     size_t rec = 0;  // floats per row in the record
@@ -324,15 +365,20 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, loss_stride, step, s));
                 // ---- backward + SGD ----
                 for (int l = m.L - 1; l >= 0; --l) {
-                    const Planes dZ = l == m.L - 1 ? dZlast : Hl[l + 1];
+                    // dZ^l: from the loss, over H^{l+1} (fused ReLU gate) or over Z^l (separate activation pass)
+                    const Planes dZ = l == m.L - 1 ? dZlast : (m.post ? Zl[l] : Hl[l + 1]);
                     RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, single_pass, s));
                     if (l > 0) {
                         // dH^l = dZ Ws^T + Abar^T (dZ Wn^T) = [dZ | Abar^T dZ] [Ws^T ; Wn^T]: aggregate first,
                         // at the layer's output width, then one product whose epilogue applies the ReLU
                         // gate and writes dZ^{l-1} over H^l
                         const Planes Q{q_hi, q_lo, (int64_t)planes_ld(m.dims[l + 1])};
-                        RTMA_TRY(launch_spmm_transposed(ctx, g, rowptr_out, col_out, inv_deg, dZ, Q, m.dims[l + 1], order, ticket, s));
-                        RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Q, Bd_hi[l], Bd_lo[l], Hl[l], single_pass, s));
+                        if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, dZ, Q, m.dims[l + 1], true, order, ticket, s));
+                        else RTMA_TRY(launch_spmm_transposed(ctx, g, rowptr_out, col_out, inv_deg, dZ, Q, m.dims[l + 1], order, ticket, s));
+                        RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZ, Q, Bd_hi[l], Bd_lo[l], Hl[l], !m.post, single_pass, s));
+                        if (m.post)  // dH^l (now in H^l's place) -> dZ^{l-1} over Z^{l-1}; gamma, beta, slope step
+                            RTMA_TRY(launch_post_backward(ctx, g, m.layer[l - 1], params, Zl[l - 1], Hl[l], stats[l - 1], post_partial,
+                                                          m.lr, tap ? taps->grads : nullptr, s));
                     }
                     RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
                 }

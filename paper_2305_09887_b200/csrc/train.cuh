@@ -53,7 +53,11 @@ inline size_t padded_ld(int64_t d) { return (size_t)((d + 3) / 4 * 4); }
 
 struct LayerShape {
     int32_t d_in, d_out;
-    int64_t param_offset;  // of Ws inside one replica; Ws, Wn, b are contiguous: a (2 d_in + 1) x d_out matrix
+    int32_t nsrc;          // weight matrices of the layer: 2 = GraphSAGE-mean (Ws, Wn), 1 = GCN (W)
+    int64_t param_offset;  // of the first weight matrix inside one replica; the weight matrices and b are
+                           // contiguous: an (nsrc d_in + 1) x d_out matrix
+    int64_t gamma_offset, beta_offset;  // Layer Normalization scale / shift [d_out]; -1 = none
+    int64_t slope_offset;               // PReLU slope [1]; -1 = ReLU
     int64_t P;             // parameters per replica
 };
 
@@ -94,6 +98,13 @@ int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t*
                                const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                                cudaStream_t s);
 
+// GCN: scale[row_ws + i] = (local degree + 1)^-1/2, and
+// out[r] = scale[r] * (scale[r] * src[r] + sum_{u in N(r)} scale[u] * src[u])   (symmetric: both passes)
+int32_t launch_gcn_scale(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* scale, cudaStream_t s);
+int32_t launch_spmm_gcn(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                        const float* scale, Planes src, Planes out, int d, bool backward, SpmmOrder order, int* ticket,
+                        cudaStream_t s);
+
 // ---- loss.cu --------------------------------------------------------------------------
 // Softmax cross-entropy over fp32 logits, mean over the part; dZ = (softmax - onehot) / n_p is
 // written as split planes and the part's loss to loss_out[part * loss_stride + loss_col] when
@@ -101,6 +112,16 @@ int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t*
 int64_t loss_tiles(const GroupDesc& g);
 int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp, Planes dZ,
                             float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s);
+
+// ---- post.cu (Layer Normalization before the activation, PReLU) ------------------------------
+int64_t post_tiles(const GroupDesc& g);
+// H = act(norm(Z)) for the layer's output; stats[row] = (mean, 1/std) when the layer normalises.
+int32_t launch_post_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const float* params, Planes Z, Planes H,
+                            float2* stats, cudaStream_t s);
+// Z <- gradient with respect to Z, given dH (the gradient with respect to H) and Z itself; then
+// gamma, beta and the slope take their SGD step.  partial: post_tiles(g) * (2 d_out + 1) floats.
+int32_t launch_post_backward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, float* params, Planes Z, Planes dH,
+                             float2* stats, float* partial, float lr, float* grads_record, cudaStream_t s);
 
 // ---- optim.cu -------------------------------------------------------------------------
 // grad = sum of the part's chunk slots; params -= lr * grad; optionally records grad.
@@ -113,8 +134,8 @@ int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float*
 // `single` = operands rounded to bf16: only the hi planes are loaded and each product is one MMA
 // instead of three.
 struct TcLayerPlan {
-    int Kf, BN_f, Npad_f;  // forward: padded K (2 x 64-blocks over d_in), column tile, padded N
-    int Kd, BN_d, Npad_d;  // dgrad: padded K (2 x 64-blocks over d_out), column tile, padded N over d_in
+    int Kf, BN_f, Npad_f;  // forward: padded K (nsrc x 64-blocks over d_in), column tile, padded N
+    int Kd, BN_d, Npad_d;  // dgrad: padded K (nsrc x 64-blocks over d_out), column tile, padded N over d_in
 };
 bool tc_available();
 TcLayerPlan tc_plan_layer(LayerShape ls);
@@ -123,17 +144,20 @@ size_t tc_prep_elems(const TcLayerPlan& p, bool with_dgrad);  // bf16 elements p
 int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, const float* params,
                               __nv_bfloat16* Bf_hi, __nv_bfloat16* Bf_lo, __nv_bfloat16* Bd_hi, __nv_bfloat16* Bd_lo,
                               cudaStream_t s);
-// out = act([H | N] [Ws; Wn] + b): split planes when out_planes.hi != NULL, else fp32 out_f32.
+// out = act([H | N] [Ws; Wn] + b), or act(N W + b) for a one-matrix layer (H is then ignored):
+// split planes when out_planes.hi != NULL, else fp32 out_f32.
 int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                           const float* params, Planes H, Planes N, const __nv_bfloat16* Bf_hi,
                           const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, bool single,
                           cudaStream_t s);
-// H <- ([dZ | Q] [Ws^T ; Wn^T]) where H > 0 else 0: on entry H holds the layer's input activations
-// (their sign is the ReLU gate), on exit the gradient with respect to the previous layer's
-// pre-activations.  Q = Abar^T dZ.
+// H <- ([dZ | Q] [Ws^T ; Wn^T]) (or Q W^T for a one-matrix layer), Q = the transposed aggregation
+// of dZ.  gate: on entry H holds the layer's input activations and entries where H <= 0 become 0
+// (the ReLU gate), so that on exit H is the gradient with respect to the previous layer's
+// pre-activations; !gate: plain product (the activation's backward pass follows separately).
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
-                        Planes dZ, Planes Q, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, Planes H, bool single,
-                        cudaStream_t s);
-// partial[slot][(2 d_in + 1) x d_out] = [H | N | 1]^T dZ over one chunk of rows.
+                        Planes dZ, Planes Q, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, Planes H, bool gate,
+                        bool single, cudaStream_t s);
+// partial[slot][(nsrc d_in + 1) x d_out] = [H | N | 1]^T dZ ([N | 1]^T dZ for a one-matrix layer)
+// over one chunk of rows.
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
                         Planes H, Planes N, Planes dZ, float* partial, bool single, cudaStream_t s);

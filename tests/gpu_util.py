@@ -95,7 +95,17 @@ def tols(gemm_dtype):
     return TOL_ACT, TOL_GRAD, TOL_PARAM, 1e-5, 2e-5, 1e-5
 
 
-def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None):
+def _param_segments(variant, dims):
+    """[(name, offset, size)] of every parameter tensor of one replica."""
+    out = []
+    for l, lay in enumerate(oracle.variant_layout(variant, dims)):
+        sizes = {"w0": dims[l] * dims[l + 1], "w1": dims[l] * dims[l + 1], "bias": dims[l + 1],
+                 "gamma": dims[l + 1], "beta": dims[l + 1], "slope": 1}
+        out += [(f"{key}{l}", off, sizes[key]) for key, off in lay.items() if off >= 0]
+    return out
+
+
+def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, variant=(0, 0, 0), params0=None):
     """Partition + induced CSR against the oracle (bit-exact), then step 0 of all M trainers
     batched as one call: every recorded intermediate, the loss, the gradient and the updated
     parameters of every part (or of the parts in only_parts) against the oracle."""
@@ -106,22 +116,25 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None):
     assert_preprocess_equal(got, want)
     M = got["M"]
     dims, n = w.dims, w.graph.n
-    P = inputs.param_count(dims)
+    params0 = w.params0 if params0 is None else params0
+    P = params0.size
+    assert P == oracle.variant_param_count(variant, dims) == binding.param_count(dims, variant)
     rec = sum(dims[l] + dims[l + 1] for l in range(len(dims) - 1))
-    params = dev(np.tile(w.params0, (M, 1)))
+    params = dev(np.tile(params0, (M, 1)))
     acts = torch.zeros(n * rec, dtype=torch.float32, device="cuda")
     grads = torch.zeros(M, P, dtype=torch.float32, device="cuda")
     loss = torch.zeros(M, 1, dtype=torch.float32, device="cuda")
     c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
                   got["Xp"], got["yp"], params, 1, loss_out=loss, taps=(acts, grads, 0), gemm_dtype=gemm_dtype,
-                  streams=streams)
+                  streams=streams, variant=variant)
     torch.cuda.synchronize()
     grads, loss, params1 = grads.cpu().numpy(), loss.cpu().numpy(), params.cpu().numpy()
-    p0 = w.params0.astype(np.float64)
+    p0 = params0.astype(np.float64)
     for p in range(M) if only_parts is None else only_parts:
         rp, cp, X, y = oracle_part(w, want, p)
         n_p = rp.size - 1
-        o_loss, o_grads, o_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True, want_preact=True)
+        o_loss, o_grads, o_acts = oracle.forward_backward_variant(variant, dims, rp, cp, X, y, p0, want_acts=True,
+                                                                  want_preact=True)
         layout, total = oracle.acts_layout(dims, n_p)
         base = int(want["part_offsets"][p]) * rec
         gpu_acts = {}
@@ -146,24 +159,25 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None):
             gates.append(g8)
         assert flipped <= 8 + flip_frac * units
         if flipped:
-            o_loss, o_grads, _ = oracle.forward_backward(dims, rp, cp, X, y, p0, gates=gates)
+            o_loss, o_grads, _ = oracle.forward_backward_variant(variant, dims, rp, cp, X, y, p0, gates=gates)
         if n_p:
             assert abs(loss[p, 0] - o_loss) <= tol_loss * max(1.0, abs(o_loss)), p
         # gradients: per parameter tensor
-        off = 0
-        for l in range(len(dims) - 1):
-            for nm, size in (("Ws", dims[l] * dims[l + 1]), ("Wn", dims[l] * dims[l + 1]), ("b", dims[l + 1])):
-                gg, og = grads[p, off:off + size], o_grads[off:off + size]
-                if np.abs(og).max() > 0:
-                    assert rel_err(gg, og) <= tol_grad, (p, l, nm)
+        for nm, off, size in _param_segments(variant, dims):
+            gg, og = grads[p, off:off + size], o_grads[off:off + size]
+            if np.abs(og).max() > 0:
+                if size == 1:   # a single number (PReLU slope): relative to itself, with an absolute floor
+                    assert abs(gg[0] - og[0]) <= tol_grad * max(abs(og[0]), 1e-3), (p, nm)
                 else:
-                    assert np.abs(gg).max() == 0
-                off += size
+                    assert rel_err(gg, og) <= tol_grad, (p, nm)
+            else:
+                assert np.abs(gg).max() == 0
         assert rel_err(params1[p], p0 - w.lr * o_grads) <= tol_param
     return got, want
 
 
-def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_parts=None):
+def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_parts=None, variant=(0, 0, 0),
+                              params0=None):
     """K local steps of all M trainers and the aggregation.  Parameters and losses of every part
     (or of the parts in only_parts) against the oracle; the average against the oracle's, or,
     when only some parts were recomputed, against the fp64 mean of the kernel's own replicas."""
@@ -171,10 +185,11 @@ def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_
     tol_loss = 10 * tols(gemm_dtype)[3]
     c = ctx()
     M, dims = got["M"], w.dims
-    params = dev(np.tile(w.params0, (M, 1)))
+    params0 = w.params0 if params0 is None else params0
+    params = dev(np.tile(params0, (M, 1)))
     loss = torch.zeros(M, K, dtype=torch.float32, device="cuda")
     c.local_steps(dims, w.lr, M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
-                  got["Xp"], got["yp"], params, K, loss_out=loss, gemm_dtype=gemm_dtype, streams=streams)
+                  got["Xp"], got["yp"], params, K, loss_out=loss, gemm_dtype=gemm_dtype, streams=streams, variant=variant)
     torch.cuda.synchronize()
     after = params.cpu().numpy().copy()
     glob = torch.empty(params.shape[1], dtype=torch.float32, device="cuda")
@@ -183,7 +198,7 @@ def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_
     o_params = after.astype(np.float64)
     for p in range(M) if only_parts is None else only_parts:
         rp, cp, X, y = oracle_part(w, want, p)
-        o_params[p], o_loss = oracle.local_steps(dims, w.lr, rp, cp, X, y, w.params0.astype(np.float64), K)
+        o_params[p], o_loss = oracle.local_steps_variant(variant, dims, w.lr, rp, cp, X, y, params0.astype(np.float64), K)
         assert rel_err(after[p], o_params[p]) <= tol_param, p
         if rp.size > 1:
             assert np.abs(loss[p].cpu().numpy() - o_loss).max() <= tol_loss * max(1.0, np.abs(o_loss).max())

@@ -39,11 +39,15 @@ def test_binding_lists_the_same_symbols():
 
 def test_param_count_and_struct_layout(lib):
     from paper_2305_09887_b200 import binding, inputs
-    assert ctypes.sizeof(binding.ModelDesc) == 4 + 4 * 9 + 4 + 4
+    assert ctypes.sizeof(binding.ModelDesc) == 4 + 4 * 9 + 4 + 4 + 3 * 4
     for dims in [(64, 64, 8), (128, 256, 256, 47), (100, 256, 256, 47), (128, 256, 2), (512, 512, 512, 47)]:
         assert binding.param_count(dims) == inputs.param_count(dims)
     assert binding.param_count((128, 256, 256, 47)) == 221231   # the Medium model
     assert binding.param_count((512, 512, 512, 47)) == 1097775  # the sweep model
+    # variants: GCN has one weight matrix per layer; hidden layers add gamma, beta (norm) and a slope (PReLU)
+    assert binding.param_count((128, 256, 256, 47), (1, 0, 0)) == 129 * 256 + 257 * 256 + 257 * 47
+    assert binding.param_count((128, 256, 256, 47), (1, 1, 1)) == 129 * 256 + 257 * 256 + 257 * 47 + 2 * (2 * 256 + 1)
+    assert binding.param_count((128, 256, 256, 47), (0, 1, 0)) == 221231 + 2
 
 
 def test_no_cpu_fallback_without_a_device():
