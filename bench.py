@@ -163,7 +163,7 @@ def cpu_sample(w, local_steps=1):
     rp, cp = oracle.part_graph(rowptr_out, col_out, part_offsets, edge_offsets, 0)
     hi = int(part_offsets[1])
     t1 = time.perf_counter()
-    oracle.local_steps(w.dims, w.lr, rp, cp, Xp[:hi], yp[:hi], w.params0, local_steps)
+    oracle.local_steps_variant(w.variant, w.dims, w.lr, rp, cp, Xp[:hi], yp[:hi], w.params0, local_steps)
     t_step = (time.perf_counter() - t1) / local_steps
     passes = 2 * L - 1
     units_full = float(kept) * passes * w.K * w.R
@@ -203,13 +203,20 @@ def make_workload(args):
     from paper_2305_09887_b200 import inputs
     s = args.scale
     if args.workload == "medium":
-        return inputs.medium(1.0 if s is None else s)
-    if args.workload == "supertma":
-        return inputs.supertma(1.0 if s is None else s, M=args.M or 16)
-    if args.workload == "sweep":
-        return inputs.supertma(1.0 if s is None else s, width=512, M=args.M or 16,
-                               use_groups=args.assign == "super", gemm_dtype=1)
-    return inputs.large(1.0 if s is None else s)
+        w = inputs.medium(1.0 if s is None else s)
+    elif args.workload == "supertma":
+        w = inputs.supertma(1.0 if s is None else s, M=args.M or 16)
+    elif args.workload == "sweep":
+        w = inputs.supertma(1.0 if s is None else s, width=512, M=args.M or 16,
+                            use_groups=args.assign == "super", gemm_dtype=1)
+    else:
+        w = inputs.large(1.0 if s is None else s)
+    variant = (1 if args.encoder == "gcn" else 0, 1 if args.act == "prelu" else 0, 1 if args.norm == "layernorm" else 0)
+    if variant != (0, 0, 0):   # the paper's own encoders (Sec. 4.1) on the same graph, features and widths
+        w.variant = variant
+        w.params0 = inputs.variant_params(variant, w.dims, inputs.SEED_WEIGHT + 7)
+        w.name += "_" + "-".join([args.encoder, args.act, args.norm])
+    return w
 
 
 def max_over_ranks(seconds: float, dist_mod=None, device=None) -> float:
@@ -233,6 +240,9 @@ def main():
     ap.add_argument("--scale", type=float, default=None, help="shrink (or grow) the workload's graph")
     ap.add_argument("--M", type=int, default=None, help="trainers (supertma / sweep)")
     ap.add_argument("--assign", default="super", choices=["node", "super"], help="sweep: assignment scheme")
+    ap.add_argument("--encoder", default="sage", choices=["sage", "gcn"])
+    ap.add_argument("--act", default="relu", choices=["relu", "prelu"])
+    ap.add_argument("--norm", default="none", choices=["none", "layernorm"])
     ap.add_argument("--streams", type=int, default=1,
                     help="CUDA streams the trainers are spread over (trainers sharing a stream are batched)")
     args = ap.parse_args()
@@ -288,7 +298,7 @@ def main():
                 for st in pool:
                     st.wait_stream(torch.cuda.current_stream())
             ctx.local_steps(w.dims, w.lr, w.M, part_host, edge_host, rowptr_out, col_out, Xp, yp, params, w.K,
-                            loss_out=loss[r], gemm_dtype=w.gemm_dtype, streams=trainer_streams)
+                            loss_out=loss[r], gemm_dtype=w.gemm_dtype, streams=trainer_streams, variant=w.variant)
             if pool:
                 for st in pool:
                     torch.cuda.current_stream().wait_stream(st)
@@ -334,7 +344,7 @@ def main():
 
     # ---- roofline of the dominant kernel class --------------------------------------
     peaks = load_peaks()
-    work = algorithmic_work(w.dims, n_parts, e_parts, w.K, w.R)
+    work = algorithmic_work(w.dims, n_parts, e_parts, w.K, w.R) if w.variant == (0, 0, 0) else {}
     total_kernel_ms = sum(ms for ms, _ in prof.values())
     shares = {k: ms / total_kernel_ms for k, (ms, _) in prof.items() if ms > 0}
     top = max(shares, key=shares.get)
@@ -382,7 +392,7 @@ def main():
     h_rowptr, h_col, h_X, h_y, h_p0 = pin(g.rowptr), pin(g.col), pin(w.X), pin(w.y), pin(w.params0)
     e2e_steps = max(1, min(args.steps, 3))
     h_gid = pin(g.group_id) if w.use_groups else None
-    host_kw = dict(group_id=h_gid, gemm_dtype=w.gemm_dtype)
+    host_kw = dict(group_id=h_gid, gemm_dtype=w.gemm_dtype, variant=w.variant)
     ctx.train_host(h_rowptr, h_col, h_X, h_y, w.dims, w.M, w.K, w.R, w.lr, w.partition_seed, h_p0, **host_kw)  # warm-up
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -411,6 +421,7 @@ def main():
                   "bf16x3-split products, f32 accumulate and elementwise"), "data": "synthetic",
         "config": {"workload": w.name, "nodes": g.n, "entries": g.num_entries, "kept_entries": int(kept), "M": w.M,
                    "dims": list(w.dims), "K": w.K, "R": w.R, "spmm_passes_per_local_step": passes,
+                   "variant": {"encoder": args.encoder, "act": args.act, "norm": args.norm},
                    "assignment": "super-node" if w.use_groups else "node",
                    "kept_fraction": kept / g.num_entries,
                    "parallelism": ("replicas only" if world > 1 else

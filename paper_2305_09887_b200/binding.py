@@ -309,7 +309,8 @@ class Context:
         self._check(st, "rtma_sgd_aggregate")
 
     # ---- whole path from host buffers -----------------------------------------------
-    def train_host(self, rowptr, col, X, y, dims, M, K, R, lr, seed, params0, group_id=None, gemm_dtype=0):
+    def train_host(self, rowptr, col, X, y, dims, M, K, R, lr, seed, params0, group_id=None, gemm_dtype=0,
+                   variant=(0, 0, 0)):
         """The whole path on HOST (numpy) buffers: copies the inputs to the device, runs
         partition, induced CSR, row gather, R rounds of (K local steps + aggregation), and
         copies the result back.  Returns (params[P] f32, losses[R, M, K] f32, kept, cut)."""
@@ -324,7 +325,7 @@ class Context:
         params0 = np.ascontiguousarray(params0, dtype=np.float32)
         gid = None if group_id is None else np.ascontiguousarray(group_id, dtype=np.int32)
         n = rowptr.size - 1
-        md = model_desc(dims, lr, gemm_dtype)
+        md = model_desc(dims, lr, gemm_dtype, variant)
         out = np.empty(params0.size, dtype=np.float32)
         losses = np.empty((R, M, K), dtype=np.float32)
         kept_cut = np.empty(2, dtype=np.int64)

@@ -203,26 +203,36 @@ post_backward_kernel(const __grid_constant__ GroupDesc g, const PostArgs a) {
     }
 }
 
+// 32 parameters per block; eight threads per parameter each add every eighth tile in order, and
+// the eight partial sums are added in a fixed order: the result does not change from run to run.
 __global__ void __launch_bounds__(256)
 post_reduce_sgd_kernel(const __grid_constant__ GroupDesc g, const LayerShape ls, const float* __restrict__ partial,
                        const float lr, float* __restrict__ params, float* __restrict__ grads_record) {
+    __shared__ float red[8][33];
     const int k = blockIdx.y;
     const int d = ls.d_out;
-    const int j = blockIdx.x * 256 + threadIdx.x;
-    if (j >= 2 * d + 1) return;
+    const int col = threadIdx.x & 31, lane_t = threadIdx.x >> 5;
+    const int j = blockIdx.x * 32 + col;
+    int64_t first = 0;
+    for (int q = 0; q < k; ++q) first += (g.rows[q] + POST_TILE_ROWS - 1) / POST_TILE_ROWS;
+    const int64_t count = (g.rows[k] + POST_TILE_ROWS - 1) / POST_TILE_ROWS;
+    float s = 0.f;
+    if (j < 2 * d + 1)
+        for (int64_t t = lane_t; t < count; t += 8) s += partial[(first + t) * (2 * d + 1) + j];
+    red[lane_t][col] = s;
+    __syncthreads();
+    if (lane_t != 0 || j >= 2 * d + 1) return;
     int64_t at;
     if (j < d) at = ls.gamma_offset < 0 ? -1 : ls.gamma_offset + j;
     else if (j < 2 * d) at = ls.beta_offset < 0 ? -1 : ls.beta_offset + (j - d);
     else at = ls.slope_offset;
     if (at < 0) return;
-    int64_t first = 0;
-    for (int q = 0; q < k; ++q) first += (g.rows[q] + POST_TILE_ROWS - 1) / POST_TILE_ROWS;
-    const int64_t count = (g.rows[k] + POST_TILE_ROWS - 1) / POST_TILE_ROWS;
-    float s = 0.f;
-    for (int64_t t = 0; t < count; ++t) s += partial[(first + t) * (2 * d + 1) + j];
+    float sum = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) sum += red[w][col];
     at += (int64_t)g.part[k] * ls.P;
-    if (grads_record) grads_record[at] = s;
-    params[at] -= lr * s;
+    if (grads_record) grads_record[at] = sum;
+    params[at] -= lr * sum;
 }
 
 }  // namespace
@@ -256,7 +266,7 @@ int32_t launch_post_backward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, f
     { KernelScope ks(ctx, KC_POST, s); RTMA_POST_DISPATCH(post_backward_kernel, ls.d_out, g, a); }
     RTMA_LAUNCH_CHECK(ctx);
     if (ls.gamma_offset >= 0 || ls.slope_offset >= 0) {
-        dim3 grid((unsigned)ceil_div(2 * ls.d_out + 1, 256), (unsigned)g.num);
+        dim3 grid((unsigned)ceil_div(2 * ls.d_out + 1, 32), (unsigned)g.num);
         { KernelScope ks(ctx, KC_POST, s); post_reduce_sgd_kernel<<<grid, 256, 0, s>>>(g, ls, partial, lr, params, grads_record); }
         RTMA_LAUNCH_CHECK(ctx);
     }

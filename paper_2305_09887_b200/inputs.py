@@ -45,6 +45,7 @@ class Workload:
     params0: np.ndarray  # float32 [P], identical start for every trainer
     use_groups: bool = False
     gemm_dtype: int = 0  # 0: fp32-accurate GEMMs, 1: bf16 inputs / fp32 accumulate
+    variant: tuple = (0, 0, 0)  # (encoder, act, norm): 0,0,0 = GraphSAGE-mean, ReLU, no normalisation
 
 
 def _sorted_unique(key: np.ndarray) -> np.ndarray:
@@ -230,6 +231,38 @@ def xavier_params(dims, seed: int) -> np.ndarray:
         a = math.sqrt(6.0 / (d_in + d_out))
         out.append(rng.uniform(-a, a, size=2 * d_in * d_out).astype(np.float32))
         out.append(np.zeros(d_out, dtype=np.float32))
+    return np.concatenate(out)
+
+
+def variant_param_count(variant, dims) -> int:
+    """Parameters of a model variant (encoder, act, norm): GCN (encoder 1) has one weight matrix
+    per layer; hidden layers add gamma, beta (norm 1) and one PReLU slope (act 1)."""
+    encoder, act, norm = variant
+    total = 0
+    for l in range(len(dims) - 1):
+        total += (1 if encoder == 1 else 2) * dims[l] * dims[l + 1] + dims[l + 1]
+        if l < len(dims) - 2:
+            total += (2 * dims[l + 1] if norm == 1 else 0) + (1 if act == 1 else 0)
+    return total
+
+
+def variant_params(variant, dims, seed: int) -> np.ndarray:
+    """Initial parameters of a model variant, in the library's order (weights, b, gamma, beta,
+    slope per layer): Xavier-uniform weights, zero biases, gamma 1, beta 0, slope 0.25."""
+    encoder, act, norm = variant
+    rng = np.random.default_rng(seed)
+    out = []
+    for l in range(len(dims) - 1):
+        d_in, d_out = dims[l], dims[l + 1]
+        a = math.sqrt(6.0 / (d_in + d_out))
+        out.append(rng.uniform(-a, a, size=(1 if encoder == 1 else 2) * d_in * d_out).astype(np.float32))
+        out.append(np.zeros(d_out, dtype=np.float32))
+        if l < len(dims) - 2:
+            if norm == 1:
+                out.append(np.ones(d_out, dtype=np.float32))
+                out.append(np.zeros(d_out, dtype=np.float32))
+            if act == 1:
+                out.append(np.full(1, 0.25, dtype=np.float32))
     return np.concatenate(out)
 
 

@@ -166,3 +166,20 @@ def test_variant_sgd_step_is_w_minus_lr_times_gradient(variant):
     r, _ = oracle.local_steps_variant(variant, dims, 0.05, rp, cp, X, y, q, 2)
     assert np.array_equal(q2, r)
     assert l2[2] < l2[0]                                   # SGD descends on a fixed batch
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_input_generator_lays_parameters_out_as_the_oracle_reads_them(variant):
+    dims = (7, 6, 5, 3)
+    p = inputs.variant_params(variant, dims, 3)
+    assert p.size == inputs.variant_param_count(variant, dims) == oracle.variant_param_count(variant, dims)
+    for l, lay in enumerate(oracle.variant_layout(variant, dims)):
+        d_out = dims[l + 1]
+        assert np.all(p[lay["bias"]:lay["bias"] + d_out] == 0)
+        if lay["gamma"] >= 0:
+            assert np.all(p[lay["gamma"]:lay["gamma"] + d_out] == 1) and np.all(p[lay["beta"]:lay["beta"] + d_out] == 0)
+        if lay["slope"] >= 0:
+            assert p[lay["slope"]] == 0.25
+        bound = np.sqrt(6.0 / (dims[l] + d_out))
+        w = p[lay["w0"]:lay["bias"]]
+        assert np.abs(w).max() <= bound and np.abs(w).max() > 0.5 * bound
