@@ -8,7 +8,8 @@ directed entries, 128-d features, 47 classes, M=8 trainers, 128-256-256-47 Graph
 20 local steps per round, 5 aggregation rounds).  --workload selects the other shapes:
 supertma (planted communities, super-node assignment, M=16), sweep (the same graph at width
 512 with bf16 GEMM operands; --M and --assign pick the point of the sweep) and large
-(--scale shrinks it; the full size needs ~60 GB of host memory to generate).
+(--scale shrinks it; the full size needs ~60 GB of host memory to generate); averaging times
+the aggregation kernel alone on a shape large enough to be bound by HBM.
 
 Metric: aggregated edges/s = (sum over parts of kept entries) x (SpMM passes per local step:
 L forward + L-1 backward) x (local steps) / time.  Local trainer-steps/s is reported beside it.
@@ -219,6 +220,44 @@ def make_workload(args):
     return w
 
 
+def run_averaging_stress(args, local_rank):
+    """`--workload averaging`: the aggregation kernel alone on a shape large enough to be bound by
+    HBM (M = 32 replicas of 16 Mi parameters, 2 GiB read and 2 GiB written per launch; the named
+    workloads average at most 4.4 MB).  One step = one rtma_aggregate."""
+    import torch
+    from paper_2305_09887_b200 import binding
+    torch.cuda.set_device(local_rank)
+    ctx = binding.Context(local_rank)
+    M, P = args.M or 32, 16 << 20
+    params = torch.randn(M, P, dtype=torch.float32, device="cuda")
+    glob = torch.empty(P, dtype=torch.float32, device="cuda")
+    for _ in range(max(args.warmup, 3)):
+        ctx.aggregate(params, glob)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ctx.aggregate(params, glob)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    seconds = e0.elapsed_time(e1) / 1e3
+    peaks = load_peaks()
+    abytes = 4.0 * P * (2 * M + 1)          # every replica read once and overwritten, the global copy written
+    achieved = abytes * args.steps / seconds / 1e9
+    print(json.dumps({
+        "metric": "averaging_bytes_per_s", "value": abytes * args.steps / seconds, "unit": "B/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * seconds / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "averaging_stress", "M": M, "P": P, "l2": "4 GiB touched per launch > L2"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "aggregate",
+                     "peak_source": peaks["source"]},
+        "gpu_launches": args.steps, "clocks": clocks}))
+
+
 def max_over_ranks(seconds: float, dist_mod=None, device=None) -> float:
     """Largest value over all ranks (the slowest rank sets the job's time)."""
     if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
@@ -236,7 +275,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="medium", choices=["medium", "supertma", "sweep", "large"])
+    ap.add_argument("--workload", default="medium", choices=["medium", "supertma", "sweep", "large", "averaging"])
     ap.add_argument("--scale", type=float, default=None, help="shrink (or grow) the workload's graph")
     ap.add_argument("--M", type=int, default=None, help="trainers (supertma / sweep)")
     ap.add_argument("--assign", default="super", choices=["node", "super"], help="sweep: assignment scheme")
@@ -253,6 +292,11 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             run_reference(args, make_workload(args))
+        return
+
+    if args.workload == "averaging":
+        if rank == 0:
+            run_averaging_stress(args, local_rank)
         return
 
     import torch

@@ -15,6 +15,8 @@ constexpr int LOSS_TILE_ROWS = 64;
 constexpr int LOSS_ROWS_PER_WARP = LOSS_TILE_ROWS / (LOSS_THREADS / 32);
 constexpr int LOSS_REG_CLASSES = 128;
 
+// J = logits a lane keeps in registers (C <= 32 J <= 128), 0 = sweep the row instead
+template <int J>
 __global__ void __launch_bounds__(LOSS_THREADS)
 softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
                     const Planes dZ, float* __restrict__ tile_loss) {
@@ -31,11 +33,11 @@ softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const
         const int64_t r = g.row_ws[k] + i;
         const float* z = logits.ptr + r * logits.ld;
         const int label = yp[g.row_abs[k] + i];
-        if (C <= LOSS_REG_CLASSES) {
-            float v[4];
+        if (J > 0) {
+            float v[J > 0 ? J : 1];
             float zmax = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < J; ++j) {
                 const int c = lane + 32 * j;
                 v[j] = c < C ? z[c] : -INFINITY;
                 zmax = fmaxf(zmax, v[j]);
@@ -44,14 +46,14 @@ softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const
             for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
             float sum = 0.f;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) sum += lane + 32 * j < C ? expf(v[j] - zmax) : 0.f;
+            for (int j = 0; j < J; ++j) sum += lane + 32 * j < C ? expf(v[j] - zmax) : 0.f;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
             const float lse = zmax + logf(sum);
             const float zl = __shfl_sync(0xffffffffu, v[label >> 5], label & 31);
             if (lane == 0) loss += lse - zl;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < J; ++j) {
                 const int c = lane + 32 * j;
                 if (c < C) {
                     __nv_bfloat16 h, l;
@@ -116,7 +118,11 @@ int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C
                             float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s) {
     const int64_t tiles = group_tiles(g, LOSS_TILE_ROWS);
     if (tiles > 0) {
-        { KernelScope ks(ctx, KC_LOSS, s); softmax_xent_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss); }
+        KernelScope ks(ctx, KC_LOSS, s);
+        if (C <= 32) softmax_xent_kernel<1><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        else if (C <= 64) softmax_xent_kernel<2><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        else if (C <= LOSS_REG_CLASSES) softmax_xent_kernel<4><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        else softmax_xent_kernel<0><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         RTMA_LAUNCH_CHECK(ctx);
     }
     if (loss_out && g.num > 0) {

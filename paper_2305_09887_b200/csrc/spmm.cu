@@ -139,6 +139,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
 #pragma unroll
     for (int c = 0; c < NCH; ++c) acc[c].zero();
     int cur = 0;  // row (relative to i0) the accumulators belong to
+    int64_t next_off = __shfl_sync(0xffffffffu, my_off, 1);  // first entry past row `cur`
 
     // finishes row `row`: scale, store, clear
     auto flush = [&](int row) {
@@ -170,24 +171,15 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     for (int64_t e0 = e_begin; e0 < e_end; e0 += 32) {
         const int cnt = (int)min((int64_t)32, e_end - e0);
         const int64_t e = e0 + lane;
-        // row of entry e = how many of the offsets rp[i0 + 1 ..] are <= e
-        int my_row = 0;
-#pragma unroll
-        for (int j = 1; j < SPMM_ROWS_PER_WARP; ++j) {
-            const int64_t oj = __shfl_sync(0xffffffffu, my_off, j);
-            my_row += (j < nrows && oj <= e) ? 1 : 0;
-        }
         const int32_t mine = lane < cnt ? __ldg(cols + e) : 0;
         const float mine_w = (MODE != 0 && lane < cnt) ? __ldg(inv_deg + ws + mine) : 0.f;
         for (int t = 0; t < cnt; t += SPMM_INFLIGHT) {
             int32_t nb[SPMM_INFLIGHT];
-            int row[SPMM_INFLIGHT];
             float wt[SPMM_INFLIGHT];
 #pragma unroll
             for (int j = 0; j < SPMM_INFLIGHT; ++j) {
                 const int tj = min(t + j, cnt - 1);
                 nb[j] = __shfl_sync(0xffffffffu, mine, tj);
-                row[j] = __shfl_sync(0xffffffffu, my_row, tj);
                 wt[j] = MODE != 0 ? __shfl_sync(0xffffffffu, mine_w, tj) : 1.f;
                 if (t + j >= cnt) nb[j] = -1;
             }
@@ -207,7 +199,11 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
 #pragma unroll
                 for (int j = 0; j < SPMM_INFLIGHT; ++j) {
                     if (nb[j] < 0) continue;
-                    while (cur < row[j]) flush(cur++);
+                    // entries come in row order: the rows that end before this entry are complete
+                    while (e0 + t + j >= next_off) {
+                        flush(cur++);
+                        next_off = __shfl_sync(0xffffffffu, my_off, cur + 1);
+                    }
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
                         if (MODE != 0) acc[c].fma_planes_mixed(wt[j], xh[j][c], xl[j][c]);
