@@ -237,6 +237,14 @@ int32_t rtma_profile(rtma_ctx* ctx, int32_t enable);
 int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launches);
 const char* rtma_kernel_class_name(int32_t cls);
 
+/* Self-test of the device-side failure path.  Every wait inside the library's kernels is
+ * bounded: a wait that runs out raises the context's device error word, the kernel winds down and
+ * the next rtma_check returns RTMA_ERR_TIMEOUT, leaving the context usable.  This call launches a
+ * one-block kernel whose wait can never be satisfied (a barrier nothing arrives at, about a
+ * thousand polls) so that the path can be exercised without faulting or hanging the device.
+ * The paper has no counterpart.                                                             */
+int32_t rtma_selftest_wait_timeout(rtma_ctx* ctx, void* stream);
+
 /* ---- the whole path on HOST buffers (Sec. 3: partition, Algorithm 2, Algorithm 1) --------
  * Every pointer here is a HOST pointer (pageable or pinned).  Copies the graph (CSR as for
  * rtma_build_induced_csr), group_id_h (NULL = RandomTMA), features X_h [n][dims[0]], labels

@@ -22,7 +22,7 @@ EXPORTS = (
     "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
-    "rtma_local_steps_var", "rtma_aggregate_masked",
+    "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout",
 )
 KERNEL_CLASSES = 20
 
@@ -307,6 +307,11 @@ class Context:
                                           ctypes.c_int64(P), ctypes.c_int32(M), _ptr(global_out),
                                           ctypes.c_void_p(_stream_handle(stream)))
         self._check(st, "rtma_sgd_aggregate")
+
+    def selftest_wait_timeout(self, stream=None):
+        """Launches a kernel whose bounded wait runs out; the next check() raises a timeout error."""
+        st = self._lib.rtma_selftest_wait_timeout(self._h, ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_selftest_wait_timeout")
 
     # ---- whole path from host buffers -----------------------------------------------
     def train_host(self, rowptr, col, X, y, dims, M, K, R, lr, seed, params0, group_id=None, gemm_dtype=0,

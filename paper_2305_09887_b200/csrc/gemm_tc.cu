@@ -601,6 +601,32 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 }
 
 // ------------------------------------------------------------------------------------
+// self-test of the bounded wait: a barrier nothing ever arrives at
+// ------------------------------------------------------------------------------------
+__global__ void wait_selftest_kernel(int* error_word, int polls) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        tc::fence_barrier_init();
+        bool done = false;
+        for (int i = 0; i < polls && !done; ++i) done = tc::mbar_try_wait(&bar, 0);
+        if (!done) atomicExch(error_word, 2);  // gave up, as the pipeline kernels do
+    }
+}
+
+}  // namespace
+
+extern "C" int32_t rtma_selftest_wait_timeout(rtma_ctx* ctx, void* stream) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->error_word, 1 << 10);
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}
+
+namespace {
+
+// ------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

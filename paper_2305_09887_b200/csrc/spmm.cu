@@ -190,8 +190,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
                         const int colx = (c * 32 + lane) * 8;
-                        xh[j][c] = xl[j][c] = make_uint4(0u, 0u, 0u, 0u);
-                        if (nb[j] >= 0 && colx < d) {
+                        if (nb[j] >= 0 && colx < d) {  // the same condition guards every use below
                             xh[j][c] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)nb[j] * src.ld + colx));
                             xl[j][c] = __ldg(reinterpret_cast<const uint4*>(sl + (int64_t)nb[j] * src.ld + colx));
                         }
@@ -206,6 +205,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
                     }
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
+                        if ((c * 32 + lane) * 8 >= d) continue;
                         if (MODE != 0) acc[c].fma_planes_mixed(wt[j], xh[j][c], xl[j][c]);
                         else acc[c].add_planes_mixed(xh[j][c], xl[j][c]);
                     }

@@ -297,6 +297,9 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             RTMA_TRY(launch_to_planes(ctx, g, Xp, m.dims[0], Hl[0], s));
             const Planes no_planes{nullptr, nullptr, 0};
             const Mat no_mat{nullptr, 0};
+            // N^0 = (aggregated input features), once for all steps of the call
+            if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], false, wave_order, ticket, s));
+            else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], wave_order, ticket, s));
             const GroupDesc wave = g;   // all parts of the wave, with their scratch rows
             const SplitPlan wave_sp = sp;
             for (int step = 0; step < wave_steps; ++step) {
@@ -332,8 +335,13 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 for (int l = 0; l < m.L; ++l)
                     RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
                 for (int l = 0; l < m.L; ++l) {
-                    if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], false, order, ticket, s));
-                    else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], order, ticket, s));
+                    if (l == 0) {
+                        // the aggregate of the input features does not change from step to step
+                    } else if (m.gcn) {
+                        RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], false, order, ticket, s));
+                    } else {
+                        RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], order, ticket, s));
+                    }
                     const bool last = l == m.L - 1;
                     if (last || !m.post) {
                         RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],

@@ -245,3 +245,16 @@ def test_whole_path_from_host_buffers(util, tiny_workload):
     assert (kept, cut) == (res["kept"], res["cut"])
     assert util.rel_err(params, res["params"][0]) <= TOL_PARAM
     assert np.abs(losses - res["losses"]).max() <= 1e-4
+
+
+def test_bounded_wait_that_runs_out_is_reported_and_leaves_the_context_usable(util, tiny_workload):
+    # the failure path of every device-side wait: a barrier nothing arrives at; no fault, no hang
+    from paper_2305_09887_b200 import binding
+    c = util.ctx()
+    c.check()
+    c.selftest_wait_timeout()
+    with pytest.raises(binding.RtmaError, match="bounded wait"):
+        c.check()
+    c.check()                                        # the error word was cleared by the report
+    w = tiny_workload                                # and the context still trains correctly
+    got, want = util.check_one_step(w)
