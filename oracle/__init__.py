@@ -324,6 +324,58 @@ def local_steps_variant(variant, dims, lr, rowptr, col, X, y, params, K):
     return params, loss
 
 
+# ---- link prediction --------------------------------------------------------------------------
+def link_param_count(variant, dims, ddims) -> int:
+    f = lib().orc_link_param_count
+    f.restype = ctypes.c_int64
+    return int(f(_p(_variant(variant), c_i32p), ctypes.c_int32(len(dims) - 1), _p(_i32(dims), c_i32p),
+                 ctypes.c_int32(len(ddims) - 1), _p(_i32(ddims), c_i32p)))
+
+
+def link_decoder_layout(variant, dims, ddims):
+    """[(theta offset, slope offset or -1)] per decoder layer."""
+    Kd = len(ddims) - 1
+    off = np.empty(2 * Kd, dtype=np.int64)
+    lib().orc_link_decoder_layout(_p(_variant(variant), c_i32p), ctypes.c_int32(len(dims) - 1), _p(_i32(dims), c_i32p),
+                                  ctypes.c_int32(Kd), _p(_i32(ddims), c_i32p), _p(off, c_i64p))
+    return [(int(off[2 * k]), int(off[2 * k + 1])) for k in range(Kd)]
+
+
+def link_init_params(variant, dims, ddims, seed) -> np.ndarray:
+    """Encoder as variant_init_params; decoder Xavier-uniform weights, slopes 0.25 (fp64)."""
+    enc = variant_init_params(variant, dims, seed)
+    rng = np.random.default_rng(seed + 1000)
+    p = np.zeros(link_param_count(variant, dims, ddims), dtype=np.float64)
+    p[:enc.size] = enc
+    for k, (theta, slope) in enumerate(link_decoder_layout(variant, dims, ddims)):
+        a = np.sqrt(6.0 / (ddims[k] + ddims[k + 1]))
+        p[theta:theta + ddims[k] * ddims[k + 1]] = rng.uniform(-a, a, size=ddims[k] * ddims[k + 1])
+        if slope >= 0:
+            p[slope] = 0.25
+    return p
+
+
+def link_forward_backward(variant, dims, ddims, rowptr, col, X, pu, pv, label, params, want_grads=True):
+    """Encoder + MLP decoder + binary cross-entropy on the given pairs of one part (fp64).
+    Returns (loss, grads or None, embeddings [n, dims[-1]], scores [B])."""
+    X = np.ascontiguousarray(X, dtype=np.float64)
+    params = np.ascontiguousarray(params, dtype=np.float64)
+    rowptr, col = _i64(rowptr), _i32(col)
+    pu, pv, label = _i32(pu), _i32(pv), _i32(label)
+    n, B = rowptr.size - 1, pu.size
+    assert ddims[0] == dims[-1] and ddims[-1] == 1 and params.size == link_param_count(variant, dims, ddims)
+    grads = np.empty(params.size, dtype=np.float64) if want_grads else None
+    emb = np.empty((n, dims[-1]), dtype=np.float64)
+    scores = np.empty(B, dtype=np.float64)
+    f = lib().orc_link_forward_backward_f64
+    f.restype = ctypes.c_double
+    loss = f(_p(_variant(variant), c_i32p), ctypes.c_int32(len(dims) - 1), _p(_i32(dims), c_i32p),
+             ctypes.c_int32(len(ddims) - 1), _p(_i32(ddims), c_i32p), ctypes.c_int64(n), _p(rowptr, c_i64p),
+             _p(col, c_i32p), _p(X, c_f64p), ctypes.c_int64(B), _p(pu, c_i32p), _p(pv, c_i32p), _p(label, c_i32p),
+             _p(params, c_f64p), _p(grads, c_f64p), _p(emb, c_f64p), _p(scores, c_f64p))
+    return float(loss), grads, emb, scores
+
+
 def average(params: np.ndarray):
     """params [M, P] -> (averaged copies [M, P], global [P])."""
     tag, ptr, dt = _fp(params.dtype)

@@ -24,6 +24,9 @@
 //   orc_*_variant         the encoders the paper's experiments use (Sec. 4.1): GCN
 //                         (Kipf & Welling) or GraphSAGE-mean layers, PReLU, Layer
 //                         Normalization before the activation.
+//   orc_link_*            the paper's task: link prediction with the Hadamard-product MLP
+//                         decoder (App. "Formulation of MLP Decoder") on given positive and
+//                         negative pairs (Sec. 4.1 "Mini-batch and Negative Sampling").
 //   orc_sigmoid_l2_grad   the 1-layer sigmoid / L2 model of Theorem 2, used
 //                         only to pin the aggregation against Eq.
 //                         (proof-2-exp-grad-central).
@@ -558,6 +561,305 @@ void local_steps_variant(const Variant& m, int32_t L, const int32_t* dims, doubl
     }
 }
 
+// ---- link prediction (Sec. 4.1 "Link Prediction Decoder", "Mini-batch and Negative Sampling";
+// App. "Formulation of MLP Decoder") -----------------------------------------------------------
+// The encoder is any model variant whose last layer outputs the node embeddings r (no softmax).
+// For a pair (u, v): e^0 = r_u (.) r_v (element-wise product), e^{k+1} = PReLU_k(e^k Theta^k) for the
+// hidden decoder layers, and the last layer gives the scalar score s = e^{Kd-1} Theta^{Kd-1}
+// (no bias anywhere, as the formula has none).  The probability of a link is sigmoid(s) and the
+// loss is the binary cross-entropy averaged over the batch (label 1: an edge of the training
+// graph, label 0: a sampled pair (u, v')).  The pairs and their labels are inputs: drawing them
+// is the caller's business.  Decoder parameters follow the encoder's in the flat vector:
+// Theta^0 [dd_0 x dd_1], [slope_0], Theta^1, [slope_1], ..., Theta^{Kd-1} [dd_{Kd-1} x 1];
+// dd_0 = the embedding width, dd_Kd = 1.
+struct DLayer {
+    int64_t d_in, d_out, theta, slope;  // offsets; slope -1 for the last layer
+};
+
+std::vector<DLayer> decoder_layers(int32_t Kd, const int32_t* ddims, int64_t first, int64_t* total) {
+    std::vector<DLayer> v(Kd);
+    int64_t off = first;
+    for (int32_t k = 0; k < Kd; ++k) {
+        v[k].d_in = ddims[k];
+        v[k].d_out = ddims[k + 1];
+        v[k].theta = off;
+        off += v[k].d_in * v[k].d_out;
+        v[k].slope = -1;
+        if (k < Kd - 1) v[k].slope = off++;
+    }
+    *total = off;
+    return v;
+}
+
+// Forward + backward of encoder and decoder on one part.  emb / scores (optional): the node
+// embeddings [n x dims[L]] and the pair scores [B].  Returns the loss.
+template <class T>
+double link_forward_backward(const Variant& m, int32_t L, const int32_t* dims, int32_t Kd, const int32_t* ddims,
+                             int64_t n, const int64_t* rowptr, const int32_t* col, const T* X, int64_t B,
+                             const int32_t* pu, const int32_t* pv, const int32_t* label, const T* params, T* grads,
+                             T* emb, T* scores) {
+    int64_t Penc = 0, P = 0;
+    const std::vector<VLayer> lv = variant_layers(m, L, dims, &Penc);
+    const std::vector<DLayer> dl = decoder_layers(Kd, ddims, Penc, &P);
+    if (grads) for (int64_t i = 0; i < P; ++i) grads[i] = (T)0;
+    if (n == 0 || B == 0) return 0.0;
+    const int64_t de = dims[L];
+
+    // ---- encoder forward (as in forward_backward_variant, without the loss) ----
+    std::vector<std::vector<T>> H(L + 1), N(L), U(L), XH(L);
+    std::vector<std::vector<double>> rstd(L);
+    std::vector<std::vector<char>> open(L);
+    H[0].assign(X, X + n * lv[0].d_in);
+    for (int32_t l = 0; l < L; ++l) {
+        const int64_t di = lv[l].d_in, dn = lv[l].d_out;
+        const bool hidden = l < L - 1;
+        N[l].resize(n * di);
+        if (m.encoder == 0) spmm_mean<T>(n, rowptr, col, di, H[l].data(), N[l].data());
+        else spmm_gcn<T>(n, rowptr, col, di, H[l].data(), N[l].data());
+        U[l].resize(n * dn);
+        H[l + 1].resize(n * dn);
+        open[l].assign(n * dn, 1);
+        if (hidden && m.norm == 1) {
+            XH[l].resize(n * dn);
+            rstd[l].resize(n);
+        }
+        const T* W0 = params + lv[l].w0;
+        const T* W1 = lv[l].w1 >= 0 ? params + lv[l].w1 : nullptr;
+        const T* b = params + lv[l].bias;
+        const double slope = !hidden ? 1.0 : (m.act == 1 ? (double)params[lv[l].slope] : 0.0);
+        std::vector<double> acc(dn);
+        std::vector<T> z(dn);
+        for (int64_t v = 0; v < n; ++v) {
+            for (int64_t j = 0; j < dn; ++j) acc[j] = (double)b[j];
+            for (int64_t k = 0; k < di; ++k) {
+                const double a0 = m.encoder == 0 ? (double)H[l][v * di + k] : (double)N[l][v * di + k];
+                const T* w0 = W0 + k * dn;
+                for (int64_t j = 0; j < dn; ++j) acc[j] += a0 * (double)w0[j];
+                if (W1) {
+                    const double a1 = (double)N[l][v * di + k];
+                    const T* w1 = W1 + k * dn;
+                    for (int64_t j = 0; j < dn; ++j) acc[j] += a1 * (double)w1[j];
+                }
+            }
+            for (int64_t j = 0; j < dn; ++j) z[j] = (T)acc[j];
+            if (!hidden) {
+                for (int64_t j = 0; j < dn; ++j) U[l][v * dn + j] = H[l + 1][v * dn + j] = z[j];
+                continue;
+            }
+            if (m.norm == 1) {
+                double mean = 0.0, var = 0.0;
+                for (int64_t j = 0; j < dn; ++j) mean += (double)z[j];
+                mean /= (double)dn;
+                for (int64_t j = 0; j < dn; ++j) var += ((double)z[j] - mean) * ((double)z[j] - mean);
+                var /= (double)dn;
+                const double rs = 1.0 / std::sqrt(var + LN_EPS);
+                rstd[l][v] = rs;
+                for (int64_t j = 0; j < dn; ++j) {
+                    const double xh = ((double)z[j] - mean) * rs;
+                    XH[l][v * dn + j] = (T)xh;
+                    U[l][v * dn + j] = (T)((double)params[lv[l].gamma + j] * xh + (double)params[lv[l].beta + j]);
+                }
+            } else {
+                for (int64_t j = 0; j < dn; ++j) U[l][v * dn + j] = z[j];
+            }
+            for (int64_t j = 0; j < dn; ++j) {
+                const T u = U[l][v * dn + j];
+                open[l][v * dn + j] = u > (T)0 ? 1 : 0;
+                H[l + 1][v * dn + j] = u > (T)0 ? u : (T)(slope * (double)u);
+            }
+        }
+    }
+    const std::vector<T>& R = H[L];
+    if (emb) std::memcpy(emb, R.data(), sizeof(T) * R.size());
+
+    // ---- decoder forward ----
+    std::vector<std::vector<T>> E(Kd + 1), ZD(Kd);
+    E[0].resize(B * de);
+    for (int64_t p = 0; p < B; ++p)
+        for (int64_t j = 0; j < de; ++j)
+            E[0][p * de + j] = (T)((double)R[(int64_t)pu[p] * de + j] * (double)R[(int64_t)pv[p] * de + j]);
+    for (int32_t k = 0; k < Kd; ++k) {
+        const int64_t di = dl[k].d_in, dn = dl[k].d_out;
+        const T* Th = params + dl[k].theta;
+        const double slope = dl[k].slope >= 0 ? (double)params[dl[k].slope] : 1.0;
+        ZD[k].resize(B * dn);
+        E[k + 1].resize(B * dn);
+        std::vector<double> acc(dn);
+        for (int64_t p = 0; p < B; ++p) {
+            for (int64_t j = 0; j < dn; ++j) acc[j] = 0.0;
+            for (int64_t i = 0; i < di; ++i) {
+                const double e = (double)E[k][p * di + i];
+                for (int64_t j = 0; j < dn; ++j) acc[j] += e * (double)Th[i * dn + j];
+            }
+            for (int64_t j = 0; j < dn; ++j) {
+                const T z = (T)acc[j];
+                ZD[k][p * dn + j] = z;
+                E[k + 1][p * dn + j] = (k == Kd - 1 || z > (T)0) ? z : (T)(slope * (double)z);
+            }
+        }
+    }
+    // ---- binary cross-entropy on the scores ----
+    std::vector<T> dZ(B);  // gradient with respect to the last layer's output
+    double loss = 0.0;
+    for (int64_t p = 0; p < B; ++p) {
+        const double s = (double)E[Kd][p];
+        if (scores) scores[p] = (T)s;
+        // log(1 + exp(-|s|)) + max(s, 0) - y s, the stable form of -[y log sig(s) + (1-y) log(1 - sig(s))]
+        loss += std::log1p(std::exp(-std::fabs(s))) + std::fmax(s, 0.0) - (double)label[p] * s;
+        const double sig = 1.0 / (1.0 + std::exp(-s));
+        dZ[p] = (T)((sig - (double)label[p]) / (double)B);
+    }
+    loss /= (double)B;
+    if (!grads) return loss;
+
+    // ---- decoder backward ----
+    std::vector<T> dE;  // gradient with respect to E[k]
+    for (int32_t k = Kd - 1; k >= 0; --k) {
+        const int64_t di = dl[k].d_in, dn = dl[k].d_out;
+        const T* Th = params + dl[k].theta;
+        std::vector<double> gt(di * dn, 0.0);
+        for (int64_t p = 0; p < B; ++p)
+            for (int64_t i = 0; i < di; ++i) {
+                const double e = (double)E[k][p * di + i];
+                for (int64_t j = 0; j < dn; ++j) gt[i * dn + j] += e * (double)dZ[p * dn + j];
+            }
+        for (int64_t i = 0; i < di * dn; ++i) grads[dl[k].theta + i] = (T)gt[i];
+        dE.assign(B * di, (T)0);
+        for (int64_t p = 0; p < B; ++p)
+            for (int64_t i = 0; i < di; ++i) {
+                double s = 0.0;
+                for (int64_t j = 0; j < dn; ++j) s += (double)dZ[p * dn + j] * (double)Th[i * dn + j];
+                dE[p * di + i] = (T)s;
+            }
+        if (k == 0) break;
+        // through the PReLU of decoder layer k-1
+        const double slope = (double)params[dl[k - 1].slope];
+        double g_slope = 0.0;
+        std::vector<T> dZprev(B * di);
+        for (int64_t i = 0; i < B * di; ++i) {
+            const double z = (double)ZD[k - 1][i], g = (double)dE[i];
+            if (z > 0.0) {
+                dZprev[i] = (T)g;
+            } else {
+                dZprev[i] = (T)(slope * g);
+                g_slope += g * z;
+            }
+        }
+        grads[dl[k - 1].slope] = (T)g_slope;
+        dZ.swap(dZprev);
+    }
+    // ---- into the embeddings: d r_u += dE0 (.) r_v, d r_v += dE0 (.) r_u ----
+    std::vector<double> dR(n * de, 0.0);
+    for (int64_t p = 0; p < B; ++p)
+        for (int64_t j = 0; j < de; ++j) {
+            const double g = (double)dE[p * de + j];
+            dR[(int64_t)pu[p] * de + j] += g * (double)R[(int64_t)pv[p] * de + j];
+            dR[(int64_t)pv[p] * de + j] += g * (double)R[(int64_t)pu[p] * de + j];
+        }
+    std::vector<T> dZe(n * de);
+    for (int64_t i = 0; i < n * de; ++i) dZe[i] = (T)dR[i];
+
+    // ---- encoder backward (as in forward_backward_variant) ----
+    for (int32_t l = L - 1; l >= 0; --l) {
+        const int64_t di = lv[l].d_in, dn = lv[l].d_out;
+        const T* W0 = params + lv[l].w0;
+        const T* W1 = lv[l].w1 >= 0 ? params + lv[l].w1 : nullptr;
+        {
+            std::vector<double> g0(di * dn, 0.0), g1(W1 ? di * dn : 0, 0.0), gb(dn, 0.0);
+            for (int64_t v = 0; v < n; ++v) {
+                const T* dz = &dZe[v * dn];
+                for (int64_t j = 0; j < dn; ++j) gb[j] += (double)dz[j];
+                for (int64_t k = 0; k < di; ++k) {
+                    const double a0 = m.encoder == 0 ? (double)H[l][v * di + k] : (double)N[l][v * di + k];
+                    for (int64_t j = 0; j < dn; ++j) g0[k * dn + j] += a0 * (double)dz[j];
+                    if (W1) {
+                        const double a1 = (double)N[l][v * di + k];
+                        for (int64_t j = 0; j < dn; ++j) g1[k * dn + j] += a1 * (double)dz[j];
+                    }
+                }
+            }
+            for (int64_t i = 0; i < di * dn; ++i) grads[lv[l].w0 + i] = (T)g0[i];
+            if (W1) for (int64_t i = 0; i < di * dn; ++i) grads[lv[l].w1 + i] = (T)g1[i];
+            for (int64_t j = 0; j < dn; ++j) grads[lv[l].bias + j] = (T)gb[j];
+        }
+        if (l == 0) break;
+        std::vector<double> dH(n * di, 0.0), dN(di);
+        for (int64_t v = 0; v < n; ++v) {
+            const T* dz = &dZe[v * dn];
+            for (int64_t k = 0; k < di; ++k) {
+                double s = 0.0, t2 = 0.0;
+                for (int64_t j = 0; j < dn; ++j) {
+                    s += (double)dz[j] * (double)W0[k * dn + j];
+                    if (W1) t2 += (double)dz[j] * (double)W1[k * dn + j];
+                }
+                if (m.encoder == 0) {
+                    dH[v * di + k] += s;
+                    dN[k] = t2;
+                } else {
+                    dN[k] = s;
+                }
+            }
+            if (m.encoder == 0) {
+                const int64_t deg = rowptr[v + 1] - rowptr[v];
+                for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e)
+                    for (int64_t k = 0; k < di; ++k) dH[(int64_t)col[e] * di + k] += dN[k] / (double)deg;
+            } else {
+                const double sv = 1.0 / std::sqrt((double)(rowptr[v + 1] - rowptr[v] + 1));
+                for (int64_t k = 0; k < di; ++k) dH[v * di + k] += sv * sv * dN[k];
+                for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+                    const int64_t u = col[e];
+                    const double su = 1.0 / std::sqrt((double)(rowptr[u + 1] - rowptr[u] + 1));
+                    for (int64_t k = 0; k < di; ++k) dH[u * di + k] += sv * su * dN[k];
+                }
+            }
+        }
+        const int32_t q = l - 1;
+        const double slope = m.act == 1 ? (double)params[lv[q].slope] : 0.0;
+        std::vector<T> dZprev(n * di);
+        std::vector<double> g_gamma(m.norm == 1 ? di : 0, 0.0), g_beta(m.norm == 1 ? di : 0, 0.0), dU(di);
+        double g_slope = 0.0;
+        for (int64_t v = 0; v < n; ++v) {
+            for (int64_t k = 0; k < di; ++k) {
+                const int64_t i = v * di + k;
+                const double g = dH[i];
+                if (open[q][i]) {
+                    dU[k] = g;
+                } else {
+                    dU[k] = slope * g;
+                    g_slope += g * (double)U[q][i];
+                }
+            }
+            if (m.norm == 1) {
+                double m1 = 0.0, m2 = 0.0;
+                for (int64_t k = 0; k < di; ++k) {
+                    const double xh = (double)XH[q][v * di + k];
+                    g_gamma[k] += dU[k] * xh;
+                    g_beta[k] += dU[k];
+                    const double dx = dU[k] * (double)params[lv[q].gamma + k];
+                    m1 += dx;
+                    m2 += dx * xh;
+                }
+                m1 /= (double)di;
+                m2 /= (double)di;
+                for (int64_t k = 0; k < di; ++k) {
+                    const double xh = (double)XH[q][v * di + k];
+                    const double dx = dU[k] * (double)params[lv[q].gamma + k];
+                    dZprev[v * di + k] = (T)(rstd[q][v] * (dx - m1 - xh * m2));
+                }
+            } else {
+                for (int64_t k = 0; k < di; ++k) dZprev[v * di + k] = (T)dU[k];
+            }
+        }
+        if (m.norm == 1) {
+            for (int64_t k = 0; k < di; ++k) grads[lv[q].gamma + k] = (T)g_gamma[k];
+            for (int64_t k = 0; k < di; ++k) grads[lv[q].beta + k] = (T)g_beta[k];
+        }
+        if (m.act == 1) grads[lv[q].slope] = (T)g_slope;
+        dZe.swap(dZprev);
+    }
+    return loss;
+}
+
 template <class T>
 void average(T* params, int64_t P, int32_t M, T* global_out) {
     for (int64_t j = 0; j < P; ++j) {
@@ -702,6 +1004,33 @@ void orc_local_steps_variant_f64(const int32_t* variant, int32_t L, const int32_
                                  double* params, int32_t K, double* loss_out) {
     local_steps_variant<double>(Variant{variant[0], variant[1], variant[2]}, L, dims, lr, n, rowptr, col, X, y, params, K,
                                 loss_out);
+}
+
+// ---- link prediction: encoder variant + MLP decoder, binary cross-entropy on given pairs ---------
+int64_t orc_link_param_count(const int32_t* variant, int32_t L, const int32_t* dims, int32_t Kd, const int32_t* ddims) {
+    int64_t Penc = 0, P = 0;
+    variant_layers(Variant{variant[0], variant[1], variant[2]}, L, dims, &Penc);
+    decoder_layers(Kd, ddims, Penc, &P);
+    return P;
+}
+// offsets[k * 2 + {0, 1}] = Theta^k, slope_k (-1 = absent) of decoder layer k
+void orc_link_decoder_layout(const int32_t* variant, int32_t L, const int32_t* dims, int32_t Kd, const int32_t* ddims,
+                             int64_t* offsets) {
+    int64_t Penc = 0, P = 0;
+    variant_layers(Variant{variant[0], variant[1], variant[2]}, L, dims, &Penc);
+    const std::vector<DLayer> dl = decoder_layers(Kd, ddims, Penc, &P);
+    for (int32_t k = 0; k < Kd; ++k) {
+        offsets[2 * k] = dl[k].theta;
+        offsets[2 * k + 1] = dl[k].slope;
+    }
+}
+double orc_link_forward_backward_f64(const int32_t* variant, int32_t L, const int32_t* dims, int32_t Kd,
+                                     const int32_t* ddims, int64_t n, const int64_t* rowptr, const int32_t* col,
+                                     const double* X, int64_t B, const int32_t* pu, const int32_t* pv,
+                                     const int32_t* label, const double* params, double* grads, double* emb,
+                                     double* scores) {
+    return link_forward_backward<double>(Variant{variant[0], variant[1], variant[2]}, L, dims, Kd, ddims, n, rowptr, col,
+                                         X, B, pu, pv, label, params, grads, emb, scores);
 }
 
 // Theorem 2's model: z_v = sigmoid((A-bar X w)_v), L = 1/2 (y_v - z_v)^2 per
