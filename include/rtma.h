@@ -206,6 +206,41 @@ int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* model, int32_
                              const int32_t* steps_host, int32_t loss_stride, float* loss_out,
                              const rtma_taps* taps, void* const* streams);
 
+/* ---- link prediction (Sec. 4.1 "Link Prediction Decoder", "Mini-batch and Negative Sampling";
+ * App. "Formulation of MLP Decoder") ---------------------------------------------------------
+ * The paper's own task.  The encoder is `model` (any variant); its last layer outputs the node
+ * embeddings r [dims[L]] instead of class scores.  For a pair (u, v): e^0 = r_u (.) r_v
+ * (element-wise), e^{k+1} = PReLU_k(e^k Theta^k) for the hidden decoder layers, the last layer
+ * gives the scalar score s = e^{Kd-1} Theta^{Kd-1} (no biases, as in the paper's formula); the
+ * link probability is sigmoid(s) and the loss the binary cross-entropy averaged over the part's
+ * pairs (label 1: an edge of the training subgraph, 0: a sampled pair (u, v')).  Pairs and labels
+ * are INPUTS (the paper draws them at random; drawing is the caller's business), as local ids of
+ * the part.  The encoder runs on the whole part (no neighbour sampling).
+ *   decoder     Kd layers, ddims[0] = dims[L], ddims[Kd] = 1.
+ *   parameters  [M][P], P = rtma_link_param_count(): the encoder's parameters, then Theta^0
+ *               [ddims[0]][ddims[1]], slope_0, Theta^1, slope_1, ..., Theta^{Kd-1} (no slope).
+ *   pair_offsets_host  HOST [M+1]: part p's pairs are pair_u/pair_v/pair_label[pair_offsets[p] ..).
+ *   loss_out [M][K] or NULL.  record_step >= 0: at that step grads_out [M][P] (or NULL) receives
+ *   the gradient applied, emb_out [n][dims[L]] (or NULL) the embeddings, score_out [pairs] (or
+ *   NULL) the scores.  Everything else as for rtma_local_steps; all trainers run K steps on the
+ *   same pairs (a caller that wants a fresh mini-batch per step calls with K = 1).
+ * The gradient of the embeddings is accumulated with floating-point atomics: its last bits, and
+ * with them the result, can differ between runs (unlike rtma_local_steps).                   */
+typedef struct {
+    int32_t Kd;
+    int32_t ddims[RTMA_MAX_LAYERS + 1];
+} rtma_decoder_desc;
+
+int64_t rtma_link_param_count(const rtma_model_desc* model, const rtma_decoder_desc* decoder);
+
+int32_t rtma_link_steps(rtma_ctx* ctx, const rtma_model_desc* model, const rtma_decoder_desc* decoder,
+                        int32_t M, const int64_t* part_offsets_host, const int64_t* edge_offsets_host,
+                        const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                        const float* Xp, const int64_t* pair_offsets_host, const int32_t* pair_u,
+                        const int32_t* pair_v, const int32_t* pair_label, float* params, int32_t K,
+                        float* loss_out, int32_t record_step, float* grads_out, float* emb_out,
+                        float* score_out, void* const* streams);
+
 /* ---- R2: aggregation (Algorithm 1, phi = plain average; Algorithm 2, overwrite) ---------
  * Wbar[j] = (1/M) sum_i params[i][j]; every replica is overwritten with Wbar; global_out
  * [P] (or NULL) also receives it.  M = 1 leaves the parameters unchanged.                 */
@@ -232,7 +267,7 @@ int32_t rtma_sgd_aggregate(rtma_ctx* ctx, float* params, const float* grads, flo
  * summed per class (ms [RTMA_KERNEL_CLASSES], milliseconds; zeros if profiling was off) and the
  * launch counts (launches [RTMA_KERNEL_CLASSES]) since the previous read, and resets both.
  * Either output may be NULL.  The paper has no counterpart; these feed the roofline report.  */
-#define RTMA_KERNEL_CLASSES 20
+#define RTMA_KERNEL_CLASSES 21
 int32_t rtma_profile(rtma_ctx* ctx, int32_t enable);
 int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launches);
 const char* rtma_kernel_class_name(int32_t cls);

@@ -355,9 +355,13 @@ def link_init_params(variant, dims, ddims, seed) -> np.ndarray:
     return p
 
 
-def link_forward_backward(variant, dims, ddims, rowptr, col, X, pu, pv, label, params, want_grads=True):
+def link_forward_backward(variant, dims, ddims, rowptr, col, X, pu, pv, label, params, want_grads=True,
+                          preact_out=None, gates=None):
     """Encoder + MLP decoder + binary cross-entropy on the given pairs of one part (fp64).
-    Returns (loss, grads or None, embeddings [n, dims[-1]], scores [B])."""
+    Returns (loss, grads or None, embeddings [n, dims[-1]], scores [B]).
+    preact_out: None or a float64 array of link_gate_count() entries that receives the input of
+    every hidden ReLU / PReLU (encoder layers, then decoder layers); gates: None or an int8 array
+    of the same length (-1 natural, 0 closed, 1 open)."""
     X = np.ascontiguousarray(X, dtype=np.float64)
     params = np.ascontiguousarray(params, dtype=np.float64)
     rowptr, col = _i64(rowptr), _i32(col)
@@ -372,8 +376,13 @@ def link_forward_backward(variant, dims, ddims, rowptr, col, X, pu, pv, label, p
     loss = f(_p(_variant(variant), c_i32p), ctypes.c_int32(len(dims) - 1), _p(_i32(dims), c_i32p),
              ctypes.c_int32(len(ddims) - 1), _p(_i32(ddims), c_i32p), ctypes.c_int64(n), _p(rowptr, c_i64p),
              _p(col, c_i32p), _p(X, c_f64p), ctypes.c_int64(B), _p(pu, c_i32p), _p(pv, c_i32p), _p(label, c_i32p),
-             _p(params, c_f64p), _p(grads, c_f64p), _p(emb, c_f64p), _p(scores, c_f64p))
+             _p(params, c_f64p), _p(grads, c_f64p), _p(emb, c_f64p), _p(scores, c_f64p), _p(preact_out, c_f64p),
+             _p(None if gates is None else np.ascontiguousarray(gates, dtype=np.int8), ctypes.POINTER(ctypes.c_int8)))
     return float(loss), grads, emb, scores
+
+
+def link_gate_count(dims, ddims, n: int, B: int) -> int:
+    return n * sum(dims[1:-1]) + B * sum(ddims[1:-1])
 
 
 def average(params: np.ndarray):

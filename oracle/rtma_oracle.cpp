@@ -592,23 +592,38 @@ std::vector<DLayer> decoder_layers(int32_t Kd, const int32_t* ddims, int64_t fir
 }
 
 // Forward + backward of encoder and decoder on one part.  emb / scores (optional): the node
-// embeddings [n x dims[L]] and the pair scores [B].  Returns the loss.
+// embeddings [n x dims[L]] and the pair scores [B].  preact (optional): the inputs of every PReLU /
+// ReLU, encoder hidden layers [n x dims[l+1]] then decoder hidden layers [B x ddims[k+1]];
+// gates (optional, same layout): -1 = the rule (open iff input > 0), 0 / 1 = closed / open
+// regardless (see forward_backward).  Returns the loss.
 template <class T>
 double link_forward_backward(const Variant& m, int32_t L, const int32_t* dims, int32_t Kd, const int32_t* ddims,
                              int64_t n, const int64_t* rowptr, const int32_t* col, const T* X, int64_t B,
                              const int32_t* pu, const int32_t* pv, const int32_t* label, const T* params, T* grads,
-                             T* emb, T* scores) {
+                             T* emb, T* scores, T* preact, const int8_t* gates) {
     int64_t Penc = 0, P = 0;
     const std::vector<VLayer> lv = variant_layers(m, L, dims, &Penc);
     const std::vector<DLayer> dl = decoder_layers(Kd, ddims, Penc, &P);
     if (grads) for (int64_t i = 0; i < P; ++i) grads[i] = (T)0;
-    if (n == 0 || B == 0) return 0.0;
+    if (n == 0) return 0.0;
     const int64_t de = dims[L];
 
     // ---- encoder forward (as in forward_backward_variant, without the loss) ----
     std::vector<std::vector<T>> H(L + 1), N(L), U(L), XH(L);
     std::vector<std::vector<double>> rstd(L);
     std::vector<std::vector<char>> open(L);
+    std::vector<int64_t> gate_off(L + Kd, 0);   // offsets into preact / gates
+    {
+        int64_t o = 0;
+        for (int32_t l = 0; l + 1 < L; ++l) {
+            gate_off[l] = o;
+            o += n * lv[l].d_out;
+        }
+        for (int32_t k = 0; k + 1 < Kd; ++k) {
+            gate_off[L + k] = o;
+            o += B * dl[k].d_out;
+        }
+    }
     H[0].assign(X, X + n * lv[0].d_in);
     for (int32_t l = 0; l < L; ++l) {
         const int64_t di = lv[l].d_in, dn = lv[l].d_out;
@@ -664,16 +679,21 @@ double link_forward_backward(const Variant& m, int32_t L, const int32_t* dims, i
             }
             for (int64_t j = 0; j < dn; ++j) {
                 const T u = U[l][v * dn + j];
-                open[l][v * dn + j] = u > (T)0 ? 1 : 0;
-                H[l + 1][v * dn + j] = u > (T)0 ? u : (T)(slope * (double)u);
+                const int8_t forced = gates ? gates[gate_off[l] + v * dn + j] : (int8_t)-1;
+                const bool is_open = forced < 0 ? (u > (T)0) : (forced != 0);
+                open[l][v * dn + j] = is_open ? 1 : 0;
+                H[l + 1][v * dn + j] = is_open ? u : (T)(slope * (double)u);
             }
         }
+        if (hidden && preact) std::memcpy(preact + gate_off[l], U[l].data(), sizeof(T) * U[l].size());
     }
     const std::vector<T>& R = H[L];
     if (emb) std::memcpy(emb, R.data(), sizeof(T) * R.size());
+    if (B == 0) return 0.0;  // no pairs: the embeddings exist, the loss and every gradient are zero
 
     // ---- decoder forward ----
     std::vector<std::vector<T>> E(Kd + 1), ZD(Kd);
+    std::vector<std::vector<char>> dopen(Kd);
     E[0].resize(B * de);
     for (int64_t p = 0; p < B; ++p)
         for (int64_t j = 0; j < de; ++j)
@@ -684,6 +704,7 @@ double link_forward_backward(const Variant& m, int32_t L, const int32_t* dims, i
         const double slope = dl[k].slope >= 0 ? (double)params[dl[k].slope] : 1.0;
         ZD[k].resize(B * dn);
         E[k + 1].resize(B * dn);
+        dopen[k].assign(B * dn, 1);
         std::vector<double> acc(dn);
         for (int64_t p = 0; p < B; ++p) {
             for (int64_t j = 0; j < dn; ++j) acc[j] = 0.0;
@@ -694,9 +715,16 @@ double link_forward_backward(const Variant& m, int32_t L, const int32_t* dims, i
             for (int64_t j = 0; j < dn; ++j) {
                 const T z = (T)acc[j];
                 ZD[k][p * dn + j] = z;
-                E[k + 1][p * dn + j] = (k == Kd - 1 || z > (T)0) ? z : (T)(slope * (double)z);
+                bool is_open = true;
+                if (k < Kd - 1) {
+                    const int8_t forced = gates ? gates[gate_off[L + k] + p * dn + j] : (int8_t)-1;
+                    is_open = forced < 0 ? (z > (T)0) : (forced != 0);
+                }
+                dopen[k][p * dn + j] = is_open ? 1 : 0;
+                E[k + 1][p * dn + j] = is_open ? z : (T)(slope * (double)z);
             }
         }
+        if (k < Kd - 1 && preact) std::memcpy(preact + gate_off[L + k], ZD[k].data(), sizeof(T) * ZD[k].size());
     }
     // ---- binary cross-entropy on the scores ----
     std::vector<T> dZ(B);  // gradient with respect to the last layer's output
@@ -738,7 +766,7 @@ double link_forward_backward(const Variant& m, int32_t L, const int32_t* dims, i
         std::vector<T> dZprev(B * di);
         for (int64_t i = 0; i < B * di; ++i) {
             const double z = (double)ZD[k - 1][i], g = (double)dE[i];
-            if (z > 0.0) {
+            if (dopen[k - 1][i]) {
                 dZprev[i] = (T)g;
             } else {
                 dZprev[i] = (T)(slope * g);
@@ -1028,9 +1056,9 @@ double orc_link_forward_backward_f64(const int32_t* variant, int32_t L, const in
                                      const int32_t* ddims, int64_t n, const int64_t* rowptr, const int32_t* col,
                                      const double* X, int64_t B, const int32_t* pu, const int32_t* pv,
                                      const int32_t* label, const double* params, double* grads, double* emb,
-                                     double* scores) {
+                                     double* scores, double* preact, const int8_t* gates) {
     return link_forward_backward<double>(Variant{variant[0], variant[1], variant[2]}, L, dims, Kd, ddims, n, rowptr, col,
-                                         X, B, pu, pv, label, params, grads, emb, scores);
+                                         X, B, pu, pv, label, params, grads, emb, scores, preact, gates);
 }
 
 // Theorem 2's model: z_v = sigmoid((A-bar X w)_v), L = 1/2 (y_v - z_v)^2 per

@@ -22,9 +22,10 @@ EXPORTS = (
     "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
-    "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout",
+    "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout", "rtma_link_param_count",
+    "rtma_link_steps",
 )
-KERNEL_CLASSES = 20
+KERNEL_CLASSES = 21
 
 _lib = None
 
@@ -37,6 +38,21 @@ class ModelDesc(ctypes.Structure):
     _fields_ = [("L", ctypes.c_int32), ("dims", ctypes.c_int32 * (MAX_LAYERS + 1)),
                 ("gemm_dtype", ctypes.c_int32), ("lr", ctypes.c_float), ("encoder", ctypes.c_int32),
                 ("act", ctypes.c_int32), ("norm", ctypes.c_int32)]
+
+
+class DecoderDesc(ctypes.Structure):
+    _fields_ = [("Kd", ctypes.c_int32), ("ddims", ctypes.c_int32 * (MAX_LAYERS + 1))]
+
+
+def decoder_desc(ddims) -> DecoderDesc:
+    Kd = len(ddims) - 1
+    if not 1 <= Kd <= MAX_LAYERS:
+        raise ValueError(f"number of decoder layers {Kd} outside [1, {MAX_LAYERS}]")
+    dd = DecoderDesc()
+    dd.Kd = Kd
+    for i, d in enumerate(ddims):
+        dd.ddims[i] = int(d)
+    return dd
 
 
 class Taps(ctypes.Structure):
@@ -74,6 +90,12 @@ def model_desc(dims, lr: float = 0.01, gemm_dtype: int = 0, variant=(0, 0, 0)) -
     md.lr = float(lr)
     md.encoder, md.act, md.norm = (int(v) for v in variant)
     return md
+
+
+def link_param_count(dims, ddims, variant=(0, 0, 0)) -> int:
+    lib = load_library()
+    lib.rtma_link_param_count.restype = ctypes.c_int64
+    return int(lib.rtma_link_param_count(ctypes.byref(model_desc(dims, variant=variant)), ctypes.byref(decoder_desc(ddims))))
 
 
 def param_count(dims, variant=(0, 0, 0)) -> int:
@@ -281,6 +303,34 @@ class Context:
                 ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), _ptr(yp), _ptr(params), steps,
                 ctypes.c_int32(stride), _ptr(loss_out), tap_ref, sarr)
             self._check(st, "rtma_local_steps_var")
+
+    def link_steps(self, dims, ddims, lr, M, part_offsets_host, edge_offsets_host, rowptr_out, col_out, Xp,
+                   pair_offsets_host, pair_u, pair_v, pair_label, params, K, loss_out=None, record_step=-1,
+                   grads_out=None, emb_out=None, score_out=None, streams=None, gemm_dtype=0, variant=(0, 0, 0),
+                   symmetric=True):
+        """K SGD steps of link prediction (encoder `dims` + MLP decoder `ddims`) on the given pairs of
+        each part, in place on params [M, P].  pair_u / pair_v / pair_label: int32 device tensors of
+        local ids and 0/1 labels, part p's pairs at pair_offsets_host[p]:pair_offsets_host[p+1]."""
+        dev = self.device
+        md = model_desc(dims, lr, gemm_dtype, variant)
+        dd = decoder_desc(ddims)
+        _need(params, torch.float32, "params", dev)
+        _need(Xp, torch.float32, "Xp", dev)
+        _need(rowptr_out, torch.int64, "rowptr_out", dev)
+        _need(col_out, torch.int32, "col_out", dev)
+        for name, t in (("pair_u", pair_u), ("pair_v", pair_v), ("pair_label", pair_label)):
+            _need(t, torch.int32, name, dev)
+        po = (ctypes.c_int64 * (M + 1))(*[int(v) for v in part_offsets_host])
+        eo = (ctypes.c_int64 * (M + 1))(*[int(v) for v in edge_offsets_host])
+        qo = (ctypes.c_int64 * (M + 1))(*[int(v) for v in pair_offsets_host])
+        handles = [_stream_handle(None)] * M if streams is None else [_stream_handle(s) for s in streams]
+        sarr = (ctypes.c_void_p * M)(*handles)
+        st = self._lib.rtma_link_steps(
+            self._h, ctypes.byref(md), ctypes.byref(dd), ctypes.c_int32(M), po, eo, _ptr(rowptr_out), _ptr(col_out),
+            ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), qo, _ptr(pair_u), _ptr(pair_v), _ptr(pair_label),
+            _ptr(params), ctypes.c_int32(K), _ptr(loss_out), ctypes.c_int32(record_step), _ptr(grads_out),
+            _ptr(emb_out), _ptr(score_out), sarr)
+        self._check(st, "rtma_link_steps")
 
     # ---- R2 -------------------------------------------------------------------------
     def aggregate(self, params, global_out=None, stream=None):

@@ -15,7 +15,7 @@
 enum KernelClass {
     KC_PART_COUNT = 0, KC_SCAN, KC_PART_SCATTER, KC_CSR_COUNT, KC_CSR_OFFSETS, KC_CSR_FILL, KC_GATHER_ROWS,
     KC_INV_DEGREE, KC_SPMM_FWD, KC_SPMM_BWD, KC_GEMM_FWD, KC_GEMM_DGRAD, KC_GEMM_WGRAD, KC_LOSS, KC_REDUCE_SGD,
-    KC_AGGREGATE, KC_COPY, KC_WEIGHT_PREP, KC_TO_PLANES, KC_POST, KC_COUNT
+    KC_AGGREGATE, KC_COPY, KC_WEIGHT_PREP, KC_TO_PLANES, KC_POST, KC_LINK, KC_COUNT
 };
 static_assert(KC_COUNT == RTMA_KERNEL_CLASSES, "kernel class table out of step with rtma.h");
 

@@ -57,7 +57,7 @@ extern "C" size_t rtma_workspace_bytes(const rtma_ctx* ctx) { return ctx ? ctx->
 static const char* const kKernelClassNames[KC_COUNT] = {
     "partition_count", "scan", "partition_scatter", "induced_count", "induced_offsets", "induced_fill", "gather_rows",
     "inv_degree", "spmm_forward", "spmm_backward", "gemm_forward", "gemm_dgrad", "gemm_wgrad", "softmax_xent",
-    "reduce_sgd", "aggregate", "copy_rows", "weight_prep", "to_planes", "norm_act"};
+    "reduce_sgd", "aggregate", "copy_rows", "weight_prep", "to_planes", "norm_act", "link_pairs"};
 
 extern "C" const char* rtma_kernel_class_name(int32_t cls) {
     return cls >= 0 && cls < KC_COUNT ? kKernelClassNames[cls] : "";

@@ -784,7 +784,7 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
     a.ld_out = out_f32.ld;
     a.params = params;
     a.P = ls.P;
-    a.bias_offset = ls.param_offset + (int64_t)ls.nsrc * ls.d_in * ls.d_out;
+    a.bias_offset = ls.has_bias ? ls.param_offset + (int64_t)ls.nsrc * ls.d_in * ls.d_out : -1;
     a.relu = relu ? 1 : 0;
     a.gate_hi = nullptr;
     return launch_rows(ctx, a, KC_GEMM_FWD, s);

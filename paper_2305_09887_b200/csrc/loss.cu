@@ -125,6 +125,11 @@ int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C
         else softmax_xent_kernel<0><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         RTMA_LAUNCH_CHECK(ctx);
     }
+    return launch_loss_finalize(ctx, g, tile_loss, loss_out, loss_stride, loss_col, s);
+}
+
+int32_t launch_loss_finalize(rtma_ctx* ctx, const GroupDesc& g, const float* tile_loss, float* loss_out,
+                             int64_t loss_stride, int64_t loss_col, cudaStream_t s) {
     if (loss_out && g.num > 0) {
         { KernelScope ks(ctx, KC_LOSS, s); loss_finalize_kernel<<<g.num, 256, 0, s>>>(g, tile_loss, loss_out, loss_stride, loss_col); }
         RTMA_LAUNCH_CHECK(ctx);

@@ -13,11 +13,12 @@ reduce_sgd_kernel(const __grid_constant__ GroupDesc g, const __grid_constant__ S
                   const float* __restrict__ partial, const float lr, float* __restrict__ params,
                   float* __restrict__ grads_record) {
     const int k = blockIdx.y;
-    const int64_t count = (int64_t)(ls.nsrc * ls.d_in + 1) * ls.d_out;  // the weight matrices and the bias row
+    const int64_t stride = (int64_t)(ls.nsrc * ls.d_in + 1) * ls.d_out;  // the weight matrices and the bias row
+    const int64_t count = ls.has_bias ? stride : stride - ls.d_out;       // the bias row is last
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (i >= count) return;
     float gsum = 0.f;
-    for (int s = sp.split_begin[k]; s < sp.split_begin[k + 1]; ++s) gsum += partial[(int64_t)s * count + i];
+    for (int s = sp.split_begin[k]; s < sp.split_begin[k + 1]; ++s) gsum += partial[(int64_t)s * stride + i];
     const int64_t at = (int64_t)g.part[k] * ls.P + ls.param_offset + i;
     if (grads_record) grads_record[at] = gsum;
     params[at] -= lr * gsum;

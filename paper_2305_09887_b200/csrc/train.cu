@@ -15,7 +15,36 @@ struct Model {
     float lr;
     bool gcn;   // GCN layers (one weight matrix, renormalised adjacency) instead of GraphSAGE-mean
     bool post;  // hidden layers normalise and / or use PReLU: the activation is a pass of its own
+    int Kd;     // link prediction: decoder layers (0: node classification)
+    int ddims[RTMA_MAX_LAYERS + 1];
+    LayerShape dec[RTMA_MAX_LAYERS];
 };
+
+// Link prediction: what rtma_link_steps adds to the training loop.
+struct LinkTask {
+    const rtma_decoder_desc* dd;
+    const int64_t* pair_offsets;  // host [M + 1]
+    const int32_t *pu, *pv, *label;
+    float *emb_out, *score_out;
+};
+
+// Decoder parameters after the encoder's: Theta^k [ddims[k]][ddims[k+1]], then (hidden layers) the slope.
+int64_t layout_decoder(const rtma_decoder_desc* dd, int64_t first, LayerShape* layer) {
+    int64_t off = first;
+    for (int k = 0; k < dd->Kd; ++k) {
+        LayerShape ls{};
+        ls.d_in = dd->ddims[k];
+        ls.d_out = dd->ddims[k + 1];
+        ls.nsrc = 1;
+        ls.has_bias = 0;
+        ls.param_offset = off;
+        off += (int64_t)ls.d_in * ls.d_out;
+        ls.gamma_offset = ls.beta_offset = -1;
+        ls.slope_offset = k < dd->Kd - 1 ? off++ : -1;
+        if (layer) layer[k] = ls;
+    }
+    return off;
+}
 
 // The parameter layout of one replica (also rtma_param_count).
 int64_t layout_model(const rtma_model_desc* md, LayerShape* layer) {
@@ -26,6 +55,7 @@ int64_t layout_model(const rtma_model_desc* md, LayerShape* layer) {
         ls.d_in = md->dims[l];
         ls.d_out = md->dims[l + 1];
         ls.nsrc = nsrc;
+        ls.has_bias = 1;
         ls.param_offset = off;
         off += (int64_t)(nsrc * md->dims[l] + 1) * md->dims[l + 1];
         ls.gamma_offset = ls.beta_offset = ls.slope_offset = -1;
@@ -58,6 +88,7 @@ int32_t parse_model(rtma_ctx* ctx, const rtma_model_desc* md, Model* m) {
     m->P = layout_model(md, m->layer);
     m->gcn = md->encoder == 1;
     m->post = md->L > 1 && (md->act == 1 || md->norm == 1);
+    m->Kd = 0;
     return RTMA_OK;
 }
 
@@ -68,6 +99,7 @@ struct ScratchPlan {
     size_t prep_bytes;        // repacked weights, per part
     int q_width;              // widest Abar^T dZ (widths of the layers above the first)
     size_t post_width;        // widest normalised / PReLU layer output (0: none)
+    size_t per_pair_bytes;    // link prediction: decoder activations per pair
 };
 
 int64_t aligned_rows(int64_t n_p) { return ceil_div(n_p, GROUP_ROW_ALIGN) * GROUP_ROW_ALIGN; }
@@ -91,6 +123,16 @@ ScratchPlan plan_scratch(const Model& m) {
     sp.q_width = q_width;
     if (q_width) per_row += 4 * planes_ld(q_width);     // Abar^T dZ
     sp.per_row_bytes = per_row;
+    // link prediction: per pair e^k and the pre-activations of every decoder layer; per node the
+    // embeddings' gradient in fp32 (the last layer's output planes serve as the embeddings)
+    sp.per_pair_bytes = 0;
+    for (int k = 0; k < m.Kd; ++k) {
+        sp.per_pair_bytes += 4 * planes_ld(m.ddims[k]) + 4 * planes_ld(m.ddims[k + 1]);
+        sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(m.ddims[k] + 1) * m.ddims[k + 1]);
+        sp.prep_bytes += sizeof(__nv_bfloat16) * tc_prep_elems(tc_plan_layer(m.dec[k]), true) + 4 * 256;
+        if (k < m.Kd - 1) sp.post_width = std::max(sp.post_width, (size_t)m.ddims[k + 1]);
+    }
+    if (m.Kd) sp.per_row_bytes += sizeof(float) * planes_ld(m.dims[m.L]);
     return sp;
 }
 
@@ -114,10 +156,13 @@ int plan_splits(const GroupDesc& g, SplitPlan* sp) {
     return slots;
 }
 
-size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p) {
+size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p, int64_t pairs) {
     const size_t rows = (size_t)aligned_rows(n_p);
-    const size_t matrices = 8 * m.L + 12;  // every matrix start is rounded up to 256 bytes
+    const size_t prows = (size_t)aligned_rows(pairs);
+    const size_t matrices = 8 * m.L + 8 * m.Kd + 16;  // every matrix start is rounded up to 256 bytes
     return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, 32) + 256) +
+           sp.per_pair_bytes * prows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(pairs, 32) + 256) +
+           sizeof(float) * ((size_t)ceil_div(pairs, 64) + 1) * (2 * sp.post_width + 1) +
            sizeof(int) * ((size_t)ceil_div(n_p, 8) + 64) +  // processing order of the aggregation kernels
            sizeof(float) * ((size_t)ceil_div(n_p, 64) + 1) * (2 * sp.post_width + 1) +  // per-tile sums of d gamma, d beta, d a
            sp.prep_bytes + 256 * matrices;
@@ -130,15 +175,38 @@ extern "C" int64_t rtma_param_count(const rtma_model_desc* md) {
     return layout_model(md, nullptr);
 }
 
-extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,
-                                        const int64_t* part_offsets, const int64_t* edge_offsets,
-                                        const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
-                                        const float* Xp, const int32_t* yp, float* params, const int32_t* steps,
-                                        int32_t loss_stride, float* loss_out, const rtma_taps* taps,
-                                        void* const* streams) {
+namespace {
+
+// The training loop behind rtma_local_steps, rtma_local_steps_var (link == NULL: softmax
+// cross-entropy on the labels yp) and rtma_link_steps (link != NULL: decoder + binary
+// cross-entropy on the given pairs).
+int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const int64_t* part_offsets,
+                   const int64_t* edge_offsets, const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                   const float* Xp, const int32_t* yp, float* params, const int32_t* steps, int32_t loss_stride,
+                   float* loss_out, const rtma_taps* taps, void* const* streams, const LinkTask* link) {
     if (!ctx) return RTMA_ERR_INVALID_ARG;
     Model m;
     RTMA_TRY(parse_model(ctx, md, &m));
+    if (link) {
+        const rtma_decoder_desc* dd = link->dd;
+        if (!dd || dd->Kd < 1 || dd->Kd > RTMA_MAX_LAYERS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "decoder layers outside [1,%d]", RTMA_MAX_LAYERS);
+        if (dd->ddims[0] != md->dims[md->L] || dd->ddims[dd->Kd] != 1)
+            return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "decoder widths must start at the embedding width %d and end at 1", md->dims[md->L]);
+        for (int k = 0; k <= dd->Kd; ++k) {
+            if (dd->ddims[k] < 1) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "ddims[%d]=%d", k, dd->ddims[k]);
+            m.ddims[k] = dd->ddims[k];
+        }
+        m.Kd = dd->Kd;
+        m.P = layout_decoder(dd, m.P, m.dec);
+        for (int l = 0; l < m.L; ++l) m.layer[l].P = m.P;
+        for (int k = 0; k < m.Kd; ++k) m.dec[k].P = m.P;
+        if (!link->pair_offsets) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_link_steps: null pair offsets");
+        for (int p = 0; p < M && M <= RTMA_MAX_PARTS; ++p)
+            if (link->pair_offsets[p + 1] < link->pair_offsets[p] || link->pair_offsets[p + 1] - link->pair_offsets[p] >= (int64_t(1) << 31))
+                return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "part %d has inconsistent pair offsets", p);
+        if (link->pair_offsets[M <= RTMA_MAX_PARTS && M >= 1 ? M : 0] > 0 && (!link->pu || !link->pv || !link->label))
+            return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_link_steps: null pairs");
+    }
     if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
     if (!part_offsets || !edge_offsets || !rowptr_out || !params || !streams || !steps)
         return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_local_steps: null pointer");
@@ -153,7 +221,7 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
     if (symmetric != 1)
         return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "directed subgraphs are not implemented: pass an undirected graph with both directions stored and symmetric=1");
     const int64_t n = part_offsets[M];
-    if (n > 0 && (!Xp || !yp)) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_local_steps: null features or labels");
+    if (n > 0 && (!Xp || (!yp && !link))) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_local_steps: null features or labels");
     if (edge_offsets[M] > 0 && !col_out) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_local_steps: null col_out");
     for (int p = 0; p < M; ++p)
         if (part_offsets[p + 1] < part_offsets[p] || edge_offsets[p + 1] < edge_offsets[p] ||
@@ -186,7 +254,8 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
     for (size_t gi = 0; gi < G; ++gi) {
         size_t sum = 0;
         for (int p : group_parts[gi]) {
-            const size_t b = part_scratch_bytes(m, plan, part_offsets[p + 1] - part_offsets[p]);
+            const size_t b = part_scratch_bytes(m, plan, part_offsets[p + 1] - part_offsets[p],
+                                                link ? link->pair_offsets[p + 1] - link->pair_offsets[p] : 0);
             sum += b;
             min_share = std::max(min_share, b);
         }
@@ -216,13 +285,15 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
         while (at < parts.size()) {
             // ---- form a wave ----
             GroupDesc g{};
+            GroupDesc gd{};   // link prediction: the same parts' pairs
             SplitPlan sp{};
             size_t bytes = 0;
-            int64_t rows = 0;
+            int64_t rows = 0, prows = 0;
             while (at < parts.size()) {
                 const int p = parts[at];
                 const int64_t n_p = part_offsets[p + 1] - part_offsets[p];
-                const size_t b = part_scratch_bytes(m, plan, n_p);
+                const int64_t pairs_p = link ? link->pair_offsets[p + 1] - link->pair_offsets[p] : 0;
+                const size_t b = part_scratch_bytes(m, plan, n_p, pairs_p);
                 if (g.num > 0 && bytes + b > share) break;
                 const int k = g.num++;
                 g.part[k] = p;
@@ -230,6 +301,13 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 g.row_abs[k] = part_offsets[p];
                 g.row_ws[k] = rows;
                 g.edge_abs[k] = edge_offsets[p];
+                gd.num = g.num;
+                gd.part[k] = p;
+                gd.rows[k] = (int32_t)pairs_p;
+                gd.row_abs[k] = link ? link->pair_offsets[p] : 0;
+                gd.row_ws[k] = prows;
+                gd.edge_abs[k] = 0;
+                prows += aligned_rows(pairs_p);
                 rows += aligned_rows(n_p);
                 bytes += b;
                 ++at;
@@ -261,8 +339,34 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 }
             }
             const int C = m.dims[m.L];
-            Mat logits{cur.take<float>((size_t)rows * planes_ld(C) + 8), (int64_t)planes_ld(C)};
+            // node classification: fp32 logits; link prediction: the embeddings as planes in their place
+            Mat logits{nullptr, (int64_t)planes_ld(C)};
+            Planes R{nullptr, nullptr, 0};
+            if (link) R = take_planes(C);
+            else logits.ptr = cur.take<float>((size_t)rows * planes_ld(C) + 8);
             Planes dZlast = take_planes(C);
+            // ---- link prediction: decoder activations per pair, fp32 gradient of the embeddings ----
+            auto take_pair_planes = [&](int d) {
+                Planes pl;
+                pl.ld = (int64_t)planes_ld(d);
+                pl.hi = cur.take<__nv_bfloat16>((size_t)prows * pl.ld + 8);
+                pl.lo = cur.take<__nv_bfloat16>((size_t)prows * pl.ld + 8);
+                return pl;
+            };
+            Planes El[RTMA_MAX_LAYERS], ZDl[RTMA_MAX_LAYERS];
+            float* dRf = nullptr;
+            float *dec_partial = nullptr, *dec_tile_loss = nullptr, *dec_post_partial = nullptr;
+            SplitPlan spd{};
+            if (link) {
+                dRf = cur.take<float>((size_t)rows * planes_ld(C) + 8);
+                for (int k = 0; k < m.Kd; ++k) {
+                    El[k] = take_pair_planes(m.ddims[k]);
+                    ZDl[k] = take_pair_planes(m.ddims[k + 1]);
+                }
+                const int dslots = plan_splits(gd, &spd);
+                dec_partial = cur.take<float>((size_t)dslots * plan.max_layer_params + 4);
+                dec_tile_loss = cur.take<float>((size_t)loss_tiles(gd) + 4);
+            }
             // Abar^T dZ of the layer in hand; carved at the widest layer, addressed at each layer's own width
             __nv_bfloat16* q_hi = plan.q_width ? cur.take<__nv_bfloat16>((size_t)rows * planes_ld(plan.q_width) + 8) : nullptr;
             __nv_bfloat16* q_lo = plan.q_width ? cur.take<__nv_bfloat16>((size_t)rows * planes_ld(plan.q_width) + 8) : nullptr;
@@ -272,6 +376,18 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
             int* heavy_list = cur.take<int>((size_t)spmm_order_entries(g) + 4);
             float* post_partial = m.post ? cur.take<float>((size_t)post_tiles(g) * (2 * plan.post_width + 1) + 4) : nullptr;
+            if (link && m.Kd > 1) dec_post_partial = cur.take<float>((size_t)post_tiles(gd) * (2 * plan.post_width + 1) + 4);
+            TcLayerPlan dtcp[RTMA_MAX_LAYERS];
+            __nv_bfloat16 *DBf_hi[RTMA_MAX_LAYERS], *DBf_lo[RTMA_MAX_LAYERS], *DBd_hi[RTMA_MAX_LAYERS], *DBd_lo[RTMA_MAX_LAYERS];
+            for (int k = 0; k < m.Kd; ++k) {
+                dtcp[k] = tc_plan_layer(m.dec[k]);
+                const size_t nf = (size_t)g.num * dtcp[k].Npad_f * dtcp[k].Kf;
+                const size_t nd = (size_t)g.num * dtcp[k].Npad_d * dtcp[k].Kd;
+                DBf_hi[k] = cur.take<__nv_bfloat16>(nf);
+                DBf_lo[k] = cur.take<__nv_bfloat16>(nf);
+                DBd_hi[k] = cur.take<__nv_bfloat16>(nd);
+                DBd_lo[k] = cur.take<__nv_bfloat16>(nd);
+            }
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
             __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
             for (int l = 0; l < m.L; ++l) {
@@ -334,6 +450,8 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                 // ---- forward ----
                 for (int l = 0; l < m.L; ++l)
                     RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
+                for (int k = 0; k < m.Kd; ++k)
+                    RTMA_TRY(launch_tc_weight_prep(ctx, g, m.dec[k], dtcp[k], params, DBf_hi[k], DBf_lo[k], DBd_hi[k], DBd_lo[k], s));
                 for (int l = 0; l < m.L; ++l) {
                     if (l == 0) {
                         // the aggregate of the input features does not change from step to step
@@ -345,14 +463,15 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                     const bool last = l == m.L - 1;
                     if (last || !m.post) {
                         RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
-                                                   last ? no_planes : Hl[l + 1], last ? logits : no_mat, !last, single_pass, s));
+                                                   last ? (link ? R : no_planes) : Hl[l + 1], (last && !link) ? logits : no_mat, !last,
+                                                   single_pass, s));
                     } else {  // pre-activations kept; normalisation and PReLU in a pass of their own
                         RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
                                                    Zl[l], no_mat, false, single_pass, s));
                         RTMA_TRY(launch_post_forward(ctx, g, m.layer[l], params, Zl[l], Hl[l + 1], stats[l], s));
                     }
                 }
-                if (tap && taps->acts) {
+                if (tap && taps->acts && !link) {
                     size_t rec = 0;  // floats per row in the record
                     for (int l = 0; l < m.L; ++l) rec += (size_t)m.dims[l] + m.dims[l + 1];
                     for (int k = 0; k < g.num; ++k) {
@@ -369,8 +488,39 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                         }
                     }
                 }
-                // ---- loss; dZ of the last layer and its tile column sums ----
-                RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, loss_stride, step, s));
+                // ---- loss; dZ of the last layer ----
+                if (!link) {
+                    RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, loss_stride, step, s));
+                } else {
+                    float* grads_rec = tap ? taps->grads : nullptr;
+                    if (tap && link->emb_out)
+                        for (int k = 0; k < g.num; ++k)
+                            RTMA_TRY(launch_from_planes(ctx, R, g.row_ws[k], g.rows[k], C, link->emb_out + (size_t)g.row_abs[k] * C, s));
+                    // decoder forward: e^0 = r_u (.) r_v; e^{k+1} = PReLU(e^k Theta^k); the last layer gives the score
+                    RTMA_TRY(launch_pair_product(ctx, gd, g, R, link->pu, link->pv, El[0], C, s));
+                    for (int k = 0; k < m.Kd && prows > 0; ++k) {
+                        RTMA_TRY(launch_tc_forward(ctx, gd, m.dec[k], dtcp[k], prows, params, El[k], El[k], DBf_hi[k], DBf_lo[k],
+                                                   ZDl[k], no_mat, false, single_pass, s));
+                        if (k < m.Kd - 1) RTMA_TRY(launch_post_forward(ctx, gd, m.dec[k], params, ZDl[k], El[k + 1], nullptr, s));
+                    }
+                    // binary cross-entropy: the scores become d loss / d score in place
+                    RTMA_TRY(launch_bce(ctx, gd, ZDl[m.Kd - 1], link->label, dec_tile_loss, tap ? link->score_out : nullptr, s));
+                    RTMA_TRY(launch_loss_finalize(ctx, gd, dec_tile_loss, loss_out, loss_stride, step, s));
+                    // decoder backward + SGD
+                    for (int k = m.Kd - 1; k >= 0 && prows > 0; --k) {
+                        RTMA_TRY(launch_tc_wgrad(ctx, gd, spd, m.dec[k], prows, El[k], El[k], ZDl[k], dec_partial, single_pass, s));
+                        // d e^k = d Z^k Theta^k^T, written over e^k
+                        RTMA_TRY(launch_tc_dgrad(ctx, gd, m.dec[k], dtcp[k], prows, ZDl[k], ZDl[k], DBd_hi[k], DBd_lo[k], El[k], false,
+                                                 single_pass, s));
+                        RTMA_TRY(launch_reduce_sgd(ctx, gd, spd, m.dec[k], dec_partial, m.lr, params, grads_rec, s));
+                        if (k > 0)
+                            RTMA_TRY(launch_post_backward(ctx, gd, m.dec[k - 1], params, ZDl[k - 1], El[k], nullptr, dec_post_partial,
+                                                          m.lr, grads_rec, s));
+                    }
+                    // into the embeddings: d r_u += d e^0 (.) r_v, d r_v += d e^0 (.) r_u
+                    RTMA_CUDA(ctx, cudaMemsetAsync(dRf, 0, sizeof(float) * (size_t)rows * planes_ld(C), s));
+                    RTMA_TRY(launch_pair_scatter(ctx, gd, g, R, link->pu, link->pv, El[0], dRf, (int64_t)planes_ld(C), C, dZlast, s));
+                }
                 // ---- backward + SGD ----
                 for (int l = m.L - 1; l >= 0; --l) {
                     // dZ^l: from the loss, over H^{l+1} (fused ReLU gate) or over Z^l (separate activation pass)
@@ -394,6 +544,40 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
         }
     }
     return RTMA_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,
+                                        const int64_t* part_offsets, const int64_t* edge_offsets,
+                                        const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                                        const float* Xp, const int32_t* yp, float* params, const int32_t* steps,
+                                        int32_t loss_stride, float* loss_out, const rtma_taps* taps,
+                                        void* const* streams) {
+    return train_impl(ctx, md, M, part_offsets, edge_offsets, rowptr_out, col_out, symmetric, Xp, yp, params, steps,
+                      loss_stride, loss_out, taps, streams, nullptr);
+}
+
+extern "C" int64_t rtma_link_param_count(const rtma_model_desc* md, const rtma_decoder_desc* dd) {
+    if (!md || md->L < 1 || md->L > RTMA_MAX_LAYERS || !dd || dd->Kd < 1 || dd->Kd > RTMA_MAX_LAYERS) return -1;
+    return layout_decoder(dd, layout_model(md, nullptr), nullptr);
+}
+
+extern "C" int32_t rtma_link_steps(rtma_ctx* ctx, const rtma_model_desc* md, const rtma_decoder_desc* dd, int32_t M,
+                                   const int64_t* part_offsets, const int64_t* edge_offsets, const int64_t* rowptr_out,
+                                   const int32_t* col_out, int32_t symmetric, const float* Xp, const int64_t* pair_offsets,
+                                   const int32_t* pair_u, const int32_t* pair_v, const int32_t* pair_label, float* params,
+                                   int32_t K, float* loss_out, int32_t record_step, float* grads_out, float* emb_out,
+                                   float* score_out, void* const* streams) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    if (K < 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "K=%d negative", K);
+    if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
+    int32_t steps[RTMA_MAX_PARTS];
+    for (int p = 0; p < M; ++p) steps[p] = K;
+    const LinkTask link{dd, pair_offsets, pair_u, pair_v, pair_label, emb_out, score_out};
+    const rtma_taps taps{nullptr, grads_out, record_step};
+    return train_impl(ctx, md, M, part_offsets, edge_offsets, rowptr_out, col_out, symmetric, Xp, nullptr, params, steps, K,
+                      loss_out, record_step >= 0 ? &taps : nullptr, streams, &link);
 }
 
 extern "C" int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,

@@ -53,7 +53,8 @@ inline size_t padded_ld(int64_t d) { return (size_t)((d + 3) / 4 * 4); }
 
 struct LayerShape {
     int32_t d_in, d_out;
-    int32_t nsrc;          // weight matrices of the layer: 2 = GraphSAGE-mean (Ws, Wn), 1 = GCN (W)
+    int32_t nsrc;          // weight matrices of the layer: 2 = GraphSAGE-mean (Ws, Wn), 1 = GCN (W), decoder
+    int32_t has_bias;      // 0: the bias row is absent from the parameters (decoder layers)
     int64_t param_offset;  // of the first weight matrix inside one replica; the weight matrices and b are
                            // contiguous: an (nsrc d_in + 1) x d_out matrix
     int64_t gamma_offset, beta_offset;  // Layer Normalization scale / shift [d_out]; -1 = none
@@ -110,6 +111,9 @@ int32_t launch_spmm_gcn(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr
 // written as split planes and the part's loss to loss_out[part * loss_stride + loss_col] when
 // loss_out != NULL.  tile_loss: loss_tiles(g) floats of scratch.
 int64_t loss_tiles(const GroupDesc& g);
+// loss_out[part * loss_stride + loss_col] = (sum of the part's tile sums) / rows of the part
+int32_t launch_loss_finalize(rtma_ctx* ctx, const GroupDesc& g, const float* tile_loss, float* loss_out,
+                             int64_t loss_stride, int64_t loss_col, cudaStream_t s);
 int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp, Planes dZ,
                             float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s);
 
@@ -122,6 +126,17 @@ int32_t launch_post_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, co
 // gamma, beta and the slope take their SGD step.  partial: post_tiles(g) * (2 d_out + 1) floats.
 int32_t launch_post_backward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, float* params, Planes Z, Planes dH,
                              float2* stats, float* partial, float lr, float* grads_record, cudaStream_t s);
+
+// ---- link.cu (link prediction on given pairs; gd addresses the pairs, g the nodes, slot by slot) ----
+// E[pair] = R[u] (.) R[v]
+int32_t launch_pair_product(rtma_ctx* ctx, const GroupDesc& gd, const GroupDesc& g, Planes R, const int32_t* pu,
+                            const int32_t* pv, Planes E, int d, cudaStream_t s);
+// dR (fp32 [scratch row][ld], zero on entry) += dE (.) R of the partner, then dR_planes = planes(dR)
+int32_t launch_pair_scatter(rtma_ctx* ctx, const GroupDesc& gd, const GroupDesc& g, Planes R, const int32_t* pu,
+                            const int32_t* pv, Planes dE, float* dR, int64_t ld, int d, Planes dR_planes, cudaStream_t s);
+// S (planes of width 1): scores in, d loss / d score out; tile_loss: loss_tiles(gd) floats
+int32_t launch_bce(rtma_ctx* ctx, const GroupDesc& gd, Planes S, const int32_t* label, float* tile_loss,
+                   float* score_out, cudaStream_t s);
 
 // ---- optim.cu -------------------------------------------------------------------------
 // grad = sum of the part's chunk slots; params -= lr * grad; optionally records grad.

@@ -69,3 +69,14 @@ def test_variant_flags_are_validated(util, tiny_workload):
     with pytest.raises(Exception):
         util.ctx().local_steps(w.dims, w.lr, w.M, got["part_host"], got["edge_host"], got["rowptr_out"],
                                got["col_out"], got["Xp"], got["yp"], params, 1, variant=(2, 0, 0))
+
+
+@pytest.mark.parametrize("variant", [(1, 1, 0), (1, 1, 1)])
+def test_variants_with_more_trainers_than_busy_parts(util, variant):
+    # 40 nodes over 16 trainers: empty parts, parts of one or two nodes, most nodes isolated
+    w = inputs.tiny()
+    g = inputs.uniform_graph(40, 100, 3)
+    w.graph, w.X, w.y = g, w.X[:40].copy(), w.y[:40].copy()
+    p0 = _start(variant, w.dims, 17)
+    got, want = util.check_one_step(w, M=16, variant=variant, params0=p0)
+    util.check_k_steps_and_average(w, got, want, 2, variant=variant, params0=p0)

@@ -99,3 +99,24 @@ def test_loss_identities():
     # an empty batch and an empty part cost nothing
     e = np.empty(0, dtype=np.int32)
     assert oracle.link_forward_backward(variant, dims, ddims, rp, cp, X, e, e, e, p)[0] == 0.0
+
+
+def test_branch_override_reproduces_the_natural_branches_and_moves_only_chosen_units():
+    rp, cp, X, pu, pv, label = _case(13)
+    variant, dims, ddims = (1, 1, 1), (6, 5, 4), (4, 3, 1)
+    p = oracle.link_init_params(variant, dims, ddims, 14)
+    n, B = rp.size - 1, pu.size
+    pre = np.zeros(oracle.link_gate_count(dims, ddims, n, B))
+    assert pre.size == n * 5 + B * 3
+    base = oracle.link_forward_backward(variant, dims, ddims, rp, cp, X, pu, pv, label, p, preact_out=pre)
+    natural = (pre > 0).astype(np.int8)
+    same = oracle.link_forward_backward(variant, dims, ddims, rp, cp, X, pu, pv, label, p, gates=natural)
+    assert same[0] == base[0] and np.array_equal(same[1], base[1])
+    free = oracle.link_forward_backward(variant, dims, ddims, rp, cp, X, pu, pv, label, p, gates=np.full(pre.size, -1, np.int8))
+    assert free[0] == base[0] and np.array_equal(free[1], base[1])
+    # flipping the unit closest to its kink changes the loss by O(|input|) only
+    i = int(np.argmin(np.abs(pre)))
+    g = natural.copy()
+    g[i] ^= 1
+    moved = oracle.link_forward_backward(variant, dims, ddims, rp, cp, X, pu, pv, label, p, gates=g)
+    assert moved[0] != base[0] and abs(moved[0] - base[0]) <= 2.0 * abs(pre[i])
