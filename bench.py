@@ -262,6 +262,139 @@ def run_averaging_stress(args, local_rank):
         "gpu_launches": args.steps, "clocks": clocks}))
 
 
+def run_link(args, rank, local_rank, world):
+    """`--task link`: the paper's own task on the workload's graph and features.  One step = the
+    whole path (partition, induced CSR, row gather, R x (K link-prediction steps on all M parts +
+    aggregation)).  Encoder: the workload's widths with the last layer as wide as the hidden ones
+    (--encoder / --act / --norm pick the variant); decoder: two layers of that width; pairs: up to
+    65,536 edges of each part as positives plus one random-tail negative each, drawn once."""
+    import torch
+    import torch.distributed as dist
+    from paper_2305_09887_b200 import binding, inputs
+
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    args.warmup = max(args.warmup, 3)
+    w = make_workload(args)
+    g = w.graph
+    hid = w.dims[1]
+    dims, ddims = tuple(w.dims[:-1]) + (hid,), (hid, hid, 1)
+    L = len(dims) - 1
+    params0 = inputs.link_params(w.variant, dims, ddims, inputs.SEED_WEIGHT + 9)
+    P = params0.size
+    ctx = binding.Context(local_rank)
+    assert P == binding.link_param_count(dims, ddims, w.variant)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    host = dict(rowptr=pin(g.rowptr), col=pin(g.col), X=pin(w.X), p0=pin(params0),
+                gid=pin(g.group_id) if w.use_groups else None)
+    res = {k: (v.to(device) if v is not None else None) for k, v in host.items()}
+
+    def preprocess():
+        part_id, part_offsets, perm, local_id = ctx.partition(g.n, res["gid"], w.partition_seed, w.M)
+        rowptr_out, col_out, edge_offsets, kept_cut, edge_host = ctx.build_induced_csr(
+            res["rowptr"], res["col"], w.M, part_id, part_offsets, perm, local_id)
+        Xp = ctx.gather_rows(res["X"], perm)
+        return part_offsets, rowptr_out, col_out, edge_offsets, edge_host, Xp
+
+    # the training pairs are inputs: drawn once from the parts' subgraphs, outside the timed region
+    part_offsets, rowptr_out, col_out, edge_offsets, edge_host, _ = preprocess()
+    pu, pv, lab, pair_off = inputs.link_pairs(rowptr_out.cpu().numpy(), col_out.cpu().numpy(), part_offsets.cpu().numpy(),
+                                              np.asarray(edge_host), w.M, 77, 65536)
+    host.update(pu=pin(pu), pv=pin(pv), lab=pin(lab))
+    res.update(pu=host["pu"].to(device), pv=host["pv"].to(device), lab=host["lab"].to(device))
+    params = torch.empty(w.M, P, dtype=torch.float32, device=device)
+    loss = torch.zeros(w.R, w.M, w.K, dtype=torch.float32, device=device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    state = {}
+
+    def step():
+        params.copy_(res["p0"].expand(w.M, P))
+        part_offsets, rowptr_out, col_out, edge_offsets, edge_host, Xp = preprocess()
+        part_host = part_offsets.cpu().tolist()
+        for r in range(w.R):
+            ctx.link_steps(dims, ddims, w.lr, w.M, part_host, edge_host, rowptr_out, col_out, Xp, pair_off,
+                           res["pu"], res["pv"], res["lab"], params, w.K, loss_out=loss[r], gemm_dtype=w.gemm_dtype,
+                           variant=w.variant)
+            ctx.aggregate(params)
+        state.update(edge_host=edge_host)
+
+    def timed(fn, n):
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        for i in range(n):
+            flush.fill_(i & 0xFF)
+            starts[i].record()
+            fn()
+            stops[i].record()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        return max_over_ranks(sum(a.elapsed_time(b) for a, b in zip(starts, stops)) / 1e3, dist if world > 1 else None, device)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    ctx.profile_read()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ctx.profile(True)
+    elapsed_s = timed(step, args.steps)
+    ctx.profile(False)
+    prof = ctx.profile_read()
+    clocks = sampler.stop()
+
+    def host_step():   # inputs from pinned host memory every step, result read back
+        for k in ("rowptr", "col", "X", "p0", "gid", "pu", "pv", "lab"):
+            if host[k] is not None:
+                res[k].copy_(host[k], non_blocking=True)
+        step()
+        state["out"] = (params[0].cpu(), loss.cpu())
+
+    e2e_steps = max(1, min(args.steps, 3))
+    host_step()
+    e2e_s = timed(host_step, e2e_steps)
+    h2d = sum(v.numel() * v.element_size() for v in host.values() if v is not None)
+    d2h = P * 4 + loss.numel() * 4 + 2 * 8 * (w.M + 1)
+
+    kept = float(state["edge_host"][-1])
+    passes = 2 * L - 1
+    units = kept * passes * w.K * w.R
+    total_ms = sum(ms for ms, _ in prof.values())
+    top = max(prof, key=lambda k: prof[k][0])
+    peaks = load_peaks()
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": world * args.steps * units / elapsed_s, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * elapsed_s / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16x3-split products, f32 accumulate and elementwise", "data": "synthetic",
+            "config": {"workload": w.name + "_link", "task": "link prediction", "nodes": g.n, "entries": g.num_entries,
+                       "kept_entries": int(kept), "M": w.M, "dims": list(dims), "decoder": list(ddims), "K": w.K, "R": w.R,
+                       "pairs": int(pair_off[-1]), "variant": {"encoder": args.encoder, "act": args.act, "norm": args.norm},
+                       "parallelism": "replicas only" if world > 1 else f"single GPU, {w.M} trainers batched on one stream",
+                       "l2": "256 MB written between timed steps"},
+            "trainer_steps_per_s": world * args.steps * w.M * w.K * w.R / elapsed_s,
+            "pairs_per_s": world * args.steps * pair_off[-1] * w.K * w.R / elapsed_s,
+            "loss_first_last": [loss[0, :, 0].mean().item(), loss[-1, :, -1].mean().item()],
+            "roofline": {"bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": None,
+                         "traffic": None, "kernel": top, "share_of_kernel_time": prof[top][0] / total_ms,
+                         "peak_source": peaks["source"]},
+            "kernels": {k: {"ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps, "share": ms / total_ms}
+                        for k, (ms, cnt) in prof.items() if cnt},
+            "gpu_launches": int(sum(cnt for _, cnt in prof.values())), "clocks": clocks,
+            "e2e": {"value": world * e2e_steps * units / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                    "d2h_bytes_per_step": int(d2h), "ms_per_step": 1e3 * e2e_s / e2e_steps, "steps": e2e_steps},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def max_over_ranks(seconds: float, dist_mod=None, device=None) -> float:
     """Largest value over all ranks (the slowest rank sets the job's time)."""
     if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
@@ -283,6 +416,8 @@ def main():
     ap.add_argument("--scale", type=float, default=None, help="shrink (or grow) the workload's graph")
     ap.add_argument("--M", type=int, default=None, help="trainers (supertma / sweep)")
     ap.add_argument("--assign", default="super", choices=["node", "super"], help="sweep: assignment scheme")
+    ap.add_argument("--task", default="node", choices=["node", "link"],
+                    help="node classification (the named workloads) or link prediction (the paper's task)")
     ap.add_argument("--encoder", default="sage", choices=["sage", "gcn"])
     ap.add_argument("--act", default="relu", choices=["relu", "prelu"])
     ap.add_argument("--norm", default="none", choices=["none", "layernorm"])
@@ -301,6 +436,9 @@ def main():
     if args.workload == "averaging":
         if rank == 0:
             run_averaging_stress(args, local_rank)
+        return
+    if args.task == "link":
+        run_link(args, rank, local_rank, world)
         return
 
     import torch

@@ -57,13 +57,13 @@ pair_scatter_kernel(const __grid_constant__ GroupDesc gd, const __grid_constant_
         load_pack(R, ru, col, a);
         load_pack(R, rv, col, b);
         load_pack(dE, src, col, ge);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            if (col + e < d) {
-                atomicAdd(dR + ru * ld + col + e, ge.v[e] * b.v[e]);
-                atomicAdd(dR + rv * ld + col + e, ge.v[e] * a.v[e]);
-            }
-        }
+        // 16-byte vector atomics; the planes' padding columns hold zeros, so whole pieces can be added
+        float4* du = reinterpret_cast<float4*>(dR + ru * ld + col);
+        float4* dv = reinterpret_cast<float4*>(dR + rv * ld + col);
+        atomicAdd(du, make_float4(ge.v[0] * b.v[0], ge.v[1] * b.v[1], ge.v[2] * b.v[2], ge.v[3] * b.v[3]));
+        atomicAdd(du + 1, make_float4(ge.v[4] * b.v[4], ge.v[5] * b.v[5], ge.v[6] * b.v[6], ge.v[7] * b.v[7]));
+        atomicAdd(dv, make_float4(ge.v[0] * a.v[0], ge.v[1] * a.v[1], ge.v[2] * a.v[2], ge.v[3] * a.v[3]));
+        atomicAdd(dv + 1, make_float4(ge.v[4] * a.v[4], ge.v[5] * a.v[5], ge.v[6] * a.v[6], ge.v[7] * a.v[7]));
     }
 }
 

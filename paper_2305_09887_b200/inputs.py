@@ -266,6 +266,51 @@ def variant_params(variant, dims, seed: int) -> np.ndarray:
     return np.concatenate(out)
 
 
+def link_param_count(variant, dims, ddims) -> int:
+    """Encoder variant + MLP decoder (Theta^k [ddims[k]][ddims[k+1]], one PReLU slope per hidden layer)."""
+    dec = sum(ddims[k] * ddims[k + 1] for k in range(len(ddims) - 1)) + (len(ddims) - 2)
+    return variant_param_count(variant, dims) + dec
+
+
+def link_params(variant, dims, ddims, seed: int) -> np.ndarray:
+    """Initial parameters for link prediction in the library's order: the encoder's
+    (variant_params), then per decoder layer Xavier-uniform Theta^k and (hidden layers) slope 0.25."""
+    rng = np.random.default_rng(seed + 1)
+    out = [variant_params(variant, dims, seed)]
+    for k in range(len(ddims) - 1):
+        a = math.sqrt(6.0 / (ddims[k] + ddims[k + 1]))
+        out.append(rng.uniform(-a, a, size=ddims[k] * ddims[k + 1]).astype(np.float32))
+        if k < len(ddims) - 2:
+            out.append(np.full(1, 0.25, dtype=np.float32))
+    return np.concatenate(out)
+
+
+def link_pairs(rowptr_out, col_out, part_offsets, edge_offsets, M: int, seed: int, max_positives: int):
+    """Training pairs per part from its induced subgraph (local ids): up to max_positives of the
+    part's undirected edges (entries with row < col) as positives, and for each positive (u, v)
+    one negative (u, v') with a uniformly drawn tail.  Returns (pair_u, pair_v, label, offsets[M+1])."""
+    rng = np.random.default_rng(seed)
+    pu, pv, lab, off = [], [], [], [0]
+    for p in range(M):
+        n_p = int(part_offsets[p + 1] - part_offsets[p])
+        base = int(part_offsets[p]) + p
+        rp = np.asarray(rowptr_out[base:base + n_p + 1])
+        cp = np.asarray(col_out[int(edge_offsets[p]):int(edge_offsets[p + 1])])
+        rows = np.repeat(np.arange(n_p, dtype=np.int32), np.diff(rp))
+        keep = np.flatnonzero(rows < cp)
+        if keep.size > max_positives:
+            keep = np.sort(rng.choice(keep, size=max_positives, replace=False))
+        k = keep.size
+        if k:
+            neg = rng.integers(0, n_p, size=k).astype(np.int32)
+            pu += [rows[keep], rows[keep]]
+            pv += [cp[keep].astype(np.int32), neg]
+            lab += [np.ones(k, np.int32), np.zeros(k, np.int32)]
+        off.append(off[-1] + 2 * k)
+    cat = lambda xs: np.concatenate(xs).astype(np.int32) if xs else np.empty(0, np.int32)
+    return cat(pu), cat(pv), cat(lab), off
+
+
 SEED_GRAPH, SEED_FEAT, SEED_LABEL, SEED_WEIGHT, SEED_PART = (
     0x5EED0001, 0x5EED0002, 0x5EED0003, 0x5EED0004, 0x5EED0005)
 
