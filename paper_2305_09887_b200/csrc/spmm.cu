@@ -133,6 +133,8 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     const int64_t my_off = (nrows > 0 && lane <= nrows) ? rp[i0 + lane] : 0;
     const int64_t e_begin = __shfl_sync(0xffffffffu, my_off, 0);
     const int64_t e_end = __shfl_sync(0xffffffffu, my_off, nrows);
+    // the rows' own weights, one coalesced load instead of a dependent load per finished row
+    const float my_w = (MODE != 1 && lane < nrows) ? inv_deg[ws + i0 + lane] : 1.f;
     if (!listed && order.heavy_count && e_end - e_begin >= order.heavy) continue;  // done as a listed group
 
     Pack8 acc[NCH];
@@ -144,7 +146,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     // finishes row `row`: scale, store, clear
     auto flush = [&](int row) {
         const int64_t r = ws + i0 + row;
-        const float w = MODE == 1 ? 1.f : inv_deg[r];
+        const float w = MODE == 1 ? 1.f : __shfl_sync(0xffffffffu, my_w, row);
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
             const int colx = (c * 32 + lane) * 8;
