@@ -181,7 +181,8 @@ typedef struct {
  *   streams  HOST array of M cudaStream_t: trainer i runs on streams[i].  Trainers that
  *            share a stream are batched into common launches; distinct streams run
  *            concurrently.  The call returns once everything is enqueued.
- * Scratch is taken from the context (grows if needed).                                    */
+ * Scratch is taken from the context (grows if needed).  A part may hold at most 2^31 - 1
+ * nodes (RTMA_ERR_INVALID_ARG) and 2^31 - 1 kept entries (RTMA_ERR_OVERFLOW).               */
 int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* model, int32_t M,
                          const int64_t* part_offsets_host, const int64_t* edge_offsets_host,
                          const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,

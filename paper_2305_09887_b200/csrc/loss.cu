@@ -2,8 +2,10 @@
 // gradient (softmax - onehot) / n_p is written as split bf16 planes (it feeds the tensor-core
 // products of the backward pass).
 //
-// One warp per row.  With up to 128 classes a lane keeps its (at most four) logits in registers,
-// so the row is read once; wider rows are swept three times (max, sum of exponentials, gradient).
+// One warp per row, eight rows per warp.  With up to 128 classes a lane keeps its (at most four,
+// consecutive) logits in registers, so a row is read once, with one vector load, and its gradient
+// leaves with one vector store per plane; wider rows are swept three times (max, sum of
+// exponentials, gradient).
 // Loss sums are reduced in a fixed order (warp -> block -> part): results do not change from
 // run to run.
 #include "train.cuh"
@@ -15,11 +17,110 @@ constexpr int LOSS_TILE_ROWS = 64;
 constexpr int LOSS_ROWS_PER_WARP = LOSS_TILE_ROWS / (LOSS_THREADS / 32);
 constexpr int LOSS_REG_CLASSES = 128;
 
-// J = logits a lane keeps in registers (C <= 32 J <= 128), 0 = sweep the row instead
+// J = consecutive logits a lane keeps in registers (C <= 32 J <= 128).  The warp's rows are
+// independent: their loads are issued together and their reductions interleave.
 template <int J>
 __global__ void __launch_bounds__(LOSS_THREADS)
 softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
                     const Planes dZ, float* __restrict__ tile_loss) {
+    __shared__ float warp_loss[LOSS_THREADS / 32];
+    int k, r0;
+    if (!locate_tile(g, LOSS_TILE_ROWS, blockIdx.x, &k, &r0)) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_p = g.rows[k];
+    const float inv_n = 1.0f / (float)n_p;
+    constexpr int R = LOSS_ROWS_PER_WARP;
+    const int i0 = r0 + warp * R;
+    const int c0 = lane * J;
+    float v[R][J];
+    int label[R];
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+        const bool row_ok = i0 + q < n_p;
+        const float* z = logits.ptr + (g.row_ws[k] + i0 + q) * logits.ld;
+        label[q] = row_ok ? yp[g.row_abs[k] + i0 + q] : 0;
+        if (J == 1) {
+            v[q][0] = (row_ok && c0 < C) ? z[c0] : 0.f;
+        } else if (J == 2) {
+            const float2 t = (row_ok && c0 < logits.ld) ? *reinterpret_cast<const float2*>(z + c0) : make_float2(0.f, 0.f);
+            v[q][0] = t.x; v[q][J > 1 ? 1 : 0] = t.y;
+        } else {
+            const float4 t = (row_ok && c0 < logits.ld) ? *reinterpret_cast<const float4*>(z + c0) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[q][0] = t.x; v[q][J > 1 ? 1 : 0] = t.y; v[q][J > 2 ? 2 : 0] = t.z; v[q][J > 3 ? 3 : 0] = t.w;
+        }
+    }
+    float zmax[R], sum[R];
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+        zmax[q] = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            if (c0 + j >= C) v[q][j] = -INFINITY;
+            zmax[q] = fmaxf(zmax[q], v[q][j]);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int q = 0; q < R; ++q) zmax[q] = fmaxf(zmax[q], __shfl_xor_sync(0xffffffffu, zmax[q], o));
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+        sum[q] = 0.f;
+#pragma unroll
+        for (int j = 0; j < J; ++j) sum[q] += c0 + j < C ? expf(v[q][j] - zmax[q]) : 0.f;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int q = 0; q < R; ++q) sum[q] += __shfl_xor_sync(0xffffffffu, sum[q], o);
+    float loss = 0.f;
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+        const bool row_ok = i0 + q < n_p;  // warp-uniform
+        const float lse = zmax[q] + logf(sum[q]);
+        float zl = 0.f;  // the label's logit, from the lane that holds it
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const float cand = __shfl_sync(0xffffffffu, v[q][j], label[q] / J);
+            if (label[q] % J == j) zl = cand;
+        }
+        if (row_ok && lane == 0) loss += lse - zl;  // rows in order: the sum does not depend on timing
+        uint32_t hb[J], lb[J];
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const int c = c0 + j;
+            hb[j] = lb[j] = 0u;  // padding columns of the planes stay zero
+            if (c < C) split_bits((expf(v[q][j] - lse) - (c == label[q] ? 1.f : 0.f)) * inv_n, hb[j], lb[j]);
+        }
+        if (row_ok && c0 < dZ.ld) {
+            const int64_t at = (g.row_ws[k] + i0 + q) * dZ.ld + c0;
+            __nv_bfloat16* ph = dZ.hi + at;
+            __nv_bfloat16* pl = dZ.lo + at;
+            if (J == 1) {
+                *ph = __ushort_as_bfloat16((unsigned short)hb[0]);
+                *pl = __ushort_as_bfloat16((unsigned short)lb[0]);
+            } else if (J == 2) {
+                *reinterpret_cast<uint32_t*>(ph) = hb[0] | (hb[J > 1 ? 1 : 0] << 16);
+                *reinterpret_cast<uint32_t*>(pl) = lb[0] | (lb[J > 1 ? 1 : 0] << 16);
+            } else {
+                *reinterpret_cast<uint2*>(ph) = make_uint2(hb[0] | (hb[J > 1 ? 1 : 0] << 16), hb[J > 2 ? 2 : 0] | (hb[J > 3 ? 3 : 0] << 16));
+                *reinterpret_cast<uint2*>(pl) = make_uint2(lb[0] | (lb[J > 1 ? 1 : 0] << 16), lb[J > 2 ? 2 : 0] | (lb[J > 3 ? 3 : 0] << 16));
+            }
+        }
+    }
+    if (lane == 0) warp_loss[warp] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int w = 0; w < LOSS_THREADS / 32; ++w) s += warp_loss[w];
+        tile_loss[blockIdx.x] = s;
+    }
+}
+
+// More than 128 classes: the row is swept three times (max, sum of exponentials, gradient).
+__global__ void __launch_bounds__(LOSS_THREADS)
+softmax_xent_wide_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
+                         const Planes dZ, float* __restrict__ tile_loss) {
     __shared__ float warp_loss[LOSS_THREADS / 32];
     int k, r0;
     if (!locate_tile(g, LOSS_TILE_ROWS, blockIdx.x, &k, &r0)) return;
@@ -33,52 +134,21 @@ softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const
         const int64_t r = g.row_ws[k] + i;
         const float* z = logits.ptr + r * logits.ld;
         const int label = yp[g.row_abs[k] + i];
-        if (J > 0) {
-            float v[J > 0 ? J : 1];
-            float zmax = -INFINITY;
+        float zmax = -INFINITY;
+        for (int c = lane; c < C; c += 32) zmax = fmaxf(zmax, z[c]);
 #pragma unroll
-            for (int j = 0; j < J; ++j) {
-                const int c = lane + 32 * j;
-                v[j] = c < C ? z[c] : -INFINITY;
-                zmax = fmaxf(zmax, v[j]);
-            }
+        for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+        float sum = 0.f;
+        for (int c = lane; c < C; c += 32) sum += expf(z[c] - zmax);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
-            float sum = 0.f;
-#pragma unroll
-            for (int j = 0; j < J; ++j) sum += lane + 32 * j < C ? expf(v[j] - zmax) : 0.f;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            const float lse = zmax + logf(sum);
-            const float zl = __shfl_sync(0xffffffffu, v[label >> 5], label & 31);
-            if (lane == 0) loss += lse - zl;
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                const int c = lane + 32 * j;
-                if (c < C) {
-                    __nv_bfloat16 h, l;
-                    split_bf16((expf(v[j] - lse) - (c == label ? 1.f : 0.f)) * inv_n, h, l);
-                    dZ.hi[r * dZ.ld + c] = h;
-                    dZ.lo[r * dZ.ld + c] = l;
-                }
-            }
-        } else {
-            float zmax = -INFINITY;
-            for (int c = lane; c < C; c += 32) zmax = fmaxf(zmax, z[c]);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
-            float sum = 0.f;
-            for (int c = lane; c < C; c += 32) sum += expf(z[c] - zmax);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            const float lse = zmax + logf(sum);
-            if (lane == 0) loss += lse - z[label];
-            for (int c = lane; c < C; c += 32) {
-                __nv_bfloat16 h, l;
-                split_bf16((expf(z[c] - lse) - (c == label ? 1.f : 0.f)) * inv_n, h, l);
-                dZ.hi[r * dZ.ld + c] = h;
-                dZ.lo[r * dZ.ld + c] = l;
-            }
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float lse = zmax + logf(sum);
+        if (lane == 0) loss += lse - z[label];
+        for (int c = lane; c < C; c += 32) {
+            __nv_bfloat16 h, l;
+            split_bf16((expf(z[c] - lse) - (c == label ? 1.f : 0.f)) * inv_n, h, l);
+            dZ.hi[r * dZ.ld + c] = h;
+            dZ.lo[r * dZ.ld + c] = l;
         }
     }
     if (lane == 0) warp_loss[warp] = loss;
@@ -122,7 +192,7 @@ int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C
         if (C <= 32) softmax_xent_kernel<1><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         else if (C <= 64) softmax_xent_kernel<2><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         else if (C <= LOSS_REG_CLASSES) softmax_xent_kernel<4><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
-        else softmax_xent_kernel<0><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        else softmax_xent_wide_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         RTMA_LAUNCH_CHECK(ctx);
     }
     return launch_loss_finalize(ctx, g, tile_loss, loss_out, loss_stride, loss_col, s);

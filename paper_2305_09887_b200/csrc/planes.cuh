@@ -106,6 +106,22 @@ struct Pack8 {
         h = make_uint4(hw[0], hw[1], hw[2], hw[3]);
         l = make_uint4(lw[0], lw[1], lw[2], lw[3]);
     }
+    // The split with the remainder x - hi formed by a mixed-precision add of -hi (the sign bits
+    // flipped in the packed word), so that hi is never unpacked; bit for bit the split below.
+    __device__ __forceinline__ void to_planes_lean(uint4& h, uint4& l) const {
+        uint32_t hw[4], lw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 hh = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+            hw[i] = *reinterpret_cast<const uint32_t*>(&hh);
+            const uint32_t neg = hw[i] ^ 0x80008000u;
+            const __nv_bfloat162 ll = __floats2bfloat162_rn(add_f32_bf16(v[2 * i], (unsigned short)(neg & 0xFFFFu)),
+                                                            add_f32_bf16(v[2 * i + 1], (unsigned short)(neg >> 16)));
+            lw[i] = *reinterpret_cast<const uint32_t*>(&ll);
+        }
+        h = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        l = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+    }
     // The same split (bit for bit, for finite inputs) through the paired conversion instruction:
     // far fewer instructions, for kernels whose special-function pipe is otherwise idle.
     __device__ __forceinline__ void to_planes_cvt(uint4& h, uint4& l) const {

@@ -9,12 +9,14 @@
 //           adjacency D~^-1/2 (A + I) D~^-1/2 of Kipf & Welling, symmetric, so the same kernel
 //           serves the backward pass.
 //
-// Gather-bound and, at the tiny local degrees random partitioning leaves (about deg/M),
-// latency-bound: a warp takes 8 consecutive rows at a time, reads their offsets with one load and their
-// column indices with one coalesced load per 32 entries (consecutive rows are consecutive
-// in the CSR), and walks the entries with eight (four for rows wider than 256) neighbours' rows in flight per lane.  Lanes
-// split the feature width in pieces of 8 values (16 bytes per plane).
+// At the tiny local degrees random partitioning leaves (about deg/M) the kernel is bound by memory
+// latency and by instruction issue, not by bandwidth: a warp takes 8 consecutive rows at a time, reads
+// their offsets with one load and their column indices with one coalesced load per 32 entries
+// (consecutive rows are consecutive in the CSR), and walks the entries with eight (four for rows
+// wider than 256) neighbours' rows in flight per lane.  Lanes split the feature width in pieces of
+// 8 values (16 bytes per plane).
 #include <algorithm>
+#include <climits>
 
 #include "train.cuh"
 
@@ -100,120 +102,173 @@ heavy_list_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict
 // MODE 0: out[v] = w[v] * sum_u src[u]                      (w = 1 / deg)
 // MODE 1: out[v] = sum_u w[u] * src[u]                      (w = 1 / deg)
 // MODE 2: out[v] = w[v] * (w[v] * src[v] + sum_u w[u] * src[u])   (w = (deg + 1)^-1/2)
+//
+// The kernel is bound by instruction issue as much as by memory latency, so the entry loop is
+// kept lean: per-lane byte offsets are fixed once (lanes past the row's width read column 0 and
+// only their stores are masked), a neighbour's address is one 32x32->64 multiply-add per plane,
+// entry positions are 32-bit numbers relative to the group's first entry, and only the last,
+// partial batch of a 32-entry piece checks how many entries it has.
 template <int NCH, int MODE>
 __global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 2 : 1)
 spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
             const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
             const int d, const int64_t total_groups, const SpmmOrder order, int* __restrict__ ticket) {
-    // neighbours' rows a lane has in flight: a hub row is a chain of entries / SPMM_INFLIGHT memory
-    // round trips, and that chain sets the length of the whole launch
-    constexpr int SPMM_INFLIGHT = NCH == 1 ? 8 : 4;
+    // neighbours' rows a lane has in flight
+    constexpr int W = NCH == 1 ? 8 : 4;
     const int lane = threadIdx.x & 31;
+    const uint32_t src_row_bytes = (uint32_t)src.ld * 2u;
+    bool live[NCH];          // the lane's 8 columns of chunk c exist
+    uint32_t col_bytes[NCH]; // their byte offset inside a row (0 for lanes without columns)
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        const int colx = (c * 32 + lane) * 8;
+        live[c] = colx < d;
+        col_bytes[c] = live[c] ? (uint32_t)colx * 2u : 0u;
+    }
+    // first group of every part, one part per lane (two for more than 32 parts): a group's part is
+    // found with one vote instead of a walk over the parts
+    // (the launch code has checked that tickets fit an int)
+    int first_lo = 0, first_hi = 0;
+    for (int k = 0; k < g.num && k < lane + 32; ++k) {
+        const int t = (g.rows[k] + SPMM_ROWS_PER_WARP - 1) / SPMM_ROWS_PER_WARP;
+        if (k < lane) first_lo += t;
+        first_hi += t;
+    }
+    if (lane >= g.num) first_lo = INT_MAX;
+    if (lane + 32 >= g.num) first_hi = INT_MAX;
+    const int n_heavy = order.heavy_count ? *order.heavy_count : 0;
+    const int last_ticket = n_heavy + (int)total_groups;
+    const int64_t heavy = order.heavy_count ? order.heavy : INT64_MAX;
+
   // Warps draw groups of 8 consecutive rows from a shared ticket counter until none are left:
   // degrees are power-law distributed, and a fixed assignment would leave most warps idle while
   // a few finish their hub rows.
   for (;;) {
-    int64_t grp = 0;
+    int grp = 0;
     if (lane == 0) grp = atomicAdd(ticket, 1);
     grp = __shfl_sync(0xffffffffu, grp, 0);
     // tickets 0 .. n_heavy-1 are the listed heavy groups, the rest all groups in row order
-    const int64_t n_heavy = order.heavy_count ? *order.heavy_count : 0;
-    if (grp >= n_heavy + total_groups) break;
+    if (grp >= last_ticket) break;
     const bool listed = grp < n_heavy;
     grp = listed ? order.heavy_list[grp] : grp - n_heavy;
-    int k, i0;
-    if (!locate_tile(g, SPMM_ROWS_PER_WARP, grp, &k, &i0)) break;
-    const int n_p = g.rows[k];
+    int k = __popc(__ballot_sync(0xffffffffu, grp >= first_lo)) - 1;
+    int first = __shfl_sync(0xffffffffu, first_lo, k & 31);
+    if (g.num > 32 && k == 31) {
+        const int more = __popc(__ballot_sync(0xffffffffu, grp >= first_hi));
+        if (more) first = __shfl_sync(0xffffffffu, first_hi, more - 1);
+        k += more;
+    }
+    if (k < 0 || k >= g.num) break;
+    const int i0 = (grp - first) * SPMM_ROWS_PER_WARP;
     const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
-    const int32_t* cols = col_out + g.edge_abs[k];
     const int64_t ws = g.row_ws[k];
-    const int nrows = max(0, min(SPMM_ROWS_PER_WARP, n_p - i0));
+    const int nrows = max(0, min(SPMM_ROWS_PER_WARP, g.rows[k] - i0));
 
     // offsets of the warp's rows: lane j holds rp[i0 + j], j = 0..nrows
     const int64_t my_off = (nrows > 0 && lane <= nrows) ? rp[i0 + lane] : 0;
-    const int64_t e_begin = __shfl_sync(0xffffffffu, my_off, 0);
-    const int64_t e_end = __shfl_sync(0xffffffffu, my_off, nrows);
     // the rows' own weights, one coalesced load instead of a dependent load per finished row
     const float my_w = (MODE != 1 && lane < nrows) ? inv_deg[ws + i0 + lane] : 1.f;
-    if (!listed && order.heavy_count && e_end - e_begin >= order.heavy) continue;  // done as a listed group
+    const int64_t e_begin = __shfl_sync(0xffffffffu, my_off, 0);
+    const int64_t e_end = __shfl_sync(0xffffffffu, my_off, nrows);
+    if (!listed && e_end - e_begin >= heavy) continue;  // done as a listed group
+    // the offsets relative to the group's first entry (a part has fewer than 2^31 entries: checked by the caller)
+    const int my_rel = (int)(my_off - e_begin);
+    const int n_entries = (int)(e_end - e_begin);
+    const int32_t* cols = col_out + g.edge_abs[k] + e_begin;
 
     Pack8 acc[NCH];
 #pragma unroll
     for (int c = 0; c < NCH; ++c) acc[c].zero();
-    int cur = 0;  // row (relative to i0) the accumulators belong to
-    int64_t next_off = __shfl_sync(0xffffffffu, my_off, 1);  // first entry past row `cur`
+    int cur = 0;                                          // row (relative to i0) the accumulators belong to
+    int next_rel = __shfl_sync(0xffffffffu, my_rel, 1);  // first entry past row `cur`
 
-    // finishes row `row`: scale, store, clear
+    // the lane's columns of the group's first output row; the rows are finished in order
+    char* out_hi[NCH];
+    char* out_lo[NCH];
+    const char* self_hi[NCH];
+    const char* self_lo[NCH];
+    const uint32_t out_row_bytes = (uint32_t)out.ld * 2u;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        out_hi[c] = reinterpret_cast<char*>(out.hi + (ws + i0) * out.ld) + col_bytes[c];
+        out_lo[c] = reinterpret_cast<char*>(out.lo + (ws + i0) * out.ld) + col_bytes[c];
+        if (MODE == 2) {
+            self_hi[c] = reinterpret_cast<const char*>(src.hi + (ws + i0) * src.ld) + col_bytes[c];
+            self_lo[c] = reinterpret_cast<const char*>(src.lo + (ws + i0) * src.ld) + col_bytes[c];
+        }
+    }
+    // finishes row `row` (= the next row in order): scale, store, clear
     auto flush = [&](int row) {
-        const int64_t r = ws + i0 + row;
         const float w = MODE == 1 ? 1.f : __shfl_sync(0xffffffffu, my_w, row);
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
-            const int colx = (c * 32 + lane) * 8;
-            if (colx < d) {
+            if (live[c]) {
                 if (MODE == 2)  // the self loop
-                    acc[c].fma_planes_mixed(w, *reinterpret_cast<const uint4*>(src.hi + r * src.ld + colx),
-                                            *reinterpret_cast<const uint4*>(src.lo + r * src.ld + colx));
+                    acc[c].fma_planes_mixed(w, *reinterpret_cast<const uint4*>(self_hi[c]), *reinterpret_cast<const uint4*>(self_lo[c]));
                 if (MODE != 1) {
 #pragma unroll
                     for (int e = 0; e < 8; ++e) acc[c].v[e] *= w;
                 }
                 uint4 h, l;
-                acc[c].to_planes_cvt(h, l);
-                *reinterpret_cast<uint4*>(out.hi + r * out.ld + colx) = h;
-                *reinterpret_cast<uint4*>(out.lo + r * out.ld + colx) = l;
+                acc[c].to_planes_lean(h, l);
+                *reinterpret_cast<uint4*>(out_hi[c]) = h;
+                *reinterpret_cast<uint4*>(out_lo[c]) = l;
             }
             acc[c].zero();
+            out_hi[c] += out_row_bytes;
+            out_lo[c] += out_row_bytes;
+            if (MODE == 2) {
+                self_hi[c] += src_row_bytes;
+                self_lo[c] += src_row_bytes;
+            }
         }
     };
 
-    const __nv_bfloat16* sh = src.hi + ws * src.ld;
-    const __nv_bfloat16* sl = src.lo + ws * src.ld;
+    // the lane's columns of the part's first source row
+    const char* base_hi[NCH];
+    const char* base_lo[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        base_hi[c] = reinterpret_cast<const char*>(src.hi + ws * src.ld) + col_bytes[c];
+        base_lo[c] = reinterpret_cast<const char*>(src.lo + ws * src.ld) + col_bytes[c];
+    }
 
-    for (int64_t e0 = e_begin; e0 < e_end; e0 += 32) {
-        const int cnt = (int)min((int64_t)32, e_end - e0);
-        const int64_t e = e0 + lane;
-        const int32_t mine = lane < cnt ? __ldg(cols + e) : 0;
+    for (int p0 = 0; p0 < n_entries; p0 += 32) {   // pieces of 32 entries
+        const int cnt = min(32, n_entries - p0);
+        const int32_t mine = lane < cnt ? __ldg(cols + p0 + lane) : 0;
         const float mine_w = (MODE != 0 && lane < cnt) ? __ldg(inv_deg + ws + mine) : 0.f;
-        for (int t = 0; t < cnt; t += SPMM_INFLIGHT) {
-            int32_t nb[SPMM_INFLIGHT];
-            float wt[SPMM_INFLIGHT];
+        // one batch: W neighbours' rows requested, then added in entry order
+        auto batch = [&](const int t, const bool full) {
+            uint4 xh[W][NCH], xl[W][NCH];
 #pragma unroll
-            for (int j = 0; j < SPMM_INFLIGHT; ++j) {
-                const int tj = min(t + j, cnt - 1);
-                nb[j] = __shfl_sync(0xffffffffu, mine, tj);
-                wt[j] = MODE != 0 ? __shfl_sync(0xffffffffu, mine_w, tj) : 1.f;
-                if (t + j >= cnt) nb[j] = -1;
-            }
-            {
-                uint4 xh[SPMM_INFLIGHT][NCH], xl[SPMM_INFLIGHT][NCH];
+            for (int j = 0; j < W; ++j) {
+                // past the end of a partial batch the last entry is read again and left out below
+                const uint32_t nb = (uint32_t)__shfl_sync(0xffffffffu, mine, full ? t + j : min(t + j, cnt - 1));
 #pragma unroll
-                for (int j = 0; j < SPMM_INFLIGHT; ++j)
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        const int colx = (c * 32 + lane) * 8;
-                        if (nb[j] >= 0 && colx < d) {  // the same condition guards every use below
-                            xh[j][c] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)nb[j] * src.ld + colx));
-                            xl[j][c] = __ldg(reinterpret_cast<const uint4*>(sl + (int64_t)nb[j] * src.ld + colx));
-                        }
-                    }
-#pragma unroll
-                for (int j = 0; j < SPMM_INFLIGHT; ++j) {
-                    if (nb[j] < 0) continue;
-                    // entries come in row order: the rows that end before this entry are complete
-                    while (e0 + t + j >= next_off) {
-                        flush(cur++);
-                        next_off = __shfl_sync(0xffffffffu, my_off, cur + 1);
-                    }
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        if ((c * 32 + lane) * 8 >= d) continue;
-                        if (MODE != 0) acc[c].fma_planes_mixed(wt[j], xh[j][c], xl[j][c]);
-                        else acc[c].add_planes_mixed(xh[j][c], xl[j][c]);
-                    }
+                for (int c = 0; c < NCH; ++c) {
+                    xh[j][c] = __ldg(reinterpret_cast<const uint4*>(base_hi[c] + (uint64_t)nb * src_row_bytes));
+                    xl[j][c] = __ldg(reinterpret_cast<const uint4*>(base_lo[c] + (uint64_t)nb * src_row_bytes));
                 }
             }
-        }
+#pragma unroll
+            for (int j = 0; j < W; ++j) {
+                if (!full && t + j >= cnt) break;
+                // entries come in row order: the rows that end before this entry are complete
+                while (p0 + t + j >= next_rel) {
+                    flush(cur++);
+                    next_rel = __shfl_sync(0xffffffffu, my_rel, cur + 1);
+                }
+                const float wj = MODE != 0 ? __shfl_sync(0xffffffffu, mine_w, t + j) : 1.f;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    if (MODE != 0) acc[c].fma_planes_mixed(wj, xh[j][c], xl[j][c]);
+                    else acc[c].add_planes_mixed(xh[j][c], xl[j][c]);
+                }
+            }
+        };
+        int t = 0;
+        for (; t + W <= cnt; t += W) batch(t, true);
+        if (t < cnt) batch(t, false);
     }
     while (cur < nrows) flush(cur++);
   }

@@ -227,6 +227,10 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
         if (part_offsets[p + 1] < part_offsets[p] || edge_offsets[p + 1] < edge_offsets[p] ||
             part_offsets[p + 1] - part_offsets[p] >= (int64_t(1) << 31))
             return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "part %d has inconsistent offsets", p);
+    for (int p = 0; p < M; ++p)  // the aggregation kernels count a part's entries in 32 bits
+        if (edge_offsets[p + 1] - edge_offsets[p] >= (int64_t(1) << 31))
+            return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "part %d has %lld entries, the limit is 2^31 - 1", p,
+                             (long long)(edge_offsets[p + 1] - edge_offsets[p]));
     if (K == 0) return RTMA_OK;
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
     const bool single_pass = md->gemm_dtype == 1;
