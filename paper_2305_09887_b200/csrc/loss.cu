@@ -2,10 +2,10 @@
 // gradient (softmax - onehot) / n_p is written as split bf16 planes (it feeds the tensor-core
 // products of the backward pass).
 //
-// One warp per row, eight rows per warp.  With up to 128 classes a lane keeps its (at most four,
-// consecutive) logits in registers, so a row is read once, with one vector load, and its gradient
-// leaves with one vector store per plane; wider rows are swept three times (max, sum of
-// exponentials, gradient).
+// Up to 64 classes: one thread per row (the kernel is bound by instruction issue, and a row in one
+// thread needs no cross-lane reductions).  Up to 128 classes: one warp per row, eight rows per warp,
+// a lane keeping four consecutive logits in registers.  Wider rows are swept three times (max, sum
+// of exponentials, gradient).
 // Loss sums are reduced in a fixed order (warp -> block -> part): results do not change from
 // run to run.
 #include "train.cuh"
@@ -117,6 +117,75 @@ softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const
     }
 }
 
+// Up to 64 classes: one thread per row.  The row sits in the thread's registers (NV4 vector loads),
+// nothing crosses lanes, and the gradient leaves as 16-byte stores; a block of 64 threads is one
+// 64-row tile.  The loss is summed by a shuffle tree and then over the two warps: a fixed order.
+template <int NV4>
+__global__ void __launch_bounds__(LOSS_TILE_ROWS)
+softmax_xent_row_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
+                        const Planes dZ, float* __restrict__ tile_loss) {
+    __shared__ float warp_loss[LOSS_TILE_ROWS / 32];
+    int k, r0;
+    if (!locate_tile(g, LOSS_TILE_ROWS, blockIdx.x, &k, &r0)) return;
+    const int n_p = g.rows[k];
+    const int i = r0 + threadIdx.x;
+    float loss = 0.f;
+    if (i < n_p) {
+        const int64_t r = g.row_ws[k] + i;
+        const float4* z = reinterpret_cast<const float4*>(logits.ptr + r * logits.ld);
+        const int label = yp[g.row_abs[k] + i];
+        const int nv = (int)(logits.ld >> 2);
+        float v[4 * NV4];
+#pragma unroll
+        for (int q = 0; q < NV4; ++q) {
+            const float4 t = q < nv ? z[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[4 * q] = t.x; v[4 * q + 1] = t.y; v[4 * q + 2] = t.z; v[4 * q + 3] = t.w;
+        }
+        float zmax = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4 * NV4; ++c) {
+            if (c >= C) v[c] = -INFINITY;
+            zmax = fmaxf(zmax, v[c]);
+        }
+        float sum = 0.f, zl = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4 * NV4; ++c) {
+            if (c == label) zl = v[c];
+            v[c] = c < C ? expf(v[c] - zmax) : 0.f;
+            sum += v[c];
+        }
+        loss = zmax + logf(sum) - zl;
+        const float scale = 1.0f / (sum * (float)n_p);  // softmax / n_p = e * scale
+        const float hot = 1.0f / (float)n_p;
+        const int n8 = (int)(dZ.ld >> 3);
+        uint4* ph = reinterpret_cast<uint4*>(dZ.hi + r * dZ.ld);
+        uint4* pl = reinterpret_cast<uint4*>(dZ.lo + r * dZ.ld);
+#pragma unroll
+        for (int q = 0; q < NV4 / 2; ++q) {
+            if (q >= n8) break;
+            Pack8 x;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int c = 8 * q + e;
+                x.v[e] = c < C ? v[c] * scale - (c == label ? hot : 0.f) : 0.f;  // padding columns stay zero
+            }
+            uint4 h, l;
+            x.to_planes_cvt(h, l);
+            ph[q] = h;
+            pl[q] = l;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+    if ((threadIdx.x & 31) == 0) warp_loss[threadIdx.x >> 5] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float sacc = 0.f;
+        for (int w = 0; w < LOSS_TILE_ROWS / 32; ++w) sacc += warp_loss[w];
+        tile_loss[blockIdx.x] = sacc;
+    }
+}
+
 // More than 128 classes: the row is swept three times (max, sum of exponentials, gradient).
 __global__ void __launch_bounds__(LOSS_THREADS)
 softmax_xent_wide_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
@@ -189,8 +258,10 @@ int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C
     const int64_t tiles = group_tiles(g, LOSS_TILE_ROWS);
     if (tiles > 0) {
         KernelScope ks(ctx, KC_LOSS, s);
-        if (C <= 32) softmax_xent_kernel<1><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
-        else if (C <= 64) softmax_xent_kernel<2><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        if (C <= 16) softmax_xent_row_kernel<4><<<(unsigned)tiles, LOSS_TILE_ROWS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        else if (C <= 32) softmax_xent_row_kernel<8><<<(unsigned)tiles, LOSS_TILE_ROWS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        else if (C <= 48) softmax_xent_row_kernel<12><<<(unsigned)tiles, LOSS_TILE_ROWS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        else if (C <= 64) softmax_xent_row_kernel<16><<<(unsigned)tiles, LOSS_TILE_ROWS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         else if (C <= LOSS_REG_CLASSES) softmax_xent_kernel<4><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         else softmax_xent_wide_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         RTMA_LAUNCH_CHECK(ctx);
