@@ -80,9 +80,25 @@ def relabel(part_id: np.ndarray, M: int):
     return part_offsets, perm, local_id
 
 
-def partition(n: int, group_id, seed: int, M: int):
+def relabel_grouped(part_id: np.ndarray, group_id: np.ndarray, M: int):
+    """Within a part: by super-node id, then by global id."""
+    n = part_id.size
+    part_id = _i32(part_id)
+    group_id = _i32(group_id)
+    part_offsets = np.empty(M + 1, dtype=np.int64)
+    perm = np.empty(n, dtype=np.int32)
+    local_id = np.empty(n, dtype=np.int32)
+    lib().orc_relabel_grouped(ctypes.c_int64(n), ctypes.c_int32(M), _p(part_id, c_i32p), _p(group_id, c_i32p),
+                              _p(part_offsets, c_i64p), _p(perm, c_i32p), _p(local_id, c_i32p))
+    return part_offsets, perm, local_id
+
+
+def partition(n: int, group_id, seed: int, M: int, grouped: bool = False):
     part_id = assign(n, group_id, seed, M)
-    part_offsets, perm, local_id = relabel(part_id, M)
+    if grouped:
+        part_offsets, perm, local_id = relabel_grouped(part_id, group_id, M)
+    else:
+        part_offsets, perm, local_id = relabel(part_id, M)
     return part_id, part_offsets, perm, local_id
 
 

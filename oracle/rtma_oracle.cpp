@@ -12,6 +12,7 @@
 //   orc_assign            RandomTMA (node level) and SuperTMA (super-node
 //                         level) assignment, Sec. 3.2.2.
 //   orc_relabel           alpha^{-1}(i) as ordered lists (Preliminaries).
+//   orc_relabel_grouped   the same lists with every super-node's members adjacent.
 //   orc_induced_csr       the node-induced subgraph G^(i) (Preliminaries).
 //   orc_spmm_mean         row-normalised aggregation, A-bar X of Theorem 2 /
 //                         Eq. (proof-2-pred): (1/d_v) sum over the effective
@@ -38,6 +39,7 @@
 // finite differences).  Convergence / accuracy against the paper's tables:
 // parity unpinned (different task, datasets not available).
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -926,6 +928,26 @@ void orc_relabel(int64_t n, int32_t M, const int32_t* part_id, int64_t* part_off
         local_id[v] = (int32_t)cursor[p];
         perm[part_offsets[p] + cursor[p]] = (int32_t)v;
         cursor[p]++;
+    }
+}
+
+// The same lists with the members of a super-node kept together (SuperTMA, Sec. 3.2.2: a
+// super-node is assigned as a whole, so all its members are in the part): within a part
+// nodes are ordered by super-node id (as a signed 32-bit number), then by global id.
+void orc_relabel_grouped(int64_t n, int32_t M, const int32_t* part_id, const int32_t* group_id,
+                         int64_t* part_offsets, int32_t* perm, int32_t* local_id) {
+    std::vector<std::vector<int32_t>> members(M);
+    for (int64_t v = 0; v < n; ++v) members[part_id[v]].push_back((int32_t)v);
+    part_offsets[0] = 0;
+    for (int32_t p = 0; p < M; ++p) {
+        std::vector<int32_t>& m = members[p];
+        // ids were pushed in ascending order; a stable sort by super-node id keeps that order inside a super-node
+        std::stable_sort(m.begin(), m.end(), [&](int32_t a, int32_t b) { return group_id[a] < group_id[b]; });
+        part_offsets[p + 1] = part_offsets[p] + (int64_t)m.size();
+        for (size_t i = 0; i < m.size(); ++i) {
+            perm[part_offsets[p] + (int64_t)i] = m[i];
+            local_id[m[i]] = (int32_t)i;
+        }
     }
 }
 

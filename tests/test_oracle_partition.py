@@ -78,6 +78,66 @@ def test_relabel_brute_force_small():
     assert local_id.tolist() == [0, 0, 1, 0, 1, 2, 2]
 
 
+def test_grouped_relabel_hand_example():
+    # parts:  node 0..7 -> [1, 0, 1, 0, 1, 0, 1, 1]; super-nodes (negative and sparse ids allowed)
+    part_id = np.array([1, 0, 1, 0, 1, 0, 1, 1], dtype=np.int32)
+    group = np.array([9, 4, -3, 4, 9, -8, -3, 9], dtype=np.int32)
+    part_offsets, perm, local_id = oracle.relabel_grouped(part_id, group, 2)
+    assert part_offsets.tolist() == [0, 3, 8]
+    # part 0 holds nodes 1, 3 (super-node 4) and 5 (super-node -8): -8 first, then 4 with ids ascending
+    # part 1 holds 2, 6 (super-node -3) then 0, 4, 7 (super-node 9)
+    assert perm.tolist() == [5, 1, 3, 2, 6, 0, 4, 7]
+    assert local_id.tolist() == [2, 1, 0, 2, 3, 0, 1, 4]
+
+
+@pytest.mark.parametrize("n,M,groups", [(1, 1, 1), (9, 4, 3), (5000, 8, 60), (60_000, 32, 700)])
+def test_grouped_relabel_is_the_lexicographic_order_part_group_id(n, M, groups):
+    rng = np.random.default_rng(n)
+    group = (rng.integers(0, groups, size=n).astype(np.int64) * 2_654_435 - 900_000_000).astype(np.int32)  # sparse, some negative
+    part_id, part_offsets, perm, local_id = oracle.partition(n, group, 77, M, grouped=True)
+    assert np.array_equal(part_id, oracle.assign(n, group, 77, M))
+    # numpy's lexsort (last key is the primary one) is the independent statement of the order
+    expect = np.lexsort((np.arange(n), group, part_id)).astype(np.int32)
+    assert np.array_equal(perm, expect)
+    assert np.array_equal(np.diff(part_offsets), np.bincount(part_id, minlength=M))
+    assert np.array_equal(perm[part_offsets[part_id] + local_id], np.arange(n))
+    # every super-node is one contiguous run of rows
+    g_in_order = group[perm]
+    runs = 1 + np.count_nonzero(np.diff(g_in_order) != 0) if n > 1 else 1
+    assert runs == np.unique(group).size
+
+
+def test_grouped_relabel_with_identity_groups_is_the_plain_relabel():
+    n, M = 20_000, 16
+    ident = np.arange(n, dtype=np.int32)
+    a = oracle.partition(n, ident, 5, M, grouped=True)
+    b = oracle.partition(n, None, 5, M)
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+
+
+def test_grouped_order_leaves_the_induced_subgraphs_isomorphic(tiny_workload):
+    # the order of the rows inside a part is a relabelling: same kept / cut counts, same degree multiset,
+    # same set of kept edges in global ids
+    g = tiny_workload.graph
+    rng = np.random.default_rng(3)
+    group = rng.integers(0, 40, size=g.n).astype(np.int32)
+    M = 4
+    res = {}
+    for grouped in (False, True):
+        part_id, part_offsets, perm, local_id = oracle.partition(g.n, group, 11, M, grouped=grouped)
+        rowptr_out, col_out, edge_offsets, kept, cut = oracle.induced_csr(g.rowptr, g.col, M, part_id, part_offsets, perm, local_id)
+        edges = set()
+        for p in range(M):
+            rp, cp = oracle.part_graph(rowptr_out, col_out, part_offsets, edge_offsets, p)
+            base = int(part_offsets[p])
+            for i in range(rp.size - 1):
+                for e in range(int(rp[i]), int(rp[i + 1])):
+                    edges.add((int(perm[base + i]), int(perm[base + int(cp[e])])))
+        res[grouped] = (kept, cut, edges)
+    assert res[False] == res[True]
+
+
 def test_supernodes_stay_whole_and_identity_groups_reproduce_node_scheme():
     n, M, seed = 30_000, 16, 1234
     rng = np.random.default_rng(0)
