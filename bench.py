@@ -159,7 +159,7 @@ def cpu_sample(w, local_steps=1):
     L = len(w.dims) - 1
     t0 = time.perf_counter()
     part_id, part_offsets, perm, local_id = oracle.partition(g.n, g.group_id if w.use_groups else None,
-                                                             w.partition_seed, w.M)
+                                                             w.partition_seed, w.M, grouped=w.use_groups and w.grouped_order)
     rowptr_out, col_out, edge_offsets, kept, cut = oracle.induced_csr(
         g.rowptr, g.col, w.M, part_id, part_offsets, perm, local_id)
     Xp = oracle.gather_rows(w.X, perm)
@@ -216,6 +216,7 @@ def make_workload(args):
                             use_groups=args.assign == "super", gemm_dtype=1)
     else:
         w = inputs.large(1.0 if s is None else s)
+    w.grouped_order = args.order == "group"   # only matters with super-node assignment
     variant = (1 if args.encoder == "gcn" else 0, 1 if args.act == "prelu" else 0, 1 if args.norm == "layernorm" else 0)
     if variant != (0, 0, 0):   # the paper's own encoders (Sec. 4.1) on the same graph, features and widths
         w.variant = variant
@@ -292,7 +293,7 @@ def run_link(args, rank, local_rank, world):
     res = {k: (v.to(device) if v is not None else None) for k, v in host.items()}
 
     def preprocess():
-        part_id, part_offsets, perm, local_id = ctx.partition(g.n, res["gid"], w.partition_seed, w.M)
+        part_id, part_offsets, perm, local_id = ctx.partition(g.n, res["gid"], w.partition_seed, w.M, grouped=w.grouped_order)
         rowptr_out, col_out, edge_offsets, kept_cut, edge_host = ctx.build_induced_csr(
             res["rowptr"], res["col"], w.M, part_id, part_offsets, perm, local_id)
         Xp = ctx.gather_rows(res["X"], perm)
@@ -416,6 +417,8 @@ def main():
     ap.add_argument("--scale", type=float, default=None, help="shrink (or grow) the workload's graph")
     ap.add_argument("--M", type=int, default=None, help="trainers (supertma / sweep)")
     ap.add_argument("--assign", default="super", choices=["node", "super"], help="sweep: assignment scheme")
+    ap.add_argument("--order", default="group", choices=["id", "group"],
+                    help="rows inside a part: by node id, or super-nodes kept together (super-node assignment only)")
     ap.add_argument("--task", default="node", choices=["node", "link"],
                     help="node classification (the named workloads) or link prediction (the paper's task)")
     ap.add_argument("--encoder", default="sage", choices=["sage", "gcn"])
@@ -471,7 +474,7 @@ def main():
 
     def step():
         params.copy_(d_params0.expand(w.M, P))                      # W_global[0] broadcast to the trainers
-        part_id, part_offsets, perm, local_id = ctx.partition(g.n, resident["gid"], w.partition_seed, w.M)
+        part_id, part_offsets, perm, local_id = ctx.partition(g.n, resident["gid"], w.partition_seed, w.M, grouped=w.grouped_order)
         rowptr_out, col_out, edge_offsets, kept_cut, edge_host = ctx.build_induced_csr(
             resident["rowptr"], resident["col"], w.M, part_id, part_offsets, perm, local_id)
         Xp = ctx.gather_rows(resident["X"], perm)
@@ -618,6 +621,7 @@ def main():
                                             "counted once per step in the unit",
                    "variant": {"encoder": args.encoder, "act": args.act, "norm": args.norm},
                    "assignment": "super-node" if w.use_groups else "node",
+                   "row_order": "super-node id, then node id" if (w.use_groups and w.grouped_order) else "node id",
                    "kept_fraction": kept / g.num_entries,
                    "parallelism": ("replicas only" if world > 1 else
                                    f"single GPU, {w.M} trainers batched on {n_streams} stream(s)"),

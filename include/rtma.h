@@ -81,6 +81,18 @@ int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group_id, uint64
                        int32_t M, int32_t* part_id, int64_t* part_offsets, int32_t* perm,
                        int32_t* local_id, void* stream);
 
+/* The same assignment with every super-node's members adjacent in memory: inside a part the
+ * nodes are ordered by super-node id (as a signed 32-bit number), then by node id, instead of
+ * by node id alone.  SuperTMA assigns a super-node as a whole (Sec. 3.2.2), so all its members
+ * are in the part, and in the graphs the scheme is meant for most of a node's neighbours are in
+ * its own super-node (mini-clusters, Sec. 3.2.2): with this order they are nearby rows of the
+ * part, which the aggregation kernels of rtma_local_steps turn into cache hits.  part_id and
+ * part_offsets equal rtma_partition's; perm and local_id differ only in the order inside each
+ * part.  group_id == NULL is rtma_partition.  Arguments, limits and errors as rtma_partition. */
+int32_t rtma_partition_grouped(rtma_ctx* ctx, int64_t n, const int32_t* group_id, uint64_t seed,
+                               int32_t M, int32_t* part_id, int64_t* part_offsets, int32_t* perm,
+                               int32_t* local_id, void* stream);
+
 /* The same partition for callers that must not allocate device memory.  (The paper has no
  * counterpart: this is a deployment variant of rtma_partition.)  Some hosts of this library
  * cannot call cudaMalloc at the point where they partition: code running while a CUDA graph is
@@ -284,8 +296,8 @@ int32_t rtma_selftest_wait_timeout(rtma_ctx* ctx, void* stream);
 /* ---- the whole path on HOST buffers (Sec. 3: partition, Algorithm 2, Algorithm 1) --------
  * Every pointer here is a HOST pointer (pageable or pinned).  Copies the graph (CSR as for
  * rtma_build_induced_csr), group_id_h (NULL = RandomTMA), features X_h [n][dims[0]], labels
- * y_h [n] and the common initial parameters params0_h [P] to the device, runs rtma_partition,
- * rtma_build_induced_csr, rtma_gather_rows, then R rounds of (rtma_local_steps with K steps on
+ * y_h [n] and the common initial parameters params0_h [P] to the device, runs rtma_partition
+ * (rtma_partition_grouped when super-node ids are given), rtma_build_induced_csr, rtma_gather_rows, then R rounds of (rtma_local_steps with K steps on
  * every part, rtma_aggregate), and copies back params_out_h [P] (the averaged parameters),
  * loss_out_h [R][M][K] (or NULL) and kept_cut_h [2] (or NULL).  The graph must be undirected
  * with both directions stored.  Allocates and frees its device buffers with cudaMalloc /

@@ -18,7 +18,7 @@ MAX_PARTS = 64
 MAX_LAYERS = 8
 
 EXPORTS = (
-    "rtma_create", "rtma_destroy", "rtma_last_error", "rtma_workspace_bytes", "rtma_partition",
+    "rtma_create", "rtma_destroy", "rtma_last_error", "rtma_workspace_bytes", "rtma_partition", "rtma_partition_grouped",
     "rtma_build_induced_csr", "rtma_gather_rows", "rtma_param_count", "rtma_local_steps",
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
@@ -205,8 +205,9 @@ class Context:
                 for i in range(KERNEL_CLASSES)}
 
     # ---- R1 -------------------------------------------------------------------------
-    def partition(self, n: int, group_id, seed: int, M: int, stream=None):
-        """Returns (part_id[n] i32, part_offsets[M+1] i64, perm[n] i32, local_id[n] i32)."""
+    def partition(self, n: int, group_id, seed: int, M: int, stream=None, grouped: bool = False):
+        """Returns (part_id[n] i32, part_offsets[M+1] i64, perm[n] i32, local_id[n] i32).
+        grouped: rtma_partition_grouped (inside a part, order by super-node id, then node id)."""
         dev = self.device
         if group_id is not None:
             _need(group_id, torch.int32, "group_id", dev)
@@ -214,10 +215,11 @@ class Context:
         part_offsets = torch.empty(M + 1, dtype=torch.int64, device=dev)
         perm = torch.empty(n, dtype=torch.int32, device=dev)
         local_id = torch.empty(n, dtype=torch.int32, device=dev)
-        st = self._lib.rtma_partition(self._h, ctypes.c_int64(n), _ptr(group_id), ctypes.c_uint64(seed),
-                                      ctypes.c_int32(M), _ptr(part_id), _ptr(part_offsets), _ptr(perm),
-                                      _ptr(local_id), ctypes.c_void_p(_stream_handle(stream)))
-        self._check(st, "rtma_partition")
+        fn = self._lib.rtma_partition_grouped if grouped else self._lib.rtma_partition
+        st = fn(self._h, ctypes.c_int64(n), _ptr(group_id), ctypes.c_uint64(seed),
+                ctypes.c_int32(M), _ptr(part_id), _ptr(part_offsets), _ptr(perm),
+                _ptr(local_id), ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_partition_grouped" if grouped else "rtma_partition")
         return part_id, part_offsets, perm, local_id
 
     def build_induced_csr(self, rowptr, col, M: int, part_id, part_offsets, perm, local_id, stream=None):

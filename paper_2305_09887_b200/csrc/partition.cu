@@ -8,6 +8,8 @@
 //      (part, chunk) the first output slot of that chunk's members;
 //   3. every warp hashes its chunk again and ranks its nodes inside the warp with
 //      match.any, 32 nodes per round, which keeps id order.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace {
@@ -33,7 +35,7 @@ __device__ __forceinline__ int part_of(int64_t v, const int32_t* __restrict__ gr
 
 __global__ void __launch_bounds__(PART_THREADS)
 part_count_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t seed, int M, int64_t num_chunks,
-                  int32_t* __restrict__ counts) {
+                  int32_t* __restrict__ counts, const int32_t* __restrict__ order_in) {
     __shared__ int32_t hist[PART_WARPS][RTMA_MAX_PARTS + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t chunk = (int64_t)blockIdx.x * PART_WARPS + warp;
@@ -41,8 +43,8 @@ part_count_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t seed
     __syncwarp();
     if (chunk >= num_chunks) return;
     for (int r = 0; r < PART_ROUNDS; ++r) {
-        const int64_t v = chunk * PART_CHUNK + r * 32 + lane;
-        const int pid = v < n ? part_of(v, group_id, seed, M) : M;
+        const int64_t pos = chunk * PART_CHUNK + r * 32 + lane;  // position in the input order (node id if none is given)
+        const int pid = pos < n ? part_of(order_in ? order_in[pos] : pos, group_id, seed, M) : M;
         const unsigned peers = __match_any_sync(0xffffffffu, pid);
         if (lane == __ffs(peers) - 1) hist[warp][pid] += __popc(peers);
         __syncwarp();
@@ -54,7 +56,7 @@ __global__ void __launch_bounds__(PART_THREADS)
 part_scatter_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t seed, int M, int64_t num_chunks,
                     const int64_t* __restrict__ scanned, int32_t* __restrict__ part_id,
                     int64_t* __restrict__ part_offsets, int32_t* __restrict__ perm,
-                    int32_t* __restrict__ local_id) {
+                    int32_t* __restrict__ local_id, const int32_t* __restrict__ order_in) {
     __shared__ int32_t cursor[PART_WARPS][RTMA_MAX_PARTS + 1];
     __shared__ int32_t first_slot[RTMA_MAX_PARTS + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -69,8 +71,9 @@ part_scatter_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t se
     if (chunk >= num_chunks) return;
     const unsigned below = (1u << lane) - 1u;
     for (int r = 0; r < PART_ROUNDS; ++r) {
-        const int64_t v = chunk * PART_CHUNK + r * 32 + lane;
-        const bool live = v < n;
+        const int64_t pos = chunk * PART_CHUNK + r * 32 + lane;
+        const bool live = pos < n;
+        const int64_t v = live && order_in ? order_in[pos] : pos;
         const int pid = live ? part_of(v, group_id, seed, M) : M;
         const unsigned peers = __match_any_sync(0xffffffffu, pid);
         const int slot = live ? cursor[warp][pid] + __popc(peers & below) : 0;
@@ -111,11 +114,118 @@ extern "C" int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group
     int64_t* scanned = cur.take<int64_t>(cells + 1);
     int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(cells));
     const unsigned blocks = (unsigned)ceil_div(num_chunks, PART_WARPS);
-    { KernelScope ks(ctx, KC_PART_COUNT, stream); part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts); }
+    { KernelScope ks(ctx, KC_PART_COUNT, stream); part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts, nullptr); }
     RTMA_LAUNCH_CHECK(ctx);
     RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, cells, scanned, scratch, stream));
     { KernelScope ks(ctx, KC_PART_SCATTER, stream); part_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, scanned, part_id,
-                                                             part_offsets, perm, local_id); }
+                                                             part_offsets, perm, local_id, nullptr); }
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}
+
+// ------------------------------------------------------------------------------------
+// Partition with every super-node's members adjacent: inside a part, order by super-node id,
+// then by node id.  The nodes are first sorted by super-node id with four stable 8-bit radix
+// passes (count per chunk and digit, scan, ranked scatter: the three steps of the partition
+// itself, with 256 buckets), then the partition pass runs over that order; being stable, it
+// keeps the super-node order inside every part.
+// ------------------------------------------------------------------------------------
+namespace {
+
+constexpr int RADIX_BUCKETS = 256;
+
+// digit of the super-node id taken as a signed number (sign bit flipped), least significant first
+__device__ __forceinline__ int radix_digit(int32_t group, int shift) {
+    return (int)((((uint32_t)group ^ 0x80000000u) >> shift) & (RADIX_BUCKETS - 1));
+}
+
+__global__ void __launch_bounds__(PART_THREADS)
+radix_count_kernel(int64_t n, const int32_t* __restrict__ order_in, const int32_t* __restrict__ group_id, int shift,
+                   int64_t num_chunks, int32_t* __restrict__ counts) {
+    __shared__ int32_t hist[PART_WARPS][RADIX_BUCKETS + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t chunk = (int64_t)blockIdx.x * PART_WARPS + warp;
+    for (int b = lane; b <= RADIX_BUCKETS; b += 32) hist[warp][b] = 0;
+    __syncwarp();
+    if (chunk >= num_chunks) return;
+    for (int r = 0; r < PART_ROUNDS; ++r) {
+        const int64_t pos = chunk * PART_CHUNK + r * 32 + lane;
+        const int dig = pos < n ? radix_digit(group_id[order_in ? order_in[pos] : pos], shift) : RADIX_BUCKETS;
+        const unsigned peers = __match_any_sync(0xffffffffu, dig);
+        if (lane == __ffs(peers) - 1) hist[warp][dig] += __popc(peers);
+        __syncwarp();
+    }
+    for (int b = lane; b < RADIX_BUCKETS; b += 32) counts[(int64_t)b * num_chunks + chunk] = hist[warp][b];
+}
+
+__global__ void __launch_bounds__(PART_THREADS)
+radix_scatter_kernel(int64_t n, const int32_t* __restrict__ order_in, const int32_t* __restrict__ group_id, int shift,
+                     int64_t num_chunks, const int64_t* __restrict__ scanned, int32_t* __restrict__ order_out) {
+    __shared__ int32_t cursor[PART_WARPS][RADIX_BUCKETS + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t chunk = (int64_t)blockIdx.x * PART_WARPS + warp;
+    if (chunk >= num_chunks) return;
+    for (int b = lane; b < RADIX_BUCKETS; b += 32) cursor[warp][b] = (int32_t)scanned[(int64_t)b * num_chunks + chunk];
+    __syncwarp();
+    const unsigned below = (1u << lane) - 1u;
+    for (int r = 0; r < PART_ROUNDS; ++r) {
+        const int64_t pos = chunk * PART_CHUNK + r * 32 + lane;
+        const bool live = pos < n;
+        const int32_t v = live ? (order_in ? order_in[pos] : (int32_t)pos) : 0;
+        const int dig = live ? radix_digit(group_id[v], shift) : RADIX_BUCKETS;
+        const unsigned peers = __match_any_sync(0xffffffffu, dig);
+        const int slot = live ? cursor[warp][dig] + __popc(peers & below) : 0;
+        __syncwarp();
+        if (live && lane == __ffs(peers) - 1) cursor[warp][dig] += __popc(peers);
+        __syncwarp();
+        if (live) order_out[slot] = v;
+    }
+}
+
+}  // namespace
+
+extern "C" int32_t rtma_partition_grouped(rtma_ctx* ctx, int64_t n, const int32_t* group_id, uint64_t seed, int32_t M,
+                                          int32_t* part_id, int64_t* part_offsets, int32_t* perm, int32_t* local_id,
+                                          void* stream_) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    if (!group_id) return rtma_partition(ctx, n, group_id, seed, M, part_id, part_offsets, perm, local_id, stream_);
+    if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
+    if (n < 0 || n >= (int64_t(1) << 31)) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "n=%lld outside [0,2^31)", (long long)n);
+    if (!part_offsets || (n > 0 && (!part_id || !perm || !local_id)))
+        return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_partition_grouped: null output pointer");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    if (n == 0) {
+        RTMA_CUDA(ctx, cudaMemsetAsync(part_offsets, 0, sizeof(int64_t) * (M + 1), stream));
+        return RTMA_OK;
+    }
+    const int64_t num_chunks = ceil_div(n, PART_CHUNK);
+    const int64_t cells = num_chunks * std::max<int64_t>(RADIX_BUCKETS, M);
+    const size_t need = 2 * ArenaCursor::granule(sizeof(int32_t) * n) + ArenaCursor::granule(sizeof(int32_t) * cells) +
+                        ArenaCursor::granule(sizeof(int64_t) * (cells + 1)) +
+                        ArenaCursor::granule(sizeof(int64_t) * scan_scratch_elems(cells));
+    RTMA_TRY(rtma_reserve(ctx, need));
+    ArenaCursor cur(ctx->arena);
+    int32_t* order[2] = {cur.take<int32_t>(n), cur.take<int32_t>(n)};
+    int32_t* counts = cur.take<int32_t>(cells);
+    int64_t* scanned = cur.take<int64_t>(cells + 1);
+    int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(cells));
+    const unsigned blocks = (unsigned)ceil_div(num_chunks, PART_WARPS);
+    const int32_t* in = nullptr;  // NULL: node id order
+    for (int pass = 0; pass < 4; ++pass) {
+        int32_t* out = order[pass & 1];
+        { KernelScope ks(ctx, KC_PART_COUNT, stream); radix_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, in, group_id, 8 * pass, num_chunks, counts); }
+        RTMA_LAUNCH_CHECK(ctx);
+        RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, num_chunks * RADIX_BUCKETS, scanned, scratch, stream));
+        { KernelScope ks(ctx, KC_PART_SCATTER, stream); radix_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, in, group_id, 8 * pass, num_chunks, scanned, out); }
+        RTMA_LAUNCH_CHECK(ctx);
+        in = out;
+    }
+    { KernelScope ks(ctx, KC_PART_COUNT, stream); part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts, in); }
+    RTMA_LAUNCH_CHECK(ctx);
+    RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, num_chunks * M, scanned, scratch, stream));
+    { KernelScope ks(ctx, KC_PART_SCATTER, stream); part_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, scanned, part_id,
+                                                             part_offsets, perm, local_id, in); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }
@@ -220,10 +330,10 @@ extern "C" int32_t rtma_partition_static(int32_t device, int64_t n, const int32_
     int32_t* counts = reinterpret_cast<int32_t*>(g_partition_scratch_ptr[device]);
     int64_t* scanned = reinterpret_cast<int64_t*>(g_partition_scratch_ptr[device] + STATIC_COUNTS_BYTES);
     const unsigned blocks = (unsigned)ceil_div(num_chunks, PART_WARPS);
-    part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts);
+    part_count_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, counts, nullptr);
     part_scan_one_block_kernel<<<1, 1024, 0, stream>>>(counts, cells, scanned);
     part_scatter_kernel<<<blocks, PART_THREADS, 0, stream>>>(n, group_id, seed, M, num_chunks, scanned, part_id,
-                                                             part_offsets, perm, local_id);
+                                                             part_offsets, perm, local_id, nullptr);
     e = cudaGetLastError();
     return e == cudaSuccess ? RTMA_OK : static_fail(RTMA_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
 }

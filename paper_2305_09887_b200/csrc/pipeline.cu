@@ -61,8 +61,9 @@ extern "C" int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_6
     int64_t* rowptr_out = static_cast<int64_t*>(at(o_rpo));
     int64_t* edge_offsets = static_cast<int64_t*>(at(o_eoff));
     int64_t* kept_cut = static_cast<int64_t*>(at(o_kc));
-    RTMA_TRY(rtma_partition(ctx, n, group_id_h ? static_cast<int32_t*>(at(o_gid)) : nullptr, seed, M, part_id,
-                            part_offsets, perm, local_id, stream));
+    // with super-nodes, their members are kept together (plain rtma_partition when there are none)
+    RTMA_TRY(rtma_partition_grouped(ctx, n, group_id_h ? static_cast<int32_t*>(at(o_gid)) : nullptr, seed, M, part_id,
+                                    part_offsets, perm, local_id, stream));
     RTMA_TRY(rtma_build_induced_csr(ctx, n, rowptr_is_64, at(o_rowptr), static_cast<int32_t*>(at(o_col)), M, part_id,
                                     part_offsets, perm, local_id, rowptr_out, nullptr, edge_offsets, kept_cut, stream));
     std::vector<int64_t> po(M + 1), eo(M + 1);

@@ -99,6 +99,38 @@ heavy_list_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict
         if (group_entries(g, rowptr_out, grp) >= heavy) list[atomicAdd(count, 1)] = (int)grp;
 }
 
+// How local are the rows' neighbourhoods?  Counts, over every 8th row, the entries whose column lies
+// within LOCAL_SPAN rows of the row itself.  When most do (super-nodes stored together), the
+// aggregation kernels hand out groups block by block, so that the warps of a block work on
+// neighbouring rows and share their source rows through L1.
+constexpr int LOCAL_SPAN = 512;
+__global__ void __launch_bounds__(256)
+locality_probe_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
+                      const int32_t* __restrict__ col_out, const int64_t total_rows, unsigned long long* __restrict__ near_total) {
+    unsigned long long near = 0, total = 0;
+    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t * 8 < total_rows; t += (int64_t)gridDim.x * 256) {
+        int k, i;
+        if (!locate_tile(g, 1, t * 8, &k, &i)) break;
+        const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
+        const int32_t* cols = col_out + g.edge_abs[k];
+        const int64_t b = rp[i], e = rp[i + 1];
+        for (int64_t x = b; x < e; ++x) {
+            const int c = cols[x];
+            near += (c - i < LOCAL_SPAN && i - c < LOCAL_SPAN) ? 1u : 0u;
+        }
+        total += (unsigned long long)(e - b);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        near += __shfl_xor_sync(0xffffffffu, near, o);
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    if ((threadIdx.x & 31) == 0 && total) {  // integer sums: the order of the additions does not matter
+        atomicAdd(near_total, near);
+        atomicAdd(near_total + 1, total);
+    }
+}
+
 // MODE 0: out[v] = w[v] * sum_u src[u]                      (w = 1 / deg)
 // MODE 1: out[v] = sum_u w[u] * src[u]                      (w = 1 / deg)
 // MODE 2: out[v] = w[v] * (w[v] * src[v] + sum_u w[u] * src[u])   (w = (deg + 1)^-1/2)
@@ -140,15 +172,29 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     const int last_ticket = n_heavy + (int)total_groups;
     const int64_t heavy = order.heavy_count ? order.heavy : INT64_MAX;
 
+    // neighbourhoods are local (see locality_probe_kernel): groups go out eight at a time, to a block
+    const bool by_block = order.near_total && order.near_total[1] > 0 && 2 * order.near_total[0] >= order.near_total[1];
+    __shared__ int block_ticket;
+
   // Warps draw groups of 8 consecutive rows from a shared ticket counter until none are left:
   // degrees are power-law distributed, and a fixed assignment would leave most warps idle while
   // a few finish their hub rows.
   for (;;) {
     int grp = 0;
-    if (lane == 0) grp = atomicAdd(ticket, 1);
-    grp = __shfl_sync(0xffffffffu, grp, 0);
+    if (by_block) {  // the same for every thread of the block: the barriers are reached by all
+        __syncthreads();
+        if (threadIdx.x == 0) block_ticket = atomicAdd(ticket, SPMM_THREADS / 32);
+        __syncthreads();
+        grp = block_ticket;
+        if (grp >= last_ticket) break;
+        grp += threadIdx.x >> 5;
+        if (grp >= last_ticket) continue;
+    } else {
+        if (lane == 0) grp = atomicAdd(ticket, 1);
+        grp = __shfl_sync(0xffffffffu, grp, 0);
+        if (grp >= last_ticket) break;
+    }
     // tickets 0 .. n_heavy-1 are the listed heavy groups, the rest all groups in row order
-    if (grp >= last_ticket) break;
     const bool listed = grp < n_heavy;
     grp = listed ? order.heavy_list[grp] : grp - n_heavy;
     int k = __popc(__ballot_sync(0xffffffffu, grp >= first_lo)) - 1;
@@ -158,7 +204,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
         if (more) first = __shfl_sync(0xffffffffu, first_hi, more - 1);
         k += more;
     }
-    if (k < 0 || k >= g.num) break;
+    if (k < 0 || k >= g.num) continue;  // cannot happen for a ticket below last_ticket
     const int i0 = (grp - first) * SPMM_ROWS_PER_WARP;
     const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
     const int64_t ws = g.row_ws[k];
@@ -282,6 +328,203 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     }
 }
 
+// Rows of at most 64 values (the backward pass of the last layer aggregates at the width of the
+// classes).  A 16-byte piece per lane would leave most of the warp idle, so the warp is cut into
+// sub-groups of LPR lanes, one per row: the 8 rows of a group advance side by side (two per
+// sub-group for LPR = 8), WN entries of every row per round, and nothing crosses lanes.  Rows longer
+// than NARROW_LONG entries would keep the whole warp waiting for one sub-group; they are done
+// afterwards by all sub-groups together, a few entries each per round, and summed across the sub-groups.
+constexpr int NARROW_LONG = 16;
+constexpr int NARROW_INFLIGHT = 4;  // neighbours' rows a lane has in flight
+
+template <int LPR, int MODE>
+__global__ void __launch_bounds__(SPMM_THREADS, 2)
+spmm_narrow_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
+                   const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src,
+                   const Planes out, const int d, const int64_t total_groups, const SpmmOrder order,
+                   int* __restrict__ ticket) {
+    constexpr int S = 32 / LPR;                   // sub-groups
+    constexpr int RPS = SPMM_ROWS_PER_WARP / S;   // rows a sub-group works on at once
+    constexpr int WN = NARROW_INFLIGHT / RPS;     // entries of each of them per round
+    static_assert(RPS >= 1 && RPS * S == SPMM_ROWS_PER_WARP, "sub-groups must tile the rows of a group");
+    const int lane = threadIdx.x & 31;
+    const int sub = lane / LPR, sl = lane % LPR;
+    const bool live = sl * 8 < d;
+    const uint32_t col_bytes = live ? (uint32_t)sl * 16u : 0u;
+    const uint32_t src_row_bytes = (uint32_t)src.ld * 2u, out_row_bytes = (uint32_t)out.ld * 2u;
+    int first_lo = 0, first_hi = 0;  // first group of every part, one part per lane (see spmm_kernel)
+    for (int k = 0; k < g.num && k < lane + 32; ++k) {
+        const int t = (g.rows[k] + SPMM_ROWS_PER_WARP - 1) / SPMM_ROWS_PER_WARP;
+        if (k < lane) first_lo += t;
+        first_hi += t;
+    }
+    if (lane >= g.num) first_lo = INT_MAX;
+    if (lane + 32 >= g.num) first_hi = INT_MAX;
+    const int n_heavy = order.heavy_count ? *order.heavy_count : 0;
+    const int last_ticket = n_heavy + (int)total_groups;
+    const int64_t heavy = order.heavy_count ? order.heavy : INT64_MAX;
+
+    const bool by_block = order.near_total && order.near_total[1] > 0 && 2 * order.near_total[0] >= order.near_total[1];
+    __shared__ int block_ticket;
+
+    for (;;) {
+        int grp = 0;
+        if (by_block) {  // as in spmm_kernel: eight groups at a time, to a block
+            __syncthreads();
+            if (threadIdx.x == 0) block_ticket = atomicAdd(ticket, SPMM_THREADS / 32);
+            __syncthreads();
+            grp = block_ticket;
+            if (grp >= last_ticket) break;
+            grp += threadIdx.x >> 5;
+            if (grp >= last_ticket) continue;
+        } else {
+            if (lane == 0) grp = atomicAdd(ticket, 1);
+            grp = __shfl_sync(0xffffffffu, grp, 0);
+            if (grp >= last_ticket) break;
+        }
+        const bool listed = grp < n_heavy;
+        grp = listed ? order.heavy_list[grp] : grp - n_heavy;
+        int k = __popc(__ballot_sync(0xffffffffu, grp >= first_lo)) - 1;
+        int first = __shfl_sync(0xffffffffu, first_lo, k & 31);
+        if (g.num > 32 && k == 31) {
+            const int more = __popc(__ballot_sync(0xffffffffu, grp >= first_hi));
+            if (more) first = __shfl_sync(0xffffffffu, first_hi, more - 1);
+            k += more;
+        }
+        if (k < 0 || k >= g.num) continue;  // cannot happen for a ticket below last_ticket
+        const int i0 = (grp - first) * SPMM_ROWS_PER_WARP;
+        const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
+        const int64_t ws = g.row_ws[k];
+        const int nrows = max(0, min(SPMM_ROWS_PER_WARP, g.rows[k] - i0));
+        const int64_t my_off = (nrows > 0 && lane <= nrows) ? rp[i0 + lane] : 0;
+        const float my_w = (MODE != 1 && lane < nrows) ? inv_deg[ws + i0 + lane] : 1.f;
+        const int64_t e_begin = __shfl_sync(0xffffffffu, my_off, 0);
+        const int64_t e_end = __shfl_sync(0xffffffffu, my_off, nrows);
+        if (!listed && e_end - e_begin >= heavy) continue;  // done as a listed group
+        const int my_rel = lane <= nrows ? (int)(my_off - e_begin) : 0;
+        const int32_t* cols = col_out + g.edge_abs[k] + e_begin;
+        const char* base_hi = reinterpret_cast<const char*>(src.hi + ws * src.ld) + col_bytes;
+        const char* base_lo = reinterpret_cast<const char*>(src.lo + ws * src.ld) + col_bytes;
+        const int my_deg = __shfl_down_sync(0xffffffffu, my_rel, 1) - my_rel;  // lane j < nrows: entries of row j
+        const unsigned long_rows = __ballot_sync(0xffffffffu, lane < nrows && my_deg > NARROW_LONG);
+        const int round_deg = (lane < nrows && my_deg <= NARROW_LONG) ? my_deg : 0;
+        const int max_deg = __reduce_max_sync(0xffffffffu, round_deg);
+
+        // finishes the lane's row r with the sums in acc
+        auto finish = [&](Pack8& acc, const int r, const float w) {
+            if (!live || r >= nrows) return;
+            const int64_t row = ws + i0 + r;
+            if (MODE == 2)  // the self loop
+                acc.fma_planes_mixed(w, *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(src.hi + row * src.ld) + col_bytes),
+                                     *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(src.lo + row * src.ld) + col_bytes));
+            if (MODE != 1) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc.v[e] *= w;
+            }
+            uint4 h, l;
+            acc.to_planes_lean(h, l);
+            *reinterpret_cast<uint4*>(reinterpret_cast<char*>(out.hi) + row * out_row_bytes + col_bytes) = h;
+            *reinterpret_cast<uint4*>(reinterpret_cast<char*>(out.lo) + row * out_row_bytes + col_bytes) = l;
+        };
+
+        // ---- the short rows, side by side ----
+        Pack8 acc[RPS];
+        int rb[RPS], re[RPS];
+        float rw[RPS];
+#pragma unroll
+        for (int q = 0; q < RPS; ++q) {
+            const int r = sub + q * S;
+            acc[q].zero();
+            rb[q] = __shfl_sync(0xffffffffu, my_rel, r);
+            re[q] = __shfl_sync(0xffffffffu, my_rel, r + 1);
+            rw[q] = __shfl_sync(0xffffffffu, my_w, r);
+            if (r >= nrows || (long_rows >> r & 1u)) re[q] = rb[q];
+        }
+        for (int t = 0; t < max_deg; t += WN) {
+            int32_t nb[RPS][WN];
+            float wt[RPS][WN];
+            uint4 xh[RPS][WN], xl[RPS][WN];
+#pragma unroll
+            for (int q = 0; q < RPS; ++q)
+#pragma unroll
+                for (int j = 0; j < WN; ++j) nb[q][j] = rb[q] + t + j < re[q] ? __ldg(cols + rb[q] + t + j) : -1;
+            if (MODE != 0) {
+#pragma unroll
+                for (int q = 0; q < RPS; ++q)
+#pragma unroll
+                    for (int j = 0; j < WN; ++j) wt[q][j] = nb[q][j] >= 0 ? __ldg(inv_deg + ws + nb[q][j]) : 0.f;
+            }
+#pragma unroll
+            for (int q = 0; q < RPS; ++q)
+#pragma unroll
+                for (int j = 0; j < WN; ++j)
+                    if (nb[q][j] >= 0) {
+                        xh[q][j] = __ldg(reinterpret_cast<const uint4*>(base_hi + (uint64_t)(uint32_t)nb[q][j] * src_row_bytes));
+                        xl[q][j] = __ldg(reinterpret_cast<const uint4*>(base_lo + (uint64_t)(uint32_t)nb[q][j] * src_row_bytes));
+                    }
+#pragma unroll
+            for (int q = 0; q < RPS; ++q)
+#pragma unroll
+                for (int j = 0; j < WN; ++j)
+                    if (nb[q][j] >= 0) {
+                        if (MODE != 0) acc[q].fma_planes_mixed(wt[q][j], xh[q][j], xl[q][j]);
+                        else acc[q].add_planes_mixed(xh[q][j], xl[q][j]);
+                    }
+        }
+#pragma unroll
+        for (int q = 0; q < RPS; ++q)
+            if (!(long_rows >> (sub + q * S) & 1u)) finish(acc[q], sub + q * S, rw[q]);
+
+        // ---- the long rows, one at a time, by all sub-groups ----
+        for (unsigned rest = long_rows; rest; rest &= rest - 1) {
+            const int r = __ffs(rest) - 1;
+            const int b = __shfl_sync(0xffffffffu, my_rel, r), e = __shfl_sync(0xffffffffu, my_rel, r + 1);
+            const float w = __shfl_sync(0xffffffffu, my_w, r);
+            Pack8 sum;
+            sum.zero();
+            for (int t = b + sub * NARROW_INFLIGHT; t < e; t += S * NARROW_INFLIGHT) {  // the bound differs by sub-group; nothing below crosses lanes
+                int32_t nb[NARROW_INFLIGHT];
+                float wt[NARROW_INFLIGHT];
+                uint4 xh[NARROW_INFLIGHT], xl[NARROW_INFLIGHT];
+#pragma unroll
+                for (int j = 0; j < NARROW_INFLIGHT; ++j) nb[j] = t + j < e ? __ldg(cols + t + j) : -1;
+                if (MODE != 0) {
+#pragma unroll
+                    for (int j = 0; j < NARROW_INFLIGHT; ++j) wt[j] = nb[j] >= 0 ? __ldg(inv_deg + ws + nb[j]) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < NARROW_INFLIGHT; ++j)
+                    if (nb[j] >= 0) {
+                        xh[j] = __ldg(reinterpret_cast<const uint4*>(base_hi + (uint64_t)(uint32_t)nb[j] * src_row_bytes));
+                        xl[j] = __ldg(reinterpret_cast<const uint4*>(base_lo + (uint64_t)(uint32_t)nb[j] * src_row_bytes));
+                    }
+#pragma unroll
+                for (int j = 0; j < NARROW_INFLIGHT; ++j)
+                    if (nb[j] >= 0) {
+                        if (MODE != 0) sum.fma_planes_mixed(wt[j], xh[j], xl[j]);
+                        else sum.add_planes_mixed(xh[j], xl[j]);
+                    }
+            }
+            __syncwarp();
+            // sub-group s adds the sums of sub-groups s + step: a fixed tree, so the order of the additions
+            // does not depend on timing; sub-group 0 ends with the row's sum
+#pragma unroll
+            for (int step = S / 2; step > 0; step >>= 1)
+#pragma unroll
+                for (int v = 0; v < 8; ++v) sum.v[v] += __shfl_down_sync(0xffffffffu, sum.v[v], step * LPR);
+            if (sub == 0) finish(sum, r, w);
+        }
+    }
+    // the last warp to run dry re-arms the ticket for the next launch
+    if (lane == 0) {
+        const int total_warps = gridDim.x * (SPMM_THREADS / 32);
+        if (atomicAdd(ticket + 1, 1) == total_warps - 1) {
+            ticket[0] = 0;
+            ticket[1] = 0;
+        }
+    }
+}
+
 template <int MODE>
 int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                       const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket, cudaStream_t s) {
@@ -298,7 +541,11 @@ int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64
         spmm_kernel<N, MODE><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, d,  \
                                                            groups, order, ticket);                        \
     } while (0)
-    if (d <= 256) RTMA_SPMM(1);
+    if (d <= 64) {
+        KernelScope ks(ctx, kclass, s);
+        if (d <= 32) spmm_narrow_kernel<4, MODE><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, d, groups, order, ticket);
+        else spmm_narrow_kernel<8, MODE><<<grid, SPMM_THREADS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out, d, groups, order, ticket);
+    } else if (d <= 256) RTMA_SPMM(1);
     else if (d <= 512) RTMA_SPMM(2);
     else if (d <= 1024) RTMA_SPMM(4);
     else return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "aggregation width %d > 1024", d);
@@ -362,9 +609,9 @@ int32_t launch_gcn_scale(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowpt
 
 int64_t spmm_order_entries(const GroupDesc& g) { return group_tiles(g, SPMM_ROWS_PER_WARP); }
 
-int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, int64_t entries, int* count,
-                          int* list, SpmmOrder* order, cudaStream_t s) {
-    *order = SpmmOrder{nullptr, nullptr, 0};
+int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                          int64_t entries, int* count, int* list, SpmmOrder* order, cudaStream_t s) {
+    *order = SpmmOrder{nullptr, nullptr, 0, nullptr};
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
     if (groups >= (int64_t(1) << 30)) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
@@ -373,6 +620,9 @@ int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, 256), 148 * 4);
     { KernelScope ks(ctx, KC_INV_DEGREE, s); heavy_list_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, groups, heavy, count, list); }
     RTMA_LAUNCH_CHECK(ctx);
-    *order = SpmmOrder{count, list, heavy};
+    unsigned long long* near_total = reinterpret_cast<unsigned long long*>(count + 2);
+    { KernelScope ks(ctx, KC_INV_DEGREE, s); locality_probe_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, col_out, group_tiles(g, 1), near_total); }
+    RTMA_LAUNCH_CHECK(ctx);
+    *order = SpmmOrder{count, list, heavy, near_total};
     return RTMA_OK;
 }

@@ -413,7 +413,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             int64_t wave_entries = 0;
             for (int k = 0; k < g.num; ++k) wave_entries += edge_offsets[g.part[k] + 1] - edge_offsets[g.part[k]];
             SpmmOrder wave_order;
-            RTMA_TRY(launch_spmm_order(ctx, g, rowptr_out, wave_entries, ticket + 16, heavy_list, &wave_order, s));
+            RTMA_TRY(launch_spmm_order(ctx, g, rowptr_out, col_out, wave_entries, ticket + 16, heavy_list, &wave_order, s));
             RTMA_TRY(launch_to_planes(ctx, g, Xp, m.dims[0], Hl[0], s));
             const Planes no_planes{nullptr, nullptr, 0};
             const Mat no_mat{nullptr, 0};
@@ -428,7 +428,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 // trainers reach the aggregation point with different step counts)
                 bool all_run = true;
                 for (int k = 0; k < wave.num; ++k) all_run = all_run && steps[wave.part[k]] > step;
-                const SpmmOrder order = all_run ? wave_order : SpmmOrder{nullptr, nullptr, 0};  // built for the whole wave
+                const SpmmOrder order = all_run ? wave_order : SpmmOrder{nullptr, nullptr, 0, nullptr};  // built for the whole wave
                 if (all_run) {
                     g = wave;
                     sp = wave_sp;

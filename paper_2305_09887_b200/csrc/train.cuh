@@ -83,11 +83,14 @@ struct SpmmOrder {
     const int* heavy_count;  // device: number of listed groups
     const int* heavy_list;   // device: their indices
     int64_t heavy;           // entries from which a group is listed
+    const unsigned long long* near_total;  // device: probed entries with a nearby column, probed entries;
+                                           // mostly nearby -> groups are handed out block by block
 };
-// list: spmm_order_entries(g) ints; count: one int, zero on entry; entries: kept entries of g's parts.
+// list: spmm_order_entries(g) ints; count: 8 ints (16-byte aligned), zero on entry: the number of listed
+// groups, then the two locality counters; entries: kept entries of g's parts.
 int64_t spmm_order_entries(const GroupDesc& g);
-int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, int64_t entries, int* count,
-                          int* list, SpmmOrder* order, cudaStream_t s);
+int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                          int64_t entries, int* count, int* list, SpmmOrder* order, cudaStream_t s);
 // out[r] = inv_deg[r] * sum_{u in N(r)} src[u]                      (forward, mean)
 // ticket: two ints of scratch, zero on entry and zero again when the kernel has finished.
 // order: from launch_spmm_order for this very g, or zeroed.

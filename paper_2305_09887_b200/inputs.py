@@ -44,6 +44,7 @@ class Workload:
     partition_seed: int
     params0: np.ndarray  # float32 [P], identical start for every trainer
     use_groups: bool = False
+    grouped_order: bool = False  # with use_groups: rows of a part ordered by super-node id, then node id
     gemm_dtype: int = 0  # 0: fp32-accurate GEMMs, 1: bf16 inputs / fp32 accumulate
     variant: tuple = (0, 0, 0)  # (encoder, act, norm): 0,0,0 = GraphSAGE-mean, ReLU, no normalisation
 

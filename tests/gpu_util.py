@@ -30,15 +30,16 @@ def rel_err(a, b):
     return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30)) if b.size else 0.0
 
 
-def gpu_preprocess(w, M=None, seed=None, use_groups=None):
+def gpu_preprocess(w, M=None, seed=None, use_groups=None, grouped=None):
     """partition + induced CSR + row gather on the GPU for workload w."""
     c = ctx()
     g = w.graph
     M = w.M if M is None else M
     seed = w.partition_seed if seed is None else seed
     use_groups = w.use_groups if use_groups is None else use_groups
+    grouped = (w.grouped_order and use_groups) if grouped is None else grouped
     gid = dev(g.group_id) if use_groups else None
-    part_id, part_offsets, perm, local_id = c.partition(g.n, gid, seed, M)
+    part_id, part_offsets, perm, local_id = c.partition(g.n, gid, seed, M, grouped=grouped)
     rowptr_out, col_out, edge_offsets, kept_cut, edge_host = c.build_induced_csr(
         dev(g.rowptr), dev(g.col), M, part_id, part_offsets, perm, local_id)
     Xp = c.gather_rows(dev(w.X), perm)
@@ -49,13 +50,14 @@ def gpu_preprocess(w, M=None, seed=None, use_groups=None):
                 edge_host=edge_host, part_host=part_offsets.cpu().tolist(), Xp=Xp, yp=yp, M=M)
 
 
-def oracle_preprocess(w, M=None, seed=None, use_groups=None):
+def oracle_preprocess(w, M=None, seed=None, use_groups=None, grouped=None):
     g = w.graph
     M = w.M if M is None else M
     seed = w.partition_seed if seed is None else seed
     use_groups = w.use_groups if use_groups is None else use_groups
+    grouped = (w.grouped_order and use_groups) if grouped is None else grouped
     gid = g.group_id if use_groups else None
-    part_id, part_offsets, perm, local_id = oracle.partition(g.n, gid, seed, M)
+    part_id, part_offsets, perm, local_id = oracle.partition(g.n, gid, seed, M, grouped=grouped)
     rowptr_out, col_out, edge_offsets, kept, cut = oracle.induced_csr(
         g.rowptr, g.col, M, part_id, part_offsets, perm, local_id)
     return dict(part_id=part_id, part_offsets=part_offsets, perm=perm, local_id=local_id,

@@ -37,6 +37,35 @@ def test_partition_empty_and_supernodes(util):
         assert np.array_equal(a.cpu().numpy(), b)
 
 
+@pytest.mark.parametrize("n,M,groups", [(1, 1, 1), (7, 3, 2), (1024, 5, 9), (1025, 64, 300), (250_000, 16, 2500),
+                                        (1_000_003, 32, 10_000)])
+def test_grouped_partition_matches_oracle(util, n, M, groups):
+    seed = 0x5EED0005 + n
+    rng = np.random.default_rng(n)
+    group = (rng.integers(0, groups, size=n).astype(np.int64) * 2_654_435 - 900_000_000).astype(np.int32)  # sparse, some negative
+    got = util.ctx().partition(n, util.dev(group), seed, M, grouped=True)
+    want = oracle.partition(n, group, seed, M, grouped=True)
+    for a, b in zip(got, want):
+        assert np.array_equal(a.cpu().numpy(), b)
+
+
+def test_grouped_partition_without_groups_and_empty(util):
+    a = util.ctx().partition(5000, None, 3, 8, grouped=True)
+    b = util.ctx().partition(5000, None, 3, 8)
+    assert all(torch.equal(x, y) for x, y in zip(a, b))
+    part_id, part_offsets, perm, local_id = util.ctx().partition(0, util.dev(np.zeros(0, dtype=np.int32)), 1, 4, grouped=True)
+    assert part_offsets.cpu().tolist() == [0] * 5
+
+
+def test_induced_csr_supernodes_grouped_order(util):
+    w = inputs.supertma(0.02)
+    got = util.gpu_preprocess(w, grouped=True)
+    want = util.oracle_preprocess(w, grouped=True)
+    util.assert_preprocess_equal(got, want)
+    plain = util.oracle_preprocess(w)
+    assert want["kept"] == plain["kept"] and want["cut"] == plain["cut"]
+
+
 def test_partition_is_deterministic(util):
     a = util.ctx().partition(300_000, None, 5, 8)
     b = util.ctx().partition(300_000, None, 5, 8)

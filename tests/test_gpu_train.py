@@ -45,6 +45,17 @@ def test_supertma_shape_scaled_feature_width_100(util):
     util.check_k_steps_and_average(w, got, want, 2)
 
 
+def test_supertma_super_nodes_kept_together(util):
+    # rows of a part ordered by super-node id: neighbourhoods become local, the aggregation kernels
+    # hand out row groups block by block; 256-wide and 47-wide aggregations
+    w = inputs.supertma(0.02, M=4)
+    w.grouped_order = True
+    w.dims = (100, 256, 47)
+    w.params0 = inputs.xavier_params(w.dims, 6)
+    got, want = util.check_one_step(w)
+    util.check_k_steps_and_average(w, got, want, 2)
+
+
 def test_bf16_operand_mode(util, tiny_workload):
     # gemm_dtype = 1: every product takes its operands rounded to bf16 and accumulates in fp32
     w = tiny_workload
