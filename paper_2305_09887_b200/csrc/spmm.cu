@@ -140,11 +140,15 @@ locality_probe_kernel(const __grid_constant__ GroupDesc g, const int64_t* __rest
 // only their stores are masked), a neighbour's address is one 32x32->64 multiply-add per plane,
 // entry positions are 32-bit numbers relative to the group's first entry, and only the last,
 // partial batch of a 32-entry piece checks how many entries it has.
-template <int NCH, int MODE>
-__global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 2 : 1)
-spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
-            const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
-            const int d, const int64_t total_groups, const SpmmOrder order, int* __restrict__ ticket) {
+// BY_BLOCK: neighbourhoods are local (see locality_probe_kernel) and groups go out eight at a time, to
+// a block.  The two ways of drawing groups are compiled separately (the kernel below picks one):
+// compiled as one loop, the barriers of the block-wise draw cost the warp-wise one a tenth more
+// instructions.
+template <int NCH, int MODE, bool BY_BLOCK>
+__device__ __forceinline__ void
+spmm_rows(const GroupDesc& g, const int64_t* __restrict__ rowptr_out,
+          const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
+          const int d, const int64_t total_groups, const SpmmOrder order, int* __restrict__ ticket) {
     // neighbours' rows a lane has in flight
     constexpr int W = NCH == 1 ? 8 : 4;
     const int lane = threadIdx.x & 31;
@@ -172,8 +176,7 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     const int last_ticket = n_heavy + (int)total_groups;
     const int64_t heavy = order.heavy_count ? order.heavy : INT64_MAX;
 
-    // neighbourhoods are local (see locality_probe_kernel): groups go out eight at a time, to a block
-    const bool by_block = order.near_total && order.near_total[1] > 0 && 2 * order.near_total[0] >= order.near_total[1];
+    constexpr bool by_block = BY_BLOCK;
     __shared__ int block_ticket;
 
   // Warps draw groups of 8 consecutive rows from a shared ticket counter until none are left:
@@ -328,6 +331,17 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
     }
 }
 
+template <int NCH, int MODE>
+__global__ void __launch_bounds__(SPMM_THREADS, NCH == 1 ? 2 : 1)
+spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
+            const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out,
+            const int d, const int64_t total_groups, const SpmmOrder order, int* __restrict__ ticket) {
+    if (order.near_total && order.near_total[1] > 0 && 2 * order.near_total[0] >= order.near_total[1])
+        spmm_rows<NCH, MODE, true>(g, rowptr_out, col_out, inv_deg, src, out, d, total_groups, order, ticket);
+    else
+        spmm_rows<NCH, MODE, false>(g, rowptr_out, col_out, inv_deg, src, out, d, total_groups, order, ticket);
+}
+
 // Rows of at most 64 values (the backward pass of the last layer aggregates at the width of the
 // classes).  A 16-byte piece per lane would leave most of the warp idle, so the warp is cut into
 // sub-groups of LPR lanes, one per row: the 8 rows of a group advance side by side (two per
@@ -337,12 +351,12 @@ spmm_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ row
 constexpr int NARROW_LONG = 16;
 constexpr int NARROW_INFLIGHT = 4;  // neighbours' rows a lane has in flight
 
-template <int LPR, int MODE>
-__global__ void __launch_bounds__(SPMM_THREADS, 2)
-spmm_narrow_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
-                   const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src,
-                   const Planes out, const int d, const int64_t total_groups, const SpmmOrder order,
-                   int* __restrict__ ticket) {
+template <int LPR, int MODE, bool BY_BLOCK>
+__device__ __forceinline__ void
+spmm_narrow_rows(const GroupDesc& g, const int64_t* __restrict__ rowptr_out,
+                 const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src,
+                 const Planes out, const int d, const int64_t total_groups, const SpmmOrder order,
+                 int* __restrict__ ticket) {
     constexpr int S = 32 / LPR;                   // sub-groups
     constexpr int RPS = SPMM_ROWS_PER_WARP / S;   // rows a sub-group works on at once
     constexpr int WN = NARROW_INFLIGHT / RPS;     // entries of each of them per round
@@ -364,7 +378,7 @@ spmm_narrow_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restric
     const int last_ticket = n_heavy + (int)total_groups;
     const int64_t heavy = order.heavy_count ? order.heavy : INT64_MAX;
 
-    const bool by_block = order.near_total && order.near_total[1] > 0 && 2 * order.near_total[0] >= order.near_total[1];
+    constexpr bool by_block = BY_BLOCK;
     __shared__ int block_ticket;
 
     for (;;) {
@@ -523,6 +537,18 @@ spmm_narrow_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restric
             ticket[1] = 0;
         }
     }
+}
+
+template <int LPR, int MODE>
+__global__ void __launch_bounds__(SPMM_THREADS, 2)
+spmm_narrow_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
+                   const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src,
+                   const Planes out, const int d, const int64_t total_groups, const SpmmOrder order,
+                   int* __restrict__ ticket) {
+    if (order.near_total && order.near_total[1] > 0 && 2 * order.near_total[0] >= order.near_total[1])
+        spmm_narrow_rows<LPR, MODE, true>(g, rowptr_out, col_out, inv_deg, src, out, d, total_groups, order, ticket);
+    else
+        spmm_narrow_rows<LPR, MODE, false>(g, rowptr_out, col_out, inv_deg, src, out, d, total_groups, order, ticket);
 }
 
 template <int MODE>
