@@ -99,8 +99,18 @@ class ClockSampler:
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
         self.proc = None
-        self.lines = []
+        self.lines = []      # (arrival time, line)
         self.thread = None
+        self.t_begin = None  # the timed region, on the host's monotonic clock
+        self.t_end = None
+
+    def begin(self):
+        """The timed region starts now (the sampler itself is started earlier: nvidia-smi takes a
+        few hundred milliseconds to deliver its first sample)."""
+        self.t_begin = time.monotonic()
+
+    def end(self):
+        self.t_end = time.monotonic()
 
     def start(self):
         try:
@@ -116,7 +126,7 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
 
     def stop(self):
         if self.proc is None:
@@ -128,7 +138,11 @@ class ClockSampler:
             self.proc.kill()
         sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        lo = self.t_begin if self.t_begin is not None else float("-inf")
+        hi = (self.t_end if self.t_end is not None else float("inf")) + 0.1   # a sample arrives up to one period late
+        for at, ln in self.lines:
+            if not (lo <= at <= hi):
+                continue
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 7:
                 continue
@@ -492,25 +506,27 @@ def main():
             ctx.aggregate(params)
         state.update(part_host=part_host, edge_host=edge_host)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()                      # started before the warm-up, windowed to the timed region below
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
     ctx.profile_read()
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     ctx.profile(True)
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
+    sampler.begin()
     for i in range(args.steps):
         flush.fill_(i & 0xFF)                                       # evict L2 between timed steps
         starts[i].record()
         step()
         stops[i].record()
     torch.cuda.synchronize()
+    sampler.end()
     if world > 1:
         dist.barrier()
     ctx.profile(False)

@@ -74,8 +74,16 @@ struct PrepArgs {
     __nv_bfloat16 *Bf_hi, *Bf_lo, *Bd_hi, *Bd_lo;  // [group slot][Npad][K]
 };
 
+constexpr int PREP_MAX_JOBS = 2 * RTMA_MAX_LAYERS;  // encoder and decoder layers of one step
+struct PrepBatch {
+    PrepArgs job[PREP_MAX_JOBS];
+};
+
+// blockIdx.z = layer (all layers of a step are repacked by one launch), blockIdx.y = part
 __global__ void __launch_bounds__(256)
-tc_weight_prep_kernel(const __grid_constant__ GroupDesc g, const PrepArgs a, const float* __restrict__ params) {
+tc_weight_prep_kernel(const __grid_constant__ GroupDesc g, const __grid_constant__ PrepBatch batch,
+                      const float* __restrict__ params) {
+    const PrepArgs& a = batch.job[blockIdx.z];
     const int k = blockIdx.y;
     const float* W = params + (int64_t)g.part[k] * a.ls.P + a.ls.param_offset;
     const int d_in = a.ls.d_in, d_out = a.ls.d_out;
@@ -716,14 +724,19 @@ size_t tc_prep_elems(const TcLayerPlan& p, bool with_dgrad) {
 
 bool tc_available() { return encode_tiled() != nullptr; }
 
-int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, const float* params,
-                              __nv_bfloat16* Bf_hi, __nv_bfloat16* Bf_lo, __nv_bfloat16* Bd_hi, __nv_bfloat16* Bd_lo,
+int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, const TcPrepJob* jobs, int njobs, const float* params,
                               cudaStream_t s) {
-    if (g.num == 0) return RTMA_OK;
-    PrepArgs a{ls, p.Npad_f, p.Kf, p.Npad_d, p.Kd, Bf_hi, Bf_lo, Bd_hi, Bd_lo};
-    const int64_t total = (int64_t)p.Npad_f * p.Kf + (Bd_hi ? (int64_t)p.Npad_d * p.Kd : 0);
-    dim3 grid((unsigned)std::min<int64_t>(ceil_div(total, 256), 64), (unsigned)g.num);
-    { KernelScope ks(ctx, KC_WEIGHT_PREP, s); tc_weight_prep_kernel<<<grid, 256, 0, s>>>(g, a, params); }
+    if (g.num == 0 || njobs == 0) return RTMA_OK;
+    if (njobs > PREP_MAX_JOBS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "internal: %d weight repack jobs", njobs);
+    PrepBatch b{};
+    int64_t most = 0;
+    for (int j = 0; j < njobs; ++j) {
+        const TcLayerPlan& p = jobs[j].plan;
+        b.job[j] = PrepArgs{jobs[j].ls, p.Npad_f, p.Kf, p.Npad_d, p.Kd, jobs[j].Bf_hi, jobs[j].Bf_lo, jobs[j].Bd_hi, jobs[j].Bd_lo};
+        most = std::max(most, (int64_t)p.Npad_f * p.Kf + (jobs[j].Bd_hi ? (int64_t)p.Npad_d * p.Kd : 0));
+    }
+    dim3 grid((unsigned)std::min<int64_t>(ceil_div(most, 256), 64), (unsigned)g.num, (unsigned)njobs);
+    { KernelScope ks(ctx, KC_WEIGHT_PREP, s); tc_weight_prep_kernel<<<grid, 256, 0, s>>>(g, b, params); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

@@ -452,10 +452,13 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                     }
                 }
                 // ---- forward ----
-                for (int l = 0; l < m.L; ++l)
-                    RTMA_TRY(launch_tc_weight_prep(ctx, g, m.layer[l], tcp[l], params, Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l], s));
-                for (int k = 0; k < m.Kd; ++k)
-                    RTMA_TRY(launch_tc_weight_prep(ctx, g, m.dec[k], dtcp[k], params, DBf_hi[k], DBf_lo[k], DBd_hi[k], DBd_lo[k], s));
+                {
+                    TcPrepJob jobs[2 * RTMA_MAX_LAYERS];
+                    int nj = 0;
+                    for (int l = 0; l < m.L; ++l) jobs[nj++] = TcPrepJob{m.layer[l], tcp[l], Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l]};
+                    for (int k = 0; k < m.Kd; ++k) jobs[nj++] = TcPrepJob{m.dec[k], dtcp[k], DBf_hi[k], DBf_lo[k], DBd_hi[k], DBd_lo[k]};
+                    RTMA_TRY(launch_tc_weight_prep(ctx, g, jobs, nj, params, s));
+                }
                 for (int l = 0; l < m.L; ++l) {
                     if (l == 0) {
                         // the aggregate of the input features does not change from step to step

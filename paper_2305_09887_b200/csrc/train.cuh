@@ -158,9 +158,14 @@ struct TcLayerPlan {
 bool tc_available();
 TcLayerPlan tc_plan_layer(LayerShape ls);
 size_t tc_prep_elems(const TcLayerPlan& p, bool with_dgrad);  // bf16 elements per part, hi and lo together
-// Repack one layer's weights of every part: transposed, zero padded, split into hi / lo.
-int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, const float* params,
-                              __nv_bfloat16* Bf_hi, __nv_bfloat16* Bf_lo, __nv_bfloat16* Bd_hi, __nv_bfloat16* Bd_lo,
+// Repack the weights of every listed layer, for every part, in one launch: transposed, zero padded,
+// split into hi / lo.  Bd_* may be NULL (no dgrad operand: the first layer).
+struct TcPrepJob {
+    LayerShape ls;
+    TcLayerPlan plan;
+    __nv_bfloat16 *Bf_hi, *Bf_lo, *Bd_hi, *Bd_lo;
+};
+int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, const TcPrepJob* jobs, int njobs, const float* params,
                               cudaStream_t s);
 // out = act([H | N] [Ws; Wn] + b), or act(N W + b) for a one-matrix layer (H is then ignored):
 // split planes when out_planes.hi != NULL, else fp32 out_f32.
