@@ -357,6 +357,11 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                     float bv[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) bv[e] = (bias && col_ok && n + e < a.N) ? __ldg(bias + n + e) : 0.f;
+                    // the thread's 16 bytes of row (lane >> 2) of the block, in either plane; the four
+                    // rows it finishes are 8 rows apart
+                    const uint32_t out_row_bytes = (uint32_t)a.out_planes.ld * 2u;
+                    char* oh = reinterpret_cast<char*>(a.out_planes.hi + (orow0 + (lane >> 2)) * a.out_planes.ld + n);
+                    char* ol = reinterpret_cast<char*>(a.out_planes.lo + (orow0 + (lane >> 2)) * a.out_planes.ld + n);
 #pragma unroll
                     for (int it = 0; it < 4; ++it) {
                         const int row = it * 8 + (lane >> 2);
@@ -366,13 +371,14 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                             Pack8 x;
                             x.v[0] = x0.x; x.v[1] = x0.y; x.v[2] = x0.z; x.v[3] = x0.w;
                             x.v[4] = x1.x; x.v[5] = x1.y; x.v[6] = x1.z; x.v[7] = x1.w;
+                            // Columns past the layer's width need no masking: the repacked weights are zero
+                            // there and so is bv, hence the accumulator, the sum and its ReLU are zero
+                            // and the padding columns of the planes stay zero.
 #pragma unroll
                             for (int e = 0; e < 8; ++e) {
-                                float tv = x.v[e] + bv[e];
-                                if (a.relu) tv = fmaxf(tv, 0.f);
-                                x.v[e] = (n + e < a.N) ? tv : 0.f;  // padding columns of the planes stay zero
+                                const float tv = x.v[e] + bv[e];
+                                x.v[e] = a.relu ? fmaxf(tv, 0.f) : tv;
                             }
-                            const int64_t at = (orow0 + row) * a.out_planes.ld + n;
                             if (a.gate_hi) {
                                 const uint32_t gw[4] = {gq[it].x, gq[it].y, gq[it].z, gq[it].w};
 #pragma unroll
@@ -382,9 +388,9 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                                 }
                             }
                             uint4 h, l;
-                            x.to_planes_cvt(h, l);
-                            *reinterpret_cast<uint4*>(a.out_planes.hi + at) = h;
-                            *reinterpret_cast<uint4*>(a.out_planes.lo + at) = l;
+                            x.to_planes_lean(h, l);
+                            *reinterpret_cast<uint4*>(oh + (size_t)(it * 8) * out_row_bytes) = h;
+                            *reinterpret_cast<uint4*>(ol + (size_t)(it * 8) * out_row_bytes) = l;
                         }
                     }
                 }
