@@ -14,7 +14,10 @@
 // their offsets with one load and their column indices with one coalesced load per 32 entries
 // (consecutive rows are consecutive in the CSR), and walks the entries with eight (four for rows
 // wider than 256) neighbours' rows in flight per lane.  Lanes split the feature width in pieces of
-// 8 values (16 bytes per plane).
+// 8 values (16 bytes per plane).  Rows of at most 64 values have a kernel of their own, in which
+// groups of lanes own one row each (spmm_narrow_kernel).  Where most neighbours of a row are rows
+// nearby (super-nodes stored together), groups are handed out eight at a time to a block, so that
+// its warps share their source rows through L1 (locality_probe_kernel decides, once per call).
 #include <algorithm>
 #include <climits>
 
