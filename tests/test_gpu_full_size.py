@@ -155,6 +155,33 @@ def test_supertma_full_size(util):
     _properties_after_training(util, w, got, 3)
 
 
+def test_trainer_count_sweep_kept_fractions(util):
+    # the SuperTMA graph under random node and random super-node assignment, M = 2 .. 32: kept and cut
+    # counts equal the oracle's, every array of the subgraphs too, and the fractions follow Sec. 3.2.2
+    # (1/M for nodes; (E_intra + E_inter / M) / E for whole super-nodes)
+    w = inputs.supertma()
+    g = w.graph
+    c = util.ctx()
+    rowptr, col, gid = util.dev(g.rowptr), util.dev(g.col), util.dev(g.group_id)
+    same_cluster = g.group_id[np.repeat(np.arange(g.n), np.diff(g.rowptr))] == g.group_id[g.col]
+    e_intra, e_all = int(np.count_nonzero(same_cluster)), g.num_entries
+    for use_groups in (False, True):
+        for M in (2, 4, 8, 16, 32):
+            gpu = c.partition(g.n, gid if use_groups else None, w.partition_seed, M, grouped=use_groups)
+            rowptr_out, col_out, edge_offsets, kept_cut, edge_host = c.build_induced_csr(rowptr, col, M, *gpu)
+            part_id, part_offsets, perm, local_id = oracle.partition(g.n, g.group_id if use_groups else None,
+                                                                     w.partition_seed, M, grouped=use_groups)
+            o_rowptr, o_col, o_edge, kept, cut = oracle.induced_csr(g.rowptr, g.col, M, part_id, part_offsets, perm, local_id)
+            assert kept_cut.cpu().tolist() == [kept, cut] and kept + cut == e_all
+            assert np.array_equal(gpu[2].cpu().numpy(), perm) and np.array_equal(gpu[3].cpu().numpy(), local_id)
+            assert np.array_equal(rowptr_out.cpu().numpy(), o_rowptr) and np.array_equal(col_out.cpu().numpy(), o_col)
+            assert np.array_equal(edge_offsets.cpu().numpy(), o_edge)
+            expect = (e_intra + (e_all - e_intra) / M) / e_all if use_groups else 1.0 / M
+            assert abs(kept / e_all - expect) < (0.01 if use_groups else 0.002)
+            del rowptr_out, col_out
+    torch.cuda.empty_cache()
+
+
 def test_large_shape_scaled(util):
     # int64 row offsets, M = 32, two classes with 1% positives, 128-256-2
     w = inputs.large(0.02)
