@@ -573,12 +573,12 @@ def main():
     else:
         roof = {"bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     # DRAM bytes per launch of the class (dram__bytes_read.sum + dram__bytes_write.sum averaged over the class's
-    # launches of one local step) from the ncu captures summarised in profiles/tc_rows_wgrad_medium.md and
-    # profiles/spmm_medium_supertma.md;
+    # launches of one local step) from ncu captures of these kernels on this workload (summaries under
+    # profiles/);
     # only for the workload and model that capture ran on
     traffic = None
     if w.name == "medium" and w.variant == (0, 0, 0) and w.gemm_dtype == 0:
-        traffic = {"gemm_forward": 463.9e6, "gemm_dgrad": 506.3e6, "gemm_wgrad": 502.9e6,
+        traffic = {"gemm_forward": 463.9e6, "gemm_dgrad": 505.6e6, "gemm_wgrad": 502.9e6,
                    "spmm_forward": 340.0e6, "spmm_backward": 194.0e6}.get(top)
     roof.update({"frac": (roof["achieved"] / roof["peak"]) if roof["achieved"] else None, "traffic": traffic,
                  "kernel": top, "launches_per_step": top_launches / args.steps,
