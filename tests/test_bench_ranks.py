@@ -70,3 +70,37 @@ def test_reference_arm_line_has_the_contract_keys():
     assert line["higher_is_better"] is True and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
     assert line["e2e"] == {"value": line["value"], "unit": "edges/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+
+
+def test_clock_samples_are_windowed_to_the_timed_region():
+    """The clock sampler starts before the warm-up (nvidia-smi is slow to deliver its first sample);
+    only samples that arrived during the timed region may enter the record, and throttle reasons
+    seen outside it must not be charged to it."""
+    sys.path.insert(0, ROOT)
+    import bench
+
+    class _Done:
+        def terminate(self):
+            pass
+
+        def wait(self, timeout=None):
+            return 0
+
+    s = bench.ClockSampler(0)
+    s.proc = _Done()
+    s.t_begin, s.t_end = 100.0, 101.0
+    s.lines = [
+        (99.0, "1200, 1965, 300.0, Not Active, Active, Not Active, Not Active"),     # warm-up: thermal flag
+        (100.2, "1800, 1965, 900.0, Not Active, Not Active, Not Active, Active"),
+        (100.6, "1900, 1965, 950.0, Not Active, Not Active, Not Active, Active"),
+        (101.05, "1850, 1965, 940.0, Not Active, Not Active, Not Active, Not Active"),  # one period late: kept
+        (102.0, "600, 1965, 100.0, Active, Not Active, Not Active, Not Active"),      # after: hardware flag
+    ]
+    rec = s.stop()
+    assert rec["samples"] == 3 and rec["sm_mhz"] == 1850.0 and rec["sm_max_mhz"] == 1965.0
+    assert rec["reasons"] == ["sw_power_cap"] and rec["power_w_max"] == 950.0
+    # without a window every sample counts
+    s2 = bench.ClockSampler(0)
+    s2.proc = _Done()
+    s2.lines = list(s.lines)
+    assert s2.stop()["samples"] == 5
