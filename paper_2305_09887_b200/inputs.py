@@ -2,8 +2,11 @@
 
 Everything here is input plumbing.  It holds none of the method's arithmetic
 (no partition hash, no aggregation, no training maths): randomness comes from
-numpy's ``default_rng(seed)``, and the arrays produced are handed unchanged to
-whichever implementation consumes them.  The shapes stand in for the paper's
+numpy's ``default_rng(seed)`` or, for the arrays with up to billions of
+elements (endpoint pairs, CSR construction, normal features), from the
+counter-based draws of the multi-threaded host library ``inputs_native.cpp``;
+the arrays produced are handed unchanged to whichever implementation consumes
+them.  The shapes stand in for the paper's
 workloads (Table 1: social / citation / e-commerce graphs with power-law
 degrees, 100-768 wide features), which are not redistributed with this code.
 
@@ -12,10 +15,56 @@ undirected edge stored, no self loops, no duplicates, columns sorted.
 """
 from __future__ import annotations
 
+import ctypes
 import dataclasses
 import math
+import os
+import subprocess
 
 import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_NATIVE_SRC = os.path.join(_HERE, "inputs_native.cpp")
+_NATIVE_LIB = os.path.join(_HERE, "libinputs_native.so")
+_native_handle = None
+
+
+def build_native(force: bool = False) -> str:
+    """Compiles inputs_native.cpp (g++, host only) next to this file."""
+    if force or not os.path.exists(_NATIVE_LIB) or os.path.getmtime(_NATIVE_LIB) < os.path.getmtime(_NATIVE_SRC):
+        tmp = f"{_NATIVE_LIB}.{os.getpid()}.tmp"
+        subprocess.run(["g++", "-O3", "-std=c++17", "-fPIC", "-shared", "-pthread", _NATIVE_SRC, "-o", tmp], check=True)
+        os.replace(tmp, _NATIVE_LIB)
+    return _NATIVE_LIB
+
+
+def _native():
+    global _native_handle
+    if _native_handle is None:
+        lib = ctypes.CDLL(build_native())
+        i64, u64, f64, ptr = ctypes.c_int64, ctypes.c_uint64, ctypes.c_double, ctypes.c_void_p
+        lib.rin_threads.restype = ctypes.c_int32
+        lib.rin_power_law_pairs.argtypes = [i64, i64, f64, f64, u64, ptr, ptr]
+        lib.rin_power_law_pairs.restype = None
+        lib.rin_csr_rows.argtypes = [i64, i64, ptr, ptr, ptr, ptr, ptr]
+        lib.rin_csr_rows.restype = i64
+        lib.rin_csr_compact.argtypes = [i64, ptr, ptr, ptr, ptr]
+        lib.rin_csr_compact.restype = None
+        lib.rin_normal_f32.argtypes = [i64, u64, ptr]
+        lib.rin_normal_f32.restype = None
+        lib.rin_add_rows_f32.argtypes = [i64, i64, ptr, ptr, ctypes.c_float, ptr]
+        lib.rin_add_rows_f32.restype = None
+        _native_handle = lib
+    return _native_handle
+
+
+def native_threads() -> int:
+    """Host threads the native producers use."""
+    return int(_native().rin_threads())
+
+
+def _p(a: np.ndarray):
+    return ctypes.c_void_p(a.ctypes.data)
 
 
 @dataclasses.dataclass
@@ -49,32 +98,20 @@ class Workload:
     variant: tuple = (0, 0, 0)  # (encoder, act, norm): 0,0,0 = GraphSAGE-mean, ReLU, no normalisation
 
 
-def _sorted_unique(key: np.ndarray) -> np.ndarray:
-    """np.unique by an in-place sort (several times faster on tens of millions of keys)."""
-    key.sort()
-    if key.size == 0:
-        return key
-    keep = np.empty(key.size, dtype=bool)
-    keep[0] = True
-    np.not_equal(key[1:], key[:-1], out=keep[1:])
-    return key[keep]
-
-
 def _csr_from_pairs(n: int, u: np.ndarray, v: np.ndarray, wide_rowptr: bool) -> Graph:
-    """Symmetrise, drop loops and duplicates, sort, and build CSR."""
-    keep = u != v
-    u = u[keep].astype(np.int64)
-    v = v[keep].astype(np.int64)
-    key = np.concatenate([u * n + v, v * n + u])
+    """Symmetrise, drop loops and duplicates, sort the columns of every row, and build CSR."""
+    u = np.ascontiguousarray(u, dtype=np.int32)
+    v = np.ascontiguousarray(v, dtype=np.int32)
+    m = int(u.size)
+    lib = _native()
+    tmp_rowptr = np.empty(n + 1, dtype=np.int64)
+    rowptr = np.empty(n + 1, dtype=np.int64)
+    col_tmp = np.empty(2 * m, dtype=np.int32)
+    entries = int(lib.rin_csr_rows(n, m, _p(u), _p(v), _p(tmp_rowptr), _p(col_tmp), _p(rowptr)))
     del u, v
-    key = _sorted_unique(key)  # sorted by (row, col), duplicates removed
-    rows = key // n
-    col = (key - rows * n).astype(np.int32)
-    del key
-    counts = np.bincount(rows, minlength=n)
-    del rows
-    rowptr = np.zeros(n + 1, dtype=np.int64)
-    np.cumsum(counts, out=rowptr[1:])
+    col = np.empty(entries, dtype=np.int32)
+    lib.rin_csr_compact(n, _p(tmp_rowptr), _p(rowptr), _p(col_tmp), _p(col))
+    del col_tmp, tmp_rowptr
     if not wide_rowptr:
         assert rowptr[-1] < 2**31
         rowptr = rowptr.astype(np.int32)
@@ -98,45 +135,50 @@ def uniform_graph(n: int, m_undirected: int, seed: int, wide_rowptr: bool = Fals
     return _csr_from_pairs(n, have // n, have % n, wide_rowptr)
 
 
-def _power_law_cdf(n: int, gamma: float, target_entries: float) -> np.ndarray:
-    """CDF of endpoint weights w_i ~ (i+i0)^(-1/(gamma-1)); i0 caps the largest
-    expected degree at sqrt(target_entries)."""
+def _power_law_offset(n: int, gamma: float, target_entries: float):
+    """Endpoint weights w(x) = (x + i0)^expo over ranks x in [0, n), expo = -1/(gamma-1).  i0 caps
+    the largest expected degree, target * W(0,1) / W(0,n) with W the integral of w, at
+    sqrt(target_entries).  Returns (i0, expo)."""
     expo = -1.0 / (gamma - 1.0)
-    idx = np.arange(n, dtype=np.float64)
+    e1 = expo + 1.0
     cap = math.sqrt(target_entries)
 
+    def integral(a: float, b: float, i0: float) -> float:
+        if abs(e1) < 1e-12:
+            return math.log((b + i0) / (a + i0))
+        return ((b + i0) ** e1 - (a + i0) ** e1) / e1
+
     def top_degree(i0: float) -> float:
-        w = (idx + i0) ** expo
-        return target_entries * w[0] / w.sum()
+        return target_entries * integral(0.0, 1.0, i0) / integral(0.0, float(n), i0)
 
     lo, hi = 1e-3, float(n)
     if top_degree(lo) <= cap:
-        i0 = lo
-    else:
-        for _ in range(60):
-            mid = math.sqrt(lo * hi)
-            if top_degree(mid) > cap:
-                lo = mid
-            else:
-                hi = mid
-        i0 = hi
-    w = (idx + i0) ** expo
-    cdf = np.cumsum(w)
-    cdf /= cdf[-1]
-    return cdf
+        return lo, expo
+    for _ in range(80):
+        mid = math.sqrt(lo * hi)
+        if top_degree(mid) > cap:
+            lo = mid
+        else:
+            hi = mid
+    return hi, expo
+
+
+def _power_law_pairs(n: int, m: int, gamma: float, target_entries: float, seed: int):
+    """m endpoint pairs, each endpoint drawn in proportion to its power-law weight; node ids are a
+    keyed permutation of the ranks, so hubs are spread over the id range."""
+    i0, expo = _power_law_offset(n, gamma, target_entries)
+    u = np.empty(m, dtype=np.int32)
+    v = np.empty(m, dtype=np.int32)
+    _native().rin_power_law_pairs(n, m, i0, expo, seed, _p(u), _p(v))
+    return u, v
 
 
 def chung_lu_graph(n: int, avg_degree: float, gamma: float, seed: int,
                    wide_rowptr: bool = False) -> Graph:
     """Chung-Lu power-law graph by endpoint sampling, node ids shuffled so that
     hubs are spread over the id range."""
-    rng = np.random.default_rng(seed)
     target = float(n) * avg_degree
-    cdf = _power_law_cdf(n, gamma, target)
-    m = int(target // 2)
-    shuffle = rng.permutation(n).astype(np.int64)
-    u = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
-    v = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
+    u, v = _power_law_pairs(n, int(target // 2), gamma, target, seed)
     return _csr_from_pairs(n, u, v, wide_rowptr)
 
 
@@ -167,11 +209,7 @@ def planted_community_graph(n_clusters: int, cluster_size: int, intra_degree: fl
 
     target = float(n) * inter_degree
     if target > 0:
-        cdf = _power_law_cdf(n, gamma, target)
-        m = int(target // 2)
-        shuffle = rng.permutation(n).astype(np.int64)
-        a = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
-        b = shuffle[np.searchsorted(cdf, rng.random(m), side="right").clip(0, n - 1)]
+        a, b = _power_law_pairs(n, int(target // 2), gamma, target, seed)
         differ = group_id[a] != group_id[b]
         us.append(a[differ])
         vs.append(b[differ])
@@ -200,13 +238,22 @@ def two_class_block_graph(n: int, avg_degree: float, h: float, seed: int):
 
 
 def normal_features(n: int, F: int, seed: int, y: np.ndarray | None = None,
-                    n_classes: int = 0, shift: float = 0.0) -> np.ndarray:
-    """N(0,1) features; with ``shift`` a class-dependent mean shift*mu_y, mu_c ~ N(0,I)."""
+                    n_classes: int = 0, shift: float = 0.0, native: bool = False) -> np.ndarray:
+    """N(0,1) features; with ``shift`` a class-dependent mean shift*mu_y, mu_c ~ N(0,I).
+    ``native``: draw with the multi-threaded host library (the named workloads, whose feature
+    matrices have up to billions of elements) instead of numpy's generator (a different stream)."""
     rng = np.random.default_rng(seed)
-    X = rng.standard_normal((n, F), dtype=np.float32)
+    if not native:
+        X = rng.standard_normal((n, F), dtype=np.float32)
+        if shift != 0.0 and y is not None:
+            mu = rng.standard_normal((n_classes, F), dtype=np.float32)
+            X += np.float32(shift) * mu[y]
+        return X
+    X = np.empty((n, F), dtype=np.float32)
+    _native().rin_normal_f32(n * F, seed, _p(X))
     if shift != 0.0 and y is not None:
         mu = rng.standard_normal((n_classes, F), dtype=np.float32)
-        X += np.float32(shift) * mu[y]
+        _native().rin_add_rows_f32(n, F, _p(np.ascontiguousarray(y, dtype=np.int32)), _p(mu), shift, _p(X))
     return X
 
 
@@ -332,7 +379,7 @@ def medium(scale: float = 1.0) -> Workload:
     n = int(200_000 * scale)
     g = chung_lu_graph(n, 25.0, 2.1, SEED_GRAPH + 1)
     y = uniform_labels(n, 47, SEED_LABEL + 1)
-    X = normal_features(n, 128, SEED_FEAT + 1, y, 47, 0.5)
+    X = normal_features(n, 128, SEED_FEAT + 1, y, 47, 0.5, native=True)
     dims = (128, 256, 256, 47)
     return Workload("medium" if scale == 1.0 else f"medium_x{scale:g}", g, X, y, dims,
                     M=8, K=20, R=5, lr=0.01, partition_seed=SEED_PART + 1,
@@ -351,7 +398,7 @@ def supertma(scale: float = 1.0, width: int | None = None, M: int = 16,
     y = cluster_label[g.group_id].astype(np.int32)
     F = 100 if width is None else width
     hid = 256 if width is None else width
-    X = normal_features(g.n, F, SEED_FEAT + 2, y, 47, 0.5)
+    X = normal_features(g.n, F, SEED_FEAT + 2, y, 47, 0.5, native=True)
     dims = (F, hid, hid, 47)
     K, R = (10, 3) if width is None else (5, 1)
     name = "supertma" if width is None else f"sweep_w{width}_M{M}_{'super' if use_groups else 'node'}"
@@ -368,7 +415,7 @@ def large(scale: float = 1.0) -> Workload:
     n = int(25_000_000 * scale)
     g = chung_lu_graph(n, 52.0, 2.0, SEED_GRAPH + 3, wide_rowptr=True)
     y = rare_positive_labels(n, 0.01, SEED_LABEL + 3)
-    X = normal_features(n, 128, SEED_FEAT + 3)
+    X = normal_features(n, 128, SEED_FEAT + 3, native=True)
     dims = (128, 256, 2)
     return Workload("large" if scale == 1.0 else f"large_x{scale:g}", g, X, y, dims,
                     M=32, K=5, R=1, lr=0.01, partition_seed=SEED_PART + 3,
