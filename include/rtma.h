@@ -24,8 +24,10 @@
  *    cudaFree, which synchronise the device) only when a call needs more than
  *    any call before it.  Every call on a context uses that scratch, so calls on
  *    one context must be ordered: the same stream, or the earlier call's stream
- *    drained first (rtma_local_steps orders its own streams).  A context must not
- *    be used from two host threads at the same time.
+ *    drained first.  The one case the library orders itself: after a local-training
+ *    call that spread its trainers over several streams, the next call on the context
+ *    (on whatever stream) first waits, on the device, for all of those streams.  A
+ *    context must not be used from two host threads at the same time.
  *  - Node ids and column indices are int32; row offsets are int32 or int64 on
  *    input and int64 on output.  At most RTMA_MAX_PARTS trainers.
  */
@@ -68,6 +70,13 @@ const char* rtma_last_error(const rtma_ctx* ctx);
 int32_t rtma_check(rtma_ctx* ctx);
 /* Bytes of scratch currently held by the context.                                        */
 size_t rtma_workspace_bytes(const rtma_ctx* ctx);
+/* Caps the scratch arena at `bytes` (0 = no cap, the default): no later call grows it beyond
+ * that, and a call that cannot work inside it returns RTMA_ERR_WORKSPACE.  An arena that is
+ * already larger is kept but only its first `bytes` are used by rtma_local_steps, which then
+ * runs the trainers of a stream in successive waves, each wave re-using the same scratch; the
+ * results are bit for bit those of a single wave.  For hosts that share the GPU with other
+ * tenants of a fixed memory budget.  The paper has no counterpart.                          */
+int32_t rtma_set_workspace_limit(rtma_ctx* ctx, size_t bytes);
 
 /* ---- R1: partition function (Sec. 3.2.2, RandomTMA and SuperTMA) -----------------------
  * part_id[v] = h(seed XOR g(v)) mod M, where h is one step of the SplitMix64 generator and

@@ -166,13 +166,24 @@ def acts_layout(dims, n: int):
     return out, off
 
 
+def round_to_bf16(x: float) -> float:
+    f = lib().orc_round_to_bf16
+    f.restype = ctypes.c_double
+    return float(f(ctypes.c_double(x)))
+
+
 def forward_backward(dims, rowptr, col, X, y, params, want_grads=True, want_acts=False, want_preact=False,
-                     gates=None):
+                     gates=None, bf16_operands=False):
     """Returns (loss, grads or None, {name: array} or None) for one part.
+    bf16_operands: the reduced-precision mode (operands of every dense product rounded to bf16; fp64 only).
     want_preact adds the hidden pre-activations as "Z1".."Z{L-1}" to the dict.
     gates: None, or a list of int8 arrays [n, d_{l+1}] for l = 0..L-2 (-1 natural, 0 closed,
     1 open) overriding the ReLU branch of individual units."""
     tag, ptr, dt = _fp(params.dtype)
+    if bf16_operands:
+        assert dt == np.float64
+        tag = "bf16ops_f64"
+        lib().orc_forward_backward_bf16ops_f64.restype = ctypes.c_double
     X = np.ascontiguousarray(X, dtype=dt)
     params = np.ascontiguousarray(params, dtype=dt)
     rowptr = _i64(rowptr)
@@ -210,9 +221,12 @@ def forward_backward(dims, rowptr, col, X, y, params, want_grads=True, want_acts
     return float(loss), grads, named
 
 
-def local_steps(dims, lr, rowptr, col, X, y, params, K):
+def local_steps(dims, lr, rowptr, col, X, y, params, K, bf16_operands=False):
     """K plain-SGD steps on one part.  Returns (new params, loss[K])."""
     tag, ptr, dt = _fp(params.dtype)
+    if bf16_operands:
+        assert dt == np.float64
+        tag = "bf16ops_f64"
     X = np.ascontiguousarray(X, dtype=dt)
     params = np.array(params, dtype=dt, copy=True)
     rowptr = _i64(rowptr)

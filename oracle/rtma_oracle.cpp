@@ -96,7 +96,29 @@ void spmm_mean(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, 
     }
 }
 
+// bf16 = the upper 16 bits of an IEEE binary32 number.  Round to nearest, ties to even, from the
+// binary32 value of x (the conversion the tensor cores' operands go through); finite inputs.
+inline double round_to_bf16(double x) {
+    const float f = (float)x;
+    uint32_t u;
+    std::memcpy(&u, &f, sizeof(u));
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    float r;
+    std::memcpy(&r, &u, sizeof(r));
+    return (double)r;
+}
+
 // One forward + backward pass over one part.  Returns the loss.
+// bf16_operands: the reduced-precision mode "GEMM inputs bf16 with fp32 accumulate".  Every operand
+// of a dense product -- H, A-bar H, the weight matrices, dZ (also under the bias gradient, the
+// product of a column of ones with dZ) -- is rounded to bf16 where it enters the product; sums,
+// aggregation, loss and update are unchanged.  Rounding does not commute with the aggregation, so
+// in this mode the gradient with respect to a layer's input is evaluated in the association
+// dH = [dZ | A-bar^T dZ] [Ws^T ; Wn^T] (aggregate, then multiply), whose second operand A-bar^T dZ
+// is rounded like any other; without the switch it is dZ Ws^T + A-bar^T (dZ Wn^T).  The two are
+// the same function in exact arithmetic.  The switch separates rounding from mistakes when a
+// bf16 implementation is compared; the plain mode remains the definition.
 // acts (optional): for l = 0..L-1: N^l [n x d_l] then H^{l+1} [n x d_{l+1}]
 // (post-ReLU for hidden layers, the logits for the last layer).
 // preact (optional): the hidden pre-activations Z^l, l = 0..L-2, [n x d_{l+1}] each.
@@ -107,7 +129,9 @@ void spmm_mean(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t d, 
 template <class T>
 double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
                         const int32_t* col, const T* X, const int32_t* y, const T* params,
-                        T* grads, T* acts, T* preact = nullptr, const int8_t* gates = nullptr) {
+                        T* grads, T* acts, T* preact = nullptr, const int8_t* gates = nullptr,
+                        bool bf16_operands = false) {
+    auto op = [bf16_operands](double x) { return bf16_operands ? round_to_bf16(x) : x; };
     const std::vector<LayerView> lv = layer_views(L, dims);
     const int64_t P = total_params(L, dims);
     if (grads) for (int64_t i = 0; i < P; ++i) grads[i] = (T)0;
@@ -128,15 +152,17 @@ double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t
         const T* Ws = params + lv[l].w_self;
         const T* Wn = params + lv[l].w_neigh;
         const T* b = params + lv[l].bias;
-        std::vector<double> acc(dn);
+        std::vector<double> acc(dn), ws_op(di * dn), wn_op(di * dn);  // the weights as they enter the product
+        for (int64_t i = 0; i < di * dn; ++i) ws_op[i] = op((double)Ws[i]);
+        for (int64_t i = 0; i < di * dn; ++i) wn_op[i] = op((double)Wn[i]);
         for (int64_t v = 0; v < n; ++v) {
             for (int64_t j = 0; j < dn; ++j) acc[j] = (double)b[j];
             for (int64_t k = 0; k < di; ++k) {
-                const double hs = (double)H[l][v * di + k];
-                const double hn = (double)N[l][v * di + k];
-                const T* ws = Ws + k * dn;
-                const T* wn = Wn + k * dn;
-                for (int64_t j = 0; j < dn; ++j) acc[j] += hs * (double)ws[j] + hn * (double)wn[j];
+                const double hs = op((double)H[l][v * di + k]);
+                const double hn = op((double)N[l][v * di + k]);
+                const double* ws = &ws_op[k * dn];
+                const double* wn = &wn_op[k * dn];
+                for (int64_t j = 0; j < dn; ++j) acc[j] += hs * ws[j] + hn * wn[j];
             }
             for (int64_t j = 0; j < dn; ++j) {
                 const T z = (T)acc[j];
@@ -190,18 +216,18 @@ double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t
         const T* Ws = params + lv[l].w_self;
         const T* Wn = params + lv[l].w_neigh;
         {   // dWs = H^T dZ, dWn = N^T dZ, db = column sums of dZ
-            std::vector<double> gs(di * dn, 0.0), gn(di * dn, 0.0), gb(dn, 0.0);
+            std::vector<double> gs(di * dn, 0.0), gn(di * dn, 0.0), gb(dn, 0.0), dz(dn);
             for (int64_t v = 0; v < n; ++v) {
-                const T* dz = &dZ[v * dn];
-                for (int64_t j = 0; j < dn; ++j) gb[j] += (double)dz[j];
+                for (int64_t j = 0; j < dn; ++j) dz[j] = op((double)dZ[v * dn + j]);
+                for (int64_t j = 0; j < dn; ++j) gb[j] += dz[j];
                 for (int64_t k = 0; k < di; ++k) {
-                    const double hs = (double)H[l][v * di + k];
-                    const double hn = (double)N[l][v * di + k];
+                    const double hs = op((double)H[l][v * di + k]);
+                    const double hn = op((double)N[l][v * di + k]);
                     double* rs = &gs[k * dn];
                     double* rn = &gn[k * dn];
                     for (int64_t j = 0; j < dn; ++j) {
-                        rs[j] += hs * (double)dz[j];
-                        rn[j] += hn * (double)dz[j];
+                        rs[j] += hs * dz[j];
+                        rn[j] += hn * dz[j];
                     }
                 }
             }
@@ -213,7 +239,28 @@ double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t
         // dH = dZ Ws^T + A-bar^T (dZ Wn^T);  dZ_prev = dH where Z_prev > 0
         std::vector<double> dH(n * di, 0.0);
         std::vector<double> dN(di);
-        for (int64_t v = 0; v < n; ++v) {
+        if (bf16_operands) {
+            // the same dH as [dZ | Q] [Ws^T ; Wn^T] with Q = A-bar^T dZ stored as T, every operand rounded
+            std::vector<double> Q(n * dn, 0.0);
+            for (int64_t v = 0; v < n; ++v) {
+                const int64_t deg = rowptr[v + 1] - rowptr[v];
+                for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e)
+                    for (int64_t j = 0; j < dn; ++j) Q[(int64_t)col[e] * dn + j] += (double)dZ[v * dn + j] / (double)deg;
+            }
+            std::vector<double> ws_op(di * dn), wn_op(di * dn), dz(dn), q(dn);
+            for (int64_t i = 0; i < di * dn; ++i) ws_op[i] = op((double)Ws[i]);
+            for (int64_t i = 0; i < di * dn; ++i) wn_op[i] = op((double)Wn[i]);
+            for (int64_t v = 0; v < n; ++v) {
+                for (int64_t j = 0; j < dn; ++j) dz[j] = op((double)dZ[v * dn + j]);
+                for (int64_t j = 0; j < dn; ++j) q[j] = op((double)(T)Q[v * dn + j]);
+                for (int64_t k = 0; k < di; ++k) {
+                    double s = 0.0;
+                    for (int64_t j = 0; j < dn; ++j) s += dz[j] * ws_op[k * dn + j] + q[j] * wn_op[k * dn + j];
+                    dH[v * di + k] = s;
+                }
+            }
+        }
+        for (int64_t v = 0; v < n && !bf16_operands; ++v) {
             const T* dz = &dZ[v * dn];
             for (int64_t k = 0; k < di; ++k) {
                 double s = 0.0, t = 0.0;
@@ -241,11 +288,12 @@ double forward_backward(int32_t L, const int32_t* dims, int64_t n, const int64_t
 template <class T>
 void local_steps(int32_t L, const int32_t* dims, double lr, int64_t n, const int64_t* rowptr,
                  const int32_t* col, const T* X, const int32_t* y, T* params, int32_t K,
-                 double* loss_out) {
+                 double* loss_out, bool bf16_operands = false) {
     const int64_t P = total_params(L, dims);
     std::vector<T> g(P);
     for (int32_t k = 0; k < K; ++k) {
-        const double loss = forward_backward<T>(L, dims, n, rowptr, col, X, y, params, g.data(), nullptr);
+        const double loss = forward_backward<T>(L, dims, n, rowptr, col, X, y, params, g.data(), nullptr, nullptr, nullptr,
+                                                bf16_operands);
         if (loss_out) loss_out[k] = loss;
         for (int64_t i = 0; i < P; ++i) params[i] = (T)((double)params[i] - lr * (double)g[i]);
     }
@@ -1020,6 +1068,20 @@ void orc_local_steps_f64(int32_t L, const int32_t* dims, double lr, int64_t n, c
                          int32_t K, double* loss_out) {
     local_steps<double>(L, dims, lr, n, rowptr, col, X, y, params, K, loss_out);
 }
+
+// The same two routines in the reduced-precision mode (operands of every dense product rounded to bf16).
+double orc_forward_backward_bf16ops_f64(int32_t L, const int32_t* dims, int64_t n, const int64_t* rowptr,
+                                        const int32_t* col, const double* X, const int32_t* y,
+                                        const double* params, double* grads, double* acts, double* preact,
+                                        const int8_t* gates) {
+    return forward_backward<double>(L, dims, n, rowptr, col, X, y, params, grads, acts, preact, gates, true);
+}
+void orc_local_steps_bf16ops_f64(int32_t L, const int32_t* dims, double lr, int64_t n, const int64_t* rowptr,
+                                 const int32_t* col, const double* X, const int32_t* y, double* params,
+                                 int32_t K, double* loss_out) {
+    local_steps<double>(L, dims, lr, n, rowptr, col, X, y, params, K, loss_out, true);
+}
+double orc_round_to_bf16(double x) { return round_to_bf16(x); }
 
 void orc_average_f32(float* params, int64_t P, int32_t M, float* global_out) { average<float>(params, P, M, global_out); }
 void orc_average_f64(double* params, int64_t P, int32_t M, double* global_out) { average<double>(params, P, M, global_out); }

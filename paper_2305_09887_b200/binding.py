@@ -23,7 +23,7 @@ EXPORTS = (
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
     "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout", "rtma_link_param_count",
-    "rtma_link_steps",
+    "rtma_link_steps", "rtma_set_workspace_limit",
 )
 KERNEL_CLASSES = 21
 
@@ -187,6 +187,10 @@ class Context:
     @property
     def workspace_bytes(self) -> int:
         return int(self._lib.rtma_workspace_bytes(self._h))
+
+    def set_workspace_limit(self, nbytes: int):
+        """Caps the context's scratch arena (0 = no cap); rtma_local_steps then runs in waves."""
+        self._check(self._lib.rtma_set_workspace_limit(self._h, ctypes.c_size_t(nbytes)), "rtma_set_workspace_limit")
 
     def check(self):
         """Synchronises and raises if a kernel gave up on a bounded device-side wait."""

@@ -33,6 +33,10 @@ struct rtma_ctx {
     std::vector<cudaEvent_t> event_pool;  // spare events
     char* arena = nullptr;        // device scratch
     size_t arena_bytes = 0;
+    size_t arena_limit = 0;       // 0: none; else the arena never grows beyond this many bytes
+    // the streams of the last local-training call and an event recorded at the end of each
+    std::vector<cudaStream_t> trained_streams;
+    std::vector<cudaEvent_t> trained_events;
     void* pinned = nullptr;       // small pinned staging block for descriptors
     size_t pinned_bytes = 0;
     char error[512] = {0};
@@ -100,6 +104,12 @@ struct KernelScope {
 
 // Makes the arena at least `bytes` large.  Growing synchronises the device.
 int32_t rtma_reserve(rtma_ctx* ctx, size_t bytes);
+
+// Ordering between calls on one context.  A local-training call may spread its work over several
+// streams; order_after_training makes `s` wait for all of them (a no-op for the streams' own
+// later work), mark_trained records the end of such a call on its streams.
+int32_t order_after_training(rtma_ctx* ctx, cudaStream_t s);
+int32_t mark_trained(rtma_ctx* ctx, const std::vector<cudaStream_t>& streams);
 
 // Bump allocator over the arena (256-byte granules).
 struct ArenaCursor {

@@ -25,6 +25,7 @@ extern "C" int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_
     if (workspace_bytes) {
         int32_t s = rtma_reserve(ctx, workspace_bytes);
         if (s != RTMA_OK) {
+            cudaFree(ctx->error_word);
             cudaFreeHost(ctx->pinned);
             delete ctx;
             return s;
@@ -46,6 +47,7 @@ extern "C" int32_t rtma_destroy(rtma_ctx* ctx) {
         cudaEventDestroy(sp.stop);
     }
     for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->trained_events) cudaEventDestroy(e);
     delete ctx;
     return RTMA_OK;
 }
@@ -102,8 +104,34 @@ extern "C" int32_t rtma_profile_read(rtma_ctx* ctx, double* ms, int64_t* launche
     return RTMA_OK;
 }
 
+extern "C" int32_t rtma_set_workspace_limit(rtma_ctx* ctx, size_t bytes) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    ctx->arena_limit = bytes;
+    return RTMA_OK;
+}
+
+int32_t order_after_training(rtma_ctx* ctx, cudaStream_t s) {
+    for (size_t i = 0; i < ctx->trained_streams.size(); ++i)
+        if (ctx->trained_streams[i] != s) RTMA_CUDA(ctx, cudaStreamWaitEvent(s, ctx->trained_events[i], 0));
+    return RTMA_OK;
+}
+
+int32_t mark_trained(rtma_ctx* ctx, const std::vector<cudaStream_t>& streams) {
+    while (ctx->trained_events.size() < streams.size()) {
+        cudaEvent_t e = nullptr;
+        RTMA_CUDA(ctx, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        ctx->trained_events.push_back(e);
+    }
+    ctx->trained_streams = streams;
+    for (size_t i = 0; i < streams.size(); ++i) RTMA_CUDA(ctx, cudaEventRecord(ctx->trained_events[i], streams[i]));
+    return RTMA_OK;
+}
+
 int32_t rtma_reserve(rtma_ctx* ctx, size_t bytes) {
     if (bytes <= ctx->arena_bytes) return RTMA_OK;
+    if (ctx->arena_limit && bytes > ctx->arena_limit)
+        return rtma_fail(ctx, RTMA_ERR_WORKSPACE, "%zu bytes of scratch needed, the limit set on this context is %zu", bytes,
+                         ctx->arena_limit);
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
     RTMA_CUDA(ctx, cudaDeviceSynchronize());
     if (ctx->arena) {

@@ -138,6 +138,7 @@ extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowp
         return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_build_induced_csr: null pointer");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_TRY(order_after_training(ctx, stream));
     const unsigned row_blocks = (unsigned)ceil_div(n, CSR_WARPS);
 
     if (col_out) {  // FILL
@@ -191,6 +192,7 @@ extern "C" int32_t rtma_gather_rows(rtma_ctx* ctx, int64_t n, int64_t row_bytes,
     if (!src || !perm || !dst) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_gather_rows: null pointer");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_TRY(order_after_training(ctx, stream));
     const unsigned blocks = (unsigned)ceil_div(n, 8);
     const uintptr_t align = reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst) | (uintptr_t)row_bytes;
     if (align % 16 == 0)

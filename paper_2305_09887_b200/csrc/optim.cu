@@ -97,6 +97,7 @@ int32_t aggregate_impl(rtma_ctx* ctx, float* params, const float* grads, float l
     if (!params) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "aggregate: null params");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_TRY(order_after_training(ctx, stream));
     const bool vec = P % 4 == 0 && reinterpret_cast<uintptr_t>(params) % 16 == 0 &&
                      (!grads || reinterpret_cast<uintptr_t>(grads) % 16 == 0) &&
                      (!global_out || reinterpret_cast<uintptr_t>(global_out) % 16 == 0);

@@ -100,6 +100,7 @@ extern "C" int32_t rtma_partition(rtma_ctx* ctx, int64_t n, const int32_t* group
         return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_partition: null output pointer");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_TRY(order_after_training(ctx, stream));
     if (n == 0) {
         RTMA_CUDA(ctx, cudaMemsetAsync(part_offsets, 0, sizeof(int64_t) * (M + 1), stream));
         return RTMA_OK;
@@ -195,6 +196,7 @@ extern "C" int32_t rtma_partition_grouped(rtma_ctx* ctx, int64_t n, const int32_
         return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_partition_grouped: null output pointer");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
+    RTMA_TRY(order_after_training(ctx, stream));
     if (n == 0) {
         RTMA_CUDA(ctx, cudaMemsetAsync(part_offsets, 0, sizeof(int64_t) * (M + 1), stream));
         return RTMA_OK;

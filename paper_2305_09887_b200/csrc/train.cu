@@ -144,11 +144,14 @@ int splits_for(int64_t n_p, int parts_in_flight) {
     return (int)std::min<int64_t>(64, std::min(want, by_rows));
 }
 
-int plan_splits(const GroupDesc& g, SplitPlan* sp) {
+// parts_in_flight: all trainers that run in this call, whatever their stream and wave, so that a
+// part's chunking (hence the order of its gradient sums) does not depend on how the trainers were
+// spread over streams or cut into waves
+int plan_splits(const GroupDesc& g, int parts_in_flight, SplitPlan* sp) {
     int slots = 0;
     for (int k = 0; k < g.num; ++k) {
         sp->split_begin[k] = slots;
-        const int nsplit = splits_for(g.rows[k], g.num);
+        const int nsplit = splits_for(g.rows[k], parts_in_flight);
         sp->rows_per_split[k] = (int32_t)std::max<int64_t>(GROUP_ROW_ALIGN, aligned_rows(ceil_div(g.rows[k], nsplit)));
         slots += (int)std::max<int64_t>(1, ceil_div(g.rows[k], sp->rows_per_split[k]));
     }
@@ -250,6 +253,11 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
         group_parts[gi].push_back(p);
     }
     const size_t G = group_stream.size();
+    int running = 0;
+    for (const std::vector<int>& parts : group_parts) running += (int)parts.size();
+    // this call's streams start after everything an earlier training call left running on other
+    // streams: the scratch shares below may be handed to different streams than last time
+    for (cudaStream_t s : group_stream) RTMA_TRY(order_after_training(ctx, s));
 
     // Scratch: every group owns an equal share of the arena; inside a share, parts run in
     // waves that fit.  Ask for enough to run every group in one wave when memory allows.
@@ -267,10 +275,11 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
     }
     want_share = ArenaCursor::granule(want_share);
     min_share = ArenaCursor::granule(min_share);
-    if (ctx->arena_bytes < want_share * G) {
+    const size_t cap = ctx->arena_limit ? ctx->arena_limit : ~size_t(0);
+    if (std::min(ctx->arena_bytes, cap) < want_share * G) {
         size_t free_b = 0, total_b = 0;
         RTMA_CUDA(ctx, cudaMemGetInfo(&free_b, &total_b));
-        const size_t reachable = ctx->arena_bytes + (size_t)((double)free_b * 0.9);
+        const size_t reachable = std::min(cap, ctx->arena_bytes + (size_t)((double)free_b * 0.9));
         size_t target = std::min(want_share * G, reachable);
         if (target < min_share * G)
             return rtma_fail(ctx, RTMA_ERR_WORKSPACE,
@@ -278,7 +287,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                              min_share, G, reachable);
         if (target > ctx->arena_bytes) RTMA_TRY(rtma_reserve(ctx, target));
     }
-    const size_t share = (ctx->arena_bytes / G) / 256 * 256;
+    const size_t share = (std::min(ctx->arena_bytes, cap) / G) / 256 * 256;
     if (share < min_share)
         return rtma_fail(ctx, RTMA_ERR_WORKSPACE, "scratch share %zu < %zu needed by the largest part", share, min_share);
 
@@ -316,7 +325,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 bytes += b;
                 ++at;
             }
-            const int slots = plan_splits(g, &sp);
+            const int slots = plan_splits(g, running, &sp);
             int wave_steps = 0;
             for (int k = 0; k < g.num; ++k) wave_steps = std::max(wave_steps, steps[g.part[k]]);
 
@@ -367,7 +376,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                     El[k] = take_pair_planes(m.ddims[k]);
                     ZDl[k] = take_pair_planes(m.ddims[k + 1]);
                 }
-                const int dslots = plan_splits(gd, &spd);
+                const int dslots = plan_splits(gd, running, &spd);
                 dec_partial = cur.take<float>((size_t)dslots * plan.max_layer_params + 4);
                 dec_tile_loss = cur.take<float>((size_t)loss_tiles(gd) + 4);
             }
@@ -550,7 +559,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             }
         }
     }
-    return RTMA_OK;
+    return mark_trained(ctx, group_stream);
 }
 
 }  // namespace

@@ -8,6 +8,11 @@ from paper_2305_09887_b200 import binding, inputs
 # relative = max|a-b| / max|b| per tensor
 TOL_ACT, TOL_GRAD, TOL_PARAM = 1e-4, 1e-3, 1e-3
 TOL_BF16 = 5e-3
+# bf16 operand mode against the oracle's own bf16 operand mode (same roundings, fp64 sums): what is
+# left is the kernel's fp32 accumulation and the few operands that round the other way
+TOL_BF16_SAME_ROUNDING = 5e-4
+# branch flips seen per check (part, flipped units, hidden units), for the test log
+FLIP_LOG = []
 
 _ctx = None
 
@@ -107,10 +112,14 @@ def _param_segments(variant, dims):
     return out
 
 
-def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, variant=(0, 0, 0), params0=None):
+def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, variant=(0, 0, 0), params0=None,
+                   gradients_against_plain=True):
     """Partition + induced CSR against the oracle (bit-exact), then step 0 of all M trainers
     batched as one call: every recorded intermediate, the loss, the gradient and the updated
-    parameters of every part (or of the parts in only_parts) against the oracle."""
+    parameters of every part (or of the parts in only_parts) against the oracle.  In bf16 operand
+    mode the step is also held, tightly, to the oracle run with the same operand roundings;
+    gradients_against_plain=False leaves the gradient comparison to that one (shapes outside the
+    named bf16 workload, where the 5e-3 bar against the unrounded oracle is not claimed)."""
     tol_act, tol_grad, tol_param, tol_loss, amb, flip_frac = tols(gemm_dtype)
     c = ctx()
     got = gpu_preprocess(w, M=M)
@@ -159,11 +168,18 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, varia
             g8 = np.full(Z.shape, -1, dtype=np.int8)
             g8[differ] = (gpu_acts[f"H{l + 1}"] > 0)[differ]
             gates.append(g8)
+        FLIP_LOG.append((w.name, gemm_dtype, p, flipped, units))
+        print(f"[relu branch] {w.name} mode {gemm_dtype} part {p}: {flipped} of {units} hidden units took the other branch")
         assert flipped <= 8 + flip_frac * units
         if flipped:
             o_loss, o_grads, _ = oracle.forward_backward_variant(variant, dims, rp, cp, X, y, p0, gates=gates)
+        if gemm_dtype == 1 and variant == (0, 0, 0):
+            same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, loss[p, 0], grads[p])
         if n_p:
             assert abs(loss[p, 0] - o_loss) <= tol_loss * max(1.0, abs(o_loss)), p
+        if not gradients_against_plain:
+            assert gemm_dtype == 1 and variant == (0, 0, 0)
+            continue
         # gradients: per parameter tensor
         for nm, off, size in _param_segments(variant, dims):
             gg, og = grads[p, off:off + size], o_grads[off:off + size]
@@ -176,6 +192,39 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, varia
                 assert np.abs(gg).max() == 0
         assert rel_err(params1[p], p0 - w.lr * o_grads) <= tol_param
     return got, want
+
+
+def same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, gpu_loss, gpu_grads):
+    """bf16 operand mode against the oracle run with the same operand roundings: separates the
+    rounding the mode is allowed (2^-9 per operand, the 5e-3 bar) from anything else."""
+    dims = w.dims
+    tol = TOL_BF16_SAME_ROUNDING
+    r_loss, r_grads, r_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True, want_preact=True,
+                                                      bf16_operands=True)
+    worst = 0.0
+    for name, a in gpu_acts.items():
+        e = rel_err(a, r_acts[name])
+        worst = max(worst, e)
+        assert e <= tol, (p, name, e)
+    gates, flipped = [], 0
+    for l in range(len(dims) - 2):
+        Z = r_acts[f"Z{l + 1}"]
+        differ = (np.abs(Z) < 1e-4 * max(1.0, np.abs(Z).max(initial=0.0))) & ((gpu_acts[f"H{l + 1}"] > 0) != (Z > 0))
+        flipped += int(differ.sum())
+        g8 = np.full(Z.shape, -1, dtype=np.int8)
+        g8[differ] = (gpu_acts[f"H{l + 1}"] > 0)[differ]
+        gates.append(g8)
+    if flipped:
+        r_loss, r_grads, _ = oracle.forward_backward(dims, rp, cp, X, y, p0, gates=gates, bf16_operands=True)
+    if rp.size > 1:
+        assert abs(gpu_loss - r_loss) <= tol * max(1.0, abs(r_loss)), p
+    worst_g = 0.0
+    for nm, off, size in _param_segments((0, 0, 0), dims):
+        if np.abs(r_grads[off:off + size]).max() > 0:
+            e = rel_err(gpu_grads[off:off + size], r_grads[off:off + size])
+            worst_g = max(worst_g, e)
+            assert e <= tol, (p, nm, e)
+    print(f"[same rounding] {w.name} part {p}: activations {worst:.2e}, gradients {worst_g:.2e}, {flipped} branch flips")
 
 
 def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_parts=None, variant=(0, 0, 0),
