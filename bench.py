@@ -3,13 +3,15 @@
 
 One step = one pass of the whole path over the workload: broadcast of the initial weights,
 partition, induced CSR (count + fill), row gather, then R x (K local steps on all M parts +
-aggregation).  The default workload is Medium (Chung-Lu power-law graph, 200k nodes, ~5M
-directed entries, 128-d features, 47 classes, M=8 trainers, 128-256-256-47 GraphSAGE-mean,
-20 local steps per round, 5 aggregation rounds).  --workload selects the other shapes:
-supertma (planted communities, super-node assignment, M=16), sweep (the same graph at width
-512 with bf16 GEMM operands; --M and --assign pick the point of the sweep) and large
-(--scale shrinks it; the full size needs ~60 GB of host memory to generate); averaging times
-the aggregation kernel alone on a shape large enough to be bound by HBM.
+aggregation).  The default workload is Large, the largest of the named shapes that one GPU
+holds (Chung-Lu power-law graph, 25M nodes, ~1.3B directed entries with 64-bit row offsets,
+128-d features, 2 classes with 1% positives, M=32 trainers, 128-256-2 GraphSAGE-mean, 5 local
+steps, one aggregation; about 35 GB of host memory and a minute of 16 host threads to
+generate).  --workload selects the other shapes: medium (200k nodes, ~5M entries, M=8,
+128-256-256-47, 20 steps x 5 rounds), supertma (planted communities, super-node assignment,
+M=16), sweep (the same graph at width 512 with bf16 GEMM operands; --M and --assign pick the
+point of the sweep); --scale shrinks any of them; averaging times the aggregation kernel
+alone on a shape large enough to be bound by HBM.
 
 Metric: aggregated edges/s = (sum over parts of kept entries) x (aggregations a local step is
 made of: L forward + L-1 backward) x (local steps) / time.  Local trainer-steps/s is reported
@@ -18,7 +20,7 @@ rtma_local_steps call instead of once per step; the unit still counts it per ste
 method defines it, and `edges_gathered_per_s` gives the rate of the gathers actually executed.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--workload medium|supertma|sweep|large] [--scale S] [--M M] [--assign node|super]
+                    [--workload large|medium|supertma|sweep|averaging] [--scale S] [--M M] [--assign node|super]
 
 Prints one JSON line (rank 0).
 """
@@ -41,6 +43,7 @@ if ROOT not in sys.path:
 
 METRIC = "aggregated_edges_per_s"
 UNIT = "edges/s"
+NOMINAL_HBM_GBS = 8000.0   # the figure the bandwidth targets are quoted on; fractions are given against both
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -60,13 +63,28 @@ def load_peaks():
 # ---------------------------------------------------------------------------------------
 # workload arithmetic (algorithmic work per kernel class for one bench step)
 # ---------------------------------------------------------------------------------------
-def algorithmic_work(dims, n_parts, e_parts, K, R):
+def algorithmic_work(dims, n_parts, e_parts, K, R, entries=0, rowptr_bytes=8, grouped=False):
     """Per kernel class: (bound, algorithmic bytes, algorithmic flops) summed over one bench
     step.  Bytes are compulsory traffic (every operand read once, every result written once)."""
     L = len(dims) - 1
     n, e = float(sum(n_parts)), float(sum(e_parts))
     steps = K * R
     work = {}
+    # preprocessing, once per bench step.  Partition: part_id, perm, local_id written (12 B per node; the
+    # super-node id read by each of its two passes); with super-nodes kept together, four radix passes
+    # of (order read, super-node id gathered) x 2 + order written
+    E = float(entries)
+    part_count = (4.0 * n if grouped else 0.0) + (4 * (8.0 * n) if grouped else 0.0)
+    part_scatter = 12.0 * n + (4.0 * n if grouped else 0.0) + (4 * (12.0 * n) if grouped else 0.0)
+    work["partition_count"] = ("hbm", part_count, 0.0)
+    work["partition_scatter"] = ("hbm", part_scatter, 0.0)
+    # induced subgraphs: per entry the column id and the part of its end point (count pass), the same
+    # again plus the end point's local id and the kept entry written (fill pass); per row its offsets,
+    # its node id and its part
+    work["induced_count"] = ("hbm", E * 8 + n * (2 * rowptr_bytes + 8 + 8), 0.0)
+    work["induced_fill"] = ("hbm", E * 8 + e * 8 + n * (2 * rowptr_bytes + 8 + 8), 0.0)
+    work["gather_rows"] = ("hbm", 2.0 * n * (4 * dims[0] + 4) + 8.0 * n, 0.0)
+    work["to_planes"] = ("hbm", R * 8.0 * n * dims[0], 0.0)
     # the aggregate of the input features is computed once per call (R times per bench step), not per step
     spmm_f = sum(n * 8 * dims[l] + 4 * e + 8 * n for l in range(1, L)) + (n * 8 * dims[0] + 4 * e + 8 * n) / K
     spmm_b = sum(n * 8 * dims[l + 1] + 4 * e + 12 * n for l in range(1, L))
@@ -164,40 +182,71 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------
 # CPU baseline: the checker program as it stands, on a bounded sample
 # ---------------------------------------------------------------------------------------
-def cpu_sample(w, local_steps=1):
-    """Times the CPU checker on a bounded sample of the workload: partition + induced CSR + row
-    gather of the whole graph, then `local_steps` local steps of trainer 0 only.  Returns the
-    whole-workload figure extrapolated from it (every other trainer-step costed like trainer 0's)."""
+def host_info():
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for ln in f:
+                if ln.lower().startswith("model name"):
+                    model = ln.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count(), "cpu_model": model}
+
+
+def cpu_sample(w, local_steps=1, flop_budget=1.2e10):
+    """Times the CPU checker, as it stands and on one core, on a bounded sample of the workload:
+    the assignment and relabelling of ALL nodes; the induced subgraph and the gathered feature /
+    label rows of trainer 0's part only; `local_steps` local steps on the first `slice_rows` rows
+    of that part (entries between those rows).  The whole-workload figure is extrapolated:
+    preprocessing as t_assign + M * t_part0, training by rows (the checker spends > 99 % of a step
+    in the per-row dense products)."""
     import oracle
     g = w.graph
     L = len(w.dims) - 1
     t0 = time.perf_counter()
     part_id, part_offsets, perm, local_id = oracle.partition(g.n, g.group_id if w.use_groups else None,
                                                              w.partition_seed, w.M, grouped=w.use_groups and w.grouped_order)
-    rowptr_out, col_out, edge_offsets, kept, cut = oracle.induced_csr(
-        g.rowptr, g.col, w.M, part_id, part_offsets, perm, local_id)
-    Xp = oracle.gather_rows(w.X, perm)
-    yp = oracle.gather_rows(w.y, perm)
-    t_pre = time.perf_counter() - t0
-    rp, cp = oracle.part_graph(rowptr_out, col_out, part_offsets, edge_offsets, 0)
-    hi = int(part_offsets[1])
+    t_assign = time.perf_counter() - t0
+    n0 = int(part_offsets[1])
+    t0 = time.perf_counter()
+    # trainer 0's part alone: the checker's routine with a single part whose members are perm[0:n0]
+    rowptr0, col0, _, kept0, _ = oracle.induced_csr(g.rowptr, g.col, 1, part_id, np.array([0, n0], dtype=np.int64),
+                                                    perm, local_id)
+    X0 = oracle.gather_rows(w.X, perm[:n0])
+    y0 = oracle.gather_rows(w.y, perm[:n0])
+    t_part0 = time.perf_counter() - t0
+    # rows whose step costs the checker about three seconds (6 flops per weight and row)
+    flops_per_row = 6.0 * sum((2 * w.dims[l] + 1) * w.dims[l + 1] for l in range(L))
+    S = min(n0, max(1024, int(flop_budget / flops_per_row)))
+    rp = rowptr0[:S + 1]
+    cols = col0[:int(rp[-1])]
+    inside = cols < S                                          # entries between the slice's rows
+    rows = np.repeat(np.arange(S), np.diff(rp))
+    srp = np.concatenate([[0], np.cumsum(np.bincount(rows[inside], minlength=S))]).astype(np.int64)
+    scol = np.ascontiguousarray(cols[inside])
     t1 = time.perf_counter()
-    oracle.local_steps_variant(w.variant, w.dims, w.lr, rp, cp, Xp[:hi], yp[:hi], w.params0, local_steps)
-    t_step = (time.perf_counter() - t1) / local_steps
+    oracle.local_steps_variant(w.variant, w.dims, w.lr, srp, scol, X0[:S], y0[:S], w.params0, local_steps)
+    t_slice = (time.perf_counter() - t1) / local_steps
+    # kept entries of the whole workload: expected value for the assignment in use, from part 0
+    kept_est = float(kept0) * g.n / max(n0, 1)
     passes = 2 * L - 1
-    units_full = float(kept) * passes * w.K * w.R
-    est_full_s = t_pre + w.K * w.R * w.M * t_step
-    return dict(value=units_full / est_full_s, t_pre_s=t_pre, t_step_s=t_step, sample_s=t_pre + t_step * local_steps,
-                trainer_steps_per_s=1.0 / t_step,
-                sample=(f"partition+induced CSR+row gather of all {g.n} nodes ({t_pre:.2f} s), then {local_steps} "
-                        f"local step(s) of trainer 0 ({hi} nodes, {cp.size} entries; {t_step:.2f} s/step); "
-                        f"whole workload extrapolated as t_pre + K*R*M*t_step"))
+    units_full = kept_est * passes * w.K * w.R
+    t_step_all_parts = t_slice * g.n / max(S, 1)               # one local step of every trainer
+    est_full_s = t_assign + w.M * t_part0 + w.K * w.R * t_step_all_parts
+    return dict(value=units_full / est_full_s, sample_s=t_assign + t_part0 + t_slice * local_steps,
+                trainer_steps_per_s=w.M / t_step_all_parts,
+                sample=(f"assignment+relabel of all {g.n} nodes ({t_assign:.2f} s); induced subgraph + row gather of "
+                        f"trainer 0's part ({n0} nodes, {kept0} kept entries; {t_part0:.2f} s); {local_steps} local "
+                        f"step(s) on its first {S} rows ({scol.size} entries; {t_slice:.2f} s/step); whole workload "
+                        f"extrapolated as t_assign + M*t_part0 + K*R*(n/{S})*t_slice"))
 
 
 def run_reference(args, w):
     """`--impl reference`: the CPU checker, single-threaded, timed on the host cores."""
     steps, warmup = args.steps, args.warmup
-    for _ in range(warmup):
+    for _ in range(min(warmup, 1)):     # the checker has no caches to warm beyond the first touch of its inputs
         cpu_sample(w)
     t0 = time.perf_counter()
     samples = [cpu_sample(w) for _ in range(steps)]
@@ -209,7 +258,8 @@ def run_reference(args, w):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "nodes": w.graph.n, "entries": w.graph.num_entries, "M": w.M,
                    "dims": list(w.dims), "K": w.K, "R": w.R, "timing": "host wall clock, bounded sample per step"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": samples[-1]["sample"]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": samples[-1]["sample"],
+                         "host": host_info()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "trainer_steps_per_s": statistics.mean(s["trainer_steps_per_s"] for s in samples),
         "gpu_launches": 0,
@@ -410,6 +460,34 @@ def run_link(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
+def kernel_sources_digest() -> str:
+    """Digest of the CUDA sources: ncu counters taken on other sources are not reported."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2305_09887_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()[:16]
+
+
+def load_dram_traffic():
+    """{(workload, kernel class): DRAM bytes per launch} from the ncu capture recorded in
+    profiles/dram_traffic.txt (lines: workload, class, bytes per launch, digest of the kernel
+    sources the capture ran on).  Entries taken on other sources than the present ones are dropped."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    out = {}
+    if not os.path.exists(path):
+        return out
+    digest = kernel_sources_digest()
+    with open(path) as f:
+        for ln in f:
+            parts = ln.split()
+            if len(parts) == 4 and not ln.startswith("#") and parts[3] == digest:
+                out[(parts[0], parts[1])] = float(parts[2])
+    return out
+
+
 def max_over_ranks(seconds: float, dist_mod=None, device=None) -> float:
     """Largest value over all ranks (the slowest rank sets the job's time)."""
     if dist_mod is None or not dist_mod.is_initialized() or dist_mod.get_world_size() == 1:
@@ -427,7 +505,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="medium", choices=["medium", "supertma", "sweep", "large", "averaging"])
+    ap.add_argument("--workload", default="large", choices=["large", "medium", "supertma", "sweep", "averaging"])
+    ap.add_argument("--profile-steps", type=int, default=1,
+                    help="steps of the separate pass that times every kernel class (CUDA events round each launch)")
     ap.add_argument("--scale", type=float, default=None, help="shrink (or grow) the workload's graph")
     ap.add_argument("--M", type=int, default=None, help="trainers (supertma / sweep)")
     ap.add_argument("--assign", default="super", choices=["node", "super"], help="sweep: assignment scheme")
@@ -511,9 +591,10 @@ def main():
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
+    ctx.check()
     ctx.profile_read()
 
-    ctx.profile(True)
+    # ---- the timed region: K steps, no per-launch instrumentation ------------------------
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     if world > 1:
@@ -529,11 +610,23 @@ def main():
     sampler.end()
     if world > 1:
         dist.barrier()
-    ctx.profile(False)
-    prof = ctx.profile_read()
+    ctx.check()                          # a kernel that gave up on a bounded wait voids the run
+    _, launch_counts = zip(*ctx.profile_read().values())
+    gpu_launches = int(sum(launch_counts))
     clocks = sampler.stop()
     elapsed_s = sum(a.elapsed_time(b) for a, b in zip(starts, stops)) / 1e3
     elapsed_s = max_over_ranks(elapsed_s, dist if world > 1 else None, device)
+
+    # ---- a separate pass with CUDA events round every launch: time per kernel class ---------
+    prof_steps = max(1, args.profile_steps)
+    ctx.profile(True)
+    for i in range(prof_steps):
+        flush.fill_(i & 0xFF)
+        step()
+    torch.cuda.synchronize()
+    ctx.profile(False)
+    ctx.check()
+    prof = ctx.profile_read()
 
     n_parts = np.diff(state["part_host"]).tolist()
     e_parts = np.diff(state["edge_host"]).tolist()
@@ -545,58 +638,76 @@ def main():
     final_loss = loss[-1, :, -1].mean().item()
     first_loss = loss[0, :, 0].mean().item()
 
-    # ---- roofline of the dominant kernel class --------------------------------------
+    # ---- roofline of the dominant kernel class, and of the aggregation (SpMM) classes ------
     peaks = load_peaks()
-    work = algorithmic_work(w.dims, n_parts, e_parts, w.K, w.R) if w.variant == (0, 0, 0) else {}
+    work = (algorithmic_work(w.dims, n_parts, e_parts, w.K, w.R, entries=g.num_entries, rowptr_bytes=g.rowptr.itemsize,
+                             grouped=w.use_groups and w.grouped_order) if w.variant == (0, 0, 0) else {})
     total_kernel_ms = sum(ms for ms, _ in prof.values())
     shares = {k: ms / total_kernel_ms for k, (ms, _) in prof.items() if ms > 0}
     top = max(shares, key=shares.get)
-    top_ms, top_launches = prof[top]
     # A layer product is three bf16 MMAs (hi*hi + lo*hi + hi*lo): the tensor pipe executes 3x the
     # algorithmic flops.  Its roofline is whichever is slower for the algorithmic work: the operand
     # bytes at the HBM peak or 3x the flops at the bf16 peak (sustained figure: timed inside a long step).
     MMAS_PER_PRODUCT = 1 if w.gemm_dtype == 1 else 3
-    if top in work:
-        bound, abytes, aflops = work[top]
-        seconds = top_ms / 1e3
-        if bound == "gemm":
-            t_hbm = abytes / (peaks["hbm_gbs"] * 1e9)
-            t_tensor = MMAS_PER_PRODUCT * aflops / (peaks["bf16_tflops_sustained"] * 1e12)
-            bound = "hbm" if t_hbm >= t_tensor else "tensor"
-        if bound == "hbm":
-            roof = {"bound": "hbm", "achieved": abytes * args.steps / seconds / 1e9, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s"}
-        else:
-            roof = {"bound": "tensor", "achieved": aflops * args.steps / seconds / 1e12,
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "note": f"algorithmic flops; the tensor pipe executes {MMAS_PER_PRODUCT} bf16 MMA(s) per product"}
-    else:
+    traffic_table = load_dram_traffic()
+
+    def roofline_of(cls):
+        ms, launches = prof[cls]
         roof = {"bound": "hbm", "achieved": None, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    # DRAM bytes per launch of the class (dram__bytes_read.sum + dram__bytes_write.sum averaged over the class's
-    # launches of one local step) from ncu captures of these kernels on this workload (summaries under
-    # profiles/);
-    # only for the workload and model that capture ran on
-    traffic = None
-    if w.name == "medium" and w.variant == (0, 0, 0) and w.gemm_dtype == 0:
-        traffic = {"gemm_forward": 463.9e6, "gemm_dgrad": 505.6e6, "gemm_wgrad": 502.9e6,
-                   "spmm_forward": 340.0e6, "spmm_backward": 194.0e6}.get(top)
-    roof.update({"frac": (roof["achieved"] / roof["peak"]) if roof["achieved"] else None, "traffic": traffic,
-                 "kernel": top, "launches_per_step": top_launches / args.steps,
-                 "avg_launch_us": 1e3 * top_ms / max(top_launches, 1), "share_of_kernel_time": shares[top],
-                 "peak_source": peaks["source"]})
+        if cls in work and ms > 0:
+            bound, abytes, aflops = work[cls]
+            seconds = ms / 1e3
+            if bound == "gemm":
+                t_hbm = abytes / (peaks["hbm_gbs"] * 1e9)
+                t_tensor = MMAS_PER_PRODUCT * aflops / (peaks["bf16_tflops_sustained"] * 1e12)
+                bound = "hbm" if t_hbm >= t_tensor else "tensor"
+            if bound == "hbm":
+                roof = {"bound": "hbm", "achieved": abytes * prof_steps / seconds / 1e9, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s"}
+                roof["frac_of_nominal_8TBps"] = roof["achieved"] / NOMINAL_HBM_GBS
+            else:
+                roof = {"bound": "tensor", "achieved": aflops * prof_steps / seconds / 1e12,
+                        "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                        "note": f"algorithmic flops; the tensor pipe executes {MMAS_PER_PRODUCT} bf16 MMA(s) per product"}
+        roof.update({"frac": (roof["achieved"] / roof["peak"]) if roof["achieved"] else None,
+                     "traffic": traffic_table.get((w.name, cls)), "kernel": cls,
+                     "launches_per_step": launches / prof_steps, "avg_launch_us": 1e3 * ms / max(launches, 1),
+                     "share_of_kernel_time": shares.get(cls), "peak_source": peaks["source"],
+                     "timing": f"CUDA events round every launch of the class, {prof_steps} step(s) after the timed region"})
+        return roof
+
+    roof = roofline_of(top)
+    spmm_ms = prof["spmm_forward"][0] + prof["spmm_backward"][0]
+    spmm_bytes = sum(work[k][1] for k in ("spmm_forward", "spmm_backward") if k in work)
+    roof_spmm = {"bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"], "peak_source": peaks["source"],
+                 "kernels": {k: roofline_of(k) for k in ("spmm_forward", "spmm_backward") if prof[k][1]}}
+    if spmm_ms > 0 and spmm_bytes > 0:
+        roof_spmm["achieved"] = spmm_bytes * prof_steps / (spmm_ms / 1e3) / 1e9
+        roof_spmm["frac"] = roof_spmm["achieved"] / peaks["hbm_gbs"]
+        roof_spmm["frac_of_nominal_8TBps"] = roof_spmm["achieved"] / NOMINAL_HBM_GBS
+        roof_spmm["share_of_kernel_time"] = spmm_ms / total_kernel_ms
     per_class = {}
     for k, (ms, cnt) in prof.items():
         if cnt == 0:
             continue
-        entry = {"ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps,
+        entry = {"ms_per_step": ms / prof_steps, "launches_per_step": cnt / prof_steps,
                  "share": ms / total_kernel_ms if total_kernel_ms else None}
-        if k in work and ms > 0:
+        if k in work and ms > 0 and work[k][1] > 0:
             bound, abytes, aflops = work[k]
-            entry["GBps"] = abytes * args.steps / (ms / 1e3) / 1e9
+            entry["GBps"] = abytes * prof_steps / (ms / 1e3) / 1e9
+            entry["frac_of_measured_hbm"] = entry["GBps"] / peaks["hbm_gbs"]
+            entry["frac_of_nominal_8TBps"] = entry["GBps"] / NOMINAL_HBM_GBS
             if aflops:
-                entry["TFLOPps"] = aflops * args.steps / (ms / 1e3) / 1e12
+                entry["TFLOPps"] = aflops * prof_steps / (ms / 1e3) / 1e12
         per_class[k] = entry
-    gpu_launches = int(sum(cnt for _, cnt in prof.values()))
+    # the partition as a whole: its count, scan and scatter launches (the scan class also holds the short
+    # scan of the induced-subgraph offsets) against the 12 B per node it must write
+    part_ms = sum(prof[k][0] for k in ("partition_count", "scan", "partition_scatter"))
+    if part_ms > 0 and work:
+        gbps = (work["partition_count"][1] + work["partition_scatter"][1]) * prof_steps / (part_ms / 1e3) / 1e9
+        per_class["partition_total"] = {"ms_per_step": part_ms / prof_steps, "GBps": gbps,
+                                        "frac_of_measured_hbm": gbps / peaks["hbm_gbs"],
+                                        "frac_of_nominal_8TBps": gbps / NOMINAL_HBM_GBS}
 
     # ---- end to end through the host-buffer entry point ------------------------------
     resident.clear()              # the host-buffer call brings its own copies
@@ -647,6 +758,7 @@ def main():
         "edges_gathered_per_s": world * args.steps * kept * ((passes - 1) * w.K + 1) * w.R / elapsed_s,
         "loss_first_last": [first_loss, final_loss],
         "roofline": roof,
+        "roofline_spmm": roof_spmm,
         "kernels": per_class,
         "gpu_launches": gpu_launches,
         "clocks": clocks,
@@ -657,7 +769,7 @@ def main():
         cb = cpu_sample(w, local_steps=2)
         line["cpu_baseline"] = {"value": cb["value"], "unit": UNIT, "cores": 1, "kind": "oracle",
                                 "sample": cb["sample"], "sample_seconds": cb["sample_s"],
-                                "trainer_steps_per_s": cb["trainer_steps_per_s"]}
+                                "trainer_steps_per_s": cb["trainer_steps_per_s"], "host": host_info()}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
