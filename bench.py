@@ -83,24 +83,43 @@ def algorithmic_work(dims, n_parts, e_parts, K, R, entries=0, rowptr_bytes=8, gr
     # its node id and its part
     work["induced_count"] = ("hbm", E * 8 + n * (2 * rowptr_bytes + 8 + 8), 0.0)
     work["induced_fill"] = ("hbm", E * 8 + e * 8 + n * (2 * rowptr_bytes + 8 + 8), 0.0)
-    work["gather_rows"] = ("hbm", 2.0 * n * (4 * dims[0] + 4) + 8.0 * n, 0.0)
-    work["to_planes"] = ("hbm", R * 8.0 * n * dims[0], 0.0)
-    # the aggregate of the input features is computed once per call (R times per bench step), not per step
-    spmm_f = sum(n * 8 * dims[l] + 4 * e + 8 * n for l in range(1, L)) + (n * 8 * dims[0] + 4 * e + 8 * n) / K
-    spmm_b = sum(n * 8 * dims[l + 1] + 4 * e + 12 * n for l in range(1, L))
-    work["spmm_forward"] = ("hbm", steps * spmm_f, steps * (sum(e * dims[l] for l in range(1, L)) + e * dims[0] / K))
-    work["spmm_backward"] = ("hbm", steps * spmm_b, steps * sum(2 * e * dims[l + 1] for l in range(1, L)))
+    work["gather_rows"] = ("hbm", 12.0 * n, 0.0)                         # labels only: perm, label in, label out
+    work["to_planes"] = ("hbm", R * (8.0 * n * dims[0] + 4.0 * n), 0.0)   # features gathered through perm into planes
+    # The last layer's aggregate is taken after its product when that is narrower (the library's rule:
+    # at most 64 classes and [H Ws | H Wn], 2 Cp wide, at most half as wide as the layer's input):
+    # scores = H Ws + Abar (H Wn) + b, dWn = H^T (Abar^T dZ).  Bytes below are those of the products and
+    # aggregations actually defined by that form.
     Mtr = len(n_parts)
-    gf_b = sum(4 * n * (2 * dims[l] + dims[l + 1]) + 4 * Mtr * (2 * dims[l] + 1) * dims[l + 1] for l in range(L))
-    gf_f = sum(2 * n * (2 * dims[l] + 1) * dims[l + 1] for l in range(L))
+    C = dims[L]
+    Cp = (C + 7) // 8 * 8
+    head = C <= 64 and 4 * Cp <= dims[L - 1]
+    full = range(L - 1) if head else range(L)          # layers whose products take [H | Abar H]
+    # aggregations per local step: Abar H^l for l >= 1 (l = 0 once per call), Abar^T dZ^l for l >= 1
+    agg_f = [dims[l] for l in full if l >= 1] + ([Cp] if head else [])
+    agg_b = [dims[l + 1] for l in range(1, L) if not (head and l == L - 1)] + ([Cp] if head else [])
+    first = (n * 8 * dims[0] + 4 * e + 8 * n) / K if (L > 1 or not head) else 0.0
+    spmm_f = sum(n * 8 * d + 4 * e + 8 * n for d in agg_f) + first
+    spmm_b = sum(n * 8 * d + 4 * e + 12 * n for d in agg_b)
+    work["spmm_forward"] = ("hbm", steps * spmm_f, steps * (sum(e * d for d in agg_f) + (e * dims[0] / K if first else 0.0)))
+    work["spmm_backward"] = ("hbm", steps * spmm_b, steps * sum(2 * e * d for d in agg_b))
+    gf_b = sum(4 * n * (2 * dims[l] + dims[l + 1]) + 4 * Mtr * (2 * dims[l] + 1) * dims[l + 1] for l in full)
+    gf_f = sum(2 * n * (2 * dims[l] + 1) * dims[l + 1] for l in full)
+    gw_b, gw_f = gf_b, gf_f
+    if head:   # T = H [Ws | Wn] (2 Cp wide out);  [dWs | dWn] = H^T [dZ | Q]
+        gf_b += 4 * n * (dims[L - 1] + 2 * Cp) + 4 * Mtr * 2 * dims[L - 1] * C
+        gf_f += 2 * n * dims[L - 1] * 2 * C
+        gw_b += 4 * n * (dims[L - 1] + 2 * Cp) + 4 * Mtr * (2 * dims[L - 1] + 1) * C
+        gw_f += 2 * n * (dims[L - 1] + 1) * 2 * C
     work["gemm_forward"] = ("gemm", steps * gf_b, steps * gf_f)
-    work["gemm_wgrad"] = ("gemm", steps * gf_b, steps * gf_f)
+    work["gemm_wgrad"] = ("gemm", steps * gw_b, steps * gw_f)
     # dgrad reads dZ and Abar^T dZ (planes), the gate (hi plane of H) and writes dZ of the layer below
-    gd_b = sum(n * (8 * dims[l + 1] + 2 * dims[l] + 4 * dims[l]) + 4 * Mtr * 2 * dims[l] * dims[l + 1] for l in range(1, L))
+    gd_b = sum(n * (8 * (Cp if head and l == L - 1 else dims[l + 1]) + 2 * dims[l] + 4 * dims[l]) +
+               4 * Mtr * 2 * dims[l] * dims[l + 1] for l in range(1, L))
     gd_f = sum(2 * n * 2 * dims[l] * dims[l + 1] for l in range(1, L))
     work["gemm_dgrad"] = ("gemm", steps * gd_b, steps * gd_f)
     P = sum((2 * dims[l] + 1) * dims[l + 1] for l in range(L))
-    work["softmax_xent"] = ("hbm", steps * (8 * n * dims[L] + 4 * n), 0.0)
+    # scores in (head form: the row's own product and the aggregated one), gradient out, label
+    work["softmax_xent"] = ("hbm", steps * ((12 * n * Cp if head else 8 * n * C) + 4 * n), 0.0)
     work["reduce_sgd"] = ("hbm", steps * 12.0 * Mtr * P, 0.0)
     work["aggregate"] = ("hbm", R * 8.0 * Mtr * P, 0.0)
     return work
@@ -571,15 +590,15 @@ def main():
         part_id, part_offsets, perm, local_id = ctx.partition(g.n, resident["gid"], w.partition_seed, w.M, grouped=w.grouped_order)
         rowptr_out, col_out, edge_offsets, kept_cut, edge_host = ctx.build_induced_csr(
             resident["rowptr"], resident["col"], w.M, part_id, part_offsets, perm, local_id)
-        Xp = ctx.gather_rows(resident["X"], perm)
         yp = ctx.gather_rows(resident["y"], perm)
         part_host = part_offsets.cpu().tolist()
         for r in range(w.R):
             if pool:  # the trainers' streams start after the preprocessing / the previous aggregation
                 for st in pool:
                     st.wait_stream(torch.cuda.current_stream())
-            ctx.local_steps(w.dims, w.lr, w.M, part_host, edge_host, rowptr_out, col_out, Xp, yp, params, w.K,
-                            loss_out=loss[r], gemm_dtype=w.gemm_dtype, streams=trainer_streams, variant=w.variant)
+            # the features stay in node order: the training call gathers them through perm
+            ctx.local_steps(w.dims, w.lr, w.M, part_host, edge_host, rowptr_out, col_out, resident["X"], yp, params, w.K,
+                            loss_out=loss[r], gemm_dtype=w.gemm_dtype, streams=trainer_streams, variant=w.variant, perm=perm)
             if pool:
                 for st in pool:
                     torch.cuda.current_stream().wait_stream(st)

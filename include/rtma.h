@@ -210,6 +210,18 @@ int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* model, int32_t M,
                          const float* Xp, const int32_t* yp, float* params, int32_t K,
                          float* loss_out, const rtma_taps* taps, void* const* streams);
 
+/* rtma_local_steps on features that are still in the graph's node order: X [n][dims[0]] as the
+ * caller holds it, perm [n] from rtma_partition; row i of the partition order is X[perm[i]] ("load
+ * G_train^(i)", Algorithm 2, done while the features are brought into the layout of the products).
+ * Saves the rtma_gather_rows pass over the features and its copy in partition order.  yp stays in
+ * partition order (rtma_gather_rows on the labels).  Everything else, and the result bit for bit,
+ * as rtma_local_steps given rtma_gather_rows(X, perm).                                        */
+int32_t rtma_local_steps_gathered(rtma_ctx* ctx, const rtma_model_desc* model, int32_t M,
+                                  const int64_t* part_offsets_host, const int64_t* edge_offsets_host,
+                                  const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                                  const float* X, const int32_t* perm, const int32_t* yp, float* params,
+                                  int32_t K, float* loss_out, const rtma_taps* taps, void* const* streams);
+
 /* Local training with a step count of its own for every trainer.  Aggregation is triggered by
  * wall time, not by a step count (Sec. 3.1), so trainers arrive at an aggregation with
  * different numbers of finished steps (Table 4 reports up to 28.8% fewer on the slowest one):
@@ -306,7 +318,7 @@ int32_t rtma_selftest_wait_timeout(rtma_ctx* ctx, void* stream);
  * Every pointer here is a HOST pointer (pageable or pinned).  Copies the graph (CSR as for
  * rtma_build_induced_csr), group_id_h (NULL = RandomTMA), features X_h [n][dims[0]], labels
  * y_h [n] and the common initial parameters params0_h [P] to the device, runs rtma_partition
- * (rtma_partition_grouped when super-node ids are given), rtma_build_induced_csr, rtma_gather_rows, then R rounds of (rtma_local_steps with K steps on
+ * (rtma_partition_grouped when super-node ids are given), rtma_build_induced_csr, rtma_gather_rows (labels), then R rounds of (rtma_local_steps_gathered with K steps on
  * every part, rtma_aggregate), and copies back params_out_h [P] (the averaged parameters),
  * loss_out_h [R][M][K] (or NULL) and kept_cut_h [2] (or NULL).  The graph must be undirected
  * with both directions stored.  Allocates and frees its device buffers with cudaMalloc /

@@ -23,7 +23,7 @@ EXPORTS = (
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
     "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout", "rtma_link_param_count",
-    "rtma_link_steps", "rtma_set_workspace_limit",
+    "rtma_link_steps", "rtma_set_workspace_limit", "rtma_local_steps_gathered",
 )
 KERNEL_CLASSES = 21
 
@@ -266,9 +266,11 @@ class Context:
     # ---- Algorithm 2 ----------------------------------------------------------------
     def local_steps(self, dims, lr, M, part_offsets_host, edge_offsets_host, rowptr_out, col_out, Xp, yp,
                     params, K, loss_out=None, streams=None, gemm_dtype=0, taps=None, symmetric=True,
-                    variant=(0, 0, 0)):
+                    variant=(0, 0, 0), perm=None):
         """K SGD steps on each of the M parts, in place on params [M, P].  K: an int, or a sequence
         of M per-trainer step counts (0 = the trainer does not run; rtma_local_steps_var).
+        perm: Xp is the feature matrix in node order and perm the partition's permutation
+        (rtma_local_steps_gathered; fixed K only).
         streams: None (all trainers on the current stream), or a list of M torch streams.
         taps: None or (acts tensor or None, grads tensor or None, step).
         variant: (encoder, act, norm) of rtma_model_desc."""
@@ -293,7 +295,14 @@ class Context:
             acts, grads, step = taps
             tap_struct = Taps(_ptr(acts), _ptr(grads), int(step))
         tap_ref = ctypes.byref(tap_struct) if tap_struct is not None else None
-        if isinstance(K, int):
+        if perm is not None:
+            _need(perm, torch.int32, "perm", dev)
+            st = self._lib.rtma_local_steps_gathered(
+                self._h, ctypes.byref(md), ctypes.c_int32(M), po, eo, _ptr(rowptr_out), _ptr(col_out),
+                ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), _ptr(perm), _ptr(yp), _ptr(params), ctypes.c_int32(int(K)),
+                _ptr(loss_out), tap_ref, sarr)
+            self._check(st, "rtma_local_steps_gathered")
+        elif isinstance(K, int):
             st = self._lib.rtma_local_steps(
                 self._h, ctypes.byref(md), ctypes.c_int32(M), po, eo, _ptr(rowptr_out), _ptr(col_out),
                 ctypes.c_int32(1 if symmetric else 0), _ptr(Xp), _ptr(yp), _ptr(params), ctypes.c_int32(K),

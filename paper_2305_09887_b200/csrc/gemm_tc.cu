@@ -67,9 +67,15 @@ __device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
 //            kk <  Kd/2 : Ws[j][kk]          (zero beyond d_in / d_out)
 //            kk >= Kd/2 : Wn[j][kk - Kd/2]
 // each written as a hi and a lo bf16 matrix.
+// Head form (head_cp > 0; the last layer when its aggregate is taken after the product,
+// Abar (H Wn) instead of (Abar H) Wn): the weight matrices side by side along n,
+//   forward  Bf[n][kk], kk < Kf = 64 * ceil(d_in / 64):
+//            n <  head_cp : Ws[kk][n]           (zero beyond d_out)
+//            n >= head_cp : Wn[kk][n - head_cp] (one-matrix layers have the first block only)
 // ------------------------------------------------------------------------------------
 struct PrepArgs {
     LayerShape ls;
+    int head_cp;
     int Npad_f, Kf, Npad_d, Kd;
     __nv_bfloat16 *Bf_hi, *Bf_lo, *Bd_hi, *Bd_lo;  // [group slot][Npad][K]
 };
@@ -94,9 +100,14 @@ tc_weight_prep_kernel(const __grid_constant__ GroupDesc g, const __grid_constant
         __nv_bfloat16 *hi, *lo;
         if (i < nf) {
             const int n = (int)(i / a.Kf), kk = (int)(i % a.Kf);
-            const int half = a.Kf / a.ls.nsrc;  // one block of K per weight matrix
-            const int src = kk < half ? kk : kk - half;
-            if (n < d_out && src < d_in) x = W[(int64_t)(kk < half ? src : d_in + src) * d_out + n];
+            if (a.head_cp > 0) {
+                const int blk = n / a.head_cp, c = n % a.head_cp;  // which weight matrix, which of its columns
+                if (blk < a.ls.nsrc && c < d_out && kk < d_in) x = W[(int64_t)(blk * d_in + kk) * d_out + c];
+            } else {
+                const int half = a.Kf / a.ls.nsrc;  // one block of K per weight matrix
+                const int src = kk < half ? kk : kk - half;
+                if (n < d_out && src < d_in) x = W[(int64_t)(kk < half ? src : d_in + src) * d_out + n];
+            }
             hi = a.Bf_hi + (int64_t)k * nf + i;
             lo = a.Bf_lo + (int64_t)k * nf + i;
         } else {
@@ -724,6 +735,13 @@ TcLayerPlan tc_plan_layer(LayerShape ls) {
     return p;
 }
 
+TcLayerPlan tc_plan_head(LayerShape ls, int head_cp) {
+    TcLayerPlan p = tc_plan_layer(ls);  // the dgrad operand is the usual one
+    p.Kf = TC_BK * (int)ceil_div(ls.d_in, TC_BK);
+    p.BN_f = p.Npad_f = (int)ceil_div(ls.nsrc * head_cp, 16) * 16;
+    return p;
+}
+
 size_t tc_prep_elems(const TcLayerPlan& p, bool with_dgrad) {
     return 2 * ((size_t)p.Npad_f * p.Kf + (with_dgrad ? (size_t)p.Npad_d * p.Kd : 0));
 }
@@ -738,7 +756,7 @@ int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, const TcPrepJob
     int64_t most = 0;
     for (int j = 0; j < njobs; ++j) {
         const TcLayerPlan& p = jobs[j].plan;
-        b.job[j] = PrepArgs{jobs[j].ls, p.Npad_f, p.Kf, p.Npad_d, p.Kd, jobs[j].Bf_hi, jobs[j].Bf_lo, jobs[j].Bd_hi, jobs[j].Bd_lo};
+        b.job[j] = PrepArgs{jobs[j].ls, jobs[j].head_cp, p.Npad_f, p.Kf, p.Npad_d, p.Kd, jobs[j].Bf_hi, jobs[j].Bf_lo, jobs[j].Bd_hi, jobs[j].Bd_lo};
         most = std::max(most, (int64_t)p.Npad_f * p.Kf + (jobs[j].Bd_hi ? (int64_t)p.Npad_d * p.Kd : 0));
     }
     dim3 grid((unsigned)std::min<int64_t>(ceil_div(most, 256), 64), (unsigned)g.num, (unsigned)njobs);

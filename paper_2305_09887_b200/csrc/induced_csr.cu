@@ -2,11 +2,13 @@
 // alpha^{-1}(i)}), emitted as one CSR per part over local ids, plus the row gather that
 // brings features and labels into partition order.
 //
-// COUNT: one warp per output row (rows taken in partition order, so part p's rows are
-// contiguous) counts the entries whose endpoint lies in the same part; an exclusive scan of
-// the counts gives every row's slot in col_out, from which the per-part zero-based offsets
-// and edge_offsets follow.  FILL: the same walk, with a warp ballot turning the keep
-// predicate into compact, order-preserving output positions.
+// COUNT: one warp per row of the input graph, rows in the input's order so that the column
+// indices stream; it counts the entries whose endpoint lies in the same part and leaves the count
+// at the row's place in partition order.  An exclusive scan of the counts gives every row's slot
+// in col_out, from which the per-part zero-based offsets and edge_offsets follow.  FILL: the same
+// walk, with a warp ballot turning the keep predicate into compact, order-preserving output
+// positions.  Per entry the only random access is the part of its endpoint; both phases first
+// pack the part ids into one byte per node, so that this table (25 MB for 25 M nodes) stays in L2.
 #include "common.cuh"
 
 namespace {
@@ -14,31 +16,33 @@ namespace {
 constexpr int CSR_THREADS = 256;
 constexpr int CSR_WARPS = CSR_THREADS / 32;
 
-__device__ __forceinline__ int find_part(const int64_t* __restrict__ offs, int M, int64_t row) {
-    int lo = 0, hi = M;  // largest p with offs[p] <= row and offs[p+1] > row
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (offs[mid] <= row) lo = mid; else hi = mid;
+// part8[v] = part_id[v] as one byte (at most 64 parts), four nodes per thread
+__global__ void __launch_bounds__(256)
+pack_parts_kernel(int64_t n, const int32_t* __restrict__ part_id, uint8_t* __restrict__ part8, const bool aligned) {
+    const int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
+    if (aligned && i + 3 < n) {
+        const int4 p = *reinterpret_cast<const int4*>(part_id + i);
+        *reinterpret_cast<uint32_t*>(part8 + i) = (uint32_t)p.x | ((uint32_t)p.y << 8) | ((uint32_t)p.z << 16) | ((uint32_t)p.w << 24);
+    } else {
+        for (int64_t v = i; v < n; ++v) part8[v] = (uint8_t)part_id[v];
     }
-    return lo;
 }
 
 template <class RowT>
 __global__ void __launch_bounds__(CSR_THREADS)
 induced_count_kernel(int64_t n, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
-                     const int32_t* __restrict__ part_id, const int32_t* __restrict__ perm,
-                     int32_t* __restrict__ counts) {
+                     const uint8_t* __restrict__ part8, const int64_t* __restrict__ part_offsets,
+                     const int32_t* __restrict__ local_id, int32_t* __restrict__ counts) {
     const int lane = threadIdx.x & 31;
-    const int64_t j = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
-    if (j >= n) return;
-    const int32_t u = perm[j];
-    const int32_t p = part_id[u];
+    const int64_t u = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
+    if (u >= n) return;
+    const int p = part8[u];
     const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
     int kept = 0;
-    for (int64_t e = begin + lane; e < end; e += 32) kept += (part_id[col[e]] == p);
+    for (int64_t e = begin + lane; e < end; e += 32) kept += (part8[__ldg(col + e)] == p);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
-    if (lane == 0) counts[j] = kept;
+    if (lane == 0) counts[part_offsets[p] + local_id[u]] = kept;  // the row's place in partition order
 }
 
 // slots[j] = global slot of row j's first kept entry (exclusive scan of counts), j = 0..n.
@@ -75,18 +79,15 @@ induced_offsets_kernel(int64_t n, int M, const int64_t* __restrict__ part_offset
 template <class RowT>
 __global__ void __launch_bounds__(CSR_THREADS)
 induced_fill_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
-                    const int32_t* __restrict__ part_id, const int64_t* __restrict__ part_offsets,
-                    const int32_t* __restrict__ perm, const int32_t* __restrict__ local_id,
+                    const uint8_t* __restrict__ part8, const int64_t* __restrict__ part_offsets,
+                    const int32_t* __restrict__ local_id,
                     const int64_t* __restrict__ rowptr_out, const int64_t* __restrict__ edge_offsets,
                     int32_t* __restrict__ col_out) {
-    __shared__ int64_t offs[RTMA_MAX_PARTS + 1];
-    for (int b = threadIdx.x; b <= M; b += CSR_THREADS) offs[b] = part_offsets[b];
-    __syncthreads();
     const int lane = threadIdx.x & 31;
-    const int64_t j = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
-    if (j >= n) return;
-    const int p = find_part(offs, M, j);
-    const int32_t u = perm[j];
+    const int64_t u = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
+    if (u >= n) return;
+    const int p = part8[u];
+    const int64_t j = part_offsets[p] + local_id[u];  // the row's place in partition order
     const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
     int64_t out = edge_offsets[p] + rowptr_out[j + p];
     const unsigned below = (1u << lane) - 1u;
@@ -95,8 +96,8 @@ induced_fill_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int
         int32_t v = 0;
         bool keep = false;
         if (e < end) {
-            v = col[e];
-            keep = part_id[v] == p;
+            v = __ldg(col + e);
+            keep = part8[v] == p;
         }
         const unsigned votes = __ballot_sync(0xffffffffu, keep);
         if (keep) col_out[out + __popc(votes & below)] = local_id[v];
@@ -141,35 +142,44 @@ extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowp
     RTMA_TRY(order_after_training(ctx, stream));
     const unsigned row_blocks = (unsigned)ceil_div(n, CSR_WARPS);
 
+    const unsigned pack_blocks = (unsigned)ceil_div(n, 1024);
     if (col_out) {  // FILL
         if (n == 0) return RTMA_OK;
+        RTMA_TRY(rtma_reserve(ctx, ArenaCursor::granule((size_t)n + 16)));
+        uint8_t* part8 = reinterpret_cast<uint8_t*>(ctx->arena);
+        { KernelScope ks(ctx, KC_CSR_FILL, stream); pack_parts_kernel<<<pack_blocks, 256, 0, stream>>>(n, part_id, part8, reinterpret_cast<uintptr_t>(part_id) % 16 == 0); }
+        RTMA_LAUNCH_CHECK(ctx);
         if (rowptr_is_64)
             { KernelScope ks(ctx, KC_CSR_FILL, stream); induced_fill_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, M, static_cast<const int64_t*>(rowptr), col, part_id, part_offsets, perm, local_id, rowptr_out,
+                n, M, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, rowptr_out,
                 edge_offsets, col_out); }
         else
             { KernelScope ks(ctx, KC_CSR_FILL, stream); induced_fill_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, M, static_cast<const int32_t*>(rowptr), col, part_id, part_offsets, perm, local_id, rowptr_out,
+                n, M, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, rowptr_out,
                 edge_offsets, col_out); }
         RTMA_LAUNCH_CHECK(ctx);
         return RTMA_OK;
     }
 
     // COUNT
-    const size_t need = ArenaCursor::granule(sizeof(int32_t) * (n + 1)) + ArenaCursor::granule(sizeof(int64_t) * (n + 2)) +
+    const size_t need = ArenaCursor::granule((size_t)n + 16) + ArenaCursor::granule(sizeof(int32_t) * (n + 1)) +
+                        ArenaCursor::granule(sizeof(int64_t) * (n + 2)) +
                         ArenaCursor::granule(sizeof(int64_t) * scan_scratch_elems(n));
     RTMA_TRY(rtma_reserve(ctx, need));
     ArenaCursor cur(ctx->arena);
+    uint8_t* part8 = cur.take<uint8_t>((size_t)n + 16);
     int32_t* counts = cur.take<int32_t>(n + 1);
     int64_t* slots = cur.take<int64_t>(n + 2);
     int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(n));
     if (n > 0) {
+        { KernelScope ks(ctx, KC_CSR_COUNT, stream); pack_parts_kernel<<<pack_blocks, 256, 0, stream>>>(n, part_id, part8, reinterpret_cast<uintptr_t>(part_id) % 16 == 0); }
+        RTMA_LAUNCH_CHECK(ctx);
         if (rowptr_is_64)
             { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, static_cast<const int64_t*>(rowptr), col, part_id, perm, counts); }
+                n, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
         else
             { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, static_cast<const int32_t*>(rowptr), col, part_id, perm, counts); }
+                n, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
         RTMA_LAUNCH_CHECK(ctx);
     }
     RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, n, slots, scratch, stream));

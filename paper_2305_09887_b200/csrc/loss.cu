@@ -186,6 +186,90 @@ softmax_xent_row_kernel(const __grid_constant__ GroupDesc g, const Mat logits, c
     }
 }
 
+// The head of the network when the last layer's aggregate is taken after the product (at most 64
+// classes): the row's scores are z = [T_self +] NT + b, with T_self the row's own product H Ws (absent
+// for one-matrix layers) and NT the aggregated product Abar (H Wn), both split planes; they are formed
+// in the thread's registers and never stored (`scores` != NULL records them, for verification).  The
+// rest is softmax_xent_row_kernel.
+template <int NV4>
+__global__ void __launch_bounds__(LOSS_TILE_ROWS)
+softmax_xent_head_kernel(const __grid_constant__ GroupDesc g, const Planes Tself, const Planes NT,
+                         const float* __restrict__ params, const int64_t P, const int64_t bias_offset, const int C,
+                         const int32_t* __restrict__ yp, const Planes dZ, const Mat scores, float* __restrict__ tile_loss) {
+    __shared__ float warp_loss[LOSS_TILE_ROWS / 32];
+    int k, r0;
+    if (!locate_tile(g, LOSS_TILE_ROWS, blockIdx.x, &k, &r0)) return;
+    const int n_p = g.rows[k];
+    const int i = r0 + threadIdx.x;
+    float loss = 0.f;
+    if (i < n_p) {
+        const int64_t r = g.row_ws[k] + i;
+        const float* bias = params + (int64_t)g.part[k] * P + bias_offset;
+        const int label = yp[g.row_abs[k] + i];
+        const int n8 = (int)(NT.ld >> 3) < NV4 / 2 ? (int)(NT.ld >> 3) : NV4 / 2;
+        float v[4 * NV4];
+#pragma unroll
+        for (int q = 0; q < NV4 / 2; ++q) {
+            Pack8 x;
+            x.zero();
+            if (q < n8) {
+                x.add_planes(*reinterpret_cast<const uint4*>(NT.hi + r * NT.ld + 8 * q), *reinterpret_cast<const uint4*>(NT.lo + r * NT.ld + 8 * q));
+                if (Tself.hi)
+                    x.add_planes(*reinterpret_cast<const uint4*>(Tself.hi + r * Tself.ld + 8 * q),
+                                 *reinterpret_cast<const uint4*>(Tself.lo + r * Tself.ld + 8 * q));
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[8 * q + e] = x.v[e] + (8 * q + e < C ? __ldg(bias + 8 * q + e) : 0.f);
+        }
+        if (scores.ptr) {
+#pragma unroll
+            for (int c = 0; c < 4 * NV4; ++c)
+                if (c < C) scores.ptr[r * scores.ld + c] = v[c];
+        }
+        float zmax = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4 * NV4; ++c) {
+            if (c >= C) v[c] = -INFINITY;
+            zmax = fmaxf(zmax, v[c]);
+        }
+        float sum = 0.f, zl = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4 * NV4; ++c) {
+            if (c == label) zl = v[c];
+            v[c] = c < C ? expf(v[c] - zmax) : 0.f;
+            sum += v[c];
+        }
+        loss = zmax + logf(sum) - zl;
+        const float scale = 1.0f / (sum * (float)n_p);  // softmax / n_p = e * scale
+        const float hot = 1.0f / (float)n_p;
+        uint4* ph = reinterpret_cast<uint4*>(dZ.hi + r * dZ.ld);
+        uint4* pl = reinterpret_cast<uint4*>(dZ.lo + r * dZ.ld);
+#pragma unroll
+        for (int q = 0; q < NV4 / 2; ++q) {
+            if (q >= n8) break;
+            Pack8 x;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int c = 8 * q + e;
+                x.v[e] = c < C ? v[c] * scale - (c == label ? hot : 0.f) : 0.f;  // padding columns stay zero
+            }
+            uint4 h, l;
+            x.to_planes_cvt(h, l);
+            ph[q] = h;
+            pl[q] = l;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+    if ((threadIdx.x & 31) == 0) warp_loss[threadIdx.x >> 5] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float sacc = 0.f;
+        for (int w = 0; w < LOSS_TILE_ROWS / 32; ++w) sacc += warp_loss[w];
+        tile_loss[blockIdx.x] = sacc;
+    }
+}
+
 // More than 128 classes: the row is swept three times (max, sum of exponentials, gradient).
 __global__ void __launch_bounds__(LOSS_THREADS)
 softmax_xent_wide_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const int C, const int32_t* __restrict__ yp,
@@ -264,6 +348,25 @@ int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C
         else if (C <= 64) softmax_xent_row_kernel<16><<<(unsigned)tiles, LOSS_TILE_ROWS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         else if (C <= LOSS_REG_CLASSES) softmax_xent_kernel<4><<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
         else softmax_xent_wide_kernel<<<(unsigned)tiles, LOSS_THREADS, 0, s>>>(g, logits, C, yp, dZ, tile_loss);
+        RTMA_LAUNCH_CHECK(ctx);
+    }
+    return launch_loss_finalize(ctx, g, tile_loss, loss_out, loss_stride, loss_col, s);
+}
+
+int32_t launch_softmax_xent_head(rtma_ctx* ctx, const GroupDesc& g, Planes Tself, Planes NT, const float* params, int64_t P,
+                                 int64_t bias_offset, int C, const int32_t* yp, Planes dZ, Mat scores, float* tile_loss,
+                                 float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s) {
+    if (C > 64) return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "internal: head kernel with %d classes", C);
+    const int64_t tiles = group_tiles(g, LOSS_TILE_ROWS);
+    if (tiles > 0) {
+        KernelScope ks(ctx, KC_LOSS, s);
+#define RTMA_HEAD(NV4) softmax_xent_head_kernel<NV4><<<(unsigned)tiles, LOSS_TILE_ROWS, 0, s>>>(g, Tself, NT, params, P, bias_offset, C, yp, dZ, scores, tile_loss)
+        if (C <= 8) RTMA_HEAD(2);
+        else if (C <= 16) RTMA_HEAD(4);
+        else if (C <= 32) RTMA_HEAD(8);
+        else if (C <= 48) RTMA_HEAD(12);
+        else RTMA_HEAD(16);
+#undef RTMA_HEAD
         RTMA_LAUNCH_CHECK(ctx);
     }
     return launch_loss_finalize(ctx, g, tile_loss, loss_out, loss_stride, loss_col, s);

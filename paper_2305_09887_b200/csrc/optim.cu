@@ -24,6 +24,28 @@ reduce_sgd_kernel(const __grid_constant__ GroupDesc g, const __grid_constant__ S
     params[at] -= lr * gsum;
 }
 
+// Head form: the chunk slots hold [(d_in + 1) x 2 cp] (see launch_reduce_sgd_head).
+__global__ void __launch_bounds__(256)
+reduce_sgd_head_kernel(const __grid_constant__ GroupDesc g, const __grid_constant__ SplitPlan sp, const LayerShape ls,
+                       const int cp, const float* __restrict__ partial, const float lr, float* __restrict__ params,
+                       float* __restrict__ grads_record) {
+    const int k = blockIdx.y;
+    const int64_t count = (int64_t)(ls.nsrc * ls.d_in + 1) * ls.d_out;  // the layer's parameters: weight matrices, bias
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= count) return;
+    const int row = (int)(i / ls.d_out), c = (int)(i % ls.d_out);
+    const int64_t stride = (int64_t)(ls.d_in + 1) * 2 * cp;
+    int64_t at_partial;
+    if (row == ls.nsrc * ls.d_in) at_partial = (int64_t)ls.d_in * 2 * cp + c;        // bias: column sums of dZ
+    else if (ls.nsrc == 2 && row < ls.d_in) at_partial = (int64_t)row * 2 * cp + c;   // Ws: H^T dZ
+    else at_partial = (int64_t)(row - (ls.nsrc - 1) * ls.d_in) * 2 * cp + cp + c;     // Wn (or W): H^T Q
+    float gsum = 0.f;
+    for (int s = sp.split_begin[k]; s < sp.split_begin[k + 1]; ++s) gsum += partial[(int64_t)s * stride + at_partial];
+    const int64_t at = (int64_t)g.part[k] * ls.P + ls.param_offset + i;
+    if (grads_record) grads_record[at] = gsum;
+    params[at] -= lr * gsum;
+}
+
 __global__ void __launch_bounds__(256)
 copy_rows_kernel(const float* __restrict__ src, const int64_t ld_src, float* __restrict__ dst, const int64_t ld_dst,
                  const int64_t rows, const int width) {
@@ -122,6 +144,16 @@ int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp
     const int64_t count = (int64_t)(ls.nsrc * ls.d_in + 1) * ls.d_out;
     dim3 grid((unsigned)ceil_div(count, 256), (unsigned)g.num);
     { KernelScope ks(ctx, KC_REDUCE_SGD, s); reduce_sgd_kernel<<<grid, 256, 0, s>>>(g, sp, ls, partial, lr, params, grads_record); }
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}
+
+int32_t launch_reduce_sgd_head(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int head_cp,
+                               const float* partial, float lr, float* params, float* grads_record, cudaStream_t s) {
+    if (g.num == 0) return RTMA_OK;
+    const int64_t count = (int64_t)(ls.nsrc * ls.d_in + 1) * ls.d_out;
+    dim3 grid((unsigned)ceil_div(count, 256), (unsigned)g.num);
+    { KernelScope ks(ctx, KC_REDUCE_SGD, s); reduce_sgd_head_kernel<<<grid, 256, 0, s>>>(g, sp, ls, head_cp, partial, lr, params, grads_record); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

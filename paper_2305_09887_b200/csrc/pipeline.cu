@@ -38,7 +38,7 @@ extern "C" int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_6
     const size_t o_X = reserve(4 * (size_t)n * F), o_y = reserve(4 * (size_t)n);
     const size_t o_pid = reserve(4 * (size_t)n), o_poff = reserve(8 * (M + 1)), o_perm = reserve(4 * (size_t)n), o_lid = reserve(4 * (size_t)n);
     const size_t o_rpo = reserve(8 * (size_t)(n + M)), o_eoff = reserve(8 * (M + 1)), o_kc = reserve(16);
-    const size_t o_Xp = reserve(4 * (size_t)n * F), o_yp = reserve(4 * (size_t)n);
+    const size_t o_yp = reserve(4 * (size_t)n);
     const size_t o_par = reserve(4 * (size_t)M * P), o_loss = reserve(4 * (size_t)R * M * (K > 0 ? K : 1));
     DeviceBlock blk, colblk;
     RTMA_CUDA(ctx, cudaMalloc(&blk.p, total));
@@ -75,15 +75,15 @@ extern "C" int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_6
     if (eo[M] > 0)
         RTMA_TRY(rtma_build_induced_csr(ctx, n, rowptr_is_64, at(o_rowptr), static_cast<int32_t*>(at(o_col)), M, part_id,
                                         part_offsets, perm, local_id, rowptr_out, col_out, edge_offsets, kept_cut, stream));
-    RTMA_TRY(rtma_gather_rows(ctx, n, 4 * F, at(o_X), perm, at(o_Xp), stream));
+    // the features stay in node order: the training call gathers them while it lays them out
     RTMA_TRY(rtma_gather_rows(ctx, n, 4, at(o_y), perm, at(o_yp), stream));
 
     std::vector<void*> streams(M, stream_);
     float* params = static_cast<float*>(at(o_par));
     float* loss = static_cast<float*>(at(o_loss));
     for (int r = 0; r < R; ++r) {
-        RTMA_TRY(rtma_local_steps(ctx, model, M, po.data(), eo.data(), rowptr_out, col_out, 1,
-                                  static_cast<float*>(at(o_Xp)), static_cast<int32_t*>(at(o_yp)), params, K,
+        RTMA_TRY(rtma_local_steps_gathered(ctx, model, M, po.data(), eo.data(), rowptr_out, col_out, 1,
+                                  static_cast<float*>(at(o_X)), perm, static_cast<int32_t*>(at(o_yp)), params, K,
                                   loss_out_h ? loss + (size_t)r * M * K : nullptr, nullptr, streams.data()));
         RTMA_TRY(rtma_aggregate(ctx, params, P, M, nullptr, stream));
     }

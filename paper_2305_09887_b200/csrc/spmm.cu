@@ -51,14 +51,16 @@ gcn_scale_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict_
 }
 
 __global__ void __launch_bounds__(256)
-to_planes_kernel(const __grid_constant__ GroupDesc g, const float* __restrict__ X, const int d, const Planes out) {
+to_planes_kernel(const __grid_constant__ GroupDesc g, const float* __restrict__ X, const int32_t* __restrict__ perm,
+                 const int d, const Planes out) {
     int k, r0;
     if (!locate_tile(g, 32, blockIdx.x, &k, &r0)) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int q = 0; q < 4; ++q) {
         const int i = r0 + warp * 4 + q;
         if (i >= g.rows[k]) return;
-        const float* x = X + (g.row_abs[k] + i) * (int64_t)d;
+        // perm: the features are still in the graph's node order; row i of the partition order is node perm[i]
+        const float* x = X + (perm ? (int64_t)perm[g.row_abs[k] + i] : g.row_abs[k] + i) * (int64_t)d;
         const int64_t o = (g.row_ws[k] + i) * out.ld;
         for (int c0 = lane * 8; c0 < out.ld; c0 += 256) {
             Pack8 p;
@@ -585,10 +587,11 @@ int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64
 
 }  // namespace
 
-int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, int d, Planes out, cudaStream_t s) {
+int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, const int32_t* perm, int d, Planes out,
+                         cudaStream_t s) {
     const int64_t tiles = group_tiles(g, 32);
     if (tiles == 0) return RTMA_OK;
-    { KernelScope ks(ctx, KC_TO_PLANES, s); to_planes_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, X, d, out); }
+    { KernelScope ks(ctx, KC_TO_PLANES, s); to_planes_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, X, perm, d, out); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

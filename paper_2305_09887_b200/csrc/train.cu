@@ -15,6 +15,9 @@ struct Model {
     float lr;
     bool gcn;   // GCN layers (one weight matrix, renormalised adjacency) instead of GraphSAGE-mean
     bool post;  // hidden layers normalise and / or use PReLU: the activation is a pass of its own
+    bool head;  // the last layer's aggregate is taken after its product, at the width of the classes:
+                // Abar (H Wn) instead of (Abar H) Wn (the same function; a fraction of the bytes)
+    int Cp;     // classes rounded up to 8 (one 16-byte piece of a plane)
     int Kd;     // link prediction: decoder layers (0: node classification)
     int ddims[RTMA_MAX_LAYERS + 1];
     LayerShape dec[RTMA_MAX_LAYERS];
@@ -89,6 +92,9 @@ int32_t parse_model(rtma_ctx* ctx, const rtma_model_desc* md, Model* m) {
     m->gcn = md->encoder == 1;
     m->post = md->L > 1 && (md->act == 1 || md->norm == 1);
     m->Kd = 0;
+    m->Cp = (int)planes_ld(md->dims[md->L]);
+    // worth it when the products' outputs ([H Ws | H Wn]) are at most half as wide as the layer's input
+    m->head = md->dims[md->L] <= 64 && 2 * m->layer[md->L - 1].nsrc * m->Cp <= md->dims[md->L - 1];
     return RTMA_OK;
 }
 
@@ -104,22 +110,25 @@ struct ScratchPlan {
 
 int64_t aligned_rows(int64_t n_p) { return ceil_div(n_p, GROUP_ROW_ALIGN) * GROUP_ROW_ALIGN; }
 
-ScratchPlan plan_scratch(const Model& m) {
+ScratchPlan plan_scratch(const Model& m, bool head, bool record) {
     ScratchPlan sp{};
     size_t per_row = sizeof(float);              // inv_deg
     per_row += 4 * planes_ld(m.dims[0]);         // X as planes
     int q_width = 0;
     for (int l = 0; l < m.L; ++l) {
-        per_row += 4 * planes_ld(m.dims[l]);     // Abar H^l
+        if (l < m.L - 1 || !head || record) per_row += 4 * planes_ld(m.dims[l]);     // Abar H^l
         if (l < m.L - 1) per_row += 4 * planes_ld(m.dims[l + 1]);  // H^{l+1}, later overwritten by dZ^l
         if (l < m.L - 1 && m.post) per_row += 4 * planes_ld(m.dims[l + 1]) + sizeof(float2);  // Z^{l}, (mean, 1/std)
-        if (l >= 1) q_width = std::max(q_width, m.dims[l + 1]);
+        if (l >= 1 && !(head && l == m.L - 1)) q_width = std::max(q_width, m.dims[l + 1]);
         sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(m.layer[l].nsrc * m.dims[l] + 1) * m.dims[l + 1]);
+        if (head && l == m.L - 1) sp.max_layer_params = std::max(sp.max_layer_params, (size_t)(m.dims[l] + 1) * 2 * m.Cp);
         if (l < m.L - 1 && m.post) sp.post_width = std::max(sp.post_width, (size_t)m.dims[l + 1]);
-        sp.prep_bytes += sizeof(__nv_bfloat16) * tc_prep_elems(tc_plan_layer(m.layer[l]), l >= 1) + 4 * 256;
+        const TcLayerPlan lp = (head && l == m.L - 1) ? tc_plan_head(m.layer[l], m.Cp) : tc_plan_layer(m.layer[l]);
+        sp.prep_bytes += sizeof(__nv_bfloat16) * tc_prep_elems(lp, l >= 1) + 4 * 256;
     }
-    per_row += sizeof(float) * planes_ld(m.dims[m.L]);  // logits
-    per_row += 4 * planes_ld(m.dims[m.L]);              // dZ of the last layer
+    if (!head || record) per_row += sizeof(float) * planes_ld(m.dims[m.L]);  // logits
+    if (head) per_row += 4 * (size_t)(m.layer[m.L - 1].nsrc + 1 + 2) * m.Cp;  // [H Ws | H Wn], its aggregate, [dZ | Abar^T dZ]
+    else per_row += 4 * planes_ld(m.dims[m.L]);         // dZ of the last layer
     sp.q_width = q_width;
     if (q_width) per_row += 4 * planes_ld(q_width);     // Abar^T dZ
     sp.per_row_bytes = per_row;
@@ -162,7 +171,7 @@ int plan_splits(const GroupDesc& g, int parts_in_flight, SplitPlan* sp) {
 size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p, int64_t pairs) {
     const size_t rows = (size_t)aligned_rows(n_p);
     const size_t prows = (size_t)aligned_rows(pairs);
-    const size_t matrices = 8 * m.L + 8 * m.Kd + 16;  // every matrix start is rounded up to 256 bytes
+    const size_t matrices = 8 * m.L + 8 * m.Kd + 24;  // every matrix start is rounded up to 256 bytes
     return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, 32) + 256) +
            sp.per_pair_bytes * prows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(pairs, 32) + 256) +
            sizeof(float) * ((size_t)ceil_div(pairs, 64) + 1) * (2 * sp.post_width + 1) +
@@ -186,7 +195,8 @@ namespace {
 int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const int64_t* part_offsets,
                    const int64_t* edge_offsets, const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
                    const float* Xp, const int32_t* yp, float* params, const int32_t* steps, int32_t loss_stride,
-                   float* loss_out, const rtma_taps* taps, void* const* streams, const LinkTask* link) {
+                   float* loss_out, const rtma_taps* taps, void* const* streams, const LinkTask* link,
+                   const int32_t* perm = nullptr) {
     if (!ctx) return RTMA_ERR_INVALID_ARG;
     Model m;
     RTMA_TRY(parse_model(ctx, md, &m));
@@ -261,7 +271,9 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
 
     // Scratch: every group owns an equal share of the arena; inside a share, parts run in
     // waves that fit.  Ask for enough to run every group in one wave when memory allows.
-    const ScratchPlan plan = plan_scratch(m);
+    const bool head = m.head && !link;
+    const bool record = taps && taps->acts;     // the verification record wants Abar H of every layer and the scores
+    const ScratchPlan plan = plan_scratch(m, head, record);
     size_t want_share = 0, min_share = 0;
     for (size_t gi = 0; gi < G; ++gi) {
         size_t sum = 0;
@@ -344,7 +356,8 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             float2* stats[RTMA_MAX_LAYERS];   // their (mean, 1/std)
             Hl[0] = take_planes(m.dims[0]);
             for (int l = 0; l < m.L; ++l) {
-                Nl[l] = take_planes(m.dims[l]);
+                if (l < m.L - 1 || !head || record) Nl[l] = take_planes(m.dims[l]);
+                else Nl[l] = Planes{nullptr, nullptr, 0};
                 if (l < m.L - 1) Hl[l + 1] = take_planes(m.dims[l + 1]);
                 if (l < m.L - 1 && m.post) {
                     Zl[l] = take_planes(m.dims[l + 1]);
@@ -356,8 +369,21 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             Mat logits{nullptr, (int64_t)planes_ld(C)};
             Planes R{nullptr, nullptr, 0};
             if (link) R = take_planes(C);
-            else logits.ptr = cur.take<float>((size_t)rows * planes_ld(C) + 8);
-            Planes dZlast = take_planes(C);
+            else if (!head || record) logits.ptr = cur.take<float>((size_t)rows * planes_ld(C) + 8);
+            // head form: T = [H Ws | H Wn] (blocks of Cp columns), NT = its aggregated second block,
+            // DQ = [dZ | Abar^T dZ]; dZlast and Qlast are the two halves of DQ
+            const int Cp = m.Cp, hsrc = m.layer[m.L - 1].nsrc;
+            Planes T{nullptr, nullptr, 0}, NT{nullptr, nullptr, 0}, DQ{nullptr, nullptr, 0}, Qlast{nullptr, nullptr, 0};
+            Planes dZlast;
+            if (head) {
+                T = take_planes(hsrc * Cp);
+                NT = take_planes(Cp);
+                DQ = take_planes(2 * Cp);
+                dZlast = DQ;
+                Qlast = Planes{DQ.hi + Cp, DQ.lo + Cp, DQ.ld};
+            } else {
+                dZlast = take_planes(C);
+            }
             // ---- link prediction: decoder activations per pair, fp32 gradient of the embeddings ----
             auto take_pair_planes = [&](int d) {
                 Planes pl;
@@ -404,7 +430,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             TcLayerPlan tcp[RTMA_MAX_LAYERS];
             __nv_bfloat16 *Bf_hi[RTMA_MAX_LAYERS], *Bf_lo[RTMA_MAX_LAYERS], *Bd_hi[RTMA_MAX_LAYERS], *Bd_lo[RTMA_MAX_LAYERS];
             for (int l = 0; l < m.L; ++l) {
-                tcp[l] = tc_plan_layer(m.layer[l]);
+                tcp[l] = (head && l == m.L - 1) ? tc_plan_head(m.layer[l], Cp) : tc_plan_layer(m.layer[l]);
                 const size_t nf = (size_t)g.num * tcp[l].Npad_f * tcp[l].Kf;
                 const size_t nd = l >= 1 ? (size_t)g.num * tcp[l].Npad_d * tcp[l].Kd : 0;
                 Bf_hi[l] = cur.take<__nv_bfloat16>(nf);
@@ -423,12 +449,14 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             for (int k = 0; k < g.num; ++k) wave_entries += edge_offsets[g.part[k] + 1] - edge_offsets[g.part[k]];
             SpmmOrder wave_order;
             RTMA_TRY(launch_spmm_order(ctx, g, rowptr_out, col_out, wave_entries, ticket + 16, heavy_list, &wave_order, s));
-            RTMA_TRY(launch_to_planes(ctx, g, Xp, m.dims[0], Hl[0], s));
+            RTMA_TRY(launch_to_planes(ctx, g, Xp, perm, m.dims[0], Hl[0], s));
             const Planes no_planes{nullptr, nullptr, 0};
             const Mat no_mat{nullptr, 0};
             // N^0 = (aggregated input features), once for all steps of the call
-            if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], false, wave_order, ticket, s));
-            else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], wave_order, ticket, s));
+            if (Nl[0].hi) {
+                if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], false, wave_order, ticket, s));
+                else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], wave_order, ticket, s));
+            }
             const GroupDesc wave = g;   // all parts of the wave, with their scratch rows
             const SplitPlan wave_sp = sp;
             for (int step = 0; step < wave_steps; ++step) {
@@ -464,11 +492,31 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 {
                     TcPrepJob jobs[2 * RTMA_MAX_LAYERS];
                     int nj = 0;
-                    for (int l = 0; l < m.L; ++l) jobs[nj++] = TcPrepJob{m.layer[l], tcp[l], Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l]};
-                    for (int k = 0; k < m.Kd; ++k) jobs[nj++] = TcPrepJob{m.dec[k], dtcp[k], DBf_hi[k], DBf_lo[k], DBd_hi[k], DBd_lo[k]};
+                    for (int l = 0; l < m.L; ++l)
+                        jobs[nj++] = TcPrepJob{m.layer[l], (head && l == m.L - 1) ? Cp : 0, tcp[l], Bf_hi[l], Bf_lo[l], Bd_hi[l], Bd_lo[l]};
+                    for (int k = 0; k < m.Kd; ++k) jobs[nj++] = TcPrepJob{m.dec[k], 0, dtcp[k], DBf_hi[k], DBf_lo[k], DBd_hi[k], DBd_lo[k]};
                     RTMA_TRY(launch_tc_weight_prep(ctx, g, jobs, nj, params, s));
                 }
                 for (int l = 0; l < m.L; ++l) {
+                    const bool head_layer = head && l == m.L - 1;
+                    if (head_layer) {
+                        // scores = H Ws + Abar (H Wn) + b: one product T = H [Ws | Wn] at the width of the
+                        // classes, then the aggregate of its second block (for GCN: Ahat (H W))
+                        LayerShape hs = m.layer[l];
+                        hs.nsrc = 1;
+                        hs.d_out = hsrc * Cp;
+                        hs.has_bias = 0;
+                        RTMA_TRY(launch_tc_forward(ctx, g, hs, tcp[l], rows, params, Hl[l], Hl[l], Bf_hi[l], Bf_lo[l], T, no_mat, false,
+                                                   single_pass, s));
+                        if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, T, NT, C, false, order, ticket, s));
+                        else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Planes{T.hi + Cp, T.lo + Cp, T.ld}, NT, C,
+                                                       order, ticket, s));
+                        if (tap && record && l > 0) {  // the record also holds Abar H of this layer (l == 0: computed before the loop)
+                            if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], false, order, ticket, s));
+                            else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[l], Nl[l], m.dims[l], order, ticket, s));
+                        }
+                        continue;
+                    }
                     if (l == 0) {
                         // the aggregate of the input features does not change from step to step
                     } else if (m.gcn) {
@@ -487,25 +535,16 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                         RTMA_TRY(launch_post_forward(ctx, g, m.layer[l], params, Zl[l], Hl[l + 1], stats[l], s));
                     }
                 }
-                if (tap && taps->acts && !link) {
-                    size_t rec = 0;  // floats per row in the record
-                    for (int l = 0; l < m.L; ++l) rec += (size_t)m.dims[l] + m.dims[l + 1];
-                    for (int k = 0; k < g.num; ++k) {
-                        float* dst = taps->acts + (size_t)g.row_abs[k] * rec;
-                        const int64_t n_p = g.rows[k];
-                        for (int l = 0; l < m.L; ++l) {
-                            RTMA_TRY(launch_from_planes(ctx, Nl[l], g.row_ws[k], n_p, m.dims[l], dst, s));
-                            dst += (size_t)n_p * m.dims[l];
-                            if (l < m.L - 1)
-                                RTMA_TRY(launch_from_planes(ctx, Hl[l + 1], g.row_ws[k], n_p, m.dims[l + 1], dst, s));
-                            else
-                                RTMA_TRY(launch_copy_rows(ctx, logits.ptr + g.row_ws[k] * logits.ld, logits.ld, dst, C, n_p, C, s));
-                            dst += (size_t)n_p * m.dims[l + 1];
-                        }
-                    }
-                }
                 // ---- loss; dZ of the last layer ----
-                if (!link) {
+                if (head) {
+                    const LayerShape& ll = m.layer[m.L - 1];
+                    RTMA_TRY(launch_softmax_xent_head(ctx, g, m.gcn ? no_planes : Planes{T.hi, T.lo, T.ld}, NT, params, ll.P,
+                                                      ll.param_offset + (int64_t)ll.nsrc * ll.d_in * ll.d_out, C, yp, dZlast,
+                                                      (tap && record) ? logits : no_mat, tile_loss, loss_out, loss_stride, step, s));
+                    // Abar^T dZ into the second half of DQ: the weight gradient needs it even in a one-layer model
+                    if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, dZlast, Qlast, C, true, order, ticket, s));
+                    else RTMA_TRY(launch_spmm_transposed(ctx, g, rowptr_out, col_out, inv_deg, dZlast, Qlast, C, order, ticket, s));
+                } else if (!link) {
                     RTMA_TRY(launch_softmax_xent(ctx, g, logits, C, yp, dZlast, tile_loss, loss_out, loss_stride, step, s));
                 } else {
                     float* grads_rec = tap ? taps->grads : nullptr;
@@ -537,10 +576,48 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                     RTMA_CUDA(ctx, cudaMemsetAsync(dRf, 0, sizeof(float) * (size_t)rows * planes_ld(C), s));
                     RTMA_TRY(launch_pair_scatter(ctx, gd, g, R, link->pu, link->pv, El[0], dRf, (int64_t)planes_ld(C), C, dZlast, s));
                 }
+                // ---- the verification record (the scores of the head form exist only after its loss kernel) ----
+                if (tap && taps->acts && !link) {
+                    size_t rec = 0;  // floats per row in the record
+                    for (int l = 0; l < m.L; ++l) rec += (size_t)m.dims[l] + m.dims[l + 1];
+                    for (int k = 0; k < g.num; ++k) {
+                        float* dst = taps->acts + (size_t)g.row_abs[k] * rec;
+                        const int64_t n_p = g.rows[k];
+                        for (int l = 0; l < m.L; ++l) {
+                            RTMA_TRY(launch_from_planes(ctx, Nl[l], g.row_ws[k], n_p, m.dims[l], dst, s));
+                            dst += (size_t)n_p * m.dims[l];
+                            if (l < m.L - 1)
+                                RTMA_TRY(launch_from_planes(ctx, Hl[l + 1], g.row_ws[k], n_p, m.dims[l + 1], dst, s));
+                            else
+                                RTMA_TRY(launch_copy_rows(ctx, logits.ptr + g.row_ws[k] * logits.ld, logits.ld, dst, C, n_p, C, s));
+                            dst += (size_t)n_p * m.dims[l + 1];
+                        }
+                    }
+                }
                 // ---- backward + SGD ----
                 for (int l = m.L - 1; l >= 0; --l) {
                     // dZ^l: from the loss, over H^{l+1} (fused ReLU gate) or over Z^l (separate activation pass)
                     const Planes dZ = l == m.L - 1 ? dZlast : (m.post ? Zl[l] : Hl[l + 1]);
+                    const bool head_layer = head && l == m.L - 1;
+                    if (head_layer) {
+                        // dWs = H^T dZ, dWn = (Abar H)^T dZ = H^T (Abar^T dZ): one product of H^T with [dZ | Q]
+                        LayerShape ws = m.layer[l];
+                        ws.nsrc = 1;
+                        ws.d_out = 2 * Cp;
+                        RTMA_TRY(launch_tc_wgrad(ctx, g, sp, ws, rows, Hl[l], Hl[l], DQ, partial, single_pass, s));
+                        if (l > 0) {
+                            if (!single_pass && dgrad_narrow_applies(m.layer[l]))
+                                RTMA_TRY(launch_dgrad_narrow(ctx, g, m.layer[l], params, dZlast, Qlast, Hl[l], !m.post, s));
+                            else
+                                RTMA_TRY(launch_tc_dgrad(ctx, g, m.layer[l], tcp[l], rows, dZlast, Qlast, Bd_hi[l], Bd_lo[l], Hl[l], !m.post,
+                                                         single_pass, s));
+                            if (m.post)
+                                RTMA_TRY(launch_post_backward(ctx, g, m.layer[l - 1], params, Zl[l - 1], Hl[l], stats[l - 1], post_partial,
+                                                              m.lr, tap ? taps->grads : nullptr, s));
+                        }
+                        RTMA_TRY(launch_reduce_sgd_head(ctx, g, sp, m.layer[l], Cp, partial, m.lr, params, tap ? taps->grads : nullptr, s));
+                        continue;
+                    }
                     RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, single_pass, s));
                     if (l > 0) {
                         // dH^l = dZ Ws^T + Abar^T (dZ Wn^T) = [dZ | Abar^T dZ] [Ws^T ; Wn^T]: aggregate first,
@@ -572,6 +649,21 @@ extern "C" int32_t rtma_local_steps_var(rtma_ctx* ctx, const rtma_model_desc* md
                                         void* const* streams) {
     return train_impl(ctx, md, M, part_offsets, edge_offsets, rowptr_out, col_out, symmetric, Xp, yp, params, steps,
                       loss_stride, loss_out, taps, streams, nullptr);
+}
+
+extern "C" int32_t rtma_local_steps_gathered(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M,
+                                             const int64_t* part_offsets, const int64_t* edge_offsets,
+                                             const int64_t* rowptr_out, const int32_t* col_out, int32_t symmetric,
+                                             const float* X, const int32_t* perm, const int32_t* yp, float* params,
+                                             int32_t K, float* loss_out, const rtma_taps* taps, void* const* streams) {
+    if (!ctx) return RTMA_ERR_INVALID_ARG;
+    if (K < 0) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "K=%d negative", K);
+    if (M < 1 || M > RTMA_MAX_PARTS) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "M=%d outside [1,%d]", M, RTMA_MAX_PARTS);
+    if (!perm) return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "rtma_local_steps_gathered: null perm");
+    int32_t steps[RTMA_MAX_PARTS];
+    for (int p = 0; p < M; ++p) steps[p] = K;
+    return train_impl(ctx, md, M, part_offsets, edge_offsets, rowptr_out, col_out, symmetric, X, yp, params, steps, K,
+                      loss_out, taps, streams, nullptr, perm);
 }
 
 extern "C" int64_t rtma_link_param_count(const rtma_model_desc* md, const rtma_decoder_desc* dd) {

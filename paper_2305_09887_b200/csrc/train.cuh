@@ -71,8 +71,10 @@ struct SplitPlan {
 };
 
 // ---- spmm.cu --------------------------------------------------------------------------
-// fp32 rows in partition order -> split planes in scratch rows.
-int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, int d, Planes out, cudaStream_t s);
+// fp32 rows in partition order (perm == NULL), or in node order with row i of the partition order at
+// X[perm[i]], -> split planes in scratch rows.
+int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, const int32_t* perm, int d, Planes out,
+                         cudaStream_t s);
 // Split planes -> dense fp32 [rows x d] (verification taps).
 int32_t launch_from_planes(rtma_ctx* ctx, Planes src, int64_t first_row, int64_t rows, int d, float* dst, cudaStream_t s);
 // inv_deg[row_ws + i] = 1 / local degree (0 for an isolated node).
@@ -120,6 +122,13 @@ int32_t launch_loss_finalize(rtma_ctx* ctx, const GroupDesc& g, const float* til
 int32_t launch_softmax_xent(rtma_ctx* ctx, const GroupDesc& g, Mat logits, int C, const int32_t* yp, Planes dZ,
                             float* tile_loss, float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s);
 
+// The head when the last layer's aggregate is taken after the product: scores = [Tself +] NT + b
+// (Tself.hi == NULL: one-matrix layer), at most 64 classes; dZ as above; scores.ptr != NULL records the
+// scores as fp32.
+int32_t launch_softmax_xent_head(rtma_ctx* ctx, const GroupDesc& g, Planes Tself, Planes NT, const float* params, int64_t P,
+                                 int64_t bias_offset, int C, const int32_t* yp, Planes dZ, Mat scores, float* tile_loss,
+                                 float* loss_out, int64_t loss_stride, int64_t loss_col, cudaStream_t s);
+
 // ---- post.cu (Layer Normalization before the activation, PReLU) ------------------------------
 int64_t post_tiles(const GroupDesc& g);
 // H = act(norm(Z)) for the layer's output; stats[row] = (mean, 1/std) when the layer normalises.
@@ -141,10 +150,21 @@ int32_t launch_pair_scatter(rtma_ctx* ctx, const GroupDesc& gd, const GroupDesc&
 int32_t launch_bce(rtma_ctx* ctx, const GroupDesc& gd, Planes S, const int32_t* label, float* tile_loss,
                    float* score_out, cudaStream_t s);
 
+// ---- dgrad_narrow.cu (the input gradient of a last layer with at most 8 products per output, on the ALUs) ----
+bool dgrad_narrow_applies(const LayerShape& ls);
+// H <- gate(dZ Ws^T + Q Wn^T) as split planes (one-matrix layers: Q W^T); gate as in launch_tc_dgrad
+int32_t launch_dgrad_narrow(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const float* params, Planes dZ, Planes Q,
+                            Planes H, bool gate, cudaStream_t s);
+
 // ---- optim.cu -------------------------------------------------------------------------
 // grad = sum of the part's chunk slots; params -= lr * grad; optionally records grad.
 int32_t launch_reduce_sgd(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, const float* partial,
                           float lr, float* params, float* grads_record, cudaStream_t s);
+// The same for the head form of the last layer: partial[slot] is [(d_in + 1) x 2 head_cp], the product of
+// [H | 1]^T with [dZ | Q]; columns c of the first block give dWs (and db in the last row), columns
+// head_cp + c give dWn (for a one-matrix layer dW, and the first block only gives db).
+int32_t launch_reduce_sgd_head(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int head_cp,
+                               const float* partial, float lr, float* params, float* grads_record, cudaStream_t s);
 int32_t launch_copy_rows(rtma_ctx* ctx, const float* src, int64_t ld_src, float* dst, int64_t ld_dst, int64_t rows,
                          int width, cudaStream_t s);
 
@@ -157,11 +177,15 @@ struct TcLayerPlan {
 };
 bool tc_available();
 TcLayerPlan tc_plan_layer(LayerShape ls);
+// The last layer with its aggregate taken after the product: forward operand [Ws | Wn] side by side in
+// blocks of head_cp columns (head_cp = the class count rounded up to 8), K = d_in alone.
+TcLayerPlan tc_plan_head(LayerShape ls, int head_cp);
 size_t tc_prep_elems(const TcLayerPlan& p, bool with_dgrad);  // bf16 elements per part, hi and lo together
 // Repack the weights of every listed layer, for every part, in one launch: transposed, zero padded,
 // split into hi / lo.  Bd_* may be NULL (no dgrad operand: the first layer).
 struct TcPrepJob {
     LayerShape ls;
+    int head_cp;  // 0: K-concatenated forward operand; > 0: the head form (tc_plan_head), blocks of head_cp columns
     TcLayerPlan plan;
     __nv_bfloat16 *Bf_hi, *Bf_lo, *Bd_hi, *Bd_lo;
 };

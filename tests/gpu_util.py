@@ -8,9 +8,14 @@ from paper_2305_09887_b200 import binding, inputs
 # relative = max|a-b| / max|b| per tensor
 TOL_ACT, TOL_GRAD, TOL_PARAM = 1e-4, 1e-3, 1e-3
 TOL_BF16 = 5e-3
-# bf16 operand mode against the oracle's own bf16 operand mode (same roundings, fp64 sums): what is
-# left is the kernel's fp32 accumulation and the few operands that round the other way
-TOL_BF16_SAME_ROUNDING = 5e-4
+# bf16 operand mode, layer by layer from the kernel's own recorded inputs (same operands, hence the same
+# roundings): what is left is fp32 accumulation against fp64
+TOL_BF16_LAYER = 5e-5
+# bf16 operand mode over a whole step against the oracle's bf16 operand mode.  Not tight: an activation
+# that differs by 1e-7 lands on the other side of a bf16 rounding boundary once in ten thousand and
+# then differs by 2^-8, which moves a whole row of the next layer by up to 3e-4 (and ReLU branches
+# flip the same way); measured 1e-3 .. 3e-3 on the named shapes.  Held to the mode's own bar.
+TOL_BF16_SAME_ROUNDING = TOL_BF16
 # branch flips seen per check (part, flipped units, hidden units), for the test log
 FLIP_LOG = []
 
@@ -174,7 +179,8 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, varia
         if flipped:
             o_loss, o_grads, _ = oracle.forward_backward_variant(variant, dims, rp, cp, X, y, p0, gates=gates)
         if gemm_dtype == 1 and variant == (0, 0, 0):
-            same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, loss[p, 0], grads[p])
+            same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, loss[p, 0], grads[p],
+                                assert_whole_step=gradients_against_plain)
         if n_p:
             assert abs(loss[p, 0] - o_loss) <= tol_loss * max(1.0, abs(o_loss)), p
         if not gradients_against_plain:
@@ -194,37 +200,75 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, varia
     return got, want
 
 
-def same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, gpu_loss, gpu_grads):
-    """bf16 operand mode against the oracle run with the same operand roundings: separates the
-    rounding the mode is allowed (2^-9 per operand, the 5e-3 bar) from anything else."""
+def _round_bf16(x):
+    """Round to nearest even into bf16 (the upper 16 bits of binary32), on the bits."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
+def layerwise_bf16_check(w, p, rp, cp, X, p0, gpu_acts):
+    """bf16 operand mode, one layer at a time from the kernel's own recorded inputs: the aggregate
+    A-bar H against the oracle's (it is not rounded), the layer output against the rounded-operand
+    product of the recorded H and A-bar H in fp64.  The last layer may be evaluated in either
+    association -- H Ws + (A-bar H) Wn or H Ws + A-bar (H Wn) -- which differ once operands are rounded."""
+    dims = w.dims
+    L = len(dims) - 1
+    r = _round_bf16
+    off = 0
+    worst = 0.0
+    for l in range(L):
+        di, dn = dims[l], dims[l + 1]
+        Ws = p0[off:off + di * dn].reshape(di, dn)
+        Wn = p0[off + di * dn:off + 2 * di * dn].reshape(di, dn)
+        b = p0[off + 2 * di * dn:off + 2 * di * dn + dn]
+        off += 2 * di * dn + dn
+        Hin = X if l == 0 else gpu_acts[f"H{l}"].astype(np.float64)
+        N = gpu_acts[f"N{l}"].astype(np.float64)
+        e_agg = rel_err(N, oracle.spmm_mean(rp, cp, Hin))
+        assert e_agg <= 2e-5, (p, f"N{l}", e_agg)
+        Z = r(Hin) @ r(Ws) + r(N) @ r(Wn) + b
+        got = gpu_acts[f"H{l + 1}"]
+        if l < L - 1:
+            e = rel_err(got, np.maximum(Z, 0.0))
+        else:
+            Z_after = r(Hin) @ r(Ws) + oracle.spmm_mean(rp, cp, r(Hin) @ r(Wn)) + b
+            e = min(rel_err(got, Z), rel_err(got, Z_after))
+        worst = max(worst, e, e_agg)
+        assert e <= TOL_BF16_LAYER, (p, f"H{l + 1}", e)
+    print(f"[bf16 layer by layer] {w.name} part {p}: worst {worst:.1e}")
+
+
+def same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, gpu_loss, gpu_grads, assert_whole_step=True):
+    """bf16 operand mode: layer by layer from the kernel's recorded inputs (tight), then the whole step
+    against the oracle run with the same operand roundings."""
+    layerwise_bf16_check(w, p, rp, cp, X, p0, gpu_acts)
     dims = w.dims
     tol = TOL_BF16_SAME_ROUNDING
     r_loss, r_grads, r_acts = oracle.forward_backward(dims, rp, cp, X, y, p0, want_acts=True, want_preact=True,
                                                       bf16_operands=True)
-    worst = 0.0
-    for name, a in gpu_acts.items():
-        e = rel_err(a, r_acts[name])
-        worst = max(worst, e)
-        assert e <= tol, (p, name, e)
+    errs = {name: rel_err(a, r_acts[name]) for name, a in gpu_acts.items()}
+    print(f"[same rounding] {w.name} part {p} activations: " + ", ".join(f"{k} {v:.1e}" for k, v in errs.items()))
     gates, flipped = [], 0
     for l in range(len(dims) - 2):
         Z = r_acts[f"Z{l + 1}"]
-        differ = (np.abs(Z) < 1e-4 * max(1.0, np.abs(Z).max(initial=0.0))) & ((gpu_acts[f"H{l + 1}"] > 0) != (Z > 0))
+        differ = (np.abs(Z) < 4e-3 * max(1.0, np.abs(Z).max(initial=0.0))) & ((gpu_acts[f"H{l + 1}"] > 0) != (Z > 0))
         flipped += int(differ.sum())
         g8 = np.full(Z.shape, -1, dtype=np.int8)
         g8[differ] = (gpu_acts[f"H{l + 1}"] > 0)[differ]
         gates.append(g8)
     if flipped:
         r_loss, r_grads, _ = oracle.forward_backward(dims, rp, cp, X, y, p0, gates=gates, bf16_operands=True)
-    if rp.size > 1:
-        assert abs(gpu_loss - r_loss) <= tol * max(1.0, abs(r_loss)), p
-    worst_g = 0.0
-    for nm, off, size in _param_segments((0, 0, 0), dims):
-        if np.abs(r_grads[off:off + size]).max() > 0:
-            e = rel_err(gpu_grads[off:off + size], r_grads[off:off + size])
-            worst_g = max(worst_g, e)
-            assert e <= tol, (p, nm, e)
-    print(f"[same rounding] {w.name} part {p}: activations {worst:.2e}, gradients {worst_g:.2e}, {flipped} branch flips")
+    gerrs = {nm: rel_err(gpu_grads[off:off + size], r_grads[off:off + size])
+             for nm, off, size in _param_segments((0, 0, 0), dims) if np.abs(r_grads[off:off + size]).max() > 0}
+    print(f"[same rounding] {w.name} part {p} gradients: " + ", ".join(f"{k} {v:.1e}" for k, v in gerrs.items()) +
+          f"; {flipped} branch flips")
+    if assert_whole_step:
+        assert max(errs.values()) <= tol, (p, errs)
+        if rp.size > 1:
+            assert abs(gpu_loss - r_loss) <= tol * max(1.0, abs(r_loss)), p
+        assert max(gerrs.values(), default=0.0) <= tol, (p, gerrs)
 
 
 def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_parts=None, variant=(0, 0, 0),

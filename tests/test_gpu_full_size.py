@@ -190,9 +190,10 @@ def test_large_shape_scaled(util):
     util.check_k_steps_and_average(w, got, want, w.K, only_parts=[21])
 
 
-@pytest.mark.skipif(os.environ.get("RTMA_TEST_LARGE") != "1",
-                    reason="25M nodes / 1.3B entries: ~10 min and ~60 GB of host memory to generate; set RTMA_TEST_LARGE=1")
+@pytest.mark.skipif(os.environ.get("RTMA_SKIP_LARGE") == "1",
+                    reason="25M nodes / 1.3B entries: about a minute on 16 host threads and ~40 GB of host memory")
 def test_large_full_size(util):
+    # the only shape whose feature (12.8 GB) and column (5.2 GB) arrays pass 2^31 bytes, with 64-bit row offsets
     w = inputs.large()
     got = util.gpu_preprocess(w)
     want = util.oracle_preprocess(w)
