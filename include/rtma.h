@@ -66,7 +66,9 @@ const char* rtma_last_error(const rtma_ctx* ctx);
 /* Synchronises the device and reports RTMA_ERR_TIMEOUT if any kernel launched through this
  * context since the last check gave up on one of its bounded device-side waits (the
  * tensor-core kernels wait on mbarriers with an iteration limit instead of spinning for
- * ever); RTMA_OK otherwise.  rtma_train_host calls it before returning.                    */
+ * ever), RTMA_ERR_INVALID_ARG if a local-training call since the last check was given a
+ * subgraph that is not symmetric; RTMA_OK otherwise.  rtma_train_host calls it before
+ * returning.                                                                               */
 int32_t rtma_check(rtma_ctx* ctx);
 /* Bytes of scratch currently held by the context.                                        */
 size_t rtma_workspace_bytes(const rtma_ctx* ctx);
@@ -196,6 +198,11 @@ typedef struct {
  *                                         subgraphs must be symmetric (undirected graph,
  *                                         both directions stored), as the paper's "simple
  *                                         graph" is; symmetric != 1 is RTMA_ERR_UNSUPPORTED.
+ *                                         The claim is verified on the device (a hash sum over
+ *                                         the entries against one over the reversed entries):
+ *                                         if it does not hold, the next rtma_check returns
+ *                                         RTMA_ERR_INVALID_ARG and the parameters written by
+ *                                         the call are not to be used.
  *   Xp [n][dims[0]] float, yp [n] int32   features / labels in partition order.
  *   params [M][P]                         in/out, one replica per trainer.
  *   loss_out [M][K] float or NULL         loss of every step of every trainer.

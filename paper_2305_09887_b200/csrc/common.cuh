@@ -26,8 +26,12 @@ struct ProfSpan {
 
 struct rtma_ctx {
     int device = 0;
+    int sm_count = 148;
     bool profiling = false;
-    int* error_word = nullptr;     // device word raised by a kernel whose bounded wait ran out
+    // device words: [0] raised by a kernel whose bounded wait ran out, [1] by the symmetry check of
+    // the local-training calls
+    int* error_word = nullptr;
+    bool rows_configured = false, wgrad_configured = false;  // shared-memory opt-in of the tensor-core kernels on this device
     int64_t launches[KC_COUNT] = {0};
     std::vector<ProfSpan> spans;        // recorded since the last read
     std::vector<cudaEvent_t> event_pool;  // spare events

@@ -12,6 +12,8 @@ extern "C" int32_t rtma_create(rtma_ctx** out, int32_t device, size_t workspace_
     if (cudaSetDevice(device) != cudaSuccess) return RTMA_ERR_CUDA;
     rtma_ctx* ctx = new rtma_ctx();
     ctx->device = device;
+    if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || ctx->sm_count <= 0)
+        ctx->sm_count = 148;
     ctx->pinned_bytes = 1 << 16;
     if (cudaMallocHost(&ctx->pinned, ctx->pinned_bytes) != cudaSuccess) {
         delete ctx;
@@ -69,12 +71,15 @@ extern "C" int32_t rtma_check(rtma_ctx* ctx) {
     if (!ctx) return RTMA_ERR_INVALID_ARG;
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
     RTMA_CUDA(ctx, cudaDeviceSynchronize());
-    int word = 0;
-    RTMA_CUDA(ctx, cudaMemcpy(&word, ctx->error_word, sizeof(int), cudaMemcpyDeviceToHost));
-    if (word != 0) {
-        cudaMemset(ctx->error_word, 0, sizeof(int));
-        return rtma_fail(ctx, RTMA_ERR_TIMEOUT, "a kernel gave up on a bounded wait (device error word %d)", word);
-    }
+    int word[2] = {0, 0};
+    RTMA_CUDA(ctx, cudaMemcpy(word, ctx->error_word, sizeof(word), cudaMemcpyDeviceToHost));
+    if (word[0] != 0 || word[1] != 0) cudaMemset(ctx->error_word, 0, sizeof(word));
+    if (word[0] != 0)
+        return rtma_fail(ctx, RTMA_ERR_TIMEOUT, "a kernel gave up on a bounded wait (device error word %d)", word[0]);
+    if (word[1] != 0)
+        return rtma_fail(ctx, RTMA_ERR_INVALID_ARG,
+                         "a local-training call was given a subgraph that is not symmetric (some entry (u,v) without (v,u)): "
+                         "its gradients are not those of the model");
     return RTMA_OK;
 }
 

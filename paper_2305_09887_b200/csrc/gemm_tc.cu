@@ -425,12 +425,17 @@ struct WgradArgs {
     int d_in, d_out, nsrc;
     int jt_per_src;   // 128-wide tiles over d_in, per source
     int n_atoms;      // 64-wide atoms over d_out (all column tiles together); a tile takes up to 4
+    int acc_cols;     // tensor-memory columns of one accumulator
     int tmem_cols, stages;
+    int bk;           // rows (k) per pipeline stage: 64 or 32
     int single;       // 1: operands rounded to bf16 (hi planes only)
     float* partial;   // [slot][(2 d_in + 1) x d_out]
     int* error_word;
 };
 
+// A block accumulates TWO 128-wide tiles of the left operand (both sources of a two-matrix layer, or
+// two neighbouring tiles of one source) against the same staged dZ tile, each into its own
+// accumulator: the dZ tile, the larger operand, crosses the shared-memory fill path once for both.
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_constant__ WgradArgs a) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ PipeBarriers pb;
@@ -441,9 +446,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     const int n_p = a.g.rows[k];
     const int v0 = min(n_p, chunk * a.sp.rows_per_split[k]);
     const int v1 = min(n_p, v0 + a.sp.rows_per_split[k]);
-    const int KB = (v1 - v0 + TC_BK - 1) / TC_BK;
-    const int src = blockIdx.x / a.jt_per_src;
-    const int j0 = (blockIdx.x % a.jt_per_src) * TC_BM;
+    const int BK = a.bk;
+    const int KB = (v1 - v0 + BK - 1) / BK;
+    const int total_a = a.nsrc * a.jt_per_src;                 // left-operand tiles of the layer
+    const int na_tiles = min(2, total_a - 2 * (int)blockIdx.x);  // of this block: 1 or 2
+    int src_of[2], j0_of[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int at = min(2 * (int)blockIdx.x + t, total_a - 1);
+        src_of[t] = at / a.jt_per_src;
+        j0_of[t] = (at % a.jt_per_src) * TC_BM;
+    }
     const int d_in = a.d_in, d_out = a.d_out;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cbase = blockIdx.z * 256;                       // first output column of this tile
@@ -453,10 +466,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     const bool bias_tile = blockIdx.x == 0;  // these blocks also produce the bias gradient of their columns
 
     if (KB == 0) {  // empty chunk: the gradient contribution is zero
-        for (int idx = threadIdx.x; idx < TC_BM * ccount; idx += TC_THREADS) {
-            const int j = j0 + idx / ccount;
-            if (j < d_in) P[(int64_t)(src * d_in + j) * d_out + cbase + idx % ccount] = 0.f;
-        }
+        for (int t = 0; t < na_tiles; ++t)
+            for (int idx = threadIdx.x; idx < TC_BM * ccount; idx += TC_THREADS) {
+                const int j = j0_of[t] + idx / ccount;
+                if (j < d_in) P[(int64_t)(src_of[t] * d_in + j) * d_out + cbase + idx % ccount] = 0.f;
+            }
         if (bias_tile)
             for (int c = threadIdx.x; c < ccount; c += TC_THREADS) P[(int64_t)a.nsrc * d_in * d_out + cbase + c] = 0.f;
         return;
@@ -464,12 +478,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 
     uint8_t* smem = align_1024(smem_raw);
     const int stages = a.stages, NA = min(4, a.n_atoms - 4 * (int)blockIdx.z);
-    constexpr uint32_t ATOM_BYTES = TC_BK * 128u;  // one 64-wide column of 64 k-rows: 8 KB
-    const uint32_t a_plane_bytes = 2u * ATOM_BYTES;
+    const uint32_t ATOM_BYTES = (uint32_t)BK * 128u;  // one 64-wide column of BK k-rows
+    const uint32_t a_tile_bytes = 2u * ATOM_BYTES;     // one plane of one left-operand tile
+    const uint32_t a_plane_bytes = 2u * a_tile_bytes;  // room for two tiles
     const uint32_t b_plane_bytes = (uint32_t)NA * ATOM_BYTES;
     const bool single = a.single != 0;
     const uint32_t np = single ? 1u : 2u;  // planes staged per operand
     const uint32_t stage_bytes = np * (a_plane_bytes + b_plane_bytes);
+    const uint32_t tx_bytes = np * ((uint32_t)na_tiles * a_tile_bytes + b_plane_bytes);
     auto a_hi = [&](int s) { return smem + (size_t)s * stage_bytes; };
     auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + a_plane_bytes; };
     auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + np * a_plane_bytes; };
@@ -483,8 +499,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
         tc::mbar_init(&pb.accum, 1);
         pb.abort = 0;
         tc::fence_barrier_init();
-        tc::prefetch_tensormap(src == 0 ? &a.mapHh : &a.mapNh);
-        tc::prefetch_tensormap(src == 0 ? &a.mapHl : &a.mapNl);
+        tc::prefetch_tensormap(&a.mapHh);
+        tc::prefetch_tensormap(&a.mapNh);
         tc::prefetch_tensormap(&a.mapZh);
         tc::prefetch_tensormap(&a.mapZl);
     }
@@ -499,20 +515,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
-            const CUtensorMap* mapAh = src == 0 ? &a.mapHh : &a.mapNh;
-            const CUtensorMap* mapAl = src == 0 ? &a.mapHl : &a.mapNl;
             const int row = (int)(a.g.row_ws[k] + v0);
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % stages;
                 if (!wait_or_abort(&pb.empty[s], ((kb / stages) & 1) ^ 1, &pb, a.error_word)) break;
-                tc::mbar_arrive_expect_tx(&pb.full[s], stage_bytes);
-                for (int t = 0; t < 2; ++t) {
-                    tc::tma_load_2d(a_hi(s) + t * ATOM_BYTES, mapAh, &pb.full[s], j0 + 64 * t, row + kb * TC_BK);
-                    if (!single) tc::tma_load_2d(a_lo(s) + t * ATOM_BYTES, mapAl, &pb.full[s], j0 + 64 * t, row + kb * TC_BK);
+                tc::mbar_arrive_expect_tx(&pb.full[s], tx_bytes);
+                for (int t = 0; t < na_tiles; ++t) {
+                    const CUtensorMap* mapAh = src_of[t] == 0 ? &a.mapHh : &a.mapNh;
+                    const CUtensorMap* mapAl = src_of[t] == 0 ? &a.mapHl : &a.mapNl;
+                    for (int h = 0; h < 2; ++h) {
+                        tc::tma_load_2d(a_hi(s) + t * a_tile_bytes + h * ATOM_BYTES, mapAh, &pb.full[s], j0_of[t] + 64 * h, row + kb * BK);
+                        if (!single)
+                            tc::tma_load_2d(a_lo(s) + t * a_tile_bytes + h * ATOM_BYTES, mapAl, &pb.full[s], j0_of[t] + 64 * h, row + kb * BK);
+                    }
                 }
                 for (int t = 0; t < NA; ++t) {
-                    tc::tma_load_2d(b_hi(s) + t * ATOM_BYTES, &a.mapZh, &pb.full[s], cbase + 64 * t, row + kb * TC_BK);
-                    if (!single) tc::tma_load_2d(b_lo(s) + t * ATOM_BYTES, &a.mapZl, &pb.full[s], cbase + 64 * t, row + kb * TC_BK);
+                    tc::tma_load_2d(b_hi(s) + t * ATOM_BYTES, &a.mapZh, &pb.full[s], cbase + 64 * t, row + kb * BK);
+                    if (!single) tc::tma_load_2d(b_lo(s) + t * ATOM_BYTES, &a.mapZl, &pb.full[s], cbase + 64 * t, row + kb * BK);
                 }
             }
         }
@@ -523,19 +542,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                 const int s = kb % stages;
                 if (!wait_or_abort(&pb.full[s], (kb / stages) & 1, &pb, a.error_word)) break;
                 tc::tc_fence_after_sync();
-                const uint32_t ah = tc::smem_u32(a_hi(s)), al = tc::smem_u32(a_lo(s));
                 const uint32_t bh = tc::smem_u32(b_hi(s)), bl = tc::smem_u32(b_lo(s));
-#pragma unroll
-                for (int ks = 0; ks < TC_BK / 16; ++ks) {
+                for (int ks = 0; ks < BK / 16; ++ks) {
                     const uint32_t off = ks * 2048;  // 16 k-rows of 128 bytes
-                    const uint64_t dah = tc::smem_desc_sw128(ah + off, ATOM_BYTES, 1024), dbh = tc::smem_desc_sw128(bh + off, ATOM_BYTES, 1024);
-                    if (single) {
-                        tc::mma_bf16(tmem_base, dah, dbh, idesc, (kb | ks) ? 1u : 0u);
-                    } else {
-                        const uint64_t dal = tc::smem_desc_sw128(al + off, ATOM_BYTES, 1024), dbl = tc::smem_desc_sw128(bl + off, ATOM_BYTES, 1024);
-                        tc::mma_bf16(tmem_base, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
-                        tc::mma_bf16(tmem_base, dah, dbl, idesc, 1u);
-                        tc::mma_bf16(tmem_base, dah, dbh, idesc, 1u);
+                    const uint64_t dbh = tc::smem_desc_sw128(bh + off, ATOM_BYTES, 1024);
+                    const uint64_t dbl = tc::smem_desc_sw128(bl + off, ATOM_BYTES, 1024);
+                    for (int t = 0; t < na_tiles; ++t) {
+                        const uint32_t d_tmem = tmem_base + (uint32_t)(t * a.acc_cols);
+                        const uint32_t ah = tc::smem_u32(a_hi(s) + t * a_tile_bytes), al = tc::smem_u32(a_lo(s) + t * a_tile_bytes);
+                        const uint64_t dah = tc::smem_desc_sw128(ah + off, ATOM_BYTES, 1024);
+                        if (single) {
+                            tc::mma_bf16(d_tmem, dah, dbh, idesc, (kb | ks) ? 1u : 0u);
+                        } else {
+                            const uint64_t dal = tc::smem_desc_sw128(al + off, ATOM_BYTES, 1024);
+                            tc::mma_bf16(d_tmem, dal, dbh, idesc, (kb | ks) ? 1u : 0u);
+                            tc::mma_bf16(d_tmem, dah, dbl, idesc, 1u);
+                            tc::mma_bf16(d_tmem, dah, dbh, idesc, 1u);
+                        }
                     }
                 }
                 tc::mma_commit(&pb.empty[s]);
@@ -545,9 +568,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
     } else {
         const int tw = threadIdx.x - 64;  // 0..127
         // Bias gradient = column sums of dZ.  While the MMAs run, the epilogue warps of the bias
-        // blocks add up the dZ tiles sitting in shared memory.  In an 8 KB atom a 16-byte chunk id
+        // blocks add up the dZ tiles sitting in shared memory.  In an atom a 16-byte chunk id
         // is (k-row r = id / 8, stored chunk s = id % 8) and holds logical chunk s ^ (r % 8).
-        // Thread tw takes ids tw, tw + 128, tw + 256, tw + 384: rows tw / 8 + 16 i, which agree
+        // Thread tw takes ids tw, tw + 128, ...: rows tw / 8 + 16 i, which agree
         // mod 8, so it always sums the same 8 columns of every atom.
         float colsum[4][8];
 #pragma unroll
@@ -565,8 +588,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
                     if (t < NA) {
                         const uint4* bh = reinterpret_cast<const uint4*>(b_hi(s) + t * ATOM_BYTES);
                         const uint4* bl = reinterpret_cast<const uint4*>(b_lo(s) + t * ATOM_BYTES);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
+                        for (int i = 0; i < BK / 16; ++i) {
                             Pack8 p;
                             p.zero();
                             p.add_planes(bh[tw + 128 * i], single ? make_uint4(0u, 0u, 0u, 0u) : bl[tw + 128 * i]);
@@ -599,22 +621,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_wgrad_kernel(const __grid_co
         }
         if (ok) {
             const int q = warp & 3;
-            const int j = j0 + q * 32 + lane;
-            const bool live = j < d_in;
-            float* o = P + (int64_t)(src * d_in + j) * d_out + cbase;
             const bool vec_ok = (d_out % 4 == 0) && (reinterpret_cast<uintptr_t>(P) % 16 == 0);
-            for (int c0 = 0; c0 < 64 * NA; c0 += 32) {
-                float v[32];
-                tc::tmem_load_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-                if (!live) continue;
+            for (int t = 0; t < na_tiles; ++t) {
+                const int j = j0_of[t] + q * 32 + lane;
+                const bool live = j < d_in;
+                float* o = P + (int64_t)(src_of[t] * d_in + j) * d_out + cbase;
+                for (int c0 = 0; c0 < 64 * NA; c0 += 32) {
+                    float v[32];
+                    tc::tmem_load_32x32(tmem_base + (uint32_t)(t * a.acc_cols) + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+                    if (!live) continue;
 #pragma unroll
-                for (int jj = 0; jj < 32; jj += 4) {
-                    const int c = c0 + jj;
-                    if (c >= ccount) break;
-                    if (vec_ok && c + 3 < ccount) {
-                        *reinterpret_cast<float4*>(o + c) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
-                    } else {
-                        for (int e = 0; e < 4 && c + e < ccount; ++e) o[c + e] = v[jj + e];
+                    for (int jj = 0; jj < 32; jj += 4) {
+                        const int c = c0 + jj;
+                        if (c >= ccount) break;
+                        if (vec_ok && c + 3 < ccount) {
+                            *reinterpret_cast<float4*>(o + c) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
+                        } else {
+                            for (int e = 0; e < 4 && c + e < ccount; ++e) o[c + e] = v[jj + e];
+                        }
                     }
                 }
             }
@@ -691,16 +715,6 @@ int32_t set_smem_limit(rtma_ctx* ctx, const void* kernel) {
     return RTMA_OK;
 }
 
-int sm_count_of(int device) {
-    static int cached = 0;
-    if (!cached) {
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || v <= 0) v = 148;
-        cached = v;
-    }
-    return cached;
-}
-
 bool plane_maps(CUtensorMap* hi, CUtensorMap* lo, Planes p, uint64_t rows, uint64_t cols, uint32_t box_cols,
                 uint32_t box_rows) {
     return make_tensor_map_bf16(hi, p.hi, rows, cols, p.ld, box_cols, box_rows) &&
@@ -766,13 +780,12 @@ int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, const TcPrepJob
 }
 
 static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
+    if (!ctx->rows_configured) {  // per device: the context is bound to one
         RTMA_CUDA(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(tc_rows_kernel<true>),
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, ROWS_SMEM_MAX));
         RTMA_CUDA(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(tc_rows_kernel<false>),
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, ROWS_SMEM_MAX));
-        configured = true;
+        ctx->rows_configured = true;
     }
     const size_t stage_bytes = (a.single ? 1 : 2) * ((size_t)PLANE_TILE_BYTES + (size_t)a.BN * 128);
     a.stages = std::max(1, std::min<int>(MAX_STAGES, (int)(ROWS_RING_BUDGET / stage_bytes)));
@@ -781,7 +794,7 @@ static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t 
     a.row_tiles = group_tiles(a.g, TC_BM);
     if (a.row_tiles == 0) return RTMA_OK;
     const int64_t total_tiles = a.row_tiles * (a.Npad / a.BN);
-    const unsigned grid = (unsigned)std::min<int64_t>(total_tiles, sm_count_of(ctx->device));
+    const unsigned grid = (unsigned)std::min<int64_t>(total_tiles, ctx->sm_count);
     // the epilogue staging slabs are only allocated for plane output: shared memory comes out of L1
     {
         KernelScope ks(ctx, kclass, s);
@@ -860,12 +873,15 @@ int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const 
     return launch_rows(ctx, a, KC_GEMM_DGRAD, s);
 }
 
+int tc_wgrad_blocks_per_slot(const LayerShape& ls) {
+    return (int)(ceil_div(ls.nsrc * ceil_div(ls.d_in, TC_BM), 2) * ceil_div(ceil_div(ls.d_out, 64), 4));
+}
+
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,
                         Planes H, Planes N, Planes dZ, float* partial, bool single, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
+    if (!ctx->wgrad_configured) {
         RTMA_TRY(set_smem_limit(ctx, reinterpret_cast<const void*>(tc_wgrad_kernel)));
-        configured = true;
+        ctx->wgrad_configured = true;
     }
     const int slots = sp.split_begin[g.num];
     if (slots == 0) return RTMA_OK;
@@ -873,27 +889,33 @@ int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, 
     WgradArgs a{};
     a.g = g;
     a.sp = sp;
-    if (!plane_maps(&a.mapHh, &a.mapHl, H, rows_total, ls.d_in, 64, TC_BK) ||
-        !plane_maps(&a.mapNh, &a.mapNl, N, rows_total, ls.d_in, 64, TC_BK) ||
-        !plane_maps(&a.mapZh, &a.mapZl, dZ, rows_total, ls.d_out, 64, TC_BK))
-        return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the wgrad operands");
     a.d_in = ls.d_in;
     a.d_out = ls.d_out;
     a.nsrc = ls.nsrc;
+    a.jt_per_src = (int)ceil_div(ls.d_in, TC_BM);
+    a.n_atoms = (int)ceil_div(ls.d_out, 64);
+    const int tile_atoms = a.n_atoms < 4 ? a.n_atoms : 4;
+    a.acc_cols = 64 * tile_atoms;
+    a.tmem_cols = (int)tmem_columns_for(2 * a.acc_cols);  // two accumulators, at most 512 columns
+    a.single = single ? 1 : 0;
+    // a stage = two left-operand tiles and the dZ tile, BK rows deep; 32-row stages where 64-row ones
+    // would leave fewer than three of them
+    const size_t stage64 = (single ? 1 : 2) * ((size_t)4 + (size_t)tile_atoms) * 64 * 128;
+    a.bk = SMEM_BUDGET / stage64 >= 3 ? 64 : 32;
+    const size_t stage_bytes = stage64 * a.bk / 64;
+    a.stages = stages_for(stage_bytes, MAX_STAGES);
+    a.partial = partial;
+    a.error_word = ctx->error_word;
+    // boxes of 64 columns x BK rows: one atom of a stage
+    if (!plane_maps(&a.mapHh, &a.mapHl, H, rows_total, ls.d_in, 64, (uint32_t)a.bk) ||
+        !plane_maps(&a.mapNh, &a.mapNl, N, rows_total, ls.d_in, 64, (uint32_t)a.bk) ||
+        !plane_maps(&a.mapZh, &a.mapZl, dZ, rows_total, ls.d_out, 64, (uint32_t)a.bk))
+        return rtma_fail(ctx, RTMA_ERR_CUDA, "cuTensorMapEncodeTiled refused the wgrad operands");
     if (ls.nsrc == 1) {  // the aggregate is the only source
         a.mapHh = a.mapNh;
         a.mapHl = a.mapNl;
     }
-    a.jt_per_src = (int)ceil_div(ls.d_in, TC_BM);
-    a.n_atoms = (int)ceil_div(ls.d_out, 64);
-    const int tile_atoms = a.n_atoms < 4 ? a.n_atoms : 4;
-    a.tmem_cols = (int)tmem_columns_for(64 * tile_atoms);
-    a.single = single ? 1 : 0;
-    const size_t stage_bytes = (single ? 1 : 2) * ((size_t)2 + (size_t)tile_atoms) * TC_BK * 128;
-    a.stages = stages_for(stage_bytes, MAX_STAGES);
-    a.partial = partial;
-    a.error_word = ctx->error_word;
-    dim3 grid((unsigned)(ls.nsrc * a.jt_per_src), (unsigned)slots, (unsigned)ceil_div(a.n_atoms, 4));
+    dim3 grid((unsigned)ceil_div(ls.nsrc * a.jt_per_src, 2), (unsigned)slots, (unsigned)ceil_div(a.n_atoms, 4));
     { KernelScope ks(ctx, KC_GEMM_WGRAD, s); tc_wgrad_kernel<<<grid, TC_THREADS, a.stages * stage_bytes + 1024, s>>>(a); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;

@@ -125,6 +125,13 @@ gather_rows_kernel(int64_t n, int64_t row_bytes, const char* __restrict__ src, c
     }
 }
 
+// rows of 4 bytes (labels, ids): one thread per row
+__global__ void __launch_bounds__(256)
+gather_words_kernel(int64_t n, const int32_t* __restrict__ src, const int32_t* __restrict__ perm, int32_t* __restrict__ dst) {
+    const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i < n) dst[i] = __ldg(src + perm[i]);
+}
+
 }  // namespace
 
 extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_64, const void* rowptr,
@@ -205,7 +212,9 @@ extern "C" int32_t rtma_gather_rows(rtma_ctx* ctx, int64_t n, int64_t row_bytes,
     RTMA_TRY(order_after_training(ctx, stream));
     const unsigned blocks = (unsigned)ceil_div(n, 8);
     const uintptr_t align = reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst) | (uintptr_t)row_bytes;
-    if (align % 16 == 0)
+    if (row_bytes == 4 && align % 4 == 0)
+        { KernelScope ks(ctx, KC_GATHER_ROWS, stream); gather_words_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, stream>>>(n, static_cast<const int32_t*>(src), perm, static_cast<int32_t*>(dst)); }
+    else if (align % 16 == 0)
         { KernelScope ks(ctx, KC_GATHER_ROWS, stream); gather_rows_kernel<16><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst)); }
     else if (align % 4 == 0)
         { KernelScope ks(ctx, KC_GATHER_ROWS, stream); gather_rows_kernel<4><<<blocks, 256, 0, stream>>>(n, row_bytes, static_cast<const char*>(src), perm, static_cast<char*>(dst)); }

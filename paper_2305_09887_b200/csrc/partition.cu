@@ -28,9 +28,19 @@ __device__ __forceinline__ uint64_t splitmix64_step(uint64_t x) {
     return z ^ (z >> 31);
 }
 
-__device__ __forceinline__ int part_of(int64_t v, const int32_t* __restrict__ group_id, uint64_t seed, int M) {
+// x mod M without a 64-bit division per node.  magic = ceil(2^64 / M) (mod_magic, computed once per
+// thread); q = floor(x * magic / 2^64) is floor(x / M) or one more (the error x * (magic - 2^64 / M) /
+// 2^64 is below 1), so x - q M is the remainder or the remainder minus M.
+__device__ __forceinline__ uint64_t mod_magic(int M) { return M > 1 ? ~0ULL / (uint64_t)M + 1ULL : 0ULL; }
+__device__ __forceinline__ int mod_small(uint64_t x, int M, uint64_t magic) {
+    const uint64_t q = __umul64hi(x, magic);
+    const int64_t r = (int64_t)(x - q * (uint64_t)M);   // M = 1: magic 0, q 0, x - 0 = x -> handled below
+    return M > 1 ? (int)(r < 0 ? r + M : r) : 0;
+}
+
+__device__ __forceinline__ int part_of(int64_t v, const int32_t* __restrict__ group_id, uint64_t seed, int M, uint64_t magic) {
     const uint64_t g = group_id ? (uint64_t)(int64_t)group_id[v] : (uint64_t)v;
-    return (int)(splitmix64_step(seed ^ g) % (uint64_t)M);
+    return mod_small(splitmix64_step(seed ^ g), M, magic);
 }
 
 __global__ void __launch_bounds__(PART_THREADS)
@@ -42,9 +52,10 @@ part_count_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t seed
     for (int b = lane; b <= RTMA_MAX_PARTS; b += 32) hist[warp][b] = 0;
     __syncwarp();
     if (chunk >= num_chunks) return;
+    const uint64_t magic = mod_magic(M);
     for (int r = 0; r < PART_ROUNDS; ++r) {
         const int64_t pos = chunk * PART_CHUNK + r * 32 + lane;  // position in the input order (node id if none is given)
-        const int pid = pos < n ? part_of(order_in ? order_in[pos] : pos, group_id, seed, M) : M;
+        const int pid = pos < n ? part_of(order_in ? order_in[pos] : pos, group_id, seed, M, magic) : M;
         const unsigned peers = __match_any_sync(0xffffffffu, pid);
         if (lane == __ffs(peers) - 1) hist[warp][pid] += __popc(peers);
         __syncwarp();
@@ -70,11 +81,12 @@ part_scatter_kernel(int64_t n, const int32_t* __restrict__ group_id, uint64_t se
     __syncthreads();
     if (chunk >= num_chunks) return;
     const unsigned below = (1u << lane) - 1u;
+    const uint64_t magic = mod_magic(M);
     for (int r = 0; r < PART_ROUNDS; ++r) {
         const int64_t pos = chunk * PART_CHUNK + r * 32 + lane;
         const bool live = pos < n;
         const int64_t v = live && order_in ? order_in[pos] : pos;
-        const int pid = live ? part_of(v, group_id, seed, M) : M;
+        const int pid = live ? part_of(v, group_id, seed, M, magic) : M;
         const unsigned peers = __match_any_sync(0xffffffffu, pid);
         const int slot = live ? cursor[warp][pid] + __popc(peers & below) : 0;
         __syncwarp();

@@ -136,6 +136,56 @@ locality_probe_kernel(const __grid_constant__ GroupDesc g, const int64_t* __rest
     }
 }
 
+// Is every part's subgraph symmetric?  The backward pass reuses the forward CSR for Abar^T, which is
+// only right when every entry (u, v) comes with (v, u).  The multiset of entries equals the multiset
+// of reversed entries exactly when two sums of a 64-bit hash over (part, row, column) and over
+// (part, column, row) agree (up to a collision chance of about 2^-64); the last block to finish
+// compares them and raises flag[0] when they differ.
+__device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
+    x ^= x >> 33;
+    x *= 0xff51afd7ed558ccdULL;
+    x ^= x >> 33;
+    x *= 0xc4ceb9fe1a85ec53ULL;
+    x ^= x >> 33;
+    return x;
+}
+__global__ void __launch_bounds__(256)
+symmetry_check_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
+                      const int32_t* __restrict__ col_out, unsigned long long* __restrict__ sums, int* __restrict__ flag) {
+    unsigned long long fwd = 0, rev = 0;
+    int k, r0;
+    if (locate_tile(g, 256, blockIdx.x, &k, &r0)) {
+        const int i = r0 + threadIdx.x;
+        if (i < g.rows[k]) {
+            const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
+            const int32_t* cols = col_out + g.edge_abs[k];
+            const unsigned long long tag = (unsigned long long)(g.part[k] + 1) << 58;
+            for (int64_t e = rp[i]; e < rp[i + 1]; ++e) {
+                const unsigned long long c = (unsigned long long)(uint32_t)cols[e], r = (unsigned long long)(uint32_t)i;
+                fwd += mix64(tag ^ (r << 29) ^ c * 0x9E3779B97F4A7C15ULL);
+                rev += mix64(tag ^ (c << 29) ^ r * 0x9E3779B97F4A7C15ULL);
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        fwd += __shfl_xor_sync(0xffffffffu, fwd, o);
+        rev += __shfl_xor_sync(0xffffffffu, rev, o);
+    }
+    if ((threadIdx.x & 31) == 0) {  // integer sums: their order does not matter
+        atomicAdd(sums, fwd);
+        atomicAdd(sums + 1, rev);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(sums + 2, 1ULL) == gridDim.x - 1) {
+            __threadfence();
+            if (atomicAdd(sums, 0ULL) != atomicAdd(sums + 1, 0ULL)) atomicExch(flag, 1);
+        }
+    }
+}
+
 // MODE 0: out[v] = w[v] * sum_u src[u]                      (w = 1 / deg)
 // MODE 1: out[v] = sum_u w[u] * src[u]                      (w = 1 / deg)
 // MODE 2: out[v] = w[v] * (w[v] * src[v] + sum_u w[u] * src[u])   (w = (deg + 1)^-1/2)
@@ -556,14 +606,77 @@ spmm_narrow_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restric
         spmm_narrow_rows<LPR, MODE, false>(g, rowptr_out, col_out, inv_deg, src, out, d, total_groups, order, ticket);
 }
 
+// Rows of at most 8 values (one 16-byte piece per plane; two-class heads): one THREAD per row.  With a
+// handful of neighbours per row and 32 bytes to fetch from each, handing rows out to warps costs more
+// than the work; here the offsets, the weights and the results are coalesced over the warp's 32 rows and
+// every thread walks its own entries, four neighbours in flight.  A hub row keeps its warp busy for as
+// many rounds as it has entries, which a launch of hundreds of thousands of warps absorbs.
+constexpr int TINY_TILE_ROWS = 256;
+template <int MODE>
+__global__ void __launch_bounds__(TINY_TILE_ROWS)
+spmm_tiny_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
+                 const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out) {
+    int k, r0;
+    if (!locate_tile(g, TINY_TILE_ROWS, blockIdx.x, &k, &r0)) return;
+    const int i = r0 + threadIdx.x;
+    if (i >= g.rows[k]) return;
+    const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
+    const int64_t ws = g.row_ws[k];
+    const int32_t* cols = col_out + g.edge_abs[k];
+    const int64_t b = rp[i], e = rp[i + 1];
+    const __nv_bfloat16* sh = src.hi + ws * src.ld;
+    const __nv_bfloat16* sl = src.lo + ws * src.ld;
+    const float* wv = inv_deg + ws;
+    Pack8 acc;
+    acc.zero();
+    for (int64_t t = b; t < e; t += 4) {
+        int32_t nb[4];
+        float wt[4];
+        uint4 xh[4], xl[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) nb[j] = t + j < e ? __ldg(cols + t + j) : -1;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (nb[j] >= 0) {
+                if (MODE != 0) wt[j] = __ldg(wv + nb[j]);
+                xh[j] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)nb[j] * src.ld));
+                xl[j] = __ldg(reinterpret_cast<const uint4*>(sl + (int64_t)nb[j] * src.ld));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (nb[j] >= 0) {
+                if (MODE != 0) acc.fma_planes_mixed(wt[j], xh[j], xl[j]);
+                else acc.add_planes_mixed(xh[j], xl[j]);
+            }
+        }
+    }
+    const float w = MODE == 1 ? 1.f : wv[i];
+    if (MODE == 2)  // the self loop
+        acc.fma_planes_mixed(w, *reinterpret_cast<const uint4*>(sh + (int64_t)i * src.ld), *reinterpret_cast<const uint4*>(sl + (int64_t)i * src.ld));
+    if (MODE != 1) {
+#pragma unroll
+        for (int v = 0; v < 8; ++v) acc.v[v] *= w;
+    }
+    uint4 h, l;
+    acc.to_planes_lean(h, l);
+    *reinterpret_cast<uint4*>(out.hi + (ws + i) * out.ld) = h;
+    *reinterpret_cast<uint4*>(out.lo + (ws + i) * out.ld) = l;
+}
+
 template <int MODE>
 int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                       const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket, cudaStream_t s) {
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
     if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
-    static int sms = 0;
-    if (!sms && (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess || sms <= 0)) sms = 148;
+    if (d <= 8) {
+        const int64_t tiles = group_tiles(g, TINY_TILE_ROWS);
+        { KernelScope ks(ctx, kclass, s); spmm_tiny_kernel<MODE><<<(unsigned)tiles, TINY_TILE_ROWS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out); }
+        RTMA_LAUNCH_CHECK(ctx);
+        return RTMA_OK;
+    }
+    const int sms = ctx->sm_count;
     const int blocks_per_sm = d <= 256 ? 2 : 1;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(groups, SPMM_THREADS / 32), (int64_t)sms * blocks_per_sm);
 #define RTMA_SPMM(N)                                                                                      \
@@ -600,6 +713,15 @@ int32_t launch_from_planes(rtma_ctx* ctx, Planes src, int64_t first_row, int64_t
     if (rows <= 0 || d <= 0) return RTMA_OK;
     const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(rows * d, 256), 148 * 16);
     { KernelScope ks(ctx, KC_COPY, s); from_planes_kernel<<<grid, 256, 0, s>>>(src, first_row, rows, d, dst); }
+    RTMA_LAUNCH_CHECK(ctx);
+    return RTMA_OK;
+}
+
+int32_t launch_symmetry_check(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                              unsigned long long* sums, cudaStream_t s) {
+    const int64_t tiles = group_tiles(g, 256);
+    if (tiles == 0) return RTMA_OK;
+    { KernelScope ks(ctx, KC_INV_DEGREE, s); symmetry_check_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, rowptr_out, col_out, sums, ctx->error_word + 1); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

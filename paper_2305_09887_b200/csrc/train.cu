@@ -1,6 +1,7 @@
 // Host-side sequencing of Algorithm 2's loop body for M trainers on one GPU: K plain-SGD
 // steps of a GraphSAGE-mean (or GCN) network on every part, trainers grouped by stream.
 #include <algorithm>
+#include <cstdint>
 #include <vector>
 
 #include "train.cuh"
@@ -147,20 +148,31 @@ ScratchPlan plan_scratch(const Model& m, bool head, bool record) {
 
 // Row chunks of the weight gradient: enough of them to give the GPU a few blocks per SM,
 // each a multiple of the row alignment.
-int splits_for(int64_t n_p, int parts_in_flight) {
-    const int64_t want = std::max<int64_t>(1, 296 / std::max(1, 4 * parts_in_flight));
-    const int64_t by_rows = std::max<int64_t>(1, ceil_div(n_p, 1024));
-    return (int)std::min<int64_t>(64, std::min(want, by_rows));
+int splits_for(int64_t n_p, int parts_in_flight, int blocks_per_slot) {
+    // The kernel runs one block per SM at a time, so its time goes as (waves of blocks) x (rows per
+    // chunk).  Taking every part for as large as this one, pick the chunk count with the smallest such
+    // product, or the fewest chunks within 3 % of it (fewer partial sums to add up afterwards).
+    constexpr int64_t SMS = 148;
+    const int64_t most = std::min<int64_t>(64, std::max<int64_t>(1, ceil_div(n_p, 1024)));
+    auto cost_of = [&](int64_t ns) {
+        const int64_t rows = aligned_rows(ceil_div(n_p, ns));
+        const int64_t blocks = (int64_t)parts_in_flight * ceil_div(n_p, rows) * blocks_per_slot;
+        return ceil_div(blocks, SMS) * rows;
+    };
+    int64_t best_cost = INT64_MAX;
+    for (int64_t ns = 1; ns <= most; ++ns) best_cost = std::min(best_cost, cost_of(ns));
+    for (int64_t ns = 1; ns <= most; ++ns)
+        if (cost_of(ns) * 100 <= best_cost * 103) return (int)ns;
+    return (int)most;
 }
 
-// parts_in_flight: all trainers that run in this call, whatever their stream and wave, so that a
-// part's chunking (hence the order of its gradient sums) does not depend on how the trainers were
-// spread over streams or cut into waves
-int plan_splits(const GroupDesc& g, int parts_in_flight, SplitPlan* sp) {
+// blocks_per_slot: blocks the weight-gradient kernel launches per chunk for the layer in hand (the
+// chunks of all running parts together should come to about two blocks per SM)
+int plan_splits(const GroupDesc& g, int parts_in_flight, int blocks_per_slot, SplitPlan* sp) {
     int slots = 0;
     for (int k = 0; k < g.num; ++k) {
         sp->split_begin[k] = slots;
-        const int nsplit = splits_for(g.rows[k], parts_in_flight);
+        const int nsplit = splits_for(g.rows[k], parts_in_flight, blocks_per_slot);
         sp->rows_per_split[k] = (int32_t)std::max<int64_t>(GROUP_ROW_ALIGN, aligned_rows(ceil_div(g.rows[k], nsplit)));
         slots += (int)std::max<int64_t>(1, ceil_div(g.rows[k], sp->rows_per_split[k]));
     }
@@ -311,7 +323,6 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             // ---- form a wave ----
             GroupDesc g{};
             GroupDesc gd{};   // link prediction: the same parts' pairs
-            SplitPlan sp{};
             size_t bytes = 0;
             int64_t rows = 0, prows = 0;
             while (at < parts.size()) {
@@ -337,7 +348,17 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 bytes += b;
                 ++at;
             }
-            const int slots = plan_splits(g, running, &sp);
+            // one chunking per layer: the number of blocks per chunk depends on the layer's shape
+            SplitPlan wave_spl[RTMA_MAX_LAYERS];
+            int slots = 0;
+            for (int l = 0; l < m.L; ++l) {
+                LayerShape shape = m.layer[l];
+                if (head && l == m.L - 1) {  // the head form's weight gradient: H^T [dZ | Q]
+                    shape.nsrc = 1;
+                    shape.d_out = 2 * m.Cp;
+                }
+                slots = std::max(slots, plan_splits(g, running, tc_wgrad_blocks_per_slot(shape), &wave_spl[l]));
+            }
             int wave_steps = 0;
             for (int k = 0; k < g.num; ++k) wave_steps = std::max(wave_steps, steps[g.part[k]]);
 
@@ -402,7 +423,10 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                     El[k] = take_pair_planes(m.ddims[k]);
                     ZDl[k] = take_pair_planes(m.ddims[k + 1]);
                 }
-                const int dslots = plan_splits(gd, running, &spd);
+                int dslots = 0;  // one chunking for all decoder layers: that of the layer with the most blocks per chunk
+                int dec_bps = 1;
+                for (int k = 0; k < m.Kd; ++k) dec_bps = std::max(dec_bps, tc_wgrad_blocks_per_slot(m.dec[k]));
+                dslots = plan_splits(gd, running, dec_bps, &spd);
                 dec_partial = cur.take<float>((size_t)dslots * plan.max_layer_params + 4);
                 dec_tile_loss = cur.take<float>((size_t)loss_tiles(gd) + 4);
             }
@@ -412,6 +436,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             float* partial = cur.take<float>((size_t)slots * plan.max_layer_params + 4);
             float* tile_loss = cur.take<float>((size_t)loss_tiles(g) + 4);
             int* ticket = cur.take<int>(64);  // work counter of the aggregation kernels (zero between launches)
+            unsigned long long* sym_sums = cur.take<unsigned long long>(4);
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
             int* heavy_list = cur.take<int>((size_t)spmm_order_entries(g) + 4);
             float* post_partial = m.post ? cur.take<float>((size_t)post_tiles(g) * (2 * plan.post_width + 1) + 4) : nullptr;
@@ -445,6 +470,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             RTMA_CUDA(ctx, cudaMemsetAsync(ctx->arena + gi * share, 0, zero_bytes, s));
             if (m.gcn) RTMA_TRY(launch_gcn_scale(ctx, g, rowptr_out, inv_deg, s));  // (deg + 1)^-1/2 in the same array
             else RTMA_TRY(launch_inv_degree(ctx, g, rowptr_out, inv_deg, s));
+            RTMA_TRY(launch_symmetry_check(ctx, g, rowptr_out, col_out, sym_sums, s));
             int64_t wave_entries = 0;
             for (int k = 0; k < g.num; ++k) wave_entries += edge_offsets[g.part[k] + 1] - edge_offsets[g.part[k]];
             SpmmOrder wave_order;
@@ -458,7 +484,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], wave_order, ticket, s));
             }
             const GroupDesc wave = g;   // all parts of the wave, with their scratch rows
-            const SplitPlan wave_sp = sp;
+
             for (int step = 0; step < wave_steps; ++step) {
                 const bool tap = taps && taps->step == step;
                 // trainers that have finished their steps drop out (time-based aggregation lets
@@ -466,21 +492,24 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 bool all_run = true;
                 for (int k = 0; k < wave.num; ++k) all_run = all_run && steps[wave.part[k]] > step;
                 const SpmmOrder order = all_run ? wave_order : SpmmOrder{nullptr, nullptr, 0, nullptr};  // built for the whole wave
+                SplitPlan spl[RTMA_MAX_LAYERS];
                 if (all_run) {
                     g = wave;
-                    sp = wave_sp;
+                    for (int l = 0; l < m.L; ++l) spl[l] = wave_spl[l];
                 } else {
                     g.num = 0;
-                    int slot = 0;
+                    int slot[RTMA_MAX_LAYERS] = {0};
                     for (int k = 0; k < wave.num; ++k) {
                         if (steps[wave.part[k]] <= step) continue;
                         const int j = g.num++;
                         // same chunking as in the whole wave: the slots still fit `partial`, and a
                         // trainer's gradient sums do not depend on who else is still running
-                        sp.split_begin[j] = slot;
-                        sp.rows_per_split[j] = wave_sp.rows_per_split[k];
-                        slot += wave_sp.split_begin[k + 1] - wave_sp.split_begin[k];
-                        sp.split_begin[j + 1] = slot;
+                        for (int l = 0; l < m.L; ++l) {
+                            spl[l].split_begin[j] = slot[l];
+                            spl[l].rows_per_split[j] = wave_spl[l].rows_per_split[k];
+                            slot[l] += wave_spl[l].split_begin[k + 1] - wave_spl[l].split_begin[k];
+                            spl[l].split_begin[j + 1] = slot[l];
+                        }
                         g.part[j] = wave.part[k];
                         g.rows[j] = wave.rows[k];
                         g.row_abs[j] = wave.row_abs[k];
@@ -604,7 +633,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                         LayerShape ws = m.layer[l];
                         ws.nsrc = 1;
                         ws.d_out = 2 * Cp;
-                        RTMA_TRY(launch_tc_wgrad(ctx, g, sp, ws, rows, Hl[l], Hl[l], DQ, partial, single_pass, s));
+                        RTMA_TRY(launch_tc_wgrad(ctx, g, spl[l], ws, rows, Hl[l], Hl[l], DQ, partial, single_pass, s));
                         if (l > 0) {
                             if (!single_pass && dgrad_narrow_applies(m.layer[l]))
                                 RTMA_TRY(launch_dgrad_narrow(ctx, g, m.layer[l], params, dZlast, Qlast, Hl[l], !m.post, s));
@@ -615,10 +644,10 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                                 RTMA_TRY(launch_post_backward(ctx, g, m.layer[l - 1], params, Zl[l - 1], Hl[l], stats[l - 1], post_partial,
                                                               m.lr, tap ? taps->grads : nullptr, s));
                         }
-                        RTMA_TRY(launch_reduce_sgd_head(ctx, g, sp, m.layer[l], Cp, partial, m.lr, params, tap ? taps->grads : nullptr, s));
+                        RTMA_TRY(launch_reduce_sgd_head(ctx, g, spl[l], m.layer[l], Cp, partial, m.lr, params, tap ? taps->grads : nullptr, s));
                         continue;
                     }
-                    RTMA_TRY(launch_tc_wgrad(ctx, g, sp, m.layer[l], rows, Hl[l], Nl[l], dZ, partial, single_pass, s));
+                    RTMA_TRY(launch_tc_wgrad(ctx, g, spl[l], m.layer[l], rows, Hl[l], Nl[l], dZ, partial, single_pass, s));
                     if (l > 0) {
                         // dH^l = dZ Ws^T + Abar^T (dZ Wn^T) = [dZ | Abar^T dZ] [Ws^T ; Wn^T]: aggregate first,
                         // at the layer's output width, then one product whose epilogue applies the ReLU
@@ -631,7 +660,7 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                             RTMA_TRY(launch_post_backward(ctx, g, m.layer[l - 1], params, Zl[l - 1], Hl[l], stats[l - 1], post_partial,
                                                           m.lr, tap ? taps->grads : nullptr, s));
                     }
-                    RTMA_TRY(launch_reduce_sgd(ctx, g, sp, m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
+                    RTMA_TRY(launch_reduce_sgd(ctx, g, spl[l], m.layer[l], partial, m.lr, params, tap ? taps->grads : nullptr, s));
                 }
             }
         }

@@ -79,6 +79,10 @@ int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, cons
 int32_t launch_from_planes(rtma_ctx* ctx, Planes src, int64_t first_row, int64_t rows, int d, float* dst, cudaStream_t s);
 // inv_deg[row_ws + i] = 1 / local degree (0 for an isolated node).
 int32_t launch_inv_degree(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, float* inv_deg, cudaStream_t s);
+// Raises the context's "not symmetric" flag (reported by rtma_check) unless every entry (u, v) of every
+// part of g comes with (v, u).  sums: three 64-bit words of scratch, zero on entry.
+int32_t launch_symmetry_check(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                              unsigned long long* sums, cudaStream_t s);
 // Processing order of the aggregation kernels' row groups (8 consecutive rows): the groups with at
 // least `heavy` entries, listed once per call, go first.  A zeroed SpmmOrder means plain row order.
 struct SpmmOrder {
@@ -204,6 +208,8 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
 int32_t launch_tc_dgrad(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                         Planes dZ, Planes Q, const __nv_bfloat16* Bd_hi, const __nv_bfloat16* Bd_lo, Planes H, bool gate,
                         bool single, cudaStream_t s);
+// Blocks launch_tc_wgrad starts per chunk of rows for a layer of this shape.
+int tc_wgrad_blocks_per_slot(const LayerShape& ls);
 // partial[slot][(nsrc d_in + 1) x d_out] = [H | N | 1]^T dZ ([N | 1]^T dZ for a one-matrix layer)
 // over one chunk of rows.
 int32_t launch_tc_wgrad(rtma_ctx* ctx, const GroupDesc& g, const SplitPlan& sp, LayerShape ls, int64_t rows_total,

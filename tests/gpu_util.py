@@ -178,9 +178,10 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, varia
         assert flipped <= 8 + flip_frac * units
         if flipped:
             o_loss, o_grads, _ = oracle.forward_backward_variant(variant, dims, rp, cp, X, y, p0, gates=gates)
+        mode_grads = None   # bf16 operand mode: the gradient of the mode's own definition (fp64 sums)
         if gemm_dtype == 1 and variant == (0, 0, 0):
-            same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, loss[p, 0], grads[p],
-                                assert_whole_step=gradients_against_plain)
+            mode_grads = same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, loss[p, 0], grads[p],
+                                             assert_whole_step=gradients_against_plain)
         if n_p:
             assert abs(loss[p, 0] - o_loss) <= tol_loss * max(1.0, abs(o_loss)), p
         if not gradients_against_plain:
@@ -208,16 +209,30 @@ def _round_bf16(x):
     return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
 
 
+def _bf16_ties(s):
+    """For recorded activations s = hi + lo (hi = the bf16 operand the kernel used, lo = the bf16
+    remainder): where s sits exactly half way between two bf16 numbers, hi cannot be told from s (a
+    remainder that rounds up to half a unit lands there, about once in 500 values).  Returns the
+    spacing of the two candidates at those places, 0 elsewhere."""
+    bits = np.ascontiguousarray(s, dtype=np.float32).view(np.uint32)
+    tie = (bits & 0xFFFF) == 0x8000
+    down = (bits & 0xFFFF0000).view(np.float32).astype(np.float64)
+    up = ((bits & 0xFFFF0000) + 0x10000).astype(np.uint32).view(np.float32).astype(np.float64)
+    return np.where(tie, np.abs(up - down), 0.0).reshape(np.shape(s))
+
+
 def layerwise_bf16_check(w, p, rp, cp, X, p0, gpu_acts):
     """bf16 operand mode, one layer at a time from the kernel's own recorded inputs: the aggregate
     A-bar H against the oracle's (it is not rounded), the layer output against the rounded-operand
     product of the recorded H and A-bar H in fp64.  The last layer may be evaluated in either
-    association -- H Ws + (A-bar H) Wn or H Ws + A-bar (H Wn) -- which differ once operands are rounded."""
+    association -- H Ws + (A-bar H) Wn or H Ws + A-bar (H Wn) -- which differ once operands are rounded.
+    Every output is held to TOL_BF16_LAYER plus what the undecidable operands (see _bf16_ties) of its
+    row can move it."""
     dims = w.dims
     L = len(dims) - 1
     r = _round_bf16
     off = 0
-    worst = 0.0
+    worst, loose = 0.0, 0
     for l in range(L):
         di, dn = dims[l], dims[l + 1]
         Ws = p0[off:off + di * dn].reshape(di, dn)
@@ -228,16 +243,24 @@ def layerwise_bf16_check(w, p, rp, cp, X, p0, gpu_acts):
         N = gpu_acts[f"N{l}"].astype(np.float64)
         e_agg = rel_err(N, oracle.spmm_mean(rp, cp, Hin))
         assert e_agg <= 2e-5, (p, f"N{l}", e_agg)
+        tie_h = np.zeros_like(Hin) if l == 0 else _bf16_ties(Hin)    # the features are rounded from fp32: no doubt there
+        tie_n = _bf16_ties(N)
+        got = gpu_acts[f"H{l + 1}"].astype(np.float64)
         Z = r(Hin) @ r(Ws) + r(N) @ r(Wn) + b
-        got = gpu_acts[f"H{l + 1}"]
+        slack = tie_h @ np.abs(r(Ws)) + tie_n @ np.abs(r(Wn))
+        scale = max(np.abs(Z).max(), 1e-30)
         if l < L - 1:
-            e = rel_err(got, np.maximum(Z, 0.0))
+            excess = np.abs(got - np.maximum(Z, 0.0)) - slack
         else:
             Z_after = r(Hin) @ r(Ws) + oracle.spmm_mean(rp, cp, r(Hin) @ r(Wn)) + b
-            e = min(rel_err(got, Z), rel_err(got, Z_after))
-        worst = max(worst, e, e_agg)
-        assert e <= TOL_BF16_LAYER, (p, f"H{l + 1}", e)
-    print(f"[bf16 layer by layer] {w.name} part {p}: worst {worst:.1e}")
+            slack_after = tie_h @ np.abs(r(Ws)) + oracle.spmm_mean(rp, cp, tie_h @ np.abs(r(Wn)))
+            e0, e1 = np.abs(got - Z) - slack, np.abs(got - Z_after) - slack_after
+            excess = e0 if e0.max() <= e1.max() else e1
+        worst = max(worst, float(excess.max()) / scale)
+        loose += int(np.count_nonzero(slack))
+        assert excess.max() <= TOL_BF16_LAYER * scale, (p, f"H{l + 1}", float(excess.max()) / scale)
+    print(f"[bf16 layer by layer] {w.name} part {p}: worst {worst:.1e} of the layer's largest output "
+          f"({loose} outputs with an undecidable operand in their row)")
 
 
 def same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, gpu_loss, gpu_grads, assert_whole_step=True):
@@ -269,6 +292,7 @@ def same_rounding_check(w, p, rp, cp, X, y, p0, gpu_acts, gpu_loss, gpu_grads, a
         if rp.size > 1:
             assert abs(gpu_loss - r_loss) <= tol * max(1.0, abs(r_loss)), p
         assert max(gerrs.values(), default=0.0) <= tol, (p, gerrs)
+    return r_grads
 
 
 def check_k_steps_and_average(w, got, want, K, gemm_dtype=0, streams=None, only_parts=None, variant=(0, 0, 0),

@@ -56,6 +56,36 @@ def test_supertma_super_nodes_kept_together(util):
     util.check_k_steps_and_average(w, got, want, 2)
 
 
+def test_directed_subgraph_is_reported(util):
+    # the backward pass reuses the forward CSR as its own transpose, which needs every entry (u, v) to
+    # come with (v, u); a caller who passes a directed subgraph as symmetric learns it at the next check
+    from paper_2305_09887_b200 import binding
+    c = binding.Context(0)
+    n, F, C = 300, 16, 4
+    g = inputs.uniform_graph(n, 900, 3)
+    rows = np.repeat(np.arange(n), np.diff(g.rowptr))
+    X = util.dev(inputs.normal_features(n, F, 4))
+    y = util.dev(inputs.uniform_labels(n, C, 5))
+    dims = (F, 8, C)
+    p0 = inputs.xavier_params(dims, 6)
+    for drop, ok in ((None, True), (7, False)):
+        keep = np.ones(g.col.size, dtype=bool)
+        if drop is not None:
+            keep[drop] = False            # one direction of one edge removed
+        rowptr = np.concatenate([[0], np.cumsum(np.bincount(rows[keep], minlength=n))]).astype(np.int64)
+        col = np.ascontiguousarray(g.col[keep])
+        params = util.dev(p0[None, :].copy())
+        c.local_steps(dims, 0.01, 1, [0, n], [0, int(col.size)], util.dev(np.concatenate([rowptr])), util.dev(col),
+                      X, y, params, 1)
+        if ok:
+            c.check()
+        else:
+            with pytest.raises(Exception, match="not symmetric"):
+                c.check()
+            c.check()                    # the flag is cleared by the report; the context stays usable
+    c.close()
+
+
 def test_features_gathered_inside_the_training_call(util, tiny_workload):
     # rtma_local_steps_gathered reads X in node order through perm: the same result, bit for bit, as
     # rtma_local_steps on the rows gathered beforehand
