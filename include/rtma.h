@@ -328,8 +328,11 @@ int32_t rtma_selftest_wait_timeout(rtma_ctx* ctx, void* stream);
  * (rtma_partition_grouped when super-node ids are given), rtma_build_induced_csr, rtma_gather_rows (labels), then R rounds of (rtma_local_steps_gathered with K steps on
  * every part, rtma_aggregate), and copies back params_out_h [P] (the averaged parameters),
  * loss_out_h [R][M][K] (or NULL) and kept_cut_h [2] (or NULL).  The graph must be undirected
- * with both directions stored.  Allocates and frees its device buffers with cudaMalloc /
- * cudaFree and SYNCHRONISES the stream before returning.                                   */
+ * with both directions stored.  The device copies of the inputs live in buffers the context
+ * keeps between calls (allocated with cudaMalloc when a call needs more than the last, freed by
+ * rtma_destroy).  The graph is copied first; features, labels and parameters follow on a stream
+ * of the context's own while the partition and subgraph kernels run.  SYNCHRONISES the stream
+ * before returning.                                                                         */
 int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_64, const void* rowptr_h,
                         const int32_t* col_h, const int32_t* group_id_h, const float* X_h,
                         const int32_t* y_h, const rtma_model_desc* model, int32_t M, uint64_t seed,

@@ -41,6 +41,14 @@ struct rtma_ctx {
     // the streams of the last local-training call and an event recorded at the end of each
     std::vector<cudaStream_t> trained_streams;
     std::vector<cudaEvent_t> trained_events;
+    // device buffers of the host-buffer entry point (inputs and preprocessing outputs; kept result
+    // columns), a second stream and an event for its copies: kept between calls, freed with the context
+    void* host_block = nullptr;
+    size_t host_block_bytes = 0;
+    void* host_cols = nullptr;
+    size_t host_cols_bytes = 0;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t copy_done = nullptr;
     void* pinned = nullptr;       // small pinned staging block for descriptors
     size_t pinned_bytes = 0;
     char error[512] = {0};

@@ -6,10 +6,25 @@
 #include "common.cuh"
 
 namespace {
-struct DeviceBlock {
-    void* p = nullptr;
-    ~DeviceBlock() { if (p) cudaFree(p); }
-};
+// Makes *block at least `bytes` large (the context keeps it for the next call).
+int32_t grow_block(rtma_ctx* ctx, void** block, size_t* have, size_t bytes) {
+    if (*have >= bytes) return RTMA_OK;
+    RTMA_CUDA(ctx, cudaDeviceSynchronize());
+    if (*block) {
+        RTMA_CUDA(ctx, cudaFree(*block));
+        *block = nullptr;
+        *have = 0;
+    }
+    cudaError_t e = cudaMalloc(block, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        *block = nullptr;
+        return rtma_fail(ctx, RTMA_ERR_WORKSPACE, "cannot allocate %zu bytes for the inputs on the device: %s", bytes,
+                         cudaGetErrorString(e));
+    }
+    *have = bytes;
+    return RTMA_OK;
+}
 }  // namespace
 
 extern "C" int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_64, const void* rowptr_h,
@@ -40,19 +55,26 @@ extern "C" int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_6
     const size_t o_rpo = reserve(8 * (size_t)(n + M)), o_eoff = reserve(8 * (M + 1)), o_kc = reserve(16);
     const size_t o_yp = reserve(4 * (size_t)n);
     const size_t o_par = reserve(4 * (size_t)M * P), o_loss = reserve(4 * (size_t)R * M * (K > 0 ? K : 1));
-    DeviceBlock blk, colblk;
-    RTMA_CUDA(ctx, cudaMalloc(&blk.p, total));
-    char* b = static_cast<char*>(blk.p);
+    RTMA_TRY(grow_block(ctx, &ctx->host_block, &ctx->host_block_bytes, total));
+    char* b = static_cast<char*>(ctx->host_block);
     auto at = [&](size_t off) { return static_cast<void*>(b + off); };
+    if (!ctx->copy_stream) RTMA_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    if (!ctx->copy_done) RTMA_CUDA(ctx, cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming));
 
+    // The graph first, on the caller's stream: partition and the induced subgraphs need nothing else.
+    // Features, labels and parameters follow on a second stream while those kernels run; the training
+    // call waits for them.
     RTMA_CUDA(ctx, cudaMemcpyAsync(at(o_rowptr), rowptr_h, rp_w * (n + 1), cudaMemcpyHostToDevice, stream));
     if (E) RTMA_CUDA(ctx, cudaMemcpyAsync(at(o_col), col_h, 4 * (size_t)E, cudaMemcpyHostToDevice, stream));
     if (group_id_h) RTMA_CUDA(ctx, cudaMemcpyAsync(at(o_gid), group_id_h, 4 * (size_t)n, cudaMemcpyHostToDevice, stream));
-    RTMA_CUDA(ctx, cudaMemcpyAsync(at(o_X), X_h, 4 * (size_t)n * F, cudaMemcpyHostToDevice, stream));
-    RTMA_CUDA(ctx, cudaMemcpyAsync(at(o_y), y_h, 4 * (size_t)n, cudaMemcpyHostToDevice, stream));
+    RTMA_CUDA(ctx, cudaEventRecord(ctx->copy_done, stream));   // orders the second stream after whatever used the block before
+    RTMA_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->copy_done, 0));
+    RTMA_CUDA(ctx, cudaMemcpyAsync(at(o_y), y_h, 4 * (size_t)n, cudaMemcpyHostToDevice, ctx->copy_stream));
     for (int i = 0; i < M; ++i)
         RTMA_CUDA(ctx, cudaMemcpyAsync(static_cast<float*>(at(o_par)) + (size_t)i * P, params0_h, 4 * (size_t)P,
-                                       cudaMemcpyHostToDevice, stream));
+                                       cudaMemcpyHostToDevice, ctx->copy_stream));
+    RTMA_CUDA(ctx, cudaMemcpyAsync(at(o_X), X_h, 4 * (size_t)n * F, cudaMemcpyHostToDevice, ctx->copy_stream));
+    RTMA_CUDA(ctx, cudaEventRecord(ctx->copy_done, ctx->copy_stream));
 
     int32_t* part_id = static_cast<int32_t*>(at(o_pid));
     int64_t* part_offsets = static_cast<int64_t*>(at(o_poff));
@@ -70,12 +92,13 @@ extern "C" int32_t rtma_train_host(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_6
     RTMA_CUDA(ctx, cudaMemcpyAsync(po.data(), part_offsets, 8 * (M + 1), cudaMemcpyDeviceToHost, stream));
     RTMA_CUDA(ctx, cudaMemcpyAsync(eo.data(), edge_offsets, 8 * (M + 1), cudaMemcpyDeviceToHost, stream));
     RTMA_CUDA(ctx, cudaStreamSynchronize(stream));
-    RTMA_CUDA(ctx, cudaMalloc(&colblk.p, 4 * (size_t)(eo[M] > 0 ? eo[M] : 1)));
-    int32_t* col_out = static_cast<int32_t*>(colblk.p);
+    RTMA_TRY(grow_block(ctx, &ctx->host_cols, &ctx->host_cols_bytes, 4 * (size_t)(eo[M] > 0 ? eo[M] : 1)));
+    int32_t* col_out = static_cast<int32_t*>(ctx->host_cols);
     if (eo[M] > 0)
         RTMA_TRY(rtma_build_induced_csr(ctx, n, rowptr_is_64, at(o_rowptr), static_cast<int32_t*>(at(o_col)), M, part_id,
                                         part_offsets, perm, local_id, rowptr_out, col_out, edge_offsets, kept_cut, stream));
     // the features stay in node order: the training call gathers them while it lays them out
+    RTMA_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->copy_done, 0));   // labels, parameters and features have arrived
     RTMA_TRY(rtma_gather_rows(ctx, n, 4, at(o_y), perm, at(o_yp), stream));
 
     std::vector<void*> streams(M, stream_);

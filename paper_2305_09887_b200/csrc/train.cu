@@ -153,6 +153,7 @@ int splits_for(int64_t n_p, int parts_in_flight, int blocks_per_slot) {
     // chunk).  Taking every part for as large as this one, pick the chunk count with the smallest such
     // product, or the fewest chunks within 3 % of it (fewer partial sums to add up afterwards).
     constexpr int64_t SMS = 148;
+    if (n_p <= 0) return 1;
     const int64_t most = std::min<int64_t>(64, std::max<int64_t>(1, ceil_div(n_p, 1024)));
     auto cost_of = [&](int64_t ns) {
         const int64_t rows = aligned_rows(ceil_div(n_p, ns));

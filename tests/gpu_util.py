@@ -194,7 +194,17 @@ def check_one_step(w, M=None, gemm_dtype=0, streams=None, only_parts=None, varia
                 if size == 1:   # a single number (PReLU slope): relative to itself, with an absolute floor
                     assert abs(gg[0] - og[0]) <= tol_grad * max(abs(og[0]), 1e-3), (p, nm)
                 else:
-                    assert rel_err(gg, og) <= tol_grad, (p, nm)
+                    e, bar = rel_err(gg, og), tol_grad
+                    if mode_grads is not None:
+                        # where rounding the operands to bf16 -- in exact sums, by the mode's definition --
+                        # already moves this tensor past the bar, no implementation of the mode can
+                        # meet it on this input: hold the kernel to what the definition delivers
+                        e_mode = rel_err(mode_grads[off:off + size], og)
+                        if e_mode > 0.8 * tol_grad:
+                            bar = max(tol_grad, 1.25 * e_mode)
+                            print(f"[bf16 bar] {w.name} part {p} {nm}: kernel {e:.2e}, the mode's definition {e_mode:.2e} "
+                                  f"from the unrounded oracle (bar {tol_grad:.0e})")
+                    assert e <= bar, (p, nm, e)
             else:
                 assert np.abs(gg).max() == 0
         assert rel_err(params1[p], p0 - w.lr * o_grads) <= tol_param
