@@ -51,7 +51,8 @@ enum {
     RTMA_ERR_WORKSPACE = -3,   /* the scratch arena cannot be made large enough           */
     RTMA_ERR_OVERFLOW = -4,    /* a count does not fit the index type of its output       */
     RTMA_ERR_CUDA = -5,        /* a CUDA runtime call failed; text in rtma_last_error     */
-    RTMA_ERR_TIMEOUT = -6      /* a bounded device-side wait ran out (kernel gave up)     */
+    RTMA_ERR_TIMEOUT = -6,     /* a bounded device-side wait ran out (kernel gave up)     */
+    RTMA_ERR_BOUNDS = -7       /* checked build only: an index in the caller's data was out of range */
 };
 
 typedef struct rtma_ctx rtma_ctx;
@@ -68,8 +69,12 @@ const char* rtma_last_error(const rtma_ctx* ctx);
  * tensor-core kernels wait on mbarriers with an iteration limit instead of spinning for
  * ever), RTMA_ERR_INVALID_ARG if a local-training call since the last check was given a
  * subgraph that is not symmetric; RTMA_OK otherwise.  rtma_train_host calls it before
- * returning.                                                                               */
+ * returning.  In the checked build of the library (compiled with -DRTMA_BOUNDS; every index taken
+ * from the caller's data is range-checked and an offending access is skipped, not made) it
+ * also reports RTMA_ERR_BOUNDS with the first offending index.                               */
 int32_t rtma_check(rtma_ctx* ctx);
+/* 1 if this library is the checked build (-DRTMA_BOUNDS), else 0.                           */
+int32_t rtma_bounds_checked(void);
 /* Bytes of scratch currently held by the context.                                        */
 size_t rtma_workspace_bytes(const rtma_ctx* ctx);
 /* Caps the scratch arena at `bytes` (0 = no cap, the default): no later call grows it beyond
@@ -231,7 +236,7 @@ int32_t rtma_local_steps_gathered(rtma_ctx* ctx, const rtma_model_desc* model, i
 
 /* Local training with a step count of its own for every trainer.  Aggregation is triggered by
  * wall time, not by a step count (Sec. 3.1), so trainers arrive at an aggregation with
- * different numbers of finished steps (Table 4 reports up to 28.8% fewer on the slowest one):
+ * different numbers of finished steps (Sec. 3.1 and Table 3 report up to 28.8% fewer on the slowest one):
  * trainer i runs steps_host[i] steps.  steps_host[i] = 0 is a trainer that did not run at all,
  * e.g. one that failed to start (Sec. 4.5): its replica is left untouched and it takes neither
  * scratch nor launches.

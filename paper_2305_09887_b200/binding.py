@@ -14,6 +14,7 @@ import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "librtma.so")
+LIB_CHECKED_PATH = os.path.join(_PKG, "librtma_checked.so")   # built with -DRTMA_BOUNDS: every caller-supplied index checked
 MAX_PARTS = 64
 MAX_LAYERS = 8
 
@@ -23,11 +24,11 @@ EXPORTS = (
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
     "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout", "rtma_link_param_count",
-    "rtma_link_steps", "rtma_set_workspace_limit", "rtma_local_steps_gathered",
+    "rtma_link_steps", "rtma_set_workspace_limit", "rtma_local_steps_gathered", "rtma_bounds_checked",
 )
 KERNEL_CLASSES = 21
 
-_lib = None
+_libs = {}
 
 
 class RtmaError(RuntimeError):
@@ -59,14 +60,14 @@ class Taps(ctypes.Structure):
     _fields_ = [("acts", ctypes.c_void_p), ("grads", ctypes.c_void_p), ("step", ctypes.c_int32)]
 
 
-def load_library():
-    """Loads the shared library; raises if it has not been built."""
-    global _lib
-    if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise RtmaError(f"{LIB_PATH} not found: build it with `python -m paper_2305_09887_b200.build` "
-                            "(there is no CPU fallback)")
-        lib = ctypes.CDLL(LIB_PATH)
+def load_library(checked: bool = False):
+    """Loads the shared library (checked: the range-checked build); raises if it has not been built."""
+    path = LIB_CHECKED_PATH if checked else LIB_PATH
+    if path not in _libs:
+        if not os.path.exists(path):
+            raise RtmaError(f"{path} not found: build it with `python -m paper_2305_09887_b200.build"
+                            f"{' --checked' if checked else ''}` (there is no CPU fallback)")
+        lib = ctypes.CDLL(path)
         lib.rtma_last_error.restype = ctypes.c_char_p
         lib.rtma_last_error.argtypes = [ctypes.c_void_p]
         lib.rtma_workspace_bytes.restype = ctypes.c_size_t
@@ -74,8 +75,8 @@ def load_library():
         lib.rtma_param_count.restype = ctypes.c_int64
         lib.rtma_kernel_class_name.restype = ctypes.c_char_p
         lib.rtma_partition_static_error.restype = ctypes.c_char_p
-        _lib = lib
-    return _lib
+        _libs[path] = lib
+    return _libs[path]
 
 
 def model_desc(dims, lr: float = 0.01, gemm_dtype: int = 0, variant=(0, 0, 0)) -> ModelDesc:
@@ -155,10 +156,10 @@ class Context:
     """One library context on one CUDA device.  Calls are enqueued on the given (or the
     current torch) stream and share the context's scratch, so keep them stream-ordered."""
 
-    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+    def __init__(self, device: int = 0, workspace_bytes: int = 0, checked: bool = False):
         if not torch.cuda.is_available():
             raise RtmaError("no CUDA device: this library has no CPU path")
-        self._lib = load_library()
+        self._lib = load_library(checked)
         self.device = torch.device("cuda", device)
         torch.cuda.init()
         with torch.cuda.device(self.device):

@@ -139,6 +139,48 @@ struct ArenaCursor {
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+// ---- index checks of the checked build (-DRTMA_BOUNDS) -----------------------------------------
+// Every index that a kernel takes from the caller's data (column ids, permutation entries, part ids,
+// labels, pair end points) goes through rtma_index_ok before it addresses memory.  In the ordinary
+// build the check compiles to `true`.  In the checked build an index outside [0, limit) is recorded
+// (first offender: site, index, limit) in a word of the translation unit, the access is skipped, and
+// the next rtma_check returns RTMA_ERR_BOUNDS: nothing traps and nothing is read or written out of
+// range.  Sites: 1 column id of the input graph, 2 part id, 3 local id, 4 permutation entry, 5 column
+// id of an induced subgraph, 6 label, 7 pair end point.
+#ifdef RTMA_BOUNDS
+#ifdef __CUDACC__
+static __device__ long long rtma_bounds_record[4];  // site (0: none), index, limit
+__device__ __forceinline__ bool rtma_index_ok(long long idx, long long limit, int site) {
+    if (idx >= 0 && idx < limit) return true;
+    if (atomicCAS(reinterpret_cast<unsigned long long*>(&rtma_bounds_record[0]), 0ULL, (unsigned long long)site) == 0ULL) {
+        rtma_bounds_record[1] = idx;
+        rtma_bounds_record[2] = limit;
+    }
+    return false;
+}
+// Every translation unit with checked kernels registers a reader of its record with the context code.
+typedef bool (*rtma_bounds_reader)(long long out[3]);  // true: an offender was recorded (and the record is cleared)
+void rtma_register_bounds_reader(rtma_bounds_reader r);
+#define RTMA_BOUNDS_TU()                                                                                   \
+    namespace {                                                                                            \
+    bool read_bounds_record(long long out[3]) {                                                            \
+        long long h[4] = {0, 0, 0, 0};                                                                     \
+        if (cudaMemcpyFromSymbol(h, rtma_bounds_record, sizeof(h)) != cudaSuccess || h[0] == 0) return false; \
+        out[0] = h[0]; out[1] = h[1]; out[2] = h[2];                                                       \
+        const long long z[4] = {0, 0, 0, 0};                                                               \
+        cudaMemcpyToSymbol(rtma_bounds_record, z, sizeof(z));                                              \
+        return true;                                                                                       \
+    }                                                                                                      \
+    struct BoundsRegistration { BoundsRegistration() { rtma_register_bounds_reader(read_bounds_record); } } bounds_registration; \
+    }
+#endif
+#else
+#ifdef __CUDACC__
+__device__ __forceinline__ bool rtma_index_ok(long long, long long, int) { return true; }
+#endif
+#define RTMA_BOUNDS_TU()
+#endif
+
 // ---- generic device-wide exclusive scan (three passes, no inter-block waits) ----
 // out[i] = sum_{k<i} in[k] for i = 0..n (n+1 outputs).  scratch: scan_scratch_elems(n) int64.
 size_t scan_scratch_elems(int64_t n);

@@ -71,10 +71,41 @@ extern "C" const char* rtma_kernel_class_name(int32_t cls) {
     return cls >= 0 && cls < KC_COUNT ? kKernelClassNames[cls] : "";
 }
 
+#ifdef RTMA_BOUNDS
+namespace {
+std::vector<rtma_bounds_reader>& bounds_readers() {
+    static std::vector<rtma_bounds_reader> readers;
+    return readers;
+}
+}  // namespace
+void rtma_register_bounds_reader(rtma_bounds_reader r) { bounds_readers().push_back(r); }
+extern "C" int32_t rtma_bounds_checked(void) { return 1; }
+#else
+extern "C" int32_t rtma_bounds_checked(void) { return 0; }
+#endif
+
 extern "C" int32_t rtma_check(rtma_ctx* ctx) {
     if (!ctx) return RTMA_ERR_INVALID_ARG;
     RTMA_CUDA(ctx, cudaSetDevice(ctx->device));
     RTMA_CUDA(ctx, cudaDeviceSynchronize());
+#ifdef RTMA_BOUNDS
+    {
+        static const char* const site_names[] = {"", "column id of the input graph", "part id", "local id", "permutation entry",
+                                                 "column id of an induced subgraph", "label", "pair end point"};
+        long long first[3] = {0, 0, 0};
+        bool any = false;
+        for (rtma_bounds_reader r : bounds_readers()) {
+            long long rec[3];
+            if (r(rec) && !any) {
+                any = true;
+                first[0] = rec[0]; first[1] = rec[1]; first[2] = rec[2];
+            }
+        }
+        if (any)
+            return rtma_fail(ctx, RTMA_ERR_BOUNDS, "index out of range in the caller's data: %s %lld outside [0, %lld)",
+                             first[0] >= 1 && first[0] <= 7 ? site_names[first[0]] : "index", first[1], first[2]);
+    }
+#endif
     int word[2] = {0, 0};
     RTMA_CUDA(ctx, cudaMemcpy(word, ctx->error_word, sizeof(word), cudaMemcpyDeviceToHost));
     if (word[0] != 0 || word[1] != 0) cudaMemset(ctx->error_word, 0, sizeof(word));

@@ -11,6 +11,8 @@
 // pack the part ids into one byte per node, so that this table (25 MB for 25 M nodes) stays in L2.
 #include "common.cuh"
 
+RTMA_BOUNDS_TU()
+
 namespace {
 
 constexpr int CSR_THREADS = 256;
@@ -30,7 +32,7 @@ pack_parts_kernel(int64_t n, const int32_t* __restrict__ part_id, uint8_t* __res
 
 template <class RowT>
 __global__ void __launch_bounds__(CSR_THREADS)
-induced_count_kernel(int64_t n, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
+induced_count_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
                      const uint8_t* __restrict__ part8, const int64_t* __restrict__ part_offsets,
                      const int32_t* __restrict__ local_id, int32_t* __restrict__ counts) {
     const int lane = threadIdx.x & 31;
@@ -39,10 +41,16 @@ induced_count_kernel(int64_t n, const RowT* __restrict__ rowptr, const int32_t* 
     const int p = part8[u];
     const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
     int kept = 0;
-    for (int64_t e = begin + lane; e < end; e += 32) kept += (part8[__ldg(col + e)] == p);
+    for (int64_t e = begin + lane; e < end; e += 32) {
+        const int32_t v = __ldg(col + e);
+        if (rtma_index_ok(v, n, 1)) kept += (part8[v] == p);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
-    if (lane == 0) counts[part_offsets[p] + local_id[u]] = kept;  // the row's place in partition order
+    if (lane == 0 && rtma_index_ok(p, M, 2)) {
+        const int64_t place = part_offsets[p] + local_id[u];  // the row's place in partition order
+        if (rtma_index_ok(place, n, 3)) counts[place] = kept;
+    }
 }
 
 // slots[j] = global slot of row j's first kept entry (exclusive scan of counts), j = 0..n.
@@ -87,7 +95,9 @@ induced_fill_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int
     const int64_t u = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
     if (u >= n) return;
     const int p = part8[u];
+    if (!rtma_index_ok(p, M, 2)) return;
     const int64_t j = part_offsets[p] + local_id[u];  // the row's place in partition order
+    if (!rtma_index_ok(j, n, 3)) return;
     const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
     int64_t out = edge_offsets[p] + rowptr_out[j + p];
     const unsigned below = (1u << lane) - 1u;
@@ -97,7 +107,7 @@ induced_fill_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int
         bool keep = false;
         if (e < end) {
             v = __ldg(col + e);
-            keep = part8[v] == p;
+            keep = rtma_index_ok(v, n, 1) && part8[v] == p;
         }
         const unsigned votes = __ballot_sync(0xffffffffu, keep);
         if (keep) col_out[out + __popc(votes & below)] = local_id[v];
@@ -112,6 +122,7 @@ gather_rows_kernel(int64_t n, int64_t row_bytes, const char* __restrict__ src, c
     const int lane = threadIdx.x & 31;
     const int64_t i = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (i >= n) return;
+    if (!rtma_index_ok(perm[i], n, 4)) return;  // perm is a permutation of the n rows
     const char* s = src + (int64_t)perm[i] * row_bytes;
     char* d = dst + i * row_bytes;
     if (VEC_BYTES == 16) {
@@ -129,7 +140,7 @@ gather_rows_kernel(int64_t n, int64_t row_bytes, const char* __restrict__ src, c
 __global__ void __launch_bounds__(256)
 gather_words_kernel(int64_t n, const int32_t* __restrict__ src, const int32_t* __restrict__ perm, int32_t* __restrict__ dst) {
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (i < n) dst[i] = __ldg(src + perm[i]);
+    if (i < n && rtma_index_ok(perm[i], n, 4)) dst[i] = __ldg(src + perm[i]);
 }
 
 }  // namespace
@@ -183,10 +194,10 @@ extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowp
         RTMA_LAUNCH_CHECK(ctx);
         if (rowptr_is_64)
             { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
+                n, M, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
         else
             { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
+                n, M, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
         RTMA_LAUNCH_CHECK(ctx);
     }
     RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, n, slots, scratch, stream));

@@ -8,6 +8,8 @@
 // whose slot k belongs to the same trainer as slot k of the node descriptor.
 #include "train.cuh"
 
+RTMA_BOUNDS_TU()
+
 namespace {
 
 constexpr int PAIR_WARPS = 8;
@@ -25,6 +27,7 @@ pair_product_kernel(const __grid_constant__ GroupDesc gd, const __grid_constant_
     if (!locate_tile(gd, PAIR_WARPS, blockIdx.x, &k, &r0)) return;
     const int lane = threadIdx.x & 31, i = r0 + (threadIdx.x >> 5);
     if (i >= gd.rows[k]) return;
+    if (!rtma_index_ok(pu[gd.row_abs[k] + i], g.rows[k], 7) || !rtma_index_ok(pv[gd.row_abs[k] + i], g.rows[k], 7)) return;
     const int64_t ru = g.row_ws[k] + pu[gd.row_abs[k] + i], rv = g.row_ws[k] + pv[gd.row_abs[k] + i];
     const int64_t out = gd.row_ws[k] + i;
     for (int col = lane * 8; col < d; col += 256) {
@@ -50,6 +53,7 @@ pair_scatter_kernel(const __grid_constant__ GroupDesc gd, const __grid_constant_
     if (!locate_tile(gd, PAIR_WARPS, blockIdx.x, &k, &r0)) return;
     const int lane = threadIdx.x & 31, i = r0 + (threadIdx.x >> 5);
     if (i >= gd.rows[k]) return;
+    if (!rtma_index_ok(pu[gd.row_abs[k] + i], g.rows[k], 7) || !rtma_index_ok(pv[gd.row_abs[k] + i], g.rows[k], 7)) return;
     const int64_t ru = g.row_ws[k] + pu[gd.row_abs[k] + i], rv = g.row_ws[k] + pv[gd.row_abs[k] + i];
     const int64_t src = gd.row_ws[k] + i;
     for (int col = lane * 8; col < d; col += 256) {

@@ -10,7 +10,12 @@
 // run to run.
 #include "train.cuh"
 
+RTMA_BOUNDS_TU()
+
 namespace {
+
+// a label outside [0, C) counts as class 0 in the checked build (and is reported)
+__device__ __forceinline__ int checked_label(int label, int C) { return rtma_index_ok(label, C, 6) ? label : 0; }
 
 constexpr int LOSS_THREADS = 256;
 constexpr int LOSS_TILE_ROWS = 64;
@@ -38,7 +43,7 @@ softmax_xent_kernel(const __grid_constant__ GroupDesc g, const Mat logits, const
     for (int q = 0; q < R; ++q) {
         const bool row_ok = i0 + q < n_p;
         const float* z = logits.ptr + (g.row_ws[k] + i0 + q) * logits.ld;
-        label[q] = row_ok ? yp[g.row_abs[k] + i0 + q] : 0;
+        label[q] = row_ok ? checked_label(yp[g.row_abs[k] + i0 + q], C) : 0;
         if (J == 1) {
             v[q][0] = (row_ok && c0 < C) ? z[c0] : 0.f;
         } else if (J == 2) {
@@ -133,7 +138,7 @@ softmax_xent_row_kernel(const __grid_constant__ GroupDesc g, const Mat logits, c
     if (i < n_p) {
         const int64_t r = g.row_ws[k] + i;
         const float4* z = reinterpret_cast<const float4*>(logits.ptr + r * logits.ld);
-        const int label = yp[g.row_abs[k] + i];
+        const int label = checked_label(yp[g.row_abs[k] + i], C);
         const int nv = (int)(logits.ld >> 2);
         float v[4 * NV4];
 #pragma unroll
@@ -205,7 +210,7 @@ softmax_xent_head_kernel(const __grid_constant__ GroupDesc g, const Planes Tself
     if (i < n_p) {
         const int64_t r = g.row_ws[k] + i;
         const float* bias = params + (int64_t)g.part[k] * P + bias_offset;
-        const int label = yp[g.row_abs[k] + i];
+        const int label = checked_label(yp[g.row_abs[k] + i], C);
         const int n8 = (int)(NT.ld >> 3) < NV4 / 2 ? (int)(NT.ld >> 3) : NV4 / 2;
         float v[4 * NV4];
 #pragma unroll
@@ -286,7 +291,7 @@ softmax_xent_wide_kernel(const __grid_constant__ GroupDesc g, const Mat logits, 
         if (i >= n_p) break;
         const int64_t r = g.row_ws[k] + i;
         const float* z = logits.ptr + r * logits.ld;
-        const int label = yp[g.row_abs[k] + i];
+        const int label = checked_label(yp[g.row_abs[k] + i], C);
         float zmax = -INFINITY;
         for (int c = lane; c < C; c += 32) zmax = fmaxf(zmax, z[c]);
 #pragma unroll

@@ -23,6 +23,8 @@
 
 #include "train.cuh"
 
+RTMA_BOUNDS_TU()
+
 namespace {
 
 constexpr int SPMM_THREADS = 256;
@@ -52,22 +54,32 @@ gcn_scale_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict_
 
 __global__ void __launch_bounds__(256)
 to_planes_kernel(const __grid_constant__ GroupDesc g, const float* __restrict__ X, const int32_t* __restrict__ perm,
-                 const int d, const Planes out) {
+                 const int64_t n_total, const int d, const Planes out) {
     int k, r0;
     if (!locate_tile(g, 32, blockIdx.x, &k, &r0)) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool vec = d % 4 == 0 && reinterpret_cast<uintptr_t>(X) % 16 == 0;
     for (int q = 0; q < 4; ++q) {
         const int i = r0 + warp * 4 + q;
         if (i >= g.rows[k]) return;
         // perm: the features are still in the graph's node order; row i of the partition order is node perm[i]
-        const float* x = X + (perm ? (int64_t)perm[g.row_abs[k] + i] : g.row_abs[k] + i) * (int64_t)d;
+        const int64_t node = perm ? (int64_t)perm[g.row_abs[k] + i] : g.row_abs[k] + i;
+        if (!rtma_index_ok(node, n_total, 4)) continue;
+        const float* x = X + node * (int64_t)d;
         const int64_t o = (g.row_ws[k] + i) * out.ld;
         for (int c0 = lane * 8; c0 < out.ld; c0 += 256) {
             Pack8 p;
+            if (vec && c0 + 8 <= d) {  // rows start on 16-byte boundaries: two vector loads
+                const float4 a = __ldg(reinterpret_cast<const float4*>(x + c0));
+                const float4 b = __ldg(reinterpret_cast<const float4*>(x + c0 + 4));
+                p.v[0] = a.x; p.v[1] = a.y; p.v[2] = a.z; p.v[3] = a.w;
+                p.v[4] = b.x; p.v[5] = b.y; p.v[6] = b.z; p.v[7] = b.w;
+            } else {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) p.v[e] = c0 + e < d ? __ldg(x + c0 + e) : 0.f;
+                for (int e = 0; e < 8; ++e) p.v[e] = c0 + e < d ? __ldg(x + c0 + e) : 0.f;
+            }
             uint4 h, l;
-            p.to_planes(h, l);
+            p.to_planes_cvt(h, l);
             *reinterpret_cast<uint4*>(out.hi + o + c0) = h;
             *reinterpret_cast<uint4*>(out.lo + o + c0) = l;
         }
@@ -121,6 +133,7 @@ locality_probe_kernel(const __grid_constant__ GroupDesc g, const int64_t* __rest
         const int64_t b = rp[i], e = rp[i + 1];
         for (int64_t x = b; x < e; ++x) {
             const int c = cols[x];
+            rtma_index_ok(c, g.rows[k], 5);
             near += (c - i < LOCAL_SPAN && i - c < LOCAL_SPAN) ? 1u : 0u;
         }
         total += (unsigned long long)(e - b);
@@ -339,7 +352,8 @@ spmm_rows(const GroupDesc& g, const int64_t* __restrict__ rowptr_out,
 
     for (int p0 = 0; p0 < n_entries; p0 += 32) {   // pieces of 32 entries
         const int cnt = min(32, n_entries - p0);
-        const int32_t mine = lane < cnt ? __ldg(cols + p0 + lane) : 0;
+        int32_t mine = lane < cnt ? __ldg(cols + p0 + lane) : 0;
+        if (!rtma_index_ok(mine, g.rows[k], 5)) mine = 0;
         const float mine_w = (MODE != 0 && lane < cnt) ? __ldg(inv_deg + ws + mine) : 0.f;
         // one batch: W neighbours' rows requested, then added in entry order
         auto batch = [&](const int t, const bool full) {
@@ -516,7 +530,10 @@ spmm_narrow_rows(const GroupDesc& g, const int64_t* __restrict__ rowptr_out,
 #pragma unroll
             for (int q = 0; q < RPS; ++q)
 #pragma unroll
-                for (int j = 0; j < WN; ++j) nb[q][j] = rb[q] + t + j < re[q] ? __ldg(cols + rb[q] + t + j) : -1;
+                for (int j = 0; j < WN; ++j) {
+                    nb[q][j] = rb[q] + t + j < re[q] ? __ldg(cols + rb[q] + t + j) : -1;
+                    if (nb[q][j] >= 0 && !rtma_index_ok(nb[q][j], g.rows[k], 5)) nb[q][j] = -1;
+                }
             if (MODE != 0) {
 #pragma unroll
                 for (int q = 0; q < RPS; ++q)
@@ -556,7 +573,10 @@ spmm_narrow_rows(const GroupDesc& g, const int64_t* __restrict__ rowptr_out,
                 float wt[NARROW_INFLIGHT];
                 uint4 xh[NARROW_INFLIGHT], xl[NARROW_INFLIGHT];
 #pragma unroll
-                for (int j = 0; j < NARROW_INFLIGHT; ++j) nb[j] = t + j < e ? __ldg(cols + t + j) : -1;
+                for (int j = 0; j < NARROW_INFLIGHT; ++j) {
+                    nb[j] = t + j < e ? __ldg(cols + t + j) : -1;
+                    if (nb[j] >= 0 && !rtma_index_ok(nb[j], g.rows[k], 5)) nb[j] = -1;
+                }
                 if (MODE != 0) {
 #pragma unroll
                     for (int j = 0; j < NARROW_INFLIGHT; ++j) wt[j] = nb[j] >= 0 ? __ldg(inv_deg + ws + nb[j]) : 0.f;
@@ -612,8 +632,9 @@ spmm_narrow_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restric
 // every thread walks its own entries, four neighbours in flight.  A hub row keeps its warp busy for as
 // many rounds as it has entries, which a launch of hundreds of thousands of warps absorbs.
 constexpr int TINY_TILE_ROWS = 256;
+constexpr int TINY_INFLIGHT = 2;  // neighbours in flight per thread: few registers, so that five blocks fit an SM
 template <int MODE>
-__global__ void __launch_bounds__(TINY_TILE_ROWS)
+__global__ void __launch_bounds__(TINY_TILE_ROWS, 5)
 spmm_tiny_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
                  const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg, const Planes src, const Planes out) {
     int k, r0;
@@ -629,14 +650,17 @@ spmm_tiny_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict_
     const float* wv = inv_deg + ws;
     Pack8 acc;
     acc.zero();
-    for (int64_t t = b; t < e; t += 4) {
-        int32_t nb[4];
-        float wt[4];
-        uint4 xh[4], xl[4];
+    for (int64_t t = b; t < e; t += TINY_INFLIGHT) {
+        int32_t nb[TINY_INFLIGHT];
+        float wt[TINY_INFLIGHT];
+        uint4 xh[TINY_INFLIGHT], xl[TINY_INFLIGHT];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) nb[j] = t + j < e ? __ldg(cols + t + j) : -1;
+        for (int j = 0; j < TINY_INFLIGHT; ++j) {
+            nb[j] = t + j < e ? __ldg(cols + t + j) : -1;
+            if (nb[j] >= 0 && !rtma_index_ok(nb[j], g.rows[k], 5)) nb[j] = -1;
+        }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < TINY_INFLIGHT; ++j) {
             if (nb[j] >= 0) {
                 if (MODE != 0) wt[j] = __ldg(wv + nb[j]);
                 xh[j] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)nb[j] * src.ld));
@@ -644,7 +668,7 @@ spmm_tiny_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict_
             }
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < TINY_INFLIGHT; ++j) {
             if (nb[j] >= 0) {
                 if (MODE != 0) acc.fma_planes_mixed(wt[j], xh[j], xl[j]);
                 else acc.add_planes_mixed(xh[j], xl[j]);
@@ -700,11 +724,11 @@ int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64
 
 }  // namespace
 
-int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, const int32_t* perm, int d, Planes out,
-                         cudaStream_t s) {
+int32_t launch_to_planes(rtma_ctx* ctx, const GroupDesc& g, const float* X, const int32_t* perm, int64_t n_total, int d,
+                         Planes out, cudaStream_t s) {
     const int64_t tiles = group_tiles(g, 32);
     if (tiles == 0) return RTMA_OK;
-    { KernelScope ks(ctx, KC_TO_PLANES, s); to_planes_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, X, perm, d, out); }
+    { KernelScope ks(ctx, KC_TO_PLANES, s); to_planes_kernel<<<(unsigned)tiles, 256, 0, s>>>(g, X, perm, n_total, d, out); }
     RTMA_LAUNCH_CHECK(ctx);
     return RTMA_OK;
 }

@@ -103,8 +103,9 @@ def tols(gemm_dtype):
     if gemm_dtype == 1:   # operands rounded to bf16 (2^-9 each), fp32 accumulation
         return TOL_BF16, TOL_BF16, TOL_BF16, TOL_BF16, 4e-3, 0.01
     # fp32-accurate products: the kernel's pre-activations carry about 1e-6 of relative error, so
-    # of the order of 1e-6 of all units straddle the kink differently from the fp64 oracle
-    return TOL_ACT, TOL_GRAD, TOL_PARAM, 1e-5, 2e-5, 1e-5
+    # of the order of 1e-6 of all units straddle the kink differently from the fp64 oracle (measured:
+    # 0 to 7 per part on the scaled shapes, 17 of 12.7 M on a whole Medium part, i.e. 1.3e-6)
+    return TOL_ACT, TOL_GRAD, TOL_PARAM, 1e-5, 2e-5, 4e-6
 
 
 def _param_segments(variant, dims):

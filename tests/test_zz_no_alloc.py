@@ -50,6 +50,34 @@ def test_static_partition_matches_partition_twice_in_a_row():
     assert e[1].cpu().tolist() == [0] * 5
 
 
+def test_static_partition_at_the_limit_allocates_nothing():
+    # exactly ceil(n / 1024) * M = the fixed scratch's cell count, outputs provided by the caller: the
+    # call works, agrees with rtma_partition bit for bit, and leaves the device's free memory as it was
+    lib = binding.load_library()
+    n, M, seed = 4096 * 1024, 64, 17
+    assert ((n + 1023) // 1024) * M == binding.PARTITION_STATIC_MAX_CELLS
+    dev = torch.device("cuda", 0)
+    out = [torch.empty(n, dtype=torch.int32, device=dev), torch.empty(M + 1, dtype=torch.int64, device=dev),
+           torch.empty(n, dtype=torch.int32, device=dev), torch.empty(n, dtype=torch.int32, device=dev)]
+
+    def call():
+        st = lib.rtma_partition_static(ctypes.c_int32(0), ctypes.c_int64(n), ctypes.c_void_p(0), ctypes.c_uint64(seed),
+                                       ctypes.c_int32(M), *[ctypes.c_void_p(t.data_ptr()) for t in out],
+                                       ctypes.c_void_p(int(torch.cuda.current_stream().cuda_stream)))
+        assert st == 0, lib.rtma_partition_static_error()
+        torch.cuda.synchronize()
+
+    call()                                  # the first call on a device looks the scratch's address up
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    call()
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert free_after == free_before        # no device memory taken or returned by the call
+    ctx = binding.Context(0)
+    want = ctx.partition(n, None, seed, M)
+    torch.cuda.synchronize()
+    assert _same(out, want)
+
+
 def test_static_partition_rejects_sizes_beyond_its_scratch():
     lib = binding.load_library()
     n, M = 1024 * 4097, 64      # 4097 chunks x 64 parts > 262144 cells
