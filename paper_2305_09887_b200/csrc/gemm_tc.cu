@@ -142,16 +142,8 @@ struct RowsArgs {
     int single;            // 1: operands rounded to bf16 (hi planes only, one MMA per product)
     const __nv_bfloat16* gate_hi;  // plane output only: entries whose gate value (same row and column,
                                    // leading dimension of out_planes) is <= 0 become 0; NULL: none
-    // Fused head (plane output, one column tile): besides H = act(...) the epilogue forms T = H Wh for the
-    // next (last) layer's head_nsrc weight matrices of head_c classes each -- at most HEAD_MAX_OUT products
-    // per row -- and writes it as planes, class c of matrix m in column m * head_cp + c.  head_w == NULL: none.
-    const float* head_w;           // parameters; the head layer's first weight matrix of part i starts at
-    int64_t head_off;              //   head_w + i * P + head_off, [N][head_c] row-major, the second one behind it
-    int head_c, head_cp, head_nsrc;
-    Planes head_T;
     int* error_word;
 };
-constexpr int HEAD_MAX_OUT = 4;
 
 // Persistent: a block walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... (tile = row tile x
 // column tile, column tiles of one row tile adjacent).  Two accumulator buffers in tensor
@@ -312,13 +304,6 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
             const float* bias = a.bias_offset >= 0 ? a.params + (int64_t)a.g.part[k] * a.P + a.bias_offset : nullptr;
             const int rows_here = min(32, a.g.rows[k] - (r0 + q * 32));  // live rows of this warp's quarter
             const int64_t orow0 = a.g.row_ws[k] + r0 + q * 32;
-            float hacc[4][HEAD_MAX_OUT];  // fused head: partial products of the thread's four rows
-#pragma unroll
-            for (int it = 0; it < 4; ++it)
-#pragma unroll
-                for (int o = 0; o < HEAD_MAX_OUT; ++o) hacc[it][o] = 0.f;
-            const int head_out = a.head_nsrc * a.head_c;
-            const float* head_w = (PLANES_OUT && a.head_w) ? a.head_w + (int64_t)a.g.part[k] * a.P + a.head_off : nullptr;
             for (int c0 = col_phase * 32; c0 < BN; c0 += 64) {
                 // the gate words this thread will need after the transpose, requested before the
                 // accumulator is read so that their latency hides behind it
@@ -383,17 +368,6 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                     float bv[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) bv[e] = (bias && col_ok && n + e < a.N) ? __ldg(bias + n + e) : 0.f;
-                    float hw[8][HEAD_MAX_OUT];  // fused head: the weights of the thread's eight columns
-                    if (head_w) {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e)
-#pragma unroll
-                            for (int o = 0; o < HEAD_MAX_OUT; ++o) {
-                                const int m = o / a.head_c, c = o - m * a.head_c;  // output o = class c of weight matrix m
-                                hw[e][o] = (o < head_out && col_ok && n + e < a.N)
-                                               ? __ldg(head_w + ((int64_t)m * a.N + n + e) * a.head_c + c) : 0.f;
-                            }
-                    }
                     // the thread's 16 bytes of row (lane >> 2) of the block, in either plane; the four
                     // rows it finishes are 8 rows apart
                     const uint32_t out_row_bytes = (uint32_t)a.out_planes.ld * 2u;
@@ -424,12 +398,6 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
                                     if (!(gate > 0.f)) x.v[e] = 0.f;
                                 }
                             }
-                            if (head_w) {
-#pragma unroll
-                                for (int e = 0; e < 8; ++e)
-#pragma unroll
-                                    for (int o = 0; o < HEAD_MAX_OUT; ++o) hacc[it][o] = fmaf(x.v[e], hw[e][o], hacc[it][o]);
-                            }
                             uint4 h, l;
                             x.to_planes_lean(h, l);
                             *reinterpret_cast<uint4*>(oh + (size_t)(it * 8) * out_row_bytes) = h;
@@ -440,47 +408,6 @@ __global__ void __launch_bounds__(ROWS_THREADS, 1) tc_rows_kernel(const __grid_c
             }
             tc::tc_fence_before_sync();
             tc::mbar_arrive(&pb.acc_empty[buf]);  // all 256 epilogue threads arrive: the buffer may be overwritten
-            if constexpr (PLANES_OUT) {
-                if (a.head_w) {  // uniform over the block
-                    // a row's products: the four lanes that share it, then the two warps of the quarter (which
-                    // took alternate column chunks) through the second warp's staging slab
-#pragma unroll
-                    for (int it = 0; it < 4; ++it)
-#pragma unroll
-                        for (int o = 0; o < HEAD_MAX_OUT; ++o) {
-                            hacc[it][o] += __shfl_xor_sync(0xffffffffu, hacc[it][o], 1);
-                            hacc[it][o] += __shfl_xor_sync(0xffffffffu, hacc[it][o], 2);
-                        }
-                    float* slab = reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes + (size_t)((ew & 3) + 4) * ROWS_STAGING_BYTES);
-                    if (col_phase == 1 && (lane & 3) == 0) {
-#pragma unroll
-                        for (int it = 0; it < 4; ++it)
-#pragma unroll
-                            for (int o = 0; o < HEAD_MAX_OUT; ++o) slab[(it * 8 + (lane >> 2)) * HEAD_MAX_OUT + o] = hacc[it][o];
-                    }
-                    asm volatile("bar.sync %0, 64;" ::"r"(2 + q) : "memory");
-                    if (col_phase == 0 && (lane & 3) == 0) {
-#pragma unroll
-                        for (int it = 0; it < 4; ++it) {
-                            const int row = it * 8 + (lane >> 2);
-                            if (row < rows_here) {
-#pragma unroll
-                                for (int o = 0; o < HEAD_MAX_OUT; ++o) {
-                                    if (o < head_out) {
-                                        const int m = o / a.head_c, c = o - m * a.head_c;
-                                        __nv_bfloat16 th, tl;
-                                        split_bf16(hacc[it][o] + slab[row * HEAD_MAX_OUT + o], th, tl);
-                                        const int64_t at = (orow0 + row) * a.head_T.ld + m * a.head_cp + c;
-                                        a.head_T.hi[at] = th;
-                                        a.head_T.lo[at] = tl;
-                                    }
-                                }
-                            }
-                        }
-                    }
-                    asm volatile("bar.sync %0, 64;" ::"r"(2 + q) : "memory");  // the slab goes back to the transposes
-                }
-            }
         }
     }
     tc::tc_fence_before_sync();
@@ -829,12 +756,6 @@ TcLayerPlan tc_plan_head(LayerShape ls, int head_cp) {
     return p;
 }
 
-bool tc_fused_head_applies(const LayerShape& below, const LayerShape& head, bool single) {
-    // one column tile holds the whole row (so a tile sees every input of the head), few enough products
-    // per row for the epilogue's registers, full-precision operands
-    return !single && below.d_out <= 256 && head.d_in == below.d_out && head.nsrc * head.d_out <= HEAD_MAX_OUT;
-}
-
 size_t tc_prep_elems(const TcLayerPlan& p, bool with_dgrad) {
     return 2 * ((size_t)p.Npad_f * p.Kf + (with_dgrad ? (size_t)p.Npad_d * p.Kd : 0));
 }
@@ -888,7 +809,7 @@ static int32_t launch_rows(rtma_ctx* ctx, RowsArgs& a, int kclass, cudaStream_t 
 int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                           const float* params, Planes H, Planes N, const __nv_bfloat16* Bf_hi,
                           const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, bool single,
-                          cudaStream_t s, const TcFusedHead* head) {
+                          cudaStream_t s) {
     RowsArgs a{};
     a.g = g;
     a.single = single ? 1 : 0;
@@ -916,16 +837,6 @@ int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, cons
     a.bias_offset = ls.has_bias ? ls.param_offset + (int64_t)ls.nsrc * ls.d_in * ls.d_out : -1;
     a.relu = relu ? 1 : 0;
     a.gate_hi = nullptr;
-    if (head) {
-        if (!tc_fused_head_applies(ls, head->layer, single) || !out_planes.hi)
-            return rtma_fail(ctx, RTMA_ERR_INVALID_ARG, "internal: fused head on a layer it does not apply to");
-        a.head_w = params;
-        a.head_off = head->layer.param_offset;
-        a.head_c = head->layer.d_out;
-        a.head_cp = head->cp;
-        a.head_nsrc = head->layer.nsrc;
-        a.head_T = head->T;
-    }
     return launch_rows(ctx, a, KC_GEMM_FWD, s);
 }
 

@@ -484,8 +484,6 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], false, wave_order, ticket, s));
                 else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Hl[0], Nl[0], m.dims[0], wave_order, ticket, s));
             }
-            // the head's product H [Ws | Wn] comes out of the epilogue of the layer below where that applies
-            const bool fused_head = head && m.L >= 2 && !m.post && tc_fused_head_applies(m.layer[m.L - 2], m.layer[m.L - 1], single_pass);
             const GroupDesc wave = g;   // all parts of the wave, with their scratch rows
 
             for (int step = 0; step < wave_steps; ++step) {
@@ -538,9 +536,8 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                         hs.nsrc = 1;
                         hs.d_out = hsrc * Cp;
                         hs.has_bias = 0;
-                        if (!fused_head)  // else T came out of the epilogue of the layer below
-                            RTMA_TRY(launch_tc_forward(ctx, g, hs, tcp[l], rows, params, Hl[l], Hl[l], Bf_hi[l], Bf_lo[l], T, no_mat, false,
-                                                       single_pass, s));
+                        RTMA_TRY(launch_tc_forward(ctx, g, hs, tcp[l], rows, params, Hl[l], Hl[l], Bf_hi[l], Bf_lo[l], T, no_mat, false,
+                                                   single_pass, s));
                         if (m.gcn) RTMA_TRY(launch_spmm_gcn(ctx, g, rowptr_out, col_out, inv_deg, T, NT, C, false, order, ticket, s));
                         else RTMA_TRY(launch_spmm_mean(ctx, g, rowptr_out, col_out, inv_deg, Planes{T.hi + Cp, T.lo + Cp, T.ld}, NT, C,
                                                        order, ticket, s));
@@ -559,10 +556,9 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                     }
                     const bool last = l == m.L - 1;
                     if (last || !m.post) {
-                        const TcFusedHead fh{m.layer[m.L - 1], Cp, T};
                         RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
                                                    last ? (link ? R : no_planes) : Hl[l + 1], (last && !link) ? logits : no_mat, !last,
-                                                   single_pass, s, (fused_head && l == m.L - 2) ? &fh : nullptr));
+                                                   single_pass, s));
                     } else {  // pre-activations kept; normalisation and PReLU in a pass of their own
                         RTMA_TRY(launch_tc_forward(ctx, g, m.layer[l], tcp[l], rows, params, Hl[l], Nl[l], Bf_hi[l], Bf_lo[l],
                                                    Zl[l], no_mat, false, single_pass, s));

@@ -197,19 +197,10 @@ int32_t launch_tc_weight_prep(rtma_ctx* ctx, const GroupDesc& g, const TcPrepJob
                               cudaStream_t s);
 // out = act([H | N] [Ws; Wn] + b), or act(N W + b) for a one-matrix layer (H is then ignored):
 // split planes when out_planes.hi != NULL, else fp32 out_f32.
-// head != NULL: the epilogue also forms T = out [Ws | Wn] of the NEXT layer `head->layer` (the last one, in
-// its head form) from the rows it has just produced, and writes it to head->T (planes, blocks of head->cp
-// columns): that layer's own product launch is then not needed.  Only where tc_fused_head_applies.
-struct TcFusedHead {
-    LayerShape layer;
-    int cp;
-    Planes T;
-};
-bool tc_fused_head_applies(const LayerShape& below, const LayerShape& head, bool single);
 int32_t launch_tc_forward(rtma_ctx* ctx, const GroupDesc& g, LayerShape ls, const TcLayerPlan& p, int64_t rows_total,
                           const float* params, Planes H, Planes N, const __nv_bfloat16* Bf_hi,
                           const __nv_bfloat16* Bf_lo, Planes out_planes, Mat out_f32, bool relu, bool single,
-                          cudaStream_t s, const TcFusedHead* head = nullptr);
+                          cudaStream_t s);
 // H <- ([dZ | Q] [Ws^T ; Wn^T]) (or Q W^T for a one-matrix layer), Q = the transposed aggregation
 // of dZ.  gate: on entry H holds the layer's input activations and entries where H <= 0 become 0
 // (the ReLU gate), so that on exit H is the gradient with respect to the previous layer's

@@ -62,6 +62,24 @@ def test_gcn_prelu_layernorm_odd_widths(util, dims):
     util.check_k_steps_and_average(w, got, want, 2, variant=(1, 1, 1), params0=p0)
 
 
+@pytest.mark.parametrize("variant,dims", [((0, 0, 0), (64, 64, 2)), ((0, 0, 0), (24, 96, 1)), ((0, 0, 0), (64, 64, 3)),
+                                          ((1, 0, 0), (64, 64, 4)), ((1, 0, 0), (40, 200, 2)), ((0, 0, 0), (32, 64, 48, 2)),
+                                          ((0, 1, 1), (64, 64, 2))])
+def test_heads_with_very_few_classes(util, variant, dims):
+    # Few classes take paths of their own: the last layer aggregated after its product at class width by one
+    # thread per row, its input gradient on the plain ALUs (up to 4 classes), and -- in a two-layer model with
+    # at most 4 products per output and no separate activation pass -- generated inside the weight-gradient
+    # kernel of the first layer instead of being written and read.  GraphSAGE (two weight matrices) and GCN
+    # (one), one to four classes, two and three layers, a PReLU + LayerNorm model (which keeps the written dgrad).
+    w = inputs.tiny()
+    w.dims = dims
+    w.X = inputs.normal_features(w.graph.n, dims[0], 31)
+    w.y = inputs.uniform_labels(w.graph.n, dims[-1], 32)
+    p0 = _start(variant, dims, 33)
+    got, want = util.check_one_step(w, M=3, variant=variant, params0=p0)
+    util.check_k_steps_and_average(w, got, want, 3, variant=variant, params0=p0)
+
+
 def test_variant_flags_are_validated(util, tiny_workload):
     w = tiny_workload
     got = util.gpu_preprocess(w)
