@@ -425,6 +425,26 @@ def average(params: np.ndarray):
     return out, glob
 
 
+def sample_hop(rowptr, col, frontier, fanout: int, seed: int, hop: int):
+    """One hop of the neighbour sampler on one part's subgraph.  frontier: ascending distinct local
+    ids.  Returns (block_rowptr[len(frontier)+1], block_col, next_frontier)."""
+    rowptr = _i64(rowptr)
+    col = _i32(col)
+    frontier = _i32(frontier)
+    n = rowptr.size - 1
+    fs = frontier.size
+    block_rowptr = np.empty(fs + 1, dtype=np.int64)
+    next_frontier = np.empty(n, dtype=np.int32)
+    f = lib().orc_sample_hop
+    f.restype = ctypes.c_int64
+    args = [ctypes.c_int64(n), _p(rowptr, c_i64p), _p(col, c_i32p), ctypes.c_int64(fs), _p(frontier, c_i32p),
+            ctypes.c_int32(fanout), ctypes.c_uint64(seed), ctypes.c_int32(hop), _p(block_rowptr, c_i64p)]
+    f(*args, None, _p(next_frontier, c_i32p))
+    block_col = np.empty(int(block_rowptr[-1]), dtype=np.int32)
+    size = f(*args, _p(block_col, c_i32p), _p(next_frontier, c_i32p))
+    return block_rowptr, block_col, next_frontier[:int(size)].copy()
+
+
 def sigmoid_l2_grad(rowptr, col, X, y, w):
     rowptr = _i64(rowptr)
     col = _i32(col)

@@ -28,6 +28,8 @@
 //   orc_link_*            the paper's task: link prediction with the Hadamard-product MLP
 //                         decoder (App. "Formulation of MLP Decoder") on given positive and
 //                         negative pairs (Sec. 4.1 "Mini-batch and Negative Sampling").
+//   orc_sample_hop        one hop of the GraphSAGE neighbour sampler that shrinks the message-flow
+//                         graph of a mini-batch (Sec. 4.1 "Mini-batch and Negative Sampling").
 //   orc_sigmoid_l2_grad   the 1-layer sigmoid / L2 model of Theorem 2, used
 //                         only to pin the aggregation against Eq.
 //                         (proof-2-exp-grad-central).
@@ -1143,6 +1145,68 @@ double orc_link_forward_backward_f64(const int32_t* variant, int32_t L, const in
                                      double* scores, double* preact, const int8_t* gates) {
     return link_forward_backward<double>(Variant{variant[0], variant[1], variant[2]}, L, dims, Kd, ddims, n, rowptr, col,
                                          X, B, pu, pv, label, params, grads, emb, scores, preact, gates);
+}
+
+// ---- neighbour sampling (Sec. 4.1 "Mini-batch and Negative Sampling") ---------------------------
+// One hop of the sampler that shrinks the message-flow graph: every node of the frontier keeps all
+// its entries when it has at most `fanout` of them, otherwise `fanout` of them drawn uniformly without
+// replacement.  The draw is counter based: entry number pos of node v at hop h gets the key
+//   key = S(S(seed xor ((h + 1) << 48)) xor ((v << 32) | pos)),   S = one SplitMix64 step,
+// and the entries with the smallest keys are kept (equal keys: the smaller position first) -- i.i.d.
+// keys make that a uniform sample.  The next frontier is the ascending union of the frontier and the
+// kept neighbours (a node needs its own features too); the hop's block is a CSR with one row per
+// frontier node, in frontier order, whose columns are positions in the next frontier and whose
+// entries keep the order they have in the node's row.  The paper gives neither fan-outs nor the
+// draw; both are inputs here.
+//   frontier        [frontier_size] ascending, distinct local ids
+//   block_rowptr    [frontier_size + 1]
+//   block_col       [at least sum of min(deg, fanout)]; NULL: sizes only
+//   next_frontier   [at most n]; returns its size
+int64_t orc_sample_hop(int64_t n, const int64_t* rowptr, const int32_t* col, int64_t frontier_size,
+                       const int32_t* frontier, int32_t fanout, uint64_t seed, int32_t hop,
+                       int64_t* block_rowptr, int32_t* block_col, int32_t* next_frontier) {
+    const uint64_t base = splitmix64_step(seed ^ ((uint64_t)(hop + 1) << 48));
+    std::vector<char> member((size_t)n, 0);
+    std::vector<std::vector<int32_t>> kept((size_t)frontier_size);
+    for (int64_t i = 0; i < frontier_size; ++i) {
+        const int64_t v = frontier[i];
+        member[(size_t)v] = 1;
+        const int64_t deg = rowptr[v + 1] - rowptr[v];
+        std::vector<int64_t> pos;  // kept positions, ascending
+        if (deg <= fanout) {
+            for (int64_t q = 0; q < deg; ++q) pos.push_back(q);
+        } else {
+            std::vector<std::pair<uint64_t, int64_t>> keyed;
+            for (int64_t q = 0; q < deg; ++q)
+                keyed.emplace_back(splitmix64_step(base ^ (((uint64_t)v << 32) | (uint64_t)q)), q);
+            std::sort(keyed.begin(), keyed.end());  // by key, then by position
+            for (int32_t q = 0; q < fanout; ++q) pos.push_back(keyed[(size_t)q].second);
+            std::sort(pos.begin(), pos.end());
+        }
+        for (int64_t q : pos) {
+            const int32_t u = col[rowptr[v] + q];
+            kept[(size_t)i].push_back(u);
+            member[(size_t)u] = 1;
+        }
+    }
+    std::vector<int64_t> index((size_t)n, -1);
+    int64_t next_size = 0;
+    for (int64_t v = 0; v < n; ++v)
+        if (member[(size_t)v]) {
+            index[(size_t)v] = next_size;
+            if (next_frontier) next_frontier[next_size] = (int32_t)v;
+            ++next_size;
+        }
+    block_rowptr[0] = 0;
+    for (int64_t i = 0; i < frontier_size; ++i) {
+        int64_t at = block_rowptr[i];
+        for (int32_t u : kept[(size_t)i]) {
+            if (block_col) block_col[at] = (int32_t)index[(size_t)u];
+            ++at;
+        }
+        block_rowptr[i + 1] = at;
+    }
+    return next_size;
 }
 
 // Theorem 2's model: z_v = sigmoid((A-bar X w)_v), L = 1/2 (y_v - z_v)^2 per
