@@ -319,17 +319,23 @@ def run_averaging_stress(args, local_rank):
     M, P = args.M or 32, 16 << 20
     params = torch.randn(M, P, dtype=torch.float32, device="cuda")
     glob = torch.empty(P, dtype=torch.float32, device="cuda")
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         ctx.aggregate(params, glob)
     torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
+    # one launch takes 0.7 ms: time at least 400 of them, so that the clock sampler (100 ms period) sees the region
+    args.steps = max(args.steps, 400)
+    time.sleep(0.5)                      # the sampler's first sample takes a few hundred milliseconds
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.begin()
     e0.record()
     for _ in range(args.steps):
         ctx.aggregate(params, glob)
     e1.record()
     torch.cuda.synchronize()
+    sampler.end()
+    ctx.check()
     clocks = sampler.stop()
     seconds = e0.elapsed_time(e1) / 1e3
     peaks = load_peaks()
@@ -341,7 +347,8 @@ def run_averaging_stress(args, local_rank):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "averaging_stress", "M": M, "P": P, "l2": "4 GiB touched per launch > L2"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "aggregate",
+                     "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
+                     "traffic": load_dram_traffic().get(("averaging_stress", "aggregate")), "kernel": "aggregate",
                      "peak_source": peaks["source"]},
         "gpu_launches": args.steps, "clocks": clocks}))
 
@@ -479,12 +486,12 @@ def run_link(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
-def kernel_sources_digest() -> str:
-    """Digest of the CUDA sources: ncu counters taken on other sources are not reported."""
+def kernel_sources_digest(files) -> str:
+    """Digest of the named CUDA sources: ncu counters taken on other sources are not reported."""
     import hashlib
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2305_09887_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
+    for name in sorted(files):
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(name.encode() + b"\0" + f.read())
     return h.hexdigest()[:16]
@@ -492,18 +499,22 @@ def kernel_sources_digest() -> str:
 
 def load_dram_traffic():
     """{(workload, kernel class): DRAM bytes per launch} from the ncu capture recorded in
-    profiles/dram_traffic.txt (lines: workload, class, bytes per launch, digest of the kernel
-    sources the capture ran on).  Entries taken on other sources than the present ones are dropped."""
+    profiles/dram_traffic.txt (lines: workload, class, bytes per launch, digest, the comma-separated
+    sources of the class's kernels the digest was taken over).  Entries whose sources have changed
+    since the capture are dropped."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     out = {}
     if not os.path.exists(path):
         return out
-    digest = kernel_sources_digest()
     with open(path) as f:
         for ln in f:
             parts = ln.split()
-            if len(parts) == 4 and not ln.startswith("#") and parts[3] == digest:
-                out[(parts[0], parts[1])] = float(parts[2])
+            if len(parts) == 5 and not ln.startswith("#"):
+                try:
+                    if kernel_sources_digest(parts[4].split(",")) == parts[3]:
+                        out[(parts[0], parts[1])] = float(parts[2])
+                except OSError:
+                    pass
     return out
 
 

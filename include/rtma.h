@@ -287,6 +287,29 @@ int32_t rtma_link_steps(rtma_ctx* ctx, const rtma_model_desc* model, const rtma_
                         float* loss_out, int32_t record_step, float* grads_out, float* emb_out,
                         float* score_out, void* const* streams);
 
+/* ---- neighbour sampling (Sec. 4.1 "Mini-batch and Negative Sampling") ---------------------
+ * One hop of the GraphSAGE neighbour sampler that shrinks the message-flow graph of a mini-batch, on
+ * one part's induced subgraph (rowptr = the part's n+1 zero-based offsets inside rowptr_out, col =
+ * its columns inside col_out).  The paper names the sampler and gives neither fan-outs nor the draw;
+ * both are inputs here.  Every frontier node with at most `fanout` entries keeps them all, otherwise
+ * it keeps the `fanout` entries with the smallest keys
+ *     key = S(S(seed ^ ((hop + 1) << 48)) ^ ((v << 32) | position)),   S = one SplitMix64 step
+ * (equal keys: the smaller position first): a uniform sample without replacement that depends only
+ * on (seed, hop, node, position).  Start with the distinct end points of the batch's pairs as the
+ * frontier and hop = 0; call again with next_frontier as the frontier and hop + 1, once per layer.
+ *   frontier      [frontier_size] int32, ascending and distinct local ids.
+ *   block_rowptr  [frontier_size + 1] int64: the hop's block, one row per frontier node.
+ *   block_col     int32, room for sum_v min(deg(v), fanout) <= frontier_size * fanout entries:
+ *                 positions in next_frontier, a row's entries in the order they have in the graph.
+ *   next_frontier [n] int32 (room for every node): ascending union of the frontier and the kept
+ *                 neighbours; next_size [1] int64 (device) receives its length.
+ * Read next_size back (after draining the stream) before the next hop.  The result is unique: no
+ * atomics on data, equal bit for bit from run to run.                                          */
+int32_t rtma_sample_hop(rtma_ctx* ctx, int64_t n, const int64_t* rowptr, const int32_t* col,
+                        int64_t frontier_size, const int32_t* frontier, int32_t fanout, uint64_t seed,
+                        int32_t hop, int64_t* block_rowptr, int32_t* block_col, int32_t* next_frontier,
+                        int64_t* next_size, void* stream);
+
 /* ---- R2: aggregation (Algorithm 1, phi = plain average; Algorithm 2, overwrite) ---------
  * Wbar[j] = (1/M) sum_i params[i][j]; every replica is overwritten with Wbar; global_out
  * [P] (or NULL) also receives it.  M = 1 leaves the parameters unchanged.                 */

@@ -24,7 +24,7 @@ EXPORTS = (
     "rtma_aggregate", "rtma_sgd_aggregate", "rtma_train_host", "rtma_profile", "rtma_profile_read",
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
     "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout", "rtma_link_param_count",
-    "rtma_link_steps", "rtma_set_workspace_limit", "rtma_local_steps_gathered", "rtma_bounds_checked",
+    "rtma_link_steps", "rtma_set_workspace_limit", "rtma_local_steps_gathered", "rtma_bounds_checked", "rtma_sample_hop",
 )
 KERNEL_CLASSES = 21
 
@@ -208,6 +208,28 @@ class Context:
         self._check(self._lib.rtma_profile_read(self._h, ms, cnt), "rtma_profile_read")
         return {self._lib.rtma_kernel_class_name(ctypes.c_int32(i)).decode(): (float(ms[i]), int(cnt[i]))
                 for i in range(KERNEL_CLASSES)}
+
+    # ---- neighbour sampling ---------------------------------------------------------
+    def sample_hop(self, rowptr, col, frontier, fanout: int, seed: int, hop: int, stream=None):
+        """One hop of the neighbour sampler on one part (rowptr: its n+1 zero-based int64 offsets, col: its
+        int32 columns, frontier: ascending distinct int32 local ids).  Returns (block_rowptr, block_col,
+        next_frontier), the last two cut to their lengths (which synchronises)."""
+        dev = self.device
+        _need(rowptr, torch.int64, "rowptr", dev)
+        _need(col, torch.int32, "col", dev)
+        _need(frontier, torch.int32, "frontier", dev)
+        n, fs = int(rowptr.numel()) - 1, int(frontier.numel())
+        block_rowptr = torch.empty(fs + 1, dtype=torch.int64, device=dev)
+        cap = min(fs * int(fanout), int(col.numel())) if fs else 0
+        block_col = torch.empty(max(cap, 1), dtype=torch.int32, device=dev)
+        next_frontier = torch.empty(max(n, 1), dtype=torch.int32, device=dev)
+        next_size = torch.zeros(1, dtype=torch.int64, device=dev)
+        st = self._lib.rtma_sample_hop(
+            self._h, ctypes.c_int64(n), _ptr(rowptr), _ptr(col), ctypes.c_int64(fs), _ptr(frontier), ctypes.c_int32(fanout),
+            ctypes.c_uint64(seed), ctypes.c_int32(hop), _ptr(block_rowptr), _ptr(block_col), _ptr(next_frontier),
+            _ptr(next_size), ctypes.c_void_p(_stream_handle(stream)))
+        self._check(st, "rtma_sample_hop")
+        return block_rowptr, block_col[:int(block_rowptr[-1].item())], next_frontier[:int(next_size.item())]
 
     # ---- R1 -------------------------------------------------------------------------
     def partition(self, n: int, group_id, seed: int, M: int, stream=None, grouped: bool = False):
