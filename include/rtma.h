@@ -84,6 +84,21 @@ size_t rtma_workspace_bytes(const rtma_ctx* ctx);
  * results are bit for bit those of a single wave.  For hosts that share the GPU with other
  * tenants of a fixed memory budget.  The paper has no counterpart.                          */
 int32_t rtma_set_workspace_limit(rtma_ctx* ctx, size_t bytes);
+/* How rtma_local_steps forms the mean aggregation Abar H (Theorem 2) and its transpose for a part:
+ *   0  always by gathering the neighbours' rows;
+ *   1  (default) per part: where at least half of the entries of a sample of its rows (every 64th)
+ *      have their column within 128 rows of the row's 128-row tile, and those rows have 4 entries or
+ *      more on average - the nodes of a super-node stored together (Sec. 3.2, rows ordered by
+ *      super-node as rtma_partition_grouped leaves them) - the entries inside that window are taken
+ *      from dense tiles on the tensor cores and only the others are gathered;
+ *   2  the tensor-core tiles for every part (for tests).
+ * The decision depends on the part alone, so a trainer's results do not depend on which other
+ * trainers share its call; a part in which some row repeats an entry inside that window always
+ * gathers.  GCN layers, and rows of fewer than 16 values, always gather.  In modes 1 and 2 the
+ * training calls wait once per wave, while they set up, for the stream to deliver the per-part
+ * decision (twice where some part takes the tiles); in mode 0 they only enqueue.
+ * Returns RTMA_ERR_INVALID_ARG for any other mode.                                           */
+int32_t rtma_set_dense_aggregation(rtma_ctx* ctx, int32_t mode);
 
 /* ---- R1: partition function (Sec. 3.2.2, RandomTMA and SuperTMA) -----------------------
  * part_id[v] = h(seed XOR g(v)) mod M, where h is one step of the SplitMix64 generator and
@@ -213,7 +228,8 @@ typedef struct {
  *   loss_out [M][K] float or NULL         loss of every step of every trainer.
  *   streams  HOST array of M cudaStream_t: trainer i runs on streams[i].  Trainers that
  *            share a stream are batched into common launches; distinct streams run
- *            concurrently.  The call returns once everything is enqueued.
+ *            concurrently.  The call returns once everything is enqueued; while it sets
+ *            up it waits for each stream once or twice unless rtma_set_dense_aggregation(ctx, 0).
  * Scratch is taken from the context (grows if needed).  A part may hold at most 2^31 - 1
  * nodes (RTMA_ERR_INVALID_ARG) and 2^31 - 1 kept entries (RTMA_ERR_OVERFLOW).               */
 int32_t rtma_local_steps(rtma_ctx* ctx, const rtma_model_desc* model, int32_t M,

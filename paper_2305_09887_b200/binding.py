@@ -25,6 +25,7 @@ EXPORTS = (
     "rtma_kernel_class_name", "rtma_check", "rtma_partition_static", "rtma_partition_static_error",
     "rtma_local_steps_var", "rtma_aggregate_masked", "rtma_selftest_wait_timeout", "rtma_link_param_count",
     "rtma_link_steps", "rtma_set_workspace_limit", "rtma_local_steps_gathered", "rtma_bounds_checked", "rtma_sample_hop",
+    "rtma_set_dense_aggregation",
 )
 KERNEL_CLASSES = 21
 
@@ -192,6 +193,10 @@ class Context:
     def set_workspace_limit(self, nbytes: int):
         """Caps the context's scratch arena (0 = no cap); rtma_local_steps then runs in waves."""
         self._check(self._lib.rtma_set_workspace_limit(self._h, ctypes.c_size_t(nbytes)), "rtma_set_workspace_limit")
+
+    def set_dense_aggregation(self, mode: int):
+        """0: always gather; 1 (default): tensor-core tiles for parts with local neighbourhoods; 2: for every part."""
+        self._check(self._lib.rtma_set_dense_aggregation(self._h, ctypes.c_int32(mode)), "rtma_set_dense_aggregation")
 
     def check(self):
         """Synchronises and raises if a kernel gave up on a bounded device-side wait."""

@@ -31,7 +31,8 @@ struct rtma_ctx {
     // device words: [0] raised by a kernel whose bounded wait ran out, [1] by the symmetry check of
     // the local-training calls
     int* error_word = nullptr;
-    bool rows_configured = false, wgrad_configured = false;  // shared-memory opt-in of the tensor-core kernels on this device
+    bool rows_configured = false, wgrad_configured = false, dense_configured = false;  // shared-memory opt-in of the tensor-core kernels on this device
+    int dense_mode = 1;           // aggregation on the tensor cores: 0 never, 1 where a part's rows are local, 2 every part
     int64_t launches[KC_COUNT] = {0};
     std::vector<ProfSpan> spans;        // recorded since the last read
     std::vector<cudaEvent_t> event_pool;  // spare events

@@ -150,6 +150,12 @@ extern "C" int32_t rtma_set_workspace_limit(rtma_ctx* ctx, size_t bytes) {
     return RTMA_OK;
 }
 
+extern "C" int32_t rtma_set_dense_aggregation(rtma_ctx* ctx, int32_t mode) {
+    if (!ctx || mode < 0 || mode > 2) return RTMA_ERR_INVALID_ARG;
+    ctx->dense_mode = mode;
+    return RTMA_OK;
+}
+
 int32_t order_after_training(rtma_ctx* ctx, cudaStream_t s) {
     for (size_t i = 0; i < ctx->trained_streams.size(); ++i)
         if (ctx->trained_streams[i] != s) RTMA_CUDA(ctx, cudaStreamWaitEvent(s, ctx->trained_events[i], 0));

@@ -17,7 +17,8 @@
 // 8 values (16 bytes per plane).  Rows of at most 64 values have a kernel of their own, in which
 // groups of lanes own one row each (spmm_narrow_kernel).  Where most neighbours of a row are rows
 // nearby (super-nodes stored together), groups are handed out eight at a time to a block, so that
-// its warps share their source rows through L1 (locality_probe_kernel decides, once per call).
+// its warps share their source rows through L1 (locality_probe_kernel decides, once per call); parts
+// that are local enough for it leave these kernels altogether for the tensor-core tiles of spmm_tc.cu.
 #include <algorithm>
 #include <climits>
 
@@ -276,6 +277,7 @@ spmm_rows(const GroupDesc& g, const int64_t* __restrict__ rowptr_out,
         k += more;
     }
     if (k < 0 || k >= g.num) continue;  // cannot happen for a ticket below last_ticket
+    if (order.dense && order.dense[g.part[k]]) continue;  // this part is aggregated on the tensor cores
     const int i0 = (grp - first) * SPMM_ROWS_PER_WARP;
     const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
     const int64_t ws = g.row_ws[k];
@@ -475,6 +477,7 @@ spmm_narrow_rows(const GroupDesc& g, const int64_t* __restrict__ rowptr_out,
             k += more;
         }
         if (k < 0 || k >= g.num) continue;  // cannot happen for a ticket below last_ticket
+        if (order.dense && order.dense[g.part[k]]) continue;  // this part is aggregated on the tensor cores
         const int i0 = (grp - first) * SPMM_ROWS_PER_WARP;
         const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
         const int64_t ws = g.row_ws[k];
@@ -694,6 +697,11 @@ int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
     if (groups >= (int64_t(1) << 31) - 65536) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
+    // parts flagged in order.dense are skipped by the kernels below and done by the tensor-core path afterwards
+    const bool dense_on = MODE != 2 && order.dense != nullptr && spmm_dense_applies(d);
+    if (!dense_on) order.dense = nullptr;
+    if (dense_on && order.all_dense)
+        return launch_spmm_dense(ctx, kclass, g, rowptr_out, col_out, inv_deg, order, src, out, d, MODE == 1, s);
     if (d <= 8) {
         const int64_t tiles = group_tiles(g, TINY_TILE_ROWS);
         { KernelScope ks(ctx, kclass, s); spmm_tiny_kernel<MODE><<<(unsigned)tiles, TINY_TILE_ROWS, 0, s>>>(g, rowptr_out, col_out, inv_deg, src, out); }
@@ -719,6 +727,8 @@ int32_t dispatch_spmm(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64
     else return rtma_fail(ctx, RTMA_ERR_UNSUPPORTED, "aggregation width %d > 1024", d);
 #undef RTMA_SPMM
     RTMA_LAUNCH_CHECK(ctx);
+    if (dense_on)
+        RTMA_TRY(launch_spmm_dense(ctx, kclass, g, rowptr_out, col_out, inv_deg, order, src, out, d, MODE == 1, s));
     return RTMA_OK;
 }
 
@@ -789,7 +799,7 @@ int64_t spmm_order_entries(const GroupDesc& g) { return group_tiles(g, SPMM_ROWS
 
 int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                           int64_t entries, int* count, int* list, SpmmOrder* order, cudaStream_t s) {
-    *order = SpmmOrder{nullptr, nullptr, 0, nullptr};
+    *order = SpmmOrder{nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr, nullptr, false};
     const int64_t groups = group_tiles(g, SPMM_ROWS_PER_WARP);
     if (groups == 0) return RTMA_OK;
     if (groups >= (int64_t(1) << 30)) return rtma_fail(ctx, RTMA_ERR_OVERFLOW, "too many row groups");
@@ -801,6 +811,6 @@ int32_t launch_spmm_order(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowp
     unsigned long long* near_total = reinterpret_cast<unsigned long long*>(count + 2);
     { KernelScope ks(ctx, KC_INV_DEGREE, s); locality_probe_kernel<<<grid, 256, 0, s>>>(g, rowptr_out, col_out, group_tiles(g, 1), near_total); }
     RTMA_LAUNCH_CHECK(ctx);
-    *order = SpmmOrder{count, list, heavy, near_total};
+    *order = SpmmOrder{count, list, heavy, near_total, nullptr, 0, nullptr, nullptr, nullptr, false};
     return RTMA_OK;
 }

@@ -114,6 +114,7 @@ int64_t aligned_rows(int64_t n_p) { return ceil_div(n_p, GROUP_ROW_ALIGN) * GROU
 ScratchPlan plan_scratch(const Model& m, bool head, bool record) {
     ScratchPlan sp{};
     size_t per_row = sizeof(float);              // inv_deg
+    per_row += DENSE_WINDOW / 8 + sizeof(int32_t) * DENSE_LEFT_CAP + 1;  // tensor-core aggregation: window masks, entries outside
     per_row += 4 * planes_ld(m.dims[0]);         // X as planes
     int q_width = 0;
     for (int l = 0; l < m.L; ++l) {
@@ -188,7 +189,7 @@ size_t part_scratch_bytes(const Model& m, const ScratchPlan& sp, int64_t n_p, in
     return sp.per_row_bytes * rows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(n_p, 32) + 256) +
            sp.per_pair_bytes * prows + sizeof(float) * (64 * sp.max_layer_params + (size_t)ceil_div(pairs, 32) + 256) +
            sizeof(float) * ((size_t)ceil_div(pairs, 64) + 1) * (2 * sp.post_width + 1) +
-           sizeof(int) * ((size_t)ceil_div(n_p, 8) + 64) +  // processing order of the aggregation kernels
+           sizeof(int) * ((size_t)ceil_div(n_p, 8) + 64 + 7 * RTMA_MAX_PARTS) +  // processing order of the aggregation kernels, per-part flags
            sizeof(float) * ((size_t)ceil_div(n_p, 64) + 1) * (2 * sp.post_width + 1) +  // per-tile sums of d gamma, d beta, d a
            sp.prep_bytes + 256 * matrices;
 }
@@ -437,9 +438,15 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             float* partial = cur.take<float>((size_t)slots * plan.max_layer_params + 4);
             float* tile_loss = cur.take<float>((size_t)loss_tiles(g) + 4);
             int* ticket = cur.take<int>(64);  // work counter of the aggregation kernels (zero between launches)
+            unsigned long long* dense_counts = cur.take<unsigned long long>(3 * RTMA_MAX_PARTS);
+            int* dense_flags = cur.take<int>(RTMA_MAX_PARTS);  // per trainer: aggregated on the tensor cores
             unsigned long long* sym_sums = cur.take<unsigned long long>(4);
             const size_t zero_bytes = cur.used;  // everything above starts from zero: rows between parts stay zero
             int* heavy_list = cur.take<int>((size_t)spmm_order_entries(g) + 4);
+            // entries outside the window of a row's tile, for the parts aggregated on the tensor cores
+            unsigned long long* win_bits = cur.take<unsigned long long>((size_t)rows * (DENSE_WINDOW / 64) + 2);
+            int32_t* left_col = cur.take<int32_t>((size_t)rows * DENSE_LEFT_CAP + 4);
+            unsigned char* left_cnt = cur.take<unsigned char>((size_t)rows + 16);
             float* post_partial = m.post ? cur.take<float>((size_t)post_tiles(g) * (2 * plan.post_width + 1) + 4) : nullptr;
             if (link && m.Kd > 1) dec_post_partial = cur.take<float>((size_t)post_tiles(gd) * (2 * plan.post_width + 1) + 4);
             TcLayerPlan dtcp[RTMA_MAX_LAYERS];
@@ -476,6 +483,37 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
             for (int k = 0; k < g.num; ++k) wave_entries += edge_offsets[g.part[k] + 1] - edge_offsets[g.part[k]];
             SpmmOrder wave_order;
             RTMA_TRY(launch_spmm_order(ctx, g, rowptr_out, col_out, wave_entries, ticket + 16, heavy_list, &wave_order, s));
+            if (ctx->dense_mode != 0 && !m.gcn && tc_available()) {
+                // Which parts take the tensor-core tiles is decided on the device; the host waits for the answer
+                // (the only synchronisation of the call), so that a wave without such parts launches nothing for them.
+                RTMA_TRY(launch_dense_probe(ctx, g, rowptr_out, col_out, ctx->dense_mode, dense_counts, dense_flags, s));
+                int* flags_host = static_cast<int*>(ctx->pinned);
+                bool any_dense = false, all_dense = true;
+                auto read_flags = [&]() -> int32_t {
+                    RTMA_CUDA(ctx, cudaMemcpyAsync(flags_host, dense_flags, sizeof(int) * RTMA_MAX_PARTS, cudaMemcpyDeviceToHost, s));
+                    RTMA_CUDA(ctx, cudaStreamSynchronize(s));
+                    any_dense = false;
+                    all_dense = true;
+                    for (int k = 0; k < g.num; ++k) {
+                        any_dense = any_dense || flags_host[g.part[k]] != 0;
+                        all_dense = all_dense && (flags_host[g.part[k]] != 0 || g.rows[k] == 0);
+                    }
+                    return RTMA_OK;
+                };
+                RTMA_TRY(read_flags());
+                if (any_dense) {  // the per-row masks and lists; a part with repeated entries is taken back: read again
+                    RTMA_TRY(launch_dense_lists(ctx, g, rowptr_out, col_out, dense_flags, win_bits, left_cnt, left_col, s));
+                    RTMA_TRY(read_flags());
+                }
+                wave_order.all_dense = any_dense && all_dense;
+                if (any_dense) {
+                    wave_order.dense = dense_flags;
+                    wave_order.rows_total = rows;
+                    wave_order.left_cnt = left_cnt;
+                    wave_order.left_col = left_col;
+                    wave_order.win_bits = win_bits;
+                }
+            }
             RTMA_TRY(launch_to_planes(ctx, g, Xp, perm, n, m.dims[0], Hl[0], s));
             const Planes no_planes{nullptr, nullptr, 0};
             const Mat no_mat{nullptr, 0};
@@ -492,7 +530,8 @@ int32_t train_impl(rtma_ctx* ctx, const rtma_model_desc* md, int32_t M, const in
                 // trainers reach the aggregation point with different step counts)
                 bool all_run = true;
                 for (int k = 0; k < wave.num; ++k) all_run = all_run && steps[wave.part[k]] > step;
-                const SpmmOrder order = all_run ? wave_order : SpmmOrder{nullptr, nullptr, 0, nullptr};  // built for the whole wave
+                // the order was built for the whole wave; which parts go to the tensor cores is a matter of each part
+                const SpmmOrder order = all_run ? wave_order : SpmmOrder{nullptr, nullptr, 0, nullptr, wave_order.dense, wave_order.rows_total, wave_order.left_cnt, wave_order.left_col, wave_order.win_bits, wave_order.all_dense};
                 SplitPlan spl[RTMA_MAX_LAYERS];
                 if (all_run) {
                     g = wave;

@@ -91,6 +91,14 @@ struct SpmmOrder {
     int64_t heavy;           // entries from which a group is listed
     const unsigned long long* near_total;  // device: probed entries with a nearby column, probed entries;
                                            // mostly nearby -> groups are handed out block by block
+    const int* dense;        // device, per trainer: 1 = the part is aggregated on the tensor cores (spmm_tc.cu);
+                             // NULL: no part is
+    int64_t rows_total;      // scratch rows of the planes (the extent the tensor-core path may address)
+    const unsigned char* left_cnt;  // device, per scratch row of such a part: its entries outside the tile's window
+                                    // (255: more than DENSE_LEFT_CAP), and their columns [row][DENSE_LEFT_CAP]
+    const int32_t* left_col;
+    const unsigned long long* win_bits;  // device, per scratch row of such a part: its window as DENSE_WINDOW bits
+    bool all_dense;          // host: every part of the wave is flagged, the gather kernels have nothing to do
 };
 // list: spmm_order_entries(g) ints; count: 8 ints (16-byte aligned), zero on entry: the number of listed
 // groups, then the two locality counters; entries: kept entries of g's parts.
@@ -107,6 +115,33 @@ int32_t launch_spmm_mean(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowpt
 int32_t launch_spmm_transposed(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
                                const float* inv_deg, Planes src, Planes out, int d, SpmmOrder order, int* ticket,
                                cudaStream_t s);
+
+// ---- spmm_tc.cu (the aggregation of parts with local neighbourhoods, on the tensor cores) ----
+// A tile of DENSE_TILE_ROWS rows takes the entries whose column lies within DENSE_HALO rows before its
+// first or after its last row from a dense product; the others are added afterwards.
+constexpr int DENSE_TILE_ROWS = 128;
+constexpr int DENSE_HALO = 128;
+constexpr int DENSE_WINDOW = DENSE_TILE_ROWS + 2 * DENSE_HALO;
+constexpr int DENSE_LEFT_CAP = 4;  // entries outside the window that are listed per row; rows with more are finished separately
+bool spmm_dense_applies(int d);
+// dense[trainer] for every part of g, from a sample of its rows (every 64th): 1 where at least half of the
+// sampled entries fall into their tile's window and the sampled rows have 4 entries or more on average.
+// mode 2: 1 for every part (launch_dense_lists may still take a part back).  counts: 3 * RTMA_MAX_PARTS 64-bit words of scratch, zero on entry.
+int32_t launch_dense_probe(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                           int mode, unsigned long long* counts, int* dense, cudaStream_t s);
+// Once per call, after launch_dense_probe, for every row of the flagged parts: the window as a bit mask and the
+// entries outside it.  win_bits: DENSE_WINDOW / 64 words per scratch row (16-byte aligned); left_cnt: one byte
+// per scratch row; left_col: DENSE_LEFT_CAP ints per scratch row (16-byte aligned).  Clears the flag of a
+// part in which a row repeats an entry inside its window.
+int32_t launch_dense_lists(rtma_ctx* ctx, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                           int* dense, unsigned long long* win_bits, unsigned char* left_cnt, int32_t* left_col,
+                           cudaStream_t s);
+// The parts of g flagged in order.dense: out = Abar src (transposed: Abar^T src on a symmetric part), window
+// entries by tensor-core tiles, the others summed into the output rows beforehand by a gather pass.  Other
+// parts are left alone.
+int32_t launch_spmm_dense(rtma_ctx* ctx, int kclass, const GroupDesc& g, const int64_t* rowptr_out, const int32_t* col_out,
+                          const float* inv_deg, const SpmmOrder& order, Planes src, Planes out, int d, bool transposed,
+                          cudaStream_t s);
 
 // GCN: scale[row_ws + i] = (local degree + 1)^-1/2, and
 // out[r] = scale[r] * (scale[r] * src[r] + sum_{u in N(r)} scale[u] * src[u])   (symmetric: both passes)

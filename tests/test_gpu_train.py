@@ -374,6 +374,21 @@ def test_whole_path_from_host_buffers(util, tiny_workload):
     assert (kept, cut) == (res["kept"], res["cut"])
     assert util.rel_err(params, res["params"][0]) <= TOL_PARAM
     assert np.abs(losses - res["losses"]).max() <= 1e-4
+    # the same path call by call on device buffers: bit for bit the host-buffer call's result (whose copies
+    # run on a second stream beside the preprocessing), also on a second call that finds its buffers kept
+    c = util.ctx()
+    got = util.gpu_preprocess(w)
+    dev_params = util.dev(np.tile(w.params0, (w.M, 1)))
+    dev_loss = torch.zeros(R, w.M, w.K, dtype=torch.float32, device="cuda")
+    for r in range(R):
+        c.local_steps(w.dims, w.lr, w.M, got["part_host"], got["edge_host"], got["rowptr_out"], got["col_out"],
+                      util.dev(w.X), got["yp"], dev_params, w.K, loss_out=dev_loss[r], perm=got["perm"])
+        c.aggregate(dev_params)
+    torch.cuda.synchronize()
+    assert np.array_equal(dev_params[0].cpu().numpy(), params)
+    assert np.array_equal(dev_loss.cpu().numpy(), losses)
+    again = c.train_host(g.rowptr, g.col, w.X, w.y, w.dims, w.M, w.K, R, w.lr, w.partition_seed, w.params0)
+    assert np.array_equal(again[0], params) and np.array_equal(again[1], losses)
 
 
 def test_bounded_wait_that_runs_out_is_reported_and_leaves_the_context_usable(util, tiny_workload):
