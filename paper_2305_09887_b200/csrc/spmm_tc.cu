@@ -44,11 +44,23 @@ constexpr int DT_KB = DENSE_WINDOW / DT_BK;
 constexpr int DT_A_BYTES = DT_BM * 128;          // one plane of A for one stage: 16 KB
 constexpr int DT_ATOM_BYTES = DT_BK * 128;       // 64 source rows x 64 columns of one plane: 8 KB
 constexpr int DT_STAGING_BYTES = 4096;           // per epilogue warp
-constexpr int DT_MAX_STAGES = 4;
+constexpr int DT_MAX_STAGES = 6;
+constexpr int DT_TILE_ATOMS = 4;                 // 64-column atoms of a column tile
 constexpr int DT_LCAP = DENSE_LEFT_CAP;          // listed entries outside the window, per row
 constexpr unsigned char DT_OVERFLOW = 255;       // left_cnt of a row with more than that
-constexpr int DT_SMEM_MAX = 226 * 1024;
+constexpr int DT_SMEM_MAX = 225 * 1024;           // with the static part (under 2 KB) within the 227 KB a block may have
 static_assert(DT_BM == 128 && DENSE_WINDOW % DT_BK == 0 && DT_HALO % DT_BK == 0, "tile shape of the MMA and whole stages");
+
+// byte of a window mask -> the four 32-bit words of the 16-byte chunk it stands for, sixteen ones per set bit
+struct MaskLut {
+    uint32_t w[256][4];
+    constexpr MaskLut() : w{} {
+        for (int b = 0; b < 256; ++b)
+            for (int p = 0; p < 4; ++p)
+                w[b][p] = (((b >> (2 * p)) & 1) ? 0x0000FFFFu : 0u) | (((b >> (2 * p + 1)) & 1) ? 0xFFFF0000u : 0u);
+    }
+};
+__device__ const MaskLut mask_lut{};
 
 struct DenseArgs {
     GroupDesc g;
@@ -61,7 +73,7 @@ struct DenseArgs {
     Planes out;
     int width;                     // columns of the planes that hold data (a multiple of 8)
     int n_atoms;                   // 64-column atoms over the width
-    int col_tiles;                 // column tiles of at most 4 atoms
+    int col_tiles;                 // column tiles of at most DT_TILE_ATOMS atoms
     int tmem_cols, stages;
     int64_t row_tiles;
     int* error_word;
@@ -72,6 +84,7 @@ struct DenseBarriers {
     uint64_t empty[DT_MAX_STAGES];  // the MMAs have read the stage
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
+    uint64_t builders;              // meeting point of the builder threads (transposed pass)
     uint32_t tmem_base;
     int abort;
 };
@@ -89,6 +102,21 @@ __device__ __forceinline__ bool dense_wait(uint64_t* bar, uint32_t parity, Dense
 // Adds to the bytes the barrier's current phase waits for, without arriving.
 __device__ __forceinline__ void expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(tc::smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+// 32 lanes x 16 consecutive 32-bit columns of tensor memory: thread i of the warp receives lane (base lane + i).
+__device__ __forceinline__ void tmem_load_32x16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // the stages of a tile: window blocks that overlap the part's rows
@@ -114,13 +142,12 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
     constexpr uint32_t NPA = TRANSPOSED ? 2u : 1u;  // planes of A
     const int n_ct = a.col_tiles;
     const int64_t total_tiles = a.row_tiles * n_ct;
-    const int NA_full = min(4, a.n_atoms);
-    const uint32_t b_plane_bytes = (uint32_t)NA_full * DT_ATOM_BYTES;
-    const uint32_t stage_bytes = NPA * DT_A_BYTES + 2u * b_plane_bytes;
+    // a stage: the plane(s) of A, then the tile's atoms of the hi plane of the source rows and, right behind
+    // them, those of the lo plane: one N-major operand of twice the tile's width
+    const uint32_t stage_bytes = NPA * DT_A_BYTES + 2u * (uint32_t)min(DT_TILE_ATOMS, a.n_atoms) * DT_ATOM_BYTES;
     auto a_hi = [&](int s) { return smem + (size_t)s * stage_bytes; };
     auto a_lo = [&](int s) { return smem + (size_t)s * stage_bytes + DT_A_BYTES; };
     auto b_hi = [&](int s) { return smem + (size_t)s * stage_bytes + NPA * DT_A_BYTES; };
-    auto b_lo = [&](int s) { return smem + (size_t)s * stage_bytes + NPA * DT_A_BYTES + b_plane_bytes; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -131,6 +158,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
             tc::mbar_init(&pb.acc_full[b], 1);
             tc::mbar_init(&pb.acc_empty[b], DT_EPI_THREADS);
         }
+        tc::mbar_init(&pb.builders, DT_BUILDERS);
         pb.abort = 0;
         tc::fence_barrier_init();
         tc::prefetch_tensormap(&a.mapSh);
@@ -156,8 +184,14 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
                 if (!locate_tile(a.g, DT_BM, tile / n_ct, &k, &r0)) break;
                 if (!a.dense[a.g.part[k]]) continue;
                 const int ct = (int)(tile % n_ct);
-                const int NA = min(4, a.n_atoms - 4 * ct);
-                const uint32_t idesc = tc::idesc_bf16(DT_BM, 64 * NA, false, true);
+                const int NA = min(DT_TILE_ATOMS, a.n_atoms - DT_TILE_ATOMS * ct);
+                // A tile of at most two atoms multiplies A with [hi | lo] (the lo atoms lie right behind the hi atoms)
+                // in ONE MMA of twice the tile's width: columns [0, 64 NA) of the accumulator take the product with the
+                // hi plane, [64 NA, 128 NA) that with the lo plane, and the epilogue adds the halves.  An MMA that
+                // narrow costs its issue, not its arithmetic.  Wider tiles take one MMA per plane into the same columns.
+                const bool joined = NA <= 2;
+                const uint32_t idesc_both = tc::idesc_bf16(DT_BM, 128 * NA, false, true);
+                const uint32_t idesc_hi = tc::idesc_bf16(DT_BM, 64 * NA, false, true);
                 int kb_first, kb_end;
                 tile_blocks(r0, a.g.rows[k], &kb_first, &kb_end);
                 const int buf = (int)(t & 1);
@@ -170,24 +204,24 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
                     ok = dense_wait(&pb.full[s], (uint32_t)((it / stages) & 1), &pb, a.error_word);
                     if (!ok) break;
                     tc::tc_fence_after_sync();
-                    const uint32_t ah = tc::smem_u32(a_hi(s)), al = tc::smem_u32(a_lo(s));
-                    const uint32_t bh = tc::smem_u32(b_hi(s)), bl = tc::smem_u32(b_lo(s));
+                    const uint32_t ah = tc::smem_u32(a_hi(s)), al = tc::smem_u32(a_lo(s)), bh = tc::smem_u32(b_hi(s));
 #pragma unroll
                     for (int ks = 0; ks < DT_BK / 16; ++ks) {
                         // A is K-major (a 128-byte row holds the 64 window rows of the stage): 16 of them = 32 bytes;
                         // the source rows are N-major (a 128-byte row per window row): 16 of them = 2048 bytes
                         const uint64_t dah = tc::smem_desc_sw128(ah + ks * 32, 16, 1024);
-                        const uint64_t dbh = tc::smem_desc_sw128(bh + ks * 2048, DT_ATOM_BYTES, 1024);
-                        const uint64_t dbl = tc::smem_desc_sw128(bl + ks * 2048, DT_ATOM_BYTES, 1024);
+                        const uint64_t db = tc::smem_desc_sw128(bh + ks * 2048, DT_ATOM_BYTES, 1024);
+                        const uint64_t dbl = tc::smem_desc_sw128(bh + NA * DT_ATOM_BYTES + ks * 2048, DT_ATOM_BYTES, 1024);
                         const uint32_t first = (kb > kb_first || ks > 0) ? 1u : 0u;
-                        if (TRANSPOSED) {
-                            const uint64_t dal = tc::smem_desc_sw128(al + ks * 32, 16, 1024);
-                            tc::mma_bf16(d_tmem, dal, dbh, idesc, first);
-                            tc::mma_bf16(d_tmem, dah, dbl, idesc, 1u);
-                            tc::mma_bf16(d_tmem, dah, dbh, idesc, 1u);
+                        if (joined) {
+                            tc::mma_bf16(d_tmem, dah, db, idesc_both, first);
                         } else {
-                            tc::mma_bf16(d_tmem, dah, dbl, idesc, first);
-                            tc::mma_bf16(d_tmem, dah, dbh, idesc, 1u);
+                            tc::mma_bf16(d_tmem, dah, dbl, idesc_hi, first);
+                            tc::mma_bf16(d_tmem, dah, db, idesc_hi, 1u);
+                        }
+                        if (TRANSPOSED) {  // + A_lo * hi (into the first half)
+                            const uint64_t dal = tc::smem_desc_sw128(al + ks * 32, 16, 1024);
+                            tc::mma_bf16(d_tmem, dal, db, idesc_hi, 1u);
                         }
                     }
                     tc::mma_commit(&pb.empty[s]);
@@ -199,10 +233,16 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
     } else if (warp < 1 + DT_BUILDERS / 32) {
         const int r = threadIdx.x - 32;  // the tile row this thread writes
         const uint32_t swz = (uint32_t)(r & 7);
-        // transposed pass: the split weights of the stage's 64 window rows, as the 32 words of a row of A
-        // with every bit set; two buffers, one barrier per stage
-        __shared__ __align__(16) uint32_t wpair[2][2][DT_BK / 2];
+        // transposed pass: the split weights 1 / deg of the tile's window rows, stage by stage as the 32 words
+        // of a row of A with every bit set; written once per tile between two barriers of the builder warps
+        __shared__ __align__(16) uint32_t wpair[DT_KB][2][DT_BK / 2];
         int64_t it = 0;
+        uint32_t meetings = 0;
+        // all builder threads meet (a bounded wait like every other: a thread that has given up is not waited for)
+        auto meet = [&]() {
+            tc::mbar_arrive(&pb.builders);
+            return dense_wait(&pb.builders, meetings++ & 1u, &pb, a.error_word);
+        };
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             int k, r0;
@@ -210,7 +250,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
             if (!a.dense[a.g.part[k]]) continue;
             const int n_p = a.g.rows[k];
             const int ct = (int)(tile % n_ct);
-            const int NA = min(4, a.n_atoms - 4 * ct);
+            const int NA = min(DT_TILE_ATOMS, a.n_atoms - DT_TILE_ATOMS * ct);
             int kb_first, kb_end;
             tile_blocks(r0, n_p, &kb_first, &kb_end);
             const int64_t ws = a.g.row_ws[k];
@@ -227,33 +267,24 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
 #pragma unroll
                 for (int q = 0; q < DT_KB; ++q) bits[q] = 0ULL;
             }
-            // 1 / deg of the window rows r, 128 + r, 256 + r: stage kb needs rows 64 kb .. 64 kb + 63
-            float wq[DENSE_WINDOW / DT_BUILDERS];
             if (TRANSPOSED) {
+                ok = meet();  // every thread has written the previous tile's last stage
+                if (!ok) break;
 #pragma unroll
                 for (int q = 0; q < DENSE_WINDOW / DT_BUILDERS; ++q) {
-                    const int u = r0 - DT_HALO + q * DT_BUILDERS + r;
-                    wq[q] = (u >= 0 && u < n_p) ? __ldg(a.inv_deg + ws + u) : 0.f;
+                    const int wr = q * DT_BUILDERS + r;  // window row
+                    const int u = r0 - DT_HALO + wr;
+                    uint32_t h = 0, l = 0;
+                    if (u >= 0 && u < n_p) split_bits(__ldg(a.inv_deg + ws + u), h, l);
+                    reinterpret_cast<unsigned short*>(wpair[wr / DT_BK][0])[wr % DT_BK] = (unsigned short)h;
+                    reinterpret_cast<unsigned short*>(wpair[wr / DT_BK][1])[wr % DT_BK] = (unsigned short)l;
                 }
+                ok = meet();
+                if (!ok) break;
             }
             for (int kb = kb_first; kb < kb_end; ++kb, ++it) {
                 const int s = (int)(it % stages);
                 ok = dense_wait(&pb.empty[s], (uint32_t)((it / stages) & 1) ^ 1u, &pb, a.error_word);
-                const int wbuf = (int)(it & 1);
-                if (TRANSPOSED) {
-                    if ((r >> 6) == (kb & 1)) {
-                        float w = wq[0];
-#pragma unroll
-                        for (int q = 1; q < DENSE_WINDOW / DT_BUILDERS; ++q) w = (kb >> 1) == q ? wq[q] : w;
-                        uint32_t h, l;
-                        split_bits(w, h, l);
-                        reinterpret_cast<unsigned short*>(wpair[wbuf][0])[r & 63] = (unsigned short)h;
-                        reinterpret_cast<unsigned short*>(wpair[wbuf][1])[r & 63] = (unsigned short)l;
-                    }
-                    // every builder thread arrives, whatever its wait said: they agree on the outcome afterwards
-                    asm volatile("bar.sync 2, %0;" ::"n"(DT_BUILDERS) : "memory");
-                    ok = ok && *reinterpret_cast<volatile int*>(&pb.abort) == 0;
-                }
                 if (!ok) break;
                 if (r == 0) {
                     // the stage's source rows, requested before this thread writes its row of A: window rows
@@ -261,8 +292,8 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
                     expect_tx(&pb.full[s], 2u * (uint32_t)NA * DT_ATOM_BYTES);
                     const int y = (int)(ws + r0 - DT_HALO + (int64_t)kb * DT_BK);  // scratch row; may be negative: reads zeros
                     for (int t = 0; t < NA; ++t) {
-                        tc::tma_load_2d(b_hi(s) + t * DT_ATOM_BYTES, &a.mapSh, &pb.full[s], (4 * ct + t) * 64, y);
-                        tc::tma_load_2d(b_lo(s) + t * DT_ATOM_BYTES, &a.mapSl, &pb.full[s], (4 * ct + t) * 64, y);
+                        tc::tma_load_2d(b_hi(s) + t * DT_ATOM_BYTES, &a.mapSh, &pb.full[s], (DT_TILE_ATOMS * ct + t) * 64, y);
+                        tc::tma_load_2d(b_hi(s) + (NA + t) * DT_ATOM_BYTES, &a.mapSl, &pb.full[s], (DT_TILE_ATOMS * ct + t) * 64, y);
                     }
                 }
                 unsigned long long m = bits[0];
@@ -272,19 +303,31 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
                 uint8_t* row_hi = a_hi(s) + r * 128;
                 uint8_t* row_lo = a_lo(s) + r * 128;
 #pragma unroll
-                for (uint32_t c = 0; c < 8; ++c) {
-                    const uint32_t b = (uint32_t)(m >> (8 * c)) & 0xFFu;
-                    uint32_t mk[4];  // 16 ones for every set bit
+                for (uint32_t c4 = 0; c4 < 8; c4 += 4) {  // four chunks at a time: all their loads, then all their stores
+                    uint4 mk[4];  // sixteen ones for every set bit
 #pragma unroll
-                    for (int p = 0; p < 4; ++p) mk[p] = ((b >> (2 * p)) & 1u ? 0x0000FFFFu : 0u) | ((b >> (2 * p + 1)) & 1u ? 0xFFFF0000u : 0u);
+                    for (uint32_t c = 0; c < 4; ++c)
+                        mk[c] = __ldg(reinterpret_cast<const uint4*>(mask_lut.w[(uint32_t)(m >> (8 * (c4 + c))) & 0xFFu]));
                     if (TRANSPOSED) {
-                        const uint4 wh = *reinterpret_cast<const uint4*>(&wpair[wbuf][0][4 * c]);
-                        const uint4 wl = *reinterpret_cast<const uint4*>(&wpair[wbuf][1][4 * c]);
-                        *reinterpret_cast<uint4*>(row_hi + ((c ^ swz) << 4)) = make_uint4(mk[0] & wh.x, mk[1] & wh.y, mk[2] & wh.z, mk[3] & wh.w);
-                        *reinterpret_cast<uint4*>(row_lo + ((c ^ swz) << 4)) = make_uint4(mk[0] & wl.x, mk[1] & wl.y, mk[2] & wl.z, mk[3] & wl.w);
+                        uint4 wh[4], wl[4];
+#pragma unroll
+                        for (uint32_t c = 0; c < 4; ++c) {
+                            wh[c] = *reinterpret_cast<const uint4*>(&wpair[kb][0][4 * (c4 + c)]);
+                            wl[c] = *reinterpret_cast<const uint4*>(&wpair[kb][1][4 * (c4 + c)]);
+                        }
+#pragma unroll
+                        for (uint32_t c = 0; c < 4; ++c) {
+                            *reinterpret_cast<uint4*>(row_hi + (((c4 + c) ^ swz) << 4)) =
+                                make_uint4(mk[c].x & wh[c].x, mk[c].y & wh[c].y, mk[c].z & wh[c].z, mk[c].w & wh[c].w);
+                            *reinterpret_cast<uint4*>(row_lo + (((c4 + c) ^ swz) << 4)) =
+                                make_uint4(mk[c].x & wl[c].x, mk[c].y & wl[c].y, mk[c].z & wl[c].z, mk[c].w & wl[c].w);
+                        }
                     } else {
                         constexpr uint32_t ONES = 0x3F803F80u;  // 1.0 | 1.0
-                        *reinterpret_cast<uint4*>(row_hi + ((c ^ swz) << 4)) = make_uint4(mk[0] & ONES, mk[1] & ONES, mk[2] & ONES, mk[3] & ONES);
+#pragma unroll
+                        for (uint32_t c = 0; c < 4; ++c)
+                            *reinterpret_cast<uint4*>(row_hi + (((c4 + c) ^ swz) << 4)) =
+                                make_uint4(mk[c].x & ONES, mk[c].y & ONES, mk[c].z & ONES, mk[c].w & ONES);
                     }
                 }
                 tc::fence_proxy_async_smem();  // the tensor core reads what this thread has just written
@@ -296,77 +339,124 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
         const int q = warp & 3;                        // the quarter of the tensor memory's lanes this warp may read
         const int col_phase = ew >> 2;                 // which of the quarter's two warps: even or odd 32-column chunks
         uint8_t* stg = smem + (size_t)stages * stage_bytes + (size_t)ew * DT_STAGING_BYTES;
-        int64_t t = 0;
-        bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            int k, r0;
-            if (!locate_tile(a.g, DT_BM, tile / n_ct, &k, &r0)) break;
-            if (!a.dense[a.g.part[k]]) continue;
-            const int ct = (int)(tile % n_ct);
-            const int BN = 64 * min(4, a.n_atoms - 4 * ct);
-            const int n0 = ct * 256;
-            const int buf = (int)(t & 1);
-            ok = dense_wait(&pb.acc_full[buf], (uint32_t)((t >> 1) & 1), &pb, a.error_word);
-            if (!ok) break;
-            tc::tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.tmem_cols);
+        float4* st = reinterpret_cast<float4*>(stg);
+        const int p = lane & 3;
+        const uint32_t out_row_bytes = (uint32_t)a.out.ld * 2u;
+        // this block's next tile at or after `from`
+        auto next_tile = [&](int64_t from, int* k, int* r0) -> int64_t {
+            for (int64_t tile = from; tile < total_tiles; tile += gridDim.x) {
+                if (!locate_tile(a.g, DT_BM, tile / n_ct, k, r0)) return -1;
+                if (a.dense[a.g.part[*k]]) return tile;
+            }
+            return -1;
+        };
+        // of the thread's four rows of a tile: the scale, and whether the output row already holds a sum to add to
+        auto row_info = [&](int k, int r0, float (&scale)[4], bool (&has_left)[4]) {
             const int rows_here = min(32, a.g.rows[k] - (r0 + q * 32));
             const int64_t orow0 = a.g.row_ws[k] + r0 + q * 32;
-            const int64_t ws = a.g.row_ws[k];
-            // of the thread's four rows: the scale, and whether the output row already holds a sum to add to
-            float scale[4] = {1.f, 1.f, 1.f, 1.f};
-            bool has_left[4] = {false, false, false, false};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int row = j * 8 + (lane >> 2);
+                scale[j] = 1.f;
+                has_left[j] = false;
                 if (row < rows_here) {
                     if (!TRANSPOSED) scale[j] = __ldg(a.inv_deg + orow0 + row);
                     has_left[j] = a.left_cnt[orow0 + row] != 0;
                 }
             }
-            for (int c0 = col_phase * 32; c0 < BN; c0 += 64) {
-                float v[32];
-                tc::tmem_load_32x32(d_tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-                if (rows_here <= 0) continue;
-                // through the warp's staging slab (16-byte chunk j of row r at chunk j ^ (r % 8)), so that a
-                // thread then owns 8 consecutive columns and a store writes whole 64-byte pieces of rows
-                float4* st = reinterpret_cast<float4*>(stg);
-                __syncwarp();
+        };
+        int k = 0, r0 = 0;
+        int64_t tile = next_tile(blockIdx.x, &k, &r0);
+        float next_scale[4];
+        bool next_left[4];
+        if (tile >= 0) row_info(k, r0, next_scale, next_left);
+        int64_t t = 0;
+        bool ok = true;
+        while (tile >= 0 && ok) {
+            float scale[4];
+            bool has_left[4];
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    st[lane * 8 + (j ^ (lane & 7))] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                __syncwarp();
-                const int p = lane & 3;
+            for (int j = 0; j < 4; ++j) {
+                scale[j] = next_scale[j];
+                has_left[j] = next_left[j];
+            }
+            const int ct = (int)(tile % n_ct);
+            const int BN = 64 * min(DT_TILE_ATOMS, a.n_atoms - DT_TILE_ATOMS * ct);
+            const int n0 = ct * 64 * DT_TILE_ATOMS;
+            const int rows_here = min(32, a.g.rows[k] - (r0 + q * 32));
+            const int64_t orow0 = a.g.row_ws[k] + r0 + q * 32;
+            // the next tile's row data is requested a tile ahead, and every chunk's existing rows before the chunk
+            // before them is finished: the epilogue is the longest chain of the kernel, and these loads its latency
+            tile = next_tile(tile + gridDim.x, &k, &r0);
+            if (tile >= 0) row_info(k, r0, next_scale, next_left);
+            uint4 gh[4], gl[4];
+            auto request = [&](int c0) {  // what the rows already hold (written by the launch before this one)
                 const int n = n0 + c0 + 8 * p;
-                const bool col_ok = n < a.width;
-                const uint32_t out_row_bytes = (uint32_t)a.out.ld * 2u;
-                char* oh = reinterpret_cast<char*>(a.out.hi + (orow0 + (lane >> 2)) * a.out.ld + n);
-                char* ol = reinterpret_cast<char*>(a.out.lo + (orow0 + (lane >> 2)) * a.out.ld + n);
-                // what the rows already hold (written by the launch before this one), requested together
-                uint4 gh[4], gl[4];
+                if (c0 >= BN || n >= a.width) return;
+                const char* oh = reinterpret_cast<const char*>(a.out.hi + (orow0 + (lane >> 2)) * a.out.ld + n);
+                const char* ol = reinterpret_cast<const char*>(a.out.lo + (orow0 + (lane >> 2)) * a.out.ld + n);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    if (has_left[j] && col_ok) {
+                    if (has_left[j]) {
                         gh[j] = __ldcg(reinterpret_cast<const uint4*>(oh + (size_t)(j * 8) * out_row_bytes));
                         gl[j] = __ldcg(reinterpret_cast<const uint4*>(ol + (size_t)(j * 8) * out_row_bytes));
                     }
                 }
+            };
+            request(col_phase * 32);
+            const int buf = (int)(t & 1);
+            ok = dense_wait(&pb.acc_full[buf], (uint32_t)((t >> 1) & 1), &pb, a.error_word);
+            if (!ok) break;
+            tc::tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.tmem_cols);
+            for (int c0 = col_phase * 32; c0 < BN && rows_here > 0; c0 += 64) {
+                // Of a tile of at most two atoms the accumulator holds the product with the hi plane and, BN columns
+                // further, that with the lo plane.  The sum goes through the warp's staging slab (16-byte chunk j of row r at chunk
+                // j ^ (r % 8)), so that a thread then owns 8 consecutive columns and a store writes whole 64-byte
+                // pieces of rows.
+                __syncwarp();
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {  // 16 accumulator columns at a time: few registers
+                    float v[16];
+                    tmem_load_32x16(d_tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c0 + 16 * half), v);
+                    if (BN <= 128) {  // the tile's planes were multiplied side by side
+                        float v2[16];
+                        tmem_load_32x16(d_tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(BN + c0 + 16 * half), v2);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) v[e] += v2[e];
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int jj = 4 * half + j;
+                        st[lane * 8 + (jj ^ (lane & 7))] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    }
+                }
+                __syncwarp();
+                const int n = n0 + c0 + 8 * p;
+                const bool col_ok = n < a.width;
+                char* oh = reinterpret_cast<char*>(a.out.hi + (orow0 + (lane >> 2)) * a.out.ld + n);
+                char* ol = reinterpret_cast<char*>(a.out.lo + (orow0 + (lane >> 2)) * a.out.ld + n);
+                Pack8 x[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int row = j * 8 + (lane >> 2);
                     const float4 x0 = st[row * 8 + ((2 * p) ^ (row & 7))];
                     const float4 x1 = st[row * 8 + ((2 * p + 1) ^ (row & 7))];
+                    x[j].v[0] = x0.x; x[j].v[1] = x0.y; x[j].v[2] = x0.z; x[j].v[3] = x0.w;
+                    x[j].v[4] = x1.x; x[j].v[5] = x1.y; x[j].v[6] = x1.z; x[j].v[7] = x1.w;
+                    if (has_left[j] && col_ok) x[j].add_planes_mixed(gh[j], gl[j]);
+                }
+                request(c0 + 64);  // the registers are free again
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int row = j * 8 + (lane >> 2);
                     if (row < rows_here && col_ok) {
-                        Pack8 x;
-                        x.v[0] = x0.x; x.v[1] = x0.y; x.v[2] = x0.z; x.v[3] = x0.w;
-                        x.v[4] = x1.x; x.v[5] = x1.y; x.v[6] = x1.z; x.v[7] = x1.w;
-                        if (has_left[j]) x.add_planes_mixed(gh[j], gl[j]);
                         if (!TRANSPOSED) {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) x.v[e] *= scale[j];
+                            for (int e = 0; e < 8; ++e) x[j].v[e] *= scale[j];
                         }
                         uint4 h, l;
-                        x.to_planes_lean(h, l);
+                        x[j].to_planes_lean(h, l);
                         *reinterpret_cast<uint4*>(oh + (size_t)(j * 8) * out_row_bytes) = h;
                         *reinterpret_cast<uint4*>(ol + (size_t)(j * 8) * out_row_bytes) = l;
                     }
@@ -671,10 +761,10 @@ int32_t launch_spmm_dense(rtma_ctx* ctx, int kclass, const GroupDesc& g, const i
     a.out = out;
     a.width = (int)planes_ld(d);
     a.n_atoms = (int)ceil_div(a.width, 64);
-    a.col_tiles = (int)ceil_div(a.n_atoms, 4);
-    const int tile_atoms = std::min(4, a.n_atoms);
-    uint32_t tmem = 32;
-    while ((int)tmem < 64 * tile_atoms) tmem <<= 1;
+    a.col_tiles = (int)ceil_div(a.n_atoms, DT_TILE_ATOMS);
+    const int tile_atoms = std::min(DT_TILE_ATOMS, a.n_atoms);
+    uint32_t tmem = 32;  // columns of one accumulator: twice the tile's width where the two planes' products lie side by side
+    while ((int)tmem < (tile_atoms <= 2 ? 128 : 64) * tile_atoms) tmem <<= 1;
     a.tmem_cols = (int)tmem;
     const size_t stage_bytes = (transposed ? 2 : 1) * (size_t)DT_A_BYTES + 2 * (size_t)tile_atoms * DT_ATOM_BYTES;
     const size_t fixed = 1024 + 8 * (size_t)DT_STAGING_BYTES;
