@@ -548,6 +548,8 @@ def main():
     ap.add_argument("--encoder", default="sage", choices=["sage", "gcn"])
     ap.add_argument("--act", default="relu", choices=["relu", "prelu"])
     ap.add_argument("--norm", default="none", choices=["none", "layernorm"])
+    ap.add_argument("--aggregation", default="auto", choices=["auto", "gather", "tiles"],
+                    help="mean aggregation: per part by itself (default), always by gathering, or tensor-core tiles for every part")
     ap.add_argument("--streams", type=int, default=1,
                     help="CUDA streams the trainers are spread over (trainers sharing a stream are batched)")
     args = ap.parse_args()
@@ -583,6 +585,7 @@ def main():
     g = w.graph
     L = len(w.dims) - 1
     ctx = binding.Context(local_rank)
+    ctx.set_dense_aggregation({"auto": 1, "gather": 0, "tiles": 2}[args.aggregation])
     resident = dict(rowptr=torch.from_numpy(g.rowptr).to(device), col=torch.from_numpy(g.col).to(device),
                     X=torch.from_numpy(w.X).to(device), y=torch.from_numpy(w.y).to(device),
                     gid=torch.from_numpy(g.group_id).to(device) if w.use_groups else None)
@@ -783,6 +786,7 @@ def main():
                    "kept_fraction": kept / g.num_entries,
                    "parallelism": ("replicas only" if world > 1 else
                                    f"single GPU, {w.M} trainers batched on {n_streams} stream(s)"),
+                   "aggregation": args.aggregation,
                    "l2": "256 MB written between timed steps"},
         "trainer_steps_per_s": world * args.steps * trainer_steps / elapsed_s,
         "edges_gathered_per_s": world * args.steps * kept * ((passes - 1) * w.K + 1) * w.R / elapsed_s,

@@ -475,17 +475,22 @@ __global__ void __launch_bounds__(DT_THREADS, 1) spmm_dense_kernel(const __grid_
 // The entries outside the window of their row's tile, before the tiles run: for every row that has any,
 // out[row] = their sum (transposed pass: weighted by 1 / deg of the column), unscaled; the tile's epilogue adds
 // its product and the scale.  A warp takes 32 consecutive rows: their counts and listed columns with one load
-// each, then the rows that have entries two at a time, all of the two rows' source rows requested together
-// (lanes split the width in pieces of 8 values).  A row with more than DT_LCAP such entries is looked up in
-// the part's CSR again, 32 entries at a time.
-template <bool TRANSPOSED>
+// each; then the rows that have entries, several at a time, two source rows of each requested together (most
+// rows have one or two).  LPR lanes own a row (pieces of 8 values per lane): 32 for rows wider than 64 values,
+// two rows at a time per warp; 8 for narrower rows, eight at a time, two per quarter of the warp.  A row with more than DT_LCAP such entries is looked
+// up in the part's CSR again, 32 entries at a time, by the whole warp.
+template <bool TRANSPOSED, int LPR>
 __global__ void __launch_bounds__(256, 2)
 spmm_outside_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restrict__ rowptr_out,
                     const int32_t* __restrict__ col_out, const float* __restrict__ inv_deg,
                     const int* __restrict__ dense, const unsigned char* __restrict__ left_cnt,
                     const int32_t* __restrict__ left_col, const Planes src, const Planes out, const int width,
                     const int64_t total_groups) {
+    constexpr int S = 32 / LPR;            // rows side by side in a warp
+    constexpr int NR = 2;                  // rows a lane works on at a time
+    constexpr int EL = 2;                  // listed entries of each of them requested together (most rows have one or two)
     const int lane = threadIdx.x & 31;
+    const int sub = lane / LPR, sl = lane % LPR;
     const int64_t warps = (int64_t)gridDim.x * 8;
     for (int64_t grp = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); grp < total_groups; grp += warps) {
         int k, i0;
@@ -496,67 +501,84 @@ spmm_outside_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restri
         const int my_cnt = i0 + lane < n_p ? (int)left_cnt[ws + i0 + lane] : 0;
         int4 my_cols = make_int4(0, 0, 0, 0);
         if (my_cnt > 0 && my_cnt <= DT_LCAP) my_cols = *reinterpret_cast<const int4*>(left_col + (ws + i0 + lane) * DT_LCAP);
-        unsigned listed = __ballot_sync(0xffffffffu, my_cnt > 0 && my_cnt <= DT_LCAP);
-        unsigned many = __ballot_sync(0xffffffffu, my_cnt == DT_OVERFLOW);
+        const unsigned listed = __ballot_sync(0xffffffffu, my_cnt > 0 && my_cnt <= DT_LCAP);
+        const unsigned many = __ballot_sync(0xffffffffu, my_cnt == DT_OVERFLOW);
         if (!(listed | many)) continue;
         const __nv_bfloat16* sh = src.hi + ws * src.ld;
-        const __nv_bfloat16* sl = src.lo + ws * src.ld;
-        for (int cb = 0; cb < width; cb += 256) {  // the same trip count for every lane: the shuffles below need the whole warp
-            const int c0 = cb + lane * 8;
+        const __nv_bfloat16* sl_ = src.lo + ws * src.ld;
+        for (int cb = 0; cb < width; cb += LPR * 8) {  // the same trip count for every lane: the shuffles below need the whole warp
+            const int c0 = cb + sl * 8;
             const bool live = c0 < width;
             const int cx = live ? c0 : 0;  // lanes past the width read column 0 and store nothing
             for (unsigned rest = listed; rest;) {
-                // two rows at a time
-                int row[2], cnt[2];
-                int4 cols[2];
+                int row[NR], cnt[NR];
+                int4 cols[NR];
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    const int owner = rest ? __ffs(rest) - 1 : 0;
-                    const bool have = rest != 0u;
-                    rest &= rest - 1;
-                    row[t] = i0 + owner;
-                    cnt[t] = __shfl_sync(0xffffffffu, my_cnt, owner);
-                    cols[t].x = __shfl_sync(0xffffffffu, my_cols.x, owner);
-                    cols[t].y = __shfl_sync(0xffffffffu, my_cols.y, owner);
-                    cols[t].z = __shfl_sync(0xffffffffu, my_cols.z, owner);
-                    cols[t].w = __shfl_sync(0xffffffffu, my_cols.w, owner);
+                for (int t = 0; t < NR; ++t) {
+                    // the (t * S + sub)-th row still to do
+                    const unsigned owner = __fns(rest, 0, t * S + sub + 1);
+                    const bool have = owner < 32u;
+                    const int from = have ? (int)owner : 0;
+                    row[t] = i0 + from;
+                    cnt[t] = __shfl_sync(0xffffffffu, my_cnt, from);
+                    cols[t].x = __shfl_sync(0xffffffffu, my_cols.x, from);
+                    cols[t].y = __shfl_sync(0xffffffffu, my_cols.y, from);
+                    cols[t].z = __shfl_sync(0xffffffffu, my_cols.z, from);
+                    cols[t].w = __shfl_sync(0xffffffffu, my_cols.w, from);
                     if (!have) cnt[t] = 0;
                 }
-                uint4 xh[2][DT_LCAP], xl[2][DT_LCAP];
-                float wt[2][DT_LCAP];
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    const int us[DT_LCAP] = {cols[t].x, cols[t].y, cols[t].z, cols[t].w};
+                for (int t = 0; t < S * NR; ++t) rest &= rest - 1;
+                Pack8 acc[NR];
 #pragma unroll
-                    for (int l = 0; l < DT_LCAP; ++l) {
-                        if (l < cnt[t]) {
-                            xh[t][l] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)us[l] * src.ld + cx));
-                            xl[t][l] = __ldg(reinterpret_cast<const uint4*>(sl + (int64_t)us[l] * src.ld + cx));
-                            if (TRANSPOSED) wt[t][l] = __ldg(inv_deg + ws + us[l]);
+                for (int t = 0; t < NR; ++t) acc[t].zero();
+                bool more = true;
+#pragma unroll
+                for (int l0 = 0; l0 < DT_LCAP; l0 += EL) {
+                    if (l0 > 0) {  // a further round only where some row of the warp has that many entries
+                        bool mine = false;
+#pragma unroll
+                        for (int t = 0; t < NR; ++t) mine = mine || cnt[t] > l0;
+                        more = __any_sync(0xffffffffu, mine);
+                    }
+                    if (!more) break;
+                    uint4 xh[NR][EL], xl[NR][EL];
+                    float wt[NR][EL];
+#pragma unroll
+                    for (int t = 0; t < NR; ++t) {
+                        const int us[DT_LCAP] = {cols[t].x, cols[t].y, cols[t].z, cols[t].w};
+#pragma unroll
+                        for (int l = 0; l < EL; ++l) {
+                            if (l0 + l < cnt[t]) {
+                                xh[t][l] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)us[l0 + l] * src.ld + cx));
+                                xl[t][l] = __ldg(reinterpret_cast<const uint4*>(sl_ + (int64_t)us[l0 + l] * src.ld + cx));
+                                if (TRANSPOSED) wt[t][l] = __ldg(inv_deg + ws + us[l0 + l]);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int t = 0; t < NR; ++t) {
+#pragma unroll
+                        for (int l = 0; l < EL; ++l) {
+                            if (l0 + l < cnt[t]) {
+                                if (TRANSPOSED) acc[t].fma_planes_mixed(wt[t][l], xh[t][l], xl[t][l]);
+                                else acc[t].add_planes_mixed(xh[t][l], xl[t][l]);
+                            }
                         }
                     }
                 }
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (cnt[t] == 0) continue;
-                    Pack8 acc;
-                    acc.zero();
-#pragma unroll
-                    for (int l = 0; l < DT_LCAP; ++l) {
-                        if (l < cnt[t]) {
-                            if (TRANSPOSED) acc.fma_planes_mixed(wt[t][l], xh[t][l], xl[t][l]);
-                            else acc.add_planes_mixed(xh[t][l], xl[t][l]);
-                        }
-                    }
-                    if (live) {
+                for (int t = 0; t < NR; ++t) {
+                    if (cnt[t] > 0 && live) {
                         uint4 h, l;
-                        acc.to_planes_lean(h, l);
+                        acc[t].to_planes_lean(h, l);
                         *reinterpret_cast<uint4*>(out.hi + (ws + row[t]) * out.ld + c0) = h;
                         *reinterpret_cast<uint4*>(out.lo + (ws + row[t]) * out.ld + c0) = l;
                     }
                 }
             }
-            // rows with more entries than are listed: the row's entries again, four source rows in flight
+            // rows with more entries than are listed: the row's entries again, one row at a time; the quarters
+            // of the warp (LPR = 8) each take every fourth of them, four source rows in flight per lane
             if (many) {
                 const int64_t* rp = rowptr_out + g.row_abs[k] + g.part[k];
                 const int32_t* cols = col_out + g.edge_abs[k];
@@ -581,17 +603,18 @@ spmm_outside_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restri
                             float wy[4];
 #pragma unroll
                             for (int b = 0; b < 4; ++b) {
-                                u[b] = -1;
-                                if (votes) {
-                                    u[b] = __shfl_sync(0xffffffffu, c, __ffs(votes) - 1);
-                                    votes &= votes - 1;
-                                }
+                                // quarter `sub` takes the entries sub, sub + S, ... of those still to do
+                                const unsigned from = __fns(votes, 0, b * S + sub + 1);
+                                u[b] = __shfl_sync(0xffffffffu, c, from < 32u ? (int)from : 0);
+                                if (from >= 32u) u[b] = -1;
                             }
+#pragma unroll
+                            for (int b = 0; b < 4 * S; ++b) votes &= votes - 1;
 #pragma unroll
                             for (int b = 0; b < 4; ++b) {
                                 if (u[b] >= 0) {
                                     yh[b] = __ldg(reinterpret_cast<const uint4*>(sh + (int64_t)u[b] * src.ld + cx));
-                                    yl[b] = __ldg(reinterpret_cast<const uint4*>(sl + (int64_t)u[b] * src.ld + cx));
+                                    yl[b] = __ldg(reinterpret_cast<const uint4*>(sl_ + (int64_t)u[b] * src.ld + cx));
                                     if (TRANSPOSED) wy[b] = __ldg(inv_deg + ws + u[b]);
                                 }
                             }
@@ -604,7 +627,12 @@ spmm_outside_kernel(const __grid_constant__ GroupDesc g, const int64_t* __restri
                             }
                         }
                     }
-                    if (live) {
+                    // the quarters' sums, added in a fixed order
+#pragma unroll
+                    for (int step = S / 2; step > 0; step >>= 1)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc.v[e] += __shfl_down_sync(0xffffffffu, acc.v[e], step * LPR);
+                    if (live && sub == 0) {
                         uint4 h, l;
                         acc.to_planes_lean(h, l);
                         *reinterpret_cast<uint4*>(out.hi + (ws + i) * out.ld + c0) = h;
@@ -781,10 +809,17 @@ int32_t launch_spmm_dense(rtma_ctx* ctx, int kclass, const GroupDesc& g, const i
     const unsigned lgrid = (unsigned)std::min<int64_t>(ceil_div(groups, 8), (int64_t)ctx->sm_count * 8);
     {
         KernelScope ks(ctx, kclass, s);
-        if (transposed)
-            spmm_outside_kernel<true><<<lgrid, 256, 0, s>>>(g, rowptr_out, col_out, inv_deg, dense, order.left_cnt, order.left_col, src, out, a.width, groups);
-        else
-            spmm_outside_kernel<false><<<lgrid, 256, 0, s>>>(g, rowptr_out, col_out, inv_deg, dense, order.left_cnt, order.left_col, src, out, a.width, groups);
+#define RTMA_OUTSIDE(T, L)                                                                                              \
+    spmm_outside_kernel<T, L><<<lgrid, 256, 0, s>>>(g, rowptr_out, col_out, inv_deg, dense, order.left_cnt, order.left_col, \
+                                                    src, out, a.width, groups)
+        if (a.width <= 64) {
+            if (transposed) RTMA_OUTSIDE(true, 8);
+            else RTMA_OUTSIDE(false, 8);
+        } else {
+            if (transposed) RTMA_OUTSIDE(true, 32);
+            else RTMA_OUTSIDE(false, 32);
+        }
+#undef RTMA_OUTSIDE
     }
     RTMA_LAUNCH_CHECK(ctx);
     const unsigned grid = (unsigned)std::min<int64_t>(row_tiles * a.col_tiles, ctx->sm_count);

@@ -1,11 +1,13 @@
 """The aggregation Abar H (Theorem 2) and its transpose taken from dense tiles on the tensor cores:
 entries whose column lies in the window around their row's 128-row tile come from an MMA against a
-0/1 (or 1/deg-weighted) tile built in shared memory, the others from a gather pass afterwards.
+0/1 (or 1/deg-weighted) tile expanded in shared memory from per-row bit masks, the others are summed
+into the output rows by a gather pass beforehand.
 
 Forced on for every part (mode 2) the path must reproduce the oracle on graphs it was not made for
-(power-law parts where most entries fall outside the window, hubs, isolated nodes, repeated entries,
-rows narrower and wider than a column tile); left to decide for itself (mode 1) it must take the
-super-node-ordered parts and leave results independent of streams, waves and of which trainers still run.
+(power-law parts where most entries fall outside the window, hubs, isolated nodes, rows narrower and
+wider than a column tile; parts with repeated entries, which a bit mask cannot count, must find their
+way back to the gather kernels); left to decide for itself (mode 1) it must take the super-node-ordered
+parts and leave results independent of streams, waves and of which trainers still run.
 """
 import numpy as np
 import pytest
@@ -63,7 +65,8 @@ def test_forced_tiles_odd_widths(util, forced, tiny_workload, dims):
 
 def test_forced_tiles_with_repeated_entries_and_unsorted_rows(util, forced, tiny_workload):
     # a multigraph: some edges occur two or three times (both directions), and every row's entries are
-    # shuffled; the mean counts an entry as often as it occurs
+    # shuffled; the mean counts an entry as often as it occurs.  Every part has rows that repeat an entry
+    # inside their window, so even when forced the tiles hand these parts back to the gather kernels
     base = inputs.uniform_graph(700, 2800, 21)
     rng = np.random.default_rng(22)
     rp = base.rowptr.astype(np.int64)
@@ -84,6 +87,41 @@ def test_forced_tiles_with_repeated_entries_and_unsorted_rows(util, forced, tiny
     w.M = 2
     got, want = util.check_one_step(w)
     util.check_k_steps_and_average(w, got, want, 2)
+
+
+def test_one_part_with_a_repeated_entry_gathers_while_the_others_take_the_tiles(util, forced):
+    # the same launch then serves both kinds of parts: the gather kernels skip the flagged parts, the tiles
+    # the others.  One edge inside one super-node is stored twice (in both directions).
+    w = inputs.supertma(0.02, M=4)
+    w.grouped_order = True
+    w.dims = (100, 64, 47)
+    w.params0 = inputs.xavier_params(w.dims, 8)
+    g = w.graph
+    rp = g.rowptr.astype(np.int64)
+    members = np.flatnonzero(g.group_id == g.group_id[0])
+    u = v = -1
+    for cand in members:   # an edge between two members of that super-node
+        row = g.col[rp[cand]:rp[cand + 1]]
+        inside = row[np.isin(row, members)]
+        if inside.size:
+            u, v = int(cand), int(inside[0])
+            break
+    assert u >= 0
+    rows = np.repeat(np.arange(g.n), np.diff(rp))
+    rows = np.concatenate([rows, [u, v]])
+    cols = np.concatenate([g.col.astype(np.int64), [v, u]])
+    order = np.lexsort((cols, rows))
+    rowptr = np.zeros(g.n + 1, dtype=g.rowptr.dtype)
+    np.cumsum(np.bincount(rows, minlength=g.n), out=rowptr[1:])
+    w.graph = inputs.Graph(n=g.n, rowptr=rowptr, col=cols[order].astype(np.int32), group_id=g.group_id)
+    got, want = util.check_one_step(w)
+    tiles = util.check_k_steps_and_average(w, got, want, 2)
+    c = forced
+    c.set_dense_aggregation(0)
+    gathered = util.check_k_steps_and_average(w, got, want, 2)
+    # the part that holds the repeated entry: the same bits either way; the other parts: not
+    same = [np.array_equal(tiles[p], gathered[p]) for p in range(w.M)]
+    assert sum(same) == 1 and same[int(want["part_id"][u])]
 
 
 def test_forced_tiles_do_not_depend_on_streams_waves_or_who_else_runs(util, forced, tiny_workload):
