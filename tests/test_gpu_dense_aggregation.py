@@ -89,6 +89,30 @@ def test_forced_tiles_with_repeated_entries_and_unsorted_rows(util, forced, tiny
     util.check_k_steps_and_average(w, got, want, 2)
 
 
+def test_forced_tiles_with_prelu_and_layer_normalization(util, forced):
+    # the paper's encoder activation and normalisation (Sec. 4.1) round the GraphSAGE aggregation on the tiles
+    import test_gpu_variants as tv
+    w = inputs.medium(0.04)
+    variant = (0, 1, 1)
+    p0 = tv._start(variant, w.dims, 11)
+    got, want = util.check_one_step(w, variant=variant, params0=p0)
+    util.check_k_steps_and_average(w, got, want, 2, variant=variant, params0=p0)
+
+
+def test_forced_tiles_in_bf16_operand_mode(util, forced, tiny_workload):
+    # the aggregation keeps its fp32 sums when the products take bf16 operands
+    w = tiny_workload
+    got, want = util.check_one_step(w, gemm_dtype=1)
+    util.check_k_steps_and_average(w, got, want, w.K, gemm_dtype=1)
+
+
+def test_forced_tiles_under_link_prediction(util, forced, tiny_workload):
+    # GraphSAGE encoder + PReLU + LayerNorm, MLP decoder on pairs (Sec. 4.1): the encoder's last layer is as
+    # wide as the hidden ones there (no head form), all its aggregations go through the tiles
+    import test_gpu_link as tl
+    tl._check_link(util, tiny_workload, (0, 1, 1), (8, 16, 5, 1), per_part=300, K=3)
+
+
 def test_one_part_with_a_repeated_entry_gathers_while_the_others_take_the_tiles(util, forced):
     # the same launch then serves both kinds of parts: the gather kernels skip the flagged parts, the tiles
     # the others.  One edge inside one super-node is stored twice (in both directions).
