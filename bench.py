@@ -78,11 +78,11 @@ def algorithmic_work(dims, n_parts, e_parts, K, R, entries=0, rowptr_bytes=8, gr
     part_scatter = 12.0 * n + (4.0 * n if grouped else 0.0) + (4 * (12.0 * n) if grouped else 0.0)
     work["partition_count"] = ("hbm", part_count, 0.0)
     work["partition_scatter"] = ("hbm", part_scatter, 0.0)
-    # induced subgraphs: per entry the column id and the part of its end point (count pass), the same
-    # again plus the end point's local id and the kept entry written (fill pass); per row its offsets,
-    # its node id and its part
-    work["induced_count"] = ("hbm", E * 8 + n * (2 * rowptr_bytes + 8 + 8), 0.0)
-    work["induced_fill"] = ("hbm", E * 8 + e * 8 + n * (2 * rowptr_bytes + 8 + 8), 0.0)
+    # induced subgraphs: per entry the column id, the part of its end point and one bit (kept or not) written
+    # (count pass); that bit, and per kept entry its column id, the end point's local id and the entry written
+    # (fill pass); per row its offsets, its node id and its part
+    work["induced_count"] = ("hbm", E * 8 + E / 8 + 4 * n + n * (2 * rowptr_bytes + 8 + 8), 0.0)
+    work["induced_fill"] = ("hbm", E / 8 + 4 * n + e * 12 + n * (2 * rowptr_bytes + 8 + 8), 0.0)
     work["gather_rows"] = ("hbm", 12.0 * n, 0.0)                         # labels only: perm, label in, label out
     work["to_planes"] = ("hbm", R * (8.0 * n * dims[0] + 4.0 * n), 0.0)   # features gathered through perm into planes
     # The last layer's aggregate is taken after its product when that is narrower (the library's rule:

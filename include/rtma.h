@@ -160,6 +160,12 @@ const char* rtma_partition_static_error(void);
  * Two phases.  col_out == NULL: COUNT -- writes rowptr_out, edge_offsets and kept_cut; read
  * edge_offsets[M] back (after draining the stream) to size col_out.  col_out != NULL: FILL --
  * reads rowptr_out and edge_offsets as the count phase left them and writes col_out only.
+ * COUNT waits for the stream once (it reads rowptr[n], 8 bytes) and leaves, in a buffer of the
+ * context of rowptr[n] / 8 + 4 n bytes (kept until the context is destroyed, not part of the
+ * scratch arena), one bit per entry: kept or not.  A FILL that follows the COUNT on the same n, M, rowptr,
+ * col and part_id pointers reads those bits and the kept entries only; any other FILL (or one
+ * after a COUNT that found no memory for the bits) looks every entry's part up again.  Same
+ * result either way.
  * part_id / part_offsets / perm / local_id are rtma_partition's outputs.                  */
 int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowptr_is_64, const void* rowptr,
                                const int32_t* col, int32_t M, const int32_t* part_id,

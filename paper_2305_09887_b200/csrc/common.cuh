@@ -48,6 +48,15 @@ struct rtma_ctx {
     size_t host_block_bytes = 0;
     void* host_cols = nullptr;
     size_t host_cols_bytes = 0;
+    // which entries the last COUNT phase of rtma_build_induced_csr kept, one bit per entry of its input graph, for
+    // the FILL phase that follows on the same arrays (keep_key: n, M, rowptr, col, part_id of that call)
+    uint32_t* keep_bits = nullptr;
+    size_t keep_words = 0;
+    int64_t keep_n = -1;
+    int32_t keep_M = 0;
+    const void* keep_rowptr = nullptr;
+    const void* keep_col = nullptr;
+    const void* keep_part = nullptr;
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t copy_done = nullptr;
     void* pinned = nullptr;       // small pinned staging block for descriptors

@@ -44,6 +44,7 @@ extern "C" int32_t rtma_destroy(rtma_ctx* ctx) {
     if (ctx->arena) cudaFree(ctx->arena);
     if (ctx->host_block) cudaFree(ctx->host_block);
     if (ctx->host_cols) cudaFree(ctx->host_cols);
+    if (ctx->keep_bits) cudaFree(ctx->keep_bits);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
     if (ctx->error_word) cudaFree(ctx->error_word);

@@ -7,8 +7,14 @@
 // at the row's place in partition order.  An exclusive scan of the counts gives every row's slot
 // in col_out, from which the per-part zero-based offsets and edge_offsets follow.  FILL: the same
 // walk, with a warp ballot turning the keep predicate into compact, order-preserving output
-// positions.  Per entry the only random access is the part of its endpoint; both phases first
-// pack the part ids into one byte per node, so that this table (25 MB for 25 M nodes) stays in L2.
+// positions.  Per entry the only random access is the part of its endpoint; the part ids are first
+// packed into one byte per node, so that this table (25 MB for 25 M nodes) stays in L2.  Even so the
+// pass runs at the rate L2 delivers 32-byte sectors, one per entry, so COUNT also leaves one bit per
+// entry (kept or not) in a buffer of the context, and a FILL that follows on the same arrays reads
+// those bits instead of looking the parts up again: a thread per row, which touches the column ids
+// of kept entries only.  The k-th 32 entries of row u (first entry `begin`) are word begin / 32 + u + k:
+// every row has words of its own (ceil(deg / 32) of them fit before the next row's first), so COUNT
+// writes whole words without atomics and nothing needs clearing.
 #include "common.cuh"
 
 RTMA_BOUNDS_TU()
@@ -34,19 +40,26 @@ template <class RowT>
 __global__ void __launch_bounds__(CSR_THREADS)
 induced_count_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
                      const uint8_t* __restrict__ part8, const int64_t* __restrict__ part_offsets,
-                     const int32_t* __restrict__ local_id, int32_t* __restrict__ counts) {
+                     const int32_t* __restrict__ local_id, int32_t* __restrict__ counts,
+                     uint32_t* __restrict__ keep_bits) {
     const int lane = threadIdx.x & 31;
     const int64_t u = (int64_t)blockIdx.x * CSR_WARPS + (threadIdx.x >> 5);
     if (u >= n) return;
     const int p = part8[u];
     const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
     int kept = 0;
-    for (int64_t e = begin + lane; e < end; e += 32) {
-        const int32_t v = __ldg(col + e);
-        if (rtma_index_ok(v, n, 1)) kept += (part8[v] == p);
+    uint32_t* words = keep_bits ? keep_bits + (begin >> 5) + u : nullptr;  // the row's own words (see the top of the file)
+    for (int64_t e0 = begin; e0 < end; e0 += 32) {
+        const int64_t e = e0 + lane;
+        bool keep = false;
+        if (e < end) {
+            const int32_t v = __ldg(col + e);
+            keep = rtma_index_ok(v, n, 1) && part8[v] == p;
+        }
+        const unsigned votes = __ballot_sync(0xffffffffu, keep);
+        kept += __popc(votes);
+        if (words && lane == 0) words[(e0 - begin) >> 5] = votes;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
     if (lane == 0 && rtma_index_ok(p, M, 2)) {
         const int64_t place = part_offsets[p] + local_id[u];  // the row's place in partition order
         if (rtma_index_ok(place, n, 3)) counts[place] = kept;
@@ -115,6 +128,68 @@ induced_fill_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int
     }
 }
 
+// FILL from the bits COUNT left: a thread per row of the input graph walks the row's words and reads the
+// column ids of the kept entries only.  Rows of more than FILL_HEAVY entries (hubs) are left to the end and
+// done by the whole warp, 32 words at a time, the output positions from a prefix sum over the lanes.
+constexpr int FILL_HEAVY = 1024;
+template <class RowT>
+__global__ void __launch_bounds__(CSR_THREADS)
+induced_fill_bits_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const int32_t* __restrict__ col,
+                         const uint8_t* __restrict__ part8, const int64_t* __restrict__ part_offsets,
+                         const int32_t* __restrict__ local_id, const int64_t* __restrict__ rowptr_out,
+                         const int64_t* __restrict__ edge_offsets, const uint32_t* __restrict__ keep_bits,
+                         int32_t* __restrict__ col_out) {
+    const int lane = threadIdx.x & 31;
+    const int64_t u = (int64_t)blockIdx.x * CSR_THREADS + threadIdx.x;
+    int64_t begin = 0, end = 0, out = 0;
+    if (u < n) {
+        const int p = part8[u];
+        if (rtma_index_ok(p, M, 2)) {
+            const int64_t j = part_offsets[p] + local_id[u];  // the row's place in partition order
+            if (rtma_index_ok(j, n, 3)) {
+                begin = (int64_t)rowptr[u];
+                end = (int64_t)rowptr[u + 1];
+                out = edge_offsets[p] + rowptr_out[j + p];
+            }
+        }
+    }
+    const bool heavy = end - begin > FILL_HEAVY;
+    if (!heavy) {
+        const uint32_t* words = keep_bits + (begin >> 5) + u;
+        for (int64_t e0 = begin; e0 < end; e0 += 32) {
+            for (unsigned bits = __ldg(words + ((e0 - begin) >> 5)); bits; bits &= bits - 1) {
+                const int32_t v = __ldg(col + e0 + (__ffs(bits) - 1));
+                col_out[out++] = local_id[v];
+            }
+        }
+    }
+    for (unsigned todo = __ballot_sync(0xffffffffu, heavy); todo; todo &= todo - 1) {
+        const int src = __ffs(todo) - 1;
+        const int64_t hu = u - lane + src;
+        const int64_t hb = __shfl_sync(0xffffffffu, begin, src), he = __shfl_sync(0xffffffffu, end, src);
+        int64_t ho = __shfl_sync(0xffffffffu, out, src);
+        const uint32_t* words = keep_bits + (hb >> 5) + hu;
+        for (int64_t k0 = 0; hb + (k0 << 5) < he; k0 += 32) {
+            const int64_t e0 = hb + ((k0 + lane) << 5);  // first entry of this lane's word
+            unsigned bits = e0 < he ? __ldg(words + k0 + lane) : 0u;
+            int before = __popc(bits);  // kept entries in the words of the lanes below: an inclusive scan, then minus its own
+            const int mine = before;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, before, o);
+                if (lane >= o) before += t;
+            }
+            const int total = __shfl_sync(0xffffffffu, before, 31);
+            int64_t at = ho + before - mine;
+            for (; bits; bits &= bits - 1) {
+                const int32_t v = __ldg(col + e0 + (__ffs(bits) - 1));
+                col_out[at++] = local_id[v];
+            }
+            ho += total;
+        }
+    }
+}
+
 template <int VEC_BYTES>
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(int64_t n, int64_t row_bytes, const char* __restrict__ src, const int32_t* __restrict__ perm,
@@ -167,14 +242,29 @@ extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowp
         uint8_t* part8 = reinterpret_cast<uint8_t*>(ctx->arena);
         { KernelScope ks(ctx, KC_CSR_FILL, stream); pack_parts_kernel<<<pack_blocks, 256, 0, stream>>>(n, part_id, part8, reinterpret_cast<uintptr_t>(part_id) % 16 == 0); }
         RTMA_LAUNCH_CHECK(ctx);
-        if (rowptr_is_64)
-            { KernelScope ks(ctx, KC_CSR_FILL, stream); induced_fill_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+        // the bits of the COUNT phase, if that was the last one and ran on these very arrays
+        const bool from_bits = ctx->keep_bits && ctx->keep_n == n && ctx->keep_M == M && ctx->keep_rowptr == rowptr &&
+                               ctx->keep_col == col && ctx->keep_part == part_id;
+        KernelScope ks(ctx, KC_CSR_FILL, stream);
+        if (from_bits) {
+            const unsigned thread_blocks = (unsigned)ceil_div(n, CSR_THREADS);
+            if (rowptr_is_64)
+                induced_fill_bits_kernel<int64_t><<<thread_blocks, CSR_THREADS, 0, stream>>>(
+                    n, M, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, rowptr_out, edge_offsets,
+                    ctx->keep_bits, col_out);
+            else
+                induced_fill_bits_kernel<int32_t><<<thread_blocks, CSR_THREADS, 0, stream>>>(
+                    n, M, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, rowptr_out, edge_offsets,
+                    ctx->keep_bits, col_out);
+        } else if (rowptr_is_64) {
+            induced_fill_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
                 n, M, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, rowptr_out,
-                edge_offsets, col_out); }
-        else
-            { KernelScope ks(ctx, KC_CSR_FILL, stream); induced_fill_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
+                edge_offsets, col_out);
+        } else {
+            induced_fill_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
                 n, M, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, rowptr_out,
-                edge_offsets, col_out); }
+                edge_offsets, col_out);
+        }
         RTMA_LAUNCH_CHECK(ctx);
         return RTMA_OK;
     }
@@ -189,16 +279,48 @@ extern "C" int32_t rtma_build_induced_csr(rtma_ctx* ctx, int64_t n, int32_t rowp
     int32_t* counts = cur.take<int32_t>(n + 1);
     int64_t* slots = cur.take<int64_t>(n + 2);
     int64_t* scratch = cur.take<int64_t>(scan_scratch_elems(n));
+    ctx->keep_n = -1;  // whatever an earlier COUNT left is void from here on
     if (n > 0) {
+        // One bit per entry for the FILL phase.  The number of entries is rowptr[n], on the device: the one place
+        // where this phase waits for the stream (8 bytes).  Without room for the bits FILL looks the parts up again.
+        int64_t entries = 0;
+        if (rowptr_is_64) {
+            RTMA_CUDA(ctx, cudaMemcpyAsync(&entries, static_cast<const int64_t*>(rowptr) + n, sizeof(int64_t), cudaMemcpyDeviceToHost, stream));
+            RTMA_CUDA(ctx, cudaStreamSynchronize(stream));
+        } else {
+            int32_t e32 = 0;
+            RTMA_CUDA(ctx, cudaMemcpyAsync(&e32, static_cast<const int32_t*>(rowptr) + n, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+            RTMA_CUDA(ctx, cudaStreamSynchronize(stream));
+            entries = e32;
+        }
+        uint32_t* keep_bits = nullptr;
+        if (entries > 0) {
+            const size_t words = (size_t)(entries / 32) + (size_t)n + 2;  // word e / 32 + u for entry e of row u
+            if (words > ctx->keep_words) {
+                if (ctx->keep_bits) cudaFree(ctx->keep_bits);
+                ctx->keep_bits = nullptr;
+                ctx->keep_words = 0;
+                if (cudaMalloc(&ctx->keep_bits, words * sizeof(uint32_t)) == cudaSuccess) ctx->keep_words = words;
+                else cudaGetLastError();
+            }
+            if (ctx->keep_bits && ctx->keep_words >= words) keep_bits = ctx->keep_bits;
+        }
         { KernelScope ks(ctx, KC_CSR_COUNT, stream); pack_parts_kernel<<<pack_blocks, 256, 0, stream>>>(n, part_id, part8, reinterpret_cast<uintptr_t>(part_id) % 16 == 0); }
         RTMA_LAUNCH_CHECK(ctx);
         if (rowptr_is_64)
             { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int64_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, M, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
+                n, M, static_cast<const int64_t*>(rowptr), col, part8, part_offsets, local_id, counts, keep_bits); }
         else
             { KernelScope ks(ctx, KC_CSR_COUNT, stream); induced_count_kernel<int32_t><<<row_blocks, CSR_THREADS, 0, stream>>>(
-                n, M, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, counts); }
+                n, M, static_cast<const int32_t*>(rowptr), col, part8, part_offsets, local_id, counts, keep_bits); }
         RTMA_LAUNCH_CHECK(ctx);
+        if (keep_bits) {
+            ctx->keep_n = n;
+            ctx->keep_M = M;
+            ctx->keep_rowptr = rowptr;
+            ctx->keep_col = col;
+            ctx->keep_part = part_id;
+        }
     }
     RTMA_TRY(exclusive_scan_i32_to_i64(ctx, counts, n, slots, scratch, stream));
     const unsigned off_blocks = (unsigned)ceil_div(n + M, CSR_THREADS);

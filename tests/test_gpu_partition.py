@@ -94,6 +94,36 @@ def test_induced_csr_supernodes(util):
     assert want["kept"] / w.graph.num_entries > 0.6                   # most edges live inside super-nodes
 
 
+def test_induced_csr_fill_with_and_without_the_count_phase_s_bits(util):
+    # COUNT leaves one bit per entry for the FILL that follows on the same arrays; a FILL after some other COUNT
+    # must not use them and looks every entry's part up again.  Rows that start and end inside a 32-entry word
+    # of the bit buffer (degrees 0..70), int32 and int64 offsets: the same col_out either way, equal to the oracle's.
+    import ctypes
+    import torch
+    from paper_2305_09887_b200 import binding
+    c = util.ctx()
+    for wide in (False, True):
+        w = inputs.medium(0.1)
+        if wide:
+            w.graph.rowptr = w.graph.rowptr.astype(np.int64)
+        M = 5
+        got = util.gpu_preprocess(w, M=M)                       # COUNT, then FILL from its bits
+        want = util.oracle_preprocess(w, M=M)
+        util.assert_preprocess_equal(got, want)
+        other = util.gpu_preprocess(inputs.tiny(), M=3)          # a COUNT (and FILL) on other arrays in between
+        g = w.graph
+        rowptr, col = util.dev(g.rowptr), util.dev(g.col)
+        again = torch.full_like(got["col_out"], -1)
+        st = c._lib.rtma_build_induced_csr(
+            c._h, ctypes.c_int64(g.n), ctypes.c_int32(1 if wide else 0), binding._ptr(rowptr), binding._ptr(col),
+            ctypes.c_int32(M), binding._ptr(got["part_id"]), binding._ptr(got["part_offsets"]), binding._ptr(got["perm"]),
+            binding._ptr(got["local_id"]), binding._ptr(got["rowptr_out"]), binding._ptr(again),
+            binding._ptr(got["edge_offsets"]), binding._ptr(got["kept_cut"]), ctypes.c_void_p(0))
+        assert st == 0
+        torch.cuda.synchronize()
+        assert torch.equal(again, got["col_out"]) and other["col_out"].numel() > 0
+
+
 def test_induced_csr_degenerate_graphs(util):
     c = util.ctx()
     # no edges at all
