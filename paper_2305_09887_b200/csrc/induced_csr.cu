@@ -49,16 +49,25 @@ induced_count_kernel(int64_t n, int M, const RowT* __restrict__ rowptr, const in
     const int64_t begin = (int64_t)rowptr[u], end = (int64_t)rowptr[u + 1];
     int kept = 0;
     uint32_t* words = keep_bits ? keep_bits + (begin >> 5) + u : nullptr;  // the row's own words (see the top of the file)
-    for (int64_t e0 = begin; e0 < end; e0 += 32) {
-        const int64_t e = e0 + lane;
-        bool keep = false;
-        if (e < end) {
-            const int32_t v = __ldg(col + e);
-            keep = rtma_index_ok(v, n, 1) && part8[v] == p;
+    // four words (128 entries) at a time: all their column ids, then all the parts, then the votes, so that the
+    // gathers of one round are in flight together
+    for (int64_t e0 = begin; e0 < end; e0 += 128) {
+        int32_t v[4];
+        bool keep[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int64_t e = e0 + 32 * c + lane;
+            keep[c] = e < end;
+            v[c] = keep[c] ? __ldg(col + e) : 0;
         }
-        const unsigned votes = __ballot_sync(0xffffffffu, keep);
-        kept += __popc(votes);
-        if (words && lane == 0) words[(e0 - begin) >> 5] = votes;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) keep[c] = keep[c] && rtma_index_ok(v[c], n, 1) && part8[v[c]] == p;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const unsigned votes = __ballot_sync(0xffffffffu, keep[c]);
+            kept += __popc(votes);
+            if (words && lane == 0 && e0 + 32 * c < end) words[((e0 - begin) >> 5) + c] = votes;
+        }
     }
     if (lane == 0 && rtma_index_ok(p, M, 2)) {
         const int64_t place = part_offsets[p] + local_id[u];  // the row's place in partition order
